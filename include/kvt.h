@@ -1,0 +1,305 @@
+/*
+ * kvt.h — C ABI of the lifecycle-aware KV cache engine hot path (GPU library libkvt.so).
+ *
+ * The library implements, for one GPU, the data-parallel part of a lifecycle-aware KV cache
+ * manager for ReAct agents:
+ *   (1) chained 16-token block hashing of agent contexts built by message-level primitives
+ *       (Section 4.1, Table 3: append / replace / remove / fork / spawn / one_off),
+ *   (2) lookup of those hashes in a GPU-resident open-addressing block table (reusable prefix),
+ *   (3) derivation of each resident block's KV-level lifecycle state from message-level states
+ *       (Section 5.2 state machine; Section 6.1 "Managing Shared KV"),
+ *   (4) state-prioritised, recency-ordered victim selection (Algorithm 1; Section 6.2), and
+ *   (5) movement of paged KV blocks between the HBM pool and a pinned host tier (Section 7).
+ *
+ * General conventions
+ *   - Plain C, no exceptions, no stdout. Every function returns an int32_t status: KVT_OK (0) or a
+ *     negative KVT_E_* code. Unless a call documents partial progress through an out-count, a call
+ *     that returns an error leaves the engine state unchanged.
+ *   - Memory ownership: the caller allocates the HBM pool, the host pool (pinned, device-mapped
+ *     memory), the device metadata arena and the device token arena, and passes raw pointers and
+ *     byte sizes in kvt_config. The library never allocates or frees device memory and never frees
+ *     caller memory. It does allocate a few MB of pinned HOST staging memory of its own in
+ *     kvt_create and frees it in kvt_destroy.
+ *   - "device pointer" = memory the GPU can dereference (cudaMalloc'd, or pinned mapped host
+ *     memory under unified addressing). "host pointer" = ordinary host memory read/written by the
+ *     CPU inside the call; it may be reused as soon as the call returns.
+ *   - stream: a cudaStream_t passed as void*. All device work of a call is enqueued on it. Calls
+ *     that return counts or data to the host synchronise that stream before returning (stated per
+ *     call); kvt_copy_blocks is asynchronous.
+ *   - An engine is not thread-safe; calls on one engine must be serialised by the caller and must
+ *     all use streams that are ordered with respect to each other.
+ *   - Every device-side loop (table probe loops) has an iteration cap; on overrun the kernel sets
+ *     a device error word and returns normally, and the call reports KVT_E_DEVICE.
+ *   - The library has no CPU fallback: without a usable CUDA device kvt_create fails with
+ *     KVT_E_CUDA.
+ */
+#ifndef KVT_H_
+#define KVT_H_
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define KVT_ABI_VERSION 1u
+#define KVT_BLOCK_TOKENS 16u
+
+/* ---- status codes -------------------------------------------------------------------------- */
+#define KVT_OK          0
+#define KVT_E_INVAL    -1  /* malformed argument (NULL pointer, bad enum, id in use, duplicate id) */
+#define KVT_E_NOCTX    -2  /* unknown or terminated context */
+#define KVT_E_RANGE    -3  /* message range or slot id out of bounds */
+#define KVT_E_STATE    -4  /* op not allowed in the current state (in-flight context / in-flight block) */
+#define KVT_E_NOSPACE  -5  /* a tier, the table or an arena is full; see the call's out-counts */
+#define KVT_E_BUFSZ    -6  /* caller-provided output buffer too small */
+#define KVT_E_DEVICE   -7  /* device error word set (probe cap exceeded, corrupt metadata) */
+#define KVT_E_CUDA     -8  /* a CUDA runtime call failed; text via kvt_last_error */
+
+/* ---- enums --------------------------------------------------------------------------------- */
+/* Tiers (Section 7: multi-tier engine; the remote tier is not part of this library). */
+#define KVT_TIER_HBM   0u
+#define KVT_TIER_HOST  1u
+#define KVT_TIER_NONE  0xFFu   /* "not resident" in block maps */
+
+/* HBM pool layouts. The host pool is always block-major. */
+#define KVT_LAYOUT_LAYER_MAJOR 0u  /* chunk (layer l, kv) of slot s at ((l*2+kv)*n_hbm_blocks + s)*chunk_bytes */
+#define KVT_LAYOUT_BLOCK_MAJOR 1u  /* slot s at s*block_bytes, chunk c at + c*chunk_bytes */
+
+/* Recency direction inside the Suspended (live-but-idle) tier (Section 6.2 and the "w/o RO"
+ * ablation of Section 8.3). */
+#define KVT_ORDER_MRU 0u   /* most recently suspended first (the paper's policy, default) */
+#define KVT_ORDER_LRU 1u   /* oldest first */
+
+/* Primitives and runtime events (Table 3; Section 5.2 "Runtime transitions"). */
+#define KVT_OP_SPAWN         1u  /* register an independent, empty context */
+#define KVT_OP_FORK          2u  /* register child `ctx` sharing messages [0, msg_end) of `parent` */
+#define KVT_OP_APPEND        3u  /* append one message (tokens) */
+#define KVT_OP_REPLACE       4u  /* replace messages [msg_start, msg_end) by one message (tokens) */
+#define KVT_OP_REMOVE        5u  /* remove messages [msg_start, msg_end) */
+#define KVT_OP_ONE_OFF       6u  /* mark the context (msg_start=0, msg_end=UINT32_MAX) or messages
+                                    [msg_start, msg_end) for one inference (Temporary) */
+#define KVT_OP_PREFILL_DONE  7u  /* prefill of the context's in-flight call completed */
+#define KVT_OP_TERMINATE     8u  /* the context ends */
+#define KVT_OP_PIN           9u  /* reserved: returns KVT_E_INVAL */
+#define KVT_OP_UNPIN        10u  /* reserved: returns KVT_E_INVAL */
+
+/* kvt_op.flags */
+#define KVT_OPF_TOKENS_ON_DEVICE 1u  /* op.tokens is a device pointer (device-to-device copy) */
+
+/* kvt_map_blocks phases */
+#define KVT_MAP_LOOKUP 0u
+#define KVT_MAP_ADMIT  1u
+
+/* kvt_copy_blocks flags */
+#define KVT_IDS_ON_DEVICE 1u  /* src/dst id arrays are device pointers */
+
+/* KV-level lifecycle ranks reported by kvt_get_states / kvt_select_victims. They follow the
+ * release order of Algorithm 1: Discarded (Expired or Temporary) < Suspended < Active < Pinned. */
+#define KVT_STATE_DEAD    0u   /* no live message version maps the block */
+#define KVT_STATE_IDLE    1u   /* live but idle: best mapped message state is Suspended */
+#define KVT_STATE_ACTIVE  2u   /* live and active */
+#define KVT_STATE_PINNED  3u   /* reserved */
+#define KVT_STATE_FREE    0xFFu /* slot holds no block */
+
+typedef struct kvt_engine kvt_engine;
+
+/* ---- configuration -------------------------------------------------------------------------- */
+typedef struct kvt_config {
+  uint32_t abi_version;      /* KVT_ABI_VERSION */
+  uint32_t block_tokens;     /* must be 16 */
+  uint32_t n_layers;         /* KV geometry: a token's KV is n_layers * 2 (K,V) * n_kv_heads * head_dim * elem_bytes */
+  uint32_t n_kv_heads;
+  uint32_t head_dim;
+  uint32_t elem_bytes;       /* 2 for bf16 */
+  uint32_t pool_layout;      /* KVT_LAYOUT_* of the HBM pool */
+  uint32_t n_hbm_blocks;     /* slots in the HBM tier (>= 1) */
+  uint32_t n_host_blocks;    /* slots in the host tier (may be 0) */
+  uint32_t table_capacity;   /* power of two, >= 2 * (n_hbm_blocks + n_host_blocks) */
+  uint32_t max_contexts;     /* context ids are 0 .. max_contexts-1 */
+  uint32_t max_batch_blocks; /* upper bound on the blocks hashed by one kvt_map_blocks call and on n of one list call */
+  uint64_t max_tokens;       /* capacity of the device token arena, in tokens */
+  uint64_t max_key_blocks;   /* capacity of the per-context key lists, in blocks (all contexts together) */
+  uint64_t hash_seed;        /* seed of the block hash */
+  uint32_t suspended_order;  /* KVT_ORDER_* */
+  uint32_t reserved;         /* must be 0 */
+  void *hbm_pool;  uint64_t hbm_pool_bytes;   /* device; NULL/0 = metadata-only engine (no payload is moved) */
+  void *host_pool; uint64_t host_pool_bytes;  /* device-accessible pinned host memory; NULL/0 if metadata-only */
+  void *dev_meta;  uint64_t dev_meta_bytes;   /* device metadata + scratch arena, 256-byte aligned */
+  void *dev_tokens; uint64_t dev_tokens_bytes;/* device token arena, 256-byte aligned */
+} kvt_config;
+
+/* Computes the byte sizes the caller must allocate for dev_meta and dev_tokens from the other
+ * fields of cfg (pointer fields are ignored). Host-only. */
+int32_t kvt_query_sizes(const kvt_config *cfg, uint64_t *meta_bytes, uint64_t *token_bytes);
+
+/* Creates an engine on the current CUDA device. Validates cfg (KVT_E_INVAL), zero-initialises
+ * the metadata arena on `stream` and synchronises it. The pools are not touched. */
+int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out);
+int32_t kvt_destroy(kvt_engine *e);
+
+/* ---- stage 0: message-level primitives (Table 3; Section 5.1; Section 5.2) ------------------ */
+typedef struct kvt_op {
+  uint32_t op;          /* KVT_OP_* */
+  uint32_t ctx;         /* context the op applies to (FORK: the new child) */
+  uint32_t parent;      /* FORK only */
+  uint32_t msg_start;   /* REPLACE / REMOVE / ONE_OFF: first message of the range */
+  uint32_t msg_end;     /* one past the last message; FORK: number of inherited messages */
+  uint32_t n_tokens;    /* APPEND / REPLACE: length of the new message (may be 0) */
+  uint32_t flags;       /* KVT_OPF_* */
+  uint32_t reserved;    /* must be 0 */
+  const uint32_t *tokens; /* APPEND / REPLACE payload: host pointer (copied before return) or device pointer */
+} kvt_op;
+
+/* Applies one primitive or runtime event to a context, strictly in program order per context
+ * (Section 5.1). Host bookkeeping plus, for token-carrying ops, a copy of the tokens into the
+ * device token arena and, for PREFILL_DONE / TERMINATE of an in-flight context, one kernel that
+ * releases the in-flight locks of the blocks the context holds.
+ *   APPEND: new message is Active, or Temporary if the context is one_off. No KV effect until the
+ *     next call (KV-existence gating, Section 5.1).
+ *   REPLACE / REMOVE at message s: the old versions of s and of every later message expire for
+ *     this context only: the context stops mapping every block from the block containing the first
+ *     token of message s on (prefix-dependent validity, Section 5.1). Requires s < e <= #messages.
+ *   FORK: the child gets Active copies of parent messages [0, msg_end) and immediately maps the
+ *     still-valid blocks they cover; parent and child evolve independently afterwards.
+ *   ONE_OFF: listed (or all current and future) messages become Temporary.
+ *   PREFILL_DONE: Active -> Suspended; advances the logical clock; stamps and unlocks held blocks.
+ *   TERMINATE: the context stops mapping anything and its id becomes free.
+ * Errors: KVT_E_NOCTX unknown context; KVT_E_INVAL id in use / bad op / NULL tokens;
+ * KVT_E_RANGE bad message range; KVT_E_STATE edit or fork-from of an in-flight context, or
+ * PREFILL_DONE of a context that is not in flight; KVT_E_NOSPACE token arena full.
+ * Does not synchronise the stream. */
+int32_t kvt_apply_op(kvt_engine *e, const kvt_op *op, void *stream);
+
+/* ---- stages 1+2 (+ admission): hash, lookup, admit ------------------------------------------- */
+typedef struct kvt_call_info {
+  uint32_t n_blocks;      /* full 16-token blocks of the context's token sequence */
+  uint32_t hit_len;       /* leading blocks found resident at LOOKUP (the reusable prefix) */
+  uint32_t n_hit_hbm;     /* of those, resident in HBM */
+  uint32_t n_hit_host;    /* of those, resident in the host tier (reload them before use) */
+  uint32_t n_admissible;  /* blocks after the prefix that may enter reusable storage (Temporary bypass) */
+  uint32_t n_admitted;    /* ADMIT: blocks this call newly holds (inserted or adopted) */
+  uint32_t n_held;        /* leading blocks locked in flight for this context after the call */
+} kvt_call_info;
+
+/* phase KVT_MAP_LOOKUP — one LLM call begins for each listed context (Section 7: call id and
+ * context id are handed to the cache engine). Advances the logical clock once per batch. For
+ * each context: reactivates its ordinary messages (Section 5.2), hashes the concatenation of its
+ * messages' tokens into chained block keys, walks the chain through the block table until the
+ * first miss, stamps and locks the hits, and makes the new token layout the context's
+ * materialised mapping. The same result as if contexts were processed one by one.
+ *
+ * phase KVT_MAP_ADMIT — Algorithm 1's admission test ("admit iff Delta <= 0") per 16-token block,
+ * in (list order, chain order), for blocks [n_held, hit_len + n_admissible): a block already
+ * resident (or inserted earlier in this batch) is adopted; otherwise it takes the lowest free
+ * HBM slot; if none is free the context stops there. Eviction is the caller's job
+ * (kvt_select_victims + kvt_offload) before ADMIT. May be called again to continue.
+ *
+ * Errors: KVT_E_NOCTX; KVT_E_INVAL duplicate context in the list, n_ctx = 0; KVT_E_STATE LOOKUP
+ * on an in-flight context or ADMIT on one that is not; KVT_E_NOSPACE batch larger than
+ * max_batch_blocks or key arena full. Synchronises the stream. `out` has n_ctx elements. */
+int32_t kvt_map_blocks(kvt_engine *e, const uint32_t *ctx_ids, uint32_t n_ctx, uint32_t phase,
+                       kvt_call_info *out, void *stream);
+
+/* Block map of a context's materialised token sequence: key, tier (KVT_TIER_* / KVT_TIER_NONE)
+ * and slot (0xFFFFFFFF if not resident) of each block as of now. Host output arrays of capacity
+ * `cap`; *n receives the block count (KVT_E_BUFSZ if cap is too small). Synchronises. */
+int32_t kvt_get_block_map(kvt_engine *e, uint32_t ctx, uint64_t *keys, uint8_t *tier,
+                          uint32_t *slot, uint32_t cap, uint32_t *n, void *stream);
+
+/* ---- stage 3: KV-level lifecycle state (Section 6.1 "Managing Shared KV") -------------------- */
+/* Recomputes, for every resident block, the highest-priority state over all (context, message
+ * version) mappings; a block nobody maps is dead. Asynchronous on `stream`. */
+int32_t kvt_classify(kvt_engine *e, void *stream);
+
+/* Copies the ranks of one tier to a host array (KVT_STATE_FREE for empty slots); classifies
+ * first if anything changed since the last classification. cap >= slots of the tier. Synchronises. */
+int32_t kvt_get_states(kvt_engine *e, uint32_t tier, uint8_t *state, uint32_t cap, void *stream);
+
+/* ---- stage 4: victim selection (Algorithm 1 order; Section 6.2 recency) ----------------------- */
+/* Returns the first min(n_req, #candidates) slots of `tier` in eviction order, with their ranks.
+ * Candidates: resident, not in flight, rank below Pinned. Order: rank ascending (dead, idle,
+ * active); within dead and active oldest stamp first; within idle newest stamp first (MRU) or
+ * oldest first if suspended_order = KVT_ORDER_LRU; then chain depth descending; then slot
+ * ascending. Classifies first if needed. Host output arrays (states_out may be NULL).
+ * KVT_E_BUFSZ if cap < min(n_req, #candidates). Synchronises. */
+int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_t *slots_out,
+                           uint8_t *states_out, uint32_t cap, uint32_t *n_out, void *stream);
+
+/* ---- stage 5: tier movement (Section 7; Algorithm 1 "release") -------------------------------- */
+/* Processes HBM slots in the given order: a dead block is dropped (key erased, slot freed, no
+ * copy); the i-th live block moves to the i-th lowest free host slot, payload byte for byte,
+ * metadata carried. Stops with KVT_E_NOSPACE when the host tier is full; *n_done = victims
+ * processed, *n_dropped = dead ones among them. A listed slot that is empty, out of range,
+ * repeated (KVT_E_INVAL / KVT_E_RANGE) or in flight (KVT_E_STATE) rejects the whole call.
+ * Host id array. Synchronises. */
+int32_t kvt_offload(kvt_engine *e, const uint32_t *hbm_slots, uint32_t n, uint32_t *n_done,
+                    uint32_t *n_dropped, void *stream);
+
+/* Mirror image: the i-th listed host slot moves to the i-th lowest free HBM slot (in-flight
+ * blocks allowed: a call reloads its own host hits). KVT_E_NOSPACE + *n_done when HBM is full. */
+int32_t kvt_reload(kvt_engine *e, const uint32_t *host_slots, uint32_t n, uint32_t *n_done,
+                   void *stream);
+
+/* Drops blocks without copying (frees host space for offloads). Same validation as kvt_offload. */
+int32_t kvt_release(kvt_engine *e, uint32_t tier, const uint32_t *slots, uint32_t n, void *stream);
+
+/* Hole-filling compaction inside a tier: with n_occ occupied slots, the i-th occupied slot
+ * >= n_occ moves to the i-th free slot < n_occ (both ascending), so that afterwards exactly slots
+ * [0, n_occ) are occupied. Metadata (including in-flight counts) is carried; callers must refresh
+ * block maps. Synchronises. */
+int32_t kvt_compact(kvt_engine *e, uint32_t tier, uint32_t *n_moved, void *stream);
+
+/* Raw paged-KV mover: copies the payload of n blocks src_tier[src[i]] -> dst_tier[dst[i]]. No
+ * metadata is read or changed. Id arrays are host pointers unless KVT_IDS_ON_DEVICE. Destinations
+ * must be distinct and disjoint from sources within a tier (not checked); ids out of range set
+ * the device error word and are skipped. n <= max_batch_blocks. Asynchronous. */
+int32_t kvt_copy_blocks(kvt_engine *e, uint32_t src_tier, const uint32_t *src, uint32_t dst_tier,
+                        const uint32_t *dst, uint32_t n, uint32_t flags, void *stream);
+
+/* ---- stand-alone hasher ----------------------------------------------------------------------- */
+/* Chained block keys of one token sequence, without an engine: d_keys[b], b < n_tokens/16.
+ * d_tokens must be 16-byte aligned. d_scratch: device scratch of at least
+ * kvt_hash_scratch_bytes(n_tokens) bytes, 8-byte aligned. Asynchronous. */
+uint64_t kvt_hash_scratch_bytes(uint64_t n_tokens);
+int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t hash_seed,
+                        uint64_t *d_keys, void *d_scratch, uint64_t scratch_bytes, void *stream);
+
+/* ---- introspection ------------------------------------------------------------------------------ */
+typedef struct kvt_stats {
+  uint64_t clock;            /* logical clock */
+  uint64_t n_contexts;       /* live contexts */
+  uint64_t occ_hbm, occ_host;/* occupied slots per tier */
+  uint64_t blocks_hashed;    /* blocks hashed by LOOKUP */
+  uint64_t hits_hbm, hits_host, misses; /* per LOOKUP block: prefix hit by tier / not in the prefix */
+  uint64_t inserted;         /* blocks inserted by ADMIT */
+  uint64_t adopted;          /* blocks adopted by ADMIT */
+  uint64_t dropped;          /* dead blocks reclaimed without copy (offload) + released */
+  uint64_t offloaded, reloaded, compacted; /* blocks moved */
+  uint64_t bytes_d2h, bytes_h2d, bytes_d2d;/* payload bytes moved by offload / reload / compact */
+  uint64_t table_rebuilds;
+  uint64_t tombstones;
+} kvt_stats;
+int32_t kvt_get_stats(kvt_engine *e, kvt_stats *out);
+
+/* Text of the last error of this engine (always NUL-terminated). */
+int32_t kvt_last_error(kvt_engine *e, char *buf, uint32_t cap);
+
+/* Copies per-slot metadata of a tier to host arrays (any may be NULL): key (0 = free), stamp,
+ * depth, in-flight count. cap >= slots of the tier. Synchronises. */
+int32_t kvt_get_entries(kvt_engine *e, uint32_t tier, uint64_t *keys, uint32_t *stamp,
+                        uint32_t *depth, uint32_t *inflight, uint32_t cap, void *stream);
+
+/* Test / benchmark hook: makes n blocks resident in `tier` at the given slots without running
+ * calls. state[i] acts as a permanent anonymous mapping of that rank (classification never reports
+ * less for the block until it is dropped). Keys must be >= 2, distinct and not resident; slots
+ * free and distinct (violations: KVT_E_INVAL, state unchanged). Advances the logical clock to at
+ * least max(stamp). Host arrays. Synchronises. */
+int32_t kvt_debug_load_resident(kvt_engine *e, const uint64_t *keys, const uint8_t *state,
+                                const uint32_t *stamp, const uint32_t *depth,
+                                const uint32_t *slot, uint32_t tier, uint32_t n, void *stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KVT_H_ */

@@ -1,0 +1,502 @@
+"""Scenario checks that take an engine factory, so the same expectations (which come from the
+paper's sentences, from hand-worked examples and from brute force) pin the CPU oracle in the
+"not gpu" tests and are re-run against the CUDA engine in the "gpu" tests."""
+import os
+
+import numpy as np
+
+HBM, HOST = 0, 1
+LOOKUP, ADMIT = 0, 1
+DEAD, IDLE, ACTIVE, FREE = 0, 1, 2, 0xFF
+E_INVAL, E_NOCTX, E_RANGE, E_STATE, E_NOSPACE, E_BUFSZ = -1, -2, -3, -4, -5, -6
+
+TOY = dict(n_layers=2, n_kv_heads=2, head_dim=64)
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def toks(rng, n):
+    return rng.integers(0, 151552, int(n), dtype=np.uint32)
+
+
+def call(eng, ctx, done=True):
+    """lookup + admit (+ prefill-done) of one context with free space assumed."""
+    a = eng.map_blocks([ctx], LOOKUP)[0]
+    b = eng.map_blocks([ctx], ADMIT)[0]
+    if done:
+        eng.prefill_done(ctx)
+    return a, b
+
+
+def states(eng, tier=HBM):
+    return [int(x) for x in eng.get_states(tier)]
+
+
+# ---- Section 5.2 runtime transitions, one context ------------------------------------------------
+def state_machine_single_context(make):
+    eng = make(n_hbm_blocks=16, n_host_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(1)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 64))                         # 4 blocks
+    a, b = call(eng, 0, done=False)
+    assert (a["n_blocks"], a["hit_len"], a["n_admissible"]) == (4, 0, 4)
+    assert (b["n_admitted"], b["n_held"]) == (4, 4)
+    assert states(eng)[:5] == [ACTIVE] * 4 + [FREE]      # participating in a request: Active
+    assert list(eng.select_victims(HBM, 16)[0]) == []    # in-flight KV is never a victim
+    eng.prefill_done(0)
+    assert states(eng)[:4] == [IDLE] * 4                 # prefill complete: Suspended
+    a = eng.map_blocks([0], LOOKUP)[0]
+    assert (a["hit_len"], a["n_hit_hbm"], a["n_admissible"]) == (4, 4, 0)
+    assert states(eng)[:4] == [ACTIVE] * 4               # next request reactivates
+    eng.map_blocks([0], ADMIT)
+    eng.prefill_done(0)
+    eng.terminate(0)
+    assert states(eng)[:4] == [DEAD] * 4                 # context terminates: Expired
+    assert eng.get_stats()["n_contexts"] == 0
+
+
+# ---- remove / replace: suffix invalidation from the edited message's first block -----------------
+def suffix_invalidation(make):
+    eng = make(n_hbm_blocks=32, n_host_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(2)
+    eng.spawn(0)
+    msgs = [toks(rng, n) for n in (40, 24, 50, 30)]      # bounds [0,40) [40,64) [64,114) [114,144): 9 blocks
+    for m in msgs:
+        eng.append(0, m)
+    call(eng, 0)
+    keys0 = eng.get_block_map(0)[0].copy()
+    assert states(eng)[:9] == [IDLE] * 9
+    eng.replace(0, 2, 3, toks(rng, 10))                  # message 2 starts at token 64 -> block 4
+    assert states(eng)[:9] == [IDLE] * 4 + [DEAD] * 5    # takes effect at the op, later messages included
+    a, b = call(eng, 0, done=False)
+    keys1 = eng.get_block_map(0)[0]
+    assert a["hit_len"] == 4 and np.array_equal(keys1[:4], keys0[:4])
+    assert not np.intersect1d(keys1[4:], keys0[4:]).size  # every key from that block on is new
+    eng.prefill_done(0)
+    # removing message 1 (starts at token 40, inside block 2): block 2 straddles and dies too
+    eng.remove(0, 1, 2)
+    st = states(eng)
+    keys, tier, slot = eng.get_block_map(0)
+    assert [st[s] for s in slot[:2]] == [IDLE, IDLE]
+    assert all(st[s] == DEAD for s in slot[2:] if s != 0xFFFFFFFF)
+    # an edit of the last message only kills its own blocks
+    eng2 = make(n_hbm_blocks=32, n_host_blocks=4, max_contexts=4, **TOY)
+    eng2.spawn(0)
+    for m in msgs:
+        eng2.append(0, m)
+    call(eng2, 0)
+    eng2.remove(0, 3, 4)                                 # starts at token 114 -> block 7
+    assert states(eng2)[:9] == [IDLE] * 7 + [DEAD] * 2
+
+
+# ---- fork: shared prefix, independent states; the paper's shared-KV example (Section 6.1) --------
+def fork_and_shared_kv(make):
+    eng = make(n_hbm_blocks=32, n_host_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(3)
+    eng.spawn(0)
+    for n in (32, 32, 32):
+        eng.append(0, toks(rng, n))                      # 6 blocks, message j = blocks 2j, 2j+1
+    call(eng, 0)
+    eng.fork(0, 1, 2)                                    # child shares messages 0,1 = blocks 0..3
+    assert states(eng)[:6] == [ACTIVE] * 4 + [IDLE] * 2  # child's inherited messages are Active
+    eng.append(1, toks(rng, 32))
+    a, b = call(eng, 1)
+    assert a["hit_len"] == 4 and b["n_admitted"] == 2    # identical prefixes hash identically
+    assert states(eng)[:8] == [IDLE] * 8
+    # parent removes message 1: its KV (blocks 2..5 for the parent) expires for the parent only;
+    # the child still holds a Suspended reference to blocks 2,3 -> they stay Suspended.
+    eng.remove(0, 1, 2)
+    assert states(eng)[:8] == [IDLE, IDLE, IDLE, IDLE, DEAD, DEAD, IDLE, IDLE]
+    # Discarded only when all mapped versions are: now the child goes too
+    eng.terminate(1)
+    assert states(eng)[:8] == [IDLE, IDLE] + [DEAD] * 6
+    # execution in one context does not touch the other's message states
+    eng.fork(0, 2, 1)
+    eng.map_blocks([2], LOOKUP)
+    assert states(eng)[:2] == [ACTIVE, ACTIVE]
+    eng.map_blocks([2], ADMIT)
+    eng.prefill_done(2)
+    eng.terminate(2)
+    assert states(eng)[:2] == [IDLE, IDLE]               # parent's Suspended reference remains
+
+
+# ---- one_off: Temporary messages bypass reuse storage (Algorithm 1; Section 5.2 (3)) --------------
+def one_off_bypass(make):
+    eng = make(n_hbm_blocks=32, n_host_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(4)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 64))
+    call(eng, 0)
+    # compaction pattern (Section 4.2): fork, declare one-off, append the instruction, run
+    eng.fork(0, 1, 1)
+    eng.one_off(1)
+    eng.append(1, toks(rng, 48))
+    a, b = call(eng, 1, done=False)
+    assert (a["n_blocks"], a["hit_len"], a["n_admissible"]) == (7, 4, 0)
+    assert (b["n_admitted"], b["n_held"]) == (0, 4)
+    assert eng.get_stats()["occ_hbm"] == 4               # nothing of the temporary context was stored
+    assert states(eng)[:4] == [IDLE] * 4                 # Temporary references do not keep KV alive
+    eng.prefill_done(1)
+    eng.terminate(1)
+    # per-message form: a scratch message at the tail; the block it shares with an ordinary message
+    # is admissible, blocks made only of temporary tokens are not
+    eng.append(0, toks(rng, 24))                         # tokens 64..88
+    eng.append(0, toks(rng, 40))                         # tokens 88..128 (scratch)
+    eng.one_off(0, 2, 3)
+    a, b = call(eng, 0, done=False)
+    assert (a["n_blocks"], a["hit_len"], a["n_admissible"]) == (8, 4, 2)   # blocks 4 and 5 (straddles 88)
+    assert b["n_held"] == 6
+    eng.prefill_done(0)
+    # a temporary message in the middle stops admission at its first pure block
+    eng.append(0, toks(rng, 64))
+    a, b = call(eng, 0, done=False)
+    assert (a["hit_len"], a["n_admissible"]) == (6, 0)
+    eng.prefill_done(0)
+
+
+# ---- hand-worked lifecycle example (8-block pool) --------------------------------------------------
+def worked_example(make):
+    eng = make(n_hbm_blocks=8, n_host_blocks=8, max_contexts=4, **TOY)
+    rng = np.random.default_rng(0)
+    A, B = 0, 1
+    eng.spawn(A)
+    for n in (20, 30, 14):
+        eng.append(A, toks(rng, n))                      # bounds [0,20) [20,50) [50,64): 4 blocks
+    a, b = call(eng, A, done=False)                      # clock 1
+    assert (b["n_admitted"],) == (4,)
+    assert list(eng.get_block_map(A)[2]) == [0, 1, 2, 3] # lowest free slots in chain order
+    assert list(eng.get_entries(HBM)["stamp"][:4]) == [1] * 4
+    eng.prefill_done(A)                                  # clock 2
+    assert list(eng.get_entries(HBM)["stamp"][:4]) == [2] * 4
+    eng.fork(A, B, 2)                                    # child maps floor(50/16) = 3 blocks
+    assert states(eng)[:4] == [ACTIVE, ACTIVE, ACTIVE, IDLE]
+    eng.append(B, toks(rng, 30))
+    a, b = call(eng, B, done=False)                      # clock 3; 80 tokens = 5 blocks
+    assert (a["n_blocks"], a["hit_len"]) == (5, 3)       # block 3 differs from A's: tokens 50.. differ
+    assert list(eng.get_block_map(B)[2]) == [0, 1, 2, 4, 5]
+    eng.prefill_done(B)                                  # clock 4
+    assert list(eng.get_entries(HBM)["stamp"][:6]) == [4, 4, 4, 2, 4, 4]
+    eng.remove(A, 1, 2)                                  # cut = floor(20/16) = 1
+    assert states(eng)[:6] == [IDLE, IDLE, IDLE, DEAD, IDLE, IDLE]
+    eng.terminate(B)
+    assert states(eng)[:6] == [IDLE, DEAD, DEAD, DEAD, DEAD, DEAD]
+    v, s = eng.select_victims(HBM, 8)
+    # dead tier oldest first (stamp 2), then stamp 4 by depth 4,3,2,1; then the one Suspended block
+    assert list(v) == [3, 5, 4, 2, 1, 0] and list(s) == [0, 0, 0, 0, 0, 1]
+    assert eng.get_stats()["clock"] == 4
+
+
+def mixed_pool_example(make, order=0):
+    """{slot: (state, stamp, depth, inflight)}; slot 5 is in flight."""
+    eng = make(n_hbm_blocks=8, n_host_blocks=8, max_contexts=4, suspended_order=order, **TOY)
+    S, D, A = IDLE, DEAD, ACTIVE
+    pool = {0: (S, 5, 0), 1: (S, 5, 1), 2: (S, 9, 2), 3: (D, 7, 3), 4: (D, 2, 1), 6: (A, 8, 4), 7: (S, 9, 3)}
+    slots = sorted(pool)
+    eng.debug_load_resident([100 + s for s in slots], [pool[s][0] for s in slots], [pool[s][1] for s in slots],
+                            [pool[s][2] for s in slots], slots, HBM)
+    # slot 5: held in flight by a real context
+    rng = np.random.default_rng(9)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 16))
+    call(eng, 0, done=False)
+    assert list(eng.get_block_map(0)[2]) == [5]
+    v, s = eng.select_victims(HBM, 8)
+    if order == 0:
+        assert list(v) == [4, 3, 7, 2, 1, 0, 6]          # idle tier newest first
+    else:
+        assert list(v) == [4, 3, 1, 0, 7, 2, 6]          # idle tier oldest first
+    assert list(s) == [0, 0, 1, 1, 1, 1, 2]
+    v3, _ = eng.select_victims(HBM, 3)
+    assert list(v3) == list(v[:3])                       # a prefix of the same order
+
+
+# ---- victim order = brute-force sort, Algorithm 1 order, LRU special cases ------------------------
+def _brute_order(ent, st, mru):
+    cands = [s for s in range(len(st)) if st[s] != FREE and ent["inflight"][s] == 0 and st[s] < 3]
+
+    def key(s):
+        rec = int(ent["stamp"][s])
+        if st[s] == IDLE and mru:
+            rec = -rec
+        return (int(st[s]), rec, -int(ent["depth"][s]), s)
+    return sorted(cands, key=key)
+
+
+def victim_order_bruteforce(make, seeds=range(30)):
+    for seed in seeds:
+        rng = np.random.default_rng(seed)
+        order = int(seed % 2)
+        n = int(rng.integers(1, 65))
+        eng = make(n_hbm_blocks=n, n_host_blocks=8, max_contexts=4, suspended_order=order, **TOY)
+        k = int(rng.integers(0, n + 1))
+        slots = rng.permutation(n)[:k]
+        eng.debug_load_resident(rng.integers(2, 1 << 62, k).astype(np.uint64), rng.integers(0, 3, k),
+                                rng.integers(0, 6, k), rng.integers(0, 4, k), slots, HBM)  # many ties
+        st = eng.get_states(HBM)
+        want = _brute_order(eng.get_entries(HBM), st, order == 0)
+        for n_req in (0, 1, k // 2, k, k + 5):
+            v, s = eng.select_victims(HBM, n_req)
+            assert list(v) == want[: n_req], (seed, n_req)
+            assert [int(x) for x in s] == [int(st[i]) for i in v]
+            # Algorithm 1: no idle victim while a dead candidate remains, no active while idle remains
+            if len(v) < len(want):
+                rest = [int(st[i]) for i in want[len(v):]]
+                assert max([int(x) for x in s], default=0) <= min(rest)
+
+
+def one_state_pools_reduce_to_lru(make):
+    rng = np.random.default_rng(5)
+    n = 40
+    stamps = rng.permutation(1000)[:n]                   # distinct stamps
+    lru = list(np.argsort(stamps))
+    for state, order, want in ((DEAD, 0, lru), (ACTIVE, 0, lru), (IDLE, 1, lru), (IDLE, 0, lru[::-1])):
+        eng = make(n_hbm_blocks=n, n_host_blocks=8, max_contexts=4, suspended_order=order, **TOY)
+        eng.debug_load_resident(np.arange(n) + 50, [state] * n, stamps, np.zeros(n), np.arange(n), HBM)
+        v, _ = eng.select_victims(HBM, n)
+        assert list(v) == want, (state, order)
+
+
+# ---- movement ------------------------------------------------------------------------------------
+def _payload(key, nbytes):
+    rng = np.random.default_rng(int(key))
+    return rng.integers(0, 256, nbytes, dtype=np.uint8)
+
+
+def offload_reload_round_trip(make, geos=None, layouts=(0, 1)):
+    geos = geos or [TOY, dict(n_layers=3, n_kv_heads=1, head_dim=16), dict(n_layers=1, n_kv_heads=8, head_dim=128)]
+    for geo in geos:
+        for layout in layouts:
+            eng = make(n_hbm_blocks=12, n_host_blocks=6, max_contexts=4, pool_layout=layout, **geo)
+            rng = np.random.default_rng(6)
+            eng.spawn(0)
+            eng.append(0, toks(rng, 16 * 10))
+            call(eng, 0)
+            keys, tier, slot = eng.get_block_map(0)
+            for k, s in zip(keys, slot):
+                eng.write_block(HBM, int(s), _payload(k, eng.block_bytes))
+            # suspended blocks are live: offload copies them to the lowest free host slots, in order
+            rc, n_done, n_dropped = eng.offload([7, 2, 9, 4])
+            assert (rc, n_done, n_dropped) == (0, 4, 0)
+            k2, t2, s2 = eng.get_block_map(0)
+            assert [int(t2[b]) for b in (7, 2, 9, 4)] == [HOST] * 4 and [int(s2[b]) for b in (7, 2, 9, 4)] == [0, 1, 2, 3]
+            for b in (7, 2, 9, 4):
+                assert np.array_equal(eng.read_block(HOST, int(s2[b])), _payload(keys[b], eng.block_bytes))
+            assert eng.get_stats()["occ_hbm"] == 6 and eng.get_stats()["occ_host"] == 4
+            # host tier has 2 slots left: the third live victim does not fit
+            rc, n_done, n_dropped = eng.offload([0, 1, 3])
+            assert (rc, n_done, n_dropped) == (E_NOSPACE, 2, 0)
+            # reload in a different order: lowest free HBM slots
+            free_hbm = sorted(set(range(12)) - {int(s) for s, t in zip(*eng.get_block_map(0)[2:0:-1]) if t == HBM})
+            hs = [int(eng.get_block_map(0)[2][b]) for b in (9, 0, 7)]
+            rc, n_done = eng.reload(hs)
+            assert (rc, n_done) == (0, 3)
+            k3, t3, s3 = eng.get_block_map(0)
+            assert [int(s3[b]) for b in (9, 0, 7)] == free_hbm[:3]
+            for b in range(10):
+                assert np.array_equal(eng.read_block(int(t3[b]), int(s3[b])), _payload(keys[b], eng.block_bytes)), (geo, layout, b)
+            # lookups find blocks in either tier and report where they are
+            a = eng.map_blocks([0], LOOKUP)[0]
+            assert (a["hit_len"], a["n_hit_hbm"], a["n_hit_host"]) == (10, 7, 3)
+            eng.prefill_done(0)
+
+
+def dead_victims_are_dropped_without_copy(make):
+    eng = make(n_hbm_blocks=8, n_host_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(7)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 64))
+    eng.append(0, toks(rng, 64))
+    call(eng, 0)
+    eng.remove(0, 1, 2)                                  # blocks 4..7 dead
+    v, s = eng.select_victims(HBM, 6)
+    assert list(s) == [0, 0, 0, 0, 1, 1]
+    rc, n_done, n_dropped = eng.offload(v)
+    assert (rc, n_done, n_dropped) == (0, 6, 4)
+    st = eng.get_stats()
+    assert (st["occ_hbm"], st["occ_host"], st["dropped"], st["offloaded"]) == (2, 2, 4, 2)
+    assert st["bytes_d2h"] == 2 * eng.block_bytes
+    a = eng.map_blocks([0], LOOKUP)[0]
+    assert (a["n_blocks"], a["hit_len"], a["n_hit_hbm"], a["n_hit_host"]) == (4, 4, 2, 2)
+    eng.prefill_done(0)
+
+
+def compaction(make):
+    eng = make(n_hbm_blocks=16, n_host_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(8)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 16 * 12))
+    call(eng, 0)
+    keys, _, slot = eng.get_block_map(0)
+    for k, s in zip(keys, slot):
+        eng.write_block(HBM, int(s), _payload(k, eng.block_bytes))
+    eng.release(HBM, [1, 4, 5, 10])
+    n_moved = eng.compact(HBM)                           # 8 occupied; movers 8, 9, 11 -> holes 1, 4, 5
+    assert n_moved == 3
+    ent = eng.get_entries(HBM)
+    assert np.all(ent["key"][:8] != 0) and np.all(ent["key"][8:] == 0)
+    assert [int(ent["key"][h]) for h in (1, 4, 5)] == [int(keys[m]) for m in (8, 9, 11)]
+    assert [int(ent["depth"][h]) for h in (1, 4, 5)] == [8, 9, 11]
+    for s in range(8):
+        assert np.array_equal(eng.read_block(HBM, s), _payload(int(ent["key"][s]), eng.block_bytes))
+    assert eng.compact(HBM) == 0
+
+
+def raw_copy_blocks(make):
+    for layout in (0, 1):
+        eng = make(n_hbm_blocks=10, n_host_blocks=10, max_contexts=2, pool_layout=layout, **TOY)
+        for s in range(10):
+            eng.write_block(HBM, s, _payload(1000 + s, eng.block_bytes))
+        eng.copy_blocks(HBM, [3, 9, 0], HOST, [5, 1, 8])
+        for s, d in ((3, 5), (9, 1), (0, 8)):
+            assert np.array_equal(eng.read_block(HOST, d), _payload(1000 + s, eng.block_bytes))
+        eng.copy_blocks(HOST, [5, 8], HBM, [6, 7])
+        assert np.array_equal(eng.read_block(HBM, 6), _payload(1003, eng.block_bytes))
+        assert np.array_equal(eng.read_block(HBM, 7), _payload(1000, eng.block_bytes))
+        eng.copy_blocks(HBM, [1, 2], HBM, [4, 5])
+        assert np.array_equal(eng.read_block(HBM, 4), _payload(1001, eng.block_bytes))
+        assert np.array_equal(eng.read_block(HBM, 3), _payload(1003, eng.block_bytes))   # untouched
+        eng.copy_blocks(HBM, [], HOST, [])                                                # empty list
+
+
+# ---- admission under a full pool; batch semantics ---------------------------------------------------
+def admission_stops_when_full(make):
+    eng = make(n_hbm_blocks=6, n_host_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(10)
+    shared = toks(rng, 32)
+    for c in (0, 1, 2):
+        eng.spawn(c)
+        eng.append(c, shared)
+        eng.append(c, toks(rng, 48))
+    info = eng.map_blocks([0, 1, 2], LOOKUP)
+    assert [int(i["n_blocks"]) for i in info] == [5, 5, 5] and [int(i["hit_len"]) for i in info] == [0, 0, 0]
+    adm = eng.map_blocks([0, 1, 2], ADMIT)
+    # context 0 inserts 5 (slots 0..4); context 1 adopts the 2 shared blocks, inserts 1 (slot 5), then
+    # the pool is full; context 2 adopts the 2 shared blocks and stops at its first absent block
+    assert [int(i["n_admitted"]) for i in adm] == [5, 3, 2]
+    assert [int(i["n_held"]) for i in adm] == [5, 3, 2]
+    ent = eng.get_entries(HBM)
+    assert list(ent["inflight"]) == [3, 3, 1, 1, 1, 1]
+    assert list(ent["depth"]) == [0, 1, 2, 3, 4, 2]
+    assert list(eng.get_block_map(1)[2][:3]) == [0, 1, 5]
+    st = eng.get_stats()
+    assert (st["inserted"], st["adopted"], st["occ_hbm"]) == (6, 4, 6)
+    # nothing evictable while everything is in flight; afterwards ADMIT can continue
+    assert len(eng.select_victims(HBM, 6)[0]) == 0
+    eng.prefill_done(0)
+    assert list(eng.get_entries(HBM)["inflight"]) == [2, 2, 0, 0, 0, 1]
+    v, s = eng.select_victims(HBM, 2)
+    assert list(v) == [4, 3] and list(s) == [1, 1]       # same stamp: chain tail first
+    rc, n_done, n_dropped = eng.offload(v)
+    assert (rc, n_done, n_dropped) == (0, 2, 0)
+    adm = eng.map_blocks([1, 2], ADMIT)
+    assert [int(i["n_admitted"]) for i in adm] == [2, 0] and [int(i["n_held"]) for i in adm] == [5, 2]
+    eng.prefill_done(1)
+    eng.prefill_done(2)
+    assert int(eng.get_entries(HBM)["inflight"].sum()) == 0
+
+
+def lookup_locks_and_orphans(make):
+    eng = make(n_hbm_blocks=8, n_host_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(12)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 96))                         # 6 blocks
+    call(eng, 0)
+    eng.release(HBM, [2])                                # hole in the chain: 3,4,5 become unreachable orphans
+    a = eng.map_blocks([0], LOOKUP)[0]
+    assert (a["hit_len"], a["n_admissible"]) == (2, 4)
+    assert list(eng.get_entries(HBM)["inflight"][:6]) == [1, 1, 0, 0, 0, 0]
+    b = eng.map_blocks([0], ADMIT)[0]
+    assert (b["n_admitted"], b["n_held"]) == (4, 6)      # block 2 re-inserted at slot 2, orphans adopted
+    st = eng.get_stats()
+    assert (st["inserted"], st["adopted"]) == (7, 3)
+    assert list(eng.get_entries(HBM)["inflight"][:6]) == [1] * 6
+    # a hit on a dead block is still a hit (content-addressed) and the block revives
+    eng.prefill_done(0)
+    eng.terminate(0)
+    assert states(eng)[:6] == [DEAD] * 6
+    eng.spawn(1)
+    rng = np.random.default_rng(12)                      # a new context with the same tokens
+    eng.append(1, toks(rng, 96))
+    a = eng.map_blocks([1], LOOKUP)[0]
+    assert a["hit_len"] == 6
+    assert states(eng)[:6] == [ACTIVE] * 6
+    eng.prefill_done(1)
+
+
+# ---- error codes -----------------------------------------------------------------------------------
+def error_codes(make, op_codes):
+    OP = op_codes
+    eng = make(n_hbm_blocks=8, n_host_blocks=2, max_contexts=4, **TOY)
+    rng = np.random.default_rng(13)
+    assert eng.apply_op_rc(OP["APPEND"], 0, tokens=toks(rng, 4)) == E_NOCTX
+    assert eng.apply_op_rc(OP["SPAWN"], 9) == E_INVAL    # id out of range
+    eng.spawn(0)
+    assert eng.apply_op_rc(OP["SPAWN"], 0) == E_INVAL    # id in use
+    assert eng.apply_op_rc(OP["PIN"], 0) == E_INVAL and eng.apply_op_rc(OP["UNPIN"], 0) == E_INVAL
+    assert eng.apply_op_rc(77, 0) == E_INVAL
+    eng.append(0, toks(rng, 40))
+    assert eng.apply_op_rc(OP["REMOVE"], 0, msg_start=0, msg_end=2) == E_RANGE
+    assert eng.apply_op_rc(OP["REMOVE"], 0, msg_start=1, msg_end=1) == E_RANGE
+    assert eng.apply_op_rc(OP["REPLACE"], 0, msg_start=1, msg_end=2, tokens=toks(rng, 4)) == E_RANGE
+    assert eng.apply_op_rc(OP["ONE_OFF"], 0, msg_start=0, msg_end=5) == E_RANGE
+    assert eng.apply_op_rc(OP["FORK"], 1, parent=0, msg_end=2) == E_RANGE
+    assert eng.apply_op_rc(OP["FORK"], 1, parent=3, msg_end=0) == E_NOCTX
+    assert eng.apply_op_rc(OP["FORK"], 0, parent=0, msg_end=0) == E_INVAL
+    assert eng.apply_op_rc(OP["PREFILL_DONE"], 0) == E_STATE
+    assert eng.map_blocks_rc([0], ADMIT)[0] == E_STATE
+    assert eng.map_blocks_rc([0, 0], LOOKUP)[0] == E_INVAL
+    assert eng.map_blocks_rc([0, 2], LOOKUP)[0] == E_NOCTX
+    assert eng.get_stats()["clock"] == 0                 # rejected calls change nothing
+    eng.map_blocks([0], LOOKUP)
+    assert eng.map_blocks_rc([0], LOOKUP)[0] == E_STATE
+    for op in ("APPEND", "REPLACE", "REMOVE", "ONE_OFF"):
+        assert eng.apply_op_rc(OP[op], 0, msg_start=0, msg_end=1, tokens=toks(rng, 4)) == E_STATE
+    assert eng.apply_op_rc(OP["FORK"], 1, parent=0, msg_end=1) == E_STATE
+    eng.map_blocks([0], ADMIT)                           # 2 blocks at slots 0, 1, in flight
+    assert eng.offload([0])[0] == E_STATE
+    assert eng.release_rc(HBM, [1]) == E_STATE
+    assert eng.offload([5])[0] == E_INVAL                # empty slot
+    assert eng.offload([8])[0] == E_RANGE
+    eng.prefill_done(0)
+    assert eng.offload([0, 0])[0] == E_INVAL             # repeated slot
+    assert eng.offload([0, 9, 5])[0] == E_RANGE          # range errors win over the others
+    assert eng.reload([0])[0] == E_INVAL
+    assert eng.release_rc(HOST, [3]) == E_RANGE
+    st = eng.get_stats()
+    assert (st["occ_hbm"], st["occ_host"], st["dropped"]) == (2, 0, 0)
+    assert eng.debug_load_resident_rc([1], [0], [0], [0], [3], HBM) == E_INVAL        # reserved key value
+    assert eng.debug_load_resident_rc([50, 50], [0, 0], [0, 0], [0, 0], [3, 4], HBM) == E_INVAL
+    assert eng.debug_load_resident_rc([50], [0], [0], [0], [0], HBM) == E_INVAL       # slot occupied
+    assert eng.debug_load_resident_rc([int(eng.get_entries(HBM)["key"][0])], [0], [0], [0], [3], HBM) == E_INVAL
+    eng.terminate(0)
+    assert eng.apply_op_rc(OP["APPEND"], 0, tokens=toks(rng, 4)) == E_NOCTX
+    eng.spawn(0)                                         # a terminated id can be reused
+
+
+# ---- zero-length and sub-block inputs ----------------------------------------------------------------
+def degenerate_inputs(make):
+    eng = make(n_hbm_blocks=8, n_host_blocks=2, max_contexts=4, **TOY)
+    rng = np.random.default_rng(14)
+    eng.spawn(0)
+    a, b = call(eng, 0)                                  # empty context
+    assert (a["n_blocks"], a["hit_len"], a["n_admissible"], b["n_held"]) == (0, 0, 0, 0)
+    eng.append(0, toks(rng, 15))                         # no full block
+    a, b = call(eng, 0)
+    assert a["n_blocks"] == 0
+    eng.append(0, toks(rng, 0))                          # empty message
+    eng.append(0, toks(rng, 1))                          # completes block 0
+    a, b = call(eng, 0)
+    assert (a["n_blocks"], b["n_admitted"]) == (1, 1)
+    assert states(eng)[0] == IDLE
+    eng.remove(0, 1, 2)                                  # removing the empty message (starts at token 15)
+    assert states(eng)[0] == DEAD                        # cut = floor(15/16) = 0
+    assert len(eng.select_victims(HBM, 0)[0]) == 0
+    assert eng.offload([])[:2] == (0, 0)
+    assert eng.reload([])[:2] == (0, 0)
+    keys, tier, slot = eng.get_block_map(0)
+    assert len(keys) == 1
+
+
+ALL = [state_machine_single_context, suffix_invalidation, fork_and_shared_kv, one_off_bypass, worked_example,
+       mixed_pool_example, victim_order_bruteforce, one_state_pools_reduce_to_lru, offload_reload_round_trip,
+       dead_victims_are_dropped_without_copy, compaction, raw_copy_blocks, admission_stops_when_full,
+       lookup_locks_and_orphans, degenerate_inputs]

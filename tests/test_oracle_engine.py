@@ -1,0 +1,114 @@
+"""Pins of the CPU oracle's engine semantics: the paper's state-machine sentences, the shared-KV
+example, Algorithm 1's order, brute force on tiny pools, round trips and global invariants."""
+import numpy as np
+import pytest
+
+import scenarios as S
+from paper_2609_39819_b200 import workloads as W
+
+
+@pytest.fixture
+def make(oracle):
+    return lambda **kw: oracle.OracleEngine(**kw)
+
+
+@pytest.mark.parametrize("scenario", S.ALL, ids=lambda f: f.__name__)
+def test_scenario(make, scenario):
+    scenario(make)
+
+
+def test_mixed_pool_lru_switch(make):
+    S.mixed_pool_example(make, order=1)
+
+
+def test_error_codes(make, oracle):
+    ops = {k[3:]: getattr(oracle, k) for k in dir(oracle) if k.startswith("OP_")}
+    S.error_codes(make, ops)
+
+
+def check_invariants(eng):
+    """Global invariants that hold after every call whatever the trace."""
+    st = eng.get_stats()
+    keys_all = []
+    for tier, n in ((0, eng.n_hbm_blocks), (1, eng.n_host_blocks)):
+        ent = eng.get_entries(tier)
+        occ = int((ent["key"] != 0).sum())
+        assert occ == st["occ_hbm" if tier == 0 else "occ_host"] <= n      # occupancy never exceeds capacity
+        keys_all.append(ent["key"][ent["key"] != 0])
+        states = eng.get_states(tier)
+        assert np.all((states == 0xFF) == (ent["key"] == 0))
+        assert np.all(ent["inflight"][ent["key"] == 0] == 0)
+    keys_all = np.concatenate(keys_all)
+    assert len(np.unique(keys_all)) == len(keys_all)                        # each key in exactly one (tier, slot)
+    assert st["hits_hbm"] + st["hits_host"] + st["misses"] == st["blocks_hashed"]
+    assert st["inserted"] - st["dropped"] == st["occ_hbm"] + st["occ_host"]
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3, 4, 5, 7, 39, 63, 86, 102, 120])
+def test_c1_replay_invariants_and_bruteforce_states(make, seed):
+    eng = make(n_hbm_blocks=128, n_host_blocks=512, max_contexts=64, **W.GEO_TOY.kwargs())
+    opt = W.ReplayOptions(payload=W.payload_normal_bf16, verify_payload_every=1)
+    for _i, kind, rec in W.replay(eng, W.trace_c1(seed), opt):
+        if kind != "call":
+            continue
+        assert rec["payload_ok"]
+        check_invariants(eng)
+        # classification equals the literal double loop over blocks x mappings
+        for tier in (0, 1):
+            assert np.array_equal(eng.get_states(tier), eng.classify_bruteforce(tier))
+        # no victim is in flight; victims come in Algorithm 1's order
+        if "vstates" in rec:
+            assert np.all(np.diff(rec["vstates"].astype(int)) >= 0)
+        assert int(eng.get_entries(0)["inflight"].sum() + eng.get_entries(1)["inflight"].sum()) == 0
+
+
+def test_c1_pool_is_under_pressure():
+    """The tiny configuration must actually exercise eviction, offload and reload."""
+    from oracle import kvt_oracle
+    tot = {"offloaded": 0, "reloaded": 0, "dropped": 0, "adopted": 0}
+    for seed in (7, 39, 63, 86, 120):
+        eng = kvt_oracle.OracleEngine(n_hbm_blocks=128, n_host_blocks=512, max_contexts=64, **W.GEO_TOY.kwargs())
+        for _ in W.replay(eng, W.trace_c1(seed), W.ReplayOptions(payload=None, record_states=False)):
+            pass
+        st = eng.get_stats()
+        for k in tot:
+            tot[k] += st[k]
+    assert tot["offloaded"] > 0 and tot["reloaded"] > 0 and tot["dropped"] > 0, tot
+
+
+def test_scaled_c2_and_c3_traces_replay(make):
+    eng = make(n_hbm_blocks=96, n_host_blocks=64, max_contexts=64, **W.GEO_TOY.kwargs())
+    n_calls = 0
+    for _i, kind, rec in W.replay(eng, W.trace_c2(1, scale=1 / 32), W.ReplayOptions(payload=W.payload_pattern, verify_payload_every=5)):
+        n_calls += kind == "call"
+    check_invariants(eng)
+    assert n_calls > 20 and W.verify_payload(eng, W.payload_pattern)
+    st = eng.get_stats()
+    assert st["offloaded"] > 0 and st["reloaded"] >= 0
+    trace, n_ctx = W.trace_c3(1, n_sessions=6, scale=1 / 64)
+    eng = make(n_hbm_blocks=256, n_host_blocks=256, max_contexts=n_ctx, **W.GEO_TOY.kwargs())
+    for _i, kind, rec in W.replay(eng, trace, W.ReplayOptions(payload=None, record_states=False)):
+        pass
+    check_invariants(eng)
+    assert eng.get_stats()["n_contexts"] == 0
+
+
+def test_incremental_appends_hash_like_one_shot(make, oracle):
+    """Hashing a context after piecewise appends equals hashing the concatenation in one shot."""
+    rng = np.random.default_rng(21)
+    eng = make(n_hbm_blocks=64, n_host_blocks=8, max_contexts=4, **S.TOY)
+    eng.spawn(0)
+    parts = []
+    for n in (5, 27, 16, 1, 100, 63):
+        parts.append(S.toks(rng, n))
+        eng.append(0, parts[-1])
+        S.call(eng, 0)
+        assert np.array_equal(eng.get_block_map(0)[0], oracle.hash_tokens(np.concatenate(parts)))
+
+
+def test_kv_size_sanity():
+    """Section 1 quotes 93 GB of KV for a 258K-token request; the GLM-scale geometry used here gives
+    a figure of the same size (within 5%)."""
+    bytes_per_token = W.GEO_GLM.block_bytes // 16
+    assert bytes_per_token == 376832
+    assert abs(258_000 * bytes_per_token / 1e9 - 93) / 93 < 0.05
