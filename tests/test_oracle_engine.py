@@ -84,7 +84,7 @@ def test_scaled_c2_and_c3_traces_replay(make):
     check_invariants(eng)
     assert n_calls > 20 and W.verify_payload(eng, W.payload_pattern)
     st = eng.get_stats()
-    assert st["offloaded"] > 0 and st["reloaded"] >= 0
+    assert st["dropped"] > 0      # a single session only ever evicts its own dead suffixes
     trace, n_ctx = W.trace_c3(1, n_sessions=6, scale=1 / 64)
     eng = make(n_hbm_blocks=256, n_host_blocks=256, max_contexts=n_ctx, **W.GEO_TOY.kwargs())
     for _i, kind, rec in W.replay(eng, trace, W.ReplayOptions(payload=None, record_states=False)):
