@@ -117,12 +117,14 @@ typedef struct kvt_config {
   uint32_t n_host_blocks;    /* slots in the host tier (may be 0) */
   uint32_t table_capacity;   /* power of two, >= 2 * (n_hbm_blocks + n_host_blocks) */
   uint32_t max_contexts;     /* context ids are 0 .. max_contexts-1 */
+  uint32_t max_messages;     /* upper bound on messages with materialised positions, all contexts together */
   uint32_t max_batch_blocks; /* upper bound on the blocks hashed by one kvt_map_blocks call and on n of one list call */
+  uint32_t reserved0;        /* must be 0 */
   uint64_t max_tokens;       /* capacity of the device token arena, in tokens */
   uint64_t max_key_blocks;   /* capacity of the per-context key lists, in blocks (all contexts together) */
   uint64_t hash_seed;        /* seed of the block hash */
   uint32_t suspended_order;  /* KVT_ORDER_* */
-  uint32_t reserved;         /* must be 0 */
+  uint32_t reserved1;        /* must be 0 */
   void *hbm_pool;  uint64_t hbm_pool_bytes;   /* device; NULL/0 = metadata-only engine (no payload is moved) */
   void *host_pool; uint64_t host_pool_bytes;  /* device-accessible pinned host memory; NULL/0 if metadata-only */
   void *dev_meta;  uint64_t dev_meta_bytes;   /* device metadata + scratch arena, 256-byte aligned */

@@ -1,0 +1,1103 @@
+// kvt_engine.cu — host control plane and C ABI of libkvt.so (see include/kvt.h for the contract).
+//
+// The host side keeps only what a data-parallel kernel cannot: per-context message lists (lengths
+// and message-level states, Section 5.2), the materialised message bounds (Section 5.1), range
+// allocators for the caller-provided arenas, counts of free slots, and the logical clock. Token
+// values, block keys, the block table, per-block metadata and payloads live on the device and are
+// only touched by the kernels in kvt_kernels.cuh. There is no CPU fallback for any stage.
+#include "kvt_kernels.cuh"
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <string>
+#include <vector>
+
+#include "../../include/kvt.h"
+
+using namespace kvt;
+
+namespace {
+
+constexpr u32 MS_ACTIVE = 0, MS_SUSPENDED = 1, MS_TEMPORARY = 3;
+inline u8 msg_rank(u8 s) { return s == MS_ACTIVE ? 2 : (s == MS_SUSPENDED ? 1 : 0); }
+
+inline u64 round_up(u64 x, u64 a) { return (x + a - 1) / a * a; }
+inline u32 cdiv(u64 a, u64 b) { return (u32)((a + b - 1) / b); }
+inline u32 bit_length(u32 x) { u32 n = 0; while (x) { ++n; x >>= 1; } return n ? n : 1; }
+
+// First-fit range allocator over a caller-provided arena (units: elements).
+struct RangeAlloc {
+  std::map<u64, u64> free_;
+  u64 align = 1;
+  void init(u64 total, u64 a) { free_.clear(); align = a; if (total) free_[0] = total / a * a; }
+  bool alloc(u64 n, u64 *off) {
+    n = round_up(std::max<u64>(n, 1), align);
+    for (auto it = free_.begin(); it != free_.end(); ++it) {
+      if (it->second >= n) {
+        *off = it->first;
+        u64 rest = it->second - n, ro = it->first + n;
+        free_.erase(it);
+        if (rest) free_[ro] = rest;
+        return true;
+      }
+    }
+    return false;
+  }
+  void release(u64 off, u64 n) {
+    n = round_up(std::max<u64>(n, 1), align);
+    auto nx = free_.lower_bound(off);
+    if (nx != free_.end() && off + n == nx->first) { n += nx->second; nx = free_.erase(nx); }
+    if (nx != free_.begin()) {
+      auto pv = std::prev(nx);
+      if (pv->first + pv->second == off) { pv->second += n; return; }
+    }
+    free_[off] = n;
+  }
+};
+
+struct Msg { u32 len; u8 state; };
+struct KeySeg { u64 off = 0, cap = 0; u32 refs = 0; };
+
+struct Ctx {
+  bool live = false, one_off = false, in_flight = false;
+  std::vector<Msg> msgs;
+  std::vector<std::pair<u32, u32>> mat_bounds;  // bounds of the leading messages still valid in the materialised layout
+  u32 mat_blocks = 0;      // blocks of the materialised token sequence (keys in the key segment)
+  u32 valid_blocks = 0, held = 0, hit_len = 0, n_hit_hbm = 0, n_hit_host = 0, n_admissible = 0;
+  u64 tok_off = 0, tok_cap = 0, tok_len = 0;   // device token buffer = concatenation of the current messages
+  int keyseg = -1;
+};
+
+struct DevLayout {
+  u64 tab, e_key, e_stamp, e_depth, e_infl, e_rank, e_tslot, e_mark, e_floor, keys, status;
+  u64 s0, s1, s2, s3, ids, ids2, pair_src, pair_dst, freelist, tiles, agg, carry, desc, ctxres;
+  u64 m_start, m_end, m_rank, keyA, keyB, valA, valB, rcounts, out_slots, out_states, map_tier, map_slot;
+  u64 total;
+  u64 LB, Nt, N;
+};
+
+DevLayout make_layout(const kvt_config &c) {
+  DevLayout L{};
+  u64 N = (u64)c.n_hbm_blocks + c.n_host_blocks, Nt = std::max(c.n_hbm_blocks, c.n_host_blocks);
+  u64 B = c.max_batch_blocks, LB = std::max<u64>(B, Nt), C = c.max_contexts, Mm = c.max_messages;
+  L.LB = LB; L.Nt = Nt; L.N = N;
+  u64 off = 0;
+  auto take = [&](u64 bytes) { u64 o = off; off = round_up(off + bytes, 256); return o; };
+  L.tab = take((u64)c.table_capacity * 16);
+  L.e_key = take(N * 8); L.e_stamp = take(N * 4); L.e_depth = take(N * 4); L.e_infl = take(N * 4);
+  L.e_rank = take(N * 4); L.e_tslot = take(N * 4); L.e_mark = take(N * 4); L.e_floor = take(N);
+  L.keys = take(c.max_key_blocks * 8);
+  L.status = take(ST_WORDS * 4);
+  L.s0 = take(LB * 4); L.s1 = take(LB * 4); L.s2 = take(LB * 4); L.s3 = take(LB * 4);
+  L.ids = take(LB * 4); L.ids2 = take(LB * 4); L.pair_src = take(LB * 4); L.pair_dst = take(LB * 4);
+  L.freelist = take(LB * 4);
+  L.tiles = take((std::max(LB, N) / SCAN_TILE + 2) * 4);
+  u64 n_chunks = B / CHUNK + C + 1;
+  L.agg = take(n_chunks * 8); L.carry = take(n_chunks * 8);
+  L.desc = take(C * 32);
+  L.ctxres = take(C * 16);
+  L.m_start = take(Mm * 4); L.m_end = take(Mm * 4); L.m_rank = take(Mm);
+  L.keyA = take(Nt * 8); L.keyB = take(Nt * 8); L.valA = take(Nt * 4); L.valB = take(Nt * 4);
+  L.rcounts = take(256ull * (Nt / SORT_TILE + 1) * 4);
+  L.out_slots = take(Nt * 4); L.out_states = take(Nt);
+  L.map_tier = take(B); L.map_slot = take(B * 4);
+  L.total = off;
+  return L;
+}
+
+}  // namespace
+
+struct kvt_engine {
+  kvt_config cfg;
+  DevLayout L;
+  u8 *meta = nullptr;
+  u32 *d_tokens = nullptr;
+  Table tab; Entries ent;
+  u64 *d_keys; u32 *d_status;
+  u64 h0;
+  u64 chunk_bytes, n_chunks, block_bytes;
+  bool metadata_only;
+  int sm_count = 148;
+  // host state
+  std::vector<Ctx> ctxs;
+  std::vector<KeySeg> segs;
+  std::vector<int> free_segs;
+  RangeAlloc tok_alloc, key_alloc;
+  u32 now = 0, max_depth = 0;
+  u32 occ[2] = {0, 0};
+  u32 tombs = 0;
+  bool dirty = true;
+  kvt_stats st{};
+  std::string err;
+  // pinned host staging
+  u8 *stage = nullptr;
+  u32 *h_status; u8 *h_desc; u32 *h_ctxres; u32 *h_mstart, *h_mend; u8 *h_mrank; u32 *h_ids, *h_ids2;
+  cudaEvent_t ev_upload = nullptr;
+  bool upload_pending = false;
+
+  template <class T> T *dp(u64 off) const { return reinterpret_cast<T *>(meta + off); }
+  u32 tier_slots(u32 t) const { return t == KVT_TIER_HBM ? cfg.n_hbm_blocks : cfg.n_host_blocks; }
+  u32 tier_e0(u32 t) const { return t == KVT_TIER_HBM ? 0 : cfg.n_hbm_blocks; }
+};
+
+namespace {
+
+#define CU(call)                                                                                   \
+  do {                                                                                             \
+    cudaError_t _e = (call);                                                                       \
+    if (_e != cudaSuccess) {                                                                       \
+      e->err = std::string(#call) + ": " + cudaGetErrorString(_e);                                 \
+      return KVT_E_CUDA;                                                                           \
+    }                                                                                              \
+  } while (0)
+
+int32_t fail(kvt_engine *e, int32_t code, const char *msg) { e->err = msg; return code; }
+
+int32_t launch_ok(kvt_engine *e) {
+  cudaError_t x = cudaGetLastError();
+  if (x != cudaSuccess) { e->err = std::string("kernel launch: ") + cudaGetErrorString(x); return KVT_E_CUDA; }
+  return KVT_OK;
+}
+#define LAUNCH_CHECK() do { int32_t _r = launch_ok(e); if (_r) return _r; } while (0)
+
+// Staging buffers are reused by every call: wait until the previous upload has been consumed.
+int32_t stage_acquire(kvt_engine *e) {
+  if (e->upload_pending) { CU(cudaEventSynchronize(e->ev_upload)); e->upload_pending = false; }
+  return KVT_OK;
+}
+int32_t stage_release(kvt_engine *e, cudaStream_t s) {
+  CU(cudaEventRecord(e->ev_upload, s));
+  e->upload_pending = true;
+  return KVT_OK;
+}
+
+int32_t status_zero(kvt_engine *e, cudaStream_t s) {
+  CU(cudaMemsetAsync(e->d_status, 0, ST_WORDS * 4, s));
+  return KVT_OK;
+}
+// Copies the status block to the host and waits for the stream.
+int32_t status_fetch(kvt_engine *e, cudaStream_t s) {
+  CU(cudaMemcpyAsync(e->h_status, e->d_status, ST_WORDS * 4, cudaMemcpyDeviceToHost, s));
+  CU(cudaStreamSynchronize(s));
+  return KVT_OK;
+}
+int32_t status_code(kvt_engine *e) {
+  u32 b = e->h_status[ST_ERR];
+  if (!b) return KVT_OK;
+  if (b & (DERR_PROBE | DERR_CORRUPT)) return fail(e, KVT_E_DEVICE, b & DERR_PROBE ? "table probe cap exceeded" : "corrupt metadata");
+  if (b & DERR_RANGE) return fail(e, KVT_E_RANGE, "slot id out of range");
+  if (b & DERR_INVAL) return fail(e, KVT_E_INVAL, "slot empty, repeated, or key already resident");
+  return fail(e, KVT_E_STATE, "block is in flight");
+}
+
+Ctx *get_ctx(kvt_engine *e, u32 id) {
+  if (id >= e->ctxs.size() || !e->ctxs[id].live) return nullptr;
+  return &e->ctxs[id];
+}
+
+void seg_deref(kvt_engine *e, int id) {
+  if (id < 0) return;
+  KeySeg &s = e->segs[id];
+  if (--s.refs == 0) { e->key_alloc.release(s.off, s.cap); e->free_segs.push_back(id); }
+}
+int seg_new(kvt_engine *e, u64 n) {
+  u64 off;
+  if (!e->key_alloc.alloc(n, &off)) return -1;
+  int id;
+  if (!e->free_segs.empty()) { id = e->free_segs.back(); e->free_segs.pop_back(); }
+  else { id = (int)e->segs.size(); e->segs.emplace_back(); }
+  e->segs[id] = KeySeg{off, round_up(std::max<u64>(n, 1), e->key_alloc.align), 1};
+  return id;
+}
+
+// ---- ordered compaction helper -----------------------------------------------------------------------
+template <class Pred, class Emit>
+int32_t compact_indices(kvt_engine *e, cudaStream_t s, Pred pred, Emit emit, u32 n, int total_word) {
+  u32 *tiles = e->dp<u32>(e->L.tiles);
+  u32 nt = cdiv(n, SCAN_TILE);
+  if (nt == 0) { CU(cudaMemsetAsync(e->d_status + total_word, 0, 4, s)); return KVT_OK; }
+  k_tile_count<<<nt, SCAN_TILE, 0, s>>>(pred, n, tiles);
+  k_scan_tiles<<<1, 1024, 0, s>>>(tiles, nt, e->d_status + total_word);
+  k_tile_scatter<<<nt, SCAN_TILE, 0, s>>>(pred, emit, n, tiles);
+  LAUNCH_CHECK();
+  return KVT_OK;
+}
+
+int32_t table_rebuild(kvt_engine *e, cudaStream_t s) {
+  k_table_clear<<<cdiv((u64)e->tab.mask + 1, 256), 256, 0, s>>>(e->tab);
+  k_table_reinsert<<<cdiv(e->ent.n_total, 256), 256, 0, s>>>(e->tab, e->ent, e->d_status);
+  LAUNCH_CHECK();
+  e->tombs = 0;
+  e->st.table_rebuilds++;
+  return KVT_OK;
+}
+
+int32_t maybe_rebuild(kvt_engine *e, cudaStream_t s) {
+  if ((u64)e->tombs * 8 > (u64)e->tab.mask + 1) return table_rebuild(e, s);
+  return KVT_OK;
+}
+
+PoolView pool_view(kvt_engine *e, u32 tier) {
+  PoolView v;
+  if (tier == KVT_TIER_HBM) {
+    v.base = (u8 *)e->cfg.hbm_pool;
+    v.n_slots = e->cfg.n_hbm_blocks;
+    if (e->cfg.pool_layout == KVT_LAYOUT_LAYER_MAJOR) { v.slot_stride = e->chunk_bytes; v.chunk_stride = e->chunk_bytes * e->cfg.n_hbm_blocks; }
+    else { v.slot_stride = e->block_bytes; v.chunk_stride = e->chunk_bytes; }
+  } else {
+    v.base = (u8 *)e->cfg.host_pool;
+    v.n_slots = e->cfg.n_host_blocks;
+    v.slot_stride = e->block_bytes; v.chunk_stride = e->chunk_bytes;
+  }
+  return v;
+}
+
+int32_t launch_mover(kvt_engine *e, cudaStream_t s, u32 st, const u32 *src, u32 dt, const u32 *dst, u32 n_max,
+                     const u32 *n_dev) {
+  if (e->metadata_only || n_max == 0) return KVT_OK;
+  MoveArgs a;
+  a.src = pool_view(e, st); a.dst = pool_view(e, dt);
+  a.src_ids = src; a.dst_ids = dst; a.n_pairs = n_max; a.n_pairs_dev = n_dev;
+  a.n_chunks = (u32)e->n_chunks; a.chunk_bytes = (u32)e->chunk_bytes; a.status = e->d_status;
+  u64 items = (u64)n_max * e->n_chunks;
+  u32 grid = (u32)std::min<u64>(items, (u64)e->sm_count * 8);
+  k_move_blocks<4><<<grid, 256, 0, s>>>(a);
+  LAUNCH_CHECK();
+  return KVT_OK;
+}
+
+// ---- classification -------------------------------------------------------------------------------------
+int32_t do_classify(kvt_engine *e, cudaStream_t s) {
+  int32_t r = stage_acquire(e);
+  if (r) return r;
+  ClsCtx *hd = reinterpret_cast<ClsCtx *>(e->h_desc);
+  u32 nc = 0, nm = 0, nmap = 0;
+  for (Ctx &c : e->ctxs) {
+    if (!c.live || c.valid_blocks == 0 || c.keyseg < 0) continue;
+    ClsCtx d;
+    d.key_off = e->segs[c.keyseg].off; d.map_base = nmap; d.valid = c.valid_blocks; d.msg_base = nm;
+    u32 k = 0;
+    for (size_t j = 0; j < c.mat_bounds.size(); ++j) {
+      if (c.mat_bounds[j].first >= c.valid_blocks * 16ull) break;  // later messages touch no mapped block
+      if (nm + k >= e->cfg.max_messages) return fail(e, KVT_E_NOSPACE, "max_messages exceeded");
+      e->h_mstart[nm + k] = c.mat_bounds[j].first;
+      e->h_mend[nm + k] = c.mat_bounds[j].second;
+      e->h_mrank[nm + k] = msg_rank(c.msgs[j].state);
+      ++k;
+    }
+    d.n_msgs = k;
+    nm += k; nmap += c.valid_blocks;
+    hd[nc++] = d;
+  }
+  k_rank_reset<<<cdiv(e->ent.n_total, 256), 256, 0, s>>>(e->ent);
+  if (nmap) {
+    CU(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nc * sizeof(ClsCtx), cudaMemcpyHostToDevice, s));
+    CU(cudaMemcpyAsync(e->dp<u8>(e->L.m_start), e->h_mstart, nm * 4ull, cudaMemcpyHostToDevice, s));
+    CU(cudaMemcpyAsync(e->dp<u8>(e->L.m_end), e->h_mend, nm * 4ull, cudaMemcpyHostToDevice, s));
+    CU(cudaMemcpyAsync(e->dp<u8>(e->L.m_rank), e->h_mrank, nm, cudaMemcpyHostToDevice, s));
+    ClsArgs a;
+    a.tab = e->tab; a.ent = e->ent; a.keys = e->d_keys; a.ctx = e->dp<ClsCtx>(e->L.desc); a.n_ctx = nc; a.n_map = nmap;
+    a.m_start = e->dp<u32>(e->L.m_start); a.m_end = e->dp<u32>(e->L.m_end); a.m_rank = e->dp<u8>(e->L.m_rank);
+    a.status = e->d_status;
+    k_classify<<<cdiv(nmap, 256), 256, 0, s>>>(a);
+    r = stage_release(e, s);
+    if (r) return r;
+  }
+  LAUNCH_CHECK();
+  e->dirty = false;
+  return KVT_OK;
+}
+
+int32_t ensure_classified(kvt_engine *e, cudaStream_t s) { return e->dirty ? do_classify(e, s) : KVT_OK; }
+
+// ---- token buffers ---------------------------------------------------------------------------------------
+int32_t copy_tokens_in(kvt_engine *e, cudaStream_t s, u64 dst_tok, const u32 *src, u32 n, bool on_device) {
+  if (!n) return KVT_OK;
+  CU(cudaMemcpyAsync(e->d_tokens + dst_tok, src, (u64)n * 4, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, s));
+  return KVT_OK;
+}
+
+u64 grow_cap(u64 need) { return round_up(std::max<u64>(need + need / 4, 1024), 64); }
+
+int32_t unlock_held(kvt_engine *e, Ctx &c, cudaStream_t s, bool stamp) {
+  if (c.held && c.keyseg >= 0) {
+    k_unlock<<<cdiv(c.held, 256), 256, 0, s>>>(e->tab, e->ent, e->d_keys + e->segs[c.keyseg].off, c.held, e->now,
+                                                stamp ? 1u : 0u, e->d_status);
+    LAUNCH_CHECK();
+  }
+  c.held = 0;
+  return KVT_OK;
+}
+
+// Index of the first block >= from made only of Temporary tokens, or n_blocks (Algorithm 1's bypass).
+u32 first_temporary_block(const Ctx &c, u32 from, u32 n_blocks) {
+  u64 pos = 0;
+  bool in_run = false;
+  u64 run_s = 0;
+  auto close_run = [&](u64 run_e) -> u32 {
+    u64 b0 = std::max<u64>((run_s + 15) / 16, from), b1 = run_e / 16;  // blocks fully inside [run_s, run_e)
+    if (b0 < b1 && b0 < n_blocks) return (u32)b0;
+    return 0xFFFFFFFFu;
+  };
+  for (const Msg &m : c.msgs) {
+    if (m.len) {
+      bool temp = msg_rank(m.state) == 0;
+      if (temp && !in_run) { in_run = true; run_s = pos; }
+      if (!temp && in_run) { in_run = false; u32 b = close_run(pos); if (b != 0xFFFFFFFFu) return b; }
+    }
+    pos += m.len;
+  }
+  if (in_run) { u32 b = close_run(pos); if (b != 0xFFFFFFFFu) return b; }
+  return n_blocks;
+}
+
+}  // namespace
+
+// =========================================================================================================
+// C ABI
+// =========================================================================================================
+extern "C" {
+
+int32_t kvt_query_sizes(const kvt_config *cfg, uint64_t *meta_bytes, uint64_t *token_bytes) {
+  if (!cfg || !meta_bytes || !token_bytes) return KVT_E_INVAL;
+  *meta_bytes = make_layout(*cfg).total;
+  *token_bytes = round_up(cfg->max_tokens * 4, 256);
+  return KVT_OK;
+}
+
+int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
+  if (!cfg || !out) return KVT_E_INVAL;
+  const kvt_config &c = *cfg;
+  if (c.abi_version != KVT_ABI_VERSION || c.block_tokens != 16 || !c.n_layers || !c.n_kv_heads || !c.head_dim ||
+      !c.elem_bytes || c.pool_layout > 1 || !c.n_hbm_blocks || !c.max_contexts || !c.max_batch_blocks ||
+      !c.max_messages || c.suspended_order > 1 || c.reserved0 || c.reserved1 || !c.dev_meta || !c.dev_tokens)
+    return KVT_E_INVAL;
+  u64 N = (u64)c.n_hbm_blocks + c.n_host_blocks;
+  if (N >= CLAIM_BIT || c.max_batch_blocks >= CLAIM_BIT) return KVT_E_INVAL;
+  if (c.table_capacity < 2 * N || (c.table_capacity & (c.table_capacity - 1))) return KVT_E_INVAL;
+  if (((uintptr_t)c.dev_meta & 255) || ((uintptr_t)c.dev_tokens & 255)) return KVT_E_INVAL;
+  DevLayout L = make_layout(c);
+  if (c.dev_meta_bytes < L.total || c.dev_tokens_bytes < c.max_tokens * 4) return KVT_E_INVAL;
+  u64 chunk_bytes = 16ull * c.n_kv_heads * c.head_dim * c.elem_bytes, n_chunks = 2ull * c.n_layers;
+  bool meta_only = c.hbm_pool == nullptr;
+  if (!meta_only) {
+    if (c.hbm_pool_bytes < chunk_bytes * n_chunks * c.n_hbm_blocks || ((uintptr_t)c.hbm_pool & 15)) return KVT_E_INVAL;
+    if (c.n_host_blocks && (!c.host_pool || c.host_pool_bytes < chunk_bytes * n_chunks * c.n_host_blocks ||
+                            ((uintptr_t)c.host_pool & 15)))
+      return KVT_E_INVAL;
+  }
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return KVT_E_CUDA;
+  kvt_engine *e = new kvt_engine();
+  e->cfg = c; e->L = L;
+  e->meta = (u8 *)c.dev_meta; e->d_tokens = (u32 *)c.dev_tokens;
+  e->chunk_bytes = chunk_bytes; e->n_chunks = n_chunks; e->block_bytes = chunk_bytes * n_chunks;
+  e->metadata_only = meta_only;
+  cudaDeviceGetAttribute(&e->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  e->tab.slots = e->dp<TSlot>(L.tab); e->tab.mask = c.table_capacity - 1;
+  e->tab.shift = 64 - (bit_length(c.table_capacity) - 1);
+  e->ent.key = e->dp<u64>(L.e_key); e->ent.stamp = e->dp<u32>(L.e_stamp); e->ent.depth = e->dp<u32>(L.e_depth);
+  e->ent.infl = e->dp<u32>(L.e_infl); e->ent.rank = e->dp<u32>(L.e_rank); e->ent.tslot = e->dp<u32>(L.e_tslot);
+  e->ent.mark = e->dp<u32>(L.e_mark); e->ent.floor = e->dp<u8>(L.e_floor);
+  e->ent.n_hbm = c.n_hbm_blocks; e->ent.n_total = (u32)N;
+  e->d_keys = e->dp<u64>(L.keys); e->d_status = e->dp<u32>(L.status);
+  e->h0 = hash_h0(c.hash_seed);
+  e->ctxs.resize(c.max_contexts);
+  e->tok_alloc.init(c.max_tokens, 64);
+  e->key_alloc.init(c.max_key_blocks, 32);
+  // pinned staging
+  u64 C = c.max_contexts, Mm = c.max_messages, LB = L.LB;
+  u64 o_status = 0, o_desc = 256, o_ctxres = o_desc + round_up(C * 32, 256), o_ms = o_ctxres + round_up(C * 16, 256),
+      o_me = o_ms + round_up(Mm * 4, 256), o_mr = o_me + round_up(Mm * 4, 256), o_ids = o_mr + round_up(Mm, 256),
+      o_ids2 = o_ids + round_up(LB * 4, 256), total = o_ids2 + round_up(LB * 4, 256);
+  if (cudaHostAlloc((void **)&e->stage, total, cudaHostAllocDefault) != cudaSuccess) { delete e; return KVT_E_CUDA; }
+  e->h_status = (u32 *)(e->stage + o_status); e->h_desc = e->stage + o_desc; e->h_ctxres = (u32 *)(e->stage + o_ctxres);
+  e->h_mstart = (u32 *)(e->stage + o_ms); e->h_mend = (u32 *)(e->stage + o_me); e->h_mrank = e->stage + o_mr;
+  e->h_ids = (u32 *)(e->stage + o_ids); e->h_ids2 = (u32 *)(e->stage + o_ids2);
+  cudaStream_t s = (cudaStream_t)stream;
+  bool ok = cudaEventCreateWithFlags(&e->ev_upload, cudaEventDisableTiming) == cudaSuccess;
+  // everything except the key arena and scratch must start at zero; the table needs ent = NONE
+  ok = ok && cudaMemsetAsync(e->meta + L.e_key, 0, L.keys - L.e_key, s) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(e->d_status, 0, ST_WORDS * 4, s) == cudaSuccess;
+  if (ok) {
+    k_table_clear<<<cdiv((u64)c.table_capacity, 256), 256, 0, s>>>(e->tab);
+    ok = cudaGetLastError() == cudaSuccess && cudaStreamSynchronize(s) == cudaSuccess;
+  }
+  if (!ok) { cudaFreeHost(e->stage); if (e->ev_upload) cudaEventDestroy(e->ev_upload); delete e; return KVT_E_CUDA; }
+  *out = e;
+  return KVT_OK;
+}
+
+int32_t kvt_destroy(kvt_engine *e) {
+  if (!e) return KVT_E_INVAL;
+  cudaDeviceSynchronize();
+  if (e->ev_upload) cudaEventDestroy(e->ev_upload);
+  if (e->stage) cudaFreeHost(e->stage);
+  delete e;
+  return KVT_OK;
+}
+
+int32_t kvt_last_error(kvt_engine *e, char *buf, uint32_t cap) {
+  if (!e || !buf || !cap) return KVT_E_INVAL;
+  std::snprintf(buf, cap, "%s", e->err.c_str());
+  return KVT_OK;
+}
+
+int32_t kvt_get_stats(kvt_engine *e, kvt_stats *out) {
+  if (!e || !out) return KVT_E_INVAL;
+  kvt_stats s = e->st;
+  s.clock = e->now;
+  s.n_contexts = 0;
+  for (const Ctx &c : e->ctxs) s.n_contexts += c.live;
+  s.occ_hbm = e->occ[0]; s.occ_host = e->occ[1];
+  s.tombstones = e->tombs;
+  *out = s;
+  return KVT_OK;
+}
+
+// ---- stage 0 -----------------------------------------------------------------------------------------------
+int32_t kvt_apply_op(kvt_engine *e, const kvt_op *op, void *stream) {
+  if (!e || !op) return KVT_E_INVAL;
+  cudaStream_t s = (cudaStream_t)stream;
+  const u32 id = op->ctx;
+  const bool on_dev = op->flags & KVT_OPF_TOKENS_ON_DEVICE;
+  if (op->op == KVT_OP_SPAWN) {
+    if (id >= e->ctxs.size() || e->ctxs[id].live) return fail(e, KVT_E_INVAL, "spawn: context id out of range or in use");
+    e->ctxs[id] = Ctx();
+    e->ctxs[id].live = true;
+    e->dirty = true;
+    return KVT_OK;
+  }
+  if (op->op == KVT_OP_FORK) {
+    if (id >= e->ctxs.size() || e->ctxs[id].live) return fail(e, KVT_E_INVAL, "fork: child id out of range or in use");
+    Ctx *p = get_ctx(e, op->parent);
+    if (!p) return fail(e, KVT_E_NOCTX, "fork: unknown parent");
+    if (p->in_flight) return fail(e, KVT_E_STATE, "fork: parent is in flight");
+    if (op->msg_end > p->msgs.size()) return fail(e, KVT_E_RANGE, "fork: end beyond the parent's messages");
+    Ctx k;
+    k.live = true;
+    u64 T = 0;
+    for (u32 j = 0; j < op->msg_end; ++j) { k.msgs.push_back(Msg{p->msgs[j].len, (u8)MS_ACTIVE}); T += p->msgs[j].len; }
+    k.tok_cap = grow_cap(T);
+    if (!e->tok_alloc.alloc(k.tok_cap, &k.tok_off)) return fail(e, KVT_E_NOSPACE, "token arena full");
+    k.tok_len = T;
+    if (T) {
+      cudaError_t ce = cudaMemcpyAsync(e->d_tokens + k.tok_off, e->d_tokens + p->tok_off, T * 4, cudaMemcpyDeviceToDevice, s);
+      if (ce != cudaSuccess) { e->tok_alloc.release(k.tok_off, k.tok_cap); e->err = cudaGetErrorString(ce); return KVT_E_CUDA; }
+    }
+    u32 m = std::min<u32>(op->msg_end, (u32)p->mat_bounds.size());
+    u32 Tm = m ? p->mat_bounds[m - 1].second : 0;
+    k.mat_bounds.assign(p->mat_bounds.begin(), p->mat_bounds.begin() + m);
+    k.mat_blocks = Tm / 16;
+    k.valid_blocks = std::min<u32>(Tm / 16, p->valid_blocks);
+    if (k.mat_blocks && p->keyseg >= 0) { k.keyseg = p->keyseg; e->segs[p->keyseg].refs++; }  // equal prefixes, equal keys
+    else { k.mat_blocks = 0; k.valid_blocks = 0; }
+    e->ctxs[id] = std::move(k);
+    e->dirty = true;
+    return KVT_OK;
+  }
+  if (op->op == 0 || op->op >= KVT_OP_PIN) return fail(e, KVT_E_INVAL, "unknown or reserved op");
+  Ctx *c = get_ctx(e, id);
+  if (!c) return fail(e, KVT_E_NOCTX, "unknown context");
+  switch (op->op) {
+    case KVT_OP_APPEND: {
+      if (c->in_flight) return fail(e, KVT_E_STATE, "append: context is in flight");
+      if (op->n_tokens && !op->tokens) return fail(e, KVT_E_INVAL, "append: NULL tokens");
+      u64 need = c->tok_len + op->n_tokens;
+      if (need > c->tok_cap) {
+        u64 ncap = grow_cap(std::max<u64>(need, 2 * c->tok_cap)), noff;
+        if (!e->tok_alloc.alloc(ncap, &noff)) return fail(e, KVT_E_NOSPACE, "token arena full");
+        if (c->tok_len) CU(cudaMemcpyAsync(e->d_tokens + noff, e->d_tokens + c->tok_off, c->tok_len * 4, cudaMemcpyDeviceToDevice, s));
+        if (c->tok_cap) e->tok_alloc.release(c->tok_off, c->tok_cap);
+        c->tok_off = noff; c->tok_cap = ncap;
+      }
+      int32_t r = copy_tokens_in(e, s, c->tok_off + c->tok_len, op->tokens, op->n_tokens, on_dev);
+      if (r) return r;
+      c->tok_len = need;
+      c->msgs.push_back(Msg{op->n_tokens, (u8)(c->one_off ? MS_TEMPORARY : MS_ACTIVE)});
+      e->dirty = true;
+      return KVT_OK;
+    }
+    case KVT_OP_REPLACE:
+    case KVT_OP_REMOVE: {
+      if (c->in_flight) return fail(e, KVT_E_STATE, "edit: context is in flight");
+      if (!(op->msg_start < op->msg_end && op->msg_end <= c->msgs.size())) return fail(e, KVT_E_RANGE, "edit: bad message range");
+      const bool rep = op->op == KVT_OP_REPLACE;
+      if (rep && op->n_tokens && !op->tokens) return fail(e, KVT_E_INVAL, "replace: NULL tokens");
+      u64 t0 = 0, t1 = 0;
+      for (u32 j = 0; j < op->msg_end; ++j) { if (j < op->msg_start) t0 += c->msgs[j].len; t1 += c->msgs[j].len; }
+      const u64 nnew = rep ? op->n_tokens : 0, tail = c->tok_len - t1, new_len = t0 + nnew + tail;
+      if (tail == 0 && t0 + nnew <= c->tok_cap) {  // edit at the end: overwrite in place
+        int32_t r = copy_tokens_in(e, s, c->tok_off + t0, op->tokens, (u32)nnew, on_dev);
+        if (r) return r;
+      } else {                                      // edit in the middle: rebuild the buffer elsewhere
+        u64 ncap = grow_cap(new_len), noff;
+        if (!e->tok_alloc.alloc(ncap, &noff)) return fail(e, KVT_E_NOSPACE, "token arena full");
+        if (t0) CU(cudaMemcpyAsync(e->d_tokens + noff, e->d_tokens + c->tok_off, t0 * 4, cudaMemcpyDeviceToDevice, s));
+        int32_t r = copy_tokens_in(e, s, noff + t0, op->tokens, (u32)nnew, on_dev);
+        if (r) return r;
+        if (tail) CU(cudaMemcpyAsync(e->d_tokens + noff + t0 + nnew, e->d_tokens + c->tok_off + t1, tail * 4, cudaMemcpyDeviceToDevice, s));
+        if (c->tok_cap) e->tok_alloc.release(c->tok_off, c->tok_cap);
+        c->tok_off = noff; c->tok_cap = ncap;
+      }
+      c->tok_len = new_len;
+      // the old versions of message msg_start and of all later messages expire for this context:
+      // it stops mapping everything from the block holding that message's first token (Section 5.1)
+      if (op->msg_start < c->mat_bounds.size()) {
+        c->valid_blocks = std::min<u32>(c->valid_blocks, c->mat_bounds[op->msg_start].first / 16);
+        c->mat_bounds.resize(op->msg_start);
+      }
+      c->msgs.erase(c->msgs.begin() + op->msg_start, c->msgs.begin() + op->msg_end);
+      if (rep) c->msgs.insert(c->msgs.begin() + op->msg_start, Msg{op->n_tokens, (u8)(c->one_off ? MS_TEMPORARY : MS_ACTIVE)});
+      e->dirty = true;
+      return KVT_OK;
+    }
+    case KVT_OP_ONE_OFF: {
+      if (c->in_flight) return fail(e, KVT_E_STATE, "one_off: context is in flight");
+      if (op->msg_start == 0 && op->msg_end == 0xFFFFFFFFu) {
+        c->one_off = true;
+        for (Msg &m : c->msgs) m.state = MS_TEMPORARY;
+      } else {
+        if (!(op->msg_start < op->msg_end && op->msg_end <= c->msgs.size())) return fail(e, KVT_E_RANGE, "one_off: bad message range");
+        for (u32 j = op->msg_start; j < op->msg_end; ++j) c->msgs[j].state = MS_TEMPORARY;
+      }
+      e->dirty = true;
+      return KVT_OK;
+    }
+    case KVT_OP_PREFILL_DONE: {
+      if (!c->in_flight) return fail(e, KVT_E_STATE, "prefill_done: context is not in flight");
+      e->now += 1;
+      int32_t r = unlock_held(e, *c, s, true);
+      if (r) return r;
+      for (Msg &m : c->msgs) if (m.state == MS_ACTIVE) m.state = MS_SUSPENDED;
+      c->in_flight = false;
+      e->dirty = true;
+      return KVT_OK;
+    }
+    case KVT_OP_TERMINATE: {
+      if (c->in_flight) { int32_t r = unlock_held(e, *c, s, false); if (r) return r; }
+      if (c->tok_cap) e->tok_alloc.release(c->tok_off, c->tok_cap);
+      seg_deref(e, c->keyseg);
+      *c = Ctx();
+      e->dirty = true;
+      return KVT_OK;
+    }
+  }
+  return KVT_E_INVAL;
+}
+
+// ---- stages 1 + 2 + admission ---------------------------------------------------------------------------
+static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_info *out, cudaStream_t s) {
+  // plan: blocks, chunks, new key segments (all-or-nothing)
+  u64 total_blocks = 0;
+  for (u32 i = 0; i < n_ctx; ++i) total_blocks += e->ctxs[ids[i]].tok_len / 16;
+  if (total_blocks > e->cfg.max_batch_blocks) return fail(e, KVT_E_NOSPACE, "batch exceeds max_batch_blocks");
+  std::vector<int> newseg(n_ctx, -1);
+  for (u32 i = 0; i < n_ctx; ++i) {
+    u64 nb = e->ctxs[ids[i]].tok_len / 16;
+    if (!nb) continue;
+    newseg[i] = seg_new(e, nb);
+    if (newseg[i] < 0) {
+      for (u32 j = 0; j < i; ++j) seg_deref(e, newseg[j]);
+      return fail(e, KVT_E_NOSPACE, "key arena full");
+    }
+  }
+  int32_t r = stage_acquire(e);
+  if (r) return r;
+  e->now += 1;
+  HashCtx *hd = reinterpret_cast<HashCtx *>(e->h_desc);
+  std::vector<int> dev_idx(n_ctx, -1);
+  u32 nd = 0, chunk_base = 0, blk_base = 0;
+  u32 *h_hit = e->h_ctxres, *h_hbm = e->h_ctxres + e->cfg.max_contexts, *h_host = e->h_ctxres + 2 * e->cfg.max_contexts;
+  for (u32 i = 0; i < n_ctx; ++i) {
+    Ctx &c = e->ctxs[ids[i]];
+    for (Msg &m : c.msgs) if (m.state == MS_SUSPENDED) m.state = MS_ACTIVE;  // reactivation (Section 5.2)
+    c.in_flight = true;
+    c.mat_bounds.clear();
+    u32 pos = 0;
+    for (const Msg &m : c.msgs) { c.mat_bounds.push_back({pos, pos + m.len}); pos += m.len; }
+    seg_deref(e, c.keyseg);
+    c.keyseg = newseg[i];
+    u32 nb = (u32)(c.tok_len / 16);
+    c.mat_blocks = c.valid_blocks = nb;
+    e->max_depth = std::max(e->max_depth, nb);
+    if (nb) {
+      HashCtx d;
+      d.tok_off = c.tok_off; d.key_off = e->segs[c.keyseg].off; d.n_blocks = nb; d.chunk_base = chunk_base; d.blk_base = blk_base; d.pad = 0;
+      h_hit[nd] = nb; h_hbm[nd] = 0; h_host[nd] = 0;
+      dev_idx[i] = (int)nd;
+      hd[nd++] = d;
+      chunk_base += cdiv(nb, CHUNK);
+      blk_base += nb;
+    }
+  }
+  e->dirty = true;
+  if (nd) {
+    u32 *d_res = e->dp<u32>(e->L.ctxres);
+    const u32 C = e->cfg.max_contexts;
+    CU(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nd * sizeof(HashCtx), cudaMemcpyHostToDevice, s));
+    CU(cudaMemcpyAsync(d_res, h_hit, nd * 4, cudaMemcpyHostToDevice, s));
+    CU(cudaMemsetAsync(d_res + C, 0, 2ull * C * 4, s));
+    r = status_zero(e, s);
+    if (r) return r;
+    HashArgs ha;
+    ha.tokens = e->d_tokens; ha.keys = e->d_keys; ha.ctx = e->dp<HashCtx>(e->L.desc); ha.n_ctx = nd;
+    ha.agg = e->dp<u64>(e->L.agg); ha.carry = e->dp<u64>(e->L.carry); ha.h0 = e->h0; ha.single = HashCtx{};
+    LookupArgs la;
+    la.tab = e->tab; la.b_ent = e->dp<u32>(e->L.s0); la.hit_len = d_res; la.status = e->d_status;
+    LockArgs lk;
+    lk.ent = e->ent; lk.b_ent = la.b_ent; lk.hit_len = d_res; lk.n_hbm = d_res + C; lk.n_host = d_res + 2 * C;
+    lk.now = e->now; lk.status = e->d_status;
+    k_hash_digest<<<chunk_base, CHUNK, 0, s>>>(ha);
+    k_hash_carry<<<cdiv(nd, 128), 128, 0, s>>>(ha);
+    k_hash_finish_lookup<<<chunk_base, CHUNK, 0, s>>>(ha, la);
+    k_lock_hits<<<chunk_base, CHUNK, 0, s>>>(ha, lk);
+    LAUNCH_CHECK();
+    CU(cudaMemcpyAsync(h_hit, d_res, 3ull * C * 4, cudaMemcpyDeviceToHost, s));
+    r = status_fetch(e, s);
+    if (r) return r;
+    r = status_code(e);
+    if (r) return r;
+  }
+  for (u32 i = 0; i < n_ctx; ++i) {
+    Ctx &c = e->ctxs[ids[i]];
+    int k = dev_idx[i];
+    c.hit_len = k >= 0 ? h_hit[k] : 0;
+    c.n_hit_hbm = k >= 0 ? h_hbm[k] : 0;
+    c.n_hit_host = k >= 0 ? h_host[k] : 0;
+    c.held = c.hit_len;
+    c.n_admissible = first_temporary_block(c, c.hit_len, c.mat_blocks) - c.hit_len;
+    e->st.blocks_hashed += c.mat_blocks;
+    e->st.hits_hbm += c.n_hit_hbm; e->st.hits_host += c.n_hit_host; e->st.misses += c.mat_blocks - c.hit_len;
+    out[i] = kvt_call_info{c.mat_blocks, c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, 0, c.held};
+  }
+  return KVT_OK;
+}
+
+static int32_t map_admit(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_info *out, cudaStream_t s) {
+  std::vector<u32> held0(n_ctx), cur(n_ctx), lim(n_ctx);
+  std::vector<bool> stopped(n_ctx, false);
+  for (u32 i = 0; i < n_ctx; ++i) {
+    Ctx &c = e->ctxs[ids[i]];
+    held0[i] = cur[i] = c.held;
+    lim[i] = c.hit_len + c.n_admissible;
+    if (cur[i] >= lim[i]) stopped[i] = true;
+  }
+  const u32 C = e->cfg.max_contexts;
+  u32 first = 0;
+  int32_t rc = KVT_OK;
+  while (rc == KVT_OK) {
+    while (first < n_ctx && stopped[first]) ++first;
+    if (first == n_ctx) break;
+    // claims may fill the table: keep live + tombstones + candidates below 3/4 of the capacity
+    u64 cap = (u64)e->tab.mask + 1, used = (u64)e->occ[0] + e->occ[1] + e->tombs;
+    if (used + 1 > cap * 3 / 4 || (e->tombs && used + e->cfg.max_batch_blocks > cap * 3 / 4)) {
+      rc = table_rebuild(e, s);
+      if (rc) break;
+      used = (u64)e->occ[0] + e->occ[1];
+    }
+    u64 budget = std::min<u64>(cap * 3 / 4 - used, e->cfg.max_batch_blocks);
+    rc = stage_acquire(e);
+    if (rc) break;
+    AdmitCtx *hd = reinterpret_cast<AdmitCtx *>(e->h_desc);
+    u32 *h_stop = e->h_ctxres + 3 * C;
+    u32 nd = 0, n_cand = 0;
+    std::vector<u32> who;
+    for (u32 i = first; i < n_ctx && n_cand < budget; ++i) {
+      if (stopped[i]) continue;
+      Ctx &c = e->ctxs[ids[i]];
+      u32 take = (u32)std::min<u64>(lim[i] - cur[i], budget - n_cand);
+      AdmitCtx d;
+      d.key_off = e->segs[c.keyseg].off; d.cand_base = n_cand; d.b_start = cur[i]; d.b_end = cur[i] + take; d.res = nd;
+      h_stop[nd] = d.b_end;
+      hd[nd++] = d;
+      who.push_back(i);
+      n_cand += take;
+      if (take < lim[i] - cur[i]) break;  // the rest of this context goes to the next round
+    }
+    u32 n_free = e->cfg.n_hbm_blocks - e->occ[0];
+    AdmitArgs a;
+    a.tab = e->tab; a.ent = e->ent; a.keys = e->d_keys; a.ctx = e->dp<AdmitCtx>(e->L.desc); a.n_ctx = nd; a.n_cand = n_cand;
+    a.cslot = e->dp<u32>(e->L.s0); a.flag = e->dp<u32>(e->L.s1); a.aux = e->dp<u32>(e->L.s2); a.krank = e->dp<u32>(e->L.s3);
+    a.freelist = e->dp<u32>(e->L.freelist); a.n_free = n_free; a.stop = e->dp<u32>(e->L.ctxres) + 3 * C;
+    a.now = e->now; a.status = e->d_status;
+    CU(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nd * sizeof(AdmitCtx), cudaMemcpyHostToDevice, s));
+    CU(cudaMemcpyAsync(a.stop, h_stop, nd * 4, cudaMemcpyHostToDevice, s));
+    rc = status_zero(e, s);
+    if (rc) break;
+    u32 g = cdiv(n_cand, 256);
+    k_admit_claim<<<g, 256, 0, s>>>(a);
+    k_admit_resolve<<<g, 256, 0, s>>>(a);
+    rc = compact_indices(e, s, PredOwner{a.flag}, EmitRank{a.krank}, n_cand, ST_NEW);
+    if (rc) break;
+    rc = compact_indices(e, s, PredFree{e->ent.key, 0}, EmitFree{e->dp<u32>(e->L.freelist), (u32)e->L.LB}, e->cfg.n_hbm_blocks, ST_FREE);
+    if (rc) break;
+    k_admit_stop<<<g, 256, 0, s>>>(a);
+    k_admit_apply<<<g, 256, 0, s>>>(a);
+    rc = launch_ok(e);
+    if (rc) break;
+    CU(cudaMemcpyAsync(h_stop, a.stop, nd * 4, cudaMemcpyDeviceToHost, s));
+    rc = status_fetch(e, s);
+    if (rc) break;
+    rc = status_code(e);
+    if (rc) break;
+    e->occ[0] += e->h_status[ST_INSERTED];
+    e->tombs += e->h_status[ST_TOMBS];
+    e->st.inserted += e->h_status[ST_INSERTED];
+    e->st.adopted += e->h_status[ST_ADOPTED];
+    for (u32 k = 0; k < nd; ++k) {
+      u32 i = who[k];
+      const AdmitCtx &d = hd[k];
+      cur[i] = h_stop[k];
+      if (h_stop[k] < d.b_end || cur[i] >= lim[i]) stopped[i] = true;
+    }
+    e->dirty = true;
+  }
+  for (u32 i = 0; i < n_ctx; ++i) {
+    Ctx &c = e->ctxs[ids[i]];
+    c.held = cur[i];
+    out[i] = kvt_call_info{c.mat_blocks, c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, cur[i] - held0[i], c.held};
+  }
+  return rc;
+}
+
+int32_t kvt_map_blocks(kvt_engine *e, const uint32_t *ctx_ids, uint32_t n_ctx, uint32_t phase, kvt_call_info *out,
+                       void *stream) {
+  if (!e || !ctx_ids || !out || n_ctx == 0 || phase > 1) return KVT_E_INVAL;
+  for (u32 i = 0; i < n_ctx; ++i)
+    if (!get_ctx(e, ctx_ids[i])) return fail(e, KVT_E_NOCTX, "map_blocks: unknown context");
+  {
+    std::vector<u32> sorted(ctx_ids, ctx_ids + n_ctx);
+    std::sort(sorted.begin(), sorted.end());
+    if (std::adjacent_find(sorted.begin(), sorted.end()) != sorted.end()) return fail(e, KVT_E_INVAL, "map_blocks: duplicate context");
+  }
+  for (u32 i = 0; i < n_ctx; ++i) {
+    bool f = e->ctxs[ctx_ids[i]].in_flight;
+    if (phase == KVT_MAP_LOOKUP && f) return fail(e, KVT_E_STATE, "lookup: context already in flight");
+    if (phase == KVT_MAP_ADMIT && !f) return fail(e, KVT_E_STATE, "admit: context not in flight");
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  return phase == KVT_MAP_LOOKUP ? map_lookup(e, ctx_ids, n_ctx, out, s) : map_admit(e, ctx_ids, n_ctx, out, s);
+}
+
+int32_t kvt_get_block_map(kvt_engine *e, uint32_t ctx, uint64_t *keys, uint8_t *tier, uint32_t *slot, uint32_t cap,
+                          uint32_t *n, void *stream) {
+  if (!e || !n) return KVT_E_INVAL;
+  Ctx *c = get_ctx(e, ctx);
+  if (!c) return fail(e, KVT_E_NOCTX, "get_block_map: unknown context");
+  cudaStream_t s = (cudaStream_t)stream;
+  u32 nb = c->mat_blocks;
+  *n = nb;
+  if (cap < nb) return KVT_E_BUFSZ;
+  if (!nb) return KVT_OK;
+  if (nb > e->cfg.max_batch_blocks) return fail(e, KVT_E_NOSPACE, "context exceeds max_batch_blocks");
+  const u64 *dk = e->d_keys + e->segs[c->keyseg].off;
+  int32_t r = status_zero(e, s);
+  if (r) return r;
+  k_block_map<<<cdiv(nb, 256), 256, 0, s>>>(e->tab, e->ent, dk, nb, e->dp<u8>(e->L.map_tier), e->dp<u32>(e->L.map_slot), e->d_status);
+  LAUNCH_CHECK();
+  if (keys) CU(cudaMemcpyAsync(keys, dk, nb * 8ull, cudaMemcpyDeviceToHost, s));
+  if (tier) CU(cudaMemcpyAsync(tier, e->dp<u8>(e->L.map_tier), nb, cudaMemcpyDeviceToHost, s));
+  if (slot) CU(cudaMemcpyAsync(slot, e->dp<u32>(e->L.map_slot), nb * 4ull, cudaMemcpyDeviceToHost, s));
+  r = status_fetch(e, s);
+  if (r) return r;
+  return status_code(e);
+}
+
+// ---- stage 3 -----------------------------------------------------------------------------------------------
+int32_t kvt_classify(kvt_engine *e, void *stream) {
+  if (!e) return KVT_E_INVAL;
+  return do_classify(e, (cudaStream_t)stream);
+}
+
+int32_t kvt_get_states(kvt_engine *e, uint32_t tier, uint8_t *state, uint32_t cap, void *stream) {
+  if (!e || !state || tier > 1) return KVT_E_INVAL;
+  u32 n = e->tier_slots(tier);
+  if (cap < n) return KVT_E_BUFSZ;
+  if (!n) return KVT_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  int32_t r = ensure_classified(e, s);
+  if (r) return r;
+  u8 *d_out = e->dp<u8>(e->L.out_states);
+  k_states_out<<<cdiv(n, 256), 256, 0, s>>>(e->ent, e->tier_e0(tier), n, d_out);
+  LAUNCH_CHECK();
+  CU(cudaMemcpyAsync(state, d_out, n, cudaMemcpyDeviceToHost, s));
+  CU(cudaStreamSynchronize(s));
+  return KVT_OK;
+}
+
+int32_t kvt_get_entries(kvt_engine *e, uint32_t tier, uint64_t *keys, uint32_t *stamp, uint32_t *depth,
+                        uint32_t *inflight, uint32_t cap, void *stream) {
+  if (!e || tier > 1) return KVT_E_INVAL;
+  u32 n = e->tier_slots(tier), e0 = e->tier_e0(tier);
+  if (cap < n) return KVT_E_BUFSZ;
+  if (!n) return KVT_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (keys) CU(cudaMemcpyAsync(keys, e->ent.key + e0, n * 8ull, cudaMemcpyDeviceToHost, s));
+  if (stamp) CU(cudaMemcpyAsync(stamp, e->ent.stamp + e0, n * 4ull, cudaMemcpyDeviceToHost, s));
+  if (depth) CU(cudaMemcpyAsync(depth, e->ent.depth + e0, n * 4ull, cudaMemcpyDeviceToHost, s));
+  if (inflight) CU(cudaMemcpyAsync(inflight, e->ent.infl + e0, n * 4ull, cudaMemcpyDeviceToHost, s));
+  CU(cudaStreamSynchronize(s));
+  return KVT_OK;
+}
+
+// ---- stage 4 -----------------------------------------------------------------------------------------------
+int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_t *slots_out, uint8_t *states_out,
+                           uint32_t cap, uint32_t *n_out, void *stream) {
+  if (!e || tier > 1 || !n_out || (!slots_out && cap)) return KVT_E_INVAL;
+  *n_out = 0;
+  u32 n = e->tier_slots(tier);
+  if (!n || !n_req) return KVT_OK;
+  cudaStream_t s = (cudaStream_t)stream;
+  int32_t r = ensure_classified(e, s);
+  if (r) return r;
+  r = status_zero(e, s);
+  if (r) return r;
+  SelArgs a;
+  a.ent = e->ent; a.e0 = e->tier_e0(tier); a.n_slots = n; a.n_req = n_req; a.now = e->now;
+  a.stamp_bits = bit_length(e->now); a.depth_bits = bit_length(e->max_depth);
+  a.mru = e->cfg.suspended_order == KVT_ORDER_MRU; a.status = e->d_status;
+  u64 *kA = e->dp<u64>(e->L.keyA), *kB = e->dp<u64>(e->L.keyB);
+  u32 *vA = e->dp<u32>(e->L.valA), *vB = e->dp<u32>(e->L.valB), *counts = e->dp<u32>(e->L.rcounts);
+  k_sel_count<<<cdiv(n, 256), 256, 0, s>>>(a);
+  r = compact_indices(e, s, PredSel{a}, EmitSel{a, kA, vA}, n, ST_M);
+  if (r) return r;
+  const u32 key_bits = 2 + a.stamp_bits + a.depth_bits, n_pass = cdiv(key_bits, 8), tiles = cdiv(n, SORT_TILE);
+  for (u32 p = 0; p < n_pass; ++p) {
+    k_radix_hist<<<tiles, 256, 0, s>>>(kA, e->d_status, 8 * p, counts);
+    k_radix_scan<<<1, 1024, 0, s>>>(counts, e->d_status);
+    k_radix_scatter<<<tiles, 256, 0, s>>>(kA, vA, kB, vB, e->d_status, 8 * p, counts);
+    std::swap(kA, kB); std::swap(vA, vB);
+  }
+  u32 n_emit = std::min(n_req, n);
+  k_sel_emit<<<cdiv(n_emit, 256), 256, 0, s>>>(kA, vA, n_emit, a.stamp_bits + a.depth_bits, e->dp<u32>(e->L.out_slots),
+                                               e->dp<u8>(e->L.out_states));
+  LAUNCH_CHECK();
+  r = status_fetch(e, s);
+  if (r) return r;
+  r = status_code(e);
+  if (r) return r;
+  u64 total = (u64)e->h_status[ST_RANK0] + e->h_status[ST_RANK1] + e->h_status[ST_RANK2];
+  u32 k = (u32)std::min<u64>(n_req, total);
+  *n_out = k;
+  if (cap < k) return KVT_E_BUFSZ;
+  if (k) {
+    CU(cudaMemcpyAsync(slots_out, e->dp<u32>(e->L.out_slots), k * 4ull, cudaMemcpyDeviceToHost, s));
+    if (states_out) CU(cudaMemcpyAsync(states_out, e->dp<u8>(e->L.out_states), k, cudaMemcpyDeviceToHost, s));
+    CU(cudaStreamSynchronize(s));
+  }
+  return KVT_OK;
+}
+
+// ---- stage 5 -----------------------------------------------------------------------------------------------
+// Shared body of offload / reload / release.
+static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier, const u32 *slots, u32 n,
+                       bool allow_inflight, bool drop_dead, bool drop_all, u32 *n_done, u32 *n_live, u32 *n_drop) {
+  *n_done = *n_live = *n_drop = 0;
+  if (n == 0) return KVT_OK;
+  if (n > e->L.LB) return fail(e, KVT_E_NOSPACE, "list longer than max_batch_blocks");
+  int32_t r = stage_acquire(e);
+  if (r) return r;
+  if (drop_dead) { r = ensure_classified(e, s); if (r) return r; r = stage_acquire(e); if (r) return r; }
+  std::memcpy(e->h_ids, slots, n * 4ull);
+  u32 *d_ids = e->dp<u32>(e->L.ids);
+  CU(cudaMemcpyAsync(d_ids, e->h_ids, n * 4ull, cudaMemcpyHostToDevice, s));
+  r = stage_release(e, s);
+  if (r) return r;
+  r = status_zero(e, s);
+  if (r) return r;
+  CU(cudaMemcpyAsync(e->d_status + ST_CUT, &n, 4, cudaMemcpyHostToDevice, s));  // pageable source: staged before return
+  ListArgs a;
+  a.tab = e->tab; a.ent = e->ent; a.ids = d_ids; a.n = n; a.e0 = e->tier_e0(src_tier); a.n_slots = e->tier_slots(src_tier);
+  a.dst_e0 = e->tier_e0(dst_tier);
+  a.live = e->dp<u32>(e->L.s1); a.lidx = e->dp<u32>(e->L.s2);
+  a.freelist = e->dp<u32>(e->L.freelist); a.n_free = e->tier_slots(dst_tier) - e->occ[dst_tier];
+  a.pair_src = e->dp<u32>(e->L.pair_src); a.pair_dst = e->dp<u32>(e->L.pair_dst);
+  a.allow_inflight = allow_inflight; a.drop_dead = drop_dead; a.drop_all = drop_all; a.status = e->d_status;
+  u32 g = cdiv(n, 256);
+  k_list_validate<<<g, 256, 0, s>>>(a);
+  r = compact_indices(e, s, PredLive{a.live}, EmitLive{a.lidx, a.n_free, e->d_status}, n, ST_TOTAL);
+  if (r) return r;
+  if (!drop_all) {
+    r = compact_indices(e, s, PredFree{e->ent.key, a.dst_e0}, EmitFree{e->dp<u32>(e->L.freelist), (u32)e->L.LB},
+                        e->tier_slots(dst_tier), ST_FREE);
+    if (r) return r;
+  }
+  k_list_apply<<<g, 256, 0, s>>>(a);
+  k_list_unmark<<<g, 256, 0, s>>>(a);
+  LAUNCH_CHECK();
+  if (!drop_all) {
+    r = launch_mover(e, s, src_tier, a.pair_src, dst_tier, a.pair_dst, std::min(n, a.n_free), e->d_status + ST_NLIVE);
+    if (r) return r;
+  }
+  r = status_fetch(e, s);
+  if (r) return r;
+  r = status_code(e);
+  if (r) return r;
+  *n_live = e->h_status[ST_NLIVE];
+  *n_drop = e->h_status[ST_NDROP];
+  *n_done = *n_live + *n_drop;
+  e->occ[src_tier] -= *n_done;
+  if (!drop_all) e->occ[dst_tier] += *n_live;
+  e->tombs += *n_drop;
+  e->st.dropped += *n_drop;
+  r = maybe_rebuild(e, s);
+  if (r) return r;
+  return *n_done < n ? KVT_E_NOSPACE : KVT_OK;
+}
+
+int32_t kvt_offload(kvt_engine *e, const uint32_t *hbm_slots, uint32_t n, uint32_t *n_done, uint32_t *n_dropped, void *stream) {
+  if (!e || (!hbm_slots && n) || !n_done || !n_dropped) return KVT_E_INVAL;
+  u32 live = 0;
+  int32_t r = list_op(e, (cudaStream_t)stream, KVT_TIER_HBM, KVT_TIER_HOST, hbm_slots, n, false, true, false, n_done, &live, n_dropped);
+  e->st.offloaded += live;
+  e->st.bytes_d2h += live * e->block_bytes;
+  if (r == KVT_E_NOSPACE) e->err = "host tier full";
+  return r;
+}
+
+int32_t kvt_reload(kvt_engine *e, const uint32_t *host_slots, uint32_t n, uint32_t *n_done, void *stream) {
+  if (!e || (!host_slots && n) || !n_done) return KVT_E_INVAL;
+  u32 live = 0, drop = 0;
+  int32_t r = list_op(e, (cudaStream_t)stream, KVT_TIER_HOST, KVT_TIER_HBM, host_slots, n, true, false, false, n_done, &live, &drop);
+  e->st.reloaded += live;
+  e->st.bytes_h2d += live * e->block_bytes;
+  if (r == KVT_E_NOSPACE) e->err = "HBM tier full";
+  return r;
+}
+
+int32_t kvt_release(kvt_engine *e, uint32_t tier, const uint32_t *slots, uint32_t n, void *stream) {
+  if (!e || tier > 1 || (!slots && n)) return KVT_E_INVAL;
+  u32 done = 0, live = 0, drop = 0;
+  return list_op(e, (cudaStream_t)stream, tier, tier, slots, n, false, false, true, &done, &live, &drop);
+}
+
+int32_t kvt_compact(kvt_engine *e, uint32_t tier, uint32_t *n_moved, void *stream) {
+  if (!e || tier > 1 || !n_moved) return KVT_E_INVAL;
+  *n_moved = 0;
+  cudaStream_t s = (cudaStream_t)stream;
+  u32 n = e->tier_slots(tier), e0 = e->tier_e0(tier), n_occ = e->occ[tier];
+  if (!n || !n_occ || n_occ == n) return KVT_OK;
+  int32_t r = status_zero(e, s);
+  if (r) return r;
+  u32 *src = e->dp<u32>(e->L.pair_src), *dst = e->dp<u32>(e->L.pair_dst);
+  r = compact_indices(e, s, PredHole{e->ent.key, e0, n_occ}, EmitList{dst}, n, ST_AUX);
+  if (r) return r;
+  r = compact_indices(e, s, PredMover{e->ent.key, e0, n_occ}, EmitList{src}, n, ST_NMOVED);
+  if (r) return r;
+  u32 n_max = std::min(n_occ, n - n_occ);
+  k_compact_apply<<<cdiv(n_max, 256), 256, 0, s>>>(e->tab, e->ent, e0, src, dst, e->d_status);
+  LAUNCH_CHECK();
+  r = launch_mover(e, s, tier, src, tier, dst, n_max, e->d_status + ST_NMOVED);
+  if (r) return r;
+  r = status_fetch(e, s);
+  if (r) return r;
+  r = status_code(e);
+  if (r) return r;
+  if (e->h_status[ST_AUX] != e->h_status[ST_NMOVED]) return fail(e, KVT_E_DEVICE, "compaction plan mismatch");
+  *n_moved = e->h_status[ST_NMOVED];
+  e->st.compacted += *n_moved;
+  e->st.bytes_d2d += *n_moved * e->block_bytes;
+  return KVT_OK;
+}
+
+int32_t kvt_copy_blocks(kvt_engine *e, uint32_t src_tier, const uint32_t *src, uint32_t dst_tier, const uint32_t *dst,
+                        uint32_t n, uint32_t flags, void *stream) {
+  if (!e || src_tier > 1 || dst_tier > 1 || ((!src || !dst) && n)) return KVT_E_INVAL;
+  if (e->metadata_only) return fail(e, KVT_E_INVAL, "copy_blocks on a metadata-only engine");
+  if (n == 0) return KVT_OK;
+  if (n > e->L.LB) return fail(e, KVT_E_NOSPACE, "list longer than max_batch_blocks");
+  cudaStream_t s = (cudaStream_t)stream;
+  const u32 *ds = src, *dd = dst;
+  if (!(flags & KVT_IDS_ON_DEVICE)) {
+    int32_t r = stage_acquire(e);
+    if (r) return r;
+    std::memcpy(e->h_ids, src, n * 4ull);
+    std::memcpy(e->h_ids2, dst, n * 4ull);
+    CU(cudaMemcpyAsync(e->dp<u32>(e->L.ids), e->h_ids, n * 4ull, cudaMemcpyHostToDevice, s));
+    CU(cudaMemcpyAsync(e->dp<u32>(e->L.ids2), e->h_ids2, n * 4ull, cudaMemcpyHostToDevice, s));
+    r = stage_release(e, s);
+    if (r) return r;
+    ds = e->dp<u32>(e->L.ids); dd = e->dp<u32>(e->L.ids2);
+  }
+  return launch_mover(e, s, src_tier, ds, dst_tier, dd, n, nullptr);
+}
+
+// ---- stand-alone hasher -----------------------------------------------------------------------------------
+uint64_t kvt_hash_scratch_bytes(uint64_t n_tokens) {
+  u64 n_chunks = (n_tokens / 16 + CHUNK - 1) / CHUNK;
+  return std::max<u64>(n_chunks, 1) * 16;
+}
+
+int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t hash_seed, uint64_t *d_keys, void *d_scratch,
+                        uint64_t scratch_bytes, void *stream) {
+  u64 nb = n_tokens / 16;
+  if (nb == 0) return KVT_OK;
+  if (!d_tokens || !d_keys || !d_scratch || ((uintptr_t)d_tokens & 15) || ((uintptr_t)d_scratch & 7)) return KVT_E_INVAL;
+  if (nb >= 0xFFFFFFFFull || scratch_bytes < kvt_hash_scratch_bytes(n_tokens)) return KVT_E_INVAL;
+  cudaStream_t s = (cudaStream_t)stream;
+  u32 n_chunks = cdiv(nb, CHUNK);
+  HashArgs ha;
+  ha.tokens = d_tokens; ha.keys = d_keys; ha.ctx = nullptr; ha.n_ctx = 1;
+  ha.single = HashCtx{0, 0, (u32)nb, 0, 0, 0};
+  ha.agg = (u64 *)d_scratch; ha.carry = (u64 *)d_scratch + n_chunks; ha.h0 = hash_h0(hash_seed);
+  LookupArgs la{};
+  k_hash_digest<<<n_chunks, CHUNK, 0, s>>>(ha);
+  k_hash_carry<<<1, 32, 0, s>>>(ha);
+  k_hash_finish_lookup<<<n_chunks, CHUNK, 0, s>>>(ha, la);
+  return cudaGetLastError() == cudaSuccess ? KVT_OK : KVT_E_CUDA;
+}
+
+// ---- debug loader -------------------------------------------------------------------------------------------
+int32_t kvt_debug_load_resident(kvt_engine *e, const uint64_t *keys, const uint8_t *state, const uint32_t *stamp,
+                                const uint32_t *depth, const uint32_t *slot, uint32_t tier, uint32_t n, void *stream) {
+  if (!e || tier > 1 || ((!keys || !state || !stamp || !depth || !slot) && n)) return KVT_E_INVAL;
+  if (n == 0) return KVT_OK;
+  u32 ns = e->tier_slots(tier);
+  if (n > ns || n > e->L.LB) return fail(e, KVT_E_INVAL, "more blocks than slots");
+  u32 max_stamp = 0, max_d = 0;
+  {
+    std::vector<u64> ks(keys, keys + n);
+    std::vector<u32> ss(slot, slot + n);
+    std::sort(ks.begin(), ks.end());
+    std::sort(ss.begin(), ss.end());
+    if (ks[0] < 2 || std::adjacent_find(ks.begin(), ks.end()) != ks.end() ||
+        std::adjacent_find(ss.begin(), ss.end()) != ss.end() || ss.back() >= ns)
+      return fail(e, KVT_E_INVAL, "bad keys or slots");
+    for (u32 i = 0; i < n; ++i) {
+      if (state[i] > 2) return fail(e, KVT_E_INVAL, "bad state");
+      max_stamp = std::max(max_stamp, stamp[i]); max_d = std::max(max_d, depth[i]);
+    }
+  }
+  if ((u64)e->occ[0] + e->occ[1] + e->tombs + n > ((u64)e->tab.mask + 1) * 3 / 4) return fail(e, KVT_E_NOSPACE, "table too full");
+  cudaStream_t s = (cudaStream_t)stream;
+  // stage the arrays in scratch: keys -> keyA, state -> out_states, stamp/depth/slot -> s1/s2/s3
+  u64 *dk = e->dp<u64>(e->L.keyA);
+  u8 *dst_state = e->dp<u8>(e->L.out_states);
+  u32 *dsp = e->dp<u32>(e->L.s1), *ddp = e->dp<u32>(e->L.s2), *dsl = e->dp<u32>(e->L.s3);
+  CU(cudaMemcpyAsync(dk, keys, n * 8ull, cudaMemcpyHostToDevice, s));
+  CU(cudaMemcpyAsync(dst_state, state, n, cudaMemcpyHostToDevice, s));
+  CU(cudaMemcpyAsync(dsp, stamp, n * 4ull, cudaMemcpyHostToDevice, s));
+  CU(cudaMemcpyAsync(ddp, depth, n * 4ull, cudaMemcpyHostToDevice, s));
+  CU(cudaMemcpyAsync(dsl, slot, n * 4ull, cudaMemcpyHostToDevice, s));
+  int32_t r = status_zero(e, s);
+  if (r) return r;
+  LoadArgs a;
+  a.tab = e->tab; a.ent = e->ent; a.keys = dk; a.state = dst_state; a.stamp = dsp; a.depth = ddp; a.slot = dsl;
+  a.n = n; a.e0 = e->tier_e0(tier); a.n_slots = ns; a.status = e->d_status;
+  k_load_check<<<cdiv(n, 256), 256, 0, s>>>(a);
+  k_load_apply<<<cdiv(n, 256), 256, 0, s>>>(a);
+  LAUNCH_CHECK();
+  r = status_fetch(e, s);
+  if (r) return r;
+  r = status_code(e);
+  if (r) return r;
+  e->occ[tier] += n;
+  e->now = std::max(e->now, max_stamp);
+  e->max_depth = std::max(e->max_depth, max_d);
+  return KVT_OK;
+}
+
+}  // extern "C"

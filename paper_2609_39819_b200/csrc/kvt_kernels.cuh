@@ -1,0 +1,809 @@
+// kvt_kernels.cuh — sm_100a kernels of the KV-cache hot path: block hasher, open-addressing block
+// table, lifecycle classifier, victim selection (ordered compaction + LSD radix sort) and paged KV
+// mover. Host-side launch logic lives in kvt_engine.cu.
+//
+// Conventions: every probe loop is capped at the table capacity and reports through the status
+// word (never traps, never spins on another thread's progress); there are no inter-CTA waits, so
+// every multi-pass algorithm is a sequence of kernels. No tensor cores: nothing here is a dense
+// contraction.
+#pragma once
+#include <cstdint>
+#include <cuda_runtime.h>
+
+namespace kvt {
+
+typedef uint8_t u8;
+typedef uint32_t u32;
+typedef uint64_t u64;
+
+constexpr u64 KEY_EMPTY = 0, KEY_TOMB = 1;
+constexpr u32 ENT_NONE = 0xFFFFFFFFu;
+constexpr u32 CLAIM_BIT = 0x80000000u;
+constexpr u32 CHUNK = 256;        // blocks hashed by one CTA
+constexpr u32 SCAN_TILE = 1024;   // items per CTA in the ordered-compaction kernels
+constexpr u32 SORT_TILE = 4096;   // items per CTA in the radix-sort kernels (8 warps x 512)
+
+// bits of the device error word
+enum : u32 { DERR_PROBE = 1, DERR_RANGE = 2, DERR_INVAL = 4, DERR_STATE = 8, DERR_CORRUPT = 16 };
+
+// words of the device status block
+enum : int {
+  ST_ERR = 0, ST_TOTAL, ST_CUT, ST_NLIVE, ST_NDROP, ST_NEW, ST_INSERTED, ST_ADOPTED, ST_TOMBS,
+  ST_RANK0, ST_RANK1, ST_RANK2, ST_M, ST_NMOVED, ST_FREE, ST_AUX, ST_WORDS = 32
+};
+
+struct __align__(16) TSlot { u64 key; u32 ent; u32 pad; };
+
+// ---- hash constants (compile-time; only H0 depends on the seed) -------------------------------------
+__host__ __device__ constexpr u64 mix64(u64 z) {
+  z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull;
+  z ^= z >> 27; z *= 0x94D049BB133111EBull;
+  z ^= z >> 31;
+  return z;
+}
+constexpr u64 GOLD = 0x9E3779B97F4A7C15ull;
+constexpr u64 HASH_P = mix64(GOLD * 17ull) | 1ull;
+__host__ __device__ constexpr u64 lane_mult(u32 t) { return mix64(GOLD * (u64)(t + 1)) | 1ull; }
+__host__ __device__ constexpr u64 hash_h0(u64 seed) { return mix64(seed ^ (GOLD * 18ull)); }
+
+__host__ __device__ __forceinline__ u64 pow_p(u32 e) {
+  u64 r = 1, b = HASH_P;
+  while (e) { if (e & 1) r *= b; b *= b; e >>= 1; }
+  return r;
+}
+
+// ---- device views -------------------------------------------------------------------------------------
+struct Table { TSlot *slots; u32 mask; u32 shift; };   // capacity = mask + 1, home = key >> shift
+
+struct Entries {            // per resident-block metadata, entry id = slot (HBM) or n_hbm + slot (host)
+  u64 *key;                 // 0 = free
+  u32 *stamp, *depth, *infl, *rank, *tslot, *mark;
+  u8 *floor;
+  u32 n_hbm, n_total;
+};
+
+__device__ __forceinline__ void set_err(u32 *status, u32 bits) { atomicOr(&status[ST_ERR], bits); }
+
+// Finds key; returns its table slot index or ENT_NONE. Stops at the first EMPTY slot.
+__device__ __forceinline__ u32 tab_find(const Table &t, u64 key, u32 *status) {
+  u32 i = (u32)(key >> t.shift);
+  for (u32 n = 0; n <= t.mask; ++n, i = (i + 1) & t.mask) {
+    u64 k = t.slots[i].key;
+    if (k == key) return i;
+    if (k == KEY_EMPTY) return ENT_NONE;
+  }
+  set_err(status, DERR_PROBE);
+  return ENT_NONE;
+}
+
+// Finds key or claims the first EMPTY slot of its probe sequence for it (tombstones are skipped,
+// never reused, so two threads inserting the same key always meet in the same slot).
+__device__ __forceinline__ u32 tab_find_or_claim(const Table &t, u64 key, u32 *status) {
+  u32 i = (u32)(key >> t.shift);
+  for (u32 n = 0; n <= t.mask;) {
+    u64 k = *(volatile u64 *)&t.slots[i].key;
+    if (k == key) return i;
+    if (k == KEY_EMPTY) {
+      u64 old = atomicCAS((unsigned long long *)&t.slots[i].key, (unsigned long long)KEY_EMPTY,
+                          (unsigned long long)key);
+      if (old == KEY_EMPTY || old == key) return i;
+      // somebody else took the slot for another key: move on
+    }
+    ++n; i = (i + 1) & t.mask;
+  }
+  set_err(status, DERR_PROBE);
+  return ENT_NONE;
+}
+
+// ======================================================================================================
+// K1: block hasher. 3 phases, no inter-CTA waits:
+//   digest : per 256-block chunk, 4 lanes per block read 16 B each, weighted sums, mix, then a CTA-wide
+//            scan of the affine chain with zero carry-in -> partial chain values + chunk aggregate
+//   carry  : one thread per context walks its chunk aggregates (<= 63 steps for a 258K-token call)
+//   finish : h = P^(i+1) * carry + partial, key = mix64(h); fused with the table probe
+// ======================================================================================================
+struct HashCtx { u64 tok_off; u64 key_off; u32 n_blocks; u32 chunk_base; u32 blk_base; u32 pad; };
+
+struct HashArgs {
+  const u32 *tokens; u64 *keys; const HashCtx *ctx; HashCtx single; u32 n_ctx;
+  u64 *agg; u64 *carry; u64 h0;
+};
+
+__device__ __forceinline__ const HashCtx &hash_ctx_of_chunk(const HashArgs &a, u32 chunk, u32 *ctx_idx) {
+  if (!a.ctx) { *ctx_idx = 0; return a.single; }
+  u32 lo = 0, hi = a.n_ctx;  // last i with chunk_base <= chunk
+  while (hi - lo > 1) { u32 mid = (lo + hi) >> 1; if (a.ctx[mid].chunk_base <= chunk) lo = mid; else hi = mid; }
+  *ctx_idx = lo;
+  return a.ctx[lo];
+}
+
+__global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
+  __shared__ u64 sd[CHUNK];
+  __shared__ u64 wagg[CHUNK / 32];
+  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  u32 ci;
+  const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci);
+  const u32 b0 = (blockIdx.x - c.chunk_base) * CHUNK;
+  const u32 nb = min(CHUNK, c.n_blocks - b0);
+  const uint4 *tok = reinterpret_cast<const uint4 *>(a.tokens + c.tok_off + (u64)b0 * 16);
+  const u32 q = tid & 3;
+  const u64 k0 = lane_mult(4 * q), k1 = lane_mult(4 * q + 1), k2 = lane_mult(4 * q + 2), k3 = lane_mult(4 * q + 3);
+  uint4 v[4];
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    u32 idx = it * CHUNK + tid;
+    v[it] = (idx >> 2) < nb ? __ldg(tok + idx) : make_uint4(0, 0, 0, 0);
+  }
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    u32 blk = (it * CHUNK + tid) >> 2;
+    u64 s = ((u64)v[it].x + 1) * k0 + ((u64)v[it].y + 1) * k1 + ((u64)v[it].z + 1) * k2 + ((u64)v[it].w + 1) * k3;
+    s += __shfl_xor_sync(0xFFFFFFFFu, s, 1);
+    s += __shfl_xor_sync(0xFFFFFFFFu, s, 2);
+    if (q == 0) sd[blk] = blk < nb ? mix64(s) : 0;
+  }
+  __syncthreads();
+  // inclusive scan of c_t = sum_{i<=t} P^(t-i) d_i
+  u64 cval = sd[tid];
+  u64 pp = HASH_P;
+#pragma unroll
+  for (u32 o = 1; o < 32; o <<= 1) {
+    u64 up = __shfl_up_sync(0xFFFFFFFFu, cval, o);
+    if (lane >= o) cval += pp * up;
+    pp *= pp;
+  }
+  if (lane == 31) wagg[warp] = cval;
+  __syncthreads();
+  u64 carry = 0;  // chain value at the end of the previous warp, with zero chunk carry-in
+  const u64 p32 = pp;  // after 5 squarings pp = P^32
+  for (u32 w = 0; w < warp; ++w) carry = p32 * carry + wagg[w];
+  cval += pow_p(lane + 1) * carry;
+  if (tid < nb) a.keys[c.key_off + b0 + tid] = cval;
+  if (tid == nb - 1) a.agg[blockIdx.x] = cval;
+}
+
+__global__ void k_hash_carry(HashArgs a) {
+  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= a.n_ctx) return;
+  const HashCtx c = a.ctx ? a.ctx[i] : a.single;
+  u64 carry = a.h0;
+  const u64 pfull = pow_p(CHUNK);
+  u32 n_chunks = (c.n_blocks + CHUNK - 1) / CHUNK;
+  for (u32 j = 0; j < n_chunks; ++j) {
+    a.carry[c.chunk_base + j] = carry;
+    u32 len = min(CHUNK, c.n_blocks - j * CHUNK);
+    carry = (len == CHUNK ? pfull : pow_p(len)) * carry + a.agg[c.chunk_base + j];
+  }
+}
+
+struct LookupArgs {
+  Table tab;            // slots == nullptr: hash only
+  u32 *b_ent;           // per batch block: entry id or ENT_NONE
+  u32 *hit_len;         // per context, pre-initialised to n_blocks
+  u32 *status;
+};
+
+__global__ void __launch_bounds__(CHUNK) k_hash_finish_lookup(HashArgs a, LookupArgs l) {
+  __shared__ u32 s_min;
+  const u32 tid = threadIdx.x;
+  u32 ci;
+  const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci);
+  const u32 b0 = (blockIdx.x - c.chunk_base) * CHUNK;
+  const u32 nb = min(CHUNK, c.n_blocks - b0);
+  if (tid == 0) s_min = 0xFFFFFFFFu;
+  __syncthreads();
+  if (tid < nb) {
+    u64 h = pow_p(tid + 1) * a.carry[blockIdx.x] + a.keys[c.key_off + b0 + tid];
+    u64 key = mix64(h);
+    if (key < 2) key += 2;
+    a.keys[c.key_off + b0 + tid] = key;
+    if (l.tab.slots) {
+      u32 s = tab_find(l.tab, key, l.status);
+      u32 ent = s == ENT_NONE ? ENT_NONE : l.tab.slots[s].ent;
+      l.b_ent[c.blk_base + b0 + tid] = ent;
+      if (ent == ENT_NONE) atomicMin(&s_min, b0 + tid);
+    }
+  }
+  __syncthreads();
+  if (l.tab.slots && tid == 0 && s_min != 0xFFFFFFFFu) atomicMin(&l.hit_len[ci], s_min);
+}
+
+// Stamps and locks the reusable prefix of every context of the batch; counts hits per tier.
+struct LockArgs { Entries ent; const u32 *b_ent; const u32 *hit_len; u32 *n_hbm; u32 *n_host; u32 now; u32 *status; };
+
+__global__ void __launch_bounds__(CHUNK) k_lock_hits(HashArgs a, LockArgs l) {
+  __shared__ u32 s_hbm, s_host;
+  const u32 tid = threadIdx.x;
+  u32 ci;
+  const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci);
+  const u32 b = (blockIdx.x - c.chunk_base) * CHUNK + tid;
+  if (tid == 0) { s_hbm = 0; s_host = 0; }
+  __syncthreads();
+  if (b < l.hit_len[ci]) {
+    u32 e = l.b_ent[c.blk_base + b];
+    if (e >= l.ent.n_total) set_err(l.status, DERR_CORRUPT);
+    else {
+      l.ent.stamp[e] = l.now;
+      atomicAdd(&l.ent.infl[e], 1u);
+      atomicAdd(e < l.ent.n_hbm ? &s_hbm : &s_host, 1u);
+    }
+  }
+  __syncthreads();
+  if (tid == 0) {
+    if (s_hbm) atomicAdd(&l.n_hbm[ci], s_hbm);
+    if (s_host) atomicAdd(&l.n_host[ci], s_host);
+  }
+}
+
+// ======================================================================================================
+// Generic ordered compaction: pred(i) for i < n -> exclusive rank among flagged items (ascending i),
+// emit(i, rank) for flagged items. Three kernels: tile counts, single-CTA scan, scatter.
+// ======================================================================================================
+template <class Pred>
+__global__ void __launch_bounds__(SCAN_TILE) k_tile_count(Pred pred, u32 n, u32 *tile_sums) {
+  __shared__ u32 s;
+  if (threadIdx.x == 0) s = 0;
+  __syncthreads();
+  u32 i = blockIdx.x * SCAN_TILE + threadIdx.x;
+  bool f = i < n && pred(i);
+  u32 m = __ballot_sync(0xFFFFFFFFu, f);
+  if ((threadIdx.x & 31) == 0 && m) atomicAdd(&s, __popc(m));
+  __syncthreads();
+  if (threadIdx.x == 0) tile_sums[blockIdx.x] = s;
+}
+
+// In-place exclusive scan of tile_sums[0..n_tiles) by one CTA; total -> *total.
+__global__ void __launch_bounds__(1024) k_scan_tiles(u32 *tile_sums, u32 n_tiles, u32 *total) {
+  __shared__ u32 warp_sums[32];
+  __shared__ u32 s_base;
+  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_base = 0;
+  __syncthreads();
+  for (u32 start = 0; start < n_tiles; start += 1024) {
+    u32 i = start + tid;
+    u32 v = i < n_tiles ? tile_sums[i] : 0;
+    u32 x = v;
+#pragma unroll
+    for (u32 o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(0xFFFFFFFFu, x, o); if (lane >= o) x += y; }
+    if (lane == 31) warp_sums[warp] = x;
+    __syncthreads();
+    if (warp == 0) {
+      u32 w = warp_sums[lane], z = w;
+#pragma unroll
+      for (u32 o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(0xFFFFFFFFu, z, o); if (lane >= o) z += y; }
+      warp_sums[lane] = z - w;  // exclusive
+    }
+    __syncthreads();
+    u32 base = s_base;
+    u32 incl = base + warp_sums[warp] + x;
+    if (i < n_tiles) tile_sums[i] = incl - v;
+    __syncthreads();
+    if (tid == 1023) s_base = incl;
+    __syncthreads();
+  }
+  if (tid == 0) *total = s_base;
+}
+
+template <class Pred, class Emit>
+__global__ void __launch_bounds__(SCAN_TILE) k_tile_scatter(Pred pred, Emit emit, u32 n, const u32 *tile_offs) {
+  __shared__ u32 warp_sums[32];
+  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  u32 i = blockIdx.x * SCAN_TILE + tid;
+  bool f = i < n && pred(i);
+  u32 m = __ballot_sync(0xFFFFFFFFu, f);
+  if (lane == 0) warp_sums[warp] = __popc(m);
+  __syncthreads();
+  if (warp == 0) {
+    u32 w = warp_sums[lane], z = w;
+#pragma unroll
+    for (u32 o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(0xFFFFFFFFu, z, o); if (lane >= o) z += y; }
+    warp_sums[lane] = z - w;
+  }
+  __syncthreads();
+  if (f) emit(i, tile_offs[blockIdx.x] + warp_sums[warp] + __popc(m & ((1u << lane) - 1)));
+}
+
+// ======================================================================================================
+// K2: block table maintenance
+// ======================================================================================================
+__global__ void k_table_clear(Table t) {
+  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i <= t.mask) { TSlot s; s.key = KEY_EMPTY; s.ent = ENT_NONE; s.pad = 0; t.slots[i] = s; }
+}
+
+// Re-inserts every resident entry (used after clearing, to drop tombstones).
+__global__ void k_table_reinsert(Table t, Entries en, u32 *status) {
+  u32 e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e >= en.n_total) return;
+  u64 key = en.key[e];
+  if (!key) return;
+  u32 s = tab_find_or_claim(t, key, status);
+  if (s == ENT_NONE) return;
+  t.slots[s].ent = e;
+  en.tslot[e] = s;
+}
+
+// ---- admission (Algorithm 1's "admit iff a slot is free", batched and deterministic) -----------------
+struct AdmitCtx { u64 key_off; u32 cand_base; u32 b_start; u32 b_end; u32 res; };  // res: index of the context's result words
+
+struct AdmitArgs {
+  Table tab; Entries ent; const u64 *keys; const AdmitCtx *ctx; u32 n_ctx; u32 n_cand;
+  u32 *cslot, *flag, *aux, *krank;   // per candidate scratch
+  const u32 *freelist; u32 n_free;   // lowest free HBM slots, ascending; n_free = free HBM slots
+  u32 *stop;                          // per context (indexed by AdmitCtx.res)
+  u32 now; u32 *status;
+};
+enum : u32 { CAND_OLD = 1, CAND_OWNER = 2, CAND_DUP = 3 };
+
+__device__ __forceinline__ u32 admit_ctx_of(const AdmitArgs &a, u32 g) {
+  u32 lo = 0, hi = a.n_ctx;
+  while (hi - lo > 1) { u32 mid = (lo + hi) >> 1; if (a.ctx[mid].cand_base <= g) lo = mid; else hi = mid; }
+  return lo;
+}
+
+// A1: every candidate finds its key or claims a slot; the lowest candidate index wins ownership.
+__global__ void k_admit_claim(AdmitArgs a) {
+  u32 g = blockIdx.x * blockDim.x + threadIdx.x;
+  if (g >= a.n_cand) return;
+  const AdmitCtx c = a.ctx[admit_ctx_of(a, g)];
+  u64 key = a.keys[c.key_off + c.b_start + (g - c.cand_base)];
+  u32 s = tab_find_or_claim(a.tab, key, a.status);
+  a.cslot[g] = s;
+  if (s != ENT_NONE) atomicMin(&a.tab.slots[s].ent, CLAIM_BIT | g);  // resident ids are < CLAIM_BIT: unchanged
+}
+
+// A2: classify candidates: already resident / owner of a new key / duplicate of an earlier candidate.
+__global__ void k_admit_resolve(AdmitArgs a) {
+  u32 g = blockIdx.x * blockDim.x + threadIdx.x;
+  if (g >= a.n_cand) return;
+  u32 s = a.cslot[g];
+  u32 f = 0, x = 0;
+  if (s != ENT_NONE) {
+    u32 v = a.tab.slots[s].ent;
+    if (v < CLAIM_BIT) { f = CAND_OLD; x = v; if (v >= a.ent.n_total) { set_err(a.status, DERR_CORRUPT); f = 0; } }
+    else {
+      x = v & ~CLAIM_BIT;
+      if (x == g) f = CAND_OWNER;
+      else if (x < g) f = CAND_DUP;
+      else { set_err(a.status, DERR_CORRUPT); f = 0; }
+    }
+  }
+  a.flag[g] = f;
+  a.aux[g] = x;
+}
+
+struct PredOwner { const u32 *flag; __device__ bool operator()(u32 g) const { return flag[g] == CAND_OWNER; } };
+struct EmitRank { u32 *krank; __device__ void operator()(u32 g, u32 r) const { krank[g] = r; } };
+
+// A3: a context stops at its first candidate that cannot be held (the pool ran out of free slots).
+__global__ void k_admit_stop(AdmitArgs a) {
+  u32 g = blockIdx.x * blockDim.x + threadIdx.x;
+  if (g >= a.n_cand) return;
+  const AdmitCtx c = a.ctx[admit_ctx_of(a, g)];
+  u32 f = a.flag[g];
+  bool ok = f == CAND_OLD || (f == CAND_OWNER && a.krank[g] < a.n_free) ||
+            (f == CAND_DUP && a.krank[a.aux[g]] < a.n_free);
+  if (!ok) atomicMin(&a.stop[c.res], c.b_start + (g - c.cand_base));
+}
+
+// A4: apply. Held candidates stamp/lock their block; owners that got a slot create the entry; owners
+// beyond the stop point give their claimed table slot back as a tombstone.
+__global__ void k_admit_apply(AdmitArgs a) {
+  u32 g = blockIdx.x * blockDim.x + threadIdx.x;
+  if (g >= a.n_cand) return;
+  if (a.status[ST_ERR]) return;
+  const AdmitCtx c = a.ctx[admit_ctx_of(a, g)];
+  u32 b = c.b_start + (g - c.cand_base);
+  u32 f = a.flag[g];
+  bool held = b < a.stop[c.res];
+  if (f == CAND_OLD) {
+    if (held) { u32 e = a.aux[g]; a.ent.stamp[e] = a.now; atomicAdd(&a.ent.infl[e], 1u); atomicAdd(&a.status[ST_ADOPTED], 1u); }
+  } else if (f == CAND_OWNER) {
+    u32 s = a.cslot[g];
+    if (held) {
+      u32 e = a.freelist[a.krank[g]];
+      a.ent.key[e] = a.keys[c.key_off + b];
+      a.ent.stamp[e] = a.now; a.ent.depth[e] = b; a.ent.rank[e] = 2; a.ent.floor[e] = 0; a.ent.tslot[e] = s;
+      atomicAdd(&a.ent.infl[e], 1u);
+      a.tab.slots[s].ent = e;
+      atomicAdd(&a.status[ST_INSERTED], 1u);
+    } else {
+      a.tab.slots[s].key = KEY_TOMB;
+      a.tab.slots[s].ent = ENT_NONE;
+      atomicAdd(&a.status[ST_TOMBS], 1u);
+    }
+  } else if (f == CAND_DUP) {
+    if (held) { u32 e = a.freelist[a.krank[a.aux[g]]]; atomicAdd(&a.ent.infl[e], 1u); atomicAdd(&a.status[ST_ADOPTED], 1u); }
+  }
+}
+
+// ---- per-context helpers -------------------------------------------------------------------------------
+// Releases the in-flight locks of blocks [0, n) of a key list (prefill done / terminate).
+__global__ void k_unlock(Table t, Entries en, const u64 *keys, u32 n, u32 now, u32 do_stamp, u32 *status) {
+  u32 b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= n) return;
+  u32 s = tab_find(t, keys[b], status);
+  if (s == ENT_NONE) { set_err(status, DERR_CORRUPT); return; }
+  u32 e = t.slots[s].ent;
+  if (e >= en.n_total) { set_err(status, DERR_CORRUPT); return; }
+  u32 old = atomicSub(&en.infl[e], 1u);
+  if (old == 0) { atomicAdd(&en.infl[e], 1u); set_err(status, DERR_CORRUPT); }
+  if (do_stamp) en.stamp[e] = now;
+}
+
+// Residency of every key of a list (block map).
+__global__ void k_block_map(Table t, Entries en, const u64 *keys, u32 n, u8 *tier, u32 *slot, u32 *status) {
+  u32 b = blockIdx.x * blockDim.x + threadIdx.x;
+  if (b >= n) return;
+  u32 s = tab_find(t, keys[b], status);
+  u32 e = s == ENT_NONE ? ENT_NONE : t.slots[s].ent;
+  if (e >= en.n_total) { tier[b] = 0xFF; slot[b] = 0xFFFFFFFFu; }
+  else if (e < en.n_hbm) { tier[b] = 0; slot[b] = e; }
+  else { tier[b] = 1; slot[b] = e - en.n_hbm; }
+}
+
+// ======================================================================================================
+// K3: classifier. rank[e] = max(floor[e], max over mappings (context, block) of the block's rank), where a
+// block's rank under a context is the highest message rank over the messages whose token span touches it.
+// ======================================================================================================
+struct ClsCtx { u64 key_off; u32 map_base; u32 valid; u32 msg_base; u32 n_msgs; };
+struct ClsArgs {
+  Table tab; Entries ent; const u64 *keys; const ClsCtx *ctx; u32 n_ctx; u32 n_map;
+  const u32 *m_start, *m_end; const u8 *m_rank; u32 *status;
+};
+
+__global__ void k_rank_reset(Entries en) {
+  u32 e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e < en.n_total) en.rank[e] = en.floor[e];
+}
+
+__global__ void k_classify(ClsArgs a) {
+  u32 g = blockIdx.x * blockDim.x + threadIdx.x;
+  if (g >= a.n_map) return;
+  u32 lo = 0, hi = a.n_ctx;
+  while (hi - lo > 1) { u32 mid = (lo + hi) >> 1; if (a.ctx[mid].map_base <= g) lo = mid; else hi = mid; }
+  const ClsCtx c = a.ctx[lo];
+  const u32 b = g - c.map_base;
+  const u32 t0 = b * 16, t1 = t0 + 16;
+  const u32 *ms = a.m_start + c.msg_base, *me = a.m_end + c.msg_base;
+  const u8 *mr = a.m_rank + c.msg_base;
+  // first message whose end is beyond t0 (ends are non-decreasing)
+  u32 l = 0, h = c.n_msgs;
+  while (l < h) { u32 mid = (l + h) >> 1; if (me[mid] > t0) h = mid; else l = mid + 1; }
+  u32 r = 0;
+  for (u32 j = l; j < c.n_msgs && ms[j] < t1; ++j)
+    if (me[j] > ms[j] && mr[j] > r) r = mr[j];
+  if (r == 0) return;
+  u32 s = tab_find(a.tab, a.keys[c.key_off + b], a.status);
+  if (s == ENT_NONE) return;  // mapped but not resident
+  u32 e = a.tab.slots[s].ent;
+  if (e < a.ent.n_total) atomicMax(&a.ent.rank[e], r);
+}
+
+// ======================================================================================================
+// K4: victim selection. Candidates of a tier: resident, not in flight, rank < 3. Whole ranks below the
+// boundary rank are taken, the ordered compaction keeps slot order, and a stable LSD radix sort on the
+// packed (rank, recency, inverted depth) key orders them; ties therefore end slot-ascending.
+// ======================================================================================================
+struct SelArgs {
+  Entries ent; u32 e0, n_slots;       // entry range of the tier
+  u32 n_req; u32 now; u32 stamp_bits, depth_bits; u32 mru;
+  u32 *status;
+};
+
+__device__ __forceinline__ bool sel_candidate(const SelArgs &a, u32 i, u32 *rank) {
+  u32 e = a.e0 + i;
+  if (!a.ent.key[e] || a.ent.infl[e]) return false;
+  u32 r = a.ent.rank[e];
+  *rank = r;
+  return r < 3;
+}
+
+__global__ void k_sel_count(SelArgs a) {
+  __shared__ u32 s[3];
+  if (threadIdx.x < 3) s[threadIdx.x] = 0;
+  __syncthreads();
+  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  u32 r = 0;
+  bool c = i < a.n_slots && sel_candidate(a, i, &r);
+  for (u32 k = 0; k < 3; ++k) {
+    u32 m = __ballot_sync(0xFFFFFFFFu, c && r == k);
+    if ((threadIdx.x & 31) == 0 && m) atomicAdd(&s[k], __popc(m));
+  }
+  __syncthreads();
+  if (threadIdx.x < 3 && s[threadIdx.x]) atomicAdd(&a.status[ST_RANK0 + threadIdx.x], s[threadIdx.x]);
+}
+
+// Highest rank that must be looked at to serve n_req victims (Algorithm 1: lower ranks go first).
+__device__ __forceinline__ u32 sel_boundary_rank(const u32 *status, u32 n_req) {
+  u32 cum = status[ST_RANK0];
+  if (cum >= n_req) return 0;
+  cum += status[ST_RANK1];
+  if (cum >= n_req) return 1;
+  return 2;
+}
+
+struct PredSel {
+  SelArgs a;
+  __device__ bool operator()(u32 i) const {
+    u32 r;
+    return sel_candidate(a, i, &r) && r <= sel_boundary_rank(a.status, a.n_req);
+  }
+};
+struct EmitSel {
+  SelArgs a; u64 *keys; u32 *vals;
+  __device__ void operator()(u32 i, u32 pos) const {
+    u32 e = a.e0 + i;
+    u64 r = a.ent.rank[e];
+    u64 st = a.ent.stamp[e];
+    u64 rec = (r == 1 && a.mru) ? (u64)a.now - st : st;       // newest first inside the idle tier
+    u64 dinv = ((1ull << a.depth_bits) - 1) - a.ent.depth[e];  // chain tail first
+    keys[pos] = (r << (a.stamp_bits + a.depth_bits)) | (rec << a.depth_bits) | dinv;
+    vals[pos] = i;
+  }
+};
+
+// ---- stable LSD radix sort, 8 bits per pass; element count read from the status block ----------------
+__global__ void __launch_bounds__(256) k_radix_hist(const u64 *keys, const u32 *status, u32 shift, u32 *counts) {
+  __shared__ u32 h[256];
+  const u32 m = status[ST_M];
+  const u32 n_tiles = (m + SORT_TILE - 1) / SORT_TILE;
+  if (blockIdx.x >= n_tiles) return;
+  h[threadIdx.x] = 0;
+  __syncthreads();
+  u32 base = blockIdx.x * SORT_TILE;
+  for (u32 k = threadIdx.x; k < SORT_TILE; k += 256) {
+    u32 i = base + k;
+    if (i < m) atomicAdd(&h[(u32)(keys[i] >> shift) & 255u], 1u);
+  }
+  __syncthreads();
+  counts[threadIdx.x * n_tiles + blockIdx.x] = h[threadIdx.x];   // digit-major
+}
+
+__global__ void __launch_bounds__(1024) k_radix_scan(u32 *counts, const u32 *status) {
+  // exclusive scan of 256 * n_tiles counts by one CTA (same scheme as k_scan_tiles)
+  __shared__ u32 warp_sums[32];
+  __shared__ u32 s_base;
+  const u32 m = status[ST_M];
+  const u32 n = 256u * ((m + SORT_TILE - 1) / SORT_TILE);
+  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) s_base = 0;
+  __syncthreads();
+  for (u32 start = 0; start < n; start += 1024) {
+    u32 i = start + tid;
+    u32 v = i < n ? counts[i] : 0, x = v;
+#pragma unroll
+    for (u32 o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(0xFFFFFFFFu, x, o); if (lane >= o) x += y; }
+    if (lane == 31) warp_sums[warp] = x;
+    __syncthreads();
+    if (warp == 0) {
+      u32 w = warp_sums[lane], z = w;
+#pragma unroll
+      for (u32 o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(0xFFFFFFFFu, z, o); if (lane >= o) z += y; }
+      warp_sums[lane] = z - w;
+    }
+    __syncthreads();
+    u32 incl = s_base + warp_sums[warp] + x;
+    if (i < n) counts[i] = incl - v;
+    __syncthreads();
+    if (tid == 1023) s_base = incl;
+    __syncthreads();
+  }
+}
+
+__global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const u32 *vals_in, u64 *keys_out, u32 *vals_out,
+                                                       const u32 *status, u32 shift, const u32 *offsets) {
+  // each warp owns 512 consecutive items of the tile and walks them in order, so equal digits keep
+  // their input order (stable)
+  __shared__ u32 cnt[8][256];
+  const u32 m = status[ST_M];
+  const u32 n_tiles = (m + SORT_TILE - 1) / SORT_TILE;
+  if (blockIdx.x >= n_tiles) return;
+  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  for (u32 k = tid; k < 8 * 256; k += 256) (&cnt[0][0])[k] = 0;
+  __syncthreads();
+  const u32 base = blockIdx.x * SORT_TILE + warp * 512;
+  u64 kreg[16];
+  u32 vreg[16];
+#pragma unroll
+  for (int it = 0; it < 16; ++it) {
+    u32 i = base + it * 32 + lane;
+    bool ok = i < m;
+    kreg[it] = ok ? keys_in[i] : 0;
+    vreg[it] = ok ? vals_in[i] : 0;
+    u32 d = (u32)(kreg[it] >> shift) & 255u;
+    u32 peers = __match_any_sync(0xFFFFFFFFu, ok ? d : 256u);
+    if (ok && (peers & ((1u << lane) - 1)) == 0) cnt[warp][d] += __popc(peers);
+    __syncwarp();
+  }
+  __syncthreads();
+  {  // per digit: exclusive scan across the 8 warps, plus the tile's global offset
+    u32 d = tid;
+    u32 run = offsets[d * n_tiles + blockIdx.x];
+#pragma unroll
+    for (int w = 0; w < 8; ++w) { u32 c = cnt[w][d]; cnt[w][d] = run; run += c; }
+  }
+  __syncthreads();
+#pragma unroll
+  for (int it = 0; it < 16; ++it) {
+    u32 i = base + it * 32 + lane;
+    bool ok = i < m;
+    u32 d = (u32)(kreg[it] >> shift) & 255u;
+    u32 peers = __match_any_sync(0xFFFFFFFFu, ok ? d : 256u);
+    u32 before = __popc(peers & ((1u << lane) - 1));
+    u32 pos = 0;
+    if (ok) pos = cnt[warp][d] + before;
+    __syncwarp();
+    if (ok && before == 0) cnt[warp][d] += __popc(peers);
+    __syncwarp();
+    if (ok) { keys_out[pos] = kreg[it]; vals_out[pos] = vreg[it]; }
+  }
+}
+
+__global__ void k_sel_emit(const u64 *keys, const u32 *vals, u32 n, u32 rank_shift, u32 *slots_out, u8 *states_out) {
+  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  slots_out[i] = vals[i];
+  states_out[i] = (u8)(keys[i] >> rank_shift);
+}
+
+// ======================================================================================================
+// Slot-list operations (offload / reload / release / compact): validate, plan, apply.
+// ======================================================================================================
+struct ListArgs {
+  Table tab; Entries ent;
+  const u32 *ids; u32 n; u32 e0, n_slots;   // listed slots of the source tier (entry = e0 + id)
+  u32 dst_e0;                                // first entry id of the destination tier
+  u32 *live;                                 // per item: 1 = must be copied
+  u32 *lidx;                                 // per item: exclusive rank among live items
+  const u32 *freelist; u32 n_free;           // lowest free destination slots
+  u32 *pair_src, *pair_dst;                  // mover pairs, indexed by lidx
+  u32 allow_inflight; u32 drop_dead; u32 drop_all;
+  u32 *status;
+};
+
+__global__ void k_list_validate(ListArgs a) {
+  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= a.n) return;
+  u32 id = a.ids[i];
+  a.live[i] = 0;
+  if (id >= a.n_slots) { set_err(a.status, DERR_RANGE); return; }
+  u32 e = a.e0 + id;
+  if (!a.ent.key[e] || atomicAdd(&a.ent.mark[e], 1u) != 0) { set_err(a.status, DERR_INVAL); return; }
+  if (a.ent.infl[e] && !a.allow_inflight) set_err(a.status, DERR_STATE);
+  a.live[i] = (a.drop_all || (a.drop_dead && a.ent.rank[e] == 0)) ? 0u : 1u;
+}
+
+__global__ void k_list_unmark(ListArgs a) {
+  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= a.n) return;
+  u32 id = a.ids[i];
+  if (id < a.n_slots) a.ent.mark[a.e0 + id] = 0;
+}
+
+struct PredLive { const u32 *live; __device__ bool operator()(u32 i) const { return live[i] != 0; } };
+// live item with rank r needs the r-th free destination slot; the first one that does not fit cuts the list
+struct EmitLive {
+  u32 *lidx; u32 n_free; u32 *status;
+  __device__ void operator()(u32 i, u32 r) const { lidx[i] = r; if (r >= n_free) atomicMin(&status[ST_CUT], i); }
+};
+struct PredFree { const u64 *key; u32 e0; __device__ bool operator()(u32 i) const { return key[e0 + i] == 0; } };
+struct EmitFree { u32 *list; u32 cap; __device__ void operator()(u32 i, u32 r) const { if (r < cap) list[r] = i; } };
+
+__device__ __forceinline__ void entry_clear(const Entries &en, u32 e) {
+  en.key[e] = 0; en.stamp[e] = 0; en.depth[e] = 0; en.infl[e] = 0; en.rank[e] = 0; en.floor[e] = 0; en.tslot[e] = ENT_NONE;
+}
+
+__device__ __forceinline__ void entry_move(const Table &t, const Entries &en, u32 src, u32 dst) {
+  en.key[dst] = en.key[src]; en.stamp[dst] = en.stamp[src]; en.depth[dst] = en.depth[src];
+  en.infl[dst] = en.infl[src]; en.rank[dst] = en.rank[src]; en.floor[dst] = en.floor[src];
+  u32 s = en.tslot[src];
+  en.tslot[dst] = s;
+  t.slots[s].ent = dst;
+  entry_clear(en, src);
+}
+
+__global__ void k_list_apply(ListArgs a) {
+  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= a.n) return;
+  if (a.status[ST_ERR]) return;
+  if (i >= a.status[ST_CUT]) return;
+  u32 id = a.ids[i];
+  u32 e = a.e0 + id;
+  if (!a.live[i]) {  // reclaim without copy: tombstone the key, free the slot
+    u32 s = a.ent.tslot[e];
+    a.tab.slots[s].key = KEY_TOMB;
+    a.tab.slots[s].ent = ENT_NONE;
+    entry_clear(a.ent, e);
+    atomicAdd(&a.status[ST_NDROP], 1u);
+  } else {
+    u32 r = a.lidx[i];
+    u32 d = a.freelist[r];
+    a.pair_src[r] = id;
+    a.pair_dst[r] = d;
+    entry_move(a.tab, a.ent, e, a.dst_e0 + d);
+    atomicAdd(&a.status[ST_NLIVE], 1u);
+  }
+}
+
+// ---- compaction plan: i-th occupied slot >= n_occ moves to the i-th free slot < n_occ ---------------
+struct PredHole { const u64 *key; u32 e0, n_occ; __device__ bool operator()(u32 i) const { return i < n_occ && key[e0 + i] == 0; } };
+struct PredMover { const u64 *key; u32 e0, n_occ; __device__ bool operator()(u32 i) const { return i >= n_occ && key[e0 + i] != 0; } };
+struct EmitList { u32 *list; __device__ void operator()(u32 i, u32 r) const { list[r] = i; } };
+
+__global__ void k_compact_apply(Table t, Entries en, u32 e0, const u32 *src, const u32 *dst, const u32 *status) {
+  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= status[ST_NMOVED] || status[ST_ERR]) return;
+  entry_move(t, en, e0 + src[i], e0 + dst[i]);
+}
+
+// ---- debug loader ---------------------------------------------------------------------------------------
+struct LoadArgs {
+  Table tab; Entries ent; const u64 *keys; const u8 *state; const u32 *stamp, *depth, *slot;
+  u32 n, e0, n_slots; u32 *status;
+};
+__global__ void k_load_check(LoadArgs a) {
+  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= a.n) return;
+  if (a.slot[i] >= a.n_slots) { set_err(a.status, DERR_RANGE); return; }
+  if (a.ent.key[a.e0 + a.slot[i]]) set_err(a.status, DERR_INVAL);
+  if (tab_find(a.tab, a.keys[i], a.status) != ENT_NONE) set_err(a.status, DERR_INVAL);
+}
+__global__ void k_load_apply(LoadArgs a) {
+  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= a.n || a.status[ST_ERR]) return;
+  u32 e = a.e0 + a.slot[i];
+  u32 s = tab_find_or_claim(a.tab, a.keys[i], a.status);
+  if (s == ENT_NONE) return;
+  a.tab.slots[s].ent = e;
+  a.ent.key[e] = a.keys[i]; a.ent.stamp[e] = a.stamp[i]; a.ent.depth[e] = a.depth[i];
+  a.ent.infl[e] = 0; a.ent.rank[e] = a.state[i]; a.ent.floor[e] = a.state[i]; a.ent.tslot[e] = s;
+}
+
+__global__ void k_states_out(Entries en, u32 e0, u32 n, u8 *out) {
+  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n) out[i] = en.key[e0 + i] ? (u8)en.rank[e0 + i] : (u8)0xFF;
+}
+
+// ======================================================================================================
+// K5: paged KV mover. A pool is addressed as base + slot * slot_stride + chunk * chunk_stride, so the
+// layer-major HBM layout, the block-major layout and the host tier all go through the same kernel.
+// Work item = (pair, chunk); each CTA streams whole chunks with 16-byte accesses, several loads in
+// flight per thread before the first store. The pair count may live in device memory.
+// ======================================================================================================
+struct PoolView { u8 *base; u64 slot_stride; u64 chunk_stride; u32 n_slots; };
+struct MoveArgs {
+  PoolView src, dst; const u32 *src_ids, *dst_ids;
+  u32 n_pairs; const u32 *n_pairs_dev;   // n_pairs_dev != nullptr: min(*n_pairs_dev, n_pairs)
+  u32 n_chunks; u32 chunk_bytes; u32 *status;
+};
+
+template <int UNROLL>
+__global__ void __launch_bounds__(256) k_move_blocks(MoveArgs a) {
+  u32 n_pairs = a.n_pairs;
+  if (a.n_pairs_dev) n_pairs = min(n_pairs, *a.n_pairs_dev);
+  const u64 n_items = (u64)n_pairs * a.n_chunks;
+  const u32 vec_per_chunk = a.chunk_bytes >> 4;
+  for (u64 item = blockIdx.x; item < n_items; item += gridDim.x) {
+    u32 pair = (u32)(item / a.n_chunks), chunk = (u32)(item % a.n_chunks);
+    u32 s = a.src_ids[pair], d = a.dst_ids[pair];
+    if (s >= a.src.n_slots || d >= a.dst.n_slots) { if (threadIdx.x == 0) set_err(a.status, DERR_RANGE); continue; }
+    const uint4 *sp = reinterpret_cast<const uint4 *>(a.src.base + s * a.src.slot_stride + chunk * a.src.chunk_stride);
+    uint4 *dp = reinterpret_cast<uint4 *>(a.dst.base + d * a.dst.slot_stride + chunk * a.dst.chunk_stride);
+    for (u32 v0 = threadIdx.x; v0 < vec_per_chunk; v0 += 256 * UNROLL) {
+      uint4 r[UNROLL];
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        u32 v = v0 + u * 256;
+        if (v < vec_per_chunk) r[u] = __ldcs(sp + v);
+      }
+#pragma unroll
+      for (int u = 0; u < UNROLL; ++u) {
+        u32 v = v0 + u * 256;
+        if (v < vec_per_chunk) __stcs(dp + v, r[u]);
+      }
+    }
+  }
+}
+
+}  // namespace kvt

@@ -1,0 +1,242 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle, element by element and
+bit-exact: all of this is integer, index and byte work, so the tolerance is zero."""
+import numpy as np
+import pytest
+
+import scenarios as S
+from paper_2609_39819_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def B():
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_39819_b200 import binding
+    binding.load_library()
+    return binding
+
+
+@pytest.fixture
+def make_gpu(B):
+    return lambda **kw: B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)
+
+
+@pytest.fixture
+def make_cpu(oracle):
+    return lambda **kw: oracle.OracleEngine(**kw)
+
+
+# ---- the scenario expectations that pin the oracle also hold for the CUDA engine -------------------
+@pytest.mark.parametrize("scenario", S.ALL, ids=lambda f: f.__name__)
+def test_scenario(make_gpu, scenario):
+    scenario(make_gpu)
+
+
+def test_mixed_pool_lru_switch(make_gpu):
+    S.mixed_pool_example(make_gpu, order=1)
+
+
+def test_error_codes(make_gpu, B):
+    ops = {k[3:]: getattr(B, k) for k in dir(B) if k.startswith("OP_") and k != "OPF_TOKENS_ON_DEVICE"}
+    S.error_codes(make_gpu, ops)
+
+
+# ---- stage 1: hashing ---------------------------------------------------------------------------------
+@pytest.mark.parametrize("n_tokens", [0, 15, 16, 17, 16 * 255, 16 * 256, 16 * 257 + 3, 16 * 1000 + 7, 258048])
+@pytest.mark.parametrize("seed", [0, 0xDEADBEEFCAFEF00D])
+def test_hash_matches_oracle(B, oracle, n_tokens, seed):
+    import torch
+    rng = np.random.default_rng(n_tokens + 1)
+    tok = rng.integers(0, W.VOCAB, n_tokens, dtype=np.uint32)
+    if n_tokens > 100:
+        tok[7] = 0
+        tok[8] = W.VOCAB - 1
+    d = torch.from_numpy(tok.view(np.int32)).cuda() if n_tokens else torch.empty(0, dtype=torch.int32, device="cuda")
+    got = B.hash_tokens(d, seed).cpu().numpy().view(np.uint64)
+    want = oracle.hash_tokens(tok, seed)
+    assert got.shape == want.shape and np.array_equal(got, want)
+
+
+def test_hash_full_size_batch_matches_oracle(B, oracle):
+    """C4-sized hashing: 64 sequences x 16,128 blocks through one kernel sequence each."""
+    import torch
+    rng = np.random.default_rng(99)
+    for _ in range(3):
+        tok = rng.integers(0, W.VOCAB, 258048, dtype=np.uint32)
+        got = B.hash_tokens(torch.from_numpy(tok.view(np.int32)).cuda(), 0).cpu().numpy().view(np.uint64)
+        assert np.array_equal(got, oracle.hash_tokens(tok, 0))
+
+
+# ---- whole path on C1 traces: every reported value and every payload byte ----------------------------
+def _replay_pair(gpu, cpu, trace, payload, check_pools=True, record_states=True, verify_every=0):
+    og = W.ReplayOptions(payload=payload, record_states=record_states, verify_payload_every=verify_every)
+    oc = W.ReplayOptions(payload=payload, record_states=record_states, verify_payload_every=verify_every)
+    n_calls = 0
+    for (i, kind, rg), (_, _, rc) in zip(W.replay(gpu, trace, og), W.replay(cpu, trace, oc)):
+        if kind == "call":
+            n_calls += 1
+            diff = W.records_equal(rg, rc, f"event[{i}]")
+            assert diff is None, diff
+            if "payload_ok" in rg:
+                assert rg["payload_ok"] and rc["payload_ok"]
+    sg, sc = gpu.get_stats(), cpu.get_stats()
+    for k in sc:
+        if k not in ("table_rebuilds", "tombstones"):
+            assert sg[k] == sc[k], k
+    if check_pools and payload is not None:
+        for tier, n in ((0, gpu.n_hbm_blocks), (1, gpu.n_host_blocks)):
+            keys = cpu.get_entries(tier)["key"]
+            for s in np.nonzero(keys)[0]:
+                assert np.array_equal(gpu.read_block(tier, int(s)), cpu.read_block(tier, int(s))), (tier, s)
+    return n_calls
+
+
+@pytest.mark.parametrize("seed", [0, 1, 2, 3, 7, 39, 63, 86, 102, 120, 136, 164])
+def test_c1_trace_parity(B, oracle, seed):
+    kw = dict(n_hbm_blocks=128, n_host_blocks=512, max_contexts=64, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    _replay_pair(gpu, cpu, W.trace_c1(seed), W.payload_normal_bf16, verify_every=2)
+
+
+@pytest.mark.parametrize("layout,order", [(0, 1), (1, 0), (1, 1)])
+def test_c1_trace_parity_other_layouts_and_orders(B, oracle, layout, order):
+    kw = dict(n_hbm_blocks=96, n_host_blocks=64, max_contexts=64, pool_layout=layout, suspended_order=order,
+              **W.GEO_TOY.kwargs())
+    for seed in (7, 63, 86):
+        gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)
+        cpu = oracle.OracleEngine(**kw)
+        _replay_pair(gpu, cpu, W.trace_c1(seed), W.payload_pattern)
+
+
+def test_scaled_c2_trace_parity(B, oracle):
+    kw = dict(n_hbm_blocks=96, n_host_blocks=64, max_contexts=8, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    n = _replay_pair(gpu, cpu, W.trace_c2(1, scale=1 / 32), W.payload_pattern, verify_every=7)
+    assert n > 20
+
+
+def test_scaled_c3_trace_parity(B, oracle):
+    trace, n_ctx = W.trace_c3(1, n_sessions=8, scale=1 / 32)
+    kw = dict(n_hbm_blocks=1024, n_host_blocks=1024, max_contexts=n_ctx, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 20, max_messages=1 << 15, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    _replay_pair(gpu, cpu, trace, W.payload_pattern, record_states=True)
+    assert cpu.get_stats()["offloaded"] > 0 and cpu.get_stats()["reloaded"] > 0
+
+
+def test_full_length_c2_session_metadata_parity(B, oracle):
+    """One 128K-token ReAct session (C2's trace at full size) on a metadata-only engine with C2's
+    block counts: every lookup, victim list, admission and state vector equals the oracle's."""
+    kw = dict(n_hbm_blocks=20480, n_host_blocks=61440, max_contexts=4, metadata_only=True, **W.GEO_8B.kwargs())
+    gpu = B.Engine(max_tokens=1 << 20, max_messages=1 << 12, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    n = _replay_pair(gpu, cpu, W.trace_c2(1), None, record_states=True)
+    assert n >= 30 and cpu.get_stats()["dropped"] > 0
+
+
+# ---- C4: metadata stress at full size -------------------------------------------------------------------
+def _c4_setup(B, oracle, n_resident, chain_blocks, n_calls):
+    inp = W.inputs_c4(1, n_resident=n_resident, chain_blocks=chain_blocks, n_calls=n_calls)
+    kw = dict(n_hbm_blocks=n_resident, n_host_blocks=0, max_contexts=n_calls + 1, metadata_only=True, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=(n_calls + 1) * chain_blocks * 16 * 2, max_messages=1024,
+                   max_batch_blocks=n_calls * chain_blocks, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    keys = np.concatenate([oracle.hash_tokens(c) for c in inp.chain_tokens])
+    for eng in (gpu, cpu):
+        eng.debug_load_resident(keys, inp.state, inp.stamp, inp.depth, inp.slot, 0)
+        for i, t in enumerate(inp.calls):
+            eng.spawn(i)
+            eng.append(i, t)
+    return inp, gpu, cpu
+
+
+@pytest.mark.parametrize("n_resident,chain_blocks,n_calls", [(5000, 700, 9), (1 << 20, 16128, 64)])
+def test_c4_lookup_and_select_parity(B, oracle, n_resident, chain_blocks, n_calls):
+    inp, gpu, cpu = _c4_setup(B, oracle, n_resident, chain_blocks, n_calls)
+    ids = list(range(n_calls))
+    # selection before any call: the whole pool is a candidate; 10% stays in the dead tier,
+    # 35% crosses into the idle (MRU) tier, 75% into the active tier
+    for frac in (0.10, 0.35, 0.75):
+        n = int(n_resident * frac)
+        vg, sg = gpu.select_victims(0, n)
+        vc, sc = cpu.select_victims(0, n)
+        assert np.array_equal(vg, vc) and np.array_equal(sg, sc), frac
+    ig = gpu.map_blocks(ids, 0)
+    ic = cpu.map_blocks(ids, 0)
+    assert np.array_equal(ig, ic)
+    assert 0.3 < ic["hit_len"].sum() / ic["n_blocks"].sum() < 0.6
+    for c in (0, n_calls // 2, n_calls - 1):
+        for a, b in zip(gpu.get_block_map(c), cpu.get_block_map(c)):
+            assert np.array_equal(a, b)
+    # with the hits locked in flight, select 10% of the pool
+    n = n_resident // 10
+    vg, sg = gpu.select_victims(0, n)
+    vc, sc = cpu.select_victims(0, n)
+    assert np.array_equal(vg, vc) and np.array_equal(sg, sc)
+    # drop them and admit the misses into the freed slots
+    assert gpu.offload(vg) == cpu.offload(vc)
+    ag = gpu.map_blocks(ids, 1)
+    ac = cpu.map_blocks(ids, 1)
+    assert np.array_equal(ag, ac)
+    for c in ids:
+        gpu.prefill_done(c)
+        cpu.prefill_done(c)
+    eg, ec = gpu.get_entries(0), cpu.get_entries(0)
+    for k in ec:
+        assert np.array_equal(eg[k], ec[k]), k
+    assert np.array_equal(gpu.get_states(0), cpu.get_states(0))
+    sg, sc = gpu.get_stats(), cpu.get_stats()
+    for k in sc:
+        if k not in ("table_rebuilds", "tombstones"):
+            assert sg[k] == sc[k], k
+
+
+# ---- C5: the raw mover ------------------------------------------------------------------------------------
+@pytest.mark.parametrize("geo", [W.GEO_TOY, W.GEO_128K, W.GEO_8B], ids=lambda g: g.name)
+@pytest.mark.parametrize("layout", [0, 1])
+def test_c5_mover_parity(B, oracle, geo, layout):
+    import torch
+    n_slots = 24 if geo.block_bytes > (1 << 20) else 200
+    kw = dict(n_hbm_blocks=n_slots, n_host_blocks=n_slots, max_contexts=2, pool_layout=layout, **geo.kwargs())
+    gpu = B.Engine(max_tokens=1 << 12, max_messages=64, max_batch_blocks=4096, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    rng = np.random.default_rng(5)
+    fill = rng.integers(0, 256, gpu.hbm_pool.numel(), dtype=np.uint8)
+    gpu.hbm_pool.copy_(torch.from_numpy(fill))
+    cpu.hbm_pool[:] = fill
+    for n in (1, 2, 7, n_slots // 2, n_slots):
+        for permuted in (False, True):
+            src = W.ids_c5(1, n, n_slots, permuted)
+            dst = W.ids_c5(2, n, n_slots, permuted)
+            for eng in (gpu, cpu):
+                eng.copy_blocks(0, src, 1, dst)          # gather HBM -> host tier
+            torch.cuda.synchronize()
+            assert np.array_equal(gpu.host_pool.numpy(), cpu.host_pool)
+            back = W.ids_c5(3, n, n_slots, permuted)
+            for eng in (gpu, cpu):
+                eng.copy_blocks(1, dst, 0, back)         # scatter host tier -> HBM
+            torch.cuda.synchronize()
+            assert np.array_equal(gpu.hbm_pool.cpu().numpy(), cpu.hbm_pool)
+    # HBM -> HBM move with disjoint halves, ids resident on the device
+    half = n_slots // 2
+    src = np.arange(half, dtype=np.uint32)
+    dst = (np.random.default_rng(6).permutation(half) + half).astype(np.uint32)
+    gpu.copy_blocks(0, torch.from_numpy(src.view(np.int32)).cuda(), 0, torch.from_numpy(dst.view(np.int32)).cuda())
+    cpu.copy_blocks(0, src, 0, dst)
+    torch.cuda.synchronize()
+    assert np.array_equal(gpu.hbm_pool.cpu().numpy(), cpu.hbm_pool)
+
+
+def test_mover_with_second_tier_in_hbm(B, oracle):
+    """The in-device measurement mode: the second tier lives in HBM; results are the same."""
+    kw = dict(n_hbm_blocks=64, n_host_blocks=64, max_contexts=4, **W.GEO_128K.kwargs())
+    gpu = B.Engine(max_tokens=1 << 16, max_messages=256, host_pool_on_device=True, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    S.offload_reload_round_trip(lambda **k: B.Engine(max_tokens=1 << 16, max_messages=256, host_pool_on_device=True, **k),
+                                geos=[W.GEO_128K.kwargs()])
+    del gpu, cpu
