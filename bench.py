@@ -1,0 +1,543 @@
+#!/usr/bin/env python
+"""Benchmark of the KV-cache hot path on one (or N independent) B200.
+
+Workload (N=1): the single long ReAct session of configuration C2 — 8B-class KV geometry
+(32 layers x 8 KV heads x 128, bf16: 2 MiB per 16-token block), 40 GiB HBM pool (20,480 blocks),
+host tier of up to 120 GiB — under tier pressure: between two LLM calls of the session, half of its
+idle KV is pushed out of HBM (the engine's own victim order), so every call hashes and looks up the
+whole context, reloads the evicted half of its prefix from the second tier, admits the new blocks
+and, after prefill, is evicted again. One step = one such call = every stage of the path:
+apply ops -> hash -> lookup -> classify -> select victims -> offload -> reload -> admit.
+
+Two measurements of the same steps:
+  value : second tier resident in HBM and tokens resident on the device (inputs in HBM when the timed
+          region starts); the mover runs HBM<->HBM and is judged against the HBM roofline.
+  e2e   : the real thing through the same C-ABI calls: tokens come from pinned host buffers, the
+          second tier is pinned host memory, every offload / reload crosses the host link inside the
+          timed region.
+`--impl reference` times the CPU oracle (plain single-threaded C++) on the same steps.
+Prints ONE JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import tempfile
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2609_39819_b200 import workloads as W  # noqa: E402
+
+METRIC = "KV block GB/s (HBM & host link) vs roofline; blocks hashed+looked up/sec"
+GiB = 1 << 30
+# DRAM traffic of the mover kernel per algorithmic byte (read + write), from the ncu capture summarised
+# in profiles/ (dram__bytes_read.sum + dram__bytes_write.sum over 2 x payload bytes of the launch);
+# None until a capture exists.
+MOVER_TRAFFIC_PER_ALGO_BYTE = None
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=8)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--hbm-gib", type=float, default=40.0)
+    ap.add_argument("--host-gib", type=float, default=120.0)
+    ap.add_argument("--cpu-steps", type=int, default=6, help="steps of the bounded CPU-oracle sample")
+    ap.add_argument("--skip-e2e", action="store_true")
+    ap.add_argument("--skip-cpu", action="store_true")
+    return ap.parse_args()
+
+
+# ---- workload ---------------------------------------------------------------------------------------------
+def split_turns(trace):
+    """Splits a C2 trace into (spawn events, [(events before the call, contexts of the call, events after
+    it)]). In C2 the only event that follows a call is the removal of that call's scratch message."""
+    setup = [ev for ev in trace if ev[0] == "spawn"]
+    turns, pre, i = [], [], len(setup)
+    while i < len(trace):
+        ev = trace[i]
+        i += 1
+        if ev[0] != "call":
+            pre.append(ev)
+            continue
+        post = []
+        if i < len(trace) and trace[i][0] == "remove":
+            post.append(trace[i])
+            i += 1
+        turns.append((pre, ev[1], post))
+        pre = []
+    return setup, turns
+
+
+def make_turns(seed, n_needed):
+    target, max_turns = 131072, 100
+    while True:
+        trace = W.trace_c2(seed, target_tokens=target, max_turns=max_turns)
+        setup, turns = split_turns(trace)
+        if len(turns) >= n_needed + 1:
+            return setup, turns, target
+        target *= 2
+        max_turns = max(max_turns, 2 * n_needed)
+
+
+def apply_event(eng, ev, tok):
+    k = ev[0]
+    if k == "spawn": eng.spawn(ev[1])
+    elif k == "append": eng.append(ev[1], tok(ev[2]))
+    elif k == "replace": eng.replace(ev[1], ev[2], ev[3], tok(ev[4]))
+    elif k == "remove": eng.remove(ev[1], ev[2], ev[3])
+    elif k == "one_off": eng.one_off(ev[1], ev[2], ev[3])
+    elif k == "terminate": eng.terminate(ev[1])
+    else: raise ValueError(k)
+
+
+CPU_PRESSURE_CAP = 512   # blocks evicted per step in the CPU-oracle runs (bounded sample: 1 GiB each way)
+
+
+def pressure_evict(eng, cap=None):
+    """Other tenants push half of the session's resident blocks out of HBM. With `cap`, at most that
+    many live blocks are moved (dead ones are dropped either way)."""
+    n = eng.get_stats()["occ_hbm"] // 2
+    if cap is not None and n:
+        _v, s = eng.select_victims(W.TIER_HBM, n)
+        n = min(n, int((s == 0).sum()) + cap)
+    if n:
+        W.evict(eng, n)
+
+
+def run_step(eng, turn, tok, opt, pressure=True, timers=None, cap=None):
+    """One LLM call of the session through the whole path, then the tier pressure between calls."""
+    pre, ctxs, post = turn
+    t0 = time.perf_counter()
+    for ev in pre:
+        apply_event(eng, ev, tok)
+    t1 = time.perf_counter()
+    W.run_call(eng, ctxs, opt)
+    t2 = time.perf_counter()
+    for ev in post:
+        apply_event(eng, ev, tok)
+    if pressure:
+        pressure_evict(eng, cap)
+    t3 = time.perf_counter()
+    if timers is not None:
+        timers["ops_ms"] += (t1 - t0) * 1e3
+        timers["call_ms"] += (t2 - t1) * 1e3
+        timers["pressure_ms"] += (t3 - t2) * 1e3
+
+
+class StageTimer:
+    """Wall-clock per API entry point (each of them synchronises its stream before returning, except
+    apply_op and classify, whose device time then shows up in the next synchronising call)."""
+
+    NAMES = ("map_blocks", "select_victims", "offload", "reload", "get_block_map", "release", "append", "replace",
+             "remove", "one_off", "prefill_done", "get_stats")
+
+    def __init__(self, eng):
+        self.ms = {}
+        self.calls = {}
+        for name in self.NAMES:
+            fn = getattr(eng, name)
+            setattr(eng, name, self._wrap(name, fn))
+
+    def _wrap(self, name, fn):
+        def inner(*a, **k):
+            t = time.perf_counter()
+            r = fn(*a, **k)
+            key = name
+            if name == "map_blocks":
+                key = "map_lookup(hash+lookup)" if a[1] == 0 else "map_admit"
+            self.ms[key] = self.ms.get(key, 0.0) + (time.perf_counter() - t) * 1e3
+            self.calls[key] = self.calls.get(key, 0) + 1
+            return r
+        return inner
+
+    def reset(self):
+        self.ms, self.calls = {}, {}
+
+
+# ---- helpers ------------------------------------------------------------------------------------------------
+def mem_available_bytes():
+    try:
+        for ln in open("/proc/meminfo"):
+            if ln.startswith("MemAvailable"):
+                avail = int(ln.split()[1]) * 1024
+                break
+        else:
+            return 0
+        try:
+            lim = open("/sys/fs/cgroup/memory.max").read().strip()
+            if lim != "max":
+                cur = int(open("/sys/fs/cgroup/memory.current").read())
+                avail = min(avail, int(lim) - cur)
+        except OSError:
+            pass
+        return avail
+    except OSError:
+        return 0
+
+
+class ClockSampler:
+    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index):
+        self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
+        try:
+            self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                                       "-i", str(gpu_index), "-lms", "200"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except OSError:
+            self.p = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.p is None:
+            return out
+        self.p.terminate()
+        try:
+            self.p.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.p.kill()
+        self.f.flush()
+        self.f.seek(0)
+        sm, mx, reasons = [], [], set()
+        names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        for ln in self.f:
+            parts = [x.strip() for x in ln.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, parts[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        self.f.close()
+        os.unlink(self.f.name)
+        if sm:
+            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        return json.load(open(p)).get("hbm_gbs", 6650.0), "measured"
+    return 6650.0, "fallback"
+
+
+def host_link_peaks(torch):
+    """1 GiB pinned cudaMemcpyAsync in each direction, best of 10 (the host-link roofline)."""
+    h = torch.empty(GiB, dtype=torch.uint8, pin_memory=True)
+    d = torch.empty(GiB, dtype=torch.uint8, device="cuda")
+    out = {}
+    for name, fn in (("h2d", lambda: d.copy_(h, non_blocking=True)), ("d2h", lambda: h.copy_(d, non_blocking=True))):
+        best = 1e9
+        for i in range(12):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record(); torch.cuda.synchronize()
+            if i >= 2:
+                best = min(best, a.elapsed_time(b))
+        out[name] = GiB / best / 1e6
+    del h, d
+    return out
+
+
+# ---- GPU arms -------------------------------------------------------------------------------------------------
+def gpu_arm(args, torch, B, setup, turns, n_ff, e2e, n_host_blocks, n_hbm_blocks, rank=0, world=1, barrier=None):
+    """Fast-forwards n_ff turns untimed, runs W warm-up steps, then times exactly K steps."""
+    W_, K = args.warmup, args.steps
+    geo = W.GEO_8B
+    max_tok = 1 << 21
+    eng = B.Engine(n_hbm_blocks=n_hbm_blocks, n_host_blocks=n_host_blocks, max_contexts=4, max_tokens=max_tok,
+                   max_messages=1 << 13, max_batch_blocks=max_tok // 16, host_pool_on_device=not e2e, zero_pools=False,
+                   **geo.kwargs())
+    eng.set_profiling(True)
+    # token sources: device tensors (value arm) or pinned host tensors (e2e arm)
+    cache = {}
+
+    def tok(arr):
+        k = id(arr)
+        if k not in cache:
+            t = torch.from_numpy(arr.view(np.int32))
+            cache[k] = t.cuda() if not e2e else t.pin_memory()
+        return cache[k]
+
+    used = turns[: n_ff + W_ + K]
+    for pre, _c, _post in used:
+        for ev in pre:
+            if ev[0] in ("append", "replace"):
+                tok(ev[2] if ev[0] == "append" else ev[4])
+    torch.cuda.synchronize()
+    opt = W.ReplayOptions(payload=None, record_states=False)
+    for ev in setup:
+        apply_event(eng, ev, tok)
+    # fast-forward; the blocks admitted here get a key-derived payload so movement can be verified later
+    base = (torch.arange(eng.block_bytes // 4, dtype=torch.int64, device="cuda") * 0x9E3779B1) & 0xFFFFFFFF
+    pool = eng.hbm_pool.view(eng.n_chunks, eng.n_hbm_blocks, eng.chunk_bytes)
+    written = {}
+    for t in range(n_ff):
+        pre, ctxs, post = used[t]
+        for ev in pre:
+            apply_event(eng, ev, tok)
+        info = eng.map_blocks(ctxs, 0)
+        adm = eng.map_blocks(ctxs, 1)
+        keys, tier, slot = eng.get_block_map(ctxs[0])
+        for b in range(int(info[0]["hit_len"]), int(adm[0]["n_held"])):
+            if tier[b] == 0 and len(written) < 512 and b % 7 == 0:
+                key = int(keys[b])
+                w = ((base + (key & 0xFFFFFFFF)) & 0xFFFFFFFF) ^ (key >> 32)
+                pool[:, int(slot[b]), :] = w.to(torch.int32).view(torch.uint8).view(eng.n_chunks, eng.chunk_bytes)
+                written[key] = True
+        for c in ctxs:
+            eng.prefill_done(c)
+        for ev in post:
+            apply_event(eng, ev, tok)
+    pressure_evict(eng)
+    for t in range(n_ff, n_ff + W_):
+        run_step(eng, used[t], tok, opt)
+    timer = StageTimer(eng)
+    timers = {"ops_ms": 0.0, "call_ms": 0.0, "pressure_ms": 0.0}
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    s0 = eng.get_stats()
+    timer.reset()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for t in range(n_ff + W_, n_ff + W_ + K):
+        run_step(eng, used[t], tok, opt, timers=timers)
+    ev1.record()
+    torch.cuda.synchronize()
+    if barrier:
+        barrier()
+    ms = ev0.elapsed_time(ev1)
+    s1 = eng.get_stats()
+    d = {k: s1[k] - s0[k] for k in s1}
+    # verification: every block written during the fast-forward still holds its key-derived payload,
+    # wherever the offload / reload cycles have left it
+    n_ok = n_seen = 0
+    for tier in (0, 1):
+        keys = eng.get_entries(tier)["key"]
+        for s in np.nonzero(keys)[0]:
+            key = int(keys[s])
+            if key in written and n_seen < 64:
+                n_seen += 1
+                w = ((base + (key & 0xFFFFFFFF)) & 0xFFFFFFFF) ^ (key >> 32)
+                want = w.to(torch.int32).view(torch.uint8).cpu().numpy()
+                n_ok += int(np.array_equal(eng.read_block(tier, int(s)), want))
+    tok_bytes = sum(4 * len(ev[2] if ev[0] == "append" else ev[4]) for pre, _c, _p in used[n_ff + W_:] for ev in pre
+                    if ev[0] in ("append", "replace"))
+    res = dict(ms=ms, stats=d, stage_ms=dict(timer.ms), stage_calls=dict(timer.calls), timers=timers,
+               verified=(n_ok, n_seen), tok_bytes=tok_bytes, block_bytes=eng.block_bytes)
+    eng.close()
+    del eng, pool, cache
+    torch.cuda.empty_cache()
+    return res
+
+
+def cpu_arm(args, setup, turns, n_ff, n_steps, n_warm, n_hbm_blocks, n_host_blocks):
+    """The CPU oracle, as it stands, on the same steps: payload copies are plain memcpy on one core."""
+    from oracle import kvt_oracle
+    kvt_oracle.build()
+    eng = kvt_oracle.OracleEngine(n_hbm_blocks=n_hbm_blocks, n_host_blocks=n_host_blocks, max_contexts=4,
+                                  **W.GEO_8B.kwargs())
+    opt = W.ReplayOptions(payload=None, record_states=False)
+    ident = lambda a: a
+    for ev in setup:
+        apply_event(eng, ev, ident)
+    for t in range(n_ff):
+        pre, ctxs, post = turns[t]
+        for ev in pre:
+            apply_event(eng, ev, ident)
+        eng.map_blocks(ctxs, 0)
+        eng.map_blocks(ctxs, 1)
+        for c in ctxs:
+            eng.prefill_done(c)
+        for ev in post:
+            apply_event(eng, ev, ident)
+    pressure_evict(eng, CPU_PRESSURE_CAP)
+    for t in range(n_ff, n_ff + n_warm):
+        run_step(eng, turns[t], ident, opt, cap=CPU_PRESSURE_CAP)
+    s0 = eng.get_stats()
+    t0 = time.perf_counter()
+    for t in range(n_ff + n_warm, n_ff + n_warm + n_steps):
+        run_step(eng, turns[t], ident, opt, cap=CPU_PRESSURE_CAP)
+    sec = time.perf_counter() - t0
+    s1 = eng.get_stats()
+    d = {k: s1[k] - s0[k] for k in s1}
+    return dict(sec=sec, stats=d, block_bytes=eng.block_bytes)
+
+
+def kv_bytes(d, block_bytes):
+    return (d["offloaded"] + d["reloaded"]) * block_bytes
+
+
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    W_, K = args.warmup, args.steps
+    n_hbm_blocks = int(args.hbm_gib * GiB) // W.GEO_8B.block_bytes
+    setup, turns, target = make_turns(args.seed + rank, W_ + K + 4)
+    n_ff = len(turns) - (W_ + K)
+    workload = (f"C2 single long ReAct session under tier pressure: seed {args.seed}, {len(turns)} turns to "
+                f"{target} tokens, fast-forward {n_ff} turns then {W_}+{K} timed calls; 8B-class KV 32x8x128 bf16 "
+                f"(2 MiB/block); HBM pool {n_hbm_blocks} blocks ({args.hbm_gib:g} GiB)")
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        n_host_blocks = min(int(args.host_gib * GiB), int(mem_available_bytes() * 0.5)) // W.GEO_8B.block_bytes
+        r = cpu_arm(args, setup, turns, n_ff, K, W_, n_hbm_blocks, n_host_blocks)
+        gbs = kv_bytes(r["stats"], r["block_bytes"]) / r["sec"] / 1e9
+        line = {
+            "impl": "reference", "metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": args.gpus, "steps": K,
+            "warmup": W_, "ms_per_step": r["sec"] * 1e3 / K, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+            "config": {"workload": workload, "host_tier_blocks": n_host_blocks},
+            "blocks_hashed_looked_up_per_s": r["stats"]["blocks_hashed"] / r["sec"],
+            "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle",
+                             "sample": f"the same {K} calls with the tier pressure capped at {CPU_PRESSURE_CAP} blocks "
+                                       f"(1 GiB each way) per step; whole path incl. payload memcpy; one thread"},
+            "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        }
+        print(json.dumps(line))
+        return
+
+    import torch
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    from paper_2609_39819_b200 import build as kbuild
+    if rank == 0 or not os.path.exists(kbuild.LIB):
+        kbuild.build_lib()
+    barrier = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        barrier = lambda: (dist.barrier(), torch.cuda.synchronize())
+        barrier()
+    from paper_2609_39819_b200 import binding as B
+    B.load_library()
+    hbm_peak, peak_kind = measured_peaks()
+    link = host_link_peaks(torch)
+
+    # ---- value arm: everything resident in HBM ------------------------------------------------------------
+    sampler = ClockSampler(local_rank)
+    free_b, _total = torch.cuda.mem_get_info()
+    want2 = int(args.host_gib * GiB) // W.GEO_8B.block_bytes
+    fit2 = int((free_b - n_hbm_blocks * W.GEO_8B.block_bytes - 6 * GiB) // W.GEO_8B.block_bytes)
+    tier2_dev_blocks = max(min(want2, fit2), 9000)
+    v = gpu_arm(args, torch, B, setup, turns, n_ff, False, tier2_dev_blocks, n_hbm_blocks, rank, world, barrier)
+    clocks = sampler.stop()
+
+    # ---- e2e arm: pinned host tier, tokens from pinned host buffers ---------------------------------------
+    e = None
+    host_blocks = 0
+    if not args.skip_e2e:
+        budget = min(int(args.host_gib * GiB), int(mem_available_bytes() * 0.5) // max(world, 1))
+        host_blocks = max(budget // W.GEO_8B.block_bytes, 9000)
+        e = gpu_arm(args, torch, B, setup, turns, n_ff, True, host_blocks, n_hbm_blocks, rank, world, barrier)
+
+    def agg(x, op):
+        if world == 1:
+            return x
+        import torch.distributed as dist
+        t = torch.tensor([float(x)], dtype=torch.float64, device="cuda")
+        dist.all_reduce(t, op=op)
+        return t.item()
+
+    vbytes = kv_bytes(v["stats"], v["block_bytes"])
+    if world > 1:
+        import torch.distributed as dist
+        ms = agg(v["ms"], dist.ReduceOp.MAX)
+        tot_bytes = agg(vbytes, dist.ReduceOp.SUM)
+        tot_hashed = agg(v["stats"]["blocks_hashed"], dist.ReduceOp.SUM)
+        launches = agg(v["stats"]["kernel_launches"], dist.ReduceOp.SUM)
+        if e:
+            e_ms = agg(e["ms"], dist.ReduceOp.MAX)
+            e_bytes = agg(kv_bytes(e["stats"], e["block_bytes"]), dist.ReduceOp.SUM)
+    else:
+        ms, tot_bytes, tot_hashed, launches = v["ms"], vbytes, v["stats"]["blocks_hashed"], v["stats"]["kernel_launches"]
+        if e:
+            e_ms, e_bytes = e["ms"], kv_bytes(e["stats"], e["block_bytes"])
+    if rank != 0:
+        return
+
+    st = v["stats"]
+    mover_s = st["mover_ns"] / 1e9
+    achieved = 2 * st["mover_bytes"] / mover_s / 1e9 if mover_s else 0.0
+    per_launch_bytes = 2 * st["mover_bytes"] / max(st["mover_launches"], 1)
+    roofline = {
+        "bound": "hbm", "kernel": "k_move_blocks", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+        "frac": achieved / hbm_peak, "peak_kind": f"{peak_kind} copy bandwidth (MEASURED_PEAKS.json hbm_gbs)",
+        "frac_of_nominal_8TBs": achieved / 8000.0,
+        "launches": st["mover_launches"], "avg_launch_ms": mover_s * 1e3 / max(st["mover_launches"], 1),
+        "algorithmic_bytes_per_launch": per_launch_bytes,
+        "traffic": None if MOVER_TRAFFIC_PER_ALGO_BYTE is None else MOVER_TRAFFIC_PER_ALGO_BYTE * per_launch_bytes,
+    }
+    line = {
+        "metric": METRIC, "value": tot_bytes / (ms / 1e3) / 1e9, "unit": "GB/s", "n_gpus": args.gpus, "steps": K,
+        "warmup": W_, "ms_per_step": ms / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "u8", "data": "synthetic",
+        "config": {"workload": workload, "second_tier_blocks_value_arm": tier2_dev_blocks,
+                   "host_tier_blocks_e2e_arm": host_blocks,
+                   "l2": "inputs larger than L2: every step streams GiBs of KV blocks; no flush needed",
+                   "per_rank": "independent session per GPU, no collective on the data path" if world > 1 else "1 GPU"},
+        "blocks_hashed_looked_up_per_s": tot_hashed / (ms / 1e3),
+        "kv_blocks_moved_per_step": (st["offloaded"] + st["reloaded"]) / K,
+        "blocks_hashed_per_step": st["blocks_hashed"] / K,
+        "gpu_launches": int(launches),
+        "clocks": clocks,
+        "roofline": roofline,
+        "stage_wall_ms_per_step": {k: round(x / K, 4) for k, x in v["stage_ms"].items()},
+        "verified_blocks": {"value_arm": v["verified"], "e2e_arm": e["verified"] if e else None},
+        "host_cpu": {"cores": os.cpu_count()},
+    }
+    if e:
+        es = e["stats"]
+        e_mover_s = es["mover_ns"] / 1e9
+        line["e2e"] = {
+            "value": e_bytes / (e_ms / 1e3) / 1e9, "unit": "GB/s", "ms_per_step": e_ms / K,
+            "h2d_bytes_per_step": (es["bytes_h2d"] + e["tok_bytes"]) / K,
+            # payload gathered to the host tier + what the calls return: two block maps per call
+            # (13 B per block), victim lists (5 B per victim), one 128-byte status block per synchronising call
+            "d2h_bytes_per_step": (es["bytes_d2h"] + 26 * es["blocks_hashed"] + 5 * (es["offloaded"] + es["dropped"])
+                                   + 128 * sum(e["stage_calls"].values())) / K,
+        }
+        line["host_link"] = {
+            "achieved": es["mover_bytes"] / e_mover_s / 1e9 if e_mover_s else 0.0, "unit": "GB/s",
+            "peak_h2d": link["h2d"], "peak_d2h": link["d2h"],
+            "frac": (es["mover_bytes"] / e_mover_s / 1e9) / (0.5 * (link["h2d"] + link["d2h"])) if e_mover_s else 0.0,
+            "peak_kind": "measured: 1 GiB pinned cudaMemcpyAsync per direction, best of 10, this run",
+            "stage_wall_ms_per_step": {k: round(x / K, 4) for k, x in e["stage_ms"].items()},
+        }
+    if not args.skip_cpu and world == 1:
+        n_host_blocks = min(int(args.host_gib * GiB), int(mem_available_bytes() * 0.5)) // W.GEO_8B.block_bytes
+        c = cpu_arm(args, setup, turns, n_ff, min(args.cpu_steps, K), 1, n_hbm_blocks, n_host_blocks)
+        line["cpu_baseline"] = {
+            "value": kv_bytes(c["stats"], c["block_bytes"]) / c["sec"] / 1e9, "unit": "GB/s", "cores": 1,
+            "kind": "oracle",
+            "sample": f"first {min(args.cpu_steps, K)} of the {K} timed calls (after 1 warm-up) with the tier pressure "
+                      f"capped at {CPU_PRESSURE_CAP} blocks (1 GiB each way) per step; whole path incl. payload "
+                      f"memcpy; {c['sec']:.1f} s on one thread",
+            "blocks_hashed_looked_up_per_s": c["stats"]["blocks_hashed"] / c["sec"],
+        }
+    print(json.dumps(line))
+
+
+if __name__ == "__main__":
+    main()

@@ -150,7 +150,9 @@ typedef struct kvt_op {
   uint32_t n_tokens;    /* APPEND / REPLACE: length of the new message (may be 0) */
   uint32_t flags;       /* KVT_OPF_* */
   uint32_t reserved;    /* must be 0 */
-  const uint32_t *tokens; /* APPEND / REPLACE payload: host pointer (copied before return) or device pointer */
+  const uint32_t *tokens; /* APPEND / REPLACE payload: host pointer (pageable memory is copied before return;
+                             pinned memory must stay unchanged until the stream has passed the call) or
+                             device pointer with KVT_OPF_TOKENS_ON_DEVICE */
 } kvt_op;
 
 /* Applies one primitive or runtime event to a context, strictly in program order per context
@@ -281,8 +283,16 @@ typedef struct kvt_stats {
   uint64_t bytes_d2h, bytes_h2d, bytes_d2d;/* payload bytes moved by offload / reload / compact */
   uint64_t table_rebuilds;
   uint64_t tombstones;
+  uint64_t kernel_launches;  /* kernels of this library launched so far */
+  uint64_t mover_launches;   /* with profiling on: mover kernels timed, their device time and payload bytes */
+  uint64_t mover_ns;
+  uint64_t mover_bytes;
 } kvt_stats;
 int32_t kvt_get_stats(kvt_engine *e, kvt_stats *out);
+
+/* Profiling switch (default off). When on, offload / reload / compact bracket their mover kernel with
+ * CUDA events on the call's stream and accumulate its device time in kvt_stats.mover_ns. */
+int32_t kvt_set_profiling(kvt_engine *e, uint32_t on);
 
 /* Text of the last error of this engine (always NUL-terminated). */
 int32_t kvt_last_error(kvt_engine *e, char *buf, uint32_t cap);

@@ -25,7 +25,7 @@ IDS_ON_DEVICE = 1
 EXPORTS = ("kvt_query_sizes", "kvt_create", "kvt_destroy", "kvt_apply_op", "kvt_map_blocks", "kvt_get_block_map",
            "kvt_classify", "kvt_get_states", "kvt_select_victims", "kvt_offload", "kvt_reload", "kvt_release",
            "kvt_compact", "kvt_copy_blocks", "kvt_hash_scratch_bytes", "kvt_hash_tokens", "kvt_get_stats",
-           "kvt_last_error", "kvt_get_entries", "kvt_debug_load_resident")
+           "kvt_last_error", "kvt_get_entries", "kvt_debug_load_resident", "kvt_set_profiling")
 
 
 class KvtError(RuntimeError):
@@ -56,7 +56,8 @@ CALL_INFO_DTYPE = np.dtype([(n, np.uint32) for n in ("n_blocks", "hit_len", "n_h
                                                        "n_admissible", "n_admitted", "n_held")])
 STATS_FIELDS = ("clock", "n_contexts", "occ_hbm", "occ_host", "blocks_hashed", "hits_hbm", "hits_host", "misses",
                 "inserted", "adopted", "dropped", "offloaded", "reloaded", "compacted", "bytes_d2h", "bytes_h2d",
-                "bytes_d2d", "table_rebuilds", "tombstones")
+                "bytes_d2d", "table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns",
+                "mover_bytes")
 
 _lib = None
 
@@ -88,6 +89,7 @@ def load_library():
             "kvt_hash_tokens": [vp, u64, u64, vp, vp, u64, vp],
             "kvt_get_stats": [vp, vp],
             "kvt_last_error": [vp, vp, u32],
+            "kvt_set_profiling": [vp, u32],
             "kvt_get_entries": [vp, u32, vp, vp, vp, vp, u32, vp],
             "kvt_debug_load_resident": [vp, vp, vp, vp, vp, vp, u32, u32, vp],
         }
@@ -136,7 +138,8 @@ class Engine:
     def __init__(self, n_layers, n_kv_heads, head_dim, elem_bytes=2, pool_layout=LAYOUT_LAYER_MAJOR,
                  n_hbm_blocks=128, n_host_blocks=512, max_contexts=64, hash_seed=0, suspended_order=ORDER_MRU,
                  metadata_only=False, table_capacity=None, max_messages=1 << 16, max_batch_blocks=None,
-                 max_tokens=1 << 22, max_key_blocks=None, host_pool_on_device=False, device="cuda"):
+                 max_tokens=1 << 22, max_key_blocks=None, host_pool_on_device=False, zero_pools=True,
+                 device="cuda"):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2609_39819_b200 needs a CUDA device (there is no CPU fallback)")
@@ -175,12 +178,13 @@ class Engine:
         if metadata_only:
             self.hbm_pool = self.host_pool = None
         else:
-            self.hbm_pool = torch.zeros(n_hbm_blocks * self.block_bytes, dtype=torch.uint8, device=self.device)
+            new = torch.zeros if zero_pools else torch.empty
+            self.hbm_pool = new(n_hbm_blocks * self.block_bytes, dtype=torch.uint8, device=self.device)
             nh = max(n_host_blocks, 1) * self.block_bytes
             if host_pool_on_device:   # second tier kept in HBM (in-device measurements)
-                self.host_pool = torch.zeros(nh, dtype=torch.uint8, device=self.device)
+                self.host_pool = new(nh, dtype=torch.uint8, device=self.device)
             else:
-                self.host_pool = torch.zeros(nh, dtype=torch.uint8, pin_memory=True)
+                self.host_pool = new(nh, dtype=torch.uint8, pin_memory=True)
             cfg.hbm_pool, cfg.hbm_pool_bytes = self.hbm_pool.data_ptr(), self.hbm_pool.numel()
             cfg.host_pool, cfg.host_pool_bytes = self.host_pool.data_ptr(), self.host_pool.numel()
         self.cfg = cfg
@@ -205,6 +209,9 @@ class Engine:
         except Exception:
             pass
 
+    def set_profiling(self, on=True):
+        self._check(self.L.kvt_set_profiling(self.h, 1 if on else 0), "set_profiling")
+
     def last_error(self):
         buf = C.create_string_buffer(256)
         self.L.kvt_last_error(self.h, buf, 256)
@@ -219,9 +226,9 @@ class Engine:
         flags, ptr, n = 0, None, 0
         keep = None
         if tokens is not None:
-            if hasattr(tokens, "data_ptr"):      # torch tensor on the device
+            if hasattr(tokens, "data_ptr"):      # torch tensor: device memory, or (pinned) host memory
                 keep = tokens
-                flags, ptr, n = OPF_TOKENS_ON_DEVICE, tokens.data_ptr(), tokens.numel()
+                flags, ptr, n = (OPF_TOKENS_ON_DEVICE if tokens.is_cuda else 0), tokens.data_ptr(), tokens.numel()
             else:
                 keep = _u32(tokens)
                 ptr, n = keep.ctypes.data, len(keep)

@@ -136,6 +136,9 @@ struct kvt_engine {
   u32 *h_status; u8 *h_desc; u32 *h_ctxres; u32 *h_mstart, *h_mend; u8 *h_mrank; u32 *h_ids, *h_ids2;
   cudaEvent_t ev_upload = nullptr;
   bool upload_pending = false;
+  // optional timing of the mover kernel (kvt_set_profiling)
+  bool profiling = false, mover_timed = false;
+  cudaEvent_t ev_m0 = nullptr, ev_m1 = nullptr;
 
   template <class T> T *dp(u64 off) const { return reinterpret_cast<T *>(meta + off); }
   u32 tier_slots(u32 t) const { return t == KVT_TIER_HBM ? cfg.n_hbm_blocks : cfg.n_host_blocks; }
@@ -151,6 +154,13 @@ namespace {
       e->err = std::string(#call) + ": " + cudaGetErrorString(_e);                                 \
       return KVT_E_CUDA;                                                                           \
     }                                                                                              \
+  } while (0)
+
+// every kernel launch of the library goes through this macro, which also counts it
+#define KL(kern, grid, block, stream, ...)                     \
+  do {                                                         \
+    kern<<<(grid), (block), 0, (stream)>>>(__VA_ARGS__);       \
+    e->st.kernel_launches++;                                   \
   } while (0)
 
 int32_t fail(kvt_engine *e, int32_t code, const char *msg) { e->err = msg; return code; }
@@ -218,16 +228,16 @@ int32_t compact_indices(kvt_engine *e, cudaStream_t s, Pred pred, Emit emit, u32
   u32 *tiles = e->dp<u32>(e->L.tiles);
   u32 nt = cdiv(n, SCAN_TILE);
   if (nt == 0) { CU(cudaMemsetAsync(e->d_status + total_word, 0, 4, s)); return KVT_OK; }
-  k_tile_count<<<nt, SCAN_TILE, 0, s>>>(pred, n, tiles);
-  k_scan_tiles<<<1, 1024, 0, s>>>(tiles, nt, e->d_status + total_word);
-  k_tile_scatter<<<nt, SCAN_TILE, 0, s>>>(pred, emit, n, tiles);
+  KL(k_tile_count, nt, SCAN_TILE, s, pred, n, tiles);
+  KL(k_scan_tiles, 1, 1024, s, tiles, nt, e->d_status + total_word);
+  KL(k_tile_scatter, nt, SCAN_TILE, s, pred, emit, n, tiles);
   LAUNCH_CHECK();
   return KVT_OK;
 }
 
 int32_t table_rebuild(kvt_engine *e, cudaStream_t s) {
-  k_table_clear<<<cdiv((u64)e->tab.mask + 1, 256), 256, 0, s>>>(e->tab);
-  k_table_reinsert<<<cdiv(e->ent.n_total, 256), 256, 0, s>>>(e->tab, e->ent, e->d_status);
+  KL(k_table_clear, cdiv((u64)e->tab.mask + 1,256), 256, s, e->tab);
+  KL(k_table_reinsert, cdiv(e->ent.n_total,256), 256, s, e->tab, e->ent, e->d_status);
   LAUNCH_CHECK();
   e->tombs = 0;
   e->st.table_rebuilds++;
@@ -263,9 +273,23 @@ int32_t launch_mover(kvt_engine *e, cudaStream_t s, u32 st, const u32 *src, u32 
   a.n_chunks = (u32)e->n_chunks; a.chunk_bytes = (u32)e->chunk_bytes; a.status = e->d_status;
   u64 items = (u64)n_max * e->n_chunks;
   u32 grid = (u32)std::min<u64>(items, (u64)e->sm_count * 8);
-  k_move_blocks<4><<<grid, 256, 0, s>>>(a);
+  const bool timed = e->profiling && n_dev != nullptr;   // only the calls that synchronise afterwards
+  if (timed) CU(cudaEventRecord(e->ev_m0, s));
+  KL(k_move_blocks<4>, grid, 256, s, a);
+  if (timed) { CU(cudaEventRecord(e->ev_m1, s)); e->mover_timed = true; }
   LAUNCH_CHECK();
   return KVT_OK;
+}
+
+// After the stream has been synchronised: adds the timed mover kernel to the statistics.
+void mover_account(kvt_engine *e, u64 blocks) {
+  if (!e->mover_timed) return;
+  e->mover_timed = false;
+  float ms = 0.f;
+  if (cudaEventElapsedTime(&ms, e->ev_m0, e->ev_m1) != cudaSuccess) return;
+  e->st.mover_launches++;
+  e->st.mover_ns += (u64)((double)ms * 1e6);
+  e->st.mover_bytes += blocks * e->block_bytes;
 }
 
 // ---- classification -------------------------------------------------------------------------------------
@@ -291,7 +315,7 @@ int32_t do_classify(kvt_engine *e, cudaStream_t s) {
     nm += k; nmap += c.valid_blocks;
     hd[nc++] = d;
   }
-  k_rank_reset<<<cdiv(e->ent.n_total, 256), 256, 0, s>>>(e->ent);
+  KL(k_rank_reset, cdiv(e->ent.n_total,256), 256, s, e->ent);
   if (nmap) {
     CU(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nc * sizeof(ClsCtx), cudaMemcpyHostToDevice, s));
     CU(cudaMemcpyAsync(e->dp<u8>(e->L.m_start), e->h_mstart, nm * 4ull, cudaMemcpyHostToDevice, s));
@@ -301,7 +325,7 @@ int32_t do_classify(kvt_engine *e, cudaStream_t s) {
     a.tab = e->tab; a.ent = e->ent; a.keys = e->d_keys; a.ctx = e->dp<ClsCtx>(e->L.desc); a.n_ctx = nc; a.n_map = nmap;
     a.m_start = e->dp<u32>(e->L.m_start); a.m_end = e->dp<u32>(e->L.m_end); a.m_rank = e->dp<u8>(e->L.m_rank);
     a.status = e->d_status;
-    k_classify<<<cdiv(nmap, 256), 256, 0, s>>>(a);
+    KL(k_classify, cdiv(nmap,256), 256, s, a);
     r = stage_release(e, s);
     if (r) return r;
   }
@@ -323,7 +347,7 @@ u64 grow_cap(u64 need) { return round_up(std::max<u64>(need + need / 4, 1024), 6
 
 int32_t unlock_held(kvt_engine *e, Ctx &c, cudaStream_t s, bool stamp) {
   if (c.held && c.keyseg >= 0) {
-    k_unlock<<<cdiv(c.held, 256), 256, 0, s>>>(e->tab, e->ent, e->d_keys + e->segs[c.keyseg].off, c.held, e->now,
+    KL(k_unlock, cdiv(c.held,256), 256, s, e->tab, e->ent, e->d_keys + e->segs[c.keyseg].off, c.held, e->now,
                                                 stamp ? 1u : 0u, e->d_status);
     LAUNCH_CHECK();
   }
@@ -417,12 +441,13 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   e->h_mstart = (u32 *)(e->stage + o_ms); e->h_mend = (u32 *)(e->stage + o_me); e->h_mrank = e->stage + o_mr;
   e->h_ids = (u32 *)(e->stage + o_ids); e->h_ids2 = (u32 *)(e->stage + o_ids2);
   cudaStream_t s = (cudaStream_t)stream;
-  bool ok = cudaEventCreateWithFlags(&e->ev_upload, cudaEventDisableTiming) == cudaSuccess;
+  bool ok = cudaEventCreateWithFlags(&e->ev_upload, cudaEventDisableTiming) == cudaSuccess &&
+            cudaEventCreate(&e->ev_m0) == cudaSuccess && cudaEventCreate(&e->ev_m1) == cudaSuccess;
   // everything except the key arena and scratch must start at zero; the table needs ent = NONE
   ok = ok && cudaMemsetAsync(e->meta + L.e_key, 0, L.keys - L.e_key, s) == cudaSuccess;
   ok = ok && cudaMemsetAsync(e->d_status, 0, ST_WORDS * 4, s) == cudaSuccess;
   if (ok) {
-    k_table_clear<<<cdiv((u64)c.table_capacity, 256), 256, 0, s>>>(e->tab);
+    KL(k_table_clear, cdiv((u64)c.table_capacity,256), 256, s, e->tab);
     ok = cudaGetLastError() == cudaSuccess && cudaStreamSynchronize(s) == cudaSuccess;
   }
   if (!ok) { cudaFreeHost(e->stage); if (e->ev_upload) cudaEventDestroy(e->ev_upload); delete e; return KVT_E_CUDA; }
@@ -434,6 +459,8 @@ int32_t kvt_destroy(kvt_engine *e) {
   if (!e) return KVT_E_INVAL;
   cudaDeviceSynchronize();
   if (e->ev_upload) cudaEventDestroy(e->ev_upload);
+  if (e->ev_m0) cudaEventDestroy(e->ev_m0);
+  if (e->ev_m1) cudaEventDestroy(e->ev_m1);
   if (e->stage) cudaFreeHost(e->stage);
   delete e;
   return KVT_OK;
@@ -442,6 +469,12 @@ int32_t kvt_destroy(kvt_engine *e) {
 int32_t kvt_last_error(kvt_engine *e, char *buf, uint32_t cap) {
   if (!e || !buf || !cap) return KVT_E_INVAL;
   std::snprintf(buf, cap, "%s", e->err.c_str());
+  return KVT_OK;
+}
+
+int32_t kvt_set_profiling(kvt_engine *e, uint32_t on) {
+  if (!e) return KVT_E_INVAL;
+  e->profiling = on != 0;
   return KVT_OK;
 }
 
@@ -650,10 +683,10 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     LockArgs lk;
     lk.ent = e->ent; lk.b_ent = la.b_ent; lk.hit_len = d_res; lk.n_hbm = d_res + C; lk.n_host = d_res + 2 * C;
     lk.now = e->now; lk.status = e->d_status;
-    k_hash_digest<<<chunk_base, CHUNK, 0, s>>>(ha);
-    k_hash_carry<<<cdiv(nd, 128), 128, 0, s>>>(ha);
-    k_hash_finish_lookup<<<chunk_base, CHUNK, 0, s>>>(ha, la);
-    k_lock_hits<<<chunk_base, CHUNK, 0, s>>>(ha, lk);
+    KL(k_hash_digest, chunk_base, CHUNK, s, ha);
+    KL(k_hash_carry, cdiv(nd,128), 128, s, ha);
+    KL(k_hash_finish_lookup, chunk_base, CHUNK, s, ha, la);
+    KL(k_lock_hits, chunk_base, CHUNK, s, ha, lk);
     LAUNCH_CHECK();
     CU(cudaMemcpyAsync(h_hit, d_res, 3ull * C * 4, cudaMemcpyDeviceToHost, s));
     r = status_fetch(e, s);
@@ -728,14 +761,14 @@ static int32_t map_admit(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_info
     rc = status_zero(e, s);
     if (rc) break;
     u32 g = cdiv(n_cand, 256);
-    k_admit_claim<<<g, 256, 0, s>>>(a);
-    k_admit_resolve<<<g, 256, 0, s>>>(a);
+    KL(k_admit_claim, g, 256, s, a);
+    KL(k_admit_resolve, g, 256, s, a);
     rc = compact_indices(e, s, PredOwner{a.flag}, EmitRank{a.krank}, n_cand, ST_NEW);
     if (rc) break;
     rc = compact_indices(e, s, PredFree{e->ent.key, 0}, EmitFree{e->dp<u32>(e->L.freelist), (u32)e->L.LB}, e->cfg.n_hbm_blocks, ST_FREE);
     if (rc) break;
-    k_admit_stop<<<g, 256, 0, s>>>(a);
-    k_admit_apply<<<g, 256, 0, s>>>(a);
+    KL(k_admit_stop, g, 256, s, a);
+    KL(k_admit_apply, g, 256, s, a);
     rc = launch_ok(e);
     if (rc) break;
     CU(cudaMemcpyAsync(h_stop, a.stop, nd * 4, cudaMemcpyDeviceToHost, s));
@@ -796,7 +829,7 @@ int32_t kvt_get_block_map(kvt_engine *e, uint32_t ctx, uint64_t *keys, uint8_t *
   const u64 *dk = e->d_keys + e->segs[c->keyseg].off;
   int32_t r = status_zero(e, s);
   if (r) return r;
-  k_block_map<<<cdiv(nb, 256), 256, 0, s>>>(e->tab, e->ent, dk, nb, e->dp<u8>(e->L.map_tier), e->dp<u32>(e->L.map_slot), e->d_status);
+  KL(k_block_map, cdiv(nb,256), 256, s, e->tab, e->ent, dk, nb, e->dp<u8>(e->L.map_tier), e->dp<u32>(e->L.map_slot), e->d_status);
   LAUNCH_CHECK();
   if (keys) CU(cudaMemcpyAsync(keys, dk, nb * 8ull, cudaMemcpyDeviceToHost, s));
   if (tier) CU(cudaMemcpyAsync(tier, e->dp<u8>(e->L.map_tier), nb, cudaMemcpyDeviceToHost, s));
@@ -821,7 +854,7 @@ int32_t kvt_get_states(kvt_engine *e, uint32_t tier, uint8_t *state, uint32_t ca
   int32_t r = ensure_classified(e, s);
   if (r) return r;
   u8 *d_out = e->dp<u8>(e->L.out_states);
-  k_states_out<<<cdiv(n, 256), 256, 0, s>>>(e->ent, e->tier_e0(tier), n, d_out);
+  KL(k_states_out, cdiv(n,256), 256, s, e->ent, e->tier_e0(tier), n, d_out);
   LAUNCH_CHECK();
   CU(cudaMemcpyAsync(state, d_out, n, cudaMemcpyDeviceToHost, s));
   CU(cudaStreamSynchronize(s));
@@ -861,18 +894,18 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   a.mru = e->cfg.suspended_order == KVT_ORDER_MRU; a.status = e->d_status;
   u64 *kA = e->dp<u64>(e->L.keyA), *kB = e->dp<u64>(e->L.keyB);
   u32 *vA = e->dp<u32>(e->L.valA), *vB = e->dp<u32>(e->L.valB), *counts = e->dp<u32>(e->L.rcounts);
-  k_sel_count<<<cdiv(n, 256), 256, 0, s>>>(a);
+  KL(k_sel_count, cdiv(n,256), 256, s, a);
   r = compact_indices(e, s, PredSel{a}, EmitSel{a, kA, vA}, n, ST_M);
   if (r) return r;
   const u32 key_bits = 2 + a.stamp_bits + a.depth_bits, n_pass = cdiv(key_bits, 8), tiles = cdiv(n, SORT_TILE);
   for (u32 p = 0; p < n_pass; ++p) {
-    k_radix_hist<<<tiles, 256, 0, s>>>(kA, e->d_status, 8 * p, counts);
-    k_radix_scan<<<1, 1024, 0, s>>>(counts, e->d_status);
-    k_radix_scatter<<<tiles, 256, 0, s>>>(kA, vA, kB, vB, e->d_status, 8 * p, counts);
+    KL(k_radix_hist, tiles, 256, s, kA, e->d_status, 8 * p, counts);
+    KL(k_radix_scan, 1, 1024, s, counts, e->d_status);
+    KL(k_radix_scatter, tiles, 256, s, kA, vA, kB, vB, e->d_status, 8 * p, counts);
     std::swap(kA, kB); std::swap(vA, vB);
   }
   u32 n_emit = std::min(n_req, n);
-  k_sel_emit<<<cdiv(n_emit, 256), 256, 0, s>>>(kA, vA, n_emit, a.stamp_bits + a.depth_bits, e->dp<u32>(e->L.out_slots),
+  KL(k_sel_emit, cdiv(n_emit,256), 256, s, kA, vA, n_emit, a.stamp_bits + a.depth_bits, e->dp<u32>(e->L.out_slots),
                                                e->dp<u8>(e->L.out_states));
   LAUNCH_CHECK();
   r = status_fetch(e, s);
@@ -917,7 +950,7 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
   a.pair_src = e->dp<u32>(e->L.pair_src); a.pair_dst = e->dp<u32>(e->L.pair_dst);
   a.allow_inflight = allow_inflight; a.drop_dead = drop_dead; a.drop_all = drop_all; a.status = e->d_status;
   u32 g = cdiv(n, 256);
-  k_list_validate<<<g, 256, 0, s>>>(a);
+  KL(k_list_validate, g, 256, s, a);
   r = compact_indices(e, s, PredLive{a.live}, EmitLive{a.lidx, a.n_free, e->d_status}, n, ST_TOTAL);
   if (r) return r;
   if (!drop_all) {
@@ -925,8 +958,8 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
                         e->tier_slots(dst_tier), ST_FREE);
     if (r) return r;
   }
-  k_list_apply<<<g, 256, 0, s>>>(a);
-  k_list_unmark<<<g, 256, 0, s>>>(a);
+  KL(k_list_apply, g, 256, s, a);
+  KL(k_list_unmark, g, 256, s, a);
   LAUNCH_CHECK();
   if (!drop_all) {
     r = launch_mover(e, s, src_tier, a.pair_src, dst_tier, a.pair_dst, std::min(n, a.n_free), e->d_status + ST_NLIVE);
@@ -938,6 +971,7 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
   if (r) return r;
   *n_live = e->h_status[ST_NLIVE];
   *n_drop = e->h_status[ST_NDROP];
+  mover_account(e, *n_live);
   *n_done = *n_live + *n_drop;
   e->occ[src_tier] -= *n_done;
   if (!drop_all) e->occ[dst_tier] += *n_live;
@@ -988,7 +1022,7 @@ int32_t kvt_compact(kvt_engine *e, uint32_t tier, uint32_t *n_moved, void *strea
   r = compact_indices(e, s, PredMover{e->ent.key, e0, n_occ}, EmitList{src}, n, ST_NMOVED);
   if (r) return r;
   u32 n_max = std::min(n_occ, n - n_occ);
-  k_compact_apply<<<cdiv(n_max, 256), 256, 0, s>>>(e->tab, e->ent, e0, src, dst, e->d_status);
+  KL(k_compact_apply, cdiv(n_max,256), 256, s, e->tab, e->ent, e0, src, dst, e->d_status);
   LAUNCH_CHECK();
   r = launch_mover(e, s, tier, src, tier, dst, n_max, e->d_status + ST_NMOVED);
   if (r) return r;
@@ -998,6 +1032,7 @@ int32_t kvt_compact(kvt_engine *e, uint32_t tier, uint32_t *n_moved, void *strea
   if (r) return r;
   if (e->h_status[ST_AUX] != e->h_status[ST_NMOVED]) return fail(e, KVT_E_DEVICE, "compaction plan mismatch");
   *n_moved = e->h_status[ST_NMOVED];
+  mover_account(e, *n_moved);
   e->st.compacted += *n_moved;
   e->st.bytes_d2d += *n_moved * e->block_bytes;
   return KVT_OK;
@@ -1087,8 +1122,8 @@ int32_t kvt_debug_load_resident(kvt_engine *e, const uint64_t *keys, const uint8
   LoadArgs a;
   a.tab = e->tab; a.ent = e->ent; a.keys = dk; a.state = dst_state; a.stamp = dsp; a.depth = ddp; a.slot = dsl;
   a.n = n; a.e0 = e->tier_e0(tier); a.n_slots = ns; a.status = e->d_status;
-  k_load_check<<<cdiv(n, 256), 256, 0, s>>>(a);
-  k_load_apply<<<cdiv(n, 256), 256, 0, s>>>(a);
+  KL(k_load_check, cdiv(n,256), 256, s, a);
+  KL(k_load_apply, cdiv(n,256), 256, s, a);
   LAUNCH_CHECK();
   r = status_fetch(e, s);
   if (r) return r;

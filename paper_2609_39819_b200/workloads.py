@@ -21,6 +21,7 @@ VOCAB = 151552
 TIER_HBM, TIER_HOST, TIER_NONE = 0, 1, 0xFF
 MAP_LOOKUP, MAP_ADMIT = 0, 1
 GiB = 1 << 30
+GPU_ONLY_STATS = ("table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns", "mover_bytes")
 
 
 # ------------------------------------------------------------------------------------------------
@@ -286,6 +287,26 @@ class ReplayOptions:
     counters: dict = field(default_factory=dict)
 
 
+def evict(eng, n):
+    """Frees n HBM slots in the engine's victim order: dead blocks are dropped, live ones go to the
+    host tier, for which room is made first by releasing the host tier's own first victims."""
+    rec = {}
+    victims, vstates = eng.select_victims(TIER_HBM, n)
+    rec["victims"] = victims.copy()
+    rec["vstates"] = vstates.copy()
+    n_live = int((vstates > 0).sum())
+    free_host = eng.n_host_blocks - eng.get_stats()["occ_host"]
+    if n_live > free_host:
+        hv, hs = eng.select_victims(TIER_HOST, n_live - free_host)
+        rec["host_victims"] = hv.copy()
+        rec["host_vstates"] = hs.copy()
+        if len(hv):
+            eng.release(TIER_HOST, hv)
+    if len(victims):
+        rec["offload"] = eng.offload(victims)
+    return rec
+
+
 def run_call(eng, ctxs, opt: ReplayOptions):
     """One LLM call per listed context through the cache path: lookup, make room following
     Algorithm 1's release order (victims come from the engine), reload host hits, admit, write the
@@ -297,19 +318,7 @@ def run_call(eng, ctxs, opt: ReplayOptions):
     free_hbm = eng.n_hbm_blocks - st["occ_hbm"]
     need = int(info["n_hit_host"].sum()) + int(info["n_admissible"].sum()) - free_hbm
     if need > 0:
-        victims, vstates = eng.select_victims(TIER_HBM, need)
-        rec["victims"] = victims.copy()
-        rec["vstates"] = vstates.copy()
-        n_live = int((vstates > 0).sum())
-        free_host = eng.n_host_blocks - st["occ_host"]
-        if n_live > free_host:
-            hv, hs = eng.select_victims(TIER_HOST, n_live - free_host)
-            rec["host_victims"] = hv.copy()
-            rec["host_vstates"] = hs.copy()
-            if len(hv):
-                eng.release(TIER_HOST, hv)
-        if len(victims):
-            rec["offload"] = eng.offload(victims)
+        rec.update(evict(eng, need))
     host_slots = []
     for c, inf in zip(ctxs, info):
         if inf["n_hit_host"]:
@@ -337,7 +346,7 @@ def run_call(eng, ctxs, opt: ReplayOptions):
     if opt.record_states:
         rec["states"] = [eng.get_states(TIER_HBM).copy(), eng.get_states(TIER_HOST).copy()]
         rec["entries"] = [eng.get_entries(TIER_HBM), eng.get_entries(TIER_HOST)]
-    rec["stats"] = {k: v for k, v in eng.get_stats().items() if k not in ("table_rebuilds", "tombstones")}
+    rec["stats"] = {k: v for k, v in eng.get_stats().items() if k not in GPU_ONLY_STATS}
     if opt.payload is not None and opt.verify_payload_every and opt.counters["calls"] % opt.verify_payload_every == 0:
         rec["payload_ok"] = verify_payload(eng, opt.payload)
     return rec

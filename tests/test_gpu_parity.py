@@ -84,7 +84,7 @@ def _replay_pair(gpu, cpu, trace, payload, check_pools=True, record_states=True,
                 assert rg["payload_ok"] and rc["payload_ok"]
     sg, sc = gpu.get_stats(), cpu.get_stats()
     for k in sc:
-        if k not in ("table_rebuilds", "tombstones"):
+        if k not in W.GPU_ONLY_STATS:
             assert sg[k] == sc[k], k
     if check_pools and payload is not None:
         for tier, n in ((0, gpu.n_hbm_blocks), (1, gpu.n_host_blocks)):
@@ -122,21 +122,25 @@ def test_scaled_c2_trace_parity(B, oracle):
 
 def test_scaled_c3_trace_parity(B, oracle):
     trace, n_ctx = W.trace_c3(1, n_sessions=8, scale=1 / 32)
-    kw = dict(n_hbm_blocks=1024, n_host_blocks=1024, max_contexts=n_ctx, **W.GEO_TOY.kwargs())
+    kw = dict(n_hbm_blocks=384, n_host_blocks=512, max_contexts=n_ctx, **W.GEO_TOY.kwargs())
     gpu = B.Engine(max_tokens=1 << 20, max_messages=1 << 15, **kw)
     cpu = oracle.OracleEngine(**kw)
     _replay_pair(gpu, cpu, trace, W.payload_pattern, record_states=True)
     assert cpu.get_stats()["offloaded"] > 0 and cpu.get_stats()["reloaded"] > 0
 
 
-def test_full_length_c2_session_metadata_parity(B, oracle):
+@pytest.mark.parametrize("n_hbm", [20480, 6144])
+def test_full_length_c2_session_metadata_parity(B, oracle, n_hbm):
     """One 128K-token ReAct session (C2's trace at full size) on a metadata-only engine with C2's
-    block counts: every lookup, victim list, admission and state vector equals the oracle's."""
-    kw = dict(n_hbm_blocks=20480, n_host_blocks=61440, max_contexts=4, metadata_only=True, **W.GEO_8B.kwargs())
+    block counts (40 GiB pool, and the 12 GiB pressure variant): every lookup, victim list,
+    admission and state vector equals the oracle's."""
+    kw = dict(n_hbm_blocks=n_hbm, n_host_blocks=61440, max_contexts=4, metadata_only=True, **W.GEO_8B.kwargs())
     gpu = B.Engine(max_tokens=1 << 20, max_messages=1 << 12, **kw)
     cpu = oracle.OracleEngine(**kw)
     n = _replay_pair(gpu, cpu, W.trace_c2(1), None, record_states=True)
-    assert n >= 30 and cpu.get_stats()["dropped"] > 0
+    assert n >= 30
+    if n_hbm < 20480:
+        assert cpu.get_stats()["dropped"] > 0
 
 
 # ---- C4: metadata stress at full size -------------------------------------------------------------------
@@ -192,7 +196,7 @@ def test_c4_lookup_and_select_parity(B, oracle, n_resident, chain_blocks, n_call
     assert np.array_equal(gpu.get_states(0), cpu.get_states(0))
     sg, sc = gpu.get_stats(), cpu.get_stats()
     for k in sc:
-        if k not in ("table_rebuilds", "tombstones"):
+        if k not in W.GPU_ONLY_STATS:
             assert sg[k] == sc[k], k
 
 
