@@ -342,7 +342,9 @@ def gpu_arm(args, torch, B, setup, turns, n_ff, e2e, n_host_blocks, n_hbm_blocks
     res = dict(ms=ms, stats=d, stage_ms=dict(timer.ms), stage_calls=dict(timer.calls), timers=timers,
                verified=(n_ok, n_seen), tok_bytes=tok_bytes, block_bytes=eng.block_bytes)
     eng.close()
-    del eng, pool, cache
+    del eng, pool, cache, base, timer
+    import gc
+    gc.collect()
     torch.cuda.empty_cache()
     return res
 

@@ -202,6 +202,7 @@ class Engine:
         if getattr(self, "h", None):
             self.L.kvt_destroy(self.h)
             self.h = None
+            self.hbm_pool = self.host_pool = self.meta = self.tokens = None   # release the memory
 
     def __del__(self):
         try:
