@@ -1,0 +1,68 @@
+"""Small, self-terminating cases of one kernel family each, sized for a profiler capture (inputs
+larger than L2, a few GB on the device at most, a handful of launches).
+
+    python -m paper_2609_39819_b200.profile_case mover      # paged KV mover, 8B-class blocks, HBM -> HBM
+    python -m paper_2609_39819_b200.profile_case mover_toy  # the same with 16 KiB blocks (4 KiB chunks)
+    python -m paper_2609_39819_b200.profile_case lookup     # hash + table lookup of 16 x 16,128-block calls
+    python -m paper_2609_39819_b200.profile_case select     # classify + select 10% of 1 Mi resident blocks
+Each prints one line with CUDA-event timings of its launches.
+"""
+from __future__ import annotations
+
+import sys
+
+import numpy as np
+
+
+def _events(torch, fn, n):
+    out = []
+    for _ in range(n):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); fn(); b.record(); torch.cuda.synchronize()
+        out.append(round(a.elapsed_time(b), 4))
+    return out
+
+
+def main(case: str):
+    import torch
+    from . import binding as B, workloads as W
+    torch.cuda.set_device(0)
+    if case in ("mover", "mover_toy"):
+        geo, n_slots, n = (W.GEO_8B, 1536, 1024) if case == "mover" else (W.GEO_TOY, 196608, 131072)
+        eng = B.Engine(n_hbm_blocks=n_slots, n_host_blocks=n_slots, max_contexts=2, max_tokens=1 << 12, max_messages=64,
+                       max_batch_blocks=max(n, 4096), host_pool_on_device=True, zero_pools=False, **geo.kwargs())
+        src = torch.from_numpy(W.ids_c5(1, n, n_slots, True).view(np.int32)).cuda()
+        dst = torch.from_numpy(W.ids_c5(2, n, n_slots, True).view(np.int32)).cuda()
+        ms = _events(torch, lambda: eng.copy_blocks(0, src, 1, dst), 3)
+        gb = n * geo.block_bytes / 1e9
+        print(f"{case}: {n} blocks x {geo.block_bytes} B, permuted ids, ms per launch {ms}, "
+              f"read+write GB/s {[round(2 * gb / (m / 1e3), 1) for m in ms]}")
+    elif case in ("lookup", "select"):
+        n_res, n_calls = (1 << 18, 16) if case == "lookup" else (1 << 20, 4)
+        inp = W.inputs_c4(1, n_resident=n_res, chain_blocks=16128, n_calls=n_calls)
+        eng = B.Engine(n_hbm_blocks=n_res, n_host_blocks=0, max_contexts=n_calls + 1, metadata_only=True,
+                       max_tokens=(n_calls + 2) * 16128 * 16 * 2, max_messages=1024, max_batch_blocks=n_calls * 16128,
+                       **W.GEO_TOY.kwargs())
+        keys = np.concatenate([B.hash_tokens(torch.from_numpy(c.view(np.int32)).cuda()).cpu().numpy().view(np.uint64)
+                               for c in inp.chain_tokens])
+        eng.debug_load_resident(keys, inp.state, inp.stamp, inp.depth, inp.slot, 0)
+        for i, t in enumerate(inp.calls):
+            eng.spawn(i)
+            eng.append(i, torch.from_numpy(t.view(np.int32)).cuda())
+        if case == "lookup":
+            ms = []
+            for _ in range(3):
+                ms += _events(torch, lambda: eng.map_blocks(list(range(n_calls)), 0), 1)
+                for c in range(n_calls):
+                    eng.prefill_done(c)
+            print(f"lookup: {n_calls} calls x 16128 blocks against {n_res} resident, ms per batch {ms}, "
+                  f"blocks/s {[round(n_calls * 16128 / (m / 1e3)) for m in ms]}")
+        else:
+            ms = _events(torch, lambda: eng.select_victims(0, n_res // 10), 3)
+            print(f"select: {n_res // 10} victims of {n_res} resident, ms per call {ms}")
+    else:
+        raise SystemExit(__doc__)
+
+
+if __name__ == "__main__":
+    main(sys.argv[1] if len(sys.argv) > 1 else "")
