@@ -269,6 +269,26 @@ uint64_t kvt_hash_scratch_bytes(uint64_t n_tokens);
 int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t hash_seed,
                         uint64_t *d_keys, void *d_scratch, uint64_t scratch_bytes, void *stream);
 
+/* Hasher variant for callers that cannot allocate. The paper has no counterpart for this call; it
+ * exists for integrations that are handed a fixed memory budget and may not call cudaMalloc (or any
+ * allocating library routine) at all: a plug-in living inside a serving engine whose allocator owns
+ * every byte of the device, or a request loop in which an allocation would stall the whole device.
+ * Same result as kvt_hash_tokens, but the per-chunk scratch is a fixed array inside the library
+ * instead of a caller buffer, so the call allocates nothing, on the host or on the device.
+ *   - d_tokens (16-byte aligned) and d_keys are device pointers supplied by the caller, as before.
+ *   - Limit: n_tokens <= KVT_HASH_NOALLOC_MAX_TOKENS; larger inputs are rejected with KVT_E_NOSPACE
+ *     and nothing is launched. The scratch array takes 16 KiB of device memory on every GPU that
+ *     loads the library, until the process exits.
+ *   - The first call on each device looks up the array's device address (no allocation, but a
+ *     runtime query): make that first call outside any stream capture.
+ *   - All calls share the one array. Nothing in it has to start at zero (each call overwrites what it
+ *     later reads), but two calls whose kernels overlap on the GPU (different streams, or different
+ *     host threads) race on it: keep calls on one device ordered.
+ * Asynchronous on `stream`. */
+#define KVT_HASH_NOALLOC_MAX_TOKENS (1ull << 22)
+int32_t kvt_hash_tokens_noalloc(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t hash_seed,
+                                uint64_t *d_keys, void *stream);
+
 /* ---- introspection ------------------------------------------------------------------------------ */
 typedef struct kvt_stats {
   uint64_t clock;            /* logical clock */

@@ -25,7 +25,8 @@ IDS_ON_DEVICE = 1
 EXPORTS = ("kvt_query_sizes", "kvt_create", "kvt_destroy", "kvt_apply_op", "kvt_map_blocks", "kvt_get_block_map",
            "kvt_classify", "kvt_get_states", "kvt_select_victims", "kvt_offload", "kvt_reload", "kvt_release",
            "kvt_compact", "kvt_copy_blocks", "kvt_hash_scratch_bytes", "kvt_hash_tokens", "kvt_get_stats",
-           "kvt_last_error", "kvt_get_entries", "kvt_debug_load_resident", "kvt_set_profiling")
+           "kvt_last_error", "kvt_get_entries", "kvt_debug_load_resident", "kvt_set_profiling",
+           "kvt_hash_tokens_noalloc")
 
 
 class KvtError(RuntimeError):
@@ -87,6 +88,7 @@ def load_library():
             "kvt_compact": [vp, u32, vp, vp],
             "kvt_copy_blocks": [vp, u32, vp, u32, vp, u32, u32, vp],
             "kvt_hash_tokens": [vp, u64, u64, vp, vp, u64, vp],
+            "kvt_hash_tokens_noalloc": [vp, u64, u64, vp, vp],
             "kvt_get_stats": [vp, vp],
             "kvt_last_error": [vp, vp, u32],
             "kvt_set_profiling": [vp, u32],
@@ -129,6 +131,17 @@ def hash_tokens(tokens_dev, seed: int = 0):
     if rc:
         raise KvtError(rc, "hash_tokens")
     return keys
+
+
+HASH_NOALLOC_MAX_TOKENS = 1 << 22
+
+
+def hash_tokens_noalloc(tokens_dev, keys_out, seed: int = 0) -> int:
+    """Block keys of a device token tensor written into the caller's `keys_out` (int64, >= n // 16
+    elements) with the library's built-in scratch: for callers that must not allocate. Returns the
+    status code (KVT_E_NOSPACE beyond HASH_NOALLOC_MAX_TOKENS)."""
+    lib = load_library()
+    return lib.kvt_hash_tokens_noalloc(tokens_dev.data_ptr(), tokens_dev.numel(), seed, keys_out.data_ptr(), _stream())
 
 
 class Engine:

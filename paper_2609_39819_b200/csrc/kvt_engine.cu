@@ -1085,6 +1085,40 @@ int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t ha
   return cudaGetLastError() == cudaSuccess ? KVT_OK : KVT_E_CUDA;
 }
 
+// ---- hasher without allocation ------------------------------------------------------------------------------
+// Scratch of the no-allocation hasher: chunk aggregates followed by chunk carries. File-scope device
+// memory: in host code this name is only a handle, so its device address is queried once per device
+// below and that pointer is what the kernels get.
+constexpr u64 NOALLOC_MAX_CHUNKS = KVT_HASH_NOALLOC_MAX_TOKENS / 16 / CHUNK;
+static __device__ __align__(256) unsigned long long g_noalloc_scratch[2 * NOALLOC_MAX_CHUNKS];
+static u64 *g_noalloc_ptr[64] = {};   // per device ordinal
+
+int32_t kvt_hash_tokens_noalloc(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t hash_seed, uint64_t *d_keys,
+                                void *stream) {
+  if (n_tokens > KVT_HASH_NOALLOC_MAX_TOKENS) return KVT_E_NOSPACE;   // beyond the built-in scratch
+  u64 nb = n_tokens / 16;
+  if (nb == 0) return KVT_OK;
+  if (!d_tokens || !d_keys || ((uintptr_t)d_tokens & 15)) return KVT_E_INVAL;
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return KVT_E_CUDA;
+  if (!g_noalloc_ptr[dev]) {   // first call on this device: resolve the array's device address
+    void *p = nullptr;
+    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return KVT_E_CUDA;
+    g_noalloc_ptr[dev] = (u64 *)p;
+  }
+  cudaStream_t s = (cudaStream_t)stream;
+  u32 n_chunks = cdiv(nb, CHUNK);
+  HashArgs ha;
+  ha.tokens = d_tokens; ha.keys = d_keys; ha.ctx = nullptr; ha.n_ctx = 1;
+  ha.single = HashCtx{0, 0, (u32)nb, 0, 0, 0};
+  ha.agg = g_noalloc_ptr[dev]; ha.carry = g_noalloc_ptr[dev] + NOALLOC_MAX_CHUNKS; ha.h0 = hash_h0(hash_seed);
+  LookupArgs la{};
+  k_hash_digest<<<n_chunks, CHUNK, 0, s>>>(ha);
+  k_hash_carry<<<1, 32, 0, s>>>(ha);
+  k_hash_finish_lookup<<<n_chunks, CHUNK, 0, s>>>(ha, la);
+  return cudaGetLastError() == cudaSuccess ? KVT_OK : KVT_E_CUDA;
+}
+
 // ---- debug loader -------------------------------------------------------------------------------------------
 int32_t kvt_debug_load_resident(kvt_engine *e, const uint64_t *keys, const uint8_t *state, const uint32_t *stamp,
                                 const uint32_t *depth, const uint32_t *slot, uint32_t tier, uint32_t n, void *stream) {
