@@ -384,6 +384,21 @@ def cpu_arm(args, setup, turns, n_ff, n_steps, n_warm, n_hbm_blocks, n_host_bloc
     return dict(sec=sec, stats=d, block_bytes=eng.block_bytes)
 
 
+def reduce_over_ranks(local, dist=None, device="cpu"):
+    """Whole-job figures from per-rank ones: 'ms' is the maximum over ranks (the job is as slow as its
+    slowest rank), every other entry is summed (units processed by all ranks). Ranks are independent
+    sessions; this is the only communication of a multi-GPU run and it happens outside the timed region."""
+    if dist is None:
+        return dict(local)
+    import torch
+    keys = sorted(local)
+    t = torch.tensor([float(local[k]) for k in keys], dtype=torch.float64, device=device)
+    mx = t.clone()
+    dist.all_reduce(t, op=dist.ReduceOp.SUM)
+    dist.all_reduce(mx, op=dist.ReduceOp.MAX)
+    return {k: (mx[i].item() if k == "ms" else t[i].item()) for i, k in enumerate(keys)}
+
+
 def kv_bytes(d, block_bytes):
     return (d["offloaded"] + d["reloaded"]) * block_bytes
 
@@ -456,28 +471,16 @@ def main():
         host_blocks = max(budget // W.GEO_8B.block_bytes, 9000)
         e = gpu_arm(args, torch, B, setup, turns, n_ff, True, host_blocks, n_hbm_blocks, rank, world, barrier)
 
-    def agg(x, op):
-        if world == 1:
-            return x
-        import torch.distributed as dist
-        t = torch.tensor([float(x)], dtype=torch.float64, device="cuda")
-        dist.all_reduce(t, op=op)
-        return t.item()
-
     vbytes = kv_bytes(v["stats"], v["block_bytes"])
+    dist = None
     if world > 1:
         import torch.distributed as dist
-        ms = agg(v["ms"], dist.ReduceOp.MAX)
-        tot_bytes = agg(vbytes, dist.ReduceOp.SUM)
-        tot_hashed = agg(v["stats"]["blocks_hashed"], dist.ReduceOp.SUM)
-        launches = agg(v["stats"]["kernel_launches"], dist.ReduceOp.SUM)
-        if e:
-            e_ms = agg(e["ms"], dist.ReduceOp.MAX)
-            e_bytes = agg(kv_bytes(e["stats"], e["block_bytes"]), dist.ReduceOp.SUM)
-    else:
-        ms, tot_bytes, tot_hashed, launches = v["ms"], vbytes, v["stats"]["blocks_hashed"], v["stats"]["kernel_launches"]
-        if e:
-            e_ms, e_bytes = e["ms"], kv_bytes(e["stats"], e["block_bytes"])
+    tot = reduce_over_ranks({"ms": v["ms"], "bytes": vbytes, "hashed": v["stats"]["blocks_hashed"],
+                             "launches": v["stats"]["kernel_launches"]}, dist, "cuda")
+    ms, tot_bytes, tot_hashed, launches = tot["ms"], tot["bytes"], tot["hashed"], tot["launches"]
+    if e:
+        te = reduce_over_ranks({"ms": e["ms"], "bytes": kv_bytes(e["stats"], e["block_bytes"])}, dist, "cuda")
+        e_ms, e_bytes = te["ms"], te["bytes"]
     if rank != 0:
         return
 
