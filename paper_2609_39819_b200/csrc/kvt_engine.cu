@@ -100,7 +100,7 @@ DevLayout make_layout(const kvt_config &c) {
   L.ctxres = take(C * 16);
   L.m_start = take(Mm * 4); L.m_end = take(Mm * 4); L.m_rank = take(Mm);
   L.keyA = take(Nt * 8); L.keyB = take(Nt * 8); L.valA = take(Nt * 4); L.valB = take(Nt * 4);
-  L.rcounts = take(256ull * (Nt / SORT_TILE + 1) * 4);
+  L.rcounts = take((256ull * (Nt / SORT_TILE + 1) + 256) * 4);
   L.out_slots = take(Nt * 4); L.out_states = take(Nt);
   L.map_tier = take(B); L.map_slot = take(B * 4);
   L.total = off;
@@ -138,6 +138,7 @@ struct kvt_engine {
   bool upload_pending = false;
   // optional timing of the mover kernel (kvt_set_profiling)
   bool profiling = false, mover_timed = false;
+  u32 mover_variant = 0;   // 0 auto, 1 CTA per chunk, 2 warp per 4 KiB tile
   cudaEvent_t ev_m0 = nullptr, ev_m1 = nullptr;
 
   template <class T> T *dp(u64 off) const { return reinterpret_cast<T *>(meta + off); }
@@ -275,7 +276,18 @@ int32_t launch_mover(kvt_engine *e, cudaStream_t s, u32 st, const u32 *src, u32 
   u32 grid = (u32)std::min<u64>(items, (u64)e->sm_count * 8);
   const bool timed = e->profiling && n_dev != nullptr;   // only the calls that synchronise afterwards
   if (timed) CU(cudaEventRecord(e->ev_m0, s));
-  KL(k_move_blocks<4>, grid, 256, s, a);
+  // a warp per 4 KiB tile keeps 8 loads per lane in flight whatever the chunk size (measured faster for
+  // 4 KiB and 32 KiB chunks alike); chunks that are not a multiple of 4 KiB take the CTA-per-chunk kernel
+  const bool tiles_ok = e->chunk_bytes % 4096 == 0;
+  const bool use_tiles = e->mover_variant != 1;
+  if (use_tiles && tiles_ok) {
+    u32 tpc = (u32)(e->chunk_bytes / 4096);
+    u64 titems = items * tpc;
+    u32 tgrid = (u32)std::min<u64>((titems + 7) / 8, (u64)e->sm_count * 8);
+    KL(k_move_tiles<8>, tgrid, 256, s, a, tpc);
+  } else {
+    KL(k_move_blocks<4>, grid, 256, s, a);
+  }
   if (timed) { CU(cudaEventRecord(e->ev_m1, s)); e->mover_timed = true; }
   LAUNCH_CHECK();
   return KVT_OK;
@@ -475,6 +487,12 @@ int32_t kvt_last_error(kvt_engine *e, char *buf, uint32_t cap) {
 int32_t kvt_set_profiling(kvt_engine *e, uint32_t on) {
   if (!e) return KVT_E_INVAL;
   e->profiling = on != 0;
+  return KVT_OK;
+}
+
+int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant) {
+  if (!e || variant > 2) return KVT_E_INVAL;
+  e->mover_variant = variant;
   return KVT_OK;
 }
 
@@ -684,7 +702,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     lk.ent = e->ent; lk.b_ent = la.b_ent; lk.hit_len = d_res; lk.n_hbm = d_res + C; lk.n_host = d_res + 2 * C;
     lk.now = e->now; lk.status = e->d_status;
     KL(k_hash_digest, chunk_base, CHUNK, s, ha);
-    KL(k_hash_carry, cdiv(nd,128), 128, s, ha);
+    KL(k_hash_carry, cdiv((u64)nd * 32, 128), 128, s, ha);
     KL(k_hash_finish_lookup, chunk_base, CHUNK, s, ha, la);
     KL(k_lock_hits, chunk_base, CHUNK, s, ha, lk);
     LAUNCH_CHECK();
@@ -894,14 +912,15 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   a.mru = e->cfg.suspended_order == KVT_ORDER_MRU; a.status = e->d_status;
   u64 *kA = e->dp<u64>(e->L.keyA), *kB = e->dp<u64>(e->L.keyB);
   u32 *vA = e->dp<u32>(e->L.valA), *vB = e->dp<u32>(e->L.valB), *counts = e->dp<u32>(e->L.rcounts);
+  u32 *row_total = counts + 256ull * (e->L.Nt / SORT_TILE + 1);
   KL(k_sel_count, cdiv(n,256), 256, s, a);
   r = compact_indices(e, s, PredSel{a}, EmitSel{a, kA, vA}, n, ST_M);
   if (r) return r;
   const u32 key_bits = 2 + a.stamp_bits + a.depth_bits, n_pass = cdiv(key_bits, 8), tiles = cdiv(n, SORT_TILE);
   for (u32 p = 0; p < n_pass; ++p) {
     KL(k_radix_hist, tiles, 256, s, kA, e->d_status, 8 * p, counts);
-    KL(k_radix_scan, 1, 1024, s, counts, e->d_status);
-    KL(k_radix_scatter, tiles, 256, s, kA, vA, kB, vB, e->d_status, 8 * p, counts);
+    KL(k_radix_scan, 32, 256, s, counts, row_total, e->d_status);
+    KL(k_radix_scatter, tiles, 256, s, kA, vA, kB, vB, e->d_status, 8 * p, counts, row_total);
     std::swap(kA, kB); std::swap(vA, vB);
   }
   u32 n_emit = std::min(n_req, n);

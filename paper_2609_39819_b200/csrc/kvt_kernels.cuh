@@ -46,11 +46,19 @@ constexpr u64 HASH_P = mix64(GOLD * 17ull) | 1ull;
 __host__ __device__ constexpr u64 lane_mult(u32 t) { return mix64(GOLD * (u64)(t + 1)) | 1ull; }
 __host__ __device__ constexpr u64 hash_h0(u64 seed) { return mix64(seed ^ (GOLD * 18ull)); }
 
-__host__ __device__ __forceinline__ u64 pow_p(u32 e) {
-  u64 r = 1, b = HASH_P;
+__host__ __device__ __forceinline__ u64 pow_u64(u64 b, u32 e) {
+  u64 r = 1;
   while (e) { if (e & 1) r *= b; b *= b; e >>= 1; }
   return r;
 }
+__host__ __device__ __forceinline__ u64 pow_p(u32 e) { return pow_u64(HASH_P, e); }
+
+// P^0 .. P^CHUNK, constant-initialised at compile time (2 KiB, L1-resident).
+struct PowTable {
+  u64 v[CHUNK + 1];
+  constexpr PowTable() : v() { u64 p = 1; for (u32 i = 0; i <= CHUNK; ++i) { v[i] = p; p *= HASH_P; } }
+};
+__device__ const PowTable g_pow_p = PowTable();
 
 // ---- device views -------------------------------------------------------------------------------------
 struct Table { TSlot *slots; u32 mask; u32 shift; };   // capacity = mask + 1, home = key >> shift
@@ -99,7 +107,7 @@ __device__ __forceinline__ u32 tab_find_or_claim(const Table &t, u64 key, u32 *s
 // K1: block hasher. 3 phases, no inter-CTA waits:
 //   digest : per 256-block chunk, 4 lanes per block read 16 B each, weighted sums, mix, then a CTA-wide
 //            scan of the affine chain with zero carry-in -> partial chain values + chunk aggregate
-//   carry  : one thread per context walks its chunk aggregates (<= 63 steps for a 258K-token call)
+//   carry  : one warp per context scans its chunk aggregates, 32 chunks per step
 //   finish : h = P^(i+1) * carry + partial, key = mix64(h); fused with the table probe
 // ======================================================================================================
 struct HashCtx { u64 tok_off; u64 key_off; u32 n_blocks; u32 chunk_base; u32 blk_base; u32 pad; };
@@ -157,22 +165,37 @@ __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   u64 carry = 0;  // chain value at the end of the previous warp, with zero chunk carry-in
   const u64 p32 = pp;  // after 5 squarings pp = P^32
   for (u32 w = 0; w < warp; ++w) carry = p32 * carry + wagg[w];
-  cval += pow_p(lane + 1) * carry;
+  cval += g_pow_p.v[lane + 1] * carry;
   if (tid < nb) a.keys[c.key_off + b0 + tid] = cval;
   if (tid == nb - 1) a.agg[blockIdx.x] = cval;
 }
 
-__global__ void k_hash_carry(HashArgs a) {
-  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+// One warp per context: the chain value entering chunk j is A^j * H0 + sum_{i<j} A^(j-1-i) * agg_i with
+// A = P^CHUNK (every chunk before the last is full), evaluated 32 chunks at a time by a warp scan.
+__global__ void __launch_bounds__(128) k_hash_carry(HashArgs a) {
+  const u32 lane = threadIdx.x & 31;
+  const u32 i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
   if (i >= a.n_ctx) return;
   const HashCtx c = a.ctx ? a.ctx[i] : a.single;
+  const u32 n_chunks = (c.n_blocks + CHUNK - 1) / CHUNK;
+  const u64 A = g_pow_p.v[CHUNK];
+  const u64 a_lane = pow_u64(A, lane + 1);
   u64 carry = a.h0;
-  const u64 pfull = pow_p(CHUNK);
-  u32 n_chunks = (c.n_blocks + CHUNK - 1) / CHUNK;
-  for (u32 j = 0; j < n_chunks; ++j) {
-    a.carry[c.chunk_base + j] = carry;
-    u32 len = min(CHUNK, c.n_blocks - j * CHUNK);
-    carry = (len == CHUNK ? pfull : pow_p(len)) * carry + a.agg[c.chunk_base + j];
+  for (u32 j0 = 0; j0 < n_chunks; j0 += 32) {
+    const u32 j = j0 + lane;
+    u64 x = j < n_chunks ? a.agg[c.chunk_base + j] : 0;
+    u64 pp = A;
+#pragma unroll
+    for (u32 o = 1; o < 32; o <<= 1) {
+      u64 up = __shfl_up_sync(0xFFFFFFFFu, x, o);
+      if (lane >= o) x += pp * up;
+      pp *= pp;
+    }
+    const u64 v = a_lane * carry + x;                       // chain value after chunk j
+    u64 in = __shfl_up_sync(0xFFFFFFFFu, v, 1);
+    if (lane == 0) in = carry;
+    if (j < n_chunks) a.carry[c.chunk_base + j] = in;
+    carry = __shfl_sync(0xFFFFFFFFu, v, 31);
   }
 }
 
@@ -193,7 +216,7 @@ __global__ void __launch_bounds__(CHUNK) k_hash_finish_lookup(HashArgs a, Lookup
   if (tid == 0) s_min = 0xFFFFFFFFu;
   __syncthreads();
   if (tid < nb) {
-    u64 h = pow_p(tid + 1) * a.carry[blockIdx.x] + a.keys[c.key_off + b0 + tid];
+    u64 h = g_pow_p.v[tid + 1] * a.carry[blockIdx.x] + a.keys[c.key_off + b0 + tid];
     u64 key = mix64(h);
     if (key < 2) key += 2;
     a.keys[c.key_off + b0 + tid] = key;
@@ -378,12 +401,24 @@ struct EmitRank { u32 *krank; __device__ void operator()(u32 g, u32 r) const { k
 // A3: a context stops at its first candidate that cannot be held (the pool ran out of free slots).
 __global__ void k_admit_stop(AdmitArgs a) {
   u32 g = blockIdx.x * blockDim.x + threadIdx.x;
-  if (g >= a.n_cand) return;
-  const AdmitCtx c = a.ctx[admit_ctx_of(a, g)];
-  u32 f = a.flag[g];
-  bool ok = f == CAND_OLD || (f == CAND_OWNER && a.krank[g] < a.n_free) ||
-            (f == CAND_DUP && a.krank[a.aux[g]] < a.n_free);
-  if (!ok) atomicMin(&a.stop[c.res], c.b_start + (g - c.cand_base));
+  u32 ci = 0xFFFFFFFFu, bad = 0xFFFFFFFFu;
+  if (g < a.n_cand) {
+    ci = admit_ctx_of(a, g);
+    const AdmitCtx c = a.ctx[ci];
+    u32 f = a.flag[g];
+    bool ok = f == CAND_OLD || (f == CAND_OWNER && a.krank[g] < a.n_free) ||
+              (f == CAND_DUP && a.krank[a.aux[g]] < a.n_free);
+    if (!ok) bad = c.b_start + (g - c.cand_base);
+    ci = c.res;
+  }
+  // one atomic per warp when the whole warp belongs to one context (the common case)
+  u32 first = __shfl_sync(0xFFFFFFFFu, ci, 0);
+  if (__all_sync(0xFFFFFFFFu, ci == first)) {
+    u32 m = __reduce_min_sync(0xFFFFFFFFu, bad);
+    if ((threadIdx.x & 31) == 0 && m != 0xFFFFFFFFu && first != 0xFFFFFFFFu) atomicMin(&a.stop[first], m);
+  } else if (bad != 0xFFFFFFFFu) {
+    atomicMin(&a.stop[ci], bad);
+  }
 }
 
 // A4: apply. Held candidates stamp/lock their block; owners that got a slot create the entry; owners
@@ -560,42 +595,32 @@ __global__ void __launch_bounds__(256) k_radix_hist(const u64 *keys, const u32 *
   counts[threadIdx.x * n_tiles + blockIdx.x] = h[threadIdx.x];   // digit-major
 }
 
-__global__ void __launch_bounds__(1024) k_radix_scan(u32 *counts, const u32 *status) {
-  // exclusive scan of 256 * n_tiles counts by one CTA (same scheme as k_scan_tiles)
-  __shared__ u32 warp_sums[32];
-  __shared__ u32 s_base;
+// One warp per digit: exclusive scan of that digit's per-tile counts in place, digit total to row_total.
+__global__ void __launch_bounds__(256) k_radix_scan(u32 *counts, u32 *row_total, const u32 *status) {
   const u32 m = status[ST_M];
-  const u32 n = 256u * ((m + SORT_TILE - 1) / SORT_TILE);
-  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  if (tid == 0) s_base = 0;
-  __syncthreads();
-  for (u32 start = 0; start < n; start += 1024) {
-    u32 i = start + tid;
-    u32 v = i < n ? counts[i] : 0, x = v;
+  const u32 n_tiles = (m + SORT_TILE - 1) / SORT_TILE;
+  const u32 lane = threadIdx.x & 31, d = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+  if (d >= 256) return;
+  u32 *row = counts + d * n_tiles;
+  u32 run = 0;
+  for (u32 t0 = 0; t0 < n_tiles; t0 += 32) {
+    u32 t = t0 + lane;
+    u32 v = t < n_tiles ? row[t] : 0, x = v;
 #pragma unroll
     for (u32 o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(0xFFFFFFFFu, x, o); if (lane >= o) x += y; }
-    if (lane == 31) warp_sums[warp] = x;
-    __syncthreads();
-    if (warp == 0) {
-      u32 w = warp_sums[lane], z = w;
-#pragma unroll
-      for (u32 o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(0xFFFFFFFFu, z, o); if (lane >= o) z += y; }
-      warp_sums[lane] = z - w;
-    }
-    __syncthreads();
-    u32 incl = s_base + warp_sums[warp] + x;
-    if (i < n) counts[i] = incl - v;
-    __syncthreads();
-    if (tid == 1023) s_base = incl;
-    __syncthreads();
+    if (t < n_tiles) row[t] = run + x - v;
+    run += __shfl_sync(0xFFFFFFFFu, x, 31);
   }
+  if (lane == 0) row_total[d] = run;
 }
 
 __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const u32 *vals_in, u64 *keys_out, u32 *vals_out,
-                                                       const u32 *status, u32 shift, const u32 *offsets) {
+                                                       const u32 *status, u32 shift, const u32 *offsets, const u32 *row_total) {
   // each warp owns 512 consecutive items of the tile and walks them in order, so equal digits keep
   // their input order (stable)
   __shared__ u32 cnt[8][256];
+  __shared__ u32 dbase[256];
+  __shared__ u32 wsum[8];
   const u32 m = status[ST_M];
   const u32 n_tiles = (m + SORT_TILE - 1) / SORT_TILE;
   if (blockIdx.x >= n_tiles) return;
@@ -617,9 +642,20 @@ __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const
     __syncwarp();
   }
   __syncthreads();
-  {  // per digit: exclusive scan across the 8 warps, plus the tile's global offset
+  {  // first position of every digit = exclusive scan of the 256 digit totals
+    u32 v = row_total[tid], x = v;
+#pragma unroll
+    for (u32 o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(0xFFFFFFFFu, x, o); if (lane >= o) x += y; }
+    if (lane == 31) wsum[warp] = x;
+    __syncthreads();
+    u32 before = 0;
+    for (u32 w = 0; w < warp; ++w) before += wsum[w];
+    dbase[tid] = before + x - v;
+  }
+  __syncthreads();
+  {  // per digit: exclusive scan across the 8 warps, plus the tile's offset inside the digit
     u32 d = tid;
-    u32 run = offsets[d * n_tiles + blockIdx.x];
+    u32 run = dbase[d] + offsets[d * n_tiles + blockIdx.x];
 #pragma unroll
     for (int w = 0; w < 8; ++w) { u32 c = cnt[w][d]; cnt[w][d] = run; run += c; }
   }
@@ -803,6 +839,34 @@ __global__ void __launch_bounds__(256) k_move_blocks(MoveArgs a) {
         if (v < vec_per_chunk) __stcs(dp + v, r[u]);
       }
     }
+  }
+}
+
+// Variant for small chunks: work item = 32 lanes x 16 B x UNROLL bytes of one chunk, one item per warp
+// at a time, so that a 4 KiB chunk keeps UNROLL loads per lane in flight instead of one.
+template <int UNROLL>
+__global__ void __launch_bounds__(256) k_move_tiles(MoveArgs a, u32 tiles_per_chunk) {
+  u32 n_pairs = a.n_pairs;
+  if (a.n_pairs_dev) n_pairs = min(n_pairs, *a.n_pairs_dev);
+  const u32 lane = threadIdx.x & 31;
+  const u64 per_pair = (u64)a.n_chunks * tiles_per_chunk;
+  const u64 n_items = (u64)n_pairs * per_pair;
+  const u64 n_warps = (u64)gridDim.x * 8;
+  for (u64 item = (u64)blockIdx.x * 8 + (threadIdx.x >> 5); item < n_items; item += n_warps) {
+    u32 pair = (u32)(item / per_pair);
+    u32 rem = (u32)(item - (u64)pair * per_pair);
+    u32 chunk = rem / tiles_per_chunk, tile = rem - chunk * tiles_per_chunk;
+    u32 s = a.src_ids[pair], d = a.dst_ids[pair];
+    if (s >= a.src.n_slots || d >= a.dst.n_slots) { if (lane == 0) set_err(a.status, DERR_RANGE); continue; }
+    const uint4 *sp = reinterpret_cast<const uint4 *>(a.src.base + s * a.src.slot_stride + chunk * a.src.chunk_stride) +
+                      (u64)tile * 32 * UNROLL + lane;
+    uint4 *dp = reinterpret_cast<uint4 *>(a.dst.base + d * a.dst.slot_stride + chunk * a.dst.chunk_stride) +
+                (u64)tile * 32 * UNROLL + lane;
+    uint4 r[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) r[u] = __ldcs(sp + u * 32);
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) __stcs(dp + u * 32, r[u]);
   }
 }
 

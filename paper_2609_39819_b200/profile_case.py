@@ -5,6 +5,7 @@ larger than L2, a few GB on the device at most, a handful of launches).
     python -m paper_2609_39819_b200.profile_case mover_toy  # the same with 16 KiB blocks (4 KiB chunks)
     python -m paper_2609_39819_b200.profile_case lookup     # hash + table lookup of 16 x 16,128-block calls
     python -m paper_2609_39819_b200.profile_case select     # classify + select 10% of 1 Mi resident blocks
+    python -m paper_2609_39819_b200.profile_case c4         # the whole metadata stress at full size (C4)
 Each prints one line with CUDA-event timings of its launches.
 """
 from __future__ import annotations
@@ -60,6 +61,30 @@ def main(case: str):
         else:
             ms = _events(torch, lambda: eng.select_victims(0, n_res // 10), 3)
             print(f"select: {n_res // 10} victims of {n_res} resident, ms per call {ms}")
+    elif case == "c4":
+        n_res, n_calls = 1 << 20, 64
+        inp = W.inputs_c4(1, n_resident=n_res, chain_blocks=16128, n_calls=n_calls)
+        eng = B.Engine(n_hbm_blocks=n_res, n_host_blocks=0, max_contexts=n_calls + 1, metadata_only=True,
+                       max_tokens=(n_calls + 2) * 16128 * 16 * 2, max_messages=1024, max_batch_blocks=n_calls * 16128,
+                       **W.GEO_TOY.kwargs())
+        keys = np.concatenate([B.hash_tokens(torch.from_numpy(c.view(np.int32)).cuda()).cpu().numpy().view(np.uint64)
+                               for c in inp.chain_tokens])
+        eng.debug_load_resident(keys, inp.state, inp.stamp, inp.depth, inp.slot, 0)
+        ids = list(range(n_calls))
+        for i, t in enumerate(inp.calls):
+            eng.spawn(i)
+            eng.append(i, torch.from_numpy(t.view(np.int32)).cuda())
+        res = {}
+        for frac in (0.10, 0.35, 0.75):
+            res[f"select_{int(frac * 100)}pct_ms"] = _events(torch, lambda: eng.select_victims(0, int(n_res * frac)), 3)
+        res["lookup_batch_ms"] = _events(torch, lambda: eng.map_blocks(ids, 0), 1)
+        res["classify_ms"] = _events(torch, lambda: eng.classify(), 3)
+        v, _s = eng.select_victims(0, n_res // 10)
+        res["drop_10pct_ms"] = _events(torch, lambda: eng.offload(v), 1)
+        res["admit_batch_ms"] = _events(torch, lambda: eng.map_blocks(ids, 1), 1)
+        st = eng.get_stats()
+        print(f"c4: {n_res} resident, {n_calls} calls x 16128 blocks; hits {st['hits_hbm']}, inserted {st['inserted']}, "
+              f"adopted {st['adopted']}, tombstones {st['tombstones']}; {res}")
     else:
         raise SystemExit(__doc__)
 
