@@ -6,6 +6,7 @@ larger than L2, a few GB on the device at most, a handful of launches).
     python -m paper_2609_39819_b200.profile_case lookup     # hash + table lookup of 16 x 16,128-block calls
     python -m paper_2609_39819_b200.profile_case select     # classify + select 10% of 1 Mi resident blocks
     python -m paper_2609_39819_b200.profile_case c4         # the whole metadata stress at full size (C4)
+    python -m paper_2609_39819_b200.profile_case sweep      # C5: movement bandwidth sweep (markdown table)
 Each prints one line with CUDA-event timings of its launches.
 """
 from __future__ import annotations
@@ -22,6 +23,52 @@ def _events(torch, fn, n):
         a.record(); fn(); b.record(); torch.cuda.synchronize()
         out.append(round(a.elapsed_time(b), 4))
     return out
+
+
+def sweep(torch, B, W):
+    """C5: n = 1 .. 65,536 blocks x block sizes x {contiguous, permuted} ids x {gather to the host tier, scatter
+    back, HBM -> HBM}; 3 warm-ups, best and median of 10 launches, CUDA events. The pools are capped at 8 GiB
+    (HBM) and 4 GiB (pinned host), which caps n for the large blocks."""
+    def bench(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(10):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(); fn(); b.record(); torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        ts.sort()
+        return ts[0], ts[len(ts) // 2]
+
+    print("| block | layout | ids | n | gather HBM->host GB/s (best / median) | scatter host->HBM GB/s | HBM->HBM GB/s read+write |")
+    print("|---|---|---|---:|---:|---:|---:|")
+    for geo in (W.GEO_TOY, W.GEO_128K, W.GEO_512K, W.GEO_8B, W.GEO_GLM):
+        n_hbm = min(131072, (8 << 30) // geo.block_bytes)
+        n_host = min(65536, (4 << 30) // geo.block_bytes)
+        for layout in (0, 1):
+            eng = B.Engine(n_hbm_blocks=n_hbm, n_host_blocks=n_host, max_contexts=2, pool_layout=layout, max_tokens=1 << 12,
+                           max_messages=64, max_batch_blocks=65536, zero_pools=False, **geo.kwargs())
+            n = 1
+            while n <= 65536:
+                nn = min(n, n_host)
+                for perm in (False, True):
+                    src = torch.from_numpy(W.ids_c5(1, nn, n_hbm // 2, perm).view(np.int32)).cuda()
+                    dst = torch.from_numpy(W.ids_c5(2, nn, n_host, perm).view(np.int32)).cuda()
+                    d2 = (torch.from_numpy(W.ids_c5(3, nn, n_hbm // 2, perm).view(np.int32)) + n_hbm // 2).cuda()
+                    gb = nn * geo.block_bytes / 1e6
+                    g = bench(lambda: eng.copy_blocks(0, src, 1, dst))
+                    sc = bench(lambda: eng.copy_blocks(1, dst, 0, src))
+                    hh = bench(lambda: eng.copy_blocks(0, src, 0, d2))
+                    print(f"| {geo.block_bytes >> 10} KiB | {'layer' if layout == 0 else 'block'}-major | "
+                          f"{'permuted' if perm else 'contiguous'} | {nn} | {gb / g[0]:.1f} / {gb / g[1]:.1f} | "
+                          f"{gb / sc[0]:.1f} / {gb / sc[1]:.1f} | {2 * gb / hh[0]:.1f} / {2 * gb / hh[1]:.1f} |", flush=True)
+                if nn < n:
+                    break
+                n *= 4
+            eng.close()
+            del eng
+            torch.cuda.empty_cache()
 
 
 def main(case: str):
@@ -85,6 +132,8 @@ def main(case: str):
         st = eng.get_stats()
         print(f"c4: {n_res} resident, {n_calls} calls x 16128 blocks; hits {st['hits_hbm']}, inserted {st['inserted']}, "
               f"adopted {st['adopted']}, tombstones {st['tombstones']}; {res}")
+    elif case == "sweep":
+        sweep(torch, B, W)
     else:
         raise SystemExit(__doc__)
 

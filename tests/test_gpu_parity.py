@@ -143,6 +143,19 @@ def test_full_length_c2_session_metadata_parity(B, oracle, n_hbm):
         assert cpu.get_stats()["dropped"] > 0
 
 
+def test_full_size_c3_metadata_parity(B, oracle):
+    """C3 at full size (32 sessions of 32K-258K tokens, forks, GLM-scale geometry, 120 GiB = 21,370-block HBM
+    pool) on metadata-only engines: every batch call's lookups, victim lists, offloads, reloads and
+    admissions equal the oracle's."""
+    trace, n_ctx = W.trace_c3(1)
+    kw = dict(n_hbm_blocks=21370, n_host_blocks=20000, max_contexts=n_ctx, metadata_only=True, **W.GEO_GLM.kwargs())
+    gpu = B.Engine(max_tokens=1 << 24, max_messages=1 << 16, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    n = _replay_pair(gpu, cpu, trace, None, record_states=True)
+    st = cpu.get_stats()
+    assert n > 100 and st["offloaded"] > 10000 and st["reloaded"] > 10000 and st["dropped"] > 10000
+
+
 # ---- C4: metadata stress at full size -------------------------------------------------------------------
 def _c4_setup(B, oracle, n_resident, chain_blocks, n_calls):
     inp = W.inputs_c4(1, n_resident=n_resident, chain_blocks=chain_blocks, n_calls=n_calls)
@@ -201,11 +214,34 @@ def test_c4_lookup_and_select_parity(B, oracle, n_resident, chain_blocks, n_call
 
 
 # ---- C5: the raw mover ------------------------------------------------------------------------------------
-@pytest.mark.parametrize("geo", [W.GEO_TOY, W.GEO_128K, W.GEO_8B], ids=lambda g: g.name)
+def test_c5_longest_id_list(B, oracle):
+    """65,536 permuted blocks in one call (the sweep's maximum), toy payloads: 1 GiB each way."""
+    import torch
+    n = 65536
+    kw = dict(n_hbm_blocks=n, n_host_blocks=n, max_contexts=2, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 12, max_messages=64, max_batch_blocks=n, zero_pools=False, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    fill = np.random.default_rng(8).integers(0, 256, gpu.hbm_pool.numel(), dtype=np.uint8)
+    gpu.hbm_pool.copy_(torch.from_numpy(fill))
+    cpu.hbm_pool[:] = fill
+    src, dst = W.ids_c5(1, n, n, True), W.ids_c5(2, n, n, True)
+    for eng in (gpu, cpu):
+        eng.copy_blocks(0, src, 1, dst)
+    torch.cuda.synchronize()
+    assert np.array_equal(gpu.host_pool.numpy(), cpu.host_pool)
+    gpu.hbm_pool.zero_()
+    cpu.hbm_pool[:] = 0
+    for eng in (gpu, cpu):
+        eng.copy_blocks(1, dst, 0, src)
+    torch.cuda.synchronize()
+    assert np.array_equal(gpu.hbm_pool.cpu().numpy(), fill) and np.array_equal(cpu.hbm_pool, fill)
+
+
+@pytest.mark.parametrize("geo", [W.GEO_TOY, W.GEO_128K, W.GEO_8B, W.GEO_GLM], ids=lambda g: g.name)
 @pytest.mark.parametrize("layout", [0, 1])
 def test_c5_mover_parity(B, oracle, geo, layout):
     import torch
-    n_slots = 24 if geo.block_bytes > (1 << 20) else 200
+    n_slots = (12 if geo.block_bytes > (4 << 20) else 24) if geo.block_bytes > (1 << 20) else 200
     kw = dict(n_hbm_blocks=n_slots, n_host_blocks=n_slots, max_contexts=2, pool_layout=layout, **geo.kwargs())
     gpu = B.Engine(max_tokens=1 << 12, max_messages=64, max_batch_blocks=4096, **kw)
     cpu = oracle.OracleEngine(**kw)
