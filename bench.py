@@ -55,6 +55,7 @@ def parse_args():
     ap.add_argument("--cpu-steps", type=int, default=6, help="steps of the bounded CPU-oracle sample")
     ap.add_argument("--skip-e2e", action="store_true")
     ap.add_argument("--skip-cpu", action="store_true")
+    ap.add_argument("--skip-stress", action="store_true", help="skip the C4-shaped metadata measurement")
     return ap.parse_args()
 
 
@@ -351,6 +352,74 @@ def gpu_arm(args, torch, B, setup, turns, n_ff, e2e, n_host_blocks, n_hbm_blocks
     return res
 
 
+def metadata_stress(torch, B, hbm_peak, reps=5):
+    """C4-shaped side measurement of the metadata stages at scale (the C2 calls above are launch-latency
+    sized): 1 Mi resident blocks, one LOOKUP batch of 64 calls x 16,128 blocks, classification of the
+    resulting 1.03 M mappings, selection of 10% of the pool. Kernel times come from the library's own
+    CUDA events, call times from events around the C-ABI call. Algorithmic bytes per unit: hash 72 B per
+    block (64 B tokens + 8 B key), fused lookup 64 B per block (two 32-byte table sectors), classify 16 B
+    per mapping + 9 B per entry, select 8 B per resident block + 4 B per victim."""
+    n_res, n_calls, cb = 1 << 20, 64, 16128
+    inp = W.inputs_c4(1, n_resident=n_res, chain_blocks=cb, n_calls=n_calls)
+    eng = B.Engine(n_hbm_blocks=n_res, n_host_blocks=0, max_contexts=n_calls + 1, metadata_only=True,
+                   max_tokens=(n_calls + 2) * cb * 16 * 2, max_messages=1024, max_batch_blocks=n_calls * cb,
+                   **W.GEO_TOY.kwargs())
+    keys = np.concatenate([B.hash_tokens(torch.from_numpy(c.view(np.int32)).cuda()).cpu().numpy().view(np.uint64)
+                           for c in inp.chain_tokens])
+    eng.debug_load_resident(keys, inp.state, inp.stamp, inp.depth, inp.slot, 0)
+    ids = list(range(n_calls))
+    for i, t in enumerate(inp.calls):
+        eng.spawn(i)
+        eng.append(i, torch.from_numpy(t.view(np.int32)).cuda())
+    eng.set_profiling(True)
+
+    def timed(fn):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(); r = fn(); b.record(); torch.cuda.synchronize()
+        return a.elapsed_time(b), r
+
+    look_ms, cls_ms, sel_ms = [], [], []
+    s0 = None
+    for rep in range(reps + 1):
+        if rep == 1:
+            s0 = eng.get_stats()          # the first repetition is the warm-up
+        ms, info = timed(lambda: eng.map_blocks(ids, 0))
+        look_ms.append(ms)
+        cls_ms.append(timed(lambda: eng.classify())[0])
+        for c in ids:
+            eng.prefill_done(c)
+        eng.classify()
+        torch.cuda.synchronize()
+        ms, (v, _st) = timed(lambda: eng.select_victims(0, n_res // 10))
+        sel_ms.append(ms)
+    s1 = eng.get_stats()
+    d = {k: s1[k] - s0[k] for k in s1}
+    n_blocks = int(info["n_blocks"].sum())
+    hit = float(info["hit_len"].sum()) / n_blocks
+    look_k = d["lookup_ns"] / 1e6 / reps
+    sel_k = d["select_ns"] / 1e6 / reps
+    med = lambda x: float(np.median(x[1:]))
+    out = {
+        "workload": f"C4: {n_res} resident blocks (dead 30 / idle 40 / active 30 %), LOOKUP batch of {n_calls} calls x {cb} "
+                    f"blocks ({hit:.0%} prefix hits), classify, select 10%; median of {reps} after 1 warm-up",
+        "hash_lookup": {"blocks_per_call": n_blocks, "call_ms": med(look_ms), "kernels_ms": look_k,
+                        "blocks_per_s": n_blocks / (med(look_ms) / 1e3), "blocks_per_s_kernels": n_blocks / (look_k / 1e3),
+                        "algorithmic_bytes_per_block": 136, "achieved_GBs": n_blocks * 136 / (look_k / 1e3) / 1e9,
+                        "frac_hbm": n_blocks * 136 / (look_k / 1e3) / 1e9 / hbm_peak},
+        "classify": {"mappings": n_blocks, "entries": n_res, "call_ms": med(cls_ms),
+                     "achieved_GBs": (16 * n_blocks + 9 * n_res) / (med(cls_ms) / 1e3) / 1e9,
+                     "frac_hbm": (16 * n_blocks + 9 * n_res) / (med(cls_ms) / 1e3) / 1e9 / hbm_peak},
+        "select": {"resident": n_res, "victims": len(v), "call_ms": med(sel_ms), "kernels_ms": sel_k,
+                   "resident_blocks_per_s": n_res / (med(sel_ms) / 1e3),
+                   "achieved_GBs": (8 * n_res + 4 * len(v)) / (sel_k / 1e3) / 1e9,
+                   "frac_hbm": (8 * n_res + 4 * len(v)) / (sel_k / 1e3) / 1e9 / hbm_peak},
+    }
+    eng.close()
+    del eng
+    torch.cuda.empty_cache()
+    return out
+
+
 def cpu_arm(args, setup, turns, n_ff, n_steps, n_warm, n_hbm_blocks, n_host_blocks):
     """The CPU oracle, as it stands, on the same steps: payload copies are plain memcpy on one core."""
     from oracle import kvt_oracle
@@ -532,6 +601,8 @@ def main():
             "peak_kind": "measured: 1 GiB pinned cudaMemcpyAsync per direction, best of 10, this run",
             "stage_wall_ms_per_step": {k: round(x / K, 4) for k, x in e["stage_ms"].items()},
         }
+    if not args.skip_stress and world == 1:
+        line["metadata_stress"] = metadata_stress(torch, B, hbm_peak)
     if not args.skip_cpu and world == 1:
         n_host_blocks = min(int(args.host_gib * GiB), int(mem_available_bytes() * 0.5)) // W.GEO_8B.block_bytes
         c = cpu_arm(args, setup, turns, n_ff, min(args.cpu_steps, K), 1, n_hbm_blocks, n_host_blocks)

@@ -307,6 +307,10 @@ typedef struct kvt_stats {
   uint64_t mover_launches;   /* with profiling on: mover kernels timed, their device time and payload bytes */
   uint64_t mover_ns;
   uint64_t mover_bytes;
+  uint64_t lookup_ns;        /* with profiling on: device time of the hash + lookup + lock kernels of LOOKUP calls */
+  uint64_t lookup_blocks;    /* and the blocks they processed */
+  uint64_t select_ns;        /* with profiling on: device time of the selection kernels (count, compaction, sort, emit) */
+  uint64_t select_slots;     /* and the tier slots they scanned */
 } kvt_stats;
 int32_t kvt_get_stats(kvt_engine *e, kvt_stats *out);
 

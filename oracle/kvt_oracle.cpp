@@ -126,7 +126,8 @@ struct CallInfo { uint32_t n_blocks, hit_len, n_hit_hbm, n_hit_host, n_admissibl
 struct Stats {
   uint64_t clock, n_contexts, occ_hbm, occ_host, blocks_hashed, hits_hbm, hits_host, misses,
       inserted, adopted, dropped, offloaded, reloaded, compacted, bytes_d2h, bytes_h2d, bytes_d2d,
-      table_rebuilds, tombstones, kernel_launches, mover_launches, mover_ns, mover_bytes;
+      table_rebuilds, tombstones, kernel_launches, mover_launches, mover_ns, mover_bytes, lookup_ns,
+      lookup_blocks, select_ns, select_slots;
 };
 
 struct Op {

@@ -139,7 +139,7 @@ struct kvt_engine {
   // optional timing of the mover kernel (kvt_set_profiling)
   bool profiling = false, mover_timed = false;
   u32 mover_variant = 0;   // 0 auto, 1 CTA per chunk, 2 warp per 4 KiB tile
-  cudaEvent_t ev_m0 = nullptr, ev_m1 = nullptr;
+  cudaEvent_t ev_m0 = nullptr, ev_m1 = nullptr, ev_h0 = nullptr, ev_h1 = nullptr;
 
   template <class T> T *dp(u64 off) const { return reinterpret_cast<T *>(meta + off); }
   u32 tier_slots(u32 t) const { return t == KVT_TIER_HBM ? cfg.n_hbm_blocks : cfg.n_host_blocks; }
@@ -454,7 +454,8 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   e->h_ids = (u32 *)(e->stage + o_ids); e->h_ids2 = (u32 *)(e->stage + o_ids2);
   cudaStream_t s = (cudaStream_t)stream;
   bool ok = cudaEventCreateWithFlags(&e->ev_upload, cudaEventDisableTiming) == cudaSuccess &&
-            cudaEventCreate(&e->ev_m0) == cudaSuccess && cudaEventCreate(&e->ev_m1) == cudaSuccess;
+            cudaEventCreate(&e->ev_m0) == cudaSuccess && cudaEventCreate(&e->ev_m1) == cudaSuccess &&
+            cudaEventCreate(&e->ev_h0) == cudaSuccess && cudaEventCreate(&e->ev_h1) == cudaSuccess;
   // everything except the key arena and scratch must start at zero; the table needs ent = NONE
   ok = ok && cudaMemsetAsync(e->meta + L.e_key, 0, L.keys - L.e_key, s) == cudaSuccess;
   ok = ok && cudaMemsetAsync(e->d_status, 0, ST_WORDS * 4, s) == cudaSuccess;
@@ -473,6 +474,8 @@ int32_t kvt_destroy(kvt_engine *e) {
   if (e->ev_upload) cudaEventDestroy(e->ev_upload);
   if (e->ev_m0) cudaEventDestroy(e->ev_m0);
   if (e->ev_m1) cudaEventDestroy(e->ev_m1);
+  if (e->ev_h0) cudaEventDestroy(e->ev_h0);
+  if (e->ev_h1) cudaEventDestroy(e->ev_h1);
   if (e->stage) cudaFreeHost(e->stage);
   delete e;
   return KVT_OK;
@@ -701,14 +704,20 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     LockArgs lk;
     lk.ent = e->ent; lk.b_ent = la.b_ent; lk.hit_len = d_res; lk.n_hbm = d_res + C; lk.n_host = d_res + 2 * C;
     lk.now = e->now; lk.status = e->d_status;
+    if (e->profiling) CU(cudaEventRecord(e->ev_h0, s));
     KL(k_hash_digest, chunk_base, CHUNK, s, ha);
     KL(k_hash_carry, cdiv((u64)nd * 32, 128), 128, s, ha);
     KL(k_hash_finish_lookup, chunk_base, CHUNK, s, ha, la);
     KL(k_lock_hits, chunk_base, CHUNK, s, ha, lk);
+    if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));
     LAUNCH_CHECK();
     CU(cudaMemcpyAsync(h_hit, d_res, 3ull * C * 4, cudaMemcpyDeviceToHost, s));
     r = status_fetch(e, s);
     if (r) return r;
+    if (e->profiling) {
+      float ms = 0.f;
+      if (cudaEventElapsedTime(&ms, e->ev_h0, e->ev_h1) == cudaSuccess) { e->st.lookup_ns += (u64)((double)ms * 1e6); e->st.lookup_blocks += blk_base; }
+    }
     r = status_code(e);
     if (r) return r;
   }
@@ -913,6 +922,7 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   u64 *kA = e->dp<u64>(e->L.keyA), *kB = e->dp<u64>(e->L.keyB);
   u32 *vA = e->dp<u32>(e->L.valA), *vB = e->dp<u32>(e->L.valB), *counts = e->dp<u32>(e->L.rcounts);
   u32 *row_total = counts + 256ull * (e->L.Nt / SORT_TILE + 1);
+  if (e->profiling) CU(cudaEventRecord(e->ev_h0, s));
   KL(k_sel_count, cdiv(n,256), 256, s, a);
   r = compact_indices(e, s, PredSel{a}, EmitSel{a, kA, vA}, n, ST_M);
   if (r) return r;
@@ -926,9 +936,14 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   u32 n_emit = std::min(n_req, n);
   KL(k_sel_emit, cdiv(n_emit,256), 256, s, kA, vA, n_emit, a.stamp_bits + a.depth_bits, e->dp<u32>(e->L.out_slots),
                                                e->dp<u8>(e->L.out_states));
+  if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));
   LAUNCH_CHECK();
   r = status_fetch(e, s);
   if (r) return r;
+  if (e->profiling) {
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, e->ev_h0, e->ev_h1) == cudaSuccess) { e->st.select_ns += (u64)((double)ms * 1e6); e->st.select_slots += n; }
+  }
   r = status_code(e);
   if (r) return r;
   u64 total = (u64)e->h_status[ST_RANK0] + e->h_status[ST_RANK1] + e->h_status[ST_RANK2];
