@@ -81,8 +81,8 @@ extern "C" {
                                     [msg_start, msg_end) for one inference (Temporary) */
 #define KVT_OP_PREFILL_DONE  7u  /* prefill of the context's in-flight call completed */
 #define KVT_OP_TERMINATE     8u  /* the context ends */
-#define KVT_OP_PIN           9u  /* reserved: returns KVT_E_INVAL */
-#define KVT_OP_UNPIN        10u  /* reserved: returns KVT_E_INVAL */
+#define KVT_OP_PIN           9u  /* declare long-term retention of messages [msg_start, msg_end) */
+#define KVT_OP_UNPIN        10u  /* release that protection */
 
 /* kvt_op.flags */
 #define KVT_OPF_TOKENS_ON_DEVICE 1u  /* op.tokens is a device pointer (device-to-device copy) */
@@ -90,6 +90,9 @@ extern "C" {
 /* kvt_map_blocks phases */
 #define KVT_MAP_LOOKUP 0u
 #define KVT_MAP_ADMIT  1u
+
+/* kvt_select_victims flags */
+#define KVT_SEL_INCLUDE_PINNED 1u  /* the incoming KV is Pinned: Pinned residents compete too (Algorithm 1, last branch) */
 
 /* kvt_copy_blocks flags */
 #define KVT_IDS_ON_DEVICE 1u  /* src/dst id arrays are device pointers */
@@ -99,7 +102,7 @@ extern "C" {
 #define KVT_STATE_DEAD    0u   /* no live message version maps the block */
 #define KVT_STATE_IDLE    1u   /* live but idle: best mapped message state is Suspended */
 #define KVT_STATE_ACTIVE  2u   /* live and active */
-#define KVT_STATE_PINNED  3u   /* reserved */
+#define KVT_STATE_PINNED  3u   /* explicitly retained: competes for space only with incoming Pinned KV */
 #define KVT_STATE_FREE    0xFFu /* slot holds no block */
 
 typedef struct kvt_engine kvt_engine;
@@ -168,7 +171,11 @@ typedef struct kvt_op {
  *     still-valid blocks they cover; parent and child evolve independently afterwards.
  *   ONE_OFF: listed (or all current and future) messages become Temporary.
  *   PREFILL_DONE: Active -> Suspended; advances the logical clock; stamps and unlocks held blocks.
- *   TERMINATE: the context stops mapping anything and its id becomes free.
+ *   PIN / UNPIN: listed messages become Pinned / Pinned ones return to Suspended (Temporary in a one_off
+ *     context). Pinned messages are not touched by call begin, PREFILL_DONE or the whole-context ONE_OFF.
+ *   TERMINATE: ordinary messages expire. Without Pinned messages the context stops mapping anything and
+ *     its id becomes free; with Pinned messages it is kept (they retain their protection), accepts only
+ *     UNPIN (which then expires them), and goes away with its last Pinned message.
  * Errors: KVT_E_NOCTX unknown context; KVT_E_INVAL id in use / bad op / NULL tokens;
  * KVT_E_RANGE bad message range; KVT_E_STATE edit or fork-from of an in-flight context, or
  * PREFILL_DONE of a context that is not in flight; KVT_E_NOSPACE token arena full.
@@ -184,6 +191,7 @@ typedef struct kvt_call_info {
   uint32_t n_admissible;  /* blocks after the prefix that may enter reusable storage (Temporary bypass) */
   uint32_t n_admitted;    /* ADMIT: blocks this call newly holds (inserted or adopted) */
   uint32_t n_held;        /* leading blocks locked in flight for this context after the call */
+  uint32_t n_pinned;      /* of the admissible blocks, those touched by a Pinned message */
 } kvt_call_info;
 
 /* phase KVT_MAP_LOOKUP — one LLM call begins for each listed context (Section 7: call id and
@@ -222,12 +230,13 @@ int32_t kvt_get_states(kvt_engine *e, uint32_t tier, uint8_t *state, uint32_t ca
 
 /* ---- stage 4: victim selection (Algorithm 1 order; Section 6.2 recency) ----------------------- */
 /* Returns the first min(n_req, #candidates) slots of `tier` in eviction order, with their ranks.
- * Candidates: resident, not in flight, rank below Pinned. Order: rank ascending (dead, idle,
- * active); within dead and active oldest stamp first; within idle newest stamp first (MRU) or
+ * Candidates: resident, not in flight, rank below Pinned (Pinned included, last, with
+ * KVT_SEL_INCLUDE_PINNED). Order: rank ascending (dead, idle, active, pinned); within dead, active and
+ * pinned oldest stamp first; within idle newest stamp first (MRU) or
  * oldest first if suspended_order = KVT_ORDER_LRU; then chain depth descending; then slot
  * ascending. Classifies first if needed. Host output arrays (states_out may be NULL).
  * KVT_E_BUFSZ if cap < min(n_req, #candidates). Synchronises. */
-int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_t *slots_out,
+int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_t flags, uint32_t *slots_out,
                            uint8_t *states_out, uint32_t cap, uint32_t *n_out, void *stream);
 
 /* ---- stage 5: tier movement (Section 7; Algorithm 1 "release") -------------------------------- */

@@ -47,12 +47,13 @@ enum : uint32_t {
   OP_TERMINATE, OP_PIN, OP_UNPIN
 };
 // message-level states (Section 5.2)
-enum : uint8_t { MS_ACTIVE = 0, MS_SUSPENDED = 1, MS_EXPIRED = 2, MS_TEMPORARY = 3 };
+enum : uint8_t { MS_ACTIVE = 0, MS_SUSPENDED = 1, MS_EXPIRED = 2, MS_TEMPORARY = 3, MS_PINNED = 4 };
 
 // Priority of a message state for the block aggregate, following Algorithm 1's release order:
-// Discarded (Expired, Temporary) lowest, then Suspended, then Active.
+// Discarded (Expired, Temporary) lowest, then Suspended, then Active, then Pinned.
 int msgrank(uint8_t s) {
   switch (s) {
+    case MS_PINNED: return 3;
     case MS_ACTIVE: return 2;
     case MS_SUSPENDED: return 1;
     default: return 0;
@@ -100,6 +101,7 @@ struct Msg { std::vector<uint32_t> tok; uint8_t state; };
 
 struct Ctx {
   bool live = false;
+  bool terminated = false;   // ended, but kept because it still has Pinned messages (Section 5.2)
   std::vector<Msg> msgs;
   bool one_off = false, in_flight = false;
   // materialised mapping: token sequence as of the last call (or inherited at fork), the bounds of
@@ -109,7 +111,7 @@ struct Ctx {
   std::vector<uint64_t> mat_keys;                          // hash of mat_tokens
   uint32_t valid_blocks = 0;  // leading blocks of mat_keys this context still maps
   uint32_t held = 0;          // leading blocks locked in flight
-  uint32_t hit_len = 0, n_hit_hbm = 0, n_hit_host = 0, n_admissible = 0;
+  uint32_t hit_len = 0, n_hit_hbm = 0, n_hit_host = 0, n_admissible = 0, n_pinned = 0;
 };
 
 struct Entry { uint64_t key = 0; uint32_t stamp = 0, depth = 0, inflight = 0; uint8_t floor = 0; };
@@ -121,7 +123,7 @@ struct Config {
   uint8_t *hbm_pool; uint8_t *host_pool;  // host memory; NULL = metadata only
 };
 
-struct CallInfo { uint32_t n_blocks, hit_len, n_hit_hbm, n_hit_host, n_admissible, n_admitted, n_held; };
+struct CallInfo { uint32_t n_blocks, hit_len, n_hit_hbm, n_hit_host, n_admissible, n_admitted, n_held, n_pinned; };
 
 struct Stats {
   uint64_t clock, n_contexts, occ_hbm, occ_host, blocks_hashed, hits_hbm, hits_host, misses,
@@ -162,8 +164,9 @@ void copy_payload(Engine &e, uint32_t st, uint32_t ss, uint32_t dt, uint32_t ds)
     std::memcpy(chunk_ptr(e, dt, ds, c), chunk_ptr(e, st, ss, c), e.chunk_bytes);
 }
 
-Ctx *get_ctx(Engine &e, uint32_t id) {
+Ctx *get_ctx(Engine &e, uint32_t id, bool allow_terminated = false) {
   if (id >= e.ctxs.size() || !e.ctxs[id].live) return nullptr;
+  if (e.ctxs[id].terminated && !allow_terminated) return nullptr;
   return &e.ctxs[id];
 }
 
@@ -311,8 +314,8 @@ int32_t kvto_apply_op(Engine *e, const Op *op) {
     }
     default: break;
   }
-  if (op->op == OP_PIN || op->op == OP_UNPIN || op->op == 0 || op->op > OP_UNPIN) return E_INVAL;
-  Ctx *c = get_ctx(*e, id);
+  if (op->op == 0 || op->op > OP_UNPIN) return E_INVAL;
+  Ctx *c = get_ctx(*e, id, op->op == OP_UNPIN);   // a terminated context with Pinned messages only accepts unpin
   if (!c) return E_NOCTX;
   switch (op->op) {
     case OP_APPEND: {
@@ -343,7 +346,8 @@ int32_t kvto_apply_op(Engine *e, const Op *op) {
       if (c->in_flight) return E_STATE;
       if (op->msg_start == 0 && op->msg_end == 0xFFFFFFFFu) {
         c->one_off = true;
-        for (Msg &m : c->msgs) m.state = MS_TEMPORARY;
+        for (Msg &m : c->msgs)
+          if (m.state != MS_PINNED) m.state = MS_TEMPORARY;   // explicit protection stays
         return OK;
       }
       if (!(op->msg_start < op->msg_end && op->msg_end <= c->msgs.size())) return E_RANGE;
@@ -361,7 +365,37 @@ int32_t kvto_apply_op(Engine *e, const Op *op) {
     }
     case OP_TERMINATE: {
       if (c->in_flight) unlock_held(*e, *c, false);
-      *c = Ctx();  // ordinary messages expire; the context maps nothing any more
+      bool pinned = false;
+      for (Msg &m : c->msgs) {
+        if (m.state == MS_PINNED) pinned = true;
+        else m.state = MS_EXPIRED;   // ordinary messages expire
+      }
+      if (pinned) {                  // Pinned messages retain their declared protection
+        c->terminated = true;
+        c->in_flight = false;
+      } else {
+        *c = Ctx();                  // the context maps nothing any more
+      }
+      return OK;
+    }
+    case OP_PIN: {
+      if (c->in_flight) return E_STATE;
+      if (!(op->msg_start < op->msg_end && op->msg_end <= c->msgs.size())) return E_RANGE;
+      for (uint32_t j = op->msg_start; j < op->msg_end; ++j) c->msgs[j].state = MS_PINNED;
+      return OK;
+    }
+    case OP_UNPIN: {
+      if (c->in_flight) return E_STATE;
+      if (!(op->msg_start < op->msg_end && op->msg_end <= c->msgs.size())) return E_RANGE;
+      // back to Suspended between calls, or to Expired if the context has terminated
+      for (uint32_t j = op->msg_start; j < op->msg_end; ++j)
+        if (c->msgs[j].state == MS_PINNED)
+          c->msgs[j].state = c->terminated ? MS_EXPIRED : (c->one_off ? MS_TEMPORARY : MS_SUSPENDED);
+      if (c->terminated) {
+        bool pinned = false;
+        for (const Msg &m : c->msgs) pinned = pinned || m.state == MS_PINNED;
+        if (!pinned) *c = Ctx();
+      }
       return OK;
     }
   }
@@ -418,13 +452,14 @@ int32_t kvto_map_blocks(Engine *e, const uint32_t *ids, uint32_t n_ctx, uint32_t
       std::vector<uint8_t> br;
       block_ranks(c, c.mat_bounds, nb, br);
       uint32_t a = h;
-      while (a < nb && br[a] != 0) ++a;
+      c.n_pinned = 0;
+      while (a < nb && br[a] != 0) { c.n_pinned += br[a] == 3; ++a; }
       c.n_admissible = a - h;
       e->st.blocks_hashed += nb;
       e->st.hits_hbm += c.n_hit_hbm;
       e->st.hits_host += c.n_hit_host;
       e->st.misses += nb - h;
-      out[i] = CallInfo{nb, h, c.n_hit_hbm, c.n_hit_host, c.n_admissible, 0, c.held};
+      out[i] = CallInfo{nb, h, c.n_hit_hbm, c.n_hit_host, c.n_admissible, 0, c.held, c.n_pinned};
     }
     return OK;
   }
@@ -453,7 +488,7 @@ int32_t kvto_map_blocks(Engine *e, const uint32_t *ids, uint32_t n_ctx, uint32_t
     }
     uint32_t adm = b - c.held;
     c.held = b;
-    out[i] = CallInfo{(uint32_t)c.mat_keys.size(), c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, adm, c.held};
+    out[i] = CallInfo{(uint32_t)c.mat_keys.size(), c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, adm, c.held, c.n_pinned};
   }
   return OK;
 }
@@ -461,7 +496,7 @@ int32_t kvto_map_blocks(Engine *e, const uint32_t *ids, uint32_t n_ctx, uint32_t
 int32_t kvto_get_block_map(Engine *e, uint32_t ctx, uint64_t *keys, uint8_t *tier, uint32_t *slot,
                            uint32_t cap, uint32_t *n) {
   if (!e || !n) return E_INVAL;
-  Ctx *c = get_ctx(*e, ctx);
+  Ctx *c = get_ctx(*e, ctx, true);
   if (!c) return E_NOCTX;
   uint32_t nb = (uint32_t)c->mat_keys.size();
   *n = nb;
@@ -512,21 +547,22 @@ int32_t kvto_classify_bruteforce(Engine *e, uint32_t tier, uint8_t *state, uint3
   return OK;
 }
 
-int32_t kvto_select_victims(Engine *e, uint32_t tier, uint32_t n_req, uint32_t *slots_out,
+int32_t kvto_select_victims(Engine *e, uint32_t tier, uint32_t n_req, uint32_t flags, uint32_t *slots_out,
                             uint8_t *states_out, uint32_t cap, uint32_t *n_out) {
-  if (!e || tier > 1 || !n_out || (!slots_out && cap)) return E_INVAL;
+  if (!e || tier > 1 || flags > 1 || !n_out || (!slots_out && cap)) return E_INVAL;
+  const int max_rank = (flags & 1) ? 3 : 2;   // Pinned KV competes only when the incoming KV is Pinned
   std::vector<uint8_t> rank[2];
   classify(*e, rank);
   struct Cand { uint32_t slot; uint8_t rank; uint32_t stamp, depth; };
   std::vector<Cand> cands;
   for (uint32_t s = 0; s < tier_size(*e, tier); ++s) {
     const Entry &x = e->ent[tier][s];
-    if (!x.key || x.inflight || rank[tier][s] >= 3) continue;
+    if (!x.key || x.inflight || rank[tier][s] > max_rank) continue;
     cands.push_back(Cand{s, rank[tier][s], x.stamp, x.depth});
   }
   const bool mru = e->cfg.suspended_order == ORDER_MRU;
   std::stable_sort(cands.begin(), cands.end(), [mru](const Cand &a, const Cand &b) {
-    if (a.rank != b.rank) return a.rank < b.rank;            // Algorithm 1: dead, idle, active
+    if (a.rank != b.rank) return a.rank < b.rank;            // Algorithm 1: dead, idle, active, (pinned)
     if (a.stamp != b.stamp) {
       if (a.rank == 1 && mru) return a.stamp > b.stamp;      // Section 6.2: most recently suspended first
       return a.stamp < b.stamp;                              // oldest first
@@ -678,7 +714,7 @@ int32_t kvto_debug_load_resident(Engine *e, const uint64_t *keys, const uint8_t 
   std::set<uint64_t> kseen;
   std::set<uint32_t> sseen;
   for (uint32_t i = 0; i < n; ++i) {
-    if (keys[i] < 2 || state[i] > 2 || slot[i] >= tier_size(*e, tier)) return E_INVAL;
+    if (keys[i] < 2 || state[i] > 3 || slot[i] >= tier_size(*e, tier)) return E_INVAL;
     if (e->where.count(keys[i]) || e->ent[tier][slot[i]].key) return E_INVAL;
     if (!kseen.insert(keys[i]).second || !sseen.insert(slot[i]).second) return E_INVAL;
   }

@@ -51,7 +51,7 @@ class _Op(C.Structure):
 
 
 CALL_INFO_DTYPE = np.dtype([(n, np.uint32) for n in ("n_blocks", "hit_len", "n_hit_hbm", "n_hit_host",
-                                                       "n_admissible", "n_admitted", "n_held")])
+                                                       "n_admissible", "n_admitted", "n_held", "n_pinned")])
 STATS_FIELDS = ("clock", "n_contexts", "occ_hbm", "occ_host", "blocks_hashed", "hits_hbm", "hits_host", "misses",
                 "inserted", "adopted", "dropped", "offloaded", "reloaded", "compacted", "bytes_d2h", "bytes_h2d",
                 "bytes_d2d", "table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns",
@@ -156,6 +156,8 @@ class OracleEngine:
     def one_off(self, ctx, s=0, e=None):
         self._op("one_off", OP_ONE_OFF, ctx, msg_start=s, msg_end=0xFFFFFFFF if e is None else e)
 
+    def pin(self, ctx, s, e): self._op("pin", OP_PIN, ctx, msg_start=s, msg_end=e)
+    def unpin(self, ctx, s, e): self._op("unpin", OP_UNPIN, ctx, msg_start=s, msg_end=e)
     def prefill_done(self, ctx): self._op("prefill_done", OP_PREFILL_DONE, ctx)
     def terminate(self, ctx): self._op("terminate", OP_TERMINATE, ctx)
 
@@ -205,11 +207,12 @@ class OracleEngine:
             raise OracleError(rc, "classify_bruteforce")
         return st
 
-    def select_victims(self, tier, n_req):
+    def select_victims(self, tier, n_req, include_pinned=False):
         cap = min(n_req, self._tier_size(tier))
         slots = np.zeros(cap, np.uint32); states = np.zeros(cap, np.uint8)
         n = C.c_uint32(0)
-        rc = self.L.kvto_select_victims(self.h, tier, n_req, _p(slots), _p(states), cap, C.byref(n))
+        rc = self.L.kvto_select_victims(self.h, tier, n_req, 1 if include_pinned else 0, _p(slots), _p(states), cap,
+                                        C.byref(n))
         if rc:
             raise OracleError(rc, "select_victims")
         return slots[:n.value].copy(), states[:n.value].copy()

@@ -54,7 +54,7 @@ class Op(C.Structure):
 
 
 CALL_INFO_DTYPE = np.dtype([(n, np.uint32) for n in ("n_blocks", "hit_len", "n_hit_hbm", "n_hit_host",
-                                                       "n_admissible", "n_admitted", "n_held")])
+                                                       "n_admissible", "n_admitted", "n_held", "n_pinned")])
 STATS_FIELDS = ("clock", "n_contexts", "occ_hbm", "occ_host", "blocks_hashed", "hits_hbm", "hits_host", "misses",
                 "inserted", "adopted", "dropped", "offloaded", "reloaded", "compacted", "bytes_d2h", "bytes_h2d",
                 "bytes_d2d", "table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns",
@@ -81,7 +81,7 @@ def load_library():
             "kvt_get_block_map": [vp, u32, vp, vp, vp, u32, vp, vp],
             "kvt_classify": [vp, vp],
             "kvt_get_states": [vp, u32, vp, u32, vp],
-            "kvt_select_victims": [vp, u32, u32, vp, vp, u32, vp, vp],
+            "kvt_select_victims": [vp, u32, u32, u32, vp, vp, u32, vp, vp],
             "kvt_offload": [vp, vp, u32, vp, vp, vp],
             "kvt_reload": [vp, vp, u32, vp, vp],
             "kvt_release": [vp, u32, vp, u32, vp],
@@ -265,6 +265,8 @@ class Engine:
     def one_off(self, ctx, s=0, e=None):
         self._op("one_off", OP_ONE_OFF, ctx, msg_start=s, msg_end=0xFFFFFFFF if e is None else e)
 
+    def pin(self, ctx, s, e): self._op("pin", OP_PIN, ctx, msg_start=s, msg_end=e)
+    def unpin(self, ctx, s, e): self._op("unpin", OP_UNPIN, ctx, msg_start=s, msg_end=e)
     def prefill_done(self, ctx): self._op("prefill_done", OP_PREFILL_DONE, ctx)
     def terminate(self, ctx): self._op("terminate", OP_TERMINATE, ctx)
 
@@ -303,12 +305,12 @@ class Engine:
         self._check(self.L.kvt_get_states(self.h, tier, _p(st), len(st), _stream()), "get_states")
         return st
 
-    def select_victims(self, tier, n_req):
+    def select_victims(self, tier, n_req, include_pinned=False):
         cap = min(n_req, self._tier_size(tier))
         slots = np.zeros(cap, np.uint32); states = np.zeros(cap, np.uint8)
         n = C.c_uint32(0)
-        self._check(self.L.kvt_select_victims(self.h, tier, n_req, _p(slots), _p(states), cap, C.byref(n), _stream()),
-                    "select_victims")
+        self._check(self.L.kvt_select_victims(self.h, tier, n_req, 1 if include_pinned else 0, _p(slots), _p(states),
+                                              cap, C.byref(n), _stream()), "select_victims")
         return slots[:n.value].copy(), states[:n.value].copy()
 
     # ---- movement -------------------------------------------------------------------------------

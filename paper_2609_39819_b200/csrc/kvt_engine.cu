@@ -20,8 +20,9 @@ using namespace kvt;
 
 namespace {
 
-constexpr u32 MS_ACTIVE = 0, MS_SUSPENDED = 1, MS_TEMPORARY = 3;
-inline u8 msg_rank(u8 s) { return s == MS_ACTIVE ? 2 : (s == MS_SUSPENDED ? 1 : 0); }
+constexpr u32 MS_ACTIVE = 0, MS_SUSPENDED = 1, MS_EXPIRED = 2, MS_TEMPORARY = 3, MS_PINNED = 4;
+// Priority of a message state in the block aggregate: Algorithm 1's release order.
+inline u8 msg_rank(u8 s) { return s == MS_PINNED ? 3 : (s == MS_ACTIVE ? 2 : (s == MS_SUSPENDED ? 1 : 0)); }
 
 inline u64 round_up(u64 x, u64 a) { return (x + a - 1) / a * a; }
 inline u32 cdiv(u64 a, u64 b) { return (u32)((a + b - 1) / b); }
@@ -62,10 +63,11 @@ struct KeySeg { u64 off = 0, cap = 0; u32 refs = 0; };
 
 struct Ctx {
   bool live = false, one_off = false, in_flight = false;
+  bool terminated = false;   // ended but kept: it still has Pinned messages
   std::vector<Msg> msgs;
   std::vector<std::pair<u32, u32>> mat_bounds;  // bounds of the leading messages still valid in the materialised layout
   u32 mat_blocks = 0;      // blocks of the materialised token sequence (keys in the key segment)
-  u32 valid_blocks = 0, held = 0, hit_len = 0, n_hit_hbm = 0, n_hit_host = 0, n_admissible = 0;
+  u32 valid_blocks = 0, held = 0, hit_len = 0, n_hit_hbm = 0, n_hit_host = 0, n_admissible = 0, n_pinned = 0;
   u64 tok_off = 0, tok_cap = 0, tok_len = 0;   // device token buffer = concatenation of the current messages
   int keyseg = -1;
 };
@@ -203,8 +205,9 @@ int32_t status_code(kvt_engine *e) {
   return fail(e, KVT_E_STATE, "block is in flight");
 }
 
-Ctx *get_ctx(kvt_engine *e, u32 id) {
+Ctx *get_ctx(kvt_engine *e, u32 id, bool allow_terminated = false) {
   if (id >= e->ctxs.size() || !e->ctxs[id].live) return nullptr;
+  if (e->ctxs[id].terminated && !allow_terminated) return nullptr;
   return &e->ctxs[id];
 }
 
@@ -389,6 +392,22 @@ u32 first_temporary_block(const Ctx &c, u32 from, u32 n_blocks) {
   return n_blocks;
 }
 
+// Blocks in [from, to) touched by a non-empty Pinned message.
+u32 count_pinned_blocks(const Ctx &c, u32 from, u32 to) {
+  u64 pos = 0;
+  u32 n = 0;
+  int64_t last = -1;   // last block already counted
+  for (const Msg &m : c.msgs) {
+    if (m.len && m.state == MS_PINNED) {
+      int64_t b0 = std::max<int64_t>((int64_t)(pos / 16), std::max<int64_t>(from, last + 1));
+      int64_t b1 = std::min<int64_t>((int64_t)((pos + m.len - 1) / 16), (int64_t)to - 1);
+      if (b1 >= b0) { n += (u32)(b1 - b0 + 1); last = b1; }
+    }
+    pos += m.len;
+  }
+  return n;
+}
+
 }  // namespace
 
 // =========================================================================================================
@@ -552,8 +571,8 @@ int32_t kvt_apply_op(kvt_engine *e, const kvt_op *op, void *stream) {
     e->dirty = true;
     return KVT_OK;
   }
-  if (op->op == 0 || op->op >= KVT_OP_PIN) return fail(e, KVT_E_INVAL, "unknown or reserved op");
-  Ctx *c = get_ctx(e, id);
+  if (op->op == 0 || op->op > KVT_OP_UNPIN) return fail(e, KVT_E_INVAL, "unknown op");
+  Ctx *c = get_ctx(e, id, op->op == KVT_OP_UNPIN);   // a terminated context kept for its Pinned messages only accepts unpin
   if (!c) return fail(e, KVT_E_NOCTX, "unknown context");
   switch (op->op) {
     case KVT_OP_APPEND: {
@@ -612,7 +631,7 @@ int32_t kvt_apply_op(kvt_engine *e, const kvt_op *op, void *stream) {
       if (c->in_flight) return fail(e, KVT_E_STATE, "one_off: context is in flight");
       if (op->msg_start == 0 && op->msg_end == 0xFFFFFFFFu) {
         c->one_off = true;
-        for (Msg &m : c->msgs) m.state = MS_TEMPORARY;
+        for (Msg &m : c->msgs) if (m.state != MS_PINNED) m.state = MS_TEMPORARY;   // explicit protection stays
       } else {
         if (!(op->msg_start < op->msg_end && op->msg_end <= c->msgs.size())) return fail(e, KVT_E_RANGE, "one_off: bad message range");
         for (u32 j = op->msg_start; j < op->msg_end; ++j) c->msgs[j].state = MS_TEMPORARY;
@@ -633,8 +652,33 @@ int32_t kvt_apply_op(kvt_engine *e, const kvt_op *op, void *stream) {
     case KVT_OP_TERMINATE: {
       if (c->in_flight) { int32_t r = unlock_held(e, *c, s, false); if (r) return r; }
       if (c->tok_cap) e->tok_alloc.release(c->tok_off, c->tok_cap);
-      seg_deref(e, c->keyseg);
-      *c = Ctx();
+      c->tok_off = c->tok_cap = c->tok_len = 0;
+      bool pinned = false;
+      for (Msg &m : c->msgs) { if (m.state == MS_PINNED) pinned = true; else m.state = MS_EXPIRED; }
+      if (pinned) {            // Pinned messages retain their protection: keep the mapping, drop the rest
+        c->terminated = true;
+        c->in_flight = false;
+      } else {
+        seg_deref(e, c->keyseg);
+        *c = Ctx();
+      }
+      e->dirty = true;
+      return KVT_OK;
+    }
+    case KVT_OP_PIN:
+    case KVT_OP_UNPIN: {
+      if (c->in_flight) return fail(e, KVT_E_STATE, "pin/unpin: context is in flight");
+      if (!(op->msg_start < op->msg_end && op->msg_end <= c->msgs.size())) return fail(e, KVT_E_RANGE, "pin/unpin: bad message range");
+      for (u32 j = op->msg_start; j < op->msg_end; ++j) {
+        Msg &m = c->msgs[j];
+        if (op->op == KVT_OP_PIN) m.state = MS_PINNED;
+        else if (m.state == MS_PINNED) m.state = c->terminated ? MS_EXPIRED : (c->one_off ? MS_TEMPORARY : MS_SUSPENDED);
+      }
+      if (c->terminated) {
+        bool pinned = false;
+        for (const Msg &m : c->msgs) pinned = pinned || m.state == MS_PINNED;
+        if (!pinned) { seg_deref(e, c->keyseg); *c = Ctx(); }
+      }
       e->dirty = true;
       return KVT_OK;
     }
@@ -729,9 +773,10 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     c.n_hit_host = k >= 0 ? h_host[k] : 0;
     c.held = c.hit_len;
     c.n_admissible = first_temporary_block(c, c.hit_len, c.mat_blocks) - c.hit_len;
+    c.n_pinned = count_pinned_blocks(c, c.hit_len, c.hit_len + c.n_admissible);
     e->st.blocks_hashed += c.mat_blocks;
     e->st.hits_hbm += c.n_hit_hbm; e->st.hits_host += c.n_hit_host; e->st.misses += c.mat_blocks - c.hit_len;
-    out[i] = kvt_call_info{c.mat_blocks, c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, 0, c.held};
+    out[i] = kvt_call_info{c.mat_blocks, c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, 0, c.held, c.n_pinned};
   }
   return KVT_OK;
 }
@@ -818,7 +863,7 @@ static int32_t map_admit(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_info
   for (u32 i = 0; i < n_ctx; ++i) {
     Ctx &c = e->ctxs[ids[i]];
     c.held = cur[i];
-    out[i] = kvt_call_info{c.mat_blocks, c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, cur[i] - held0[i], c.held};
+    out[i] = kvt_call_info{c.mat_blocks, c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, cur[i] - held0[i], c.held, c.n_pinned};
   }
   return rc;
 }
@@ -845,7 +890,7 @@ int32_t kvt_map_blocks(kvt_engine *e, const uint32_t *ctx_ids, uint32_t n_ctx, u
 int32_t kvt_get_block_map(kvt_engine *e, uint32_t ctx, uint64_t *keys, uint8_t *tier, uint32_t *slot, uint32_t cap,
                           uint32_t *n, void *stream) {
   if (!e || !n) return KVT_E_INVAL;
-  Ctx *c = get_ctx(e, ctx);
+  Ctx *c = get_ctx(e, ctx, true);
   if (!c) return fail(e, KVT_E_NOCTX, "get_block_map: unknown context");
   cudaStream_t s = (cudaStream_t)stream;
   u32 nb = c->mat_blocks;
@@ -904,9 +949,9 @@ int32_t kvt_get_entries(kvt_engine *e, uint32_t tier, uint64_t *keys, uint32_t *
 }
 
 // ---- stage 4 -----------------------------------------------------------------------------------------------
-int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_t *slots_out, uint8_t *states_out,
-                           uint32_t cap, uint32_t *n_out, void *stream) {
-  if (!e || tier > 1 || !n_out || (!slots_out && cap)) return KVT_E_INVAL;
+int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_t flags, uint32_t *slots_out,
+                           uint8_t *states_out, uint32_t cap, uint32_t *n_out, void *stream) {
+  if (!e || tier > 1 || flags > 1 || !n_out || (!slots_out && cap)) return KVT_E_INVAL;
   *n_out = 0;
   u32 n = e->tier_slots(tier);
   if (!n || !n_req) return KVT_OK;
@@ -919,6 +964,7 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   a.ent = e->ent; a.e0 = e->tier_e0(tier); a.n_slots = n; a.n_req = n_req; a.now = e->now;
   a.stamp_bits = bit_length(e->now); a.depth_bits = bit_length(e->max_depth);
   a.mru = e->cfg.suspended_order == KVT_ORDER_MRU; a.status = e->d_status;
+  a.max_rank = (flags & KVT_SEL_INCLUDE_PINNED) ? 3 : 2;
   u64 *kA = e->dp<u64>(e->L.keyA), *kB = e->dp<u64>(e->L.keyB);
   u32 *vA = e->dp<u32>(e->L.valA), *vB = e->dp<u32>(e->L.valB), *counts = e->dp<u32>(e->L.rcounts);
   u32 *row_total = counts + 256ull * (e->L.Nt / SORT_TILE + 1);
@@ -946,7 +992,7 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   }
   r = status_code(e);
   if (r) return r;
-  u64 total = (u64)e->h_status[ST_RANK0] + e->h_status[ST_RANK1] + e->h_status[ST_RANK2];
+  u64 total = (u64)e->h_status[ST_RANK0] + e->h_status[ST_RANK1] + e->h_status[ST_RANK2] + e->h_status[ST_RANK3];
   u32 k = (u32)std::min<u64>(n_req, total);
   *n_out = k;
   if (cap < k) return KVT_E_BUFSZ;
@@ -1170,7 +1216,7 @@ int32_t kvt_debug_load_resident(kvt_engine *e, const uint64_t *keys, const uint8
         std::adjacent_find(ss.begin(), ss.end()) != ss.end() || ss.back() >= ns)
       return fail(e, KVT_E_INVAL, "bad keys or slots");
     for (u32 i = 0; i < n; ++i) {
-      if (state[i] > 2) return fail(e, KVT_E_INVAL, "bad state");
+      if (state[i] > 3) return fail(e, KVT_E_INVAL, "bad state");
       max_stamp = std::max(max_stamp, stamp[i]); max_d = std::max(max_d, depth[i]);
     }
   }

@@ -29,7 +29,7 @@ enum : u32 { DERR_PROBE = 1, DERR_RANGE = 2, DERR_INVAL = 4, DERR_STATE = 8, DER
 // words of the device status block
 enum : int {
   ST_ERR = 0, ST_TOTAL, ST_CUT, ST_NLIVE, ST_NDROP, ST_NEW, ST_INSERTED, ST_ADOPTED, ST_TOMBS,
-  ST_RANK0, ST_RANK1, ST_RANK2, ST_M, ST_NMOVED, ST_FREE, ST_AUX, ST_WORDS = 32
+  ST_RANK0, ST_RANK1, ST_RANK2, ST_RANK3, ST_M, ST_NMOVED, ST_FREE, ST_AUX, ST_WORDS = 32
 };
 
 struct __align__(16) TSlot { u64 key; u32 ent; u32 pad; };
@@ -516,13 +516,14 @@ __global__ void k_classify(ClsArgs a) {
 }
 
 // ======================================================================================================
-// K4: victim selection. Candidates of a tier: resident, not in flight, rank < 3. Whole ranks below the
+// K4: victim selection. Candidates of a tier: resident, not in flight, rank <= max_rank (2, or 3 when the
+// incoming KV is Pinned). Whole ranks below the
 // boundary rank are taken, the ordered compaction keeps slot order, and a stable LSD radix sort on the
 // packed (rank, recency, inverted depth) key orders them; ties therefore end slot-ascending.
 // ======================================================================================================
 struct SelArgs {
   Entries ent; u32 e0, n_slots;       // entry range of the tier
-  u32 n_req; u32 now; u32 stamp_bits, depth_bits; u32 mru;
+  u32 n_req; u32 now; u32 stamp_bits, depth_bits; u32 mru; u32 max_rank;
   u32 *status;
 };
 
@@ -531,22 +532,22 @@ __device__ __forceinline__ bool sel_candidate(const SelArgs &a, u32 i, u32 *rank
   if (!a.ent.key[e] || a.ent.infl[e]) return false;
   u32 r = a.ent.rank[e];
   *rank = r;
-  return r < 3;
+  return r <= a.max_rank;
 }
 
 __global__ void k_sel_count(SelArgs a) {
-  __shared__ u32 s[3];
-  if (threadIdx.x < 3) s[threadIdx.x] = 0;
+  __shared__ u32 s[4];
+  if (threadIdx.x < 4) s[threadIdx.x] = 0;
   __syncthreads();
   u32 i = blockIdx.x * blockDim.x + threadIdx.x;
   u32 r = 0;
   bool c = i < a.n_slots && sel_candidate(a, i, &r);
-  for (u32 k = 0; k < 3; ++k) {
+  for (u32 k = 0; k < 4; ++k) {
     u32 m = __ballot_sync(0xFFFFFFFFu, c && r == k);
     if ((threadIdx.x & 31) == 0 && m) atomicAdd(&s[k], __popc(m));
   }
   __syncthreads();
-  if (threadIdx.x < 3 && s[threadIdx.x]) atomicAdd(&a.status[ST_RANK0 + threadIdx.x], s[threadIdx.x]);
+  if (threadIdx.x < 4 && s[threadIdx.x]) atomicAdd(&a.status[ST_RANK0 + threadIdx.x], s[threadIdx.x]);
 }
 
 // Highest rank that must be looked at to serve n_req victims (Algorithm 1: lower ranks go first).
@@ -555,7 +556,9 @@ __device__ __forceinline__ u32 sel_boundary_rank(const u32 *status, u32 n_req) {
   if (cum >= n_req) return 0;
   cum += status[ST_RANK1];
   if (cum >= n_req) return 1;
-  return 2;
+  cum += status[ST_RANK2];
+  if (cum >= n_req) return 2;
+  return 3;
 }
 
 struct PredSel {

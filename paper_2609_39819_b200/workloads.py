@@ -64,6 +64,7 @@ GEO_GLM = Geometry("glm-92x8x128", 92, 8, 128)      # 5.75 MiB / block (368 KiB 
 # Traces: lists of events
 #   ("spawn", ctx) ("fork", parent, child, end) ("append", ctx, tokens) ("replace", ctx, s, e, tokens)
 #   ("remove", ctx, s, e) ("one_off", ctx, s, e_or_None) ("terminate", ctx) ("call", [ctx, ...])
+#   ("pin", ctx, s, e) ("unpin", ctx, s, e)
 # A "call" is one LLM call per listed context, carried through the whole cache path by `replay`.
 # ------------------------------------------------------------------------------------------------
 def _tokens(rng, n):
@@ -78,16 +79,21 @@ def trace_c1(seed: int):
     """C1: one root context, 3 calls, 2-6 appended messages of 50-400 tokens per call; per appended
     message replace (p=0.1), remove (p=0.05) or fork a subagent (p=0.05). A subagent appends 1-2
     messages (one_off with p=0.5), runs one call, idles through the parent's next call, then appends
-    once more, runs a second call and terminates."""
+    once more, runs a second call and terminates. Every third seed pins the root's first message
+    right after appending it (a system prompt); every sixth unpins it again before the last call."""
     rng = np.random.default_rng([1, seed])
     ev = [("spawn", 0)]
     n_msgs = 0
     next_ctx = 1
     pending = []
     for _call in range(3):
+        if _call == 2 and seed % 6 == 0:
+            ev.append(("unpin", 0, 0, 1))
         for _ in range(int(rng.integers(2, 7))):
             ev.append(("append", 0, _tokens(rng, rng.integers(50, 401))))
             n_msgs += 1
+            if n_msgs == 1 and _call == 0 and seed % 3 == 0:
+                ev.append(("pin", 0, 0, 1))
             u = rng.random()
             if u < 0.10 and n_msgs:
                 j = int(rng.integers(0, n_msgs))
@@ -164,6 +170,8 @@ def trace_c3(seed: int, n_sessions: int = 32, min_len: int = 32768, max_len: int
         n = max(16, int(600 * scale))
         ev.append(("append", s, _tokens(rng, n)))
         lens[s].append(n)
+        if s % 4 == 0:
+            ev.append(("pin", s, 0, 1))   # every fourth session pins its system prompt
     live = set(range(n_sessions))
     while live:
         batch = []
@@ -288,11 +296,15 @@ class ReplayOptions:
     counters: dict = field(default_factory=dict)
 
 
-def evict(eng, n):
+def evict(eng, n, n_pinned_incoming=0):
     """Frees n HBM slots in the engine's victim order: dead blocks are dropped, live ones go to the
-    host tier, for which room is made first by releasing the host tier's own first victims."""
+    host tier, for which room is made first by releasing the host tier's own first victims. Pinned
+    blocks are only asked for when Pinned blocks are coming in, and only for as many (Algorithm 1)."""
     rec = {}
     victims, vstates = eng.select_victims(TIER_HBM, n)
+    if len(victims) < n and n_pinned_incoming > 0:
+        want = len(victims) + min(n - len(victims), n_pinned_incoming)
+        victims, vstates = eng.select_victims(TIER_HBM, want, include_pinned=True)
     rec["victims"] = victims.copy()
     rec["vstates"] = vstates.copy()
     n_live = int((vstates > 0).sum())
@@ -319,7 +331,7 @@ def run_call(eng, ctxs, opt: ReplayOptions):
     free_hbm = eng.n_hbm_blocks - st["occ_hbm"]
     need = int(info["n_hit_host"].sum()) + int(info["n_admissible"].sum()) - free_hbm
     if need > 0:
-        rec.update(evict(eng, need))
+        rec.update(evict(eng, need, int(info["n_pinned"].sum())))
     host_slots = []
     for c, inf in zip(ctxs, info):
         if inf["n_hit_host"]:
@@ -382,6 +394,10 @@ def replay(eng, trace, opt: ReplayOptions | None = None):
             eng.one_off(ev[1], ev[2], ev[3]); rec = None
         elif kind == "terminate":
             eng.terminate(ev[1]); rec = None
+        elif kind == "pin":
+            eng.pin(ev[1], ev[2], ev[3]); rec = None
+        elif kind == "unpin":
+            eng.unpin(ev[1], ev[2], ev[3]); rec = None
         elif kind == "call":
             rec = run_call(eng, ev[1], opt)
         else:

@@ -7,7 +7,7 @@ import numpy as np
 
 HBM, HOST = 0, 1
 LOOKUP, ADMIT = 0, 1
-DEAD, IDLE, ACTIVE, FREE = 0, 1, 2, 0xFF
+DEAD, IDLE, ACTIVE, PINNED, FREE = 0, 1, 2, 3, 0xFF
 E_INVAL, E_NOCTX, E_RANGE, E_STATE, E_NOSPACE, E_BUFSZ = -1, -2, -3, -4, -5, -6
 
 TOY = dict(n_layers=2, n_kv_heads=2, head_dim=64)
@@ -151,6 +151,75 @@ def one_off_bypass(make):
     a, b = call(eng, 0, done=False)
     assert (a["hit_len"], a["n_admissible"]) == (6, 0)
     eng.prefill_done(0)
+
+
+# ---- pin / unpin: explicit retention (Table 3; Section 5.2; Algorithm 1's last branch) ---------------
+def pinned_retention(make):
+    eng = make(n_hbm_blocks=8, n_host_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(15)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 32))                         # system message: blocks 0, 1
+    eng.pin(0, 0, 1)                                     # pinned at initialisation (Section 4.2)
+    eng.append(0, toks(rng, 32))                         # blocks 2, 3
+    a, b = call(eng, 0, done=False)
+    assert (a["n_admissible"], a["n_pinned"], b["n_held"]) == (4, 2, 4)
+    assert states(eng)[:4] == [PINNED, PINNED, ACTIVE, ACTIVE]
+    eng.prefill_done(0)
+    assert states(eng)[:4] == [PINNED, PINNED, IDLE, IDLE]      # prefill-done does not touch Pinned messages
+    v, s = eng.select_victims(HBM, 8)
+    assert list(v) == [3, 2] and list(s) == [1, 1]              # Pinned KV is out of ordinary contention
+    v, s = eng.select_victims(HBM, 8, include_pinned=True)
+    assert list(v) == [3, 2, 1, 0] and list(s) == [1, 1, 3, 3]  # it competes last, oldest / deepest first
+    eng.map_blocks([0], LOOKUP)
+    assert states(eng)[:4] == [PINNED, PINNED, ACTIVE, ACTIVE]
+    eng.map_blocks([0], ADMIT)
+    eng.prefill_done(0)
+    # unpin between calls: back to Suspended
+    eng.unpin(0, 0, 1)
+    assert states(eng)[:4] == [IDLE] * 4
+    eng.pin(0, 0, 2)
+    assert states(eng)[:4] == [PINNED] * 4
+    eng.unpin(0, 1, 2)
+    # termination: ordinary messages expire, Pinned ones keep their protection
+    eng.terminate(0)
+    assert states(eng)[:4] == [PINNED, PINNED, DEAD, DEAD]
+    assert eng.get_stats()["n_contexts"] == 1
+    assert eng.apply_op_rc(3, 0, tokens=toks(rng, 4)) == E_NOCTX     # (3 = append) the context has ended
+    assert eng.apply_op_rc(1, 0) == E_INVAL                          # (1 = spawn) its id is still in use
+    assert eng.map_blocks_rc([0], LOOKUP)[0] == E_NOCTX
+    # releasing the protection of a terminated context: Expired, and the context goes away
+    eng.unpin(0, 0, 1)
+    assert states(eng)[:4] == [DEAD] * 4
+    assert eng.get_stats()["n_contexts"] == 0
+    eng.spawn(0)
+
+
+def pinned_competes_only_with_pinned(make, run_call, options):
+    eng = make(n_hbm_blocks=4, n_host_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(16)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 64))
+    eng.pin(0, 0, 1)
+    run_call(eng, [0], options())                       # 4 pinned blocks fill the pool
+    assert states(eng) == [PINNED] * 4
+    eng.spawn(1)
+    eng.append(1, toks(rng, 32))
+    rec = run_call(eng, [1], options())                  # ordinary KV cannot displace Pinned KV
+    assert int(rec["admit"][0]["n_admitted"]) == 0 and len(rec["victims"]) == 0
+    assert states(eng) == [PINNED] * 4
+    eng.spawn(2)
+    eng.append(2, toks(rng, 32))
+    eng.pin(2, 0, 1)
+    rec = run_call(eng, [2], options())                  # Pinned incoming KV competes with Pinned residents
+    assert list(rec["victims"]) == [3, 2] and list(rec["vstates"]) == [3, 3]
+    assert rec["offload"] == (0, 2, 0)                   # live: moved to the host tier, not dropped
+    assert int(rec["admit"][0]["n_admitted"]) == 2
+    assert states(eng) == [PINNED] * 4 and states(eng, HOST)[:2] == [PINNED, PINNED]
+    # one_off on a context does not strip explicit protection
+    eng.one_off(2)
+    assert states(eng)[2:] == [PINNED, PINNED]
+    eng.one_off(2, 0, 1)                                 # the per-message declaration does
+    assert states(eng)[2:] == [DEAD, DEAD]
 
 
 # ---- hand-worked lifecycle example (8-block pool) --------------------------------------------------
@@ -431,13 +500,15 @@ def error_codes(make, op_codes):
     assert eng.apply_op_rc(OP["SPAWN"], 9) == E_INVAL    # id out of range
     eng.spawn(0)
     assert eng.apply_op_rc(OP["SPAWN"], 0) == E_INVAL    # id in use
-    assert eng.apply_op_rc(OP["PIN"], 0) == E_INVAL and eng.apply_op_rc(OP["UNPIN"], 0) == E_INVAL
-    assert eng.apply_op_rc(77, 0) == E_INVAL
+    assert eng.apply_op_rc(77, 0) == E_INVAL and eng.apply_op_rc(0, 0) == E_INVAL
     eng.append(0, toks(rng, 40))
     assert eng.apply_op_rc(OP["REMOVE"], 0, msg_start=0, msg_end=2) == E_RANGE
     assert eng.apply_op_rc(OP["REMOVE"], 0, msg_start=1, msg_end=1) == E_RANGE
     assert eng.apply_op_rc(OP["REPLACE"], 0, msg_start=1, msg_end=2, tokens=toks(rng, 4)) == E_RANGE
     assert eng.apply_op_rc(OP["ONE_OFF"], 0, msg_start=0, msg_end=5) == E_RANGE
+    assert eng.apply_op_rc(OP["PIN"], 0, msg_start=0, msg_end=2) == E_RANGE
+    assert eng.apply_op_rc(OP["UNPIN"], 0, msg_start=1, msg_end=1) == E_RANGE
+    assert eng.apply_op_rc(OP["PIN"], 2, msg_start=0, msg_end=1) == E_NOCTX
     assert eng.apply_op_rc(OP["FORK"], 1, parent=0, msg_end=2) == E_RANGE
     assert eng.apply_op_rc(OP["FORK"], 1, parent=3, msg_end=0) == E_NOCTX
     assert eng.apply_op_rc(OP["FORK"], 0, parent=0, msg_end=0) == E_INVAL
@@ -448,7 +519,7 @@ def error_codes(make, op_codes):
     assert eng.get_stats()["clock"] == 0                 # rejected calls change nothing
     eng.map_blocks([0], LOOKUP)
     assert eng.map_blocks_rc([0], LOOKUP)[0] == E_STATE
-    for op in ("APPEND", "REPLACE", "REMOVE", "ONE_OFF"):
+    for op in ("APPEND", "REPLACE", "REMOVE", "ONE_OFF", "PIN", "UNPIN"):
         assert eng.apply_op_rc(OP[op], 0, msg_start=0, msg_end=1, tokens=toks(rng, 4)) == E_STATE
     assert eng.apply_op_rc(OP["FORK"], 1, parent=0, msg_end=1) == E_STATE
     eng.map_blocks([0], ADMIT)                           # 2 blocks at slots 0, 1, in flight
@@ -499,4 +570,4 @@ def degenerate_inputs(make):
 ALL = [state_machine_single_context, suffix_invalidation, fork_and_shared_kv, one_off_bypass, worked_example,
        mixed_pool_example, victim_order_bruteforce, one_state_pools_reduce_to_lru, offload_reload_round_trip,
        dead_victims_are_dropped_without_copy, compaction, raw_copy_blocks, admission_stops_when_full,
-       lookup_locks_and_orphans, degenerate_inputs]
+       lookup_locks_and_orphans, degenerate_inputs, pinned_retention]

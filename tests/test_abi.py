@@ -39,4 +39,4 @@ def test_struct_sizes_match_the_header():
     from paper_2609_39819_b200 import binding
     assert ctypes.sizeof(binding.Config) == 14 * 4 + 3 * 8 + 2 * 4 + 8 * 8
     assert ctypes.sizeof(binding.Op) == 8 * 4 + 8
-    assert binding.CALL_INFO_DTYPE.itemsize == 7 * 4
+    assert binding.CALL_INFO_DTYPE.itemsize == 8 * 4

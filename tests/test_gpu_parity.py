@@ -35,6 +35,10 @@ def test_scenario(make_gpu, scenario):
     scenario(make_gpu)
 
 
+def test_pinned_competes_only_with_pinned(make_gpu):
+    S.pinned_competes_only_with_pinned(make_gpu, W.run_call, lambda: W.ReplayOptions(payload=None, record_states=False))
+
+
 def test_mixed_pool_lru_switch(make_gpu):
     S.mixed_pool_example(make_gpu, order=1)
 

@@ -17,6 +17,10 @@ def test_scenario(make, scenario):
     scenario(make)
 
 
+def test_pinned_competes_only_with_pinned(make):
+    S.pinned_competes_only_with_pinned(make, W.run_call, lambda: W.ReplayOptions(payload=None, record_states=False))
+
+
 def test_mixed_pool_lru_switch(make):
     S.mixed_pool_example(make, order=1)
 
@@ -90,7 +94,12 @@ def test_scaled_c2_and_c3_traces_replay(make):
     for _i, kind, rec in W.replay(eng, trace, W.ReplayOptions(payload=None, record_states=False)):
         pass
     check_invariants(eng)
+    # sessions 0 and 4 pinned their system prompt: they outlive their termination until it is unpinned
+    assert eng.get_stats()["n_contexts"] == 2 and int((eng.get_states(0) == 3).sum() + (eng.get_states(1) == 3).sum()) > 0
+    eng.unpin(0, 0, 1)
+    eng.unpin(4, 0, 1)
     assert eng.get_stats()["n_contexts"] == 0
+    assert int((eng.get_states(0) == 3).sum() + (eng.get_states(1) == 3).sum()) == 0
 
 
 def test_incremental_appends_hash_like_one_shot(make, oracle):
