@@ -135,7 +135,7 @@ struct kvt_engine {
   std::string err;
   // pinned host staging
   u8 *stage = nullptr;
-  u32 *h_status; u8 *h_desc; u32 *h_ctxres; u32 *h_mstart, *h_mend; u8 *h_mrank; u32 *h_ids, *h_ids2;
+  u32 *h_status; u8 *h_desc; u32 *h_ctxres; u32 *h_mstart, *h_mend; u8 *h_mrank; u32 *h_ids, *h_ids2; u8 *h_out;   // h_out: results staged for the caller (block maps, victim lists)
   cudaEvent_t ev_upload = nullptr;
   bool upload_pending = false;
   // optional timing of the mover kernel (kvt_set_profiling)
@@ -466,11 +466,12 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   u64 C = c.max_contexts, Mm = c.max_messages, LB = L.LB;
   u64 o_status = 0, o_desc = 256, o_ctxres = o_desc + round_up(C * 32, 256), o_ms = o_ctxres + round_up(C * 16, 256),
       o_me = o_ms + round_up(Mm * 4, 256), o_mr = o_me + round_up(Mm * 4, 256), o_ids = o_mr + round_up(Mm, 256),
-      o_ids2 = o_ids + round_up(LB * 4, 256), total = o_ids2 + round_up(LB * 4, 256);
+      o_ids2 = o_ids + round_up(LB * 4, 256), o_out = o_ids2 + round_up(LB * 4, 256),
+      total = o_out + round_up(LB * 16, 256);
   if (cudaHostAlloc((void **)&e->stage, total, cudaHostAllocDefault) != cudaSuccess) { delete e; return KVT_E_CUDA; }
   e->h_status = (u32 *)(e->stage + o_status); e->h_desc = e->stage + o_desc; e->h_ctxres = (u32 *)(e->stage + o_ctxres);
   e->h_mstart = (u32 *)(e->stage + o_ms); e->h_mend = (u32 *)(e->stage + o_me); e->h_mrank = e->stage + o_mr;
-  e->h_ids = (u32 *)(e->stage + o_ids); e->h_ids2 = (u32 *)(e->stage + o_ids2);
+  e->h_ids = (u32 *)(e->stage + o_ids); e->h_ids2 = (u32 *)(e->stage + o_ids2); e->h_out = e->stage + o_out;
   cudaStream_t s = (cudaStream_t)stream;
   bool ok = cudaEventCreateWithFlags(&e->ev_upload, cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreate(&e->ev_m0) == cudaSuccess && cudaEventCreate(&e->ev_m1) == cudaSuccess &&
@@ -903,12 +904,19 @@ int32_t kvt_get_block_map(kvt_engine *e, uint32_t ctx, uint64_t *keys, uint8_t *
   if (r) return r;
   KL(k_block_map, cdiv(nb,256), 256, s, e->tab, e->ent, dk, nb, e->dp<u8>(e->L.map_tier), e->dp<u32>(e->L.map_slot), e->d_status);
   LAUNCH_CHECK();
-  if (keys) CU(cudaMemcpyAsync(keys, dk, nb * 8ull, cudaMemcpyDeviceToHost, s));
-  if (tier) CU(cudaMemcpyAsync(tier, e->dp<u8>(e->L.map_tier), nb, cudaMemcpyDeviceToHost, s));
-  if (slot) CU(cudaMemcpyAsync(slot, e->dp<u32>(e->L.map_slot), nb * 4ull, cudaMemcpyDeviceToHost, s));
+  // results go through pinned staging: one synchronisation for everything
+  u64 *hk = (u64 *)e->h_out; u32 *hs = (u32 *)(e->h_out + nb * 8ull); u8 *ht = e->h_out + nb * 12ull;
+  if (keys) CU(cudaMemcpyAsync(hk, dk, nb * 8ull, cudaMemcpyDeviceToHost, s));
+  if (slot) CU(cudaMemcpyAsync(hs, e->dp<u32>(e->L.map_slot), nb * 4ull, cudaMemcpyDeviceToHost, s));
+  if (tier) CU(cudaMemcpyAsync(ht, e->dp<u8>(e->L.map_tier), nb, cudaMemcpyDeviceToHost, s));
   r = status_fetch(e, s);
   if (r) return r;
-  return status_code(e);
+  r = status_code(e);
+  if (r) return r;
+  if (keys) std::memcpy(keys, hk, nb * 8ull);
+  if (slot) std::memcpy(slot, hs, nb * 4ull);
+  if (tier) std::memcpy(tier, ht, nb);
+  return KVT_OK;
 }
 
 // ---- stage 3 -----------------------------------------------------------------------------------------------
@@ -984,6 +992,10 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
                                                e->dp<u8>(e->L.out_states));
   if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));
   LAUNCH_CHECK();
+  // the victim list (at most n_emit entries) travels with the status block: one synchronisation
+  u32 *h_slots = (u32 *)e->h_out; u8 *h_states = e->h_out + n_emit * 4ull;
+  CU(cudaMemcpyAsync(h_slots, e->dp<u32>(e->L.out_slots), n_emit * 4ull, cudaMemcpyDeviceToHost, s));
+  if (states_out) CU(cudaMemcpyAsync(h_states, e->dp<u8>(e->L.out_states), n_emit, cudaMemcpyDeviceToHost, s));
   r = status_fetch(e, s);
   if (r) return r;
   if (e->profiling) {
@@ -997,9 +1009,8 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   *n_out = k;
   if (cap < k) return KVT_E_BUFSZ;
   if (k) {
-    CU(cudaMemcpyAsync(slots_out, e->dp<u32>(e->L.out_slots), k * 4ull, cudaMemcpyDeviceToHost, s));
-    if (states_out) CU(cudaMemcpyAsync(states_out, e->dp<u8>(e->L.out_states), k, cudaMemcpyDeviceToHost, s));
-    CU(cudaStreamSynchronize(s));
+    std::memcpy(slots_out, h_slots, k * 4ull);
+    if (states_out) std::memcpy(states_out, h_states, k);
   }
   return KVT_OK;
 }
