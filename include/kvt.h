@@ -71,6 +71,12 @@ extern "C" {
 #define KVT_ORDER_MRU 0u   /* most recently suspended first (the paper's policy, default) */
 #define KVT_ORDER_LRU 1u   /* oldest first */
 
+/* kvt_config.policy_flags */
+#define KVT_POLICY_NO_LIFECYCLE 1u  /* the "w/o LT" ablation of Section 8.3: no lifecycle information reaches the
+                                       policy. Every resident block is one tier ordered by suspended_order alone,
+                                       offload copies every victim (nothing is known to be dead) and nothing bypasses
+                                       admission. kvt_get_states still reports the true states (for metrics). */
+
 /* Primitives and runtime events (Table 3; Section 5.2 "Runtime transitions"). */
 #define KVT_OP_SPAWN         1u  /* register an independent, empty context */
 #define KVT_OP_FORK          2u  /* register child `ctx` sharing messages [0, msg_end) of `parent` */
@@ -122,7 +128,7 @@ typedef struct kvt_config {
   uint32_t max_contexts;     /* context ids are 0 .. max_contexts-1 */
   uint32_t max_messages;     /* upper bound on messages with materialised positions, all contexts together */
   uint32_t max_batch_blocks; /* upper bound on the blocks hashed by one kvt_map_blocks call and on n of one list call */
-  uint32_t reserved0;        /* must be 0 */
+  uint32_t policy_flags;     /* KVT_POLICY_* (0 = the paper's policy) */
   uint64_t max_tokens;       /* capacity of the device token arena, in tokens */
   uint64_t max_key_blocks;   /* capacity of the per-context key lists, in blocks (all contexts together) */
   uint64_t hash_seed;        /* seed of the block hash */

@@ -42,6 +42,7 @@ enum : int32_t {
 enum : uint32_t { TIER_HBM = 0, TIER_HOST = 1 };
 enum : uint32_t { LAYOUT_LAYER_MAJOR = 0, LAYOUT_BLOCK_MAJOR = 1 };
 enum : uint32_t { ORDER_MRU = 0, ORDER_LRU = 1 };
+enum : uint32_t { POLICY_NO_LIFECYCLE = 1 };   // the "w/o LT" variant of Section 8.3
 enum : uint32_t {
   OP_SPAWN = 1, OP_FORK, OP_APPEND, OP_REPLACE, OP_REMOVE, OP_ONE_OFF, OP_PREFILL_DONE,
   OP_TERMINATE, OP_PIN, OP_UNPIN
@@ -118,7 +119,7 @@ struct Entry { uint64_t key = 0; uint32_t stamp = 0, depth = 0, inflight = 0; ui
 
 struct Config {
   uint32_t n_layers, n_kv_heads, head_dim, elem_bytes, pool_layout;
-  uint32_t n_hbm_blocks, n_host_blocks, max_contexts, suspended_order, reserved;
+  uint32_t n_hbm_blocks, n_host_blocks, max_contexts, suspended_order, policy_flags;
   uint64_t hash_seed;
   uint8_t *hbm_pool; uint8_t *host_pool;  // host memory; NULL = metadata only
 };
@@ -246,7 +247,7 @@ extern "C" {
 int32_t kvto_create(const Config *cfg, Engine **out) {
   if (!cfg || !out) return E_INVAL;
   if (!cfg->n_layers || !cfg->n_kv_heads || !cfg->head_dim || !cfg->elem_bytes || !cfg->n_hbm_blocks ||
-      !cfg->max_contexts || cfg->pool_layout > 1 || cfg->suspended_order > 1)
+      !cfg->max_contexts || cfg->pool_layout > 1 || cfg->suspended_order > 1 || cfg->policy_flags > 1)
     return E_INVAL;
   Engine *e = new Engine();
   e->cfg = *cfg;
@@ -453,7 +454,11 @@ int32_t kvto_map_blocks(Engine *e, const uint32_t *ids, uint32_t n_ctx, uint32_t
       block_ranks(c, c.mat_bounds, nb, br);
       uint32_t a = h;
       c.n_pinned = 0;
-      while (a < nb && br[a] != 0) { c.n_pinned += br[a] == 3; ++a; }
+      if (e->cfg.policy_flags & POLICY_NO_LIFECYCLE) {
+        a = nb;   // no lifecycle information: nothing is known to be Temporary, everything is admitted
+      } else {
+        while (a < nb && br[a] != 0) { c.n_pinned += br[a] == 3; ++a; }
+      }
       c.n_admissible = a - h;
       e->st.blocks_hashed += nb;
       e->st.hits_hbm += c.n_hit_hbm;
@@ -553,6 +558,8 @@ int32_t kvto_select_victims(Engine *e, uint32_t tier, uint32_t n_req, uint32_t f
   const int max_rank = (flags & 1) ? 3 : 2;   // Pinned KV competes only when the incoming KV is Pinned
   std::vector<uint8_t> rank[2];
   classify(*e, rank);
+  if (e->cfg.policy_flags & POLICY_NO_LIFECYCLE)   // without lifecycle tracking every resident block is one tier
+    for (uint8_t &r : rank[tier]) if (r != 0xFF) r = 1;
   struct Cand { uint32_t slot; uint8_t rank; uint32_t stamp, depth; };
   std::vector<Cand> cands;
   for (uint32_t s = 0; s < tier_size(*e, tier); ++s) {
@@ -612,9 +619,10 @@ int32_t kvto_offload(Engine *e, const uint32_t *slots, uint32_t n, uint32_t *n_d
   if (v != OK) return v;
   std::vector<uint8_t> rank[2];
   classify(*e, rank);
+  const bool knows_dead = !(e->cfg.policy_flags & POLICY_NO_LIFECYCLE);
   for (uint32_t i = 0; i < n; ++i) {
     uint32_t s = slots[i];
-    if (rank[0][s] == 0) {  // reclaim dead KV without a copy
+    if (knows_dead && rank[0][s] == 0) {  // reclaim dead KV without a copy
       free_slot(*e, TIER_HBM, s);
       e->st.dropped++;
       (*n_dropped)++;

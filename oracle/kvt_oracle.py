@@ -20,6 +20,7 @@ OK, E_INVAL, E_NOCTX, E_RANGE, E_STATE, E_NOSPACE, E_BUFSZ = 0, -1, -2, -3, -4, 
 TIER_HBM, TIER_HOST, TIER_NONE = 0, 1, 0xFF
 LAYOUT_LAYER_MAJOR, LAYOUT_BLOCK_MAJOR = 0, 1
 ORDER_MRU, ORDER_LRU = 0, 1
+POLICY_NO_LIFECYCLE = 1
 (OP_SPAWN, OP_FORK, OP_APPEND, OP_REPLACE, OP_REMOVE, OP_ONE_OFF, OP_PREFILL_DONE, OP_TERMINATE,
  OP_PIN, OP_UNPIN) = range(1, 11)
 MAP_LOOKUP, MAP_ADMIT = 0, 1
@@ -41,7 +42,7 @@ def build(force: bool = False) -> str:
 class _Config(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in ("n_layers", "n_kv_heads", "head_dim", "elem_bytes", "pool_layout",
                                            "n_hbm_blocks", "n_host_blocks", "max_contexts", "suspended_order",
-                                           "reserved")] + \
+                                           "policy_flags")] + \
                [("hash_seed", C.c_uint64), ("hbm_pool", C.c_void_p), ("host_pool", C.c_void_p)]
 
 
@@ -100,7 +101,7 @@ class OracleEngine:
 
     def __init__(self, n_layers, n_kv_heads, head_dim, elem_bytes=2, pool_layout=LAYOUT_LAYER_MAJOR,
                  n_hbm_blocks=128, n_host_blocks=512, max_contexts=64, hash_seed=0,
-                 suspended_order=ORDER_MRU, metadata_only=False, **_ignored):
+                 suspended_order=ORDER_MRU, metadata_only=False, policy_flags=0, **_ignored):
         self.L = lib()
         self.n_layers, self.n_kv_heads, self.head_dim, self.elem_bytes = n_layers, n_kv_heads, head_dim, elem_bytes
         self.pool_layout = pool_layout
@@ -115,7 +116,7 @@ class OracleEngine:
             self.hbm_pool = np.zeros(n_hbm_blocks * self.block_bytes, dtype=np.uint8)
             self.host_pool = np.zeros(max(n_host_blocks, 1) * self.block_bytes, dtype=np.uint8)
         cfg = _Config(n_layers, n_kv_heads, head_dim, elem_bytes, pool_layout, n_hbm_blocks, n_host_blocks,
-                      max_contexts, suspended_order, 0, hash_seed,
+                      max_contexts, suspended_order, policy_flags, hash_seed,
                       None if metadata_only else self.hbm_pool.ctypes.data,
                       None if metadata_only else self.host_pool.ctypes.data)
         h = C.c_void_p()

@@ -16,6 +16,7 @@ OK, E_INVAL, E_NOCTX, E_RANGE, E_STATE, E_NOSPACE, E_BUFSZ, E_DEVICE, E_CUDA = 0
 TIER_HBM, TIER_HOST, TIER_NONE = 0, 1, 0xFF
 LAYOUT_LAYER_MAJOR, LAYOUT_BLOCK_MAJOR = 0, 1
 ORDER_MRU, ORDER_LRU = 0, 1
+POLICY_NO_LIFECYCLE = 1
 (OP_SPAWN, OP_FORK, OP_APPEND, OP_REPLACE, OP_REMOVE, OP_ONE_OFF, OP_PREFILL_DONE, OP_TERMINATE,
  OP_PIN, OP_UNPIN) = range(1, 11)
 OPF_TOKENS_ON_DEVICE = 1
@@ -39,7 +40,7 @@ class Config(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in ("abi_version", "block_tokens", "n_layers", "n_kv_heads", "head_dim",
                                            "elem_bytes", "pool_layout", "n_hbm_blocks", "n_host_blocks",
                                            "table_capacity", "max_contexts", "max_messages", "max_batch_blocks",
-                                           "reserved0")] + \
+                                           "policy_flags")] + \
                [("max_tokens", C.c_uint64), ("max_key_blocks", C.c_uint64), ("hash_seed", C.c_uint64),
                 ("suspended_order", C.c_uint32), ("reserved1", C.c_uint32),
                 ("hbm_pool", C.c_void_p), ("hbm_pool_bytes", C.c_uint64),
@@ -152,7 +153,7 @@ class Engine:
     def __init__(self, n_layers, n_kv_heads, head_dim, elem_bytes=2, pool_layout=LAYOUT_LAYER_MAJOR,
                  n_hbm_blocks=128, n_host_blocks=512, max_contexts=64, hash_seed=0, suspended_order=ORDER_MRU,
                  metadata_only=False, table_capacity=None, max_messages=1 << 16, max_batch_blocks=None,
-                 max_tokens=1 << 22, max_key_blocks=None, host_pool_on_device=False, zero_pools=True,
+                 max_tokens=1 << 22, max_key_blocks=None, host_pool_on_device=False, zero_pools=True, policy_flags=0,
                  device="cuda"):
         import torch
         if not torch.cuda.is_available():
@@ -180,7 +181,7 @@ class Engine:
         cfg.pool_layout, cfg.n_hbm_blocks, cfg.n_host_blocks = pool_layout, n_hbm_blocks, n_host_blocks
         cfg.table_capacity, cfg.max_contexts, cfg.max_messages = table_capacity, max_contexts, max_messages
         cfg.max_batch_blocks, cfg.max_tokens, cfg.max_key_blocks = max_batch_blocks, max_tokens, max_key_blocks
-        cfg.hash_seed, cfg.suspended_order = hash_seed, suspended_order
+        cfg.hash_seed, cfg.suspended_order, cfg.policy_flags = hash_seed, suspended_order, policy_flags
         mb, tb = C.c_uint64(0), C.c_uint64(0)
         rc = self.L.kvt_query_sizes(C.byref(cfg), C.byref(mb), C.byref(tb))
         if rc:

@@ -427,7 +427,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   const kvt_config &c = *cfg;
   if (c.abi_version != KVT_ABI_VERSION || c.block_tokens != 16 || !c.n_layers || !c.n_kv_heads || !c.head_dim ||
       !c.elem_bytes || c.pool_layout > 1 || !c.n_hbm_blocks || !c.max_contexts || !c.max_batch_blocks ||
-      !c.max_messages || c.suspended_order > 1 || c.reserved0 || c.reserved1 || !c.dev_meta || !c.dev_tokens)
+      !c.max_messages || c.suspended_order > 1 || c.policy_flags > 1 || c.reserved1 || !c.dev_meta || !c.dev_tokens)
     return KVT_E_INVAL;
   u64 N = (u64)c.n_hbm_blocks + c.n_host_blocks;
   if (N >= CLAIM_BIT || c.max_batch_blocks >= CLAIM_BIT) return KVT_E_INVAL;
@@ -773,8 +773,13 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     c.n_hit_hbm = k >= 0 ? h_hbm[k] : 0;
     c.n_hit_host = k >= 0 ? h_host[k] : 0;
     c.held = c.hit_len;
-    c.n_admissible = first_temporary_block(c, c.hit_len, c.mat_blocks) - c.hit_len;
-    c.n_pinned = count_pinned_blocks(c, c.hit_len, c.hit_len + c.n_admissible);
+    if (e->cfg.policy_flags & KVT_POLICY_NO_LIFECYCLE) {   // nothing is known to be Temporary or Pinned
+      c.n_admissible = c.mat_blocks - c.hit_len;
+      c.n_pinned = 0;
+    } else {
+      c.n_admissible = first_temporary_block(c, c.hit_len, c.mat_blocks) - c.hit_len;
+      c.n_pinned = count_pinned_blocks(c, c.hit_len, c.hit_len + c.n_admissible);
+    }
     e->st.blocks_hashed += c.mat_blocks;
     e->st.hits_hbm += c.n_hit_hbm; e->st.hits_host += c.n_hit_host; e->st.misses += c.mat_blocks - c.hit_len;
     out[i] = kvt_call_info{c.mat_blocks, c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, 0, c.held, c.n_pinned};
@@ -973,6 +978,7 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   a.stamp_bits = bit_length(e->now); a.depth_bits = bit_length(e->max_depth);
   a.mru = e->cfg.suspended_order == KVT_ORDER_MRU; a.status = e->d_status;
   a.max_rank = (flags & KVT_SEL_INCLUDE_PINNED) ? 3 : 2;
+  a.one_tier = (e->cfg.policy_flags & KVT_POLICY_NO_LIFECYCLE) ? 1 : 0;
   u64 *kA = e->dp<u64>(e->L.keyA), *kB = e->dp<u64>(e->L.keyB);
   u32 *vA = e->dp<u32>(e->L.valA), *vB = e->dp<u32>(e->L.valB), *counts = e->dp<u32>(e->L.rcounts);
   u32 *row_total = counts + 256ull * (e->L.Nt / SORT_TILE + 1);
@@ -1076,7 +1082,8 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
 int32_t kvt_offload(kvt_engine *e, const uint32_t *hbm_slots, uint32_t n, uint32_t *n_done, uint32_t *n_dropped, void *stream) {
   if (!e || (!hbm_slots && n) || !n_done || !n_dropped) return KVT_E_INVAL;
   u32 live = 0;
-  int32_t r = list_op(e, (cudaStream_t)stream, KVT_TIER_HBM, KVT_TIER_HOST, hbm_slots, n, false, true, false, n_done, &live, n_dropped);
+  const bool knows_dead = !(e->cfg.policy_flags & KVT_POLICY_NO_LIFECYCLE);
+  int32_t r = list_op(e, (cudaStream_t)stream, KVT_TIER_HBM, KVT_TIER_HOST, hbm_slots, n, false, knows_dead, false, n_done, &live, n_dropped);
   e->st.offloaded += live;
   e->st.bytes_d2h += live * e->block_bytes;
   if (r == KVT_E_NOSPACE) e->err = "host tier full";

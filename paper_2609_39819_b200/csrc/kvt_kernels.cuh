@@ -523,14 +523,14 @@ __global__ void k_classify(ClsArgs a) {
 // ======================================================================================================
 struct SelArgs {
   Entries ent; u32 e0, n_slots;       // entry range of the tier
-  u32 n_req; u32 now; u32 stamp_bits, depth_bits; u32 mru; u32 max_rank;
+  u32 n_req; u32 now; u32 stamp_bits, depth_bits; u32 mru; u32 max_rank; u32 one_tier;
   u32 *status;
 };
 
 __device__ __forceinline__ bool sel_candidate(const SelArgs &a, u32 i, u32 *rank) {
   u32 e = a.e0 + i;
   if (!a.ent.key[e] || a.ent.infl[e]) return false;
-  u32 r = a.ent.rank[e];
+  u32 r = a.one_tier ? 1u : a.ent.rank[e];   // without lifecycle tracking every block is one tier
   *rank = r;
   return r <= a.max_rank;
 }
@@ -572,7 +572,7 @@ struct EmitSel {
   SelArgs a; u64 *keys; u32 *vals;
   __device__ void operator()(u32 i, u32 pos) const {
     u32 e = a.e0 + i;
-    u64 r = a.ent.rank[e];
+    u64 r = a.one_tier ? 1u : a.ent.rank[e];
     u64 st = a.ent.stamp[e];
     u64 rec = (r == 1 && a.mru) ? (u64)a.now - st : st;       // newest first inside the idle tier
     u64 dinv = ((1ull << a.depth_bits) - 1) - a.ent.depth[e];  // chain tail first

@@ -222,6 +222,31 @@ def pinned_competes_only_with_pinned(make, run_call, options):
     assert states(eng)[2:] == [DEAD, DEAD]
 
 
+# ---- "w/o LT" ablation (Section 8.3): no lifecycle information reaches the policy -----------------------
+def no_lifecycle_policy(make):
+    eng = make(n_hbm_blocks=8, n_host_blocks=8, max_contexts=4, policy_flags=1, **TOY)
+    rng = np.random.default_rng(17)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 64))                         # blocks 0..3, clock 1..2
+    call(eng, 0)
+    eng.spawn(1)
+    eng.one_off(1)
+    eng.append(1, toks(rng, 32))                         # a one-off context: its KV would bypass storage
+    a, b = call(eng, 1)
+    assert (a["n_admissible"], b["n_admitted"]) == (2, 2)    # nothing is known to be Temporary: admitted
+    eng.terminate(1)
+    eng.remove(0, 0, 1)
+    assert states(eng)[:6] == [DEAD] * 6                 # the true states are still reported (for metrics) ...
+    v, s = eng.select_victims(HBM, 8)
+    assert list(v) == [5, 4, 3, 2, 1, 0] and list(s) == [1] * 6   # ... but the policy sees one tier, newest first
+    rc, n_done, n_dropped = eng.offload(v[:3])
+    assert (rc, n_done, n_dropped) == (0, 3, 0)          # and cannot reclaim zombies without a copy
+    assert eng.get_stats()["occ_host"] == 3
+    eng2 = make(n_hbm_blocks=8, n_host_blocks=8, max_contexts=4, policy_flags=1, suspended_order=1, **TOY)
+    eng2.debug_load_resident([10, 11, 12], [2, 0, 1], [5, 9, 7], [0, 0, 0], [0, 1, 2], HBM)
+    assert list(eng2.select_victims(HBM, 3)[0]) == [0, 2, 1]      # plain LRU
+
+
 # ---- hand-worked lifecycle example (8-block pool) --------------------------------------------------
 def worked_example(make):
     eng = make(n_hbm_blocks=8, n_host_blocks=8, max_contexts=4, **TOY)
@@ -570,4 +595,4 @@ def degenerate_inputs(make):
 ALL = [state_machine_single_context, suffix_invalidation, fork_and_shared_kv, one_off_bypass, worked_example,
        mixed_pool_example, victim_order_bruteforce, one_state_pools_reduce_to_lru, offload_reload_round_trip,
        dead_victims_are_dropped_without_copy, compaction, raw_copy_blocks, admission_stops_when_full,
-       lookup_locks_and_orphans, degenerate_inputs, pinned_retention]
+       lookup_locks_and_orphans, degenerate_inputs, pinned_retention, no_lifecycle_policy]

@@ -116,6 +116,24 @@ def test_c1_trace_parity_other_layouts_and_orders(B, oracle, layout, order):
         _replay_pair(gpu, cpu, W.trace_c1(seed), W.payload_pattern)
 
 
+@pytest.mark.parametrize("order,flags", [(0, 1), (1, 1)])
+def test_trace_parity_without_lifecycle_tracking(B, oracle, order, flags):
+    """The "w/o LT" ablation and plain LRU: same replays, same results as the oracle."""
+    for seed in (7, 63):
+        kw = dict(n_hbm_blocks=96, n_host_blocks=256, max_contexts=64, suspended_order=order, policy_flags=flags,
+                  **W.GEO_TOY.kwargs())
+        gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)
+        cpu = oracle.OracleEngine(**kw)
+        _replay_pair(gpu, cpu, W.trace_c1(seed), W.payload_pattern)
+    trace, n_ctx = W.trace_c3(1, n_sessions=8, scale=1 / 32)
+    kw = dict(n_hbm_blocks=256, n_host_blocks=256, max_contexts=n_ctx, metadata_only=True, suspended_order=order,
+              policy_flags=flags, **W.GEO_TOY.kwargs())
+    from paper_2609_39819_b200 import policy_metrics as PM
+    mg = PM.replay_metrics(B.Engine(max_tokens=1 << 20, max_messages=1 << 15, **kw), trace)
+    mc = PM.replay_metrics(oracle.OracleEngine(**kw), trace)
+    assert mg == mc
+
+
 def test_scaled_c2_trace_parity(B, oracle):
     kw = dict(n_hbm_blocks=96, n_host_blocks=64, max_contexts=8, **W.GEO_TOY.kwargs())
     gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)

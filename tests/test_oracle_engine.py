@@ -121,3 +121,20 @@ def test_kv_size_sanity():
     bytes_per_token = W.GEO_GLM.block_bytes // 16
     assert bytes_per_token == 376832
     assert abs(258_000 * bytes_per_token / 1e9 - 93) / 93 < 0.05
+
+
+def test_policy_metrics_on_a_small_trace(make):
+    """Hit ratio, zombie share and wrong-direction ratio are well defined and the ablations behave as
+    Section 8.3 describes: without lifecycle tracking zombies pile up and are copied instead of dropped."""
+    from paper_2609_39819_b200 import policy_metrics as PM
+    trace, n_ctx = W.trace_c3(1, n_sessions=8, scale=1 / 32)
+    res = {}
+    for name, (order, flags) in PM.POLICIES.items():
+        eng = make(n_hbm_blocks=256, n_host_blocks=256, max_contexts=n_ctx, metadata_only=True, suspended_order=order,
+                   policy_flags=flags, **W.GEO_TOY.kwargs())
+        res[name] = PM.replay_metrics(eng, trace)
+        m = res[name]
+        assert 0 < m["hit_ratio"] < 1 and 0 <= m["wrong_direction_ratio"] <= 1 and m["zombie_share_peak"] <= 1
+    paper, no_lt = res["lifecycle + MRU (paper)"], res["w/o LT (MRU only)"]
+    assert no_lt["zombie_share_mean"] > paper["zombie_share_mean"]
+    assert no_lt["offloaded"] > paper["offloaded"]
