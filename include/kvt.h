@@ -77,6 +77,12 @@ extern "C" {
                                        offload copies every victim (nothing is known to be dead) and nothing bypasses
                                        admission. kvt_get_states still reports the true states (for metrics). */
 
+#define KVT_POLICY_INCLUSIVE 2u     /* inclusive tiers (Section 7: a tier may retain a fast copy): kvt_reload leaves the
+                                       block's bytes in its host slot as a clean copy linked to the HBM block; a later
+                                       kvt_offload of that block hands it back to the copy without moving a byte.
+                                       Copies occupy host slots, are the first victims of the host tier (state
+                                       KVT_STATE_COPY), can be released on their own, and go away with their block. */
+
 /* Primitives and runtime events (Table 3; Section 5.2 "Runtime transitions"). */
 #define KVT_OP_SPAWN         1u  /* register an independent, empty context */
 #define KVT_OP_FORK          2u  /* register child `ctx` sharing messages [0, msg_end) of `parent` */
@@ -110,6 +116,8 @@ extern "C" {
 #define KVT_STATE_ACTIVE  2u   /* live and active */
 #define KVT_STATE_PINNED  3u   /* explicitly retained: competes for space only with incoming Pinned KV */
 #define KVT_STATE_FREE    0xFFu /* slot holds no block */
+#define KVT_STATE_COPY    0xFEu /* host slot holding only the clean copy of a block whose home is HBM (inclusive tiers) */
+#define KVT_STATE_HAS_COPY 0x80u /* or-ed into the rank of an HBM victim that still has a clean host copy */
 
 typedef struct kvt_engine kvt_engine;
 
@@ -326,6 +334,7 @@ typedef struct kvt_stats {
   uint64_t lookup_blocks;    /* and the blocks they processed */
   uint64_t select_ns;        /* with profiling on: device time of the selection kernels (count, compaction, sort, emit) */
   uint64_t select_slots;     /* and the tier slots they scanned */
+  uint64_t offloaded_clean;  /* of `offloaded`, blocks handed to an existing clean host copy (no bytes moved) */
 } kvt_stats;
 int32_t kvt_get_stats(kvt_engine *e, kvt_stats *out);
 
@@ -342,9 +351,10 @@ int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant);
 int32_t kvt_last_error(kvt_engine *e, char *buf, uint32_t cap);
 
 /* Copies per-slot metadata of a tier to host arrays (any may be NULL): key (0 = free), stamp,
- * depth, in-flight count. cap >= slots of the tier. Synchronises. */
+ * depth, in-flight count, and link = the slot of the other tier that holds this block's clean copy /
+ * the block this copy belongs to (0xFFFFFFFF: none). cap >= slots of the tier. Synchronises. */
 int32_t kvt_get_entries(kvt_engine *e, uint32_t tier, uint64_t *keys, uint32_t *stamp,
-                        uint32_t *depth, uint32_t *inflight, uint32_t cap, void *stream);
+                        uint32_t *depth, uint32_t *inflight, uint32_t *link, uint32_t cap, void *stream);
 
 /* Test / benchmark hook: makes n blocks resident in `tier` at the given slots without running
  * calls. state[i] acts as a permanent anonymous mapping of that rank (classification never reports

@@ -42,7 +42,10 @@ enum : int32_t {
 enum : uint32_t { TIER_HBM = 0, TIER_HOST = 1 };
 enum : uint32_t { LAYOUT_LAYER_MAJOR = 0, LAYOUT_BLOCK_MAJOR = 1 };
 enum : uint32_t { ORDER_MRU = 0, ORDER_LRU = 1 };
-enum : uint32_t { POLICY_NO_LIFECYCLE = 1 };   // the "w/o LT" variant of Section 8.3
+enum : uint32_t {
+  POLICY_NO_LIFECYCLE = 1,   // the "w/o LT" variant of Section 8.3
+  POLICY_INCLUSIVE = 2       // a reloaded block keeps its host copy (Section 7: per-tier caching keeps a fast copy)
+};
 enum : uint32_t {
   OP_SPAWN = 1, OP_FORK, OP_APPEND, OP_REPLACE, OP_REMOVE, OP_ONE_OFF, OP_PREFILL_DONE,
   OP_TERMINATE, OP_PIN, OP_UNPIN
@@ -115,7 +118,12 @@ struct Ctx {
   uint32_t hit_len = 0, n_hit_hbm = 0, n_hit_host = 0, n_admissible = 0, n_pinned = 0;
 };
 
-struct Entry { uint64_t key = 0; uint32_t stamp = 0, depth = 0, inflight = 0; uint8_t floor = 0; };
+struct Entry {
+  uint64_t key = 0; uint32_t stamp = 0, depth = 0, inflight = 0; uint8_t floor = 0;
+  // inclusive tiering: an HBM block and its clean host copy ("shadow") point at each other by slot
+  int64_t link = -1;
+  bool shadow = false;   // host slot that only holds a copy of a block whose home is in HBM
+};
 
 struct Config {
   uint32_t n_layers, n_kv_heads, head_dim, elem_bytes, pool_layout;
@@ -130,7 +138,7 @@ struct Stats {
   uint64_t clock, n_contexts, occ_hbm, occ_host, blocks_hashed, hits_hbm, hits_host, misses,
       inserted, adopted, dropped, offloaded, reloaded, compacted, bytes_d2h, bytes_h2d, bytes_d2d,
       table_rebuilds, tombstones, kernel_launches, mover_launches, mover_ns, mover_bytes, lookup_ns,
-      lookup_blocks, select_ns, select_slots;
+      lookup_blocks, select_ns, select_slots, offloaded_clean;
 };
 
 struct Op {
@@ -179,7 +187,15 @@ Entry *find_entry(Engine &e, uint64_t key) {
 
 void free_slot(Engine &e, uint32_t tier, uint32_t slot) {
   Entry &x = e.ent[tier][slot];
-  e.where.erase(x.key);
+  if (x.shadow) {                      // dropping a host copy: the block lives on in HBM
+    e.ent[TIER_HBM][x.link].link = -1;
+  } else {
+    e.where.erase(x.key);
+    if (x.link >= 0) {                 // dropping a block that has a host copy: the copy goes too
+      e.ent[TIER_HOST][x.link] = Entry();
+      e.free_slots[TIER_HOST].insert((uint32_t)x.link);
+    }
+  }
   x = Entry();
   e.free_slots[tier].insert(slot);
 }
@@ -205,7 +221,7 @@ void classify(Engine &e, std::vector<uint8_t> rank[2]) {
   for (int t = 0; t < 2; ++t) {
     rank[t].assign(e.ent[t].size(), 0xFF);
     for (size_t s = 0; s < e.ent[t].size(); ++s)
-      if (e.ent[t][s].key) rank[t][s] = e.ent[t][s].floor;
+      if (e.ent[t][s].key) rank[t][s] = e.ent[t][s].shadow ? 0xFE : e.ent[t][s].floor;
   }
   std::vector<uint8_t> br;
   for (const Ctx &c : e.ctxs) {
@@ -247,7 +263,7 @@ extern "C" {
 int32_t kvto_create(const Config *cfg, Engine **out) {
   if (!cfg || !out) return E_INVAL;
   if (!cfg->n_layers || !cfg->n_kv_heads || !cfg->head_dim || !cfg->elem_bytes || !cfg->n_hbm_blocks ||
-      !cfg->max_contexts || cfg->pool_layout > 1 || cfg->suspended_order > 1 || cfg->policy_flags > 1)
+      !cfg->max_contexts || cfg->pool_layout > 1 || cfg->suspended_order > 1 || cfg->policy_flags > 3)
     return E_INVAL;
   Engine *e = new Engine();
   e->cfg = *cfg;
@@ -533,6 +549,7 @@ int32_t kvto_classify_bruteforce(Engine *e, uint32_t tier, uint8_t *state, uint3
   for (uint32_t s = 0; s < tier_size(*e, tier); ++s) {
     const Entry &x = e->ent[tier][s];
     if (!x.key) { state[s] = 0xFF; continue; }
+    if (x.shadow) { state[s] = 0xFE; continue; }
     int best = x.floor;
     for (const Ctx &c : e->ctxs) {
       if (!c.live) continue;
@@ -560,21 +577,26 @@ int32_t kvto_select_victims(Engine *e, uint32_t tier, uint32_t n_req, uint32_t f
   classify(*e, rank);
   if (e->cfg.policy_flags & POLICY_NO_LIFECYCLE)   // without lifecycle tracking every resident block is one tier
     for (uint8_t &r : rank[tier]) if (r != 0xFF) r = 1;
-  struct Cand { uint32_t slot; uint8_t rank; uint32_t stamp, depth; };
+  struct Cand { uint32_t slot; uint8_t rank; uint32_t stamp, depth; bool shadow; };
   std::vector<Cand> cands;
   for (uint32_t s = 0; s < tier_size(*e, tier); ++s) {
     const Entry &x = e->ent[tier][s];
-    if (!x.key || x.inflight || rank[tier][s] > max_rank) continue;
-    cands.push_back(Cand{s, rank[tier][s], x.stamp, x.depth});
+    if (!x.key) continue;
+    if (x.shadow) { cands.push_back(Cand{s, 0xFE, x.stamp, x.depth, true}); continue; }   // free to drop: first
+    if (x.inflight || rank[tier][s] > max_rank) continue;
+    // an HBM victim that still has a clean host copy is flagged: moving it out needs no copy
+    cands.push_back(Cand{s, (uint8_t)(rank[tier][s] | (x.link >= 0 ? 0x80 : 0)), x.stamp, x.depth, false});
   }
   const bool mru = e->cfg.suspended_order == ORDER_MRU;
   std::stable_sort(cands.begin(), cands.end(), [mru](const Cand &a, const Cand &b) {
-    if (a.rank != b.rank) return a.rank < b.rank;            // Algorithm 1: dead, idle, active, (pinned)
+    if (a.shadow != b.shadow) return a.shadow;                // host copies of HBM blocks go first
+    int ra = a.shadow ? 0 : (a.rank & 0x7F), rb = b.shadow ? 0 : (b.rank & 0x7F);
+    if (ra != rb) return ra < rb;                              // Algorithm 1: dead, idle, active, (pinned)
     if (a.stamp != b.stamp) {
-      if (a.rank == 1 && mru) return a.stamp > b.stamp;      // Section 6.2: most recently suspended first
-      return a.stamp < b.stamp;                              // oldest first
+      if (ra == 1 && mru && !a.shadow) return a.stamp > b.stamp;   // Section 6.2: most recently suspended first
+      return a.stamp < b.stamp;                                // oldest first
     }
-    if (a.depth != b.depth) return a.depth > b.depth;        // chain tail before its prefix
+    if (a.depth != b.depth) return a.depth > b.depth;          // chain tail before its prefix
     return a.slot < b.slot;
   });
   uint32_t n = std::min<uint32_t>(n_req, (uint32_t)cands.size());
@@ -587,13 +609,14 @@ int32_t kvto_select_victims(Engine *e, uint32_t tier, uint32_t n_req, uint32_t f
   return OK;
 }
 
-static int32_t validate_slots(Engine *e, uint32_t tier, const uint32_t *slots, uint32_t n, bool allow_inflight) {
+static int32_t validate_slots(Engine *e, uint32_t tier, const uint32_t *slots, uint32_t n, bool allow_inflight,
+                              bool allow_shadow = true) {
   bool bad_range = false, bad_inval = false, bad_state = false;
   std::set<uint32_t> seen;
   for (uint32_t i = 0; i < n; ++i) {
     if (slots[i] >= tier_size(*e, tier)) { bad_range = true; continue; }
     const Entry &x = e->ent[tier][slots[i]];
-    if (!x.key || !seen.insert(slots[i]).second) { bad_inval = true; continue; }
+    if (!x.key || !seen.insert(slots[i]).second || (x.shadow && !allow_shadow)) { bad_inval = true; continue; }
     if (x.inflight && !allow_inflight) bad_state = true;
   }
   if (bad_range) return E_RANGE;
@@ -609,7 +632,8 @@ static void move_entry(Engine *e, uint32_t st, uint32_t ss, uint32_t dt, uint32_
   e->free_slots[st].insert(ss);
   e->free_slots[dt].erase(ds);
   e->ent[dt][ds] = x;
-  e->where[x.key] = {dt, ds};
+  if (!x.shadow) e->where[x.key] = {dt, ds};
+  if (x.link >= 0) e->ent[x.shadow ? TIER_HBM : TIER_HOST][x.link].link = ds;   // the partner follows (compaction)
 }
 
 int32_t kvto_offload(Engine *e, const uint32_t *slots, uint32_t n, uint32_t *n_done, uint32_t *n_dropped) {
@@ -626,6 +650,15 @@ int32_t kvto_offload(Engine *e, const uint32_t *slots, uint32_t n, uint32_t *n_d
       free_slot(*e, TIER_HBM, s);
       e->st.dropped++;
       (*n_dropped)++;
+    } else if (e->ent[TIER_HBM][s].link >= 0) {  // a clean host copy exists: hand the block over, no copy
+      Entry x = e->ent[TIER_HBM][s];
+      Entry &h = e->ent[TIER_HOST][x.link];
+      h.shadow = false; h.link = -1; h.stamp = x.stamp; h.depth = x.depth; h.floor = x.floor; h.inflight = x.inflight;
+      e->where[x.key] = {TIER_HOST, (uint32_t)x.link};
+      e->ent[TIER_HBM][s] = Entry();
+      e->free_slots[TIER_HBM].insert(s);
+      e->st.offloaded++;
+      e->st.offloaded_clean++;
     } else {
       if (e->free_slots[TIER_HOST].empty()) return E_NOSPACE;
       uint32_t d = *e->free_slots[TIER_HOST].begin();
@@ -641,12 +674,25 @@ int32_t kvto_offload(Engine *e, const uint32_t *slots, uint32_t n, uint32_t *n_d
 int32_t kvto_reload(Engine *e, const uint32_t *slots, uint32_t n, uint32_t *n_done) {
   if (!e || (!slots && n) || !n_done) return E_INVAL;
   *n_done = 0;
-  int32_t v = validate_slots(e, TIER_HOST, slots, n, true);
+  int32_t v = validate_slots(e, TIER_HOST, slots, n, true, false);
   if (v != OK) return v;
   for (uint32_t i = 0; i < n; ++i) {
     if (e->free_slots[TIER_HBM].empty()) return E_NOSPACE;
     uint32_t d = *e->free_slots[TIER_HBM].begin();
-    move_entry(e, TIER_HOST, slots[i], TIER_HBM, d);
+    if (e->cfg.policy_flags & POLICY_INCLUSIVE) {   // the host slot keeps the bytes as a clean copy
+      uint32_t h = slots[i];
+      copy_payload(*e, TIER_HOST, h, TIER_HBM, d);
+      Entry x = e->ent[TIER_HOST][h];
+      x.link = h;
+      e->ent[TIER_HBM][d] = x;
+      e->free_slots[TIER_HBM].erase(d);
+      e->ent[TIER_HOST][h].shadow = true;
+      e->ent[TIER_HOST][h].link = d;
+      e->ent[TIER_HOST][h].inflight = 0;
+      e->where[x.key] = {TIER_HBM, d};
+    } else {
+      move_entry(e, TIER_HOST, slots[i], TIER_HBM, d);
+    }
     e->st.reloaded++;
     e->st.bytes_h2d += e->block_bytes;
     (*n_done)++;
@@ -703,7 +749,7 @@ int32_t kvto_get_stats(Engine *e, Stats *out) {
 }
 
 int32_t kvto_get_entries(Engine *e, uint32_t tier, uint64_t *keys, uint32_t *stamp, uint32_t *depth,
-                         uint32_t *inflight, uint32_t cap) {
+                         uint32_t *inflight, uint32_t *link, uint32_t cap) {
   if (!e || tier > 1) return E_INVAL;
   if (cap < tier_size(*e, tier)) return E_BUFSZ;
   for (uint32_t s = 0; s < tier_size(*e, tier); ++s) {
@@ -712,6 +758,7 @@ int32_t kvto_get_entries(Engine *e, uint32_t tier, uint64_t *keys, uint32_t *sta
     if (stamp) stamp[s] = x.stamp;
     if (depth) depth[s] = x.depth;
     if (inflight) inflight[s] = x.inflight;
+    if (link) link[s] = x.link >= 0 ? (uint32_t)x.link : 0xFFFFFFFFu;
   }
   return OK;
 }

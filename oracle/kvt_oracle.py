@@ -20,7 +20,7 @@ OK, E_INVAL, E_NOCTX, E_RANGE, E_STATE, E_NOSPACE, E_BUFSZ = 0, -1, -2, -3, -4, 
 TIER_HBM, TIER_HOST, TIER_NONE = 0, 1, 0xFF
 LAYOUT_LAYER_MAJOR, LAYOUT_BLOCK_MAJOR = 0, 1
 ORDER_MRU, ORDER_LRU = 0, 1
-POLICY_NO_LIFECYCLE = 1
+POLICY_NO_LIFECYCLE, POLICY_INCLUSIVE = 1, 2
 (OP_SPAWN, OP_FORK, OP_APPEND, OP_REPLACE, OP_REMOVE, OP_ONE_OFF, OP_PREFILL_DONE, OP_TERMINATE,
  OP_PIN, OP_UNPIN) = range(1, 11)
 MAP_LOOKUP, MAP_ADMIT = 0, 1
@@ -56,7 +56,7 @@ CALL_INFO_DTYPE = np.dtype([(n, np.uint32) for n in ("n_blocks", "hit_len", "n_h
 STATS_FIELDS = ("clock", "n_contexts", "occ_hbm", "occ_host", "blocks_hashed", "hits_hbm", "hits_host", "misses",
                 "inserted", "adopted", "dropped", "offloaded", "reloaded", "compacted", "bytes_d2h", "bytes_h2d",
                 "bytes_d2d", "table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns",
-                "mover_bytes", "lookup_ns", "lookup_blocks", "select_ns", "select_slots")
+                "mover_bytes", "lookup_ns", "lookup_blocks", "select_ns", "select_slots", "offloaded_clean")
 
 _lib = None
 
@@ -260,11 +260,11 @@ class OracleEngine:
     def get_entries(self, tier):
         n = self._tier_size(tier)
         keys = np.zeros(n, np.uint64); stamp = np.zeros(n, np.uint32)
-        depth = np.zeros(n, np.uint32); infl = np.zeros(n, np.uint32)
-        rc = self.L.kvto_get_entries(self.h, tier, _p(keys), _p(stamp), _p(depth), _p(infl), n)
+        depth = np.zeros(n, np.uint32); infl = np.zeros(n, np.uint32); link = np.zeros(n, np.uint32)
+        rc = self.L.kvto_get_entries(self.h, tier, _p(keys), _p(stamp), _p(depth), _p(infl), _p(link), n)
         if rc:
             raise OracleError(rc, "get_entries")
-        return {"key": keys, "stamp": stamp, "depth": depth, "inflight": infl}
+        return {"key": keys, "stamp": stamp, "depth": depth, "inflight": infl, "link": link}
 
     def debug_load_resident_rc(self, keys, state, stamp, depth, slot, tier):
         k = np.ascontiguousarray(np.asarray(keys, np.uint64)); st = np.ascontiguousarray(np.asarray(state, np.uint8))

@@ -73,7 +73,7 @@ struct Ctx {
 };
 
 struct DevLayout {
-  u64 tab, e_key, e_stamp, e_depth, e_infl, e_rank, e_tslot, e_mark, e_floor, keys, status;
+  u64 tab, e_key, e_stamp, e_depth, e_infl, e_rank, e_tslot, e_mark, e_link, e_floor, keys, status;
   u64 s0, s1, s2, s3, ids, ids2, pair_src, pair_dst, freelist, tiles, agg, carry, desc, ctxres;
   u64 m_start, m_end, m_rank, keyA, keyB, valA, valB, rcounts, out_slots, out_states, map_tier, map_slot;
   u64 total;
@@ -89,7 +89,7 @@ DevLayout make_layout(const kvt_config &c) {
   auto take = [&](u64 bytes) { u64 o = off; off = round_up(off + bytes, 256); return o; };
   L.tab = take((u64)c.table_capacity * 16);
   L.e_key = take(N * 8); L.e_stamp = take(N * 4); L.e_depth = take(N * 4); L.e_infl = take(N * 4);
-  L.e_rank = take(N * 4); L.e_tslot = take(N * 4); L.e_mark = take(N * 4); L.e_floor = take(N);
+  L.e_rank = take(N * 4); L.e_tslot = take(N * 4); L.e_mark = take(N * 4); L.e_link = take(N * 4); L.e_floor = take(N);
   L.keys = take(c.max_key_blocks * 8);
   L.status = take(ST_WORDS * 4);
   L.s0 = take(LB * 4); L.s1 = take(LB * 4); L.s2 = take(LB * 4); L.s3 = take(LB * 4);
@@ -427,7 +427,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   const kvt_config &c = *cfg;
   if (c.abi_version != KVT_ABI_VERSION || c.block_tokens != 16 || !c.n_layers || !c.n_kv_heads || !c.head_dim ||
       !c.elem_bytes || c.pool_layout > 1 || !c.n_hbm_blocks || !c.max_contexts || !c.max_batch_blocks ||
-      !c.max_messages || c.suspended_order > 1 || c.policy_flags > 1 || c.reserved1 || !c.dev_meta || !c.dev_tokens)
+      !c.max_messages || c.suspended_order > 1 || c.policy_flags > 3 || c.reserved1 || !c.dev_meta || !c.dev_tokens)
     return KVT_E_INVAL;
   u64 N = (u64)c.n_hbm_blocks + c.n_host_blocks;
   if (N >= CLAIM_BIT || c.max_batch_blocks >= CLAIM_BIT) return KVT_E_INVAL;
@@ -455,7 +455,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   e->tab.shift = 64 - (bit_length(c.table_capacity) - 1);
   e->ent.key = e->dp<u64>(L.e_key); e->ent.stamp = e->dp<u32>(L.e_stamp); e->ent.depth = e->dp<u32>(L.e_depth);
   e->ent.infl = e->dp<u32>(L.e_infl); e->ent.rank = e->dp<u32>(L.e_rank); e->ent.tslot = e->dp<u32>(L.e_tslot);
-  e->ent.mark = e->dp<u32>(L.e_mark); e->ent.floor = e->dp<u8>(L.e_floor);
+  e->ent.mark = e->dp<u32>(L.e_mark); e->ent.floor = e->dp<u8>(L.e_floor); e->ent.link = e->dp<u32>(L.e_link);
   e->ent.n_hbm = c.n_hbm_blocks; e->ent.n_total = (u32)N;
   e->d_keys = e->dp<u64>(L.keys); e->d_status = e->dp<u32>(L.status);
   e->h0 = hash_h0(c.hash_seed);
@@ -479,6 +479,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   // everything except the key arena and scratch must start at zero; the table needs ent = NONE
   ok = ok && cudaMemsetAsync(e->meta + L.e_key, 0, L.keys - L.e_key, s) == cudaSuccess;
   ok = ok && cudaMemsetAsync(e->d_status, 0, ST_WORDS * 4, s) == cudaSuccess;
+  ok = ok && cudaMemsetAsync(e->ent.link, 0xFF, N * 4, s) == cudaSuccess;   // no links
   if (ok) {
     KL(k_table_clear, cdiv((u64)c.table_capacity,256), 256, s, e->tab);
     ok = cudaGetLastError() == cudaSuccess && cudaStreamSynchronize(s) == cudaSuccess;
@@ -947,7 +948,7 @@ int32_t kvt_get_states(kvt_engine *e, uint32_t tier, uint8_t *state, uint32_t ca
 }
 
 int32_t kvt_get_entries(kvt_engine *e, uint32_t tier, uint64_t *keys, uint32_t *stamp, uint32_t *depth,
-                        uint32_t *inflight, uint32_t cap, void *stream) {
+                        uint32_t *inflight, uint32_t *link, uint32_t cap, void *stream) {
   if (!e || tier > 1) return KVT_E_INVAL;
   u32 n = e->tier_slots(tier), e0 = e->tier_e0(tier);
   if (cap < n) return KVT_E_BUFSZ;
@@ -957,7 +958,10 @@ int32_t kvt_get_entries(kvt_engine *e, uint32_t tier, uint64_t *keys, uint32_t *
   if (stamp) CU(cudaMemcpyAsync(stamp, e->ent.stamp + e0, n * 4ull, cudaMemcpyDeviceToHost, s));
   if (depth) CU(cudaMemcpyAsync(depth, e->ent.depth + e0, n * 4ull, cudaMemcpyDeviceToHost, s));
   if (inflight) CU(cudaMemcpyAsync(inflight, e->ent.infl + e0, n * 4ull, cudaMemcpyDeviceToHost, s));
+  if (link) CU(cudaMemcpyAsync(link, e->ent.link + e0, n * 4ull, cudaMemcpyDeviceToHost, s));
   CU(cudaStreamSynchronize(s));
+  if (link && tier == KVT_TIER_HBM)   // entry ids of host copies -> host slot numbers
+    for (u32 i = 0; i < n; ++i) if (link[i] != ENT_NONE) link[i] -= e->cfg.n_hbm_blocks;
   return KVT_OK;
 }
 
@@ -986,7 +990,7 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   KL(k_sel_count, cdiv(n,256), 256, s, a);
   r = compact_indices(e, s, PredSel{a}, EmitSel{a, kA, vA}, n, ST_M);
   if (r) return r;
-  const u32 key_bits = 2 + a.stamp_bits + a.depth_bits, n_pass = cdiv(key_bits, 8), tiles = cdiv(n, SORT_TILE);
+  const u32 key_bits = 3 + a.stamp_bits + a.depth_bits, n_pass = cdiv(key_bits, 8), tiles = cdiv(n, SORT_TILE);
   for (u32 p = 0; p < n_pass; ++p) {
     KL(k_radix_hist, tiles, 256, s, kA, e->d_status, 8 * p, counts);
     KL(k_radix_scan, 32, 256, s, counts, row_total, e->d_status);
@@ -994,7 +998,7 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
     std::swap(kA, kB); std::swap(vA, vB);
   }
   u32 n_emit = std::min(n_req, n);
-  KL(k_sel_emit, cdiv(n_emit,256), 256, s, kA, vA, n_emit, a.stamp_bits + a.depth_bits, e->dp<u32>(e->L.out_slots),
+  KL(k_sel_emit, cdiv(n_emit,256), 256, s, e->ent, a.e0, n, kA, vA, n_emit, e->d_status, a.stamp_bits + a.depth_bits, e->dp<u32>(e->L.out_slots),
                                                e->dp<u8>(e->L.out_states));
   if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));
   LAUNCH_CHECK();
@@ -1010,7 +1014,8 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   }
   r = status_code(e);
   if (r) return r;
-  u64 total = (u64)e->h_status[ST_RANK0] + e->h_status[ST_RANK1] + e->h_status[ST_RANK2] + e->h_status[ST_RANK3];
+  u64 total = (u64)e->h_status[ST_RANK0] + e->h_status[ST_RANK1] + e->h_status[ST_RANK2] + e->h_status[ST_RANK3] +
+              e->h_status[ST_SHADOW];
   u32 k = (u32)std::min<u64>(n_req, total);
   *n_out = k;
   if (cap < k) return KVT_E_BUFSZ;
@@ -1023,14 +1028,17 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
 
 // ---- stage 5 -----------------------------------------------------------------------------------------------
 // Shared body of offload / reload / release.
+struct ListMode { bool allow_inflight, drop_dead, drop_all, reject_shadow, clean_ok, keep_copy; };
+struct ListCounts { u32 done = 0, copied = 0, dropped = 0, clean = 0; };
+
 static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier, const u32 *slots, u32 n,
-                       bool allow_inflight, bool drop_dead, bool drop_all, u32 *n_done, u32 *n_live, u32 *n_drop) {
-  *n_done = *n_live = *n_drop = 0;
+                       const ListMode &m, ListCounts *out) {
+  *out = ListCounts();
   if (n == 0) return KVT_OK;
   if (n > e->L.LB) return fail(e, KVT_E_NOSPACE, "list longer than max_batch_blocks");
   int32_t r = stage_acquire(e);
   if (r) return r;
-  if (drop_dead) { r = ensure_classified(e, s); if (r) return r; r = stage_acquire(e); if (r) return r; }
+  if (m.drop_dead) { r = ensure_classified(e, s); if (r) return r; r = stage_acquire(e); if (r) return r; }
   std::memcpy(e->h_ids, slots, n * 4ull);
   u32 *d_ids = e->dp<u32>(e->L.ids);
   CU(cudaMemcpyAsync(d_ids, e->h_ids, n * 4ull, cudaMemcpyHostToDevice, s));
@@ -1045,12 +1053,13 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
   a.live = e->dp<u32>(e->L.s1); a.lidx = e->dp<u32>(e->L.s2);
   a.freelist = e->dp<u32>(e->L.freelist); a.n_free = e->tier_slots(dst_tier) - e->occ[dst_tier];
   a.pair_src = e->dp<u32>(e->L.pair_src); a.pair_dst = e->dp<u32>(e->L.pair_dst);
-  a.allow_inflight = allow_inflight; a.drop_dead = drop_dead; a.drop_all = drop_all; a.status = e->d_status;
+  a.allow_inflight = m.allow_inflight; a.drop_dead = m.drop_dead; a.drop_all = m.drop_all;
+  a.reject_shadow = m.reject_shadow; a.clean_ok = m.clean_ok; a.keep_copy = m.keep_copy; a.status = e->d_status;
   u32 g = cdiv(n, 256);
   KL(k_list_validate, g, 256, s, a);
   r = compact_indices(e, s, PredLive{a.live}, EmitLive{a.lidx, a.n_free, e->d_status}, n, ST_TOTAL);
   if (r) return r;
-  if (!drop_all) {
+  if (!m.drop_all) {
     r = compact_indices(e, s, PredFree{e->ent.key, a.dst_e0}, EmitFree{e->dp<u32>(e->L.freelist), (u32)e->L.LB},
                         e->tier_slots(dst_tier), ST_FREE);
     if (r) return r;
@@ -1058,7 +1067,7 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
   KL(k_list_apply, g, 256, s, a);
   KL(k_list_unmark, g, 256, s, a);
   LAUNCH_CHECK();
-  if (!drop_all) {
+  if (!m.drop_all) {
     r = launch_mover(e, s, src_tier, a.pair_src, dst_tier, a.pair_dst, std::min(n, a.n_free), e->d_status + ST_NLIVE);
     if (r) return r;
   }
@@ -1066,44 +1075,59 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
   if (r) return r;
   r = status_code(e);
   if (r) return r;
-  *n_live = e->h_status[ST_NLIVE];
-  *n_drop = e->h_status[ST_NDROP];
-  mover_account(e, *n_live);
-  *n_done = *n_live + *n_drop;
-  e->occ[src_tier] -= *n_done;
-  if (!drop_all) e->occ[dst_tier] += *n_live;
-  e->tombs += *n_drop;
-  e->st.dropped += *n_drop;
+  out->copied = e->h_status[ST_NLIVE];
+  out->dropped = e->h_status[ST_NDROP];
+  out->clean = e->h_status[ST_NCLEAN];
+  out->done = out->copied + out->dropped + out->clean;
+  mover_account(e, out->copied);
+  // occupancy: listed blocks leave the source tier unless they stay behind as clean copies; copies that
+  // belonged to dropped blocks free their host slots as well
+  e->occ[src_tier] -= out->done - (m.keep_copy ? out->copied : 0);
+  if (!m.drop_all) e->occ[dst_tier] += out->copied;
+  e->occ[KVT_TIER_HOST] -= e->h_status[ST_NSHDROP];
+  e->tombs += e->h_status[ST_TOMBS];
+  e->st.dropped += out->dropped;
   r = maybe_rebuild(e, s);
   if (r) return r;
-  return *n_done < n ? KVT_E_NOSPACE : KVT_OK;
+  return out->done < n ? KVT_E_NOSPACE : KVT_OK;
 }
 
 int32_t kvt_offload(kvt_engine *e, const uint32_t *hbm_slots, uint32_t n, uint32_t *n_done, uint32_t *n_dropped, void *stream) {
   if (!e || (!hbm_slots && n) || !n_done || !n_dropped) return KVT_E_INVAL;
-  u32 live = 0;
-  const bool knows_dead = !(e->cfg.policy_flags & KVT_POLICY_NO_LIFECYCLE);
-  int32_t r = list_op(e, (cudaStream_t)stream, KVT_TIER_HBM, KVT_TIER_HOST, hbm_slots, n, false, knows_dead, false, n_done, &live, n_dropped);
-  e->st.offloaded += live;
-  e->st.bytes_d2h += live * e->block_bytes;
+  ListMode m{};
+  m.drop_dead = !(e->cfg.policy_flags & KVT_POLICY_NO_LIFECYCLE);
+  m.clean_ok = true;
+  ListCounts c;
+  int32_t r = list_op(e, (cudaStream_t)stream, KVT_TIER_HBM, KVT_TIER_HOST, hbm_slots, n, m, &c);
+  *n_done = c.done; *n_dropped = c.dropped;
+  e->st.offloaded += c.copied + c.clean;
+  e->st.offloaded_clean += c.clean;
+  e->st.bytes_d2h += c.copied * e->block_bytes;
   if (r == KVT_E_NOSPACE) e->err = "host tier full";
   return r;
 }
 
 int32_t kvt_reload(kvt_engine *e, const uint32_t *host_slots, uint32_t n, uint32_t *n_done, void *stream) {
   if (!e || (!host_slots && n) || !n_done) return KVT_E_INVAL;
-  u32 live = 0, drop = 0;
-  int32_t r = list_op(e, (cudaStream_t)stream, KVT_TIER_HOST, KVT_TIER_HBM, host_slots, n, true, false, false, n_done, &live, &drop);
-  e->st.reloaded += live;
-  e->st.bytes_h2d += live * e->block_bytes;
+  ListMode m{};
+  m.allow_inflight = true;
+  m.reject_shadow = true;
+  m.keep_copy = e->cfg.policy_flags & KVT_POLICY_INCLUSIVE;
+  ListCounts c;
+  int32_t r = list_op(e, (cudaStream_t)stream, KVT_TIER_HOST, KVT_TIER_HBM, host_slots, n, m, &c);
+  *n_done = c.done;
+  e->st.reloaded += c.copied;
+  e->st.bytes_h2d += c.copied * e->block_bytes;
   if (r == KVT_E_NOSPACE) e->err = "HBM tier full";
   return r;
 }
 
 int32_t kvt_release(kvt_engine *e, uint32_t tier, const uint32_t *slots, uint32_t n, void *stream) {
   if (!e || tier > 1 || (!slots && n)) return KVT_E_INVAL;
-  u32 done = 0, live = 0, drop = 0;
-  return list_op(e, (cudaStream_t)stream, tier, tier, slots, n, false, false, true, &done, &live, &drop);
+  ListMode m{};
+  m.drop_all = true;
+  ListCounts c;
+  return list_op(e, (cudaStream_t)stream, tier, tier, slots, n, m, &c);
 }
 
 int32_t kvt_compact(kvt_engine *e, uint32_t tier, uint32_t *n_moved, void *stream) {

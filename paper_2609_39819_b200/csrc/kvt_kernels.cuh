@@ -29,7 +29,8 @@ enum : u32 { DERR_PROBE = 1, DERR_RANGE = 2, DERR_INVAL = 4, DERR_STATE = 8, DER
 // words of the device status block
 enum : int {
   ST_ERR = 0, ST_TOTAL, ST_CUT, ST_NLIVE, ST_NDROP, ST_NEW, ST_INSERTED, ST_ADOPTED, ST_TOMBS,
-  ST_RANK0, ST_RANK1, ST_RANK2, ST_RANK3, ST_M, ST_NMOVED, ST_FREE, ST_AUX, ST_WORDS = 32
+  ST_RANK0, ST_RANK1, ST_RANK2, ST_RANK3, ST_M, ST_NMOVED, ST_FREE, ST_AUX, ST_SHADOW, ST_NCLEAN, ST_NSHDROP,
+  ST_WORDS = 32
 };
 
 struct __align__(16) TSlot { u64 key; u32 ent; u32 pad; };
@@ -66,9 +67,13 @@ struct Table { TSlot *slots; u32 mask; u32 shift; };   // capacity = mask + 1, h
 struct Entries {            // per resident-block metadata, entry id = slot (HBM) or n_hbm + slot (host)
   u64 *key;                 // 0 = free
   u32 *stamp, *depth, *infl, *rank, *tslot, *mark;
+  u32 *link;                // inclusive tiering: an HBM block and its clean host copy point at each other (else ENT_NONE)
   u8 *floor;
   u32 n_hbm, n_total;
 };
+
+// A host entry that only holds a clean copy of a block whose home is in HBM.
+__device__ __forceinline__ bool is_shadow(const Entries &en, u32 e) { return e >= en.n_hbm && en.link[e] != ENT_NONE; }
 
 __device__ __forceinline__ void set_err(u32 *status, u32 bits) { atomicOr(&status[ST_ERR], bits); }
 
@@ -339,7 +344,7 @@ __global__ void k_table_reinsert(Table t, Entries en, u32 *status) {
   u32 e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e >= en.n_total) return;
   u64 key = en.key[e];
-  if (!key) return;
+  if (!key || is_shadow(en, e)) return;   // a clean host copy is not in the table: its block is
   u32 s = tab_find_or_claim(t, key, status);
   if (s == ENT_NONE) return;
   t.slots[s].ent = e;
@@ -438,7 +443,7 @@ __global__ void k_admit_apply(AdmitArgs a) {
     if (held) {
       u32 e = a.freelist[a.krank[g]];
       a.ent.key[e] = a.keys[c.key_off + b];
-      a.ent.stamp[e] = a.now; a.ent.depth[e] = b; a.ent.rank[e] = 2; a.ent.floor[e] = 0; a.ent.tslot[e] = s;
+      a.ent.stamp[e] = a.now; a.ent.depth[e] = b; a.ent.rank[e] = 2; a.ent.floor[e] = 0; a.ent.tslot[e] = s; a.ent.link[e] = ENT_NONE;
       atomicAdd(&a.ent.infl[e], 1u);
       a.tab.slots[s].ent = e;
       atomicAdd(&a.status[ST_INSERTED], 1u);
@@ -527,32 +532,39 @@ struct SelArgs {
   u32 *status;
 };
 
-__device__ __forceinline__ bool sel_candidate(const SelArgs &a, u32 i, u32 *rank) {
+// Class of slot i for the selection: 0..3 = candidate of that rank, SEL_SHADOW = clean host copy of an HBM
+// block (always a candidate, goes first: dropping it loses nothing), SEL_NOT = not a candidate.
+constexpr u32 SEL_SHADOW = 0xFE, SEL_NOT = 0xFF;
+__device__ __forceinline__ u32 sel_class(const SelArgs &a, u32 i) {
   u32 e = a.e0 + i;
-  if (!a.ent.key[e] || a.ent.infl[e]) return false;
+  if (!a.ent.key[e]) return SEL_NOT;
+  if (is_shadow(a.ent, e)) return SEL_SHADOW;
+  if (a.ent.infl[e]) return SEL_NOT;
   u32 r = a.one_tier ? 1u : a.ent.rank[e];   // without lifecycle tracking every block is one tier
-  *rank = r;
-  return r <= a.max_rank;
+  return r <= a.max_rank ? r : SEL_NOT;
 }
 
 __global__ void k_sel_count(SelArgs a) {
-  __shared__ u32 s[4];
-  if (threadIdx.x < 4) s[threadIdx.x] = 0;
+  __shared__ u32 s[5];
+  if (threadIdx.x < 5) s[threadIdx.x] = 0;
   __syncthreads();
   u32 i = blockIdx.x * blockDim.x + threadIdx.x;
-  u32 r = 0;
-  bool c = i < a.n_slots && sel_candidate(a, i, &r);
-  for (u32 k = 0; k < 4; ++k) {
-    u32 m = __ballot_sync(0xFFFFFFFFu, c && r == k);
+  u32 c = i < a.n_slots ? sel_class(a, i) : SEL_NOT;
+  for (u32 k = 0; k < 5; ++k) {
+    u32 m = __ballot_sync(0xFFFFFFFFu, c == (k == 4 ? SEL_SHADOW : k));
     if ((threadIdx.x & 31) == 0 && m) atomicAdd(&s[k], __popc(m));
   }
   __syncthreads();
   if (threadIdx.x < 4 && s[threadIdx.x]) atomicAdd(&a.status[ST_RANK0 + threadIdx.x], s[threadIdx.x]);
+  if (threadIdx.x == 4 && s[4]) atomicAdd(&a.status[ST_SHADOW], s[4]);
 }
 
-// Highest rank that must be looked at to serve n_req victims (Algorithm 1: lower ranks go first).
-__device__ __forceinline__ u32 sel_boundary_rank(const u32 *status, u32 n_req) {
-  u32 cum = status[ST_RANK0];
+// Highest rank that must be looked at to serve n_req victims (Algorithm 1: lower ranks go first; clean host
+// copies go before everything). -1: the copies alone suffice.
+__device__ __forceinline__ int sel_boundary_rank(const u32 *status, u32 n_req) {
+  u32 cum = status[ST_SHADOW];
+  if (cum >= n_req) return -1;
+  cum += status[ST_RANK0];
   if (cum >= n_req) return 0;
   cum += status[ST_RANK1];
   if (cum >= n_req) return 1;
@@ -564,19 +576,23 @@ __device__ __forceinline__ u32 sel_boundary_rank(const u32 *status, u32 n_req) {
 struct PredSel {
   SelArgs a;
   __device__ bool operator()(u32 i) const {
-    u32 r;
-    return sel_candidate(a, i, &r) && r <= sel_boundary_rank(a.status, a.n_req);
+    u32 c = sel_class(a, i);
+    if (c == SEL_NOT) return false;
+    return c == SEL_SHADOW || (int)c <= sel_boundary_rank(a.status, a.n_req);
   }
 };
 struct EmitSel {
   SelArgs a; u64 *keys; u32 *vals;
   __device__ void operator()(u32 i, u32 pos) const {
     u32 e = a.e0 + i;
-    u64 r = a.one_tier ? 1u : a.ent.rank[e];
+    const bool sh = is_shadow(a.ent, e);
+    u64 r = sh ? 0u : (a.one_tier ? 1u : a.ent.rank[e]);
     u64 st = a.ent.stamp[e];
-    u64 rec = (r == 1 && a.mru) ? (u64)a.now - st : st;       // newest first inside the idle tier
-    u64 dinv = ((1ull << a.depth_bits) - 1) - a.ent.depth[e];  // chain tail first
-    keys[pos] = (r << (a.stamp_bits + a.depth_bits)) | (rec << a.depth_bits) | dinv;
+    u64 rec = (r == 1 && a.mru && !sh) ? (u64)a.now - st : st;  // newest first inside the idle tier
+    u64 dinv = ((1ull << a.depth_bits) - 1) - a.ent.depth[e];   // chain tail first
+    u64 primary = sh ? 0u : 1u;                                  // copies sort before resident blocks
+    keys[pos] = (primary << (2 + a.stamp_bits + a.depth_bits)) | (r << (a.stamp_bits + a.depth_bits)) |
+                (rec << a.depth_bits) | dinv;
     vals[pos] = i;
   }
 };
@@ -679,11 +695,19 @@ __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const
   }
 }
 
-__global__ void k_sel_emit(const u64 *keys, const u32 *vals, u32 n, u32 rank_shift, u32 *slots_out, u8 *states_out) {
+// Victim list for the caller: slot, and its state: the rank, | 0x80 for an HBM block that still has a clean host
+// copy (moving it out needs no copy), or 0xFE for a host slot that is such a copy.
+__global__ void k_sel_emit(Entries en, u32 e0, u32 n_slots, const u64 *keys, const u32 *vals, u32 n, const u32 *status,
+                           u32 rank_shift, u32 *slots_out, u8 *states_out) {
   u32 i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n) return;
-  slots_out[i] = vals[i];
-  states_out[i] = (u8)(keys[i] >> rank_shift);
+  if (i >= n || i >= status[ST_M]) return;   // only the first ST_M entries of the sorted list exist
+  u32 slot = vals[i];
+  if (slot >= n_slots) return;
+  slots_out[i] = slot;
+  u64 k = keys[i] >> rank_shift;
+  bool primary = (k >> 2) & 1;
+  u32 link = en.link[e0 + slot];
+  states_out[i] = !primary ? (u8)0xFE : (u8)((k & 3) | (link != ENT_NONE ? 0x80 : 0));
 }
 
 // ======================================================================================================
@@ -693,24 +717,34 @@ struct ListArgs {
   Table tab; Entries ent;
   const u32 *ids; u32 n; u32 e0, n_slots;   // listed slots of the source tier (entry = e0 + id)
   u32 dst_e0;                                // first entry id of the destination tier
-  u32 *live;                                 // per item: 1 = must be copied
-  u32 *lidx;                                 // per item: exclusive rank among live items
+  u32 *live;                                 // per item: LIST_DROP, LIST_COPY (needs a free destination slot), LIST_CLEAN
+  u32 *lidx;                                 // per item: exclusive rank among LIST_COPY items
   const u32 *freelist; u32 n_free;           // lowest free destination slots
   u32 *pair_src, *pair_dst;                  // mover pairs, indexed by lidx
   u32 allow_inflight; u32 drop_dead; u32 drop_all;
+  u32 reject_shadow;                         // reload: a host slot that is only a copy is not a resident block
+  u32 clean_ok;                              // offload: a block with a clean host copy is handed over without a copy
+  u32 keep_copy;                             // reload with inclusive tiers: the host slot stays as a clean copy
   u32 *status;
 };
+enum : u32 { LIST_DROP = 0, LIST_COPY = 1, LIST_CLEAN = 2 };
 
 __global__ void k_list_validate(ListArgs a) {
   u32 i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= a.n) return;
   u32 id = a.ids[i];
-  a.live[i] = 0;
+  a.live[i] = LIST_DROP;
   if (id >= a.n_slots) { set_err(a.status, DERR_RANGE); return; }
   u32 e = a.e0 + id;
-  if (!a.ent.key[e] || atomicAdd(&a.ent.mark[e], 1u) != 0) { set_err(a.status, DERR_INVAL); return; }
+  if (!a.ent.key[e] || atomicAdd(&a.ent.mark[e], 1u) != 0 || (a.reject_shadow && is_shadow(a.ent, e))) {
+    set_err(a.status, DERR_INVAL);
+    return;
+  }
   if (a.ent.infl[e] && !a.allow_inflight) set_err(a.status, DERR_STATE);
-  a.live[i] = (a.drop_all || (a.drop_dead && a.ent.rank[e] == 0)) ? 0u : 1u;
+  u32 cat = LIST_COPY;
+  if (a.drop_all || (a.drop_dead && a.ent.rank[e] == 0)) cat = LIST_DROP;
+  else if (a.clean_ok && a.ent.link[e] != ENT_NONE) cat = LIST_CLEAN;
+  a.live[i] = cat;
 }
 
 __global__ void k_list_unmark(ListArgs a) {
@@ -720,8 +754,8 @@ __global__ void k_list_unmark(ListArgs a) {
   if (id < a.n_slots) a.ent.mark[a.e0 + id] = 0;
 }
 
-struct PredLive { const u32 *live; __device__ bool operator()(u32 i) const { return live[i] != 0; } };
-// live item with rank r needs the r-th free destination slot; the first one that does not fit cuts the list
+struct PredLive { const u32 *live; __device__ bool operator()(u32 i) const { return live[i] == LIST_COPY; } };
+// item with rank r needs the r-th free destination slot; the first one that does not fit cuts the list
 struct EmitLive {
   u32 *lidx; u32 n_free; u32 *status;
   __device__ void operator()(u32 i, u32 r) const { lidx[i] = r; if (r >= n_free) atomicMin(&status[ST_CUT], i); }
@@ -731,14 +765,19 @@ struct EmitFree { u32 *list; u32 cap; __device__ void operator()(u32 i, u32 r) c
 
 __device__ __forceinline__ void entry_clear(const Entries &en, u32 e) {
   en.key[e] = 0; en.stamp[e] = 0; en.depth[e] = 0; en.infl[e] = 0; en.rank[e] = 0; en.floor[e] = 0; en.tslot[e] = ENT_NONE;
+  en.link[e] = ENT_NONE;
 }
 
+// Moves an entry (and whatever points at it: its table slot, its linked copy / block) to a free entry.
 __device__ __forceinline__ void entry_move(const Table &t, const Entries &en, u32 src, u32 dst) {
   en.key[dst] = en.key[src]; en.stamp[dst] = en.stamp[src]; en.depth[dst] = en.depth[src];
   en.infl[dst] = en.infl[src]; en.rank[dst] = en.rank[src]; en.floor[dst] = en.floor[src];
   u32 s = en.tslot[src];
   en.tslot[dst] = s;
-  t.slots[s].ent = dst;
+  if (s != ENT_NONE) t.slots[s].ent = dst;
+  u32 l = en.link[src];
+  en.link[dst] = l;
+  if (l != ENT_NONE) en.link[l] = dst;
   entry_clear(en, src);
 }
 
@@ -749,18 +788,47 @@ __global__ void k_list_apply(ListArgs a) {
   if (i >= a.status[ST_CUT]) return;
   u32 id = a.ids[i];
   u32 e = a.e0 + id;
-  if (!a.live[i]) {  // reclaim without copy: tombstone the key, free the slot
-    u32 s = a.ent.tslot[e];
-    a.tab.slots[s].key = KEY_TOMB;
-    a.tab.slots[s].ent = ENT_NONE;
+  u32 cat = a.live[i];
+  if (cat == LIST_DROP) {
+    if (is_shadow(a.ent, e)) {           // dropping a copy: the block lives on in HBM
+      a.ent.link[a.ent.link[e]] = ENT_NONE;
+    } else {                             // reclaim without copy: tombstone the key; a clean copy goes too
+      u32 s = a.ent.tslot[e];
+      a.tab.slots[s].key = KEY_TOMB;
+      a.tab.slots[s].ent = ENT_NONE;
+      atomicAdd(&a.status[ST_TOMBS], 1u);
+      u32 l = a.ent.link[e];
+      if (l != ENT_NONE) { entry_clear(a.ent, l); atomicAdd(&a.status[ST_NSHDROP], 1u); }
+    }
     entry_clear(a.ent, e);
     atomicAdd(&a.status[ST_NDROP], 1u);
+  } else if (cat == LIST_CLEAN) {        // hand the block over to its clean host copy: metadata only
+    u32 h = a.ent.link[e];
+    a.ent.stamp[h] = a.ent.stamp[e]; a.ent.depth[h] = a.ent.depth[e]; a.ent.infl[h] = a.ent.infl[e];
+    a.ent.rank[h] = a.ent.rank[e]; a.ent.floor[h] = a.ent.floor[e];
+    u32 s = a.ent.tslot[e];
+    a.ent.tslot[h] = s;
+    a.tab.slots[s].ent = h;
+    a.ent.link[h] = ENT_NONE;
+    entry_clear(a.ent, e);
+    atomicAdd(&a.status[ST_NCLEAN], 1u);
   } else {
     u32 r = a.lidx[i];
     u32 d = a.freelist[r];
     a.pair_src[r] = id;
     a.pair_dst[r] = d;
-    entry_move(a.tab, a.ent, e, a.dst_e0 + d);
+    u32 de = a.dst_e0 + d;
+    if (a.keep_copy) {                   // the block moves to HBM, the host slot stays behind as its clean copy
+      a.ent.key[de] = a.ent.key[e]; a.ent.stamp[de] = a.ent.stamp[e]; a.ent.depth[de] = a.ent.depth[e];
+      a.ent.infl[de] = a.ent.infl[e]; a.ent.rank[de] = a.ent.rank[e]; a.ent.floor[de] = a.ent.floor[e];
+      u32 s = a.ent.tslot[e];
+      a.ent.tslot[de] = s;
+      a.tab.slots[s].ent = de;
+      a.ent.link[de] = e;
+      a.ent.link[e] = de; a.ent.tslot[e] = ENT_NONE; a.ent.infl[e] = 0;
+    } else {
+      entry_move(a.tab, a.ent, e, de);
+    }
     atomicAdd(&a.status[ST_NLIVE], 1u);
   }
 }
@@ -796,12 +864,12 @@ __global__ void k_load_apply(LoadArgs a) {
   if (s == ENT_NONE) return;
   a.tab.slots[s].ent = e;
   a.ent.key[e] = a.keys[i]; a.ent.stamp[e] = a.stamp[i]; a.ent.depth[e] = a.depth[i];
-  a.ent.infl[e] = 0; a.ent.rank[e] = a.state[i]; a.ent.floor[e] = a.state[i]; a.ent.tslot[e] = s;
+  a.ent.infl[e] = 0; a.ent.rank[e] = a.state[i]; a.ent.floor[e] = a.state[i]; a.ent.tslot[e] = s; a.ent.link[e] = ENT_NONE;
 }
 
 __global__ void k_states_out(Entries en, u32 e0, u32 n, u8 *out) {
   u32 i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) out[i] = en.key[e0 + i] ? (u8)en.rank[e0 + i] : (u8)0xFF;
+  if (i < n) out[i] = en.key[e0 + i] ? (is_shadow(en, e0 + i) ? (u8)0xFE : (u8)en.rank[e0 + i]) : (u8)0xFF;
 }
 
 // ======================================================================================================

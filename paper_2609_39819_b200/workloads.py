@@ -23,6 +23,7 @@ MAP_LOOKUP, MAP_ADMIT = 0, 1
 GiB = 1 << 30
 GPU_ONLY_STATS = ("table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns", "mover_bytes",
                   "lookup_ns", "lookup_blocks", "select_ns", "select_slots")
+STATE_COPY, STATE_HAS_COPY = 0xFE, 0x80
 
 
 # ------------------------------------------------------------------------------------------------
@@ -307,7 +308,8 @@ def evict(eng, n, n_pinned_incoming=0):
         victims, vstates = eng.select_victims(TIER_HBM, want, include_pinned=True)
     rec["victims"] = victims.copy()
     rec["vstates"] = vstates.copy()
-    n_live = int((vstates > 0).sum())
+    # victims that need a free host slot: live ones without a clean host copy
+    n_live = int((((vstates & 0x7F) > 0) & ((vstates & STATE_HAS_COPY) == 0)).sum())
     free_host = eng.n_host_blocks - eng.get_stats()["occ_host"]
     if n_live > free_host:
         hv, hs = eng.select_victims(TIER_HOST, n_live - free_host)

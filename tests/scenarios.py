@@ -247,6 +247,71 @@ def no_lifecycle_policy(make):
     assert list(eng2.select_victims(HBM, 3)[0]) == [0, 2, 1]      # plain LRU
 
 
+# ---- inclusive tiering: a reloaded block keeps its host copy, a later offload of it needs no copy ----------
+SHADOW, HAS_COPY, NONE = 0xFE, 0x80, 0xFFFFFFFF
+
+
+def inclusive_tiers(make):
+    eng = make(n_hbm_blocks=6, n_host_blocks=6, max_contexts=4, policy_flags=2, **TOY)
+    rng = np.random.default_rng(18)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 64))
+    call(eng, 0)                                         # blocks 0..3 at HBM slots 0..3
+    keys = eng.get_block_map(0)[0]
+    for b in range(4):
+        eng.write_block(HBM, b, _payload(keys[b], eng.block_bytes))
+    assert eng.offload([3, 2]) == (0, 2, 0)              # copied to host slots 0 (block 3) and 1 (block 2)
+    a = eng.map_blocks([0], LOOKUP)[0]
+    assert (a["hit_len"], a["n_hit_hbm"], a["n_hit_host"]) == (4, 2, 2)
+    assert eng.reload([1, 0]) == (0, 2)                  # block 2 -> HBM slot 2, block 3 -> HBM slot 3
+    st = eng.get_stats()
+    assert (st["occ_hbm"], st["occ_host"], st["bytes_h2d"]) == (4, 2, 2 * eng.block_bytes)   # host copies stay
+    assert states(eng, HOST)[:3] == [SHADOW, SHADOW, FREE]
+    assert list(eng.get_entries(HBM)["link"][:4]) == [NONE, NONE, 1, 0]
+    assert list(eng.get_entries(HOST)["link"][:2]) == [3, 2]
+    assert list(eng.get_block_map(0)[1]) == [HBM] * 4    # the block's home is HBM again
+    assert eng.reload([0])[0] == E_INVAL                 # a copy is not a resident block of the host tier
+    eng.map_blocks([0], ADMIT)
+    eng.prefill_done(0)
+    v, s = eng.select_victims(HBM, 4)
+    assert list(v) == [3, 2, 1, 0] and list(s) == [IDLE | HAS_COPY, IDLE | HAS_COPY, IDLE, IDLE]
+    d2h = eng.get_stats()["bytes_d2h"]
+    assert eng.offload([3, 2]) == (0, 2, 0)              # handed over to their host copies: nothing is copied
+    st = eng.get_stats()
+    assert (st["occ_hbm"], st["occ_host"], st["bytes_d2h"], st["offloaded"], st["offloaded_clean"]) == (2, 2, d2h, 4, 2)
+    assert states(eng, HOST)[:2] == [IDLE, IDLE] and list(eng.get_entries(HOST)["link"][:2]) == [NONE, NONE]
+    k, t, sl = eng.get_block_map(0)
+    assert list(t) == [HBM, HBM, HOST, HOST] and list(sl) == [0, 1, 1, 0]
+    for b in range(4):
+        assert np.array_equal(eng.read_block(int(t[b]), int(sl[b])), _payload(keys[b], eng.block_bytes))
+    # copies are the first victims of the host tier (dropping them loses nothing) and may be released
+    assert eng.reload([1, 0]) == (0, 2)
+    v, s = eng.select_victims(HOST, 6)
+    assert list(v) == [0, 1] and list(s) == [SHADOW, SHADOW]     # same stamp: deeper block first
+    eng.release(HOST, [0])                               # drop the copy of block 3
+    assert list(eng.get_entries(HBM)["link"][:4]) == [NONE, NONE, 1, NONE]
+    assert eng.get_stats()["occ_host"] == 1
+    eng.release(HBM, [2])                                # drop block 2: its copy goes with it
+    st = eng.get_stats()
+    assert (st["occ_hbm"], st["occ_host"]) == (3, 0)
+    assert list(eng.get_block_map(0)[1]) == [HBM, HBM, 0xFF, HBM]
+    # compaction keeps block and copy linked
+    assert eng.offload([3]) == (0, 1, 0)                 # block 3 -> host slot 0 (copied again: its copy was dropped)
+    assert eng.reload([0]) == (0, 1)                     # back to HBM slot 2, host slot 0 is its copy
+    eng.release(HBM, [0])
+    assert eng.compact(HBM) == 1                         # 2 occupied: slot 2 moves to slot 0
+    assert list(eng.get_entries(HBM)["link"][:3]) == [0, NONE, NONE]
+    assert list(eng.get_entries(HOST)["link"][:1]) == [0]
+    assert list(eng.get_block_map(0)[2]) == [NONE, 1, NONE, 0]
+    # a dead block with a copy: both are reclaimed
+    eng.terminate(0)
+    v, s = eng.select_victims(HBM, 6)
+    assert list(s) == [DEAD | HAS_COPY, DEAD]
+    assert eng.offload(v) == (0, 2, 2)
+    st = eng.get_stats()
+    assert (st["occ_hbm"], st["occ_host"]) == (0, 0)
+
+
 # ---- hand-worked lifecycle example (8-block pool) --------------------------------------------------
 def worked_example(make):
     eng = make(n_hbm_blocks=8, n_host_blocks=8, max_contexts=4, **TOY)
@@ -595,4 +660,4 @@ def degenerate_inputs(make):
 ALL = [state_machine_single_context, suffix_invalidation, fork_and_shared_kv, one_off_bypass, worked_example,
        mixed_pool_example, victim_order_bruteforce, one_state_pools_reduce_to_lru, offload_reload_round_trip,
        dead_victims_are_dropped_without_copy, compaction, raw_copy_blocks, admission_stops_when_full,
-       lookup_locks_and_orphans, degenerate_inputs, pinned_retention, no_lifecycle_policy]
+       lookup_locks_and_orphans, degenerate_inputs, pinned_retention, no_lifecycle_policy, inclusive_tiers]

@@ -134,6 +134,34 @@ def test_trace_parity_without_lifecycle_tracking(B, oracle, order, flags):
     assert mg == mc
 
 
+@pytest.mark.parametrize("flags", [2, 3])
+def test_trace_parity_with_inclusive_tiers(B, oracle, flags):
+    """Inclusive tiering (and its combination with the no-lifecycle policy): reloaded blocks keep a clean host
+    copy, later offloads of them move no bytes; every reported value and every payload byte still matches."""
+    for seed in (7, 63, 86):
+        kw = dict(n_hbm_blocks=96, n_host_blocks=256, max_contexts=64, policy_flags=flags, **W.GEO_TOY.kwargs())
+        gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)
+        cpu = oracle.OracleEngine(**kw)
+        _replay_pair(gpu, cpu, W.trace_c1(seed), W.payload_pattern, verify_every=1)
+    trace, n_ctx = W.trace_c3(1, n_sessions=8, scale=1 / 32)
+    kw = dict(n_hbm_blocks=256, n_host_blocks=320, max_contexts=n_ctx, policy_flags=flags, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 20, max_messages=1 << 15, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    _replay_pair(gpu, cpu, trace, W.payload_pattern, verify_every=5)
+    st = cpu.get_stats()
+    assert st["offloaded_clean"] > 0 and st["reloaded"] > 0
+    # force a table rebuild with copies present, then look everything up again
+    keys = cpu.get_entries(0)["key"]
+    for eng in (gpu, cpu):
+        v, s = eng.select_victims(0, int((keys != 0).sum()))
+        eng.offload(v)
+    for tier in (0, 1):
+        eg, ec = gpu.get_entries(tier), cpu.get_entries(tier)
+        for k in ec:
+            assert np.array_equal(eg[k], ec[k]), (tier, k)
+        assert np.array_equal(gpu.get_states(tier), cpu.get_states(tier))
+
+
 def test_scaled_c2_trace_parity(B, oracle):
     kw = dict(n_hbm_blocks=96, n_host_blocks=64, max_contexts=8, **W.GEO_TOY.kwargs())
     gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)
