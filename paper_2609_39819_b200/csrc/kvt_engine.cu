@@ -752,7 +752,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     lk.now = e->now; lk.status = e->d_status;
     if (e->profiling) CU(cudaEventRecord(e->ev_h0, s));
     KL(k_hash_digest, chunk_base, CHUNK, s, ha);
-    KL(k_hash_carry, cdiv((u64)nd * 32, 128), 128, s, ha);
+    KL(k_hash_carry, nd, 1024, s, ha);
     KL(k_hash_finish_lookup, chunk_base, CHUNK, s, ha, la);
     KL(k_lock_hits, chunk_base, CHUNK, s, ha, lk);
     if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));
@@ -1202,7 +1202,7 @@ int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t ha
   ha.agg = (u64 *)d_scratch; ha.carry = (u64 *)d_scratch + n_chunks; ha.h0 = hash_h0(hash_seed);
   LookupArgs la{};
   k_hash_digest<<<n_chunks, CHUNK, 0, s>>>(ha);
-  k_hash_carry<<<1, 32, 0, s>>>(ha);
+  k_hash_carry<<<1, 1024, 0, s>>>(ha);
   k_hash_finish_lookup<<<n_chunks, CHUNK, 0, s>>>(ha, la);
   return cudaGetLastError() == cudaSuccess ? KVT_OK : KVT_E_CUDA;
 }
@@ -1236,7 +1236,7 @@ int32_t kvt_hash_tokens_noalloc(const uint32_t *d_tokens, uint64_t n_tokens, uin
   ha.agg = g_noalloc_ptr[dev]; ha.carry = g_noalloc_ptr[dev] + NOALLOC_MAX_CHUNKS; ha.h0 = hash_h0(hash_seed);
   LookupArgs la{};
   k_hash_digest<<<n_chunks, CHUNK, 0, s>>>(ha);
-  k_hash_carry<<<1, 32, 0, s>>>(ha);
+  k_hash_carry<<<1, 1024, 0, s>>>(ha);
   k_hash_finish_lookup<<<n_chunks, CHUNK, 0, s>>>(ha, la);
   return cudaGetLastError() == cudaSuccess ? KVT_OK : KVT_E_CUDA;
 }

@@ -112,7 +112,7 @@ __device__ __forceinline__ u32 tab_find_or_claim(const Table &t, u64 key, u32 *s
 // K1: block hasher. 3 phases, no inter-CTA waits:
 //   digest : per 256-block chunk, 4 lanes per block read 16 B each, weighted sums, mix, then a CTA-wide
 //            scan of the affine chain with zero carry-in -> partial chain values + chunk aggregate
-//   carry  : one warp per context scans its chunk aggregates, 32 chunks per step
+//   carry  : one CTA per context scans its chunk aggregates, 1024 chunks per step
 //   finish : h = P^(i+1) * carry + partial, key = mix64(h); fused with the table probe
 // ======================================================================================================
 struct HashCtx { u64 tok_off; u64 key_off; u32 n_blocks; u32 chunk_base; u32 blk_base; u32 pad; };
@@ -130,6 +130,21 @@ __device__ __forceinline__ const HashCtx &hash_ctx_of_chunk(const HashArgs &a, u
   return a.ctx[lo];
 }
 
+// Lane multipliers K[0..15] as a constant-initialised table (read once per thread, L1-resident).
+struct LaneTable {
+  u64 v[16];
+  constexpr LaneTable() : v() { for (u32 t = 0; t < 16; ++t) v[t] = lane_mult(t); }
+};
+__device__ const LaneTable g_lane_mult = LaneTable();
+
+// tok * K mod 2^64 for a 32-bit token: one widening multiply-add for the low word of K, one 32-bit multiply for
+// its high word (a full 64 x 64 multiply costs twice as much on the integer pipe, which bounds this kernel).
+__device__ __forceinline__ u64 mul_tok(u32 tok, u64 k) {
+  u64 lo = (u64)tok * (u32)k;
+  u32 hi = tok * (u32)(k >> 32);
+  return lo + ((u64)hi << 32);
+}
+
 __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   __shared__ u64 sd[CHUNK];
   __shared__ u64 wagg[CHUNK / 32];
@@ -140,20 +155,28 @@ __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   const u32 nb = min(CHUNK, c.n_blocks - b0);
   const uint4 *tok = reinterpret_cast<const uint4 *>(a.tokens + c.tok_off + (u64)b0 * 16);
   const u32 q = tid & 3;
-  const u64 k0 = lane_mult(4 * q), k1 = lane_mult(4 * q + 1), k2 = lane_mult(4 * q + 2), k3 = lane_mult(4 * q + 3);
+  const u64 k0 = g_lane_mult.v[4 * q], k1 = g_lane_mult.v[4 * q + 1], k2 = g_lane_mult.v[4 * q + 2],
+            k3 = g_lane_mult.v[4 * q + 3];
+  const u64 ksum = k0 + k1 + k2 + k3;   // sum (tok + 1) K = sum tok K + sum K
   uint4 v[4];
 #pragma unroll
   for (int it = 0; it < 4; ++it) {
     u32 idx = it * CHUNK + tid;
     v[it] = (idx >> 2) < nb ? __ldg(tok + idx) : make_uint4(0, 0, 0, 0);
   }
+  // iteration `it` covers blocks it*64 .. it*64+63, four lanes per block; after the two exchange steps every
+  // lane of a quad holds the four block sums, and lane q finishes the block of iteration q
+  u64 mine = 0;
 #pragma unroll
   for (int it = 0; it < 4; ++it) {
-    u32 blk = (it * CHUNK + tid) >> 2;
-    u64 s = ((u64)v[it].x + 1) * k0 + ((u64)v[it].y + 1) * k1 + ((u64)v[it].z + 1) * k2 + ((u64)v[it].w + 1) * k3;
+    u64 s = ksum + mul_tok(v[it].x, k0) + mul_tok(v[it].y, k1) + mul_tok(v[it].z, k2) + mul_tok(v[it].w, k3);
     s += __shfl_xor_sync(0xFFFFFFFFu, s, 1);
     s += __shfl_xor_sync(0xFFFFFFFFu, s, 2);
-    if (q == 0) sd[blk] = blk < nb ? mix64(s) : 0;
+    if ((u32)it == q) mine = s;
+  }
+  {
+    u32 blk = (q * CHUNK + tid) >> 2;
+    sd[blk] = blk < nb ? mix64(mine) : 0;
   }
   __syncthreads();
   // inclusive scan of c_t = sum_{i<=t} P^(t-i) d_i
@@ -175,19 +198,23 @@ __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   if (tid == nb - 1) a.agg[blockIdx.x] = cval;
 }
 
-// One warp per context: the chain value entering chunk j is A^j * H0 + sum_{i<j} A^(j-1-i) * agg_i with
-// A = P^CHUNK (every chunk before the last is full), evaluated 32 chunks at a time by a warp scan.
-__global__ void __launch_bounds__(128) k_hash_carry(HashArgs a) {
-  const u32 lane = threadIdx.x & 31;
-  const u32 i = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+// One CTA per context: the chain value entering chunk j is A^j * H0 + sum_{i<j} A^(j-1-i) * agg_i with
+// A = P^CHUNK (every chunk before the last is full), evaluated 1024 chunks at a time: a warp scan per 32 chunks,
+// a scan of the 32 warp totals, then the carry of the previous 1024.
+__global__ void __launch_bounds__(1024) k_hash_carry(HashArgs a) {
+  __shared__ u64 wtot[32], wpre[32], sv[1024];
+  const u32 i = blockIdx.x;
   if (i >= a.n_ctx) return;
+  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const HashCtx c = a.ctx ? a.ctx[i] : a.single;
   const u32 n_chunks = (c.n_blocks + CHUNK - 1) / CHUNK;
   const u64 A = g_pow_p.v[CHUNK];
-  const u64 a_lane = pow_u64(A, lane + 1);
+  const u64 A32 = pow_u64(A, 32);
+  const u64 a_lane = pow_u64(A, lane + 1);          // A^(lane+1)
+  const u64 a_tid = pow_u64(A32, warp) * a_lane;    // A^(tid+1)
   u64 carry = a.h0;
-  for (u32 j0 = 0; j0 < n_chunks; j0 += 32) {
-    const u32 j = j0 + lane;
+  for (u32 base = 0; base < n_chunks; base += 1024) {
+    const u32 j = base + tid;
     u64 x = j < n_chunks ? a.agg[c.chunk_base + j] : 0;
     u64 pp = A;
 #pragma unroll
@@ -196,11 +223,25 @@ __global__ void __launch_bounds__(128) k_hash_carry(HashArgs a) {
       if (lane >= o) x += pp * up;
       pp *= pp;
     }
-    const u64 v = a_lane * carry + x;                       // chain value after chunk j
-    u64 in = __shfl_up_sync(0xFFFFFFFFu, v, 1);
-    if (lane == 0) in = carry;
-    if (j < n_chunks) a.carry[c.chunk_base + j] = in;
-    carry = __shfl_sync(0xFFFFFFFFu, v, 31);
+    if (lane == 31) wtot[warp] = x;
+    __syncthreads();
+    if (warp == 0) {   // value at the end of every earlier warp of this round, with zero carry-in
+      u64 y = wtot[lane], qq = A32;
+#pragma unroll
+      for (u32 o = 1; o < 32; o <<= 1) {
+        u64 up = __shfl_up_sync(0xFFFFFFFFu, y, o);
+        if (lane >= o) y += qq * up;
+        qq *= qq;
+      }
+      u64 e = __shfl_up_sync(0xFFFFFFFFu, y, 1);
+      wpre[lane] = lane ? e : 0;
+    }
+    __syncthreads();
+    sv[tid] = a_tid * carry + a_lane * wpre[warp] + x;   // chain value after chunk j
+    __syncthreads();
+    if (j < n_chunks) a.carry[c.chunk_base + j] = tid ? sv[tid - 1] : carry;
+    carry = sv[1023];
+    __syncthreads();
   }
 }
 

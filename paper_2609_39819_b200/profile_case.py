@@ -3,6 +3,8 @@ larger than L2, a few GB on the device at most, a handful of launches).
 
     python -m paper_2609_39819_b200.profile_case mover      # paged KV mover, 8B-class blocks, HBM -> HBM
     python -m paper_2609_39819_b200.profile_case mover_toy  # the same with 16 KiB blocks (4 KiB chunks)
+    python -m paper_2609_39819_b200.profile_case mover_host # the same blocks, HBM -> pinned host tier and back
+    python -m paper_2609_39819_b200.profile_case hash_big   # stand-alone hasher on 64 Mi tokens (256 MiB > L2)
     python -m paper_2609_39819_b200.profile_case lookup     # hash + table lookup of 16 x 16,128-block calls
     python -m paper_2609_39819_b200.profile_case select     # classify + select 10% of 1 Mi resident blocks
     python -m paper_2609_39819_b200.profile_case c4         # the whole metadata stress at full size (C4)
@@ -85,6 +87,24 @@ def main(case: str):
         gb = n * geo.block_bytes / 1e9
         print(f"{case}: {n} blocks x {geo.block_bytes} B, permuted ids, ms per launch {ms}, "
               f"read+write GB/s {[round(2 * gb / (m / 1e3), 1) for m in ms]}")
+    elif case == "mover_host":
+        geo, n_slots, n = W.GEO_8B, 768, 512
+        eng = B.Engine(n_hbm_blocks=n_slots, n_host_blocks=n, max_contexts=2, max_tokens=1 << 12, max_messages=64,
+                       max_batch_blocks=4096, zero_pools=False, **geo.kwargs())
+        src = torch.from_numpy(W.ids_c5(1, n, n_slots, True).view(np.int32)).cuda()
+        dst = torch.from_numpy(W.ids_c5(2, n, n, True).view(np.int32)).cuda()
+        g = _events(torch, lambda: eng.copy_blocks(0, src, 1, dst), 2)
+        sc = _events(torch, lambda: eng.copy_blocks(1, dst, 0, src), 2)
+        gb = n * geo.block_bytes / 1e9
+        print(f"mover_host: {n} blocks x {geo.block_bytes} B; gather to host ms {g} = {[round(gb / (m / 1e3), 1) for m in g]} GB/s; "
+              f"scatter from host ms {sc} = {[round(gb / (m / 1e3), 1) for m in sc]} GB/s")
+    elif case == "hash_big":
+        n_tok = 64 << 20
+        tok = torch.randint(0, W.VOCAB, (n_tok,), dtype=torch.int32, device="cuda")
+        ms = _events(torch, lambda: B.hash_tokens(tok, 0), 3)
+        nb = n_tok // 16
+        print(f"hash_big: {nb} blocks, ms per call {ms}, blocks/s {[round(nb / (m / 1e3)) for m in ms]}, "
+              f"GB/s at 72 B per block {[round(72 * nb / (m / 1e3) / 1e9, 1) for m in ms]}")
     elif case in ("lookup", "select"):
         n_res, n_calls = (1 << 18, 16) if case == "lookup" else (1 << 20, 4)
         inp = W.inputs_c4(1, n_resident=n_res, chain_blocks=16128, n_calls=n_calls)
