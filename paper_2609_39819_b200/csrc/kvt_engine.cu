@@ -983,6 +983,7 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   a.mru = e->cfg.suspended_order == KVT_ORDER_MRU; a.status = e->d_status;
   a.max_rank = (flags & KVT_SEL_INCLUDE_PINNED) ? 3 : 2;
   a.one_tier = (e->cfg.policy_flags & KVT_POLICY_NO_LIFECYCLE) ? 1 : 0;
+  a.copy_bit = (tier == KVT_TIER_HOST && (e->cfg.policy_flags & KVT_POLICY_INCLUSIVE)) ? 1 : 0;
   u64 *kA = e->dp<u64>(e->L.keyA), *kB = e->dp<u64>(e->L.keyB);
   u32 *vA = e->dp<u32>(e->L.valA), *vB = e->dp<u32>(e->L.valB), *counts = e->dp<u32>(e->L.rcounts);
   u32 *row_total = counts + 256ull * (e->L.Nt / SORT_TILE + 1);
@@ -990,7 +991,7 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   KL(k_sel_count, cdiv(n,256), 256, s, a);
   r = compact_indices(e, s, PredSel{a}, EmitSel{a, kA, vA}, n, ST_M);
   if (r) return r;
-  const u32 key_bits = 3 + a.stamp_bits + a.depth_bits, n_pass = cdiv(key_bits, 8), tiles = cdiv(n, SORT_TILE);
+  const u32 key_bits = 2 + a.copy_bit + a.stamp_bits + a.depth_bits, n_pass = cdiv(key_bits, 8), tiles = cdiv(n, SORT_TILE);
   for (u32 p = 0; p < n_pass; ++p) {
     KL(k_radix_hist, tiles, 256, s, kA, e->d_status, 8 * p, counts);
     KL(k_radix_scan, 32, 256, s, counts, row_total, e->d_status);
@@ -998,7 +999,7 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
     std::swap(kA, kB); std::swap(vA, vB);
   }
   u32 n_emit = std::min(n_req, n);
-  KL(k_sel_emit, cdiv(n_emit,256), 256, s, e->ent, a.e0, n, kA, vA, n_emit, e->d_status, a.stamp_bits + a.depth_bits, e->dp<u32>(e->L.out_slots),
+  KL(k_sel_emit, cdiv(n_emit,256), 256, s, e->ent, a.e0, n, kA, vA, n_emit, e->d_status, a.stamp_bits + a.depth_bits, a.copy_bit, e->dp<u32>(e->L.out_slots),
                                                e->dp<u8>(e->L.out_states));
   if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));
   LAUNCH_CHECK();

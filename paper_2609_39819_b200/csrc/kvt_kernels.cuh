@@ -570,6 +570,7 @@ __global__ void k_classify(ClsArgs a) {
 struct SelArgs {
   Entries ent; u32 e0, n_slots;       // entry range of the tier
   u32 n_req; u32 now; u32 stamp_bits, depth_bits; u32 mru; u32 max_rank; u32 one_tier;
+  u32 copy_bit;                       // 1: the key carries a leading "resident block" bit (host tier with clean copies)
   u32 *status;
 };
 
@@ -632,7 +633,7 @@ struct EmitSel {
     u64 rec = (r == 1 && a.mru && !sh) ? (u64)a.now - st : st;  // newest first inside the idle tier
     u64 dinv = ((1ull << a.depth_bits) - 1) - a.ent.depth[e];   // chain tail first
     u64 primary = sh ? 0u : 1u;                                  // copies sort before resident blocks
-    keys[pos] = (primary << (2 + a.stamp_bits + a.depth_bits)) | (r << (a.stamp_bits + a.depth_bits)) |
+    keys[pos] = (a.copy_bit ? primary << (2 + a.stamp_bits + a.depth_bits) : 0) | (r << (a.stamp_bits + a.depth_bits)) |
                 (rec << a.depth_bits) | dinv;
     vals[pos] = i;
   }
@@ -739,14 +740,14 @@ __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const
 // Victim list for the caller: slot, and its state: the rank, | 0x80 for an HBM block that still has a clean host
 // copy (moving it out needs no copy), or 0xFE for a host slot that is such a copy.
 __global__ void k_sel_emit(Entries en, u32 e0, u32 n_slots, const u64 *keys, const u32 *vals, u32 n, const u32 *status,
-                           u32 rank_shift, u32 *slots_out, u8 *states_out) {
+                           u32 rank_shift, u32 copy_bit, u32 *slots_out, u8 *states_out) {
   u32 i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= n || i >= status[ST_M]) return;   // only the first ST_M entries of the sorted list exist
   u32 slot = vals[i];
   if (slot >= n_slots) return;
   slots_out[i] = slot;
   u64 k = keys[i] >> rank_shift;
-  bool primary = (k >> 2) & 1;
+  bool primary = copy_bit ? (k >> 2) & 1 : true;
   u32 link = en.link[e0 + slot];
   states_out[i] = !primary ? (u8)0xFE : (u8)((k & 3) | (link != ENT_NONE ? 0x80 : 0));
 }

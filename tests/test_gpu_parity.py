@@ -330,3 +330,86 @@ def test_mover_with_second_tier_in_hbm(B, oracle):
     S.offload_reload_round_trip(lambda **k: B.Engine(max_tokens=1 << 16, max_messages=256, host_pool_on_device=True, **k),
                                 geos=[W.GEO_128K.kwargs()])
     del gpu, cpu
+
+
+# ---- table maintenance and limits -------------------------------------------------------------------------
+def test_tombstones_trigger_rebuild_and_lookups_survive(B, oracle):
+    """Insert / drop cycles leave tombstones; the table is rebuilt when they pile up; every resident key is still
+    found afterwards, and the results stay equal to the oracle's."""
+    kw = dict(n_hbm_blocks=64, n_host_blocks=0, max_contexts=8, metadata_only=True, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 16, max_messages=256, table_capacity=128, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    base = np.random.default_rng(4).integers(0, W.VOCAB, 16 * 20, dtype=np.uint32)
+    for eng in (gpu, cpu):
+        eng.spawn(0)
+        eng.append(0, base)
+        eng.map_blocks([0], 0); eng.map_blocks([0], 1); eng.prefill_done(0)
+    for round_ in range(12):                       # each round: a new 40-block context is admitted, then dropped
+        toks = np.random.default_rng(100 + round_).integers(0, W.VOCAB, 16 * 40, dtype=np.uint32)
+        for eng in (gpu, cpu):
+            eng.spawn(1)
+            eng.append(1, toks)
+            eng.map_blocks([1], 0)
+            info = eng.map_blocks([1], 1)
+            assert int(info[0]["n_admitted"]) == 40
+            eng.prefill_done(1)
+            eng.terminate(1)
+            v, s = eng.select_victims(0, 40)
+            assert len(v) == 40 and np.all(s == 0)
+            assert eng.offload(v) == (0, 40, 40)
+    assert gpu.get_stats()["table_rebuilds"] >= 1
+    a, b = gpu.map_blocks([0], 0), cpu.map_blocks([0], 0)
+    assert np.array_equal(a, b) and int(a[0]["hit_len"]) == 20
+    for x, y in zip(gpu.get_block_map(0), cpu.get_block_map(0)):
+        assert np.array_equal(x, y)
+
+
+def test_admission_in_rounds_when_the_table_is_tight(B, oracle):
+    """A batch with more candidate blocks than the table may safely claim at once is admitted in several
+    rounds; the result equals one sequential pass."""
+    n = 256
+    kw = dict(n_hbm_blocks=n, n_host_blocks=0, max_contexts=8, metadata_only=True, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 18, max_messages=256, table_capacity=2 * n, **kw)   # claims capped at 3/4 * 512
+    cpu = oracle.OracleEngine(**kw)
+    rng = np.random.default_rng(5)
+    shared = rng.integers(0, W.VOCAB, 16 * 30, dtype=np.uint32)
+    toks = [np.concatenate([shared, rng.integers(0, W.VOCAB, 16 * 150, dtype=np.uint32)]) for _ in range(4)]
+    for eng in (gpu, cpu):
+        for c, t in enumerate(toks):
+            eng.spawn(c)
+            eng.append(c, t)
+        eng.map_blocks([0, 1, 2, 3], 0)
+    ag, ac = gpu.map_blocks([0, 1, 2, 3], 1), cpu.map_blocks([0, 1, 2, 3], 1)   # 720 candidates, 256 slots
+    assert np.array_equal(ag, ac)
+    assert [int(x) for x in ac["n_held"]] == [180, 106, 30, 30]
+    eg, ec = gpu.get_entries(0), cpu.get_entries(0)
+    for k in ec:
+        assert np.array_equal(eg[k], ec[k]), k
+    sg, sc = gpu.get_stats(), cpu.get_stats()
+    assert (sg["inserted"], sg["adopted"]) == (sc["inserted"], sc["adopted"]) == (256, 90)
+
+
+def test_capacity_errors_leave_the_engine_usable(B):
+    kw = dict(n_hbm_blocks=16, n_host_blocks=4, max_contexts=4, **W.GEO_TOY.kwargs())
+    eng = B.Engine(max_tokens=4096, max_messages=8, max_batch_blocks=64, max_key_blocks=128, **kw)
+    rng = np.random.default_rng(6)
+    eng.spawn(0)
+    eng.append(0, rng.integers(0, W.VOCAB, 1500, dtype=np.uint32))
+    assert eng.apply_op_rc(B.OP_APPEND, 0, tokens=rng.integers(0, W.VOCAB, 4000, dtype=np.uint32)) == B.E_NOSPACE  # token arena
+    eng.spawn(1)
+    eng.append(1, rng.integers(0, W.VOCAB, 16 * 60, dtype=np.uint32))
+    assert eng.map_blocks_rc([0, 1], 0)[0] == B.E_NOSPACE        # 93 + 60 blocks > max_batch_blocks
+    assert eng.get_stats()["clock"] == 0
+    info = eng.map_blocks([1], 0)
+    assert int(info[0]["n_blocks"]) == 60
+    adm = eng.map_blocks([1], 1)
+    assert int(adm[0]["n_admitted"]) == 16                       # pool of 16
+    eng.prefill_done(1)
+    v, s = eng.select_victims(0, 16)
+    rc, n_done, n_dropped = eng.offload(v)                       # live blocks, host tier of 4
+    assert (rc, n_done, n_dropped) == (B.E_NOSPACE, 4, 0)
+    assert "host tier full" in eng.last_error()
+    st = eng.get_stats()
+    assert (st["occ_hbm"], st["occ_host"]) == (12, 4)
+    with pytest.raises(B.KvtError):
+        eng.select_victims(2, 1)                                 # bad tier
