@@ -335,6 +335,7 @@ typedef struct kvt_stats {
   uint64_t select_ns;        /* with profiling on: device time of the selection kernels (count, compaction, sort, emit) */
   uint64_t select_slots;     /* and the tier slots they scanned */
   uint64_t offloaded_clean;  /* of `offloaded`, blocks handed to an existing clean host copy (no bytes moved) */
+  uint64_t blocks_rehashed;  /* of `blocks_hashed`, blocks whose digest was actually recomputed (the rest kept their keys) */
 } kvt_stats;
 int32_t kvt_get_stats(kvt_engine *e, kvt_stats *out);
 

@@ -56,7 +56,8 @@ CALL_INFO_DTYPE = np.dtype([(n, np.uint32) for n in ("n_blocks", "hit_len", "n_h
 STATS_FIELDS = ("clock", "n_contexts", "occ_hbm", "occ_host", "blocks_hashed", "hits_hbm", "hits_host", "misses",
                 "inserted", "adopted", "dropped", "offloaded", "reloaded", "compacted", "bytes_d2h", "bytes_h2d",
                 "bytes_d2d", "table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns",
-                "mover_bytes", "lookup_ns", "lookup_blocks", "select_ns", "select_slots", "offloaded_clean")
+                "mover_bytes", "lookup_ns", "lookup_blocks", "select_ns", "select_slots", "offloaded_clean",
+                "blocks_rehashed")
 
 _lib = None
 

@@ -59,7 +59,9 @@ struct RangeAlloc {
 };
 
 struct Msg { u32 len; u8 state; };
-struct KeySeg { u64 off = 0, cap = 0; u32 refs = 0; };
+// A key list in the key arena: keycap keys followed by one chain carry per CHUNK keys (kept so that the next
+// call can resume hashing at a chunk boundary instead of block 0).
+struct KeySeg { u64 off = 0, cap = 0, keycap = 0; u32 refs = 0; };
 
 struct Ctx {
   bool live = false, one_off = false, in_flight = false;
@@ -90,7 +92,7 @@ DevLayout make_layout(const kvt_config &c) {
   L.tab = take((u64)c.table_capacity * 16);
   L.e_key = take(N * 8); L.e_stamp = take(N * 4); L.e_depth = take(N * 4); L.e_infl = take(N * 4);
   L.e_rank = take(N * 4); L.e_tslot = take(N * 4); L.e_mark = take(N * 4); L.e_link = take(N * 4); L.e_floor = take(N);
-  L.keys = take(c.max_key_blocks * 8);
+  L.keys = take((c.max_key_blocks + c.max_key_blocks / CHUNK + 64ull * c.max_contexts) * 8);   // keys + per-chunk carries
   L.status = take(ST_WORDS * 4);
   L.s0 = take(LB * 4); L.s1 = take(LB * 4); L.s2 = take(LB * 4); L.s3 = take(LB * 4);
   L.ids = take(LB * 4); L.ids2 = take(LB * 4); L.pair_src = take(LB * 4); L.pair_dst = take(LB * 4);
@@ -98,7 +100,7 @@ DevLayout make_layout(const kvt_config &c) {
   L.tiles = take((std::max(LB, N) / SCAN_TILE + 2) * 4);
   u64 n_chunks = B / CHUNK + C + 1;
   L.agg = take(n_chunks * 8); L.carry = take(n_chunks * 8);
-  L.desc = take(C * 32);
+  L.desc = take(C * 64);
   L.ctxres = take(C * 16);
   L.m_start = take(Mm * 4); L.m_end = take(Mm * 4); L.m_rank = take(Mm);
   L.keyA = take(Nt * 8); L.keyB = take(Nt * 8); L.valA = take(Nt * 4); L.valB = take(Nt * 4);
@@ -217,12 +219,12 @@ void seg_deref(kvt_engine *e, int id) {
   if (--s.refs == 0) { e->key_alloc.release(s.off, s.cap); e->free_segs.push_back(id); }
 }
 int seg_new(kvt_engine *e, u64 n) {
-  u64 off;
-  if (!e->key_alloc.alloc(n, &off)) return -1;
+  u64 keycap = round_up(std::max<u64>(n, 1), 32), total = keycap + keycap / CHUNK + 1, off;
+  if (!e->key_alloc.alloc(total, &off)) return -1;
   int id;
   if (!e->free_segs.empty()) { id = e->free_segs.back(); e->free_segs.pop_back(); }
   else { id = (int)e->segs.size(); e->segs.emplace_back(); }
-  e->segs[id] = KeySeg{off, round_up(std::max<u64>(n, 1), e->key_alloc.align), 1};
+  e->segs[id] = KeySeg{off, round_up(total, e->key_alloc.align), keycap, 1};
   return id;
 }
 
@@ -461,10 +463,10 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   e->h0 = hash_h0(c.hash_seed);
   e->ctxs.resize(c.max_contexts);
   e->tok_alloc.init(c.max_tokens, 64);
-  e->key_alloc.init(c.max_key_blocks, 32);
+  e->key_alloc.init(c.max_key_blocks + c.max_key_blocks / CHUNK + 64ull * c.max_contexts, 32);
   // pinned staging
   u64 C = c.max_contexts, Mm = c.max_messages, LB = L.LB;
-  u64 o_status = 0, o_desc = 256, o_ctxres = o_desc + round_up(C * 32, 256), o_ms = o_ctxres + round_up(C * 16, 256),
+  u64 o_status = 0, o_desc = 256, o_ctxres = o_desc + round_up(C * 64, 256), o_ms = o_ctxres + round_up(C * 16, 256),
       o_me = o_ms + round_up(Mm * 4, 256), o_mr = o_me + round_up(Mm * 4, 256), o_ids = o_mr + round_up(Mm, 256),
       o_ids2 = o_ids + round_up(LB * 4, 256), o_out = o_ids2 + round_up(LB * 4, 256),
       total = o_out + round_up(LB * 16, 256);
@@ -709,7 +711,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
   e->now += 1;
   HashCtx *hd = reinterpret_cast<HashCtx *>(e->h_desc);
   std::vector<int> dev_idx(n_ctx, -1);
-  u32 nd = 0, chunk_base = 0, blk_base = 0;
+  u32 nd = 0, chunk_base = 0, dchunk_base = 0, blk_base = 0;
   u32 *h_hit = e->h_ctxres, *h_hbm = e->h_ctxres + e->cfg.max_contexts, *h_host = e->h_ctxres + 2 * e->cfg.max_contexts;
   for (u32 i = 0; i < n_ctx; ++i) {
     Ctx &c = e->ctxs[ids[i]];
@@ -718,19 +720,33 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     c.mat_bounds.clear();
     u32 pos = 0;
     for (const Msg &m : c.msgs) { c.mat_bounds.push_back({pos, pos + m.len}); pos += m.len; }
-    seg_deref(e, c.keyseg);
-    c.keyseg = newseg[i];
     u32 nb = (u32)(c.tok_len / 16);
+    // incremental hashing: the leading blocks this context still maps have unchanged tokens, so their keys
+    // (and the chain carries kept per chunk) are taken over; hashing resumes at the last chunk boundary
+    u32 first = 0;
+    u64 old_key_off = 0, old_carry_off = 0;
+    if (c.keyseg >= 0 && nb) {
+      first = std::min(c.valid_blocks, nb) / CHUNK * CHUNK;
+      old_key_off = e->segs[c.keyseg].off;
+      old_carry_off = old_key_off + e->segs[c.keyseg].keycap;
+    }
+    seg_deref(e, c.keyseg);   // the old list stays readable for the kernels of this call (stream order)
+    c.keyseg = newseg[i];
     c.mat_blocks = c.valid_blocks = nb;
     e->max_depth = std::max(e->max_depth, nb);
     if (nb) {
+      const KeySeg &sg = e->segs[c.keyseg];
       HashCtx d;
-      d.tok_off = c.tok_off; d.key_off = e->segs[c.keyseg].off; d.n_blocks = nb; d.chunk_base = chunk_base; d.blk_base = blk_base; d.pad = 0;
+      d.tok_off = c.tok_off; d.key_off = sg.off; d.carry_off = sg.off + sg.keycap;
+      d.old_key_off = old_key_off; d.old_carry_off = old_carry_off;
+      d.n_blocks = nb; d.first = first; d.chunk_base = chunk_base; d.dchunk_base = dchunk_base; d.blk_base = blk_base; d.pad = 0;
       h_hit[nd] = nb; h_hbm[nd] = 0; h_host[nd] = 0;
       dev_idx[i] = (int)nd;
       hd[nd++] = d;
       chunk_base += cdiv(nb, CHUNK);
+      dchunk_base += cdiv(nb - first, CHUNK);
       blk_base += nb;
+      e->st.blocks_rehashed += nb - first;
     }
   }
   e->dirty = true;
@@ -743,15 +759,15 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     r = status_zero(e, s);
     if (r) return r;
     HashArgs ha;
-    ha.tokens = e->d_tokens; ha.keys = e->d_keys; ha.ctx = e->dp<HashCtx>(e->L.desc); ha.n_ctx = nd;
-    ha.agg = e->dp<u64>(e->L.agg); ha.carry = e->dp<u64>(e->L.carry); ha.h0 = e->h0; ha.single = HashCtx{};
+    ha.tokens = e->d_tokens; ha.keys = e->d_keys; ha.carry_base = e->d_keys; ha.ctx = e->dp<HashCtx>(e->L.desc); ha.n_ctx = nd;
+    ha.agg = e->dp<u64>(e->L.agg); ha.h0 = e->h0; ha.single = HashCtx{};
     LookupArgs la;
     la.tab = e->tab; la.b_ent = e->dp<u32>(e->L.s0); la.hit_len = d_res; la.status = e->d_status;
     LockArgs lk;
     lk.ent = e->ent; lk.b_ent = la.b_ent; lk.hit_len = d_res; lk.n_hbm = d_res + C; lk.n_host = d_res + 2 * C;
     lk.now = e->now; lk.status = e->d_status;
     if (e->profiling) CU(cudaEventRecord(e->ev_h0, s));
-    KL(k_hash_digest, chunk_base, CHUNK, s, ha);
+    if (dchunk_base) KL(k_hash_digest, dchunk_base, CHUNK, s, ha);
     KL(k_hash_carry, nd, 1024, s, ha);
     KL(k_hash_finish_lookup, chunk_base, CHUNK, s, ha, la);
     KL(k_lock_hits, chunk_base, CHUNK, s, ha, lk);
@@ -1186,7 +1202,7 @@ int32_t kvt_copy_blocks(kvt_engine *e, uint32_t src_tier, const uint32_t *src, u
 // ---- stand-alone hasher -----------------------------------------------------------------------------------
 uint64_t kvt_hash_scratch_bytes(uint64_t n_tokens) {
   u64 n_chunks = (n_tokens / 16 + CHUNK - 1) / CHUNK;
-  return std::max<u64>(n_chunks, 1) * 16;
+  return (2 * std::max<u64>(n_chunks, 1) + 1) * 8;   // chunk aggregates, then chunk carries plus the final value
 }
 
 int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t hash_seed, uint64_t *d_keys, void *d_scratch,
@@ -1199,8 +1215,9 @@ int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t ha
   u32 n_chunks = cdiv(nb, CHUNK);
   HashArgs ha;
   ha.tokens = d_tokens; ha.keys = d_keys; ha.ctx = nullptr; ha.n_ctx = 1;
-  ha.single = HashCtx{0, 0, (u32)nb, 0, 0, 0};
-  ha.agg = (u64 *)d_scratch; ha.carry = (u64 *)d_scratch + n_chunks; ha.h0 = hash_h0(hash_seed);
+  ha.single = HashCtx{};
+  ha.single.n_blocks = (u32)nb;
+  ha.agg = (u64 *)d_scratch; ha.carry_base = (u64 *)d_scratch + n_chunks; ha.h0 = hash_h0(hash_seed);
   LookupArgs la{};
   k_hash_digest<<<n_chunks, CHUNK, 0, s>>>(ha);
   k_hash_carry<<<1, 1024, 0, s>>>(ha);
@@ -1213,7 +1230,7 @@ int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t ha
 // memory: in host code this name is only a handle, so its device address is queried once per device
 // below and that pointer is what the kernels get.
 constexpr u64 NOALLOC_MAX_CHUNKS = KVT_HASH_NOALLOC_MAX_TOKENS / 16 / CHUNK;
-static __device__ __align__(256) unsigned long long g_noalloc_scratch[2 * NOALLOC_MAX_CHUNKS];
+static __device__ __align__(256) unsigned long long g_noalloc_scratch[2 * NOALLOC_MAX_CHUNKS + 1];
 static u64 *g_noalloc_ptr[64] = {};   // per device ordinal
 
 int32_t kvt_hash_tokens_noalloc(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t hash_seed, uint64_t *d_keys,
@@ -1233,8 +1250,9 @@ int32_t kvt_hash_tokens_noalloc(const uint32_t *d_tokens, uint64_t n_tokens, uin
   u32 n_chunks = cdiv(nb, CHUNK);
   HashArgs ha;
   ha.tokens = d_tokens; ha.keys = d_keys; ha.ctx = nullptr; ha.n_ctx = 1;
-  ha.single = HashCtx{0, 0, (u32)nb, 0, 0, 0};
-  ha.agg = g_noalloc_ptr[dev]; ha.carry = g_noalloc_ptr[dev] + NOALLOC_MAX_CHUNKS; ha.h0 = hash_h0(hash_seed);
+  ha.single = HashCtx{};
+  ha.single.n_blocks = (u32)nb;
+  ha.agg = g_noalloc_ptr[dev]; ha.carry_base = g_noalloc_ptr[dev] + NOALLOC_MAX_CHUNKS; ha.h0 = hash_h0(hash_seed);
   LookupArgs la{};
   k_hash_digest<<<n_chunks, CHUNK, 0, s>>>(ha);
   k_hash_carry<<<1, 1024, 0, s>>>(ha);

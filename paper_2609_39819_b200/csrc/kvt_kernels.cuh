@@ -113,19 +113,41 @@ __device__ __forceinline__ u32 tab_find_or_claim(const Table &t, u64 key, u32 *s
 //   digest : per 256-block chunk, 4 lanes per block read 16 B each, weighted sums, mix, then a CTA-wide
 //            scan of the affine chain with zero carry-in -> partial chain values + chunk aggregate
 //   carry  : one CTA per context scans its chunk aggregates, 1024 chunks per step
+// Incremental: a sequence whose leading blocks are unchanged since its previous key list only digests from the
+// last chunk boundary before the first changed block (the chain restarts from the carry kept for that chunk).
 //   finish : h = P^(i+1) * carry + partial, key = mix64(h); fused with the table probe
 // ======================================================================================================
-struct HashCtx { u64 tok_off; u64 key_off; u32 n_blocks; u32 chunk_base; u32 blk_base; u32 pad; };
-
-struct HashArgs {
-  const u32 *tokens; u64 *keys; const HashCtx *ctx; HashCtx single; u32 n_ctx;
-  u64 *agg; u64 *carry; u64 h0;
+// One sequence of a batch. Blocks [0, first) keep the keys of the previous key list (first is a multiple of
+// CHUNK): only chunks from first / CHUNK on are digested, restarting the chain from the carry stored for that
+// chunk. The per-chunk carries of a sequence are kept next to its keys for exactly this purpose.
+struct HashCtx {
+  u64 tok_off;        // token buffer (u32 index into HashArgs.tokens)
+  u64 key_off;        // key list (u64 index into HashArgs.keys)
+  u64 carry_off;      // per-chunk carries (u64 index into HashArgs.carry_base)
+  u64 old_key_off;    // previous key list and carries, read when first > 0
+  u64 old_carry_off;
+  u32 n_blocks;
+  u32 first;
+  u32 chunk_base;     // first chunk of this sequence in the all-blocks grid (finish / lock kernels)
+  u32 dchunk_base;    // first chunk in the digest grid (chunks >= first / CHUNK only)
+  u32 blk_base;       // first block of this sequence in the batch-wide result arrays
+  u32 pad;
 };
 
-__device__ __forceinline__ const HashCtx &hash_ctx_of_chunk(const HashArgs &a, u32 chunk, u32 *ctx_idx) {
+struct HashArgs {
+  const u32 *tokens; u64 *keys; u64 *carry_base; const HashCtx *ctx; HashCtx single; u32 n_ctx;
+  u64 *agg; u64 h0;
+};
+
+// Sequence that owns chunk `chunk` of the all-blocks grid (dgrid = false) or of the digest grid (dgrid = true):
+// the last one whose base is <= chunk (sequences with no chunk of their own share a base with their successor).
+__device__ __forceinline__ const HashCtx &hash_ctx_of_chunk(const HashArgs &a, u32 chunk, u32 *ctx_idx, bool dgrid = false) {
   if (!a.ctx) { *ctx_idx = 0; return a.single; }
-  u32 lo = 0, hi = a.n_ctx;  // last i with chunk_base <= chunk
-  while (hi - lo > 1) { u32 mid = (lo + hi) >> 1; if (a.ctx[mid].chunk_base <= chunk) lo = mid; else hi = mid; }
+  u32 lo = 0, hi = a.n_ctx;
+  while (hi - lo > 1) {
+    u32 mid = (lo + hi) >> 1;
+    if ((dgrid ? a.ctx[mid].dchunk_base : a.ctx[mid].chunk_base) <= chunk) lo = mid; else hi = mid;
+  }
   *ctx_idx = lo;
   return a.ctx[lo];
 }
@@ -150,8 +172,8 @@ __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   __shared__ u64 wagg[CHUNK / 32];
   const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   u32 ci;
-  const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci);
-  const u32 b0 = (blockIdx.x - c.chunk_base) * CHUNK;
+  const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci, true);
+  const u32 b0 = c.first + (blockIdx.x - c.dchunk_base) * CHUNK;
   const u32 nb = min(CHUNK, c.n_blocks - b0);
   const uint4 *tok = reinterpret_cast<const uint4 *>(a.tokens + c.tok_off + (u64)b0 * 16);
   const u32 q = tid & 3;
@@ -198,24 +220,28 @@ __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   if (tid == nb - 1) a.agg[blockIdx.x] = cval;
 }
 
-// One CTA per context: the chain value entering chunk j is A^j * H0 + sum_{i<j} A^(j-1-i) * agg_i with
-// A = P^CHUNK (every chunk before the last is full), evaluated 1024 chunks at a time: a warp scan per 32 chunks,
-// a scan of the 32 warp totals, then the carry of the previous 1024.
+// One CTA per sequence: the chain value entering chunk g0 + j is A^j * C0 + sum_{i<j} A^(j-1-i) * agg_i with
+// A = P^CHUNK (every chunk before the last is full) and C0 the value entering chunk g0 = first / CHUNK (H0, or the
+// carry kept from the previous key list), evaluated 1024 chunks at a time: a warp scan per 32 chunks, a scan of
+// the 32 warp totals, then the carry of the previous 1024. Also copies the kept carries of chunks < g0.
 __global__ void __launch_bounds__(1024) k_hash_carry(HashArgs a) {
   __shared__ u64 wtot[32], wpre[32], sv[1024];
   const u32 i = blockIdx.x;
   if (i >= a.n_ctx) return;
   const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const HashCtx c = a.ctx ? a.ctx[i] : a.single;
-  const u32 n_chunks = (c.n_blocks + CHUNK - 1) / CHUNK;
+  const u32 g0 = c.first / CHUNK;
+  const u32 n_chunks = (c.n_blocks - c.first + CHUNK - 1) / CHUNK;   // chunks that were digested
+  for (u32 k = tid; k < g0; k += 1024) a.carry_base[c.carry_off + k] = a.carry_base[c.old_carry_off + k];
   const u64 A = g_pow_p.v[CHUNK];
   const u64 A32 = pow_u64(A, 32);
   const u64 a_lane = pow_u64(A, lane + 1);          // A^(lane+1)
   const u64 a_tid = pow_u64(A32, warp) * a_lane;    // A^(tid+1)
-  u64 carry = a.h0;
+  u64 carry = g0 ? a.carry_base[c.old_carry_off + g0] : a.h0;
+  if (n_chunks == 0 && tid == 0) a.carry_base[c.carry_off + g0] = carry;   // nothing new: keep the resume point
   for (u32 base = 0; base < n_chunks; base += 1024) {
     const u32 j = base + tid;
-    u64 x = j < n_chunks ? a.agg[c.chunk_base + j] : 0;
+    u64 x = j < n_chunks ? a.agg[c.dchunk_base + j] : 0;
     u64 pp = A;
 #pragma unroll
     for (u32 o = 1; o < 32; o <<= 1) {
@@ -237,9 +263,11 @@ __global__ void __launch_bounds__(1024) k_hash_carry(HashArgs a) {
       wpre[lane] = lane ? e : 0;
     }
     __syncthreads();
-    sv[tid] = a_tid * carry + a_lane * wpre[warp] + x;   // chain value after chunk j
+    sv[tid] = a_tid * carry + a_lane * wpre[warp] + x;   // chain value after chunk g0 + j
     __syncthreads();
-    if (j < n_chunks) a.carry[c.chunk_base + j] = tid ? sv[tid - 1] : carry;
+    if (j < n_chunks) a.carry_base[c.carry_off + g0 + j] = tid ? sv[tid - 1] : carry;
+    // value after the last chunk: the resume point of a later call if that chunk is full
+    if (j == n_chunks - 1) a.carry_base[c.carry_off + g0 + n_chunks] = sv[tid];
     carry = sv[1023];
     __syncthreads();
   }
@@ -262,9 +290,14 @@ __global__ void __launch_bounds__(CHUNK) k_hash_finish_lookup(HashArgs a, Lookup
   if (tid == 0) s_min = 0xFFFFFFFFu;
   __syncthreads();
   if (tid < nb) {
-    u64 h = g_pow_p.v[tid + 1] * a.carry[blockIdx.x] + a.keys[c.key_off + b0 + tid];
-    u64 key = mix64(h);
-    if (key < 2) key += 2;
+    u64 key;
+    if (b0 < c.first) {          // unchanged prefix: the key of the previous list still holds
+      key = a.keys[c.old_key_off + b0 + tid];
+    } else {
+      u64 h = g_pow_p.v[tid + 1] * a.carry_base[c.carry_off + (blockIdx.x - c.chunk_base)] + a.keys[c.key_off + b0 + tid];
+      key = mix64(h);
+      if (key < 2) key += 2;
+    }
     a.keys[c.key_off + b0 + tid] = key;
     if (l.tab.slots) {
       u32 s = tab_find(l.tab, key, l.status);

@@ -22,7 +22,7 @@ TIER_HBM, TIER_HOST, TIER_NONE = 0, 1, 0xFF
 MAP_LOOKUP, MAP_ADMIT = 0, 1
 GiB = 1 << 30
 GPU_ONLY_STATS = ("table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns", "mover_bytes",
-                  "lookup_ns", "lookup_blocks", "select_ns", "select_slots")
+                  "lookup_ns", "lookup_blocks", "select_ns", "select_slots", "blocks_rehashed")
 STATE_COPY, STATE_HAS_COPY = 0xFE, 0x80
 
 

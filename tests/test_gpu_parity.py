@@ -413,3 +413,45 @@ def test_capacity_errors_leave_the_engine_usable(B):
     assert (st["occ_hbm"], st["occ_host"]) == (12, 4)
     with pytest.raises(B.KvtError):
         eng.select_victims(2, 1)                                 # bad tier
+
+
+def test_incremental_hashing_resumes_at_chunk_boundaries(B, oracle):
+    """Appends, edits, forks and repeated calls around multiples of 256 blocks: only the changed tail is digested
+    again, and every key still equals the one-shot hash of the whole sequence."""
+    kw = dict(n_hbm_blocks=4096, n_host_blocks=0, max_contexts=8, metadata_only=True, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 18, max_messages=1024, **kw)
+    rng = np.random.default_rng(30)
+    msgs = []
+
+    def check(ctx):
+        before = gpu.get_stats()["blocks_rehashed"]
+        gpu.map_blocks([ctx], 0); gpu.map_blocks([ctx], 1); gpu.prefill_done(ctx)
+        return gpu.get_stats()["blocks_rehashed"] - before
+
+    gpu.spawn(0)
+    # (tokens appended, blocks digested by the next call): 256 | 512 (resume at 256) | 512 (+7 tokens: nothing new)
+    # | 813 (resume at 512) | 1024 (resume at 768)
+    for n_tok, want in ((16 * 256, 256), (16 * 256, 256), (7, 0), (16 * 300 + 9, 301), (16 * 211, 256)):
+        t = rng.integers(0, W.VOCAB, n_tok, dtype=np.uint32)
+        msgs.append(t)
+        gpu.append(0, t)
+        assert check(0) == want
+        assert np.array_equal(gpu.get_block_map(0)[0], oracle.hash_tokens(np.concatenate(msgs)))
+    assert check(0) == 0                   # a call with no change digests nothing (1024 blocks, all kept)
+    # an edit in the middle: everything from the chunk holding the edited message's first block is redone
+    msgs[3] = rng.integers(0, W.VOCAB, 100, dtype=np.uint32)
+    gpu.replace(0, 3, 4, msgs[3])
+    got = check(0)
+    keys = gpu.get_block_map(0)[0]
+    assert np.array_equal(keys, oracle.hash_tokens(np.concatenate(msgs)))
+    assert got == len(keys) - 512          # message 3 starts at token 8199 -> block 512
+    # a fork resumes from its parent's list
+    gpu.fork(0, 1, 3)
+    extra = rng.integers(0, W.VOCAB, 16 * 40, dtype=np.uint32)
+    gpu.append(1, extra)
+    got = check(1)
+    keys = gpu.get_block_map(1)[0]
+    assert np.array_equal(keys, oracle.hash_tokens(np.concatenate(msgs[:3] + [extra])))
+    assert got == len(keys) - 512
+    st = gpu.get_stats()
+    assert st["blocks_rehashed"] < st["blocks_hashed"]
