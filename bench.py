@@ -189,7 +189,9 @@ def mem_available_bytes():
 
 
 class ClockSampler:
-    FIELDS = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+    """nvidia-smi polled every 50 ms in the background; stop(t0, t1) keeps the samples taken inside the timed
+    window [t0, t1] (host wall clock), or all samples of the run if the window saw fewer than two."""
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
@@ -197,14 +199,16 @@ class ClockSampler:
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                                       "-i", str(gpu_index), "-lms", "200"], stdout=self.f, stderr=subprocess.DEVNULL)
+                                       "-i", str(gpu_index), "-lms", "50"], stdout=self.f, stderr=subprocess.DEVNULL)
         except OSError:
             self.p = None
 
-    def stop(self):
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+    def stop(self, t0=None, t1=None):
+        import datetime
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": "none"}
         if self.p is None:
             return out
+        time.sleep(0.06)
         self.p.terminate()
         try:
             self.p.wait(timeout=5)
@@ -212,23 +216,25 @@ class ClockSampler:
             self.p.kill()
         self.f.flush()
         self.f.seek(0)
-        sm, mx, reasons = [], [], set()
         names = ("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap")
+        rows = []
         for ln in self.f:
             parts = [x.strip() for x in ln.split(",")]
             if len(parts) < 9:
                 continue
             try:
-                sm.append(float(parts[1])); mx.append(float(parts[2]))
+                ts = datetime.datetime.strptime(parts[0], "%Y/%m/%d %H:%M:%S.%f").timestamp()
+                rows.append((ts, float(parts[1]), float(parts[2]),
+                             [nm for nm, v in zip(names, parts[5:9]) if v.lower().startswith("active")]))
             except ValueError:
                 continue
-            for nm, v in zip(names, parts[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(nm)
         self.f.close()
         os.unlink(self.f.name)
-        if sm:
-            out.update(sm_mhz=float(np.median(sm)), sm_max_mhz=float(max(mx)), reasons=sorted(reasons), samples=len(sm))
+        inside = [r for r in rows if t0 is not None and t0 - 0.05 <= r[0] <= t1 + 0.05]
+        use, out["window"] = (inside, "timed region") if len(inside) >= 2 else (rows, "whole arm (timed region shorter than the sampling period)")
+        if use:
+            out.update(sm_mhz=float(np.median([r[1] for r in use])), sm_max_mhz=float(max(r[2] for r in use)),
+                       reasons=sorted({x for r in use for x in r[3]}), samples=len(use))
         return out
 
 
@@ -318,6 +324,7 @@ def gpu_arm(args, torch, B, setup, turns, n_ff, e2e, n_host_blocks, n_hbm_blocks
     s0 = eng.get_stats()
     timer.reset()
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    wall0 = time.time()
     ev0.record()
     torch.cuda.nvtx.range_push("kvt_timed")      # lets a profiler restrict its launch list to the timed steps
     for t in range(n_ff + W_, n_ff + W_ + K):
@@ -325,6 +332,7 @@ def gpu_arm(args, torch, B, setup, turns, n_ff, e2e, n_host_blocks, n_hbm_blocks
     torch.cuda.nvtx.range_pop()
     ev1.record()
     torch.cuda.synchronize()
+    wall1 = time.time()
     if barrier:
         barrier()
     ms = ev0.elapsed_time(ev1)
@@ -345,7 +353,7 @@ def gpu_arm(args, torch, B, setup, turns, n_ff, e2e, n_host_blocks, n_hbm_blocks
     tok_bytes = sum(4 * len(ev[2] if ev[0] == "append" else ev[4]) for pre, _c, _p in used[n_ff + W_:] for ev in pre
                     if ev[0] in ("append", "replace"))
     res = dict(ms=ms, stats=d, stage_ms=dict(timer.ms), stage_calls=dict(timer.calls), timers=timers,
-               verified=(n_ok, n_seen), tok_bytes=tok_bytes, block_bytes=eng.block_bytes)
+               verified=(n_ok, n_seen), tok_bytes=tok_bytes, block_bytes=eng.block_bytes, wall=(wall0, wall1))
     eng.close()
     del eng, pool, cache, base, timer
     import gc
@@ -532,7 +540,7 @@ def main():
     fit2 = int((free_b - n_hbm_blocks * W.GEO_8B.block_bytes - 6 * GiB) // W.GEO_8B.block_bytes)
     tier2_dev_blocks = max(min(want2, fit2), 9000)
     v = gpu_arm(args, torch, B, setup, turns, n_ff, False, tier2_dev_blocks, n_hbm_blocks, rank, world, barrier)
-    clocks = sampler.stop()
+    clocks = sampler.stop(*v["wall"])
 
     # ---- e2e arm: pinned host tier, tokens from pinned host buffers ---------------------------------------
     e = None
@@ -540,7 +548,9 @@ def main():
     if not args.skip_e2e:
         budget = min(int(args.host_gib * GiB), int(mem_available_bytes() * 0.5) // max(world, 1))
         host_blocks = max(budget // W.GEO_8B.block_bytes, 9000)
+        sampler = ClockSampler(local_rank)
         e = gpu_arm(args, torch, B, setup, turns, n_ff, True, host_blocks, n_hbm_blocks, rank, world, barrier)
+        clocks_e2e = sampler.stop(*e["wall"])
 
     vbytes = kv_bytes(v["stats"], v["block_bytes"])
     dist = None
@@ -588,6 +598,7 @@ def main():
     if e:
         es = e["stats"]
         e_mover_s = es["mover_ns"] / 1e9
+        line["clocks_e2e"] = clocks_e2e
         line["e2e"] = {
             "value": e_bytes / (e_ms / 1e3) / 1e9, "unit": "GB/s", "ms_per_step": e_ms / K,
             "h2d_bytes_per_step": (es["bytes_h2d"] + e["tok_bytes"]) / K,
