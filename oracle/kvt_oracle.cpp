@@ -644,6 +644,10 @@ int32_t kvto_offload(Engine *e, const uint32_t *slots, uint32_t n, uint32_t *n_d
   std::vector<uint8_t> rank[2];
   classify(*e, rank);
   const bool knows_dead = !(e->cfg.policy_flags & POLICY_NO_LIFECYCLE);
+  // destination slots: the host slots that are free when the call begins, lowest first (slots freed by this
+  // call's own drops are not reused within it)
+  std::vector<uint32_t> dests(e->free_slots[TIER_HOST].begin(), e->free_slots[TIER_HOST].end());
+  size_t next_dest = 0;
   for (uint32_t i = 0; i < n; ++i) {
     uint32_t s = slots[i];
     if (knows_dead && rank[0][s] == 0) {  // reclaim dead KV without a copy
@@ -660,8 +664,8 @@ int32_t kvto_offload(Engine *e, const uint32_t *slots, uint32_t n, uint32_t *n_d
       e->st.offloaded++;
       e->st.offloaded_clean++;
     } else {
-      if (e->free_slots[TIER_HOST].empty()) return E_NOSPACE;
-      uint32_t d = *e->free_slots[TIER_HOST].begin();
+      if (next_dest == dests.size()) return E_NOSPACE;
+      uint32_t d = dests[next_dest++];
       move_entry(e, TIER_HBM, s, TIER_HOST, d);
       e->st.offloaded++;
       e->st.bytes_d2h += e->block_bytes;

@@ -1,0 +1,24 @@
+"""Random differential test: the same random stream of API calls (valid and invalid, every policy switch) goes to
+the CUDA engine and to the CPU oracle; every status code, every returned list and, every few calls, all metadata,
+states, statistics and payload bytes must be identical."""
+import pytest
+
+import fuzz_driver as F
+from paper_2609_39819_b200 import workloads as W
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("seed", range(24))
+@pytest.mark.parametrize("flags", [0, 1, 2, 3])
+@pytest.mark.parametrize("pools", [(24, 16), (8, 4), (40, 0)], ids=lambda p: f"hbm{p[0]}-host{p[1]}")
+def test_random_api_streams_match_the_oracle(oracle, seed, flags, pools):
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_39819_b200 import binding as B
+    kw = dict(n_hbm_blocks=pools[0], n_host_blocks=pools[1], max_contexts=6, policy_flags=flags, suspended_order=seed % 2,
+              pool_layout=seed % 2, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 16, max_messages=2048, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    F.run([gpu, cpu], seed, steps=300, inclusive=bool(flags & 2), check_every=10)
