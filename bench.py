@@ -546,11 +546,13 @@ def main():
     e = None
     host_blocks = 0
     if not args.skip_e2e:
+        # pinned host tier: the configured size, but never more than this rank's share of half the free host RAM
         budget = min(int(args.host_gib * GiB), int(mem_available_bytes() * 0.5) // max(world, 1))
-        host_blocks = max(budget // W.GEO_8B.block_bytes, 9000)
-        sampler = ClockSampler(local_rank)
-        e = gpu_arm(args, torch, B, setup, turns, n_ff, True, host_blocks, n_hbm_blocks, rank, world, barrier)
-        clocks_e2e = sampler.stop(*e["wall"])
+        host_blocks = budget // W.GEO_8B.block_bytes
+        if host_blocks >= 5000:      # the session keeps up to ~4.5 K blocks in the host tier
+            sampler = ClockSampler(local_rank)
+            e = gpu_arm(args, torch, B, setup, turns, n_ff, True, host_blocks, n_hbm_blocks, rank, world, barrier)
+            clocks_e2e = sampler.stop(*e["wall"])
 
     vbytes = kv_bytes(v["stats"], v["block_bytes"])
     dist = None

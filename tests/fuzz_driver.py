@@ -60,16 +60,18 @@ def check_invariants(eng, inclusive):
 
 
 class Fuzzer:
-    def __init__(self, engines, seed, max_ctx=6):
+    def __init__(self, engines, seed, max_ctx=6, max_tok=90):
         self.engs = engines
         self.rng = np.random.default_rng([77, seed])
         self.max_ctx = max_ctx
+        self.max_tok = max_tok
         self.n_msgs = {}            # mirror: live contexts -> message count (retained contexts excluded)
         self.in_flight = set()
         self.log = []
 
-    def toks(self, lo=1, hi=90):
-        return self.rng.integers(0, 50, int(self.rng.integers(lo, hi + 1)), dtype=np.uint32)  # tiny vocabulary: shared blocks
+    def toks(self, lo=1):
+        n = int(self.rng.integers(lo, self.max_tok + 1))
+        return self.rng.integers(0, 50, n, dtype=np.uint32)  # tiny vocabulary: blocks shared across contexts do occur
 
     def all_rc(self, fn):
         """Calls fn(engine) on every engine; the results must be equal; returns the first."""
@@ -228,8 +230,8 @@ class Fuzzer:
                         e.write_block(HBM, int(slot[b]), payload(keys[b], e.block_bytes))
 
 
-def run(engines, seed, steps=250, inclusive=False, check_every=10, invariants=True):
-    f = Fuzzer(engines, seed)
+def run(engines, seed, steps=250, inclusive=False, check_every=10, invariants=True, max_tok=90):
+    f = Fuzzer(engines, seed, max_tok=max_tok)
     for i in range(steps):
         f.step()
         if (i + 1) % check_every == 0 or i == steps - 1:

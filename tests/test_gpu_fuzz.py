@@ -22,3 +22,21 @@ def test_random_api_streams_match_the_oracle(oracle, seed, flags, pools):
     gpu = B.Engine(max_tokens=1 << 16, max_messages=2048, **kw)
     cpu = oracle.OracleEngine(**kw)
     F.run([gpu, cpu], seed, steps=300, inclusive=bool(flags & 2), check_every=10)
+
+
+@pytest.mark.parametrize("seed", range(6))
+@pytest.mark.parametrize("flags", [0, 2])
+def test_random_api_streams_with_long_messages(oracle, seed, flags):
+    """Messages of up to 6,000 tokens: contexts span several 256-block hash chunks, so edits, forks and repeated
+    calls exercise the incremental hasher's resume points inside the random stream."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_39819_b200 import binding as B
+    kw = dict(n_hbm_blocks=1500, n_host_blocks=600, max_contexts=6, policy_flags=flags, metadata_only=True,
+              **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 20, max_messages=4096, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    F.run([gpu, cpu], seed, steps=200, inclusive=bool(flags & 2), check_every=10, invariants=False, max_tok=6000)
+    st = gpu.get_stats()
+    assert st["blocks_rehashed"] < st["blocks_hashed"]
