@@ -549,6 +549,11 @@ def main():
         # pinned host tier: the configured size, but never more than this rank's share of half the free host RAM
         budget = min(int(args.host_gib * GiB), int(mem_available_bytes() * 0.5) // max(world, 1))
         host_blocks = budget // W.GEO_8B.block_bytes
+        if world > 1:                # every rank must take the same decision below
+            import torch.distributed as dist
+            hb = torch.tensor([host_blocks], dtype=torch.int64, device="cuda")
+            dist.all_reduce(hb, op=dist.ReduceOp.MIN)
+            host_blocks = int(hb.item())
         if host_blocks >= 5000:      # the session keeps up to ~4.5 K blocks in the host tier
             sampler = ClockSampler(local_rank)
             e = gpu_arm(args, torch, B, setup, turns, n_ff, True, host_blocks, n_hbm_blocks, rank, world, barrier)
