@@ -345,7 +345,8 @@ int32_t kvt_set_profiling(kvt_engine *e, uint32_t on);
 
 /* Tuning hook: which mover kernel offload / reload / compact / copy_blocks launch. 0 = automatic (variant 2
  * whenever it applies, default), 1 = one CTA per (block, chunk), 2 = one warp per 4 KiB tile (needs chunk_bytes % 4096 == 0,
- * otherwise variant 1 is used). Results are identical. */
+ * otherwise variant 1 is used), 3 = TMA bulk copies through a shared-memory ring (chunks of at most 16 KiB or a
+ * multiple of 16 KiB). Results are identical. */
 int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant);
 
 /* Text of the last error of this engine (always NUL-terminated). */

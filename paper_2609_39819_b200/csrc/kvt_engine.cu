@@ -142,7 +142,8 @@ struct kvt_engine {
   bool upload_pending = false;
   // optional timing of the mover kernel (kvt_set_profiling)
   bool profiling = false, mover_timed = false;
-  u32 mover_variant = 0;   // 0 auto, 1 CTA per chunk, 2 warp per 4 KiB tile
+  u32 mover_variant = 0;   // 0 auto, 1 CTA per chunk, 2 warp per 4 KiB tile, 3 TMA ring
+  bool tma_attr_set = false;
   cudaEvent_t ev_m0 = nullptr, ev_m1 = nullptr, ev_h0 = nullptr, ev_h1 = nullptr;
 
   template <class T> T *dp(u64 off) const { return reinterpret_cast<T *>(meta + off); }
@@ -285,7 +286,21 @@ int32_t launch_mover(kvt_engine *e, cudaStream_t s, u32 st, const u32 *src, u32 
   // 4 KiB and 32 KiB chunks alike); chunks that are not a multiple of 4 KiB take the CTA-per-chunk kernel
   const bool tiles_ok = e->chunk_bytes % 4096 == 0;
   const bool use_tiles = e->mover_variant != 1;
-  if (use_tiles && tiles_ok) {
+  if (e->mover_variant == 3 && e->chunk_bytes % 16 == 0) {   // TMA ring (experimental variant)
+    u32 tile = (u32)(e->chunk_bytes <= 16384 ? e->chunk_bytes : (e->chunk_bytes % 16384 == 0 ? 16384 : 0));
+    if (tile == 0 || tile > 49152) return fail(e, KVT_E_INVAL, "chunk size not supported by the TMA mover");
+    u32 tpc = (u32)(e->chunk_bytes / tile);
+    u64 titems = items * tpc;
+    size_t smem = (size_t)TMA_STAGES * tile;
+    if (!e->tma_attr_set) {
+      CU(cudaFuncSetAttribute(k_move_tma, cudaFuncAttributeMaxDynamicSharedMemorySize, 196608));
+      e->tma_attr_set = true;
+    }
+    u32 per_sm = (u32)std::max<size_t>(1, std::min<size_t>(8, (200 * 1024) / (smem + 1024)));
+    u32 tgrid = (u32)std::min<u64>(titems, (u64)e->sm_count * per_sm);
+    k_move_tma<<<tgrid, 32, smem, s>>>(a, tile, tpc);
+    e->st.kernel_launches++;
+  } else if (use_tiles && tiles_ok) {
     u32 tpc = (u32)(e->chunk_bytes / 4096);
     u64 titems = items * tpc;
     u32 tgrid = (u32)std::min<u64>((titems + 7) / 8, (u64)e->sm_count * 8);
@@ -517,7 +532,7 @@ int32_t kvt_set_profiling(kvt_engine *e, uint32_t on) {
 }
 
 int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant) {
-  if (!e || variant > 2) return KVT_E_INVAL;
+  if (!e || variant > 3) return KVT_E_INVAL;
   e->mover_variant = variant;
   return KVT_OK;
 }

@@ -1016,4 +1016,94 @@ __global__ void __launch_bounds__(256) k_move_tiles(MoveArgs a, u32 tiles_per_ch
   }
 }
 
+// ------------------------------------------------------------------------------------------------------
+// TMA variant: one elected thread per CTA drives a ring of shared-memory stages with untiled bulk copies
+// (cp.async.bulk global -> shared, completion on an mbarrier; shared -> global as a bulk group). No registers
+// carry payload; every wait is bounded and reports through the status word. No multicast, no clusters.
+// ------------------------------------------------------------------------------------------------------
+constexpr int TMA_STAGES = 4;
+constexpr u32 TMA_WAIT_LIMIT = 1u << 20;
+
+__device__ __forceinline__ u32 smem_u32(const void *p) { return (u32)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(u64 *bar, u32 count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(u64 *bar, u32 bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Polls the barrier's phase; gives up after TMA_WAIT_LIMIT polls (returns false).
+__device__ __forceinline__ bool mbar_wait(u64 *bar, u32 parity) {
+  u32 done = 0;
+  for (u32 n = 0; n < TMA_WAIT_LIMIT && !done; ++n) {
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  }
+  return done != 0;
+}
+__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, u32 bytes, u64 *bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void *gdst, const void *smem_src, u32 bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(smem_src)), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(32) k_move_tma(MoveArgs a, u32 tile_bytes, u32 tiles_per_chunk) {
+  extern __shared__ __align__(128) u8 smem[];
+  __shared__ __align__(8) u64 bars[TMA_STAGES];
+  if (threadIdx.x != 0) return;            // one thread issues everything; the copies run in the async proxy
+  u32 n_pairs = a.n_pairs;
+  if (a.n_pairs_dev) n_pairs = min(n_pairs, *a.n_pairs_dev);
+  const u64 per_pair = (u64)a.n_chunks * tiles_per_chunk;
+  const u64 n_items = (u64)n_pairs * per_pair;
+  if (blockIdx.x >= n_items) return;
+  const u64 n_mine = (n_items - blockIdx.x + gridDim.x - 1) / gridDim.x;   // my tiles: blockIdx + k * gridDim
+  for (int s = 0; s < TMA_STAGES; ++s) mbar_init(&bars[s], 1);
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+
+  auto locate = [&](u64 k, const u8 *&src, u8 *&dst) -> bool {
+    u64 item = blockIdx.x + k * gridDim.x;
+    u32 pair = (u32)(item / per_pair);
+    u32 rem = (u32)(item - (u64)pair * per_pair);
+    u32 chunk = rem / tiles_per_chunk, tile = rem - chunk * tiles_per_chunk;
+    u32 sid = a.src_ids[pair], did = a.dst_ids[pair];
+    if (sid >= a.src.n_slots || did >= a.dst.n_slots) { set_err(a.status, DERR_RANGE); return false; }
+    src = a.src.base + sid * a.src.slot_stride + chunk * a.src.chunk_stride + (u64)tile * tile_bytes;
+    dst = a.dst.base + did * a.dst.slot_stride + chunk * a.dst.chunk_stride + (u64)tile * tile_bytes;
+    return true;
+  };
+  auto issue_load = [&](u64 k) {
+    const u8 *src; u8 *dst;
+    int s = (int)(k % TMA_STAGES);
+    if (locate(k, src, dst)) {
+      mbar_expect_tx(&bars[s], tile_bytes);
+      bulk_load(smem + (size_t)s * tile_bytes, src, tile_bytes, &bars[s]);
+    } else {
+      mbar_expect_tx(&bars[s], 0);          // keep the phase sequence going for a skipped tile
+    }
+  };
+
+  const u64 prologue = n_mine < TMA_STAGES ? n_mine : TMA_STAGES;
+  for (u64 k = 0; k < prologue; ++k) issue_load(k);
+  bool ok = true;
+  for (u64 k = 0; k < n_mine && ok; ++k) {
+    int s = (int)(k % TMA_STAGES);
+    ok = mbar_wait(&bars[s], (u32)((k / TMA_STAGES) & 1));
+    if (!ok) break;
+    const u8 *src; u8 *dst;
+    if (locate(k, src, dst)) bulk_store(dst, smem + (size_t)s * tile_bytes, tile_bytes);
+    else asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+    // the stage of tile k-1 may be refilled once its store has finished reading shared memory
+    if (k >= 1 && k - 1 + TMA_STAGES < n_mine) {
+      asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");
+      issue_load(k - 1 + TMA_STAGES);
+    }
+  }
+  if (!ok) set_err(a.status, DERR_PROBE);
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // all my stores are complete before the CTA ends
+}
+
 }  // namespace kvt

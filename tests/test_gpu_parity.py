@@ -289,11 +289,13 @@ def test_c5_longest_id_list(B, oracle):
 
 @pytest.mark.parametrize("geo", [W.GEO_TOY, W.GEO_128K, W.GEO_8B, W.GEO_GLM], ids=lambda g: g.name)
 @pytest.mark.parametrize("layout", [0, 1])
-def test_c5_mover_parity(B, oracle, geo, layout):
+@pytest.mark.parametrize("variant", [1, 2, 3], ids=["cta-per-chunk", "warp-tiles", "tma-ring"])
+def test_c5_mover_parity(B, oracle, geo, layout, variant):
     import torch
     n_slots = (12 if geo.block_bytes > (4 << 20) else 24) if geo.block_bytes > (1 << 20) else 200
     kw = dict(n_hbm_blocks=n_slots, n_host_blocks=n_slots, max_contexts=2, pool_layout=layout, **geo.kwargs())
     gpu = B.Engine(max_tokens=1 << 12, max_messages=64, max_batch_blocks=4096, **kw)
+    gpu.set_mover_variant(variant)
     cpu = oracle.OracleEngine(**kw)
     rng = np.random.default_rng(5)
     fill = rng.integers(0, 256, gpu.hbm_pool.numel(), dtype=np.uint8)
