@@ -70,8 +70,12 @@ def load_library():
     global _lib
     if _lib is None:
         if not os.path.exists(LIB_PATH):
-            raise RuntimeError(f"{LIB_PATH} is missing: run `python -m paper_2609_39819_b200.build` "
-                               "(there is no CPU fallback)")
+            try:                                   # a build step, not a fallback: compile the CUDA library in-tree
+                from . import build
+                build.build_lib()
+            except Exception as exc:
+                raise RuntimeError(f"{LIB_PATH} is missing and could not be built with nvcc ({exc}); "
+                                   "there is no CPU fallback") from exc
         lib = C.CDLL(LIB_PATH)
         vp, u32, u64, i32 = C.c_void_p, C.c_uint32, C.c_uint64, C.c_int32
         sig = {
