@@ -238,6 +238,25 @@ class ClockSampler:
         return out
 
 
+def host_info():
+    model = "unknown"
+    try:
+        for ln in open("/proc/cpuinfo"):
+            if ln.lower().startswith("model name"):
+                model = ln.split(":", 1)[1].strip()
+                break
+    except OSError:
+        pass
+    mem = 0
+    try:
+        for ln in open("/proc/meminfo"):
+            if ln.startswith("MemTotal"):
+                mem = int(ln.split()[1]) // (1 << 20)
+    except OSError:
+        pass
+    return {"model": model, "cores": os.cpu_count(), "mem_total_gib": mem}
+
+
 def measured_peaks():
     p = os.path.join(ROOT, "MEASURED_PEAKS.json")
     if os.path.exists(p):
@@ -453,14 +472,16 @@ def cpu_arm(args, setup, turns, n_ff, n_steps, n_warm, n_hbm_blocks, n_host_bloc
     pressure_evict(eng, CPU_PRESSURE_CAP)
     for t in range(n_ff, n_ff + n_warm):
         run_step(eng, turns[t], ident, opt, cap=CPU_PRESSURE_CAP)
+    timer = StageTimer(eng)
     s0 = eng.get_stats()
+    timer.reset()
     t0 = time.perf_counter()
     for t in range(n_ff + n_warm, n_ff + n_warm + n_steps):
         run_step(eng, turns[t], ident, opt, cap=CPU_PRESSURE_CAP)
     sec = time.perf_counter() - t0
     s1 = eng.get_stats()
     d = {k: s1[k] - s0[k] for k in s1}
-    return dict(sec=sec, stats=d, block_bytes=eng.block_bytes)
+    return dict(sec=sec, stats=d, block_bytes=eng.block_bytes, stage_ms=dict(timer.ms))
 
 
 def reduce_over_ranks(local, dist=None, device="cpu"):
@@ -507,7 +528,8 @@ def main():
             "vs_baseline": None, "dtype": "u8", "data": "synthetic",
             "config": {"workload": workload, "host_tier_blocks": n_host_blocks},
             "blocks_hashed_looked_up_per_s": r["stats"]["blocks_hashed"] / r["sec"],
-            "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle",
+            "cpu_baseline": {"value": gbs, "unit": "GB/s", "cores": 1, "kind": "oracle", "host": host_info(),
+                             "stage_wall_ms_per_step": {k: round(x / K, 3) for k, x in r["stage_ms"].items()},
                              "sample": f"the same {K} calls with the tier pressure capped at {CPU_PRESSURE_CAP} blocks "
                                        f"(1 GiB each way) per step; whole path incl. payload memcpy; one thread"},
             "e2e": {"value": gbs, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
@@ -600,7 +622,7 @@ def main():
         "roofline": roofline,
         "stage_wall_ms_per_step": {k: round(x / K, 4) for k, x in v["stage_ms"].items()},
         "verified_blocks": {"value_arm": v["verified"], "e2e_arm": e["verified"] if e else None},
-        "host_cpu": {"cores": os.cpu_count()},
+        "host_cpu": host_info(),
     }
     if e:
         es = e["stats"]
@@ -645,6 +667,8 @@ def main():
                       f"capped at {CPU_PRESSURE_CAP} blocks (1 GiB each way) per step; whole path incl. payload "
                       f"memcpy; {c['sec']:.1f} s on one thread",
             "blocks_hashed_looked_up_per_s": c["stats"]["blocks_hashed"] / c["sec"],
+            "stage_wall_ms_per_step": {k: round(x / min(args.cpu_steps, K), 3) for k, x in c["stage_ms"].items()},
+            "host": host_info(),
         }
     print(json.dumps(line))
 
