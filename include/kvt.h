@@ -248,27 +248,34 @@ int32_t kvt_get_states(kvt_engine *e, uint32_t tier, uint8_t *state, uint32_t ca
  * KVT_SEL_INCLUDE_PINNED). Order: rank ascending (dead, idle, active, pinned); within dead, active and
  * pinned oldest stamp first; within idle newest stamp first (MRU) or
  * oldest first if suspended_order = KVT_ORDER_LRU; then chain depth descending; then slot
- * ascending. Classifies first if needed. Host output arrays (states_out may be NULL).
- * KVT_E_BUFSZ if cap < min(n_req, #candidates). Synchronises. */
+ * ascending. With inclusive tiers the host tier's clean copies (KVT_STATE_COPY) come before everything
+ * else, oldest first. states_out[i] is the rank, with KVT_STATE_HAS_COPY or-ed in for an HBM victim that
+ * still has a clean host copy (offloading it moves no bytes and needs no host slot), or KVT_STATE_COPY.
+ * With KVT_POLICY_NO_LIFECYCLE every candidate counts as rank 1. Classifies first if needed. Host output
+ * arrays (states_out may be NULL). KVT_E_BUFSZ if cap < min(n_req, #candidates). Synchronises. */
 int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_t flags, uint32_t *slots_out,
                            uint8_t *states_out, uint32_t cap, uint32_t *n_out, void *stream);
 
 /* ---- stage 5: tier movement (Section 7; Algorithm 1 "release") -------------------------------- */
 /* Processes HBM slots in the given order: a dead block is dropped (key erased, slot freed, no
- * copy); the i-th live block moves to the i-th lowest free host slot, payload byte for byte,
- * metadata carried. Stops with KVT_E_NOSPACE when the host tier is full; *n_done = victims
- * processed, *n_dropped = dead ones among them. A listed slot that is empty, out of range,
+ * copy; its clean host copy, if any, is freed too); a live block that has a clean host copy is handed
+ * over to it (metadata only); the i-th other live block moves to the i-th lowest host slot that was
+ * free when the call began, payload byte for byte, metadata carried. Stops with KVT_E_NOSPACE at the
+ * first block that finds no host slot; *n_done = victims processed, *n_dropped = dead ones among them. A listed slot that is empty, out of range,
  * repeated (KVT_E_INVAL / KVT_E_RANGE) or in flight (KVT_E_STATE) rejects the whole call.
  * Host id array. Synchronises. */
 int32_t kvt_offload(kvt_engine *e, const uint32_t *hbm_slots, uint32_t n, uint32_t *n_done,
                     uint32_t *n_dropped, void *stream);
 
 /* Mirror image: the i-th listed host slot moves to the i-th lowest free HBM slot (in-flight
- * blocks allowed: a call reloads its own host hits). KVT_E_NOSPACE + *n_done when HBM is full. */
+ * blocks allowed: a call reloads its own host hits). With inclusive tiers the host slot stays occupied
+ * as the block's clean copy. A listed slot that only holds such a copy is rejected (KVT_E_INVAL).
+ * KVT_E_NOSPACE + *n_done when HBM is full. Synchronises. */
 int32_t kvt_reload(kvt_engine *e, const uint32_t *host_slots, uint32_t n, uint32_t *n_done,
                    void *stream);
 
-/* Drops blocks without copying (frees host space for offloads). Same validation as kvt_offload. */
+/* Drops blocks without copying (frees host space for offloads). Same validation as kvt_offload.
+ * Releasing an HBM block frees its clean host copy too; releasing a clean copy leaves its block alone. */
 int32_t kvt_release(kvt_engine *e, uint32_t tier, const uint32_t *slots, uint32_t n, void *stream);
 
 /* Hole-filling compaction inside a tier: with n_occ occupied slots, the i-th occupied slot
