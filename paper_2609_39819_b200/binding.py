@@ -381,6 +381,23 @@ class Engine:
         pool = self.hbm_pool if tier == TIER_HBM else self.host_pool
         return pool.view(-1, self.n_chunks, self.chunk_bytes)[slot]
 
+    # Device-side counterpart of workloads.payload_pattern for large blocks (harness helpers, torch ops only).
+    def _pattern(self, key):
+        torch = self.torch
+        if getattr(self, "_pat_base", None) is None:
+            self._pat_base = (torch.arange(self.block_bytes // 4, dtype=torch.int64, device=self.device) * 0x9E3779B1) & 0xFFFFFFFF
+        w = ((self._pat_base + (int(key) & 0xFFFFFFFF)) & 0xFFFFFFFF) ^ (int(key) >> 32)
+        return w.to(torch.int32).view(torch.uint8).view(self.n_chunks, self.chunk_bytes)
+
+    def fill_block_pattern(self, tier, slot, key):
+        dst = self._chunks(tier, slot)
+        dst.copy_(self._pattern(key).to(dst.device))
+
+    def check_block_pattern(self, tier, slot, key) -> bool:
+        self.torch.cuda.current_stream().synchronize()
+        got = self._chunks(tier, slot).to(self.device)
+        return bool(self.torch.equal(got, self._pattern(key)))
+
     def write_block(self, tier, slot, payload):
         t = self.torch.from_numpy(np.ascontiguousarray(np.asarray(payload, np.uint8))).view(self.n_chunks, self.chunk_bytes)
         dst = self._chunks(tier, slot)

@@ -292,6 +292,7 @@ def payload_pattern(key: int, block_bytes: int) -> np.ndarray:
 @dataclass
 class ReplayOptions:
     payload: object = None        # callable(key, block_bytes) -> uint8 array, or None (metadata only)
+    writer: object = None         # callable(engine, slot, key): writes a new HBM block's payload in place (large blocks)
     record_states: bool = True    # record per-tier states / entries after every call (slow on big pools)
     verify_payload_every: int = 0 # every k-th call, read back every occupied slot and compare with payload(key)
     counters: dict = field(default_factory=dict)
@@ -350,10 +351,13 @@ def run_call(eng, ctxs, opt: ReplayOptions):
     for c, inf in zip(ctxs, adm):
         keys, tier, slot = eng.get_block_map(c)
         maps.append((keys.copy(), tier.copy(), slot.copy()))
-        if opt.payload is not None:
+        if opt.payload is not None or opt.writer is not None:
             for b in range(int(inf["hit_len"]), int(inf["n_held"])):
                 if tier[b] == TIER_HBM:
-                    eng.write_block(TIER_HBM, int(slot[b]), opt.payload(int(keys[b]), eng.block_bytes))
+                    if opt.writer is not None:
+                        opt.writer(eng, int(slot[b]), int(keys[b]))
+                    else:
+                        eng.write_block(TIER_HBM, int(slot[b]), opt.payload(int(keys[b]), eng.block_bytes))
     rec["maps"] = maps
     for c in ctxs:
         eng.prefill_done(c)

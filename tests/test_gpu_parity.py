@@ -206,6 +206,89 @@ def test_full_size_c3_metadata_parity(B, oracle):
     assert n > 100 and st["offloaded"] > 10000 and st["reloaded"] > 10000 and st["dropped"] > 10000
 
 
+def test_bench_steps_at_full_size_match_the_oracle(B, oracle):
+    """The benchmark's own step sequence (C2 session, 8B-class blocks, 20,480-block HBM pool, 61,440-block second
+    tier kept in HBM as in the bench's in-device arm, tier pressure after every call) against the metadata-only
+    oracle: every call's reports and the statistics are equal, and every resident block's payload survives."""
+    import sys
+    import torch
+    sys.path.insert(0, str(__import__("pathlib").Path(__file__).resolve().parents[1]))
+    import bench
+    geo = W.GEO_8B
+    free_b, _ = torch.cuda.mem_get_info()
+    if free_b < (20480 + 61440) * geo.block_bytes + (6 << 30):
+        pytest.skip("needs 160 GiB of HBM")
+    setup, turns, _target = bench.make_turns(1, 12)
+    kw = dict(n_hbm_blocks=20480, n_host_blocks=61440, max_contexts=4, **geo.kwargs())
+    gpu = B.Engine(max_tokens=1 << 21, max_messages=1 << 13, host_pool_on_device=True, zero_pools=False, **kw)
+    cpu = oracle.OracleEngine(metadata_only=True, **kw)
+    og = W.ReplayOptions(payload=None, record_states=False, writer=lambda e, slot, key: e.fill_block_pattern(0, slot, key))
+    oc = W.ReplayOptions(payload=None, record_states=False)
+    ident = lambda a: a
+    for ev in setup:
+        bench.apply_event(gpu, ev, ident)
+        bench.apply_event(cpu, ev, ident)
+    for t, (pre, ctxs, post) in enumerate(turns):
+        recs = []
+        for eng, opt in ((gpu, og), (cpu, oc)):
+            for ev in pre:
+                bench.apply_event(eng, ev, ident)
+            rec = W.run_call(eng, ctxs, opt)
+            for ev in post:
+                bench.apply_event(eng, ev, ident)
+            n = eng.get_stats()["occ_hbm"] // 2
+            rec["pressure"] = W.evict(eng, n) if n else {}
+            recs.append(rec)
+        diff = W.records_equal(recs[0], recs[1], f"turn {t}")
+        assert diff is None, diff
+    sg, sc = gpu.get_stats(), cpu.get_stats()
+    for k in sc:
+        if k not in W.GPU_ONLY_STATS:
+            assert sg[k] == sc[k], k
+    assert sc["offloaded"] > 50000 and sc["reloaded"] > 50000
+    bad = n_checked = 0
+    for tier in (0, 1):
+        keys = gpu.get_entries(tier)["key"]
+        for s in np.nonzero(keys)[0]:
+            n_checked += 1
+            bad += not gpu.check_block_pattern(tier, int(s), int(keys[s]))
+    assert bad == 0 and n_checked > 5000
+
+
+def test_full_size_c3_with_payload(B, oracle):
+    """C3 at full size with real payloads on the GPU: GLM-scale blocks (5.75 MiB), the 120 GiB HBM pool
+    (21,370 blocks) and a pinned host tier of 24 GiB (4,274 blocks; the oracle runs the same sizes metadata-only).
+    Every call's results equal the oracle's and, at the end, every occupied slot of both tiers holds the payload
+    of the key it is registered for, after ~50 K blocks have crossed the host link."""
+    import torch
+    free_b, _ = torch.cuda.mem_get_info()
+    geo = W.GEO_GLM
+    n_hbm = 21370
+    if free_b < (n_hbm * geo.block_bytes + (6 << 30)):
+        pytest.skip("needs a 120 GiB HBM pool")
+    trace, n_ctx = W.trace_c3(1)
+    kw = dict(n_hbm_blocks=n_hbm, n_host_blocks=4274, max_contexts=n_ctx, **geo.kwargs())
+    gpu = B.Engine(max_tokens=1 << 24, max_messages=1 << 16, zero_pools=False, **kw)
+    cpu = oracle.OracleEngine(metadata_only=True, **kw)
+    og = W.ReplayOptions(payload=None, record_states=False, writer=lambda e, slot, key: e.fill_block_pattern(0, slot, key))
+    oc = W.ReplayOptions(payload=None, record_states=False)
+    for (i, kind, rg), (_, _, rc) in zip(W.replay(gpu, trace, og), W.replay(cpu, trace, oc)):
+        if kind == "call":
+            diff = W.records_equal(rg, rc, f"event[{i}]")
+            assert diff is None, diff
+    sg, sc = gpu.get_stats(), cpu.get_stats()
+    for k in sc:
+        if k not in W.GPU_ONLY_STATS:
+            assert sg[k] == sc[k], k
+    assert sc["offloaded"] > 10000 and sc["reloaded"] > 5000
+    bad = 0
+    for tier in (0, 1):
+        keys = gpu.get_entries(tier)["key"]
+        for s in np.nonzero(keys)[0]:
+            bad += not gpu.check_block_pattern(tier, int(s), int(keys[s]))
+    assert bad == 0
+
+
 # ---- C4: metadata stress at full size -------------------------------------------------------------------
 def _c4_setup(B, oracle, n_resident, chain_blocks, n_calls):
     inp = W.inputs_c4(1, n_resident=n_resident, chain_blocks=chain_blocks, n_calls=n_calls)
