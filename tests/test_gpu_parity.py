@@ -215,6 +215,9 @@ def test_bench_steps_at_full_size_match_the_oracle(B, oracle):
     sys.path.insert(0, str(__import__("pathlib").Path(__file__).resolve().parents[1]))
     import bench
     geo = W.GEO_8B
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()          # memory cached from earlier tests counts as used otherwise
     free_b, _ = torch.cuda.mem_get_info()
     if free_b < (20480 + 61440) * geo.block_bytes + (6 << 30):
         pytest.skip("needs 160 GiB of HBM")
@@ -260,7 +263,10 @@ def test_full_size_c3_with_payload(B, oracle):
     (21,370 blocks) and a pinned host tier of 24 GiB (4,274 blocks; the oracle runs the same sizes metadata-only).
     Every call's results equal the oracle's and, at the end, every occupied slot of both tiers holds the payload
     of the key it is registered for, after ~50 K blocks have crossed the host link."""
+    import gc
     import torch
+    gc.collect()
+    torch.cuda.empty_cache()          # memory cached from earlier tests counts as used otherwise
     free_b, _ = torch.cuda.mem_get_info()
     geo = W.GEO_GLM
     n_hbm = 21370
