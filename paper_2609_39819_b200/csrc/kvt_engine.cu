@@ -142,6 +142,11 @@ struct kvt_engine {
   bool upload_pending = false;
   // optional timing of the mover kernel (kvt_set_profiling)
   bool profiling = false, mover_timed = false;
+  // CUDA graph of the radix-sort passes of kvt_select_victims, one per tier
+  struct SortGraph { cudaGraphExec_t exec = nullptr; u32 n_pass = 0; };
+  SortGraph sort_graph[2];
+  cudaStream_t capture_stream = nullptr;   // only ever used for stream capture, never executes work
+  bool use_graphs = true;
   u32 mover_variant = 0;   // 0 auto, 1 CTA per chunk, 2 warp per 4 KiB tile, 3 TMA ring
   bool tma_attr_set = false;
   cudaEvent_t ev_m0 = nullptr, ev_m1 = nullptr, ev_h0 = nullptr, ev_h1 = nullptr;
@@ -490,6 +495,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   e->h_mstart = (u32 *)(e->stage + o_ms); e->h_mend = (u32 *)(e->stage + o_me); e->h_mrank = e->stage + o_mr;
   e->h_ids = (u32 *)(e->stage + o_ids); e->h_ids2 = (u32 *)(e->stage + o_ids2); e->h_out = e->stage + o_out;
   cudaStream_t s = (cudaStream_t)stream;
+  if (cudaStreamCreateWithFlags(&e->capture_stream, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); e->use_graphs = false; }
   bool ok = cudaEventCreateWithFlags(&e->ev_upload, cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreate(&e->ev_m0) == cudaSuccess && cudaEventCreate(&e->ev_m1) == cudaSuccess &&
             cudaEventCreate(&e->ev_h0) == cudaSuccess && cudaEventCreate(&e->ev_h1) == cudaSuccess;
@@ -509,6 +515,8 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
 int32_t kvt_destroy(kvt_engine *e) {
   if (!e) return KVT_E_INVAL;
   cudaDeviceSynchronize();
+  for (auto &g : e->sort_graph) if (g.exec) cudaGraphExecDestroy(g.exec);
+  if (e->capture_stream) cudaStreamDestroy(e->capture_stream);
   if (e->ev_upload) cudaEventDestroy(e->ev_upload);
   if (e->ev_m0) cudaEventDestroy(e->ev_m0);
   if (e->ev_m1) cudaEventDestroy(e->ev_m1);
@@ -1023,11 +1031,42 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   r = compact_indices(e, s, PredSel{a}, EmitSel{a, kA, vA}, n, ST_M);
   if (r) return r;
   const u32 key_bits = 2 + a.copy_bit + a.stamp_bits + a.depth_bits, n_pass = cdiv(key_bits, 8), tiles = cdiv(n, SORT_TILE);
-  for (u32 p = 0; p < n_pass; ++p) {
-    KL(k_radix_hist, tiles, 256, s, kA, e->d_status, 8 * p, counts);
-    KL(k_radix_scan, 32, 256, s, counts, row_total, e->d_status);
-    KL(k_radix_scatter, tiles, 256, s, kA, vA, kB, vB, e->d_status, 8 * p, counts, row_total);
-    std::swap(kA, kB); std::swap(vA, vB);
+  // The radix passes are a fixed sequence of short kernels (same buffers, same grids, element count read from
+  // the status block), i.e. launch-bound: they are captured once per (tier, pass count) into a CUDA graph on a
+  // private capture stream and replayed on the caller's stream with one launch.
+  {
+    kvt_engine::SortGraph &g = e->sort_graph[tier];
+    if (e->use_graphs && (!g.exec || g.n_pass != n_pass)) {
+      if (g.exec) { cudaGraphExecDestroy(g.exec); g.exec = nullptr; }
+      cudaGraph_t graph = nullptr;
+      bool ok = cudaStreamBeginCapture(e->capture_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
+      if (ok) {
+        u64 *ka = kA, *kb = kB; u32 *va = vA, *vb = vB;
+        for (u32 p = 0; p < n_pass; ++p) {
+          k_radix_hist<<<tiles, 256, 0, e->capture_stream>>>(ka, e->d_status, 8 * p, counts);
+          k_radix_scan<<<32, 256, 0, e->capture_stream>>>(counts, row_total, e->d_status);
+          k_radix_scatter<<<tiles, 256, 0, e->capture_stream>>>(ka, va, kb, vb, e->d_status, 8 * p, counts, row_total);
+          std::swap(ka, kb); std::swap(va, vb);
+        }
+        ok = cudaStreamEndCapture(e->capture_stream, &graph) == cudaSuccess && graph;
+      }
+      if (ok) ok = cudaGraphInstantiate(&g.exec, graph, 0) == cudaSuccess;
+      if (graph) cudaGraphDestroy(graph);
+      if (!ok) { cudaGetLastError(); g.exec = nullptr; e->use_graphs = false; }   // fall back to plain launches
+      g.n_pass = n_pass;
+    }
+    if (e->use_graphs && g.exec) {
+      CU(cudaGraphLaunch(g.exec, s));
+      e->st.kernel_launches += 3ull * n_pass;
+      if (n_pass & 1) { std::swap(kA, kB); std::swap(vA, vB); }
+    } else {
+      for (u32 p = 0; p < n_pass; ++p) {
+        KL(k_radix_hist, tiles, 256, s, kA, e->d_status, 8 * p, counts);
+        KL(k_radix_scan, 32, 256, s, counts, row_total, e->d_status);
+        KL(k_radix_scatter, tiles, 256, s, kA, vA, kB, vB, e->d_status, 8 * p, counts, row_total);
+        std::swap(kA, kB); std::swap(vA, vB);
+      }
+    }
   }
   u32 n_emit = std::min(n_req, n);
   KL(k_sel_emit, cdiv(n_emit,256), 256, s, e->ent, a.e0, n, kA, vA, n_emit, e->d_status, a.stamp_bits + a.depth_bits, a.copy_bit, e->dp<u32>(e->L.out_slots),
