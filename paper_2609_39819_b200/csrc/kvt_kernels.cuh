@@ -21,7 +21,8 @@ constexpr u32 ENT_NONE = 0xFFFFFFFFu;
 constexpr u32 CLAIM_BIT = 0x80000000u;
 constexpr u32 CHUNK = 256;        // blocks hashed by one CTA
 constexpr u32 SCAN_TILE = 1024;   // items per CTA in the ordered-compaction kernels
-constexpr u32 SORT_TILE = 4096;   // items per CTA in the radix-sort kernels (8 warps x 512)
+constexpr u32 SORT_TILE = 1024;   // items per CTA in the radix-sort kernels (8 warps x 128): small tiles keep all SMs busy
+constexpr int SORT_ITERS = SORT_TILE / 256;   // items per thread
 
 // bits of the device error word
 enum : u32 { DERR_PROBE = 1, DERR_RANGE = 2, DERR_INVAL = 4, DERR_STATE = 8, DERR_CORRUPT = 16 };
@@ -710,7 +711,7 @@ __global__ void __launch_bounds__(256) k_radix_scan(u32 *counts, u32 *row_total,
 
 __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const u32 *vals_in, u64 *keys_out, u32 *vals_out,
                                                        const u32 *status, u32 shift, const u32 *offsets, const u32 *row_total) {
-  // each warp owns 512 consecutive items of the tile and walks them in order, so equal digits keep
+  // each warp owns SORT_TILE / 8 consecutive items of the tile and walks them in order, so equal digits keep
   // their input order (stable)
   __shared__ u32 cnt[8][256];
   __shared__ u32 dbase[256];
@@ -721,11 +722,11 @@ __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const
   const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   for (u32 k = tid; k < 8 * 256; k += 256) (&cnt[0][0])[k] = 0;
   __syncthreads();
-  const u32 base = blockIdx.x * SORT_TILE + warp * 512;
-  u64 kreg[16];
-  u32 vreg[16];
+  const u32 base = blockIdx.x * SORT_TILE + warp * (SORT_TILE / 8);
+  u64 kreg[SORT_ITERS];
+  u32 vreg[SORT_ITERS];
 #pragma unroll
-  for (int it = 0; it < 16; ++it) {
+  for (int it = 0; it < SORT_ITERS; ++it) {
     u32 i = base + it * 32 + lane;
     bool ok = i < m;
     kreg[it] = ok ? keys_in[i] : 0;
@@ -755,7 +756,7 @@ __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const
   }
   __syncthreads();
 #pragma unroll
-  for (int it = 0; it < 16; ++it) {
+  for (int it = 0; it < SORT_ITERS; ++it) {
     u32 i = base + it * 32 + lane;
     bool ok = i < m;
     u32 d = (u32)(kreg[it] >> shift) & 255u;
