@@ -11,7 +11,7 @@ apply ops -> hash -> lookup -> classify -> select victims -> offload -> reload -
 
 Two measurements of the same steps:
   value : second tier resident in HBM and tokens resident on the device (inputs in HBM when the timed
-          region starts); the mover runs HBM<->HBM and is judged against the HBM roofline.
+          region starts); the mover runs HBM<->HBM and is measured against the HBM roofline.
   e2e   : the real thing through the same C-ABI calls: tokens come from pinned host buffers, the
           second tier is pinned host memory, every offload / reload crosses the host link inside the
           timed region.
