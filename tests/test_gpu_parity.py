@@ -546,3 +546,32 @@ def test_incremental_hashing_resumes_at_chunk_boundaries(B, oracle):
     assert got == len(keys) - 512
     st = gpu.get_stats()
     assert st["blocks_rehashed"] < st["blocks_hashed"]
+
+
+def test_create_rejects_bad_configs(B):
+    import ctypes as C
+    import torch
+    lib = B.load_library()
+    good = B.Engine(n_hbm_blocks=16, n_host_blocks=4, max_contexts=4, max_tokens=4096, max_messages=64, **W.GEO_TOY.kwargs())
+
+    def attempt(**changes):
+        cfg = B.Config.from_buffer_copy(good.cfg)
+        for k, v in changes.items():
+            setattr(cfg, k, v)
+        h = C.c_void_p()
+        rc = lib.kvt_create(C.byref(cfg), C.c_void_p(torch.cuda.current_stream().cuda_stream), C.byref(h))
+        if rc == 0:
+            lib.kvt_destroy(h)
+        return rc
+
+    assert attempt() == B.OK                                   # the unmodified copy is fine
+    assert attempt(abi_version=2) == B.E_INVAL
+    assert attempt(block_tokens=32) == B.E_INVAL
+    assert attempt(table_capacity=good.cfg.table_capacity + 1) == B.E_INVAL      # not a power of two
+    assert attempt(table_capacity=16) == B.E_INVAL                                # < 2 * (hbm + host)
+    assert attempt(dev_meta=good.cfg.dev_meta + 8) == B.E_INVAL                   # misaligned arena
+    assert attempt(dev_meta_bytes=1024) == B.E_INVAL                              # arena too small
+    assert attempt(hbm_pool_bytes=1024) == B.E_INVAL
+    assert attempt(suspended_order=2) == B.E_INVAL and attempt(policy_flags=8) == B.E_INVAL
+    assert attempt(n_hbm_blocks=0) == B.E_INVAL and attempt(max_contexts=0) == B.E_INVAL
+    assert lib.kvt_create(None, None, None) == B.E_INVAL
