@@ -274,6 +274,16 @@ int32_t kvt_offload(kvt_engine *e, const uint32_t *hbm_slots, uint32_t n, uint32
 int32_t kvt_reload(kvt_engine *e, const uint32_t *host_slots, uint32_t n, uint32_t *n_done,
                    void *stream);
 
+/* Reload and offload in one call, for the common step "bring my prefix back and push other blocks out": the
+ * listed host slots move to the HBM slots that are free when the call begins (as kvt_reload does), the listed
+ * HBM slots are dropped / handed over / moved to the host slots that are free when the call begins (as
+ * kvt_offload does). Because neither list depends on slots the other one frees, the two payload streams are
+ * issued by ONE mover launch and cross the host link in both directions at the same time (the link is full
+ * duplex). Both lists are validated before anything changes (same codes as the single calls). KVT_E_NOSPACE if
+ * either direction ran out of destination slots; the three counts tell how far each got. Synchronises. */
+int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_out, const uint32_t *host_slots_in,
+                     uint32_t n_in, uint32_t *n_out_done, uint32_t *n_dropped, uint32_t *n_in_done, void *stream);
+
 /* Drops blocks without copying (frees host space for offloads). Same validation as kvt_offload.
  * Releasing an HBM block frees its clean host copy too; releasing a clean copy leaves its block alone. */
 int32_t kvt_release(kvt_engine *e, uint32_t tier, const uint32_t *slots, uint32_t n, void *stream);

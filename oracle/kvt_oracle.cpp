@@ -704,6 +704,70 @@ int32_t kvto_reload(Engine *e, const uint32_t *slots, uint32_t n, uint32_t *n_do
   return OK;
 }
 
+// Reload and offload in one call, both with destinations taken from the slots that are free when the call
+// begins (the two payload streams are independent, so a device can run them concurrently over a duplex link).
+int32_t kvto_exchange(Engine *e, const uint32_t *out_slots, uint32_t n_out, const uint32_t *in_slots, uint32_t n_in,
+                      uint32_t *n_out_done, uint32_t *n_dropped, uint32_t *n_in_done) {
+  if (!e || (!out_slots && n_out) || (!in_slots && n_in) || !n_out_done || !n_dropped || !n_in_done) return E_INVAL;
+  *n_out_done = *n_dropped = *n_in_done = 0;
+  int32_t va = validate_slots(e, TIER_HOST, in_slots, n_in, true, false);
+  int32_t vb = validate_slots(e, TIER_HBM, out_slots, n_out, false);
+  for (int32_t code : {E_RANGE, E_INVAL, E_STATE})
+    if (va == code || vb == code) return code;
+  std::vector<uint8_t> rank[2];
+  classify(*e, rank);
+  const bool knows_dead = !(e->cfg.policy_flags & POLICY_NO_LIFECYCLE);
+  std::vector<uint32_t> hbm_dests(e->free_slots[TIER_HBM].begin(), e->free_slots[TIER_HBM].end());
+  std::vector<uint32_t> host_dests(e->free_slots[TIER_HOST].begin(), e->free_slots[TIER_HOST].end());
+  bool full = false;
+  for (uint32_t i = 0; i < n_in; ++i) {               // incoming blocks
+    if (i == hbm_dests.size()) { full = true; break; }
+    uint32_t h = in_slots[i], d = hbm_dests[i];
+    if (e->cfg.policy_flags & POLICY_INCLUSIVE) {
+      copy_payload(*e, TIER_HOST, h, TIER_HBM, d);
+      Entry x = e->ent[TIER_HOST][h];
+      x.link = h;
+      e->ent[TIER_HBM][d] = x;
+      e->free_slots[TIER_HBM].erase(d);
+      e->ent[TIER_HOST][h].shadow = true;
+      e->ent[TIER_HOST][h].link = d;
+      e->ent[TIER_HOST][h].inflight = 0;
+      e->where[x.key] = {TIER_HBM, d};
+    } else {
+      move_entry(e, TIER_HOST, h, TIER_HBM, d);
+    }
+    e->st.reloaded++;
+    e->st.bytes_h2d += e->block_bytes;
+    (*n_in_done)++;
+  }
+  size_t next_dest = 0;
+  for (uint32_t i = 0; i < n_out; ++i) {              // outgoing blocks
+    uint32_t s = out_slots[i];
+    if (knows_dead && rank[0][s] == 0) {
+      free_slot(*e, TIER_HBM, s);
+      e->st.dropped++;
+      (*n_dropped)++;
+    } else if (e->ent[TIER_HBM][s].link >= 0) {
+      Entry x = e->ent[TIER_HBM][s];
+      Entry &h = e->ent[TIER_HOST][x.link];
+      h.shadow = false; h.link = -1; h.stamp = x.stamp; h.depth = x.depth; h.floor = x.floor; h.inflight = x.inflight;
+      e->where[x.key] = {TIER_HOST, (uint32_t)x.link};
+      e->ent[TIER_HBM][s] = Entry();
+      e->free_slots[TIER_HBM].insert(s);
+      e->st.offloaded++;
+      e->st.offloaded_clean++;
+    } else {
+      if (next_dest == host_dests.size()) { full = true; break; }
+      uint32_t d = host_dests[next_dest++];
+      move_entry(e, TIER_HBM, s, TIER_HOST, d);
+      e->st.offloaded++;
+      e->st.bytes_d2h += e->block_bytes;
+    }
+    (*n_out_done)++;
+  }
+  return full ? E_NOSPACE : OK;
+}
+
 int32_t kvto_release(Engine *e, uint32_t tier, const uint32_t *slots, uint32_t n) {
   if (!e || tier > 1 || (!slots && n)) return E_INVAL;
   int32_t v = validate_slots(e, tier, slots, n, false);

@@ -230,6 +230,12 @@ class OracleEngine:
         rc = self.L.kvto_reload(self.h, _p(s), len(s), C.byref(nd))
         return rc, nd.value
 
+    def exchange(self, out_slots, in_slots):
+        o, i = _u32(out_slots), _u32(in_slots)
+        a, b, c = C.c_uint32(0), C.c_uint32(0), C.c_uint32(0)
+        rc = self.L.kvto_exchange(self.h, _p(o), len(o), _p(i), len(i), C.byref(a), C.byref(b), C.byref(c))
+        return rc, a.value, b.value, c.value
+
     def release_rc(self, tier, slots):
         s = _u32(slots)
         return self.L.kvto_release(self.h, tier, _p(s), len(s))

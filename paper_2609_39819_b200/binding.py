@@ -27,7 +27,7 @@ EXPORTS = ("kvt_query_sizes", "kvt_create", "kvt_destroy", "kvt_apply_op", "kvt_
            "kvt_classify", "kvt_get_states", "kvt_select_victims", "kvt_offload", "kvt_reload", "kvt_release",
            "kvt_compact", "kvt_copy_blocks", "kvt_hash_scratch_bytes", "kvt_hash_tokens", "kvt_get_stats",
            "kvt_last_error", "kvt_get_entries", "kvt_debug_load_resident", "kvt_set_profiling",
-           "kvt_hash_tokens_noalloc", "kvt_debug_set_mover_variant")
+           "kvt_hash_tokens_noalloc", "kvt_debug_set_mover_variant", "kvt_exchange")
 
 
 class KvtError(RuntimeError):
@@ -90,6 +90,7 @@ def load_library():
             "kvt_select_victims": [vp, u32, u32, u32, vp, vp, u32, vp, vp],
             "kvt_offload": [vp, vp, u32, vp, vp, vp],
             "kvt_reload": [vp, vp, u32, vp, vp],
+            "kvt_exchange": [vp, vp, u32, vp, u32, vp, vp, vp, vp],
             "kvt_release": [vp, u32, vp, u32, vp],
             "kvt_compact": [vp, u32, vp, vp],
             "kvt_copy_blocks": [vp, u32, vp, u32, vp, u32, u32, vp],
@@ -329,6 +330,12 @@ class Engine:
         s = _u32(slots); nd = C.c_uint32(0)
         rc = self.L.kvt_reload(self.h, _p(s), len(s), C.byref(nd), _stream())
         return rc, nd.value
+
+    def exchange(self, out_slots, in_slots):
+        o, i = _u32(out_slots), _u32(in_slots)
+        a, b, c = C.c_uint32(0), C.c_uint32(0), C.c_uint32(0)
+        rc = self.L.kvt_exchange(self.h, _p(o), len(o), _p(i), len(i), C.byref(a), C.byref(b), C.byref(c), _stream())
+        return rc, a.value, b.value, c.value
 
     def release_rc(self, tier, slots):
         s = _u32(slots)

@@ -76,7 +76,7 @@ struct Ctx {
 
 struct DevLayout {
   u64 tab, e_key, e_stamp, e_depth, e_infl, e_rank, e_tslot, e_mark, e_link, e_floor, keys, status;
-  u64 s0, s1, s2, s3, ids, ids2, pair_src, pair_dst, freelist, tiles, agg, carry, desc, ctxres;
+  u64 s0, s1, s2, s3, ids, ids2, pair_src, pair_dst, pair_src2, pair_dst2, freelist, freelist2, tiles, agg, carry, desc, ctxres;
   u64 m_start, m_end, m_rank, keyA, keyB, valA, valB, rcounts, out_slots, out_states, map_tier, map_slot;
   u64 total;
   u64 LB, Nt, N;
@@ -96,7 +96,7 @@ DevLayout make_layout(const kvt_config &c) {
   L.status = take(ST_WORDS * 4);
   L.s0 = take(LB * 4); L.s1 = take(LB * 4); L.s2 = take(LB * 4); L.s3 = take(LB * 4);
   L.ids = take(LB * 4); L.ids2 = take(LB * 4); L.pair_src = take(LB * 4); L.pair_dst = take(LB * 4);
-  L.freelist = take(LB * 4);
+  L.freelist = take(LB * 4); L.freelist2 = take(LB * 4); L.pair_src2 = take(LB * 4); L.pair_dst2 = take(LB * 4);
   L.tiles = take((std::max(LB, N) / SCAN_TILE + 2) * 4);
   u64 n_chunks = B / CHUNK + C + 1;
   L.agg = take(n_chunks * 8); L.carry = take(n_chunks * 8);
@@ -1126,9 +1126,10 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
   a.pair_src = e->dp<u32>(e->L.pair_src); a.pair_dst = e->dp<u32>(e->L.pair_dst);
   a.allow_inflight = m.allow_inflight; a.drop_dead = m.drop_dead; a.drop_all = m.drop_all;
   a.reject_shadow = m.reject_shadow; a.clean_ok = m.clean_ok; a.keep_copy = m.keep_copy; a.status = e->d_status;
+  a.w_cut = ST_CUT; a.w_nlive = ST_NLIVE; a.w_ndrop = ST_NDROP; a.w_nclean = ST_NCLEAN; a.w_nshdrop = ST_NSHDROP;
   u32 g = cdiv(n, 256);
   KL(k_list_validate, g, 256, s, a);
-  r = compact_indices(e, s, PredLive{a.live}, EmitLive{a.lidx, a.n_free, e->d_status}, n, ST_TOTAL);
+  r = compact_indices(e, s, PredLive{a.live}, EmitLive{a.lidx, a.n_free, e->d_status + ST_CUT}, n, ST_TOTAL);
   if (r) return r;
   if (!m.drop_all) {
     r = compact_indices(e, s, PredFree{e->ent.key, a.dst_e0}, EmitFree{e->dp<u32>(e->L.freelist), (u32)e->L.LB},
@@ -1191,6 +1192,106 @@ int32_t kvt_reload(kvt_engine *e, const uint32_t *host_slots, uint32_t n, uint32
   e->st.bytes_h2d += c.copied * e->block_bytes;
   if (r == KVT_E_NOSPACE) e->err = "HBM tier full";
   return r;
+}
+
+int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_out, const uint32_t *host_slots_in,
+                     uint32_t n_in, uint32_t *n_out_done, uint32_t *n_dropped, uint32_t *n_in_done, void *stream) {
+  if (!e || (!hbm_slots_out && n_out) || (!host_slots_in && n_in) || !n_out_done || !n_dropped || !n_in_done) return KVT_E_INVAL;
+  *n_out_done = *n_dropped = *n_in_done = 0;
+  cudaStream_t s = (cudaStream_t)stream;
+  if (n_out == 0 && n_in == 0) return KVT_OK;
+  if (n_out > e->L.LB || n_in > e->L.LB) return fail(e, KVT_E_NOSPACE, "list longer than max_batch_blocks");
+  int32_t r = ensure_classified(e, s);
+  if (r) return r;
+  r = stage_acquire(e);
+  if (r) return r;
+  u32 *d_in = e->dp<u32>(e->L.ids), *d_out = e->dp<u32>(e->L.ids2);
+  if (n_in) { std::memcpy(e->h_ids, host_slots_in, n_in * 4ull); CU(cudaMemcpyAsync(d_in, e->h_ids, n_in * 4ull, cudaMemcpyHostToDevice, s)); }
+  if (n_out) { std::memcpy(e->h_ids2, hbm_slots_out, n_out * 4ull); CU(cudaMemcpyAsync(d_out, e->h_ids2, n_out * 4ull, cudaMemcpyHostToDevice, s)); }
+  r = stage_release(e, s);
+  if (r) return r;
+  r = status_zero(e, s);
+  if (r) return r;
+  CU(cudaMemcpyAsync(e->d_status + ST_CUT, &n_in, 4, cudaMemcpyHostToDevice, s));
+  CU(cudaMemcpyAsync(e->d_status + ST_B_CUT, &n_out, 4, cudaMemcpyHostToDevice, s));
+  // list A: incoming (host -> HBM); list B: outgoing (HBM -> host). Both plans use the free slots of call begin.
+  ListArgs a{}, b{};
+  a.tab = b.tab = e->tab; a.ent = b.ent = e->ent; a.status = b.status = e->d_status;
+  a.ids = d_in; a.n = n_in; a.e0 = e->tier_e0(KVT_TIER_HOST); a.n_slots = e->cfg.n_host_blocks; a.dst_e0 = 0;
+  a.live = e->dp<u32>(e->L.s1); a.lidx = e->dp<u32>(e->L.s2); a.freelist = e->dp<u32>(e->L.freelist);
+  a.n_free = e->cfg.n_hbm_blocks - e->occ[0];
+  a.pair_src = e->dp<u32>(e->L.pair_src); a.pair_dst = e->dp<u32>(e->L.pair_dst);
+  a.allow_inflight = 1; a.reject_shadow = 1; a.keep_copy = (e->cfg.policy_flags & KVT_POLICY_INCLUSIVE) ? 1 : 0;
+  a.w_cut = ST_CUT; a.w_nlive = ST_NLIVE; a.w_ndrop = ST_NDROP; a.w_nclean = ST_NCLEAN; a.w_nshdrop = ST_NSHDROP;
+  b.ids = d_out; b.n = n_out; b.e0 = 0; b.n_slots = e->cfg.n_hbm_blocks; b.dst_e0 = e->tier_e0(KVT_TIER_HOST);
+  b.live = e->dp<u32>(e->L.s3); b.lidx = e->dp<u32>(e->L.s0); b.freelist = e->dp<u32>(e->L.freelist2);
+  b.n_free = e->cfg.n_host_blocks - e->occ[1];
+  b.pair_src = e->dp<u32>(e->L.pair_src2); b.pair_dst = e->dp<u32>(e->L.pair_dst2);
+  b.drop_dead = !(e->cfg.policy_flags & KVT_POLICY_NO_LIFECYCLE); b.clean_ok = 1;
+  b.w_cut = ST_B_CUT; b.w_nlive = ST_B_NLIVE; b.w_ndrop = ST_B_NDROP; b.w_nclean = ST_B_NCLEAN; b.w_nshdrop = ST_B_NSHDROP;
+  const u32 ga = cdiv(n_in, 256), gb = cdiv(n_out, 256);
+  if (n_in) KL(k_list_validate, ga, 256, s, a);
+  if (n_out) KL(k_list_validate, gb, 256, s, b);
+  if (n_in) { r = compact_indices(e, s, PredLive{a.live}, EmitLive{a.lidx, a.n_free, e->d_status + ST_CUT}, n_in, ST_TOTAL); if (r) return r; }
+  if (n_out) { r = compact_indices(e, s, PredLive{b.live}, EmitLive{b.lidx, b.n_free, e->d_status + ST_B_CUT}, n_out, ST_B_TOTAL); if (r) return r; }
+  r = compact_indices(e, s, PredFree{e->ent.key, 0}, EmitFree{e->dp<u32>(e->L.freelist), (u32)e->L.LB}, e->cfg.n_hbm_blocks, ST_FREE);
+  if (r) return r;
+  if (e->cfg.n_host_blocks) {
+    r = compact_indices(e, s, PredFree{e->ent.key, b.dst_e0}, EmitFree{e->dp<u32>(e->L.freelist2), (u32)e->L.LB}, e->cfg.n_host_blocks, ST_B_FREE);
+    if (r) return r;
+  }
+  if (n_in) { KL(k_list_apply, ga, 256, s, a); KL(k_list_unmark, ga, 256, s, a); }
+  if (n_out) { KL(k_list_apply, gb, 256, s, b); KL(k_list_unmark, gb, 256, s, b); }
+  LAUNCH_CHECK();
+  // one mover launch for both directions
+  if (!e->metadata_only) {
+    MoveArgs ma{}, mb{};
+    ma.src = pool_view(e, KVT_TIER_HOST); ma.dst = pool_view(e, KVT_TIER_HBM); ma.src_ids = a.pair_src; ma.dst_ids = a.pair_dst;
+    ma.n_pairs = std::min(n_in, a.n_free); ma.n_pairs_dev = e->d_status + ST_NLIVE;
+    mb.src = pool_view(e, KVT_TIER_HBM); mb.dst = pool_view(e, KVT_TIER_HOST); mb.src_ids = b.pair_src; mb.dst_ids = b.pair_dst;
+    mb.n_pairs = std::min(n_out, b.n_free); mb.n_pairs_dev = e->d_status + ST_B_NLIVE;
+    ma.n_chunks = mb.n_chunks = (u32)e->n_chunks; ma.chunk_bytes = mb.chunk_bytes = (u32)e->chunk_bytes; ma.status = mb.status = e->d_status;
+    u64 items = ((u64)ma.n_pairs + mb.n_pairs) * e->n_chunks;
+    if (items) {
+      const bool timed = e->profiling;
+      if (timed) CU(cudaEventRecord(e->ev_m0, s));
+      if (e->chunk_bytes % 4096 == 0) {
+        u32 tpc = (u32)(e->chunk_bytes / 4096);
+        u32 grid = (u32)std::min<u64>((items * tpc + 7) / 8, (u64)e->sm_count * 8);
+        KL(k_move_tiles_dual<8>, grid, 256, s, ma, mb, tpc);
+      } else {   // chunk sizes the tile kernel cannot split: one direction after the other
+        u32 g1 = (u32)std::min<u64>((u64)ma.n_pairs * e->n_chunks, (u64)e->sm_count * 8);
+        u32 g2 = (u32)std::min<u64>((u64)mb.n_pairs * e->n_chunks, (u64)e->sm_count * 8);
+        if (g1) KL(k_move_blocks<4>, g1, 256, s, ma);
+        if (g2) KL(k_move_blocks<4>, g2, 256, s, mb);
+      }
+      if (timed) { CU(cudaEventRecord(e->ev_m1, s)); e->mover_timed = true; }
+      LAUNCH_CHECK();
+    }
+  }
+  r = status_fetch(e, s);
+  if (r) return r;
+  r = status_code(e);
+  if (r) return r;
+  const u32 *h = e->h_status;
+  const u32 in_copied = h[ST_NLIVE], out_copied = h[ST_B_NLIVE], out_drop = h[ST_B_NDROP], out_clean = h[ST_B_NCLEAN];
+  mover_account(e, (u64)in_copied + out_copied);
+  *n_in_done = in_copied;
+  *n_out_done = out_copied + out_drop + out_clean;
+  *n_dropped = out_drop;
+  e->occ[KVT_TIER_HBM] += in_copied;
+  if (!a.keep_copy) e->occ[KVT_TIER_HOST] -= in_copied;
+  e->occ[KVT_TIER_HBM] -= *n_out_done;
+  e->occ[KVT_TIER_HOST] += out_copied;
+  e->occ[KVT_TIER_HOST] -= h[ST_B_NSHDROP];
+  e->tombs += h[ST_TOMBS];
+  e->st.dropped += out_drop;
+  e->st.reloaded += in_copied; e->st.bytes_h2d += in_copied * e->block_bytes;
+  e->st.offloaded += out_copied + out_clean; e->st.offloaded_clean += out_clean; e->st.bytes_d2h += out_copied * e->block_bytes;
+  r = maybe_rebuild(e, s);
+  if (r) return r;
+  if (*n_in_done < n_in || *n_out_done < n_out) return fail(e, KVT_E_NOSPACE, "exchange: a tier ran out of free slots");
+  return KVT_OK;
 }
 
 int32_t kvt_release(kvt_engine *e, uint32_t tier, const uint32_t *slots, uint32_t n, void *stream) {

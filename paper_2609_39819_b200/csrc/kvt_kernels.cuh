@@ -31,6 +31,7 @@ enum : u32 { DERR_PROBE = 1, DERR_RANGE = 2, DERR_INVAL = 4, DERR_STATE = 8, DER
 enum : int {
   ST_ERR = 0, ST_TOTAL, ST_CUT, ST_NLIVE, ST_NDROP, ST_NEW, ST_INSERTED, ST_ADOPTED, ST_TOMBS,
   ST_RANK0, ST_RANK1, ST_RANK2, ST_RANK3, ST_M, ST_NMOVED, ST_FREE, ST_AUX, ST_SHADOW, ST_NCLEAN, ST_NSHDROP,
+  ST_B_CUT, ST_B_NLIVE, ST_B_NDROP, ST_B_NCLEAN, ST_B_NSHDROP, ST_B_TOTAL, ST_B_FREE,   // second list of an exchange
   ST_WORDS = 32
 };
 
@@ -801,6 +802,7 @@ struct ListArgs {
   u32 reject_shadow;                         // reload: a host slot that is only a copy is not a resident block
   u32 clean_ok;                              // offload: a block with a clean host copy is handed over without a copy
   u32 keep_copy;                             // reload with inclusive tiers: the host slot stays as a clean copy
+  u32 w_cut, w_nlive, w_ndrop, w_nclean, w_nshdrop;   // status words this list counts in
   u32 *status;
 };
 enum : u32 { LIST_DROP = 0, LIST_COPY = 1, LIST_CLEAN = 2 };
@@ -833,8 +835,8 @@ __global__ void k_list_unmark(ListArgs a) {
 struct PredLive { const u32 *live; __device__ bool operator()(u32 i) const { return live[i] == LIST_COPY; } };
 // item with rank r needs the r-th free destination slot; the first one that does not fit cuts the list
 struct EmitLive {
-  u32 *lidx; u32 n_free; u32 *status;
-  __device__ void operator()(u32 i, u32 r) const { lidx[i] = r; if (r >= n_free) atomicMin(&status[ST_CUT], i); }
+  u32 *lidx; u32 n_free; u32 *cut;
+  __device__ void operator()(u32 i, u32 r) const { lidx[i] = r; if (r >= n_free) atomicMin(cut, i); }
 };
 struct PredFree { const u64 *key; u32 e0; __device__ bool operator()(u32 i) const { return key[e0 + i] == 0; } };
 struct EmitFree { u32 *list; u32 cap; __device__ void operator()(u32 i, u32 r) const { if (r < cap) list[r] = i; } };
@@ -861,7 +863,7 @@ __global__ void k_list_apply(ListArgs a) {
   u32 i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= a.n) return;
   if (a.status[ST_ERR]) return;
-  if (i >= a.status[ST_CUT]) return;
+  if (i >= a.status[a.w_cut]) return;
   u32 id = a.ids[i];
   u32 e = a.e0 + id;
   u32 cat = a.live[i];
@@ -874,10 +876,10 @@ __global__ void k_list_apply(ListArgs a) {
       a.tab.slots[s].ent = ENT_NONE;
       atomicAdd(&a.status[ST_TOMBS], 1u);
       u32 l = a.ent.link[e];
-      if (l != ENT_NONE) { entry_clear(a.ent, l); atomicAdd(&a.status[ST_NSHDROP], 1u); }
+      if (l != ENT_NONE) { entry_clear(a.ent, l); atomicAdd(&a.status[a.w_nshdrop], 1u); }
     }
     entry_clear(a.ent, e);
-    atomicAdd(&a.status[ST_NDROP], 1u);
+    atomicAdd(&a.status[a.w_ndrop], 1u);
   } else if (cat == LIST_CLEAN) {        // hand the block over to its clean host copy: metadata only
     u32 h = a.ent.link[e];
     a.ent.stamp[h] = a.ent.stamp[e]; a.ent.depth[h] = a.ent.depth[e]; a.ent.infl[h] = a.ent.infl[e];
@@ -887,7 +889,7 @@ __global__ void k_list_apply(ListArgs a) {
     a.tab.slots[s].ent = h;
     a.ent.link[h] = ENT_NONE;
     entry_clear(a.ent, e);
-    atomicAdd(&a.status[ST_NCLEAN], 1u);
+    atomicAdd(&a.status[a.w_nclean], 1u);
   } else {
     u32 r = a.lidx[i];
     u32 d = a.freelist[r];
@@ -905,7 +907,7 @@ __global__ void k_list_apply(ListArgs a) {
     } else {
       entry_move(a.tab, a.ent, e, de);
     }
-    atomicAdd(&a.status[ST_NLIVE], 1u);
+    atomicAdd(&a.status[a.w_nlive], 1u);
   }
 }
 
@@ -1008,6 +1010,40 @@ __global__ void __launch_bounds__(256) k_move_tiles(MoveArgs a, u32 tiles_per_ch
     const uint4 *sp = reinterpret_cast<const uint4 *>(a.src.base + s * a.src.slot_stride + chunk * a.src.chunk_stride) +
                       (u64)tile * 32 * UNROLL + lane;
     uint4 *dp = reinterpret_cast<uint4 *>(a.dst.base + d * a.dst.slot_stride + chunk * a.dst.chunk_stride) +
+                (u64)tile * 32 * UNROLL + lane;
+    uint4 r[UNROLL];
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) r[u] = __ldcs(sp + u * 32);
+#pragma unroll
+    for (int u = 0; u < UNROLL; ++u) __stcs(dp + u * 32, r[u]);
+  }
+}
+
+// Two independent pair lists in one launch (kvt_exchange): list a and list b alternate tile by tile while both
+// last, so that loads from and stores to the host tier are in flight at the same time (the link is full duplex).
+template <int UNROLL>
+__global__ void __launch_bounds__(256) k_move_tiles_dual(MoveArgs a, MoveArgs b, u32 tiles_per_chunk) {
+  u32 na = a.n_pairs, nb = b.n_pairs;
+  if (a.n_pairs_dev) na = min(na, *a.n_pairs_dev);
+  if (b.n_pairs_dev) nb = min(nb, *b.n_pairs_dev);
+  const u32 lane = threadIdx.x & 31;
+  const u64 per_pair = (u64)a.n_chunks * tiles_per_chunk;
+  const u64 ia = (u64)na * per_pair, ib = (u64)nb * per_pair, both = 2 * min(ia, ib), n_items = ia + ib;
+  const u64 n_warps = (u64)gridDim.x * 8;
+  for (u64 item = (u64)blockIdx.x * 8 + (threadIdx.x >> 5); item < n_items; item += n_warps) {
+    bool from_b;
+    u64 k;
+    if (item < both) { from_b = item & 1; k = item >> 1; }
+    else { from_b = ib > ia; k = item - min(ia, ib); }
+    const MoveArgs &m = from_b ? b : a;
+    u32 pair = (u32)(k / per_pair);
+    u32 rem = (u32)(k - (u64)pair * per_pair);
+    u32 chunk = rem / tiles_per_chunk, tile = rem - chunk * tiles_per_chunk;
+    u32 s = m.src_ids[pair], d = m.dst_ids[pair];
+    if (s >= m.src.n_slots || d >= m.dst.n_slots) { if (lane == 0) set_err(m.status, DERR_RANGE); continue; }
+    const uint4 *sp = reinterpret_cast<const uint4 *>(m.src.base + s * m.src.slot_stride + chunk * m.src.chunk_stride) +
+                      (u64)tile * 32 * UNROLL + lane;
+    uint4 *dp = reinterpret_cast<uint4 *>(m.dst.base + d * m.dst.slot_stride + chunk * m.dst.chunk_stride) +
                 (u64)tile * 32 * UNROLL + lane;
     uint4 r[UNROLL];
 #pragma unroll

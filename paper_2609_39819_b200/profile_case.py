@@ -5,6 +5,7 @@ larger than L2, a few GB on the device at most, a handful of launches).
     python -m paper_2609_39819_b200.profile_case mover_toy  # the same with 16 KiB blocks (4 KiB chunks)
     python -m paper_2609_39819_b200.profile_case mover_host # the same blocks, HBM -> pinned host tier and back
     python -m paper_2609_39819_b200.profile_case hash_big   # stand-alone hasher on 64 Mi tokens (256 MiB > L2)
+    python -m paper_2609_39819_b200.profile_case exchange   # 1024 blocks each way over the host link: one call vs two
     python -m paper_2609_39819_b200.profile_case lookup     # hash + table lookup of 16 x 16,128-block calls
     python -m paper_2609_39819_b200.profile_case select     # classify + select 10% of 1 Mi resident blocks
     python -m paper_2609_39819_b200.profile_case c4         # the whole metadata stress at full size (C4)
@@ -98,6 +99,33 @@ def main(case: str):
         gb = n * geo.block_bytes / 1e9
         print(f"mover_host: {n} blocks x {geo.block_bytes} B; gather to host ms {g} = {[round(gb / (m / 1e3), 1) for m in g]} GB/s; "
               f"scatter from host ms {sc} = {[round(gb / (m / 1e3), 1) for m in sc]} GB/s")
+    elif case == "exchange":
+        geo, n = W.GEO_8B, 1024
+        eng = B.Engine(n_hbm_blocks=3 * n, n_host_blocks=3 * n, max_contexts=2, max_tokens=1 << 12, max_messages=64,
+                       max_batch_blocks=4 * n, zero_pools=False, **geo.kwargs())
+        ar = np.arange(n, dtype=np.uint32)
+        eng.debug_load_resident(ar + 1000, np.ones(n, np.uint8), ar, ar, ar, 0)            # n idle blocks in HBM
+        eng.debug_load_resident(ar + 100000, np.ones(n, np.uint8), ar, ar, ar, 1)          # n idle blocks on the host
+        gb = n * geo.block_bytes / 1e9
+
+        def lists():
+            return np.nonzero(eng.get_entries(0)["key"])[0], np.nonzero(eng.get_entries(1)["key"])[0]
+
+        res = {"exchange": [], "reload_then_offload": []}
+        for rep in range(4):
+            for mode in ("exchange", "reload_then_offload"):
+                out, inn = lists()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                if mode == "exchange":
+                    r = eng.exchange(out, inn)
+                else:
+                    r = (eng.reload(inn), eng.offload(out))
+                b.record(); torch.cuda.synchronize()
+                if rep:
+                    res[mode].append(round(a.elapsed_time(b), 2))
+        print(f"exchange: {n} blocks x {geo.block_bytes} B in each direction per call; ms {res}; "
+              f"GB/s both directions together { {k: [round(2 * gb / (m / 1e3), 1) for m in v] for k, v in res.items()} }")
     elif case == "hash_big":
         n_tok = 64 << 20
         tok = torch.randint(0, W.VOCAB, (n_tok,), dtype=torch.int32, device="cuda")

@@ -7,7 +7,7 @@ from paper_2609_39819_b200 import workloads as W
 HBM, HOST = 0, 1
 OPS = ("append", "append", "append", "replace", "remove", "one_off_ctx", "one_off_msg", "pin", "unpin", "fork", "spawn",
        "terminate", "call", "call", "call", "lookup_only", "admit_only", "prefill_done", "evict", "evict_pinned",
-       "release_hbm", "release_host", "reload_some", "compact_hbm", "compact_host", "bad")
+       "release_hbm", "release_host", "reload_some", "compact_hbm", "compact_host", "exchange", "exchange", "bad")
 
 
 def payload(key, nbytes):
@@ -192,6 +192,14 @@ class Fuzzer:
             if len(occ) and r.random() < 0.8:
                 slots = r.choice(occ, size=min(len(occ), int(r.integers(1, 6))), replace=False)
             self.all_rc(lambda e: e.reload(slots))
+        elif op == "exchange":
+            occ_h = np.nonzero(E.get_entries(HBM)["key"])[0]
+            occ_s = np.nonzero(E.get_entries(HOST)["key"])[0]
+            out = r.choice(occ_h, size=min(len(occ_h), int(r.integers(0, 5))), replace=False) if len(occ_h) else []
+            inn = r.choice(occ_s, size=min(len(occ_s), int(r.integers(0, 5))), replace=False) if len(occ_s) else []
+            if r.random() < 0.1:
+                out = list(out) + [int(r.integers(0, E.n_hbm_blocks + 2))]
+            self.all_rc(lambda e: e.exchange(out, inn))
         elif op in ("compact_hbm", "compact_host"):
             tier = HBM if op == "compact_hbm" else HOST
             self.all_rc(lambda e: e.compact(tier))

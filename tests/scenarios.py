@@ -312,6 +312,64 @@ def inclusive_tiers(make):
     assert (st["occ_hbm"], st["occ_host"]) == (0, 0)
 
 
+# ---- exchange: reload and offload in one call, destinations = slots free when the call begins ------------------
+def exchange_both_ways(make):
+    for flags in (0, 2):
+        eng = make(n_hbm_blocks=8, n_host_blocks=8, max_contexts=4, policy_flags=flags, **TOY)
+        rng = np.random.default_rng(19)
+        keys = {}
+        for c in (0, 1):
+            eng.spawn(c)
+            eng.append(c, toks(rng, 64))
+            call(eng, c)                                  # context 0: HBM slots 0..3, context 1: slots 4..7
+            k, _t, sl = eng.get_block_map(c)
+            keys[c] = k
+            for kk, s_ in zip(k, sl):
+                eng.write_block(HBM, int(s_), _payload(kk, eng.block_bytes))
+        assert eng.offload([7, 6]) == (0, 2, 0)           # context 1's blocks 3, 2 -> host slots 0, 1
+        # bring them back while pushing context 0's tail out: the incoming blocks take the HBM slots that are free
+        # now (6, 7), the outgoing ones the host slots that are free now (2, 3; 0 and 1 are still occupied)
+        assert eng.exchange([3, 2], [1, 0]) == (0, 2, 0, 2)
+        _k, t1, s1 = eng.get_block_map(1)
+        assert list(t1) == [HBM] * 4 and list(s1) == [4, 5, 6, 7]
+        _k, t0, s0 = eng.get_block_map(0)
+        assert list(t0) == [HBM, HBM, HOST, HOST] and list(s0) == [0, 1, 3, 2]
+        st = eng.get_stats()
+        assert (st["occ_hbm"], st["occ_host"]) == ((6, 2) if flags == 0 else (6, 4))   # inclusive keeps the copies
+        for c in (0, 1):
+            _k, t, sl = eng.get_block_map(c)
+            for b in range(4):
+                assert np.array_equal(eng.read_block(int(t[b]), int(sl[b])), _payload(keys[c][b], eng.block_bytes))
+        # second exchange: context 0's tail comes back into HBM slots 2, 3 while its block 0 goes out; the host
+        # slots 0, 1 are free again without inclusive tiers, and still hold clean copies with them
+        assert eng.exchange([0], [3, 2]) == (0, 1, 0, 2)
+        _k, t0, s0 = eng.get_block_map(0)
+        assert list(t0) == [HOST, HBM, HBM, HBM] and list(s0) == [0 if flags == 0 else 4, 1, 2, 3]
+        # validation covers both lists before anything moves
+        watch = ("occ_hbm", "occ_host", "offloaded", "reloaded", "dropped", "bytes_d2h", "bytes_h2d")
+        before = {k: eng.get_stats()[k] for k in watch}
+        assert eng.exchange([1, 1], [])[0] == E_INVAL and eng.exchange([], [7])[0] == E_INVAL
+        assert eng.exchange([9], [])[0] == E_RANGE and eng.exchange([1], [9])[0] == E_RANGE
+        assert {k: eng.get_stats()[k] for k in watch} == before
+        for c in (0, 1):
+            _k, t, sl = eng.get_block_map(c)
+            for b in range(4):
+                assert np.array_equal(eng.read_block(int(t[b]), int(sl[b])), _payload(keys[c][b], eng.block_bytes))
+    # more incoming blocks than free HBM slots: what fits is done, the rest is reported
+    eng = make(n_hbm_blocks=4, n_host_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(20)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 64))
+    call(eng, 0)
+    assert eng.offload([3, 2]) == (0, 2, 0)
+    eng.spawn(1)
+    eng.append(1, toks(rng, 16))
+    call(eng, 1)                                          # takes HBM slot 2; slot 3 is the only free one
+    assert eng.exchange([], [0, 1]) == (E_NOSPACE, 0, 0, 1)
+    assert list(eng.get_block_map(0)[2]) == [0, 1, 1, 3]  # block 3 came back to HBM slot 3, block 2 still at host slot 1
+    assert eng.exchange([], []) == (0, 0, 0, 0)
+
+
 # ---- hand-worked lifecycle example (8-block pool) --------------------------------------------------
 def worked_example(make):
     eng = make(n_hbm_blocks=8, n_host_blocks=8, max_contexts=4, **TOY)
@@ -660,4 +718,4 @@ def degenerate_inputs(make):
 ALL = [state_machine_single_context, suffix_invalidation, fork_and_shared_kv, one_off_bypass, worked_example,
        mixed_pool_example, victim_order_bruteforce, one_state_pools_reduce_to_lru, offload_reload_round_trip,
        dead_victims_are_dropped_without_copy, compaction, raw_copy_blocks, admission_stops_when_full,
-       lookup_locks_and_orphans, degenerate_inputs, pinned_retention, no_lifecycle_policy, inclusive_tiers]
+       lookup_locks_and_orphans, degenerate_inputs, pinned_retention, no_lifecycle_policy, inclusive_tiers, exchange_both_ways]
