@@ -540,7 +540,8 @@ int32_t kvt_set_profiling(kvt_engine *e, uint32_t on) {
 }
 
 int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant) {
-  if (!e || variant > 3) return KVT_E_INVAL;
+  if (!e) return KVT_E_INVAL;
+  if (variant > 3) return KVT_E_INVAL;
   e->mover_variant = variant;
   return KVT_OK;
 }
@@ -1258,7 +1259,7 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
       if (e->chunk_bytes % 4096 == 0) {
         u32 tpc = (u32)(e->chunk_bytes / 4096);
         u32 grid = (u32)std::min<u64>((items * tpc + 7) / 8, (u64)e->sm_count * 8);
-        KL(k_move_tiles_dual<8>, grid, 256, s, ma, mb, tpc);
+        KL(k_move_tiles_dual<8>, grid, 256, s, ma, mb, tpc, 2u);   // CTAs alternate between the two directions
       } else {   // chunk sizes the tile kernel cannot split: one direction after the other
         u32 g1 = (u32)std::min<u64>((u64)ma.n_pairs * e->n_chunks, (u64)e->sm_count * 8);
         u32 g2 = (u32)std::min<u64>((u64)mb.n_pairs * e->n_chunks, (u64)e->sm_count * 8);

@@ -1019,37 +1019,52 @@ __global__ void __launch_bounds__(256) k_move_tiles(MoveArgs a, u32 tiles_per_ch
   }
 }
 
-// Two independent pair lists in one launch (kvt_exchange): list a and list b alternate tile by tile while both
-// last, so that loads from and stores to the host tier are in flight at the same time (the link is full duplex).
+// Two independent pair lists in one launch (kvt_exchange): even CTAs work on list a, odd CTAs on list b (or all
+// CTAs on the one that has work), so that loads from and stores to the host tier are in flight at the same time
+// (the link is full duplex) and neither direction waits for the other's latency.
 template <int UNROLL>
-__global__ void __launch_bounds__(256) k_move_tiles_dual(MoveArgs a, MoveArgs b, u32 tiles_per_chunk) {
+__global__ void __launch_bounds__(256) k_move_tiles_dual(MoveArgs a, MoveArgs b, u32 tiles_per_chunk, u32 b_every) {
   u32 na = a.n_pairs, nb = b.n_pairs;
   if (a.n_pairs_dev) na = min(na, *a.n_pairs_dev);
   if (b.n_pairs_dev) nb = min(nb, *b.n_pairs_dev);
   const u32 lane = threadIdx.x & 31;
   const u64 per_pair = (u64)a.n_chunks * tiles_per_chunk;
-  const u64 ia = (u64)na * per_pair, ib = (u64)nb * per_pair, both = 2 * min(ia, ib), n_items = ia + ib;
-  const u64 n_warps = (u64)gridDim.x * 8;
-  for (u64 item = (u64)blockIdx.x * 8 + (threadIdx.x >> 5); item < n_items; item += n_warps) {
+  // CTA roles: with work on both sides and at least two CTAs the grid is split in two halves; otherwise every CTA
+  // serves list a and then list b
+  const bool split = na && nb && gridDim.x >= b_every;
+  for (int pass = 0; pass < 2; ++pass) {
     bool from_b;
-    u64 k;
-    if (item < both) { from_b = item & 1; k = item >> 1; }
-    else { from_b = ib > ia; k = item - min(ia, ib); }
+    u32 my_cta, n_cta;
+    if (split) {
+      if (pass) break;
+      // every b_every-th CTA serves list b, the others list a
+      const u32 q = blockIdx.x / b_every, rmd = blockIdx.x % b_every;
+      from_b = rmd == b_every - 1;
+      const u32 n_b = gridDim.x / b_every, n_a = gridDim.x - n_b;
+      my_cta = from_b ? q : q * (b_every - 1) + rmd;
+      n_cta = from_b ? n_b : n_a;
+    } else {
+      from_b = pass; my_cta = blockIdx.x; n_cta = gridDim.x;
+    }
     const MoveArgs &m = from_b ? b : a;
-    u32 pair = (u32)(k / per_pair);
-    u32 rem = (u32)(k - (u64)pair * per_pair);
-    u32 chunk = rem / tiles_per_chunk, tile = rem - chunk * tiles_per_chunk;
-    u32 s = m.src_ids[pair], d = m.dst_ids[pair];
-    if (s >= m.src.n_slots || d >= m.dst.n_slots) { if (lane == 0) set_err(m.status, DERR_RANGE); continue; }
-    const uint4 *sp = reinterpret_cast<const uint4 *>(m.src.base + s * m.src.slot_stride + chunk * m.src.chunk_stride) +
-                      (u64)tile * 32 * UNROLL + lane;
-    uint4 *dp = reinterpret_cast<uint4 *>(m.dst.base + d * m.dst.slot_stride + chunk * m.dst.chunk_stride) +
-                (u64)tile * 32 * UNROLL + lane;
-    uint4 r[UNROLL];
+    const u64 n_items = (u64)(from_b ? nb : na) * per_pair;
+    const u64 n_warps = (u64)n_cta * 8;
+    for (u64 k = (u64)my_cta * 8 + (threadIdx.x >> 5); k < n_items; k += n_warps) {
+      u32 pair = (u32)(k / per_pair);
+      u32 rem = (u32)(k - (u64)pair * per_pair);
+      u32 chunk = rem / tiles_per_chunk, tile = rem - chunk * tiles_per_chunk;
+      u32 s = m.src_ids[pair], d = m.dst_ids[pair];
+      if (s >= m.src.n_slots || d >= m.dst.n_slots) { if (lane == 0) set_err(m.status, DERR_RANGE); continue; }
+      const uint4 *sp = reinterpret_cast<const uint4 *>(m.src.base + s * m.src.slot_stride + chunk * m.src.chunk_stride) +
+                        (u64)tile * 32 * UNROLL + lane;
+      uint4 *dp = reinterpret_cast<uint4 *>(m.dst.base + d * m.dst.slot_stride + chunk * m.dst.chunk_stride) +
+                  (u64)tile * 32 * UNROLL + lane;
+      uint4 r[UNROLL];
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) r[u] = __ldcs(sp + u * 32);
+      for (int u = 0; u < UNROLL; ++u) r[u] = __ldcs(sp + u * 32);
 #pragma unroll
-    for (int u = 0; u < UNROLL; ++u) __stcs(dp + u * 32, r[u]);
+      for (int u = 0; u < UNROLL; ++u) __stcs(dp + u * 32, r[u]);
+    }
   }
 }
 
