@@ -616,7 +616,7 @@ def main():
     achieved = 2 * st["mover_bytes"] / mover_s / 1e9 if mover_s else 0.0
     per_launch_bytes = 2 * st["mover_bytes"] / max(st["mover_launches"], 1)
     roofline = {
-        "bound": "hbm", "kernel": "k_move_blocks", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
+        "bound": "hbm", "kernel": "k_move_tiles<8>", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
         "frac": achieved / hbm_peak, "peak_kind": f"{peak_kind} copy bandwidth (MEASURED_PEAKS.json hbm_gbs)",
         "frac_of_nominal_8TBs": achieved / 8000.0, "torch_copy_gbs_this_run": hbm_now,
         "launches": st["mover_launches"], "avg_launch_ms": mover_s * 1e3 / max(st["mover_launches"], 1),

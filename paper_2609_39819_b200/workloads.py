@@ -295,13 +295,16 @@ class ReplayOptions:
     writer: object = None         # callable(engine, slot, key): writes a new HBM block's payload in place (large blocks)
     record_states: bool = True    # record per-tier states / entries after every call (slow on big pools)
     verify_payload_every: int = 0 # every k-th call, read back every occupied slot and compare with payload(key)
+    use_exchange: bool = False    # a call's reloads and the offloads that make room for them go out as one exchange
     counters: dict = field(default_factory=dict)
 
 
-def evict(eng, n, n_pinned_incoming=0):
+def evict(eng, n, n_pinned_incoming=0, reload_slots=None):
     """Frees n HBM slots in the engine's victim order: dead blocks are dropped, live ones go to the
     host tier, for which room is made first by releasing the host tier's own first victims. Pinned
-    blocks are only asked for when Pinned blocks are coming in, and only for as many (Algorithm 1)."""
+    blocks are only asked for when Pinned blocks are coming in, and only for as many (Algorithm 1).
+    With `reload_slots` (host slots the caller wants back in HBM) the offload and that reload are issued
+    together."""
     rec = {}
     victims, vstates = eng.select_victims(TIER_HBM, n)
     if len(victims) < n and n_pinned_incoming > 0:
@@ -318,7 +321,13 @@ def evict(eng, n, n_pinned_incoming=0):
         rec["host_vstates"] = hs.copy()
         if len(hv):
             eng.release(TIER_HOST, hv)
-    if len(victims):
+    if reload_slots is not None and len(reload_slots):
+        # both directions in one call; what found no free HBM slot at the start follows once the offload has made room
+        rc, n_out, n_drop, n_in = eng.exchange(victims, reload_slots)
+        rec["exchange"] = (rc, n_out, n_drop, n_in)
+        if n_in < len(reload_slots):
+            rec["reload"] = eng.reload(reload_slots[n_in:])
+    elif len(victims):
         rec["offload"] = eng.offload(victims)
     return rec
 
@@ -333,18 +342,23 @@ def run_call(eng, ctxs, opt: ReplayOptions):
     st = eng.get_stats()
     free_hbm = eng.n_hbm_blocks - st["occ_hbm"]
     need = int(info["n_hit_host"].sum()) + int(info["n_admissible"].sum()) - free_hbm
-    if need > 0:
-        rec.update(evict(eng, need, int(info["n_pinned"].sum())))
     host_slots = []
     for c, inf in zip(ctxs, info):
         if inf["n_hit_host"]:
             _keys, tier, slot = eng.get_block_map(c)
             h = int(inf["hit_len"])
             host_slots.append(slot[:h][tier[:h] == TIER_HOST])
+    hs = None
     if host_slots:
         hs = np.concatenate(host_slots)
         hs = hs[np.sort(np.unique(hs, return_index=True)[1])]  # a shared host block is reloaded once
-        rec["reload"] = eng.reload(hs)
+    if need > 0 and opt.use_exchange and hs is not None:
+        rec.update(evict(eng, need, int(info["n_pinned"].sum()), reload_slots=hs))
+    else:
+        if need > 0:
+            rec.update(evict(eng, need, int(info["n_pinned"].sum())))
+        if hs is not None:
+            rec["reload"] = eng.reload(hs)
     adm = eng.map_blocks(ctxs, MAP_ADMIT)
     rec["admit"] = adm.copy()
     maps = []

@@ -75,9 +75,11 @@ def test_hash_full_size_batch_matches_oracle(B, oracle):
 
 
 # ---- whole path on C1 traces: every reported value and every payload byte ----------------------------
-def _replay_pair(gpu, cpu, trace, payload, check_pools=True, record_states=True, verify_every=0):
-    og = W.ReplayOptions(payload=payload, record_states=record_states, verify_payload_every=verify_every)
-    oc = W.ReplayOptions(payload=payload, record_states=record_states, verify_payload_every=verify_every)
+def _replay_pair(gpu, cpu, trace, payload, check_pools=True, record_states=True, verify_every=0, use_exchange=False):
+    og = W.ReplayOptions(payload=payload, record_states=record_states, verify_payload_every=verify_every,
+                         use_exchange=use_exchange)
+    oc = W.ReplayOptions(payload=payload, record_states=record_states, verify_payload_every=verify_every,
+                         use_exchange=use_exchange)
     n_calls = 0
     for (i, kind, rg), (_, _, rc) in zip(W.replay(gpu, trace, og), W.replay(cpu, trace, oc)):
         if kind == "call":
@@ -160,6 +162,34 @@ def test_trace_parity_with_inclusive_tiers(B, oracle, flags):
         for k in ec:
             assert np.array_equal(eg[k], ec[k]), (tier, k)
         assert np.array_equal(gpu.get_states(tier), cpu.get_states(tier))
+
+
+@pytest.mark.parametrize("flags", [0, 2])
+def test_trace_parity_with_exchange_calls(B, oracle, flags):
+    """The replay driver in exchange mode: a call's reloads and the offloads that make room for them are one
+    kvt_exchange (both directions in one mover launch), the rest of the reload follows. Every reported value,
+    every state and every payload byte matches the oracle's exchange."""
+    n_x = 0
+    for seed in (7, 63, 86):
+        kw = dict(n_hbm_blocks=96, n_host_blocks=256, max_contexts=64, policy_flags=flags, **W.GEO_TOY.kwargs())
+        gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)
+        cpu = oracle.OracleEngine(**kw)
+        _replay_pair(gpu, cpu, W.trace_c1(seed), W.payload_pattern, verify_every=1, use_exchange=True)
+    trace, n_ctx = W.trace_c3(1, n_sessions=8, scale=1 / 32)
+    kw = dict(n_hbm_blocks=256, n_host_blocks=320, max_contexts=n_ctx, policy_flags=flags, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 20, max_messages=1 << 15, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    og = W.ReplayOptions(payload=W.payload_pattern, verify_payload_every=5, use_exchange=True)
+    oc = W.ReplayOptions(payload=W.payload_pattern, verify_payload_every=5, use_exchange=True)
+    for (i, kind, rg), (_, _, rc) in zip(W.replay(gpu, trace, og), W.replay(cpu, trace, oc)):
+        if kind == "call":
+            n_x += "exchange" in rc
+            diff = W.records_equal(rg, rc, f"event[{i}]")
+            assert diff is None, diff
+            assert rg.get("payload_ok", True) and rc.get("payload_ok", True)
+    assert n_x > 0
+    sg, sc = gpu.get_stats(), cpu.get_stats()
+    assert all(sg[k] == sc[k] for k in sc if k not in W.GPU_ONLY_STATS)
 
 
 def test_scaled_c2_trace_parity(B, oracle):

@@ -102,6 +102,31 @@ def test_scaled_c2_and_c3_traces_replay(make):
     assert int((eng.get_states(0) == 3).sum() + (eng.get_states(1) == 3).sum()) == 0
 
 
+@pytest.mark.parametrize("flags", [0, 2])
+def test_replay_with_exchange_moves_the_same_blocks(make, flags):
+    """The driver's exchange mode (reloads and the offloads that make room for them in one call) changes which slots
+    blocks land in, not which blocks move: hit counts, admissions and the set of resident keys equal those of the
+    separate offload + reload calls, and every payload byte survives."""
+    trace, n_ctx = W.trace_c3(1, n_sessions=8, scale=1 / 32)
+    out = []
+    for use in (False, True):
+        eng = make(n_hbm_blocks=256, n_host_blocks=320, max_contexts=n_ctx, policy_flags=flags, **W.GEO_TOY.kwargs())
+        opt = W.ReplayOptions(payload=W.payload_pattern, record_states=False, verify_payload_every=9, use_exchange=use)
+        n_x = 0
+        for _i, kind, rec in W.replay(eng, trace, opt):
+            if kind == "call":
+                n_x += "exchange" in rec
+                assert rec.get("payload_ok", True)
+        check_invariants(eng) if not flags else None
+        assert W.verify_payload(eng, W.payload_pattern)
+        st = eng.get_stats()
+        keys = [np.sort(eng.get_entries(t)["key"][eng.get_states(t) < 0xFE]) for t in (0, 1)]
+        out.append((n_x, {k: st[k] for k in ("hits_hbm", "hits_host", "misses", "inserted", "reloaded", "occ_hbm")}, keys))
+    assert out[0][0] == 0 and out[1][0] > 0
+    assert out[0][1] == out[1][1]
+    assert np.array_equal(out[0][2][0], out[1][2][0]) and np.array_equal(out[0][2][1], out[1][2][1])
+
+
 def test_incremental_appends_hash_like_one_shot(make, oracle):
     """Hashing a context after piecewise appends equals hashing the concatenation in one shot."""
     rng = np.random.default_rng(21)
