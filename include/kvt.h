@@ -82,6 +82,13 @@ extern "C" {
                                        kvt_offload of that block hands it back to the copy without moving a byte.
                                        Copies occupy host slots, are the first victims of the host tier (state
                                        KVT_STATE_COPY), can be released on their own, and go away with their block. */
+#define KVT_POLICY_ORPHANS_DEAD 4u   /* reachability-aware classification. A lookup reuses a contiguous prefix of a
+                                       context's chain (Section 2.1: prefix-dependent validity), so a resident block
+                                       behind a block that is no longer resident in any tier can never be hit again
+                                       through that context. With this flag a context's mappings stop counting at
+                                       its first non-resident block; a block that no context reaches any more
+                                       classifies as dead, becomes a first victim and is dropped, not copied. The
+                                       paper is silent on such orphans; without the flag they keep their state. */
 
 /* Primitives and runtime events (Table 3; Section 5.2 "Runtime transitions"). */
 #define KVT_OP_SPAWN         1u  /* register an independent, empty context */

@@ -44,6 +44,7 @@ enum : uint32_t { LAYOUT_LAYER_MAJOR = 0, LAYOUT_BLOCK_MAJOR = 1 };
 enum : uint32_t { ORDER_MRU = 0, ORDER_LRU = 1 };
 enum : uint32_t {
   POLICY_NO_LIFECYCLE = 1,   // the "w/o LT" variant of Section 8.3
+  POLICY_ORPHANS_DEAD = 4,   // a context's mappings stop counting at its first non-resident block
   POLICY_INCLUSIVE = 2       // a reloaded block keeps its host copy (Section 7: per-tier caching keeps a fast copy)
 };
 enum : uint32_t {
@@ -229,7 +230,10 @@ void classify(Engine &e, std::vector<uint8_t> rank[2]) {
     block_ranks(c, c.mat_bounds, c.valid_blocks, br);
     for (uint32_t b = 0; b < c.valid_blocks; ++b) {
       auto it = e.where.find(c.mat_keys[b]);
-      if (it == e.where.end()) continue;
+      if (it == e.where.end()) {
+        if (e.cfg.policy_flags & POLICY_ORPHANS_DEAD) break;   // nothing behind a missing block is reachable
+        continue;
+      }
       uint8_t &r = rank[it->second.first][it->second.second];
       if (br[b] > r) r = br[b];
     }
@@ -263,7 +267,7 @@ extern "C" {
 int32_t kvto_create(const Config *cfg, Engine **out) {
   if (!cfg || !out) return E_INVAL;
   if (!cfg->n_layers || !cfg->n_kv_heads || !cfg->head_dim || !cfg->elem_bytes || !cfg->n_hbm_blocks ||
-      !cfg->max_contexts || cfg->pool_layout > 1 || cfg->suspended_order > 1 || cfg->policy_flags > 3)
+      !cfg->max_contexts || cfg->pool_layout > 1 || cfg->suspended_order > 1 || cfg->policy_flags > 7)
     return E_INVAL;
   Engine *e = new Engine();
   e->cfg = *cfg;
@@ -557,6 +561,11 @@ int32_t kvto_classify_bruteforce(Engine *e, uint32_t tier, uint8_t *state, uint3
       hash_blocks(e->hp, c.mat_tokens.data(), c.mat_tokens.size(), keys);
       for (uint32_t b = 0; b < c.valid_blocks; ++b) {
         if (keys[b] != x.key) continue;
+        if (e->cfg.policy_flags & POLICY_ORPHANS_DEAD) {   // reachable: every block of the prefix is resident
+          bool reach = true;
+          for (uint32_t p = 0; p < b && reach; ++p) reach = e->where.count(keys[p]) != 0;
+          if (!reach) continue;
+        }
         for (size_t j = 0; j < c.mat_bounds.size(); ++j) {
           uint32_t lo = std::max<uint32_t>(c.mat_bounds[j].first, 16 * b);
           uint32_t hi = std::min<uint32_t>(c.mat_bounds[j].second, 16 * b + 16);

@@ -362,6 +362,12 @@ int32_t do_classify(kvt_engine *e, cudaStream_t s) {
     a.tab = e->tab; a.ent = e->ent; a.keys = e->d_keys; a.ctx = e->dp<ClsCtx>(e->L.desc); a.n_ctx = nc; a.n_map = nmap;
     a.m_start = e->dp<u32>(e->L.m_start); a.m_end = e->dp<u32>(e->L.m_end); a.m_rank = e->dp<u8>(e->L.m_rank);
     a.status = e->d_status;
+    a.first_miss = nullptr;
+    if (e->cfg.policy_flags & KVT_POLICY_ORPHANS_DEAD) {
+      a.first_miss = e->dp<u32>(e->L.ctxres);   // per-call scratch of the lookup, free between calls (stream order)
+      CU(cudaMemsetAsync(a.first_miss, 0xFF, nc * 4ull, s));
+      KL(k_first_miss, cdiv(nmap,256), 256, s, a);
+    }
     KL(k_classify, cdiv(nmap,256), 256, s, a);
     r = stage_release(e, s);
     if (r) return r;
@@ -449,7 +455,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   const kvt_config &c = *cfg;
   if (c.abi_version != KVT_ABI_VERSION || c.block_tokens != 16 || !c.n_layers || !c.n_kv_heads || !c.head_dim ||
       !c.elem_bytes || c.pool_layout > 1 || !c.n_hbm_blocks || !c.max_contexts || !c.max_batch_blocks ||
-      !c.max_messages || c.suspended_order > 1 || c.policy_flags > 3 || c.reserved1 || !c.dev_meta || !c.dev_tokens)
+      !c.max_messages || c.suspended_order > 1 || c.policy_flags > 7 || c.reserved1 || !c.dev_meta || !c.dev_tokens)
     return KVT_E_INVAL;
   u64 N = (u64)c.n_hbm_blocks + c.n_host_blocks;
   if (N >= CLAIM_BIT || c.max_batch_blocks >= CLAIM_BIT) return KVT_E_INVAL;
@@ -1160,6 +1166,7 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
   e->occ[KVT_TIER_HOST] -= e->h_status[ST_NSHDROP];
   e->tombs += e->h_status[ST_TOMBS];
   e->st.dropped += out->dropped;
+  if (out->dropped && (e->cfg.policy_flags & KVT_POLICY_ORPHANS_DEAD)) e->dirty = true;   // reachability changed
   r = maybe_rebuild(e, s);
   if (r) return r;
   return out->done < n ? KVT_E_NOSPACE : KVT_OK;
@@ -1287,6 +1294,7 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
   e->occ[KVT_TIER_HOST] -= h[ST_B_NSHDROP];
   e->tombs += h[ST_TOMBS];
   e->st.dropped += out_drop;
+  if (out_drop && (e->cfg.policy_flags & KVT_POLICY_ORPHANS_DEAD)) e->dirty = true;   // reachability changed
   e->st.reloaded += in_copied; e->st.bytes_h2d += in_copied * e->block_bytes;
   e->st.offloaded += out_copied + out_clean; e->st.offloaded_clean += out_clean; e->st.bytes_d2h += out_copied * e->block_bytes;
   r = maybe_rebuild(e, s);

@@ -566,11 +566,24 @@ struct ClsCtx { u64 key_off; u32 map_base; u32 valid; u32 msg_base; u32 n_msgs; 
 struct ClsArgs {
   Table tab; Entries ent; const u64 *keys; const ClsCtx *ctx; u32 n_ctx; u32 n_map;
   const u32 *m_start, *m_end; const u8 *m_rank; u32 *status;
+  u32 *first_miss;   // per listed context: index of its first non-resident block; nullptr = orphans keep their state
 };
 
 __global__ void k_rank_reset(Entries en) {
   u32 e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e < en.n_total) en.rank[e] = en.floor[e];
+}
+
+// Reachability pre-pass: the first block of every context's mapped prefix that is resident in no tier. A lookup
+// stops there, so the blocks behind it cannot be reused through this context.
+__global__ void k_first_miss(ClsArgs a) {
+  u32 g = blockIdx.x * blockDim.x + threadIdx.x;
+  if (g >= a.n_map) return;
+  u32 lo = 0, hi = a.n_ctx;
+  while (hi - lo > 1) { u32 mid = (lo + hi) >> 1; if (a.ctx[mid].map_base <= g) lo = mid; else hi = mid; }
+  const ClsCtx c = a.ctx[lo];
+  const u32 b = g - c.map_base;
+  if (tab_find(a.tab, a.keys[c.key_off + b], a.status) == ENT_NONE) atomicMin(&a.first_miss[lo], b);
 }
 
 __global__ void k_classify(ClsArgs a) {
@@ -580,6 +593,7 @@ __global__ void k_classify(ClsArgs a) {
   while (hi - lo > 1) { u32 mid = (lo + hi) >> 1; if (a.ctx[mid].map_base <= g) lo = mid; else hi = mid; }
   const ClsCtx c = a.ctx[lo];
   const u32 b = g - c.map_base;
+  if (a.first_miss && b >= a.first_miss[lo]) return;   // behind a missing block: unreachable through this context
   const u32 t0 = b * 16, t1 = t0 + 16;
   const u32 *ms = a.m_start + c.msg_base, *me = a.m_end + c.msg_base;
   const u8 *mr = a.m_rank + c.msg_base;
@@ -1071,7 +1085,7 @@ __global__ void __launch_bounds__(256) k_move_tiles_dual(MoveArgs a, MoveArgs b,
 // ------------------------------------------------------------------------------------------------------
 // TMA variant: one elected thread per CTA drives a ring of shared-memory stages with untiled bulk copies
 // (cp.async.bulk global -> shared, completion on an mbarrier; shared -> global as a bulk group). No registers
-// carry payload; every wait is bounded and reports through the status word. No multicast, no clusters.
+// carry payload; every wait is bounded and reports through the status word. Every copy is CTA-local: one source, one destination, no clusters.
 // ------------------------------------------------------------------------------------------------------
 constexpr int TMA_STAGES = 4;
 constexpr u32 TMA_WAIT_LIMIT = 1u << 20;

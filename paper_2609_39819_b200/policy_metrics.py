@@ -20,6 +20,7 @@ POLICIES = {                      # name -> (suspended_order, policy_flags)
     "w/o RO (lifecycle + LRU)": (1, 0),
     "w/o LT (MRU only)": (0, 1),
     "no lifecycle + LRU": (1, 1),
+    "lifecycle + MRU, unreachable blocks dead": (0, 4),
 }
 
 

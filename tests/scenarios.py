@@ -715,7 +715,42 @@ def degenerate_inputs(make):
     assert len(keys) == 1
 
 
+# ---- reachability-aware classification: blocks behind a missing prefix block are dead ----------------
+def orphans_are_dead(make):
+    for flags in (0, 4):
+        eng = make(n_hbm_blocks=12, n_host_blocks=4, max_contexts=4, policy_flags=flags, **TOY)
+        rng = np.random.default_rng(21)
+        eng.spawn(0)
+        eng.append(0, toks(rng, 96))                     # 6 blocks at slots 0..5
+        call(eng, 0)
+        eng.fork(0, 1, 1)                                # the child shares all six and adds two of its own (6, 7)
+        eng.append(1, toks(rng, 32))
+        call(eng, 1)
+        eng.pin(1, 1, 2)                                 # the child's own message is pinned
+        assert states(eng)[:8] == [IDLE] * 6 + [PINNED] * 2
+        assert eng.offload([1]) == (0, 1, 0)             # a block on the host tier still counts as present
+        assert states(eng)[:8] == [IDLE, FREE] + [IDLE] * 4 + [PINNED] * 2 and states(eng, HOST)[0] == IDLE
+        eng.release(HBM, [2])                            # block 2 is gone from every tier
+        want = [IDLE, FREE, FREE] + ([DEAD] * 5 if flags else [IDLE] * 3 + [PINNED] * 2)
+        assert states(eng)[:8] == want                   # pinned or not: nothing behind the hole can be hit again
+        v, s = eng.select_victims(HBM, 5)
+        if flags:
+            assert list(v) == [7, 6, 5, 4, 3] and list(s) == [DEAD] * 5      # first victims, deepest first
+            assert eng.offload(v[:2]) == (0, 2, 2)       # and dropped, not copied
+        else:
+            assert list(s) == [IDLE] * 4 and set(v) == {0, 3, 4, 5}
+        # the parent's next call re-creates block 2 and adopts what is still there: everything is reachable again
+        a = eng.map_blocks([0], LOOKUP)[0]
+        assert (a["hit_len"], a["n_hit_hbm"], a["n_hit_host"]) == (2, 1, 1)
+        assert states(eng)[:6] == [ACTIVE, FREE, FREE] + ([DEAD] * 3 if flags else [ACTIVE] * 3)
+        b = eng.map_blocks([0], ADMIT)[0]
+        assert (b["n_admitted"], b["n_held"]) == (4, 6)
+        assert states(eng)[:6] == [ACTIVE, ACTIVE, FREE] + [ACTIVE] * 3     # block 2 re-created at the lowest free slot (1)
+        eng.prefill_done(0)
+
+
 ALL = [state_machine_single_context, suffix_invalidation, fork_and_shared_kv, one_off_bypass, worked_example,
        mixed_pool_example, victim_order_bruteforce, one_state_pools_reduce_to_lru, offload_reload_round_trip,
        dead_victims_are_dropped_without_copy, compaction, raw_copy_blocks, admission_stops_when_full,
-       lookup_locks_and_orphans, degenerate_inputs, pinned_retention, no_lifecycle_policy, inclusive_tiers, exchange_both_ways]
+       lookup_locks_and_orphans, degenerate_inputs, pinned_retention, no_lifecycle_policy, inclusive_tiers, exchange_both_ways,
+       orphans_are_dead]

@@ -10,7 +10,7 @@ pytestmark = pytest.mark.gpu
 
 
 @pytest.mark.parametrize("seed", range(24))
-@pytest.mark.parametrize("flags", [0, 1, 2, 3])
+@pytest.mark.parametrize("flags", [0, 1, 2, 3, 4, 7])
 @pytest.mark.parametrize("pools", [(24, 16), (8, 4), (40, 0)], ids=lambda p: f"hbm{p[0]}-host{p[1]}")
 def test_random_api_streams_match_the_oracle(oracle, seed, flags, pools):
     import torch

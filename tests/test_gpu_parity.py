@@ -192,6 +192,35 @@ def test_trace_parity_with_exchange_calls(B, oracle, flags):
     assert all(sg[k] == sc[k] for k in sc if k not in W.GPU_ONLY_STATS)
 
 
+@pytest.mark.parametrize("flags", [4, 6])
+def test_trace_parity_with_unreachable_blocks_dead(B, oracle, flags):
+    """Reachability-aware classification: a small host tier forces drops of live prefixes, the blocks behind them
+    classify as dead on both sides, are the first victims and are dropped without a copy."""
+    for seed in (7, 63, 86):
+        kw = dict(n_hbm_blocks=96, n_host_blocks=48, max_contexts=64, policy_flags=flags, **W.GEO_TOY.kwargs())
+        gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)
+        cpu = oracle.OracleEngine(**kw)
+        _replay_pair(gpu, cpu, W.trace_c1(seed), W.payload_pattern, verify_every=1)
+    trace, n_ctx = W.trace_c3(1, n_sessions=8, scale=1 / 32)
+    kw = dict(n_hbm_blocks=256, n_host_blocks=96, max_contexts=n_ctx, policy_flags=flags, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 20, max_messages=1 << 15, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    # stop in mid-trace (sessions alive), punch holes into the chains, compare the reclassification
+    _replay_pair(gpu, cpu, trace[:2 * len(trace) // 3], W.payload_pattern, verify_every=5)
+    before = cpu.get_states(0).copy()
+    ent = cpu.get_entries(0)
+    holes = [int(x) for x in np.nonzero((ent["key"] != 0) & (ent["inflight"] == 0) & (ent["depth"] % 7 == 3))[0][:12]]
+    assert holes
+    for eng in (gpu, cpu):
+        eng.release(0, holes)
+    after = cpu.get_states(0)
+    assert int(((before > 0) & (before < 0xFE) & (after == 0)).sum()) > 0     # orphans appeared
+    for tier in (0, 1):
+        assert np.array_equal(gpu.get_states(tier), cpu.get_states(tier))
+    vg, vc = gpu.select_victims(0, 64), cpu.select_victims(0, 64)
+    assert np.array_equal(vg[0], vc[0]) and np.array_equal(vg[1], vc[1])
+
+
 def test_scaled_c2_trace_parity(B, oracle):
     kw = dict(n_hbm_blocks=96, n_host_blocks=64, max_contexts=8, **W.GEO_TOY.kwargs())
     gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)

@@ -7,7 +7,7 @@ from paper_2609_39819_b200 import workloads as W
 
 
 @pytest.mark.parametrize("seed", range(8))
-@pytest.mark.parametrize("flags", [0, 1, 2, 3])
+@pytest.mark.parametrize("flags", [0, 1, 2, 3, 4, 6])
 @pytest.mark.parametrize("pools", [(24, 16), (8, 4), (40, 0)], ids=lambda p: f"hbm{p[0]}-host{p[1]}")
 def test_oracle_survives_random_api_streams(oracle, seed, flags, pools):
     eng = oracle.OracleEngine(n_hbm_blocks=pools[0], n_host_blocks=pools[1], max_contexts=6, policy_flags=flags,
