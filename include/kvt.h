@@ -373,6 +373,12 @@ int32_t kvt_set_profiling(kvt_engine *e, uint32_t on);
  * multiple of 16 KiB). Results are identical. */
 int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant);
 
+/* Tuning hook: how kvt_map_blocks(LOOKUP) hashes and probes. 0 / 1 = three kernels (digest, carry scan, finish +
+ * probe; default), 2 = one single-pass kernel in which chunks hand their chain values forward through device
+ * memory (bounded waits; a wait that runs out makes the call return KVT_E_DEVICE). Results are identical; the
+ * single pass measured slower on B200 (its CTAs live too long to keep enough token bytes in flight). */
+int32_t kvt_debug_set_lookup_variant(kvt_engine *e, uint32_t variant);
+
 /* Text of the last error of this engine (always NUL-terminated). */
 int32_t kvt_last_error(kvt_engine *e, char *buf, uint32_t cap);
 

@@ -16,7 +16,7 @@ OK, E_INVAL, E_NOCTX, E_RANGE, E_STATE, E_NOSPACE, E_BUFSZ, E_DEVICE, E_CUDA = 0
 TIER_HBM, TIER_HOST, TIER_NONE = 0, 1, 0xFF
 LAYOUT_LAYER_MAJOR, LAYOUT_BLOCK_MAJOR = 0, 1
 ORDER_MRU, ORDER_LRU = 0, 1
-POLICY_NO_LIFECYCLE, POLICY_INCLUSIVE = 1, 2
+POLICY_NO_LIFECYCLE, POLICY_INCLUSIVE, POLICY_ORPHANS_DEAD = 1, 2, 4
 (OP_SPAWN, OP_FORK, OP_APPEND, OP_REPLACE, OP_REMOVE, OP_ONE_OFF, OP_PREFILL_DONE, OP_TERMINATE,
  OP_PIN, OP_UNPIN) = range(1, 11)
 OPF_TOKENS_ON_DEVICE = 1
@@ -27,7 +27,7 @@ EXPORTS = ("kvt_query_sizes", "kvt_create", "kvt_destroy", "kvt_apply_op", "kvt_
            "kvt_classify", "kvt_get_states", "kvt_select_victims", "kvt_offload", "kvt_reload", "kvt_release",
            "kvt_compact", "kvt_copy_blocks", "kvt_hash_scratch_bytes", "kvt_hash_tokens", "kvt_get_stats",
            "kvt_last_error", "kvt_get_entries", "kvt_debug_load_resident", "kvt_set_profiling",
-           "kvt_hash_tokens_noalloc", "kvt_debug_set_mover_variant", "kvt_exchange")
+           "kvt_hash_tokens_noalloc", "kvt_debug_set_mover_variant", "kvt_exchange", "kvt_debug_set_lookup_variant")
 
 
 class KvtError(RuntimeError):
@@ -100,6 +100,7 @@ def load_library():
             "kvt_last_error": [vp, vp, u32],
             "kvt_set_profiling": [vp, u32],
             "kvt_debug_set_mover_variant": [vp, u32],
+            "kvt_debug_set_lookup_variant": [vp, u32],
             "kvt_get_entries": [vp, u32, vp, vp, vp, vp, vp, u32, vp],
             "kvt_debug_load_resident": [vp, vp, vp, vp, vp, vp, u32, u32, vp],
         }
@@ -236,6 +237,9 @@ class Engine:
 
     def set_mover_variant(self, variant):
         self._check(self.L.kvt_debug_set_mover_variant(self.h, variant), "set_mover_variant")
+
+    def set_lookup_variant(self, variant):
+        self._check(self.L.kvt_debug_set_lookup_variant(self.h, variant), "set_lookup_variant")
 
     def last_error(self):
         buf = C.create_string_buffer(256)

@@ -76,7 +76,7 @@ struct Ctx {
 
 struct DevLayout {
   u64 tab, e_key, e_stamp, e_depth, e_infl, e_rank, e_tslot, e_mark, e_link, e_floor, keys, status;
-  u64 s0, s1, s2, s3, ids, ids2, pair_src, pair_dst, pair_src2, pair_dst2, freelist, freelist2, tiles, agg, carry, desc, ctxres;
+  u64 s0, s1, s2, s3, ids, ids2, pair_src, pair_dst, pair_src2, pair_dst2, freelist, freelist2, tiles, agg, carry, cflags, desc, ctxres;
   u64 m_start, m_end, m_rank, keyA, keyB, valA, valB, rcounts, out_slots, out_states, map_tier, map_slot;
   u64 total;
   u64 LB, Nt, N;
@@ -99,7 +99,8 @@ DevLayout make_layout(const kvt_config &c) {
   L.freelist = take(LB * 4); L.freelist2 = take(LB * 4); L.pair_src2 = take(LB * 4); L.pair_dst2 = take(LB * 4);
   L.tiles = take((std::max(LB, N) / SCAN_TILE + 2) * 4);
   u64 n_chunks = B / CHUNK + C + 1;
-  L.agg = take(n_chunks * 8); L.carry = take(n_chunks * 8);
+  L.agg = take(n_chunks * 8); L.carry = take(n_chunks * 8);   // per-chunk aggregates / chain values of a LOOKUP batch
+  L.cflags = take((n_chunks + 1) * 4);                         // per-chunk publication flags + the ticket word
   L.desc = take(C * 64);
   L.ctxres = take(C * 16);
   L.m_start = take(Mm * 4); L.m_end = take(Mm * 4); L.m_rank = take(Mm);
@@ -148,6 +149,7 @@ struct kvt_engine {
   cudaStream_t capture_stream = nullptr;   // only ever used for stream capture, never executes work
   bool use_graphs = true;
   u32 mover_variant = 0;   // 0 auto, 1 CTA per chunk, 2 warp per 4 KiB tile, 3 TMA ring
+  u32 lookup_variant = 0;  // 0 / 1 digest / carry / finish kernels, 2 single-pass hash + probe kernel
   bool tma_attr_set = false;
   cudaEvent_t ev_m0 = nullptr, ev_m1 = nullptr, ev_h0 = nullptr, ev_h1 = nullptr;
 
@@ -207,6 +209,7 @@ int32_t status_fetch(kvt_engine *e, cudaStream_t s) {
 int32_t status_code(kvt_engine *e) {
   u32 b = e->h_status[ST_ERR];
   if (!b) return KVT_OK;
+  if (b & DERR_WAIT) return fail(e, KVT_E_DEVICE, "a chunk's wait for its predecessor ran out");
   if (b & (DERR_PROBE | DERR_CORRUPT)) return fail(e, KVT_E_DEVICE, b & DERR_PROBE ? "table probe cap exceeded" : "corrupt metadata");
   if (b & DERR_RANGE) return fail(e, KVT_E_RANGE, "slot id out of range");
   if (b & DERR_INVAL) return fail(e, KVT_E_INVAL, "slot empty, repeated, or key already resident");
@@ -225,7 +228,7 @@ void seg_deref(kvt_engine *e, int id) {
   if (--s.refs == 0) { e->key_alloc.release(s.off, s.cap); e->free_segs.push_back(id); }
 }
 int seg_new(kvt_engine *e, u64 n) {
-  u64 keycap = round_up(std::max<u64>(n, 1), 32), total = keycap + keycap / CHUNK + 1, off;
+  u64 keycap = round_up(std::max<u64>(n, 1), 32), total = keycap + cdiv(keycap, (u64)CHUNK) + 1, off;   // one carry per chunk (the last may be partial) + the resume point
   if (!e->key_alloc.alloc(total, &off)) return -1;
   int id;
   if (!e->free_segs.empty()) { id = e->free_segs.back(); e->free_segs.pop_back(); }
@@ -552,6 +555,12 @@ int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant) {
   return KVT_OK;
 }
 
+int32_t kvt_debug_set_lookup_variant(kvt_engine *e, uint32_t variant) {
+  if (!e || variant > 2) return KVT_E_INVAL;
+  e->lookup_variant = variant;
+  return KVT_OK;
+}
+
 int32_t kvt_get_stats(kvt_engine *e, kvt_stats *out) {
   if (!e || !out) return KVT_E_INVAL;
   kvt_stats s = e->st;
@@ -797,9 +806,17 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     lk.ent = e->ent; lk.b_ent = la.b_ent; lk.hit_len = d_res; lk.n_hbm = d_res + C; lk.n_host = d_res + 2 * C;
     lk.now = e->now; lk.status = e->d_status;
     if (e->profiling) CU(cudaEventRecord(e->ev_h0, s));
-    if (dchunk_base) KL(k_hash_digest, dchunk_base, CHUNK, s, ha);
-    KL(k_hash_carry, nd, 1024, s, ha);
-    KL(k_hash_finish_lookup, chunk_base, CHUNK, s, ha, la);
+    if (e->lookup_variant != 2) {
+      if (dchunk_base) KL(k_hash_digest, dchunk_base, CHUNK, s, ha);
+      KL(k_hash_carry, nd, 1024, s, ha);
+      KL(k_hash_finish_lookup, chunk_base, CHUNK, s, ha, la);
+    } else {
+      ChainState cs;
+      cs.flags = e->dp<u32>(e->L.cflags); cs.ticket = cs.flags + chunk_base; cs.incl = e->dp<u64>(e->L.carry);
+      cs.spin_limit = 1u << 18;   // x (one L2 round trip + 40 ns): far beyond any real wait, still bounded
+      CU(cudaMemsetAsync(cs.flags, 0, (chunk_base + 1) * 4ull, s));
+      KL(k_hash_lookup_fused, chunk_base, CHUNK, s, ha, la, cs);
+    }
     KL(k_lock_hits, chunk_base, CHUNK, s, ha, lk);
     if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));
     LAUNCH_CHECK();

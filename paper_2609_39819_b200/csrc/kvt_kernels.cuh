@@ -25,7 +25,7 @@ constexpr u32 SORT_TILE = 1024;   // items per CTA in the radix-sort kernels (8 
 constexpr int SORT_ITERS = SORT_TILE / 256;   // items per thread
 
 // bits of the device error word
-enum : u32 { DERR_PROBE = 1, DERR_RANGE = 2, DERR_INVAL = 4, DERR_STATE = 8, DERR_CORRUPT = 16 };
+enum : u32 { DERR_PROBE = 1, DERR_RANGE = 2, DERR_INVAL = 4, DERR_STATE = 8, DERR_CORRUPT = 16, DERR_WAIT = 32 };
 
 // words of the device status block
 enum : int {
@@ -310,6 +310,167 @@ __global__ void __launch_bounds__(CHUNK) k_hash_finish_lookup(HashArgs a, Lookup
   }
   __syncthreads();
   if (l.tab.slots && tid == 0 && s_min != 0xFFFFFFFFu) atomicMin(&l.hit_len[ci], s_min);
+}
+
+// ------------------------------------------------------------------------------------------------------
+// Single-pass form of digest + carry + finish + probe for a LOOKUP batch. A CTA takes the next chunk of the
+// all-blocks grid from a ticket counter (so every chunk with a lower number is already running or done),
+// digests it, publishes its aggregate, finds the chain value entering it by looking back over the
+// aggregates / chain values its predecessors of the same sequence have published (32 predecessors per step,
+// folded as affine maps), publishes its own chain value and finishes + probes its 256 keys. The streaming
+// token reads of some chunks overlap the random table reads of others. Every wait is bounded: a CTA that
+// gives up sets DERR_WAIT and carries on with a zero carry (the call then fails; no table word is written by
+// this kernel).
+// ------------------------------------------------------------------------------------------------------
+struct ChainState {
+  u32 *flags;    // per chunk of the all-blocks grid: 0 nothing, 1 aggregate published, 2 chain value published
+  u64 *incl;     // chain value after the chunk
+  u32 *ticket;   // next chunk to hand out (zero at launch, like the flags)
+  u32 spin_limit;
+};
+
+__device__ __forceinline__ u32 ld_acquire_u32(const u32 *p) {
+  u32 v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release_u32(u32 *p, u32 v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+
+__global__ void __launch_bounds__(CHUNK) k_hash_lookup_fused(HashArgs a, LookupArgs l, ChainState cs) {
+  __shared__ u64 sd[CHUNK];
+  __shared__ u64 wagg[CHUNK / 32];
+  __shared__ u64 s_carry;
+  __shared__ u32 s_chunk, s_min;
+  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) { s_chunk = atomicAdd(cs.ticket, 1u); s_min = 0xFFFFFFFFu; }
+  __syncthreads();
+  const u32 chunk = s_chunk;
+  u32 ci;
+  const HashCtx c = hash_ctx_of_chunk(a, chunk, &ci);
+  const u32 j = chunk - c.chunk_base;            // chunk index inside the sequence
+  const u32 b0 = j * CHUNK;
+  const u32 nb = min(CHUNK, c.n_blocks - b0);
+  const u32 g0 = c.first / CHUNK;
+  u64 key = 0;
+  if (b0 < c.first) {
+    // unchanged prefix: keys and the carry entering this chunk are taken over from the previous list
+    if (tid < nb) key = a.keys[c.old_key_off + b0 + tid];
+    if (tid == 0) {
+      a.carry_base[c.carry_off + j] = a.carry_base[c.old_carry_off + j];
+      if (b0 + CHUNK == c.n_blocks) a.carry_base[c.carry_off + j + 1] = a.carry_base[c.old_carry_off + j + 1];
+    }
+  } else {
+    const uint4 *tok = reinterpret_cast<const uint4 *>(a.tokens + c.tok_off + (u64)b0 * 16);
+    const u32 q = tid & 3;
+    const u64 k0 = g_lane_mult.v[4 * q], k1 = g_lane_mult.v[4 * q + 1], k2 = g_lane_mult.v[4 * q + 2],
+              k3 = g_lane_mult.v[4 * q + 3];
+    const u64 ksum = k0 + k1 + k2 + k3;
+    uint4 v[4];
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      u32 idx = it * CHUNK + tid;
+      v[it] = (idx >> 2) < nb ? __ldg(tok + idx) : make_uint4(0, 0, 0, 0);
+    }
+    u64 mine = 0;
+#pragma unroll
+    for (int it = 0; it < 4; ++it) {
+      u64 s = ksum + mul_tok(v[it].x, k0) + mul_tok(v[it].y, k1) + mul_tok(v[it].z, k2) + mul_tok(v[it].w, k3);
+      s += __shfl_xor_sync(0xFFFFFFFFu, s, 1);
+      s += __shfl_xor_sync(0xFFFFFFFFu, s, 2);
+      if ((u32)it == q) mine = s;
+    }
+    {
+      u32 blk = (q * CHUNK + tid) >> 2;
+      sd[blk] = blk < nb ? mix64(mine) : 0;
+    }
+    __syncthreads();
+    u64 cval = sd[tid];
+    u64 pp = HASH_P;
+#pragma unroll
+    for (u32 o = 1; o < 32; o <<= 1) {
+      u64 up = __shfl_up_sync(0xFFFFFFFFu, cval, o);
+      if (lane >= o) cval += pp * up;
+      pp *= pp;
+    }
+    if (lane == 31) wagg[warp] = cval;
+    __syncthreads();
+    u64 wc = 0;
+    const u64 p32 = pp;
+    for (u32 w = 0; w < warp; ++w) wc = p32 * wc + wagg[w];
+    cval += g_pow_p.v[lane + 1] * wc;      // chain value of block b0 + tid with zero carry-in
+    if (tid == nb - 1) sd[0] = cval;       // sd[] was consumed before the last barrier: reuse word 0 for the aggregate
+    __syncthreads();
+    if (warp == 0) {
+      const u64 agg = sd[0];
+      u64 cin;
+      if (j == g0) {
+        cin = g0 ? a.carry_base[c.old_carry_off + g0] : a.h0;
+      } else {
+        if (lane == 0) { a.agg[chunk] = agg; st_release_u32(cs.flags + chunk, 1u); }
+        const u64 A = g_pow_p.v[CHUNK];    // every predecessor is a full chunk
+        u64 acc_m = 1, acc_a = 0;
+        int k_hi = (int)j - 1;
+        bool failed = false;
+        while (true) {
+          const int k = k_hi - (int)lane;
+          u64 m = 1, ad = 0;
+          u32 f = 2;
+          const bool mine_k = k >= (int)g0;
+          const u32 idx = c.chunk_base + (u32)(mine_k ? k : 0);
+          u32 it = 0;
+          do {
+            f = mine_k ? ld_acquire_u32(cs.flags + idx) : 2u;
+            if (!__any_sync(0xFFFFFFFFu, f == 0)) break;
+            __nanosleep(40);
+          } while (++it < cs.spin_limit);
+          if (mine_k) {
+            if (f == 2) { m = 0; ad = __ldcg(cs.incl + idx); }
+            else if (f == 1) { m = A; ad = __ldcg(a.agg + idx); }
+            else { m = 0; ad = 0; failed = true; }
+          }
+          // fold the window: lane 0 ends with M_0 o M_1 o ... o M_31 (M_31 applied first)
+#pragma unroll
+          for (u32 o = 1; o < 32; o <<= 1) {
+            u64 m2 = __shfl_down_sync(0xFFFFFFFFu, m, o), a2 = __shfl_down_sync(0xFFFFFFFFu, ad, o);
+            if (lane + o < 32) { ad = m * a2 + ad; m = m * m2; }
+          }
+          const u64 wm = __shfl_sync(0xFFFFFFFFu, m, 0), wa = __shfl_sync(0xFFFFFFFFu, ad, 0);
+          acc_a = acc_m * wa + acc_a;
+          acc_m = acc_m * wm;
+          failed = __any_sync(0xFFFFFFFFu, failed);
+          if (acc_m == 0 || failed) break;   // a published chain value ends the walk (A is odd: no other zero)
+          k_hi -= 32;
+          if (k_hi < (int)g0) { failed = true; break; }   // cannot happen: chunk g0 always publishes its chain value
+        }
+        if (failed && lane == 0) set_err(l.status, DERR_WAIT);
+        cin = failed ? 0 : acc_a;
+      }
+      if (lane == 0) {
+        const u64 after = g_pow_p.v[nb] * cin + agg;
+        cs.incl[chunk] = after;
+        st_release_u32(cs.flags + chunk, 2u);
+        a.carry_base[c.carry_off + j] = cin;
+        if (b0 + nb == c.n_blocks) a.carry_base[c.carry_off + j + 1] = after;   // resume point of a later call
+        s_carry = cin;
+      }
+    }
+    __syncthreads();
+    if (tid < nb) {
+      key = mix64(g_pow_p.v[tid + 1] * s_carry + cval);
+      if (key < 2) key += 2;
+    }
+  }
+  if (tid < nb) {
+    a.keys[c.key_off + b0 + tid] = key;
+    u32 s = tab_find(l.tab, key, l.status);
+    u32 ent = s == ENT_NONE ? ENT_NONE : l.tab.slots[s].ent;
+    l.b_ent[c.blk_base + b0 + tid] = ent;
+    if (ent == ENT_NONE) atomicMin(&s_min, b0 + tid);
+  }
+  __syncthreads();
+  if (tid == 0 && s_min != 0xFFFFFFFFu) atomicMin(&l.hit_len[ci], s_min);
 }
 
 // Stamps and locks the reusable prefix of every context of the batch; counts hits per tier.

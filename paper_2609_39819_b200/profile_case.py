@@ -153,7 +153,7 @@ def main(case: str):
         print(f"hash_big: {nb} blocks, ms per call {ms}, blocks/s {[round(nb / (m / 1e3)) for m in ms]}, "
               f"GB/s at 72 B per block {[round(72 * nb / (m / 1e3) / 1e9, 1) for m in ms]}")
     elif case in ("lookup", "select"):
-        n_res, n_calls = (1 << 18, 16) if case == "lookup" else (1 << 20, 4)
+        n_res, n_calls = (1 << 20, 64) if case == "lookup" else (1 << 20, 4)
         inp = W.inputs_c4(1, n_resident=n_res, chain_blocks=16128, n_calls=n_calls)
         eng = B.Engine(n_hbm_blocks=n_res, n_host_blocks=0, max_contexts=n_calls + 1, metadata_only=True,
                        max_tokens=(n_calls + 2) * 16128 * 16 * 2, max_messages=1024, max_batch_blocks=n_calls * 16128,
@@ -161,17 +161,31 @@ def main(case: str):
         keys = np.concatenate([B.hash_tokens(torch.from_numpy(c.view(np.int32)).cuda()).cpu().numpy().view(np.uint64)
                                for c in inp.chain_tokens])
         eng.debug_load_resident(keys, inp.state, inp.stamp, inp.depth, inp.slot, 0)
-        for i, t in enumerate(inp.calls):
-            eng.spawn(i)
-            eng.append(i, torch.from_numpy(t.view(np.int32)).cuda())
+        call_tok = [torch.from_numpy(t.view(np.int32)).cuda() for t in inp.calls]
+
+        def fresh_contexts():
+            for i, t in enumerate(call_tok):
+                eng.spawn(i)
+                eng.append(i, t)
+        if case == "select":
+            fresh_contexts()
         if case == "lookup":
-            ms = []
-            for _ in range(3):
-                ms += _events(torch, lambda: eng.map_blocks(list(range(n_calls)), 0), 1)
-                for c in range(n_calls):
-                    eng.prefill_done(c)
-            print(f"lookup: {n_calls} calls x 16128 blocks against {n_res} resident, ms per batch {ms}, "
-                  f"blocks/s {[round(n_calls * 16128 / (m / 1e3)) for m in ms]}")
+            # both forms of the hash + probe stage, each with a cold L2 (a 512 MiB fill before every batch)
+            eng.set_profiling(True)
+            flush = torch.empty(1 << 29, dtype=torch.uint8, device="cuda")
+            for variant in (1, 2, 1, 2):
+                eng.set_lookup_variant(variant)
+                ms, kms = [], []
+                for rep in range(4):
+                    fresh_contexts()          # nothing to resume from: every block is digested
+                    flush.fill_(rep)
+                    k0 = eng.get_stats()["lookup_ns"]
+                    ms += _events(torch, lambda: eng.map_blocks(list(range(n_calls)), 0), 1)
+                    kms.append(round((eng.get_stats()["lookup_ns"] - k0) / 1e6, 4))
+                    for c in range(n_calls):
+                        eng.terminate(c)
+                print(f"lookup variant {variant}: {n_calls} calls x 16128 blocks against {n_res} resident, cold L2: "
+                      f"ms per batch {ms}, kernels ms {kms}, blocks/s (kernels) {[round(n_calls * 16128 / (m / 1e3)) for m in kms]}")
         else:
             ms = _events(torch, lambda: eng.select_victims(0, n_res // 10), 3)
             print(f"select: {n_res // 10} victims of {n_res} resident, ms per call {ms}")

@@ -370,9 +370,11 @@ def _c4_setup(B, oracle, n_resident, chain_blocks, n_calls):
     return inp, gpu, cpu
 
 
+@pytest.mark.parametrize("lookup_variant", [1, 2], ids=["three-kernels", "single-pass"])
 @pytest.mark.parametrize("n_resident,chain_blocks,n_calls", [(5000, 700, 9), (1 << 20, 16128, 64)])
-def test_c4_lookup_and_select_parity(B, oracle, n_resident, chain_blocks, n_calls):
+def test_c4_lookup_and_select_parity(B, oracle, n_resident, chain_blocks, n_calls, lookup_variant):
     inp, gpu, cpu = _c4_setup(B, oracle, n_resident, chain_blocks, n_calls)
+    gpu.set_lookup_variant(lookup_variant)
     ids = list(range(n_calls))
     # selection before any call: the whole pool is a candidate; 10% stays in the dead tier,
     # 35% crosses into the idle (MRU) tier, 75% into the active tier
@@ -565,11 +567,13 @@ def test_capacity_errors_leave_the_engine_usable(B):
         eng.select_victims(2, 1)                                 # bad tier
 
 
-def test_incremental_hashing_resumes_at_chunk_boundaries(B, oracle):
+@pytest.mark.parametrize("lookup_variant", [1, 2], ids=["three-kernels", "single-pass"])
+def test_incremental_hashing_resumes_at_chunk_boundaries(B, oracle, lookup_variant):
     """Appends, edits, forks and repeated calls around multiples of 256 blocks: only the changed tail is digested
     again, and every key still equals the one-shot hash of the whole sequence."""
     kw = dict(n_hbm_blocks=4096, n_host_blocks=0, max_contexts=8, metadata_only=True, **W.GEO_TOY.kwargs())
     gpu = B.Engine(max_tokens=1 << 18, max_messages=1024, **kw)
+    gpu.set_lookup_variant(lookup_variant)
     rng = np.random.default_rng(30)
     msgs = []
 
@@ -605,6 +609,33 @@ def test_incremental_hashing_resumes_at_chunk_boundaries(B, oracle):
     assert got == len(keys) - 512
     st = gpu.get_stats()
     assert st["blocks_rehashed"] < st["blocks_hashed"]
+
+
+@pytest.mark.parametrize("lookup_variant", [1, 2], ids=["three-kernels", "single-pass"])
+def test_adjacent_key_lists_do_not_overlap(B, oracle, lookup_variant):
+    """Key lists of one batch sit back to back in the key arena, each followed by its per-chunk carries and the
+    resume point: sizes whose rounded lists leave no slack (e.g. 7,937..7,968 blocks) must not spill into the
+    next list."""
+    rng = np.random.default_rng(31)
+    for sizes in ((7950, 300, 7968), (7937, 7968, 31), (16130, 16160, 288), (255, 256, 257, 32, 1)):
+        kw = dict(n_hbm_blocks=64, n_host_blocks=0, max_contexts=8, metadata_only=True, **W.GEO_TOY.kwargs())
+        gpu = B.Engine(max_tokens=1 << 21, max_messages=64, **kw)
+        gpu.set_lookup_variant(lookup_variant)
+        toks = []
+        for c, nb in enumerate(sizes):
+            toks.append(rng.integers(0, W.VOCAB, nb * 16 + 5, dtype=np.uint32))
+            gpu.spawn(c)
+            gpu.append(c, toks[c])
+        for rnd in range(2):       # second round: everything is resumed from the kept carries
+            gpu.map_blocks(list(range(len(sizes))), 0)
+            for c in range(len(sizes)):
+                assert np.array_equal(gpu.get_block_map(c)[0], oracle.hash_tokens(toks[c])), (sizes, rnd, c)
+            for c in range(len(sizes)):
+                gpu.prefill_done(c)
+            for c in range(len(sizes)):
+                extra = rng.integers(0, W.VOCAB, 16 * 3, dtype=np.uint32)
+                toks[c] = np.concatenate([toks[c], extra])
+                gpu.append(c, extra)
 
 
 def test_create_rejects_bad_configs(B):
