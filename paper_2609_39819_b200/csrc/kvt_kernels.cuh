@@ -143,12 +143,22 @@ struct HashArgs {
 
 // Sequence that owns chunk `chunk` of the all-blocks grid (dgrid = false) or of the digest grid (dgrid = true):
 // the last one whose base is <= chunk (sequences with no chunk of their own share a base with their successor).
+// Called by every thread of the CTA with the same arguments: the bases are staged in shared memory with one
+// round of loads, so a cold start costs one memory latency instead of one per step of the binary search.
+constexpr u32 CTX_STAGE = 1024;
 __device__ __forceinline__ const HashCtx &hash_ctx_of_chunk(const HashArgs &a, u32 chunk, u32 *ctx_idx, bool dgrid = false) {
   if (!a.ctx) { *ctx_idx = 0; return a.single; }
+  __shared__ u32 s_base[CTX_STAGE];
+  const bool staged = a.n_ctx <= CTX_STAGE;
+  if (staged) {
+    for (u32 t = threadIdx.x; t < a.n_ctx; t += blockDim.x) s_base[t] = dgrid ? a.ctx[t].dchunk_base : a.ctx[t].chunk_base;
+    __syncthreads();
+  }
   u32 lo = 0, hi = a.n_ctx;
   while (hi - lo > 1) {
     u32 mid = (lo + hi) >> 1;
-    if ((dgrid ? a.ctx[mid].dchunk_base : a.ctx[mid].chunk_base) <= chunk) lo = mid; else hi = mid;
+    u32 base = staged ? s_base[mid] : (dgrid ? a.ctx[mid].dchunk_base : a.ctx[mid].chunk_base);
+    if (base <= chunk) lo = mid; else hi = mid;
   }
   *ctx_idx = lo;
   return a.ctx[lo];
@@ -730,6 +740,23 @@ struct ClsArgs {
   u32 *first_miss;   // per listed context: index of its first non-resident block; nullptr = orphans keep their state
 };
 
+// Context that owns mapping g (the last one whose map_base is <= g). Every thread of the CTA calls it: the
+// bases are staged in shared memory by one round of loads when they fit.
+__device__ __forceinline__ u32 cls_ctx_of_mapping(const ClsArgs &a, u32 g) {
+  __shared__ u32 s_base[CTX_STAGE];
+  const bool staged = a.n_ctx <= CTX_STAGE;
+  if (staged) {
+    for (u32 t = threadIdx.x; t < a.n_ctx; t += blockDim.x) s_base[t] = a.ctx[t].map_base;
+    __syncthreads();
+  }
+  u32 lo = 0, hi = a.n_ctx;
+  while (hi - lo > 1) {
+    u32 mid = (lo + hi) >> 1;
+    if ((staged ? s_base[mid] : a.ctx[mid].map_base) <= g) lo = mid; else hi = mid;
+  }
+  return lo;
+}
+
 __global__ void k_rank_reset(Entries en) {
   u32 e = blockIdx.x * blockDim.x + threadIdx.x;
   if (e < en.n_total) en.rank[e] = en.floor[e];
@@ -739,9 +766,8 @@ __global__ void k_rank_reset(Entries en) {
 // stops there, so the blocks behind it cannot be reused through this context.
 __global__ void k_first_miss(ClsArgs a) {
   u32 g = blockIdx.x * blockDim.x + threadIdx.x;
+  const u32 lo = cls_ctx_of_mapping(a, g);
   if (g >= a.n_map) return;
-  u32 lo = 0, hi = a.n_ctx;
-  while (hi - lo > 1) { u32 mid = (lo + hi) >> 1; if (a.ctx[mid].map_base <= g) lo = mid; else hi = mid; }
   const ClsCtx c = a.ctx[lo];
   const u32 b = g - c.map_base;
   if (tab_find(a.tab, a.keys[c.key_off + b], a.status) == ENT_NONE) atomicMin(&a.first_miss[lo], b);
@@ -749,9 +775,8 @@ __global__ void k_first_miss(ClsArgs a) {
 
 __global__ void k_classify(ClsArgs a) {
   u32 g = blockIdx.x * blockDim.x + threadIdx.x;
+  const u32 lo = cls_ctx_of_mapping(a, g);
   if (g >= a.n_map) return;
-  u32 lo = 0, hi = a.n_ctx;
-  while (hi - lo > 1) { u32 mid = (lo + hi) >> 1; if (a.ctx[mid].map_base <= g) lo = mid; else hi = mid; }
   const ClsCtx c = a.ctx[lo];
   const u32 b = g - c.map_base;
   if (a.first_miss && b >= a.first_miss[lo]) return;   // behind a missing block: unreachable through this context
