@@ -39,7 +39,7 @@ namespace {
 enum : int32_t {
   OK = 0, E_INVAL = -1, E_NOCTX = -2, E_RANGE = -3, E_STATE = -4, E_NOSPACE = -5, E_BUFSZ = -6
 };
-enum : uint32_t { TIER_HBM = 0, TIER_HOST = 1 };
+enum : uint32_t { TIER_HBM = 0, TIER_HOST = 1, TIER_REMOTE = 2, N_TIERS = 3 };
 enum : uint32_t { LAYOUT_LAYER_MAJOR = 0, LAYOUT_BLOCK_MAJOR = 1 };
 enum : uint32_t { ORDER_MRU = 0, ORDER_LRU = 1 };
 enum : uint32_t {
@@ -116,7 +116,7 @@ struct Ctx {
   std::vector<uint64_t> mat_keys;                          // hash of mat_tokens
   uint32_t valid_blocks = 0;  // leading blocks of mat_keys this context still maps
   uint32_t held = 0;          // leading blocks locked in flight
-  uint32_t hit_len = 0, n_hit_hbm = 0, n_hit_host = 0, n_admissible = 0, n_pinned = 0;
+  uint32_t hit_len = 0, n_hit_hbm = 0, n_hit_host = 0, n_hit_remote = 0, n_admissible = 0, n_pinned = 0;
 };
 
 struct Entry {
@@ -131,15 +131,18 @@ struct Config {
   uint32_t n_hbm_blocks, n_host_blocks, max_contexts, suspended_order, policy_flags;
   uint64_t hash_seed;
   uint8_t *hbm_pool; uint8_t *host_pool;  // host memory; NULL = metadata only
+  uint32_t n_remote_blocks, pad;          // third tier (Section 7: remote memory), stood in for by one more buffer
+  uint8_t *remote_pool;
 };
 
-struct CallInfo { uint32_t n_blocks, hit_len, n_hit_hbm, n_hit_host, n_admissible, n_admitted, n_held, n_pinned; };
+struct CallInfo { uint32_t n_blocks, hit_len, n_hit_hbm, n_hit_host, n_admissible, n_admitted, n_held, n_pinned, n_hit_remote; };
 
 struct Stats {
   uint64_t clock, n_contexts, occ_hbm, occ_host, blocks_hashed, hits_hbm, hits_host, misses,
       inserted, adopted, dropped, offloaded, reloaded, compacted, bytes_d2h, bytes_h2d, bytes_d2d,
       table_rebuilds, tombstones, kernel_launches, mover_launches, mover_ns, mover_bytes, lookup_ns,
-      lookup_blocks, select_ns, select_slots, offloaded_clean, blocks_rehashed;
+      lookup_blocks, select_ns, select_slots, offloaded_clean, blocks_rehashed, occ_remote, hits_remote, demoted,
+      promoted;
 };
 
 struct Op {
@@ -152,19 +155,21 @@ struct Engine {
   HashParams hp;
   uint64_t chunk_bytes, n_chunks, block_bytes;
   std::vector<Ctx> ctxs;
-  std::vector<Entry> ent[2];          // per tier, indexed by slot; key == 0 means free
-  std::set<uint32_t> free_slots[2];   // lowest-numbered free slot first
+  std::vector<Entry> ent[N_TIERS];          // per tier, indexed by slot; key == 0 means free
+  std::set<uint32_t> free_slots[N_TIERS];   // lowest-numbered free slot first
   std::map<uint64_t, std::pair<uint32_t, uint32_t>> where;  // key -> (tier, slot)
   uint32_t now = 0;
   Stats st{};
 };
 
-uint32_t tier_size(const Engine &e, uint32_t t) { return t == TIER_HBM ? e.cfg.n_hbm_blocks : e.cfg.n_host_blocks; }
+uint32_t tier_size(const Engine &e, uint32_t t) {
+  return t == TIER_HBM ? e.cfg.n_hbm_blocks : t == TIER_HOST ? e.cfg.n_host_blocks : e.cfg.n_remote_blocks;
+}
 
 uint8_t *chunk_ptr(const Engine &e, uint32_t tier, uint32_t slot, uint64_t c) {
   if (tier == TIER_HBM && e.cfg.pool_layout == LAYOUT_LAYER_MAJOR)
     return e.cfg.hbm_pool + (c * (uint64_t)e.cfg.n_hbm_blocks + slot) * e.chunk_bytes;
-  uint8_t *base = tier == TIER_HBM ? e.cfg.hbm_pool : e.cfg.host_pool;
+  uint8_t *base = tier == TIER_HBM ? e.cfg.hbm_pool : tier == TIER_HOST ? e.cfg.host_pool : e.cfg.remote_pool;
   return base + (uint64_t)slot * e.block_bytes + c * e.chunk_bytes;
 }
 
@@ -218,8 +223,8 @@ void block_ranks(const Ctx &c, const std::vector<std::pair<uint32_t, uint32_t>> 
 // KV-level state of every resident block (Section 6.1): the highest-priority state over all
 // mappings (context c, block b < valid_blocks, same key); dead if nobody maps it. `floor` is the
 // anonymous mapping installed by the debug loader.
-void classify(Engine &e, std::vector<uint8_t> rank[2]) {
-  for (int t = 0; t < 2; ++t) {
+void classify(Engine &e, std::vector<uint8_t> rank[N_TIERS]) {
+  for (int t = 0; t < (int)N_TIERS; ++t) {
     rank[t].assign(e.ent[t].size(), 0xFF);
     for (size_t s = 0; s < e.ent[t].size(); ++s)
       if (e.ent[t][s].key) rank[t][s] = e.ent[t][s].shadow ? 0xFE : e.ent[t][s].floor;
@@ -278,8 +283,10 @@ int32_t kvto_create(const Config *cfg, Engine **out) {
   e->ctxs.resize(cfg->max_contexts);
   e->ent[0].resize(cfg->n_hbm_blocks);
   e->ent[1].resize(cfg->n_host_blocks);
+  e->ent[2].resize(cfg->n_remote_blocks);
   for (uint32_t s = 0; s < cfg->n_hbm_blocks; ++s) e->free_slots[0].insert(s);
   for (uint32_t s = 0; s < cfg->n_host_blocks; ++s) e->free_slots[1].insert(s);
+  for (uint32_t s = 0; s < cfg->n_remote_blocks; ++s) e->free_slots[2].insert(s);
   *out = e;
   return OK;
 }
@@ -457,14 +464,16 @@ int32_t kvto_map_blocks(Engine *e, const uint32_t *ids, uint32_t n_ctx, uint32_t
       c.valid_blocks = nb;
       // reusable prefix: walk the chain until the first block that is not resident
       uint32_t h = 0;
-      c.n_hit_hbm = c.n_hit_host = 0;
+      c.n_hit_hbm = c.n_hit_host = c.n_hit_remote = 0;
       while (h < nb) {
         auto it = e->where.find(c.mat_keys[h]);
         if (it == e->where.end()) break;
         Entry &x = e->ent[it->second.first][it->second.second];
         x.stamp = e->now;
         x.inflight += 1;
-        if (it->second.first == TIER_HBM) c.n_hit_hbm++; else c.n_hit_host++;
+        if (it->second.first == TIER_HBM) c.n_hit_hbm++;
+        else if (it->second.first == TIER_HOST) c.n_hit_host++;
+        else c.n_hit_remote++;
         ++h;
       }
       c.hit_len = h;
@@ -483,8 +492,9 @@ int32_t kvto_map_blocks(Engine *e, const uint32_t *ids, uint32_t n_ctx, uint32_t
       e->st.blocks_hashed += nb;
       e->st.hits_hbm += c.n_hit_hbm;
       e->st.hits_host += c.n_hit_host;
+      e->st.hits_remote += c.n_hit_remote;
       e->st.misses += nb - h;
-      out[i] = CallInfo{nb, h, c.n_hit_hbm, c.n_hit_host, c.n_admissible, 0, c.held, c.n_pinned};
+      out[i] = CallInfo{nb, h, c.n_hit_hbm, c.n_hit_host, c.n_admissible, 0, c.held, c.n_pinned, c.n_hit_remote};
     }
     return OK;
   }
@@ -513,7 +523,8 @@ int32_t kvto_map_blocks(Engine *e, const uint32_t *ids, uint32_t n_ctx, uint32_t
     }
     uint32_t adm = b - c.held;
     c.held = b;
-    out[i] = CallInfo{(uint32_t)c.mat_keys.size(), c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, adm, c.held, c.n_pinned};
+    out[i] = CallInfo{(uint32_t)c.mat_keys.size(), c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, adm, c.held, c.n_pinned,
+                      c.n_hit_remote};
   }
   return OK;
 }
@@ -536,9 +547,9 @@ int32_t kvto_get_block_map(Engine *e, uint32_t ctx, uint64_t *keys, uint8_t *tie
 }
 
 int32_t kvto_get_states(Engine *e, uint32_t tier, uint8_t *state, uint32_t cap) {
-  if (!e || !state || tier > 1) return E_INVAL;
+  if (!e || !state || tier >= N_TIERS) return E_INVAL;
   if (cap < tier_size(*e, tier)) return E_BUFSZ;
-  std::vector<uint8_t> rank[2];
+  std::vector<uint8_t> rank[N_TIERS];
   classify(*e, rank);
   if (!rank[tier].empty()) std::memcpy(state, rank[tier].data(), rank[tier].size());
   return OK;
@@ -548,7 +559,7 @@ int32_t kvto_get_states(Engine *e, uint32_t tier, uint8_t *state, uint32_t cap) 
 // mapping of every context), with block ranks recomputed from token spans per block. Quadratic:
 // tiny pools only. Serves as a pin for classify().
 int32_t kvto_classify_bruteforce(Engine *e, uint32_t tier, uint8_t *state, uint32_t cap) {
-  if (!e || !state || tier > 1) return E_INVAL;
+  if (!e || !state || tier >= N_TIERS) return E_INVAL;
   if (cap < tier_size(*e, tier)) return E_BUFSZ;
   for (uint32_t s = 0; s < tier_size(*e, tier); ++s) {
     const Entry &x = e->ent[tier][s];
@@ -580,9 +591,9 @@ int32_t kvto_classify_bruteforce(Engine *e, uint32_t tier, uint8_t *state, uint3
 
 int32_t kvto_select_victims(Engine *e, uint32_t tier, uint32_t n_req, uint32_t flags, uint32_t *slots_out,
                             uint8_t *states_out, uint32_t cap, uint32_t *n_out) {
-  if (!e || tier > 1 || flags > 1 || !n_out || (!slots_out && cap)) return E_INVAL;
+  if (!e || tier >= N_TIERS || flags > 1 || !n_out || (!slots_out && cap)) return E_INVAL;
   const int max_rank = (flags & 1) ? 3 : 2;   // Pinned KV competes only when the incoming KV is Pinned
-  std::vector<uint8_t> rank[2];
+  std::vector<uint8_t> rank[N_TIERS];
   classify(*e, rank);
   if (e->cfg.policy_flags & POLICY_NO_LIFECYCLE)   // without lifecycle tracking every resident block is one tier
     for (uint8_t &r : rank[tier]) if (r != 0xFF) r = 1;
@@ -650,7 +661,7 @@ int32_t kvto_offload(Engine *e, const uint32_t *slots, uint32_t n, uint32_t *n_d
   *n_done = *n_dropped = 0;
   int32_t v = validate_slots(e, TIER_HBM, slots, n, false);
   if (v != OK) return v;
-  std::vector<uint8_t> rank[2];
+  std::vector<uint8_t> rank[N_TIERS];
   classify(*e, rank);
   const bool knows_dead = !(e->cfg.policy_flags & POLICY_NO_LIFECYCLE);
   // destination slots: the host slots that are free when the call begins, lowest first (slots freed by this
@@ -713,6 +724,44 @@ int32_t kvto_reload(Engine *e, const uint32_t *slots, uint32_t n, uint32_t *n_do
   return OK;
 }
 
+// Movement between any two neighbouring levels of the hierarchy (Section 7: HBM, host memory, remote memory), plus
+// the direct way up from the remote tier into HBM. Downward (host -> remote) behaves like an offload: dead blocks
+// are dropped, live ones go to the destination slots that are free when the call begins, lowest first. Upward
+// (remote -> host, remote -> HBM) behaves like a reload: the i-th listed block goes to the i-th lowest free slot;
+// blocks in flight may move up (a call fetches its own hits). Clean host copies of HBM blocks cannot be moved.
+int32_t kvto_move(Engine *e, uint32_t st, uint32_t dt, const uint32_t *slots, uint32_t n, uint32_t *n_done,
+                  uint32_t *n_dropped) {
+  if (!e || (!slots && n) || !n_done || !n_dropped) return E_INVAL;
+  *n_done = *n_dropped = 0;
+  if (st == TIER_HBM && dt == TIER_HOST) return kvto_offload(e, slots, n, n_done, n_dropped);
+  if (st == TIER_HOST && dt == TIER_HBM) return kvto_reload(e, slots, n, n_done);
+  const bool down = st == TIER_HOST && dt == TIER_REMOTE;
+  const bool up = st == TIER_REMOTE && (dt == TIER_HOST || dt == TIER_HBM);
+  if (!down && !up) return E_INVAL;
+  int32_t v = validate_slots(e, st, slots, n, up, false);
+  if (v != OK) return v;
+  std::vector<uint8_t> rank[N_TIERS];
+  classify(*e, rank);
+  const bool knows_dead = !(e->cfg.policy_flags & POLICY_NO_LIFECYCLE);
+  std::vector<uint32_t> dests(e->free_slots[dt].begin(), e->free_slots[dt].end());
+  size_t next_dest = 0;
+  for (uint32_t i = 0; i < n; ++i) {
+    uint32_t s = slots[i];
+    if (down && knows_dead && rank[st][s] == 0) {
+      free_slot(*e, st, s);
+      e->st.dropped++;
+      (*n_dropped)++;
+    } else {
+      if (next_dest == dests.size()) return E_NOSPACE;
+      move_entry(e, st, s, dt, dests[next_dest++]);
+      if (down) e->st.demoted++; else e->st.promoted++;
+      if (dt == TIER_HBM) e->st.bytes_h2d += e->block_bytes;
+    }
+    (*n_done)++;
+  }
+  return OK;
+}
+
 // Reload and offload in one call, both with destinations taken from the slots that are free when the call
 // begins (the two payload streams are independent, so a device can run them concurrently over a duplex link).
 int32_t kvto_exchange(Engine *e, const uint32_t *out_slots, uint32_t n_out, const uint32_t *in_slots, uint32_t n_in,
@@ -723,7 +772,7 @@ int32_t kvto_exchange(Engine *e, const uint32_t *out_slots, uint32_t n_out, cons
   int32_t vb = validate_slots(e, TIER_HBM, out_slots, n_out, false);
   for (int32_t code : {E_RANGE, E_INVAL, E_STATE})
     if (va == code || vb == code) return code;
-  std::vector<uint8_t> rank[2];
+  std::vector<uint8_t> rank[N_TIERS];
   classify(*e, rank);
   const bool knows_dead = !(e->cfg.policy_flags & POLICY_NO_LIFECYCLE);
   std::vector<uint32_t> hbm_dests(e->free_slots[TIER_HBM].begin(), e->free_slots[TIER_HBM].end());
@@ -778,7 +827,7 @@ int32_t kvto_exchange(Engine *e, const uint32_t *out_slots, uint32_t n_out, cons
 }
 
 int32_t kvto_release(Engine *e, uint32_t tier, const uint32_t *slots, uint32_t n) {
-  if (!e || tier > 1 || (!slots && n)) return E_INVAL;
+  if (!e || tier >= N_TIERS || (!slots && n)) return E_INVAL;
   int32_t v = validate_slots(e, tier, slots, n, false);
   if (v != OK) return v;
   for (uint32_t i = 0; i < n; ++i) {
@@ -789,7 +838,7 @@ int32_t kvto_release(Engine *e, uint32_t tier, const uint32_t *slots, uint32_t n
 }
 
 int32_t kvto_compact(Engine *e, uint32_t tier, uint32_t *n_moved) {
-  if (!e || tier > 1 || !n_moved) return E_INVAL;
+  if (!e || tier >= N_TIERS || !n_moved) return E_INVAL;
   uint32_t n = tier_size(*e, tier);
   uint32_t n_occ = n - (uint32_t)e->free_slots[tier].size();
   std::vector<uint32_t> holes, movers;
@@ -805,7 +854,7 @@ int32_t kvto_compact(Engine *e, uint32_t tier, uint32_t *n_moved) {
 }
 
 int32_t kvto_copy_blocks(Engine *e, uint32_t st, const uint32_t *src, uint32_t dt, const uint32_t *dst, uint32_t n) {
-  if (!e || st > 1 || dt > 1 || ((!src || !dst) && n)) return E_INVAL;
+  if (!e || st >= N_TIERS || dt >= N_TIERS || ((!src || !dst) && n)) return E_INVAL;
   if (!e->cfg.hbm_pool) return E_INVAL;
   for (uint32_t i = 0; i < n; ++i)
     if (src[i] >= tier_size(*e, st) || dst[i] >= tier_size(*e, dt)) return E_RANGE;
@@ -821,13 +870,14 @@ int32_t kvto_get_stats(Engine *e, Stats *out) {
   for (const Ctx &c : e->ctxs) s.n_contexts += c.live;
   s.occ_hbm = e->cfg.n_hbm_blocks - e->free_slots[0].size();
   s.occ_host = e->cfg.n_host_blocks - e->free_slots[1].size();
+  s.occ_remote = e->cfg.n_remote_blocks - e->free_slots[2].size();
   *out = s;
   return OK;
 }
 
 int32_t kvto_get_entries(Engine *e, uint32_t tier, uint64_t *keys, uint32_t *stamp, uint32_t *depth,
                          uint32_t *inflight, uint32_t *link, uint32_t cap) {
-  if (!e || tier > 1) return E_INVAL;
+  if (!e || tier >= N_TIERS) return E_INVAL;
   if (cap < tier_size(*e, tier)) return E_BUFSZ;
   for (uint32_t s = 0; s < tier_size(*e, tier); ++s) {
     const Entry &x = e->ent[tier][s];
@@ -842,7 +892,7 @@ int32_t kvto_get_entries(Engine *e, uint32_t tier, uint64_t *keys, uint32_t *sta
 
 int32_t kvto_debug_load_resident(Engine *e, const uint64_t *keys, const uint8_t *state, const uint32_t *stamp,
                                  const uint32_t *depth, const uint32_t *slot, uint32_t tier, uint32_t n) {
-  if (!e || tier > 1 || ((!keys || !state || !stamp || !depth || !slot) && n)) return E_INVAL;
+  if (!e || tier >= N_TIERS || ((!keys || !state || !stamp || !depth || !slot) && n)) return E_INVAL;
   std::set<uint64_t> kseen;
   std::set<uint32_t> sseen;
   for (uint32_t i = 0; i < n; ++i) {

@@ -17,7 +17,7 @@ _SRC = os.path.join(_HERE, "kvt_oracle.cpp")
 _LIB = os.path.join(_HERE, "libkvt_oracle.so")
 
 OK, E_INVAL, E_NOCTX, E_RANGE, E_STATE, E_NOSPACE, E_BUFSZ = 0, -1, -2, -3, -4, -5, -6
-TIER_HBM, TIER_HOST, TIER_NONE = 0, 1, 0xFF
+TIER_HBM, TIER_HOST, TIER_REMOTE, TIER_NONE = 0, 1, 2, 0xFF
 LAYOUT_LAYER_MAJOR, LAYOUT_BLOCK_MAJOR = 0, 1
 ORDER_MRU, ORDER_LRU = 0, 1
 POLICY_NO_LIFECYCLE, POLICY_INCLUSIVE = 1, 2
@@ -43,7 +43,8 @@ class _Config(C.Structure):
     _fields_ = [(n, C.c_uint32) for n in ("n_layers", "n_kv_heads", "head_dim", "elem_bytes", "pool_layout",
                                            "n_hbm_blocks", "n_host_blocks", "max_contexts", "suspended_order",
                                            "policy_flags")] + \
-               [("hash_seed", C.c_uint64), ("hbm_pool", C.c_void_p), ("host_pool", C.c_void_p)]
+               [("hash_seed", C.c_uint64), ("hbm_pool", C.c_void_p), ("host_pool", C.c_void_p),
+                ("n_remote_blocks", C.c_uint32), ("pad", C.c_uint32), ("remote_pool", C.c_void_p)]
 
 
 class _Op(C.Structure):
@@ -52,12 +53,13 @@ class _Op(C.Structure):
 
 
 CALL_INFO_DTYPE = np.dtype([(n, np.uint32) for n in ("n_blocks", "hit_len", "n_hit_hbm", "n_hit_host",
-                                                       "n_admissible", "n_admitted", "n_held", "n_pinned")])
+                                                       "n_admissible", "n_admitted", "n_held", "n_pinned",
+                                                       "n_hit_remote")])
 STATS_FIELDS = ("clock", "n_contexts", "occ_hbm", "occ_host", "blocks_hashed", "hits_hbm", "hits_host", "misses",
                 "inserted", "adopted", "dropped", "offloaded", "reloaded", "compacted", "bytes_d2h", "bytes_h2d",
                 "bytes_d2d", "table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns",
                 "mover_bytes", "lookup_ns", "lookup_blocks", "select_ns", "select_slots", "offloaded_clean",
-                "blocks_rehashed")
+                "blocks_rehashed", "occ_remote", "hits_remote", "demoted", "promoted")
 
 _lib = None
 
@@ -102,24 +104,26 @@ class OracleEngine:
 
     def __init__(self, n_layers, n_kv_heads, head_dim, elem_bytes=2, pool_layout=LAYOUT_LAYER_MAJOR,
                  n_hbm_blocks=128, n_host_blocks=512, max_contexts=64, hash_seed=0,
-                 suspended_order=ORDER_MRU, metadata_only=False, policy_flags=0, **_ignored):
+                 suspended_order=ORDER_MRU, metadata_only=False, policy_flags=0, n_remote_blocks=0, **_ignored):
         self.L = lib()
         self.n_layers, self.n_kv_heads, self.head_dim, self.elem_bytes = n_layers, n_kv_heads, head_dim, elem_bytes
         self.pool_layout = pool_layout
-        self.n_hbm_blocks, self.n_host_blocks = n_hbm_blocks, n_host_blocks
+        self.n_hbm_blocks, self.n_host_blocks, self.n_remote_blocks = n_hbm_blocks, n_host_blocks, n_remote_blocks
         self.chunk_bytes = 16 * n_kv_heads * head_dim * elem_bytes
         self.n_chunks = 2 * n_layers
         self.block_bytes = self.chunk_bytes * self.n_chunks
         self.metadata_only = metadata_only
         if metadata_only:
-            self.hbm_pool = self.host_pool = None
+            self.hbm_pool = self.host_pool = self.remote_pool = None
         else:
             self.hbm_pool = np.zeros(n_hbm_blocks * self.block_bytes, dtype=np.uint8)
             self.host_pool = np.zeros(max(n_host_blocks, 1) * self.block_bytes, dtype=np.uint8)
+            self.remote_pool = np.zeros(max(n_remote_blocks, 1) * self.block_bytes, dtype=np.uint8)
         cfg = _Config(n_layers, n_kv_heads, head_dim, elem_bytes, pool_layout, n_hbm_blocks, n_host_blocks,
                       max_contexts, suspended_order, policy_flags, hash_seed,
                       None if metadata_only else self.hbm_pool.ctypes.data,
-                      None if metadata_only else self.host_pool.ctypes.data)
+                      None if metadata_only else self.host_pool.ctypes.data,
+                      n_remote_blocks, 0, None if metadata_only else self.remote_pool.ctypes.data)
         h = C.c_void_p()
         rc = self.L.kvto_create(C.byref(cfg), C.byref(h))
         if rc:
@@ -193,7 +197,7 @@ class OracleEngine:
         pass  # the oracle derives states from the definition whenever they are asked for
 
     def _tier_size(self, tier):
-        return self.n_hbm_blocks if tier == TIER_HBM else self.n_host_blocks
+        return (self.n_hbm_blocks, self.n_host_blocks, self.n_remote_blocks)[tier]
 
     def get_states(self, tier):
         st = np.zeros(self._tier_size(tier), np.uint8)
@@ -229,6 +233,11 @@ class OracleEngine:
         s = _u32(slots); nd = C.c_uint32(0)
         rc = self.L.kvto_reload(self.h, _p(s), len(s), C.byref(nd))
         return rc, nd.value
+
+    def move(self, src_tier, dst_tier, slots):
+        s = _u32(slots); nd = C.c_uint32(0); nx = C.c_uint32(0)
+        rc = self.L.kvto_move(self.h, src_tier, dst_tier, _p(s), len(s), C.byref(nd), C.byref(nx))
+        return rc, nd.value, nx.value
 
     def exchange(self, out_slots, in_slots):
         o, i = _u32(out_slots), _u32(in_slots)
@@ -288,7 +297,7 @@ class OracleEngine:
         if tier == TIER_HBM and self.pool_layout == LAYOUT_LAYER_MAJOR:
             v = self.hbm_pool.reshape(self.n_chunks, self.n_hbm_blocks, self.chunk_bytes)
             return v[:, slot, :]
-        pool = self.hbm_pool if tier == TIER_HBM else self.host_pool
+        pool = (self.hbm_pool, self.host_pool, self.remote_pool)[tier]
         return pool.reshape(-1, self.n_chunks, self.chunk_bytes)[slot]
 
     def write_block(self, tier, slot, payload):

@@ -13,7 +13,7 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkvt.so")
 
 OK, E_INVAL, E_NOCTX, E_RANGE, E_STATE, E_NOSPACE, E_BUFSZ, E_DEVICE, E_CUDA = 0, -1, -2, -3, -4, -5, -6, -7, -8
-TIER_HBM, TIER_HOST, TIER_NONE = 0, 1, 0xFF
+TIER_HBM, TIER_HOST, TIER_REMOTE, TIER_NONE = 0, 1, 2, 0xFF
 LAYOUT_LAYER_MAJOR, LAYOUT_BLOCK_MAJOR = 0, 1
 ORDER_MRU, ORDER_LRU = 0, 1
 POLICY_NO_LIFECYCLE, POLICY_INCLUSIVE, POLICY_ORPHANS_DEAD = 1, 2, 4

@@ -18,7 +18,7 @@ from dataclasses import dataclass, field
 import numpy as np
 
 VOCAB = 151552
-TIER_HBM, TIER_HOST, TIER_NONE = 0, 1, 0xFF
+TIER_HBM, TIER_HOST, TIER_REMOTE, TIER_NONE = 0, 1, 2, 0xFF
 MAP_LOOKUP, MAP_ADMIT = 0, 1
 GiB = 1 << 30
 GPU_ONLY_STATS = ("table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns", "mover_bytes",

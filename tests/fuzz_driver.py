@@ -4,10 +4,19 @@ import numpy as np
 
 from paper_2609_39819_b200 import workloads as W
 
-HBM, HOST = 0, 1
+HBM, HOST, REMOTE = 0, 1, 2
 OPS = ("append", "append", "append", "replace", "remove", "one_off_ctx", "one_off_msg", "pin", "unpin", "fork", "spawn",
        "terminate", "call", "call", "call", "lookup_only", "admit_only", "prefill_done", "evict", "evict_pinned",
        "release_hbm", "release_host", "reload_some", "compact_hbm", "compact_host", "exchange", "exchange", "bad")
+OPS_REMOTE = ("demote", "demote", "promote_host", "promote_hbm", "release_remote", "compact_remote", "bad_move")
+
+
+def tiers(eng):
+    return (HBM, HOST, REMOTE) if getattr(eng, "n_remote_blocks", 0) else (HBM, HOST)
+
+
+def tier_size(eng, tier):
+    return (eng.n_hbm_blocks, eng.n_host_blocks, getattr(eng, "n_remote_blocks", 0))[tier]
 
 
 def payload(key, nbytes):
@@ -17,7 +26,7 @@ def payload(key, nbytes):
 def observe(eng):
     """Everything an engine lets a caller see, as a comparable structure."""
     out = {"stats": {k: v for k, v in eng.get_stats().items() if k not in W.GPU_ONLY_STATS}}
-    for tier in (HBM, HOST):
+    for tier in tiers(eng):
         out[f"states{tier}"] = eng.get_states(tier)
         out[f"entries{tier}"] = eng.get_entries(tier)
     return out
@@ -27,7 +36,7 @@ def check_payload(eng):
     """Every occupied slot (blocks and clean copies) holds the payload of its key."""
     if eng.metadata_only:
         return True
-    for tier in (HBM, HOST):
+    for tier in tiers(eng):
         keys = eng.get_entries(tier)["key"]
         for s in np.nonzero(keys)[0]:
             if not np.array_equal(eng.read_block(tier, int(s)), payload(keys[s], eng.block_bytes)):
@@ -37,11 +46,11 @@ def check_payload(eng):
 
 def check_invariants(eng, inclusive):
     st = eng.get_stats()
-    ent = [eng.get_entries(HBM), eng.get_entries(HOST)]
-    states = [eng.get_states(HBM), eng.get_states(HOST)]
-    for tier, n in ((HBM, eng.n_hbm_blocks), (HOST, eng.n_host_blocks)):
+    ent = [eng.get_entries(t) for t in tiers(eng)]
+    states = [eng.get_states(t) for t in tiers(eng)]
+    for tier in tiers(eng):
         occ = int((ent[tier]["key"] != 0).sum())
-        assert occ == st["occ_hbm" if tier == HBM else "occ_host"] <= n
+        assert occ == st[("occ_hbm", "occ_host", "occ_remote")[tier]] <= tier_size(eng, tier)
         assert np.all((states[tier] == 0xFF) == (ent[tier]["key"] == 0))
         assert np.all(ent[tier]["inflight"][ent[tier]["key"] == 0] == 0)
     copies = states[HOST] == 0xFE
@@ -51,11 +60,12 @@ def check_invariants(eng, inclusive):
     for h in np.nonzero(copies)[0]:
         b = int(ent[HOST]["link"][h])
         assert int(ent[HBM]["link"][b]) == h and ent[HBM]["key"][b] == ent[HOST]["key"][h]
-    prim = np.concatenate([ent[HBM]["key"][ent[HBM]["key"] != 0], ent[HOST]["key"][(ent[HOST]["key"] != 0) & ~copies]])
+    prim = np.concatenate([ent[HBM]["key"][ent[HBM]["key"] != 0], ent[HOST]["key"][(ent[HOST]["key"] != 0) & ~copies]] +
+                          [ent[t]["key"][ent[t]["key"] != 0] for t in tiers(eng)[2:]])
     assert len(np.unique(prim)) == len(prim)
-    assert st["hits_hbm"] + st["hits_host"] + st["misses"] == st["blocks_hashed"]
+    assert st["hits_hbm"] + st["hits_host"] + st["hits_remote"] + st["misses"] == st["blocks_hashed"]
     if hasattr(eng, "classify_bruteforce"):
-        for tier in (HBM, HOST):
+        for tier in tiers(eng):
             assert np.array_equal(states[tier], eng.classify_bruteforce(tier))
 
 
@@ -96,7 +106,7 @@ class Fuzzer:
 
     def step(self):
         r = self.rng
-        op = str(r.choice(OPS))
+        op = str(r.choice(OPS + OPS_REMOTE if len(tiers(self.engs[0])) == 3 else OPS))
         self.log.append(op)
         E = self.engs[0]
         if op == "spawn":
@@ -153,7 +163,7 @@ class Fuzzer:
                 if need:
                     self.evict(need, False)
             if op == "call" and r.random() < 0.7:        # bring the host-tier part of the prefixes back
-                hs = []
+                hs, rs = [], []
                 for c in ctxs:
                     if c in self.n_msgs:
                         try:
@@ -161,9 +171,13 @@ class Fuzzer:
                         except Exception:
                             continue
                         hs += [int(x) for x, t in zip(slot, tier) if t == HOST]
+                        rs += [int(x) for x, t in zip(slot, tier) if t == REMOTE]
                 if hs:
                     hs = list(dict.fromkeys(hs))
                     self.all_rc(lambda e: e.reload(hs))
+                if rs:
+                    rs = list(dict.fromkeys(rs))
+                    self.all_rc(lambda e: e.move(REMOTE, HBM, rs))
             if op != "lookup_only":
                 rc, info = self.all_rc(lambda e: e.map_blocks_rc(ctxs, 1))
                 if rc == 0:
@@ -200,9 +214,27 @@ class Fuzzer:
             if r.random() < 0.1:
                 out = list(out) + [int(r.integers(0, E.n_hbm_blocks + 2))]
             self.all_rc(lambda e: e.exchange(out, inn))
-        elif op in ("compact_hbm", "compact_host"):
-            tier = HBM if op == "compact_hbm" else HOST
+        elif op in ("compact_hbm", "compact_host", "compact_remote"):
+            tier = {"compact_hbm": HBM, "compact_host": HOST, "compact_remote": REMOTE}[op]
             self.all_rc(lambda e: e.compact(tier))
+        elif op in ("demote", "promote_host", "promote_hbm"):
+            src, dst = {"demote": (HOST, REMOTE), "promote_host": (REMOTE, HOST), "promote_hbm": (REMOTE, HBM)}[op]
+            n = tier_size(E, src)
+            slots = r.integers(0, n + 1, int(r.integers(0, 4)))
+            occ = np.nonzero(E.get_entries(src)["key"])[0]
+            if len(occ) and r.random() < 0.85:
+                slots = r.choice(occ, size=min(len(occ), int(r.integers(1, 6))), replace=False)
+            if op == "demote" and r.random() < 0.5:       # the usual way down: the host tier's own victims
+                k = int(r.integers(1, 6))
+                slots, _s = self.all_rc(lambda e: e.select_victims(HOST, k))
+            self.all_rc(lambda e: e.move(src, dst, slots))
+        elif op == "release_remote":
+            occ = np.nonzero(E.get_entries(REMOTE)["key"])[0]
+            slots = r.choice(occ, size=min(len(occ), int(r.integers(1, 4))), replace=False) if len(occ) else [0]
+            self.all_rc(lambda e: e.release_rc(REMOTE, slots))
+        elif op == "bad_move":
+            src, dst = [(HBM, REMOTE), (REMOTE, REMOTE), (HBM, HBM), (3, 0), (HOST, HOST)][int(r.integers(0, 5))]
+            self.all_rc(lambda e: e.move(src, dst, [0]))
         elif op == "bad":
             which = int(r.integers(0, 4))
             if which == 0:

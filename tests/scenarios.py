@@ -749,8 +749,74 @@ def orphans_are_dead(make):
         eng.prefill_done(0)
 
 
+# ---- three tiers: HBM, host memory, remote memory (Section 7) ------------------------------------------
+REMOTE = 2
+
+
+def three_tiers(make):
+    eng = make(n_hbm_blocks=6, n_host_blocks=3, n_remote_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(22)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 96))
+    call(eng, 0)                                         # blocks 0..5 at HBM slots 0..5
+    keys = eng.get_block_map(0)[0]
+    for b in range(6):
+        eng.write_block(HBM, b, _payload(keys[b], eng.block_bytes))
+    assert eng.offload([5, 4, 3]) == (0, 3, 0)           # host slots 0, 1, 2 hold blocks 5, 4, 3
+    v, s = eng.select_victims(HOST, 2)                   # same stamp everywhere: the chain's tail goes first
+    assert list(v) == [0, 1] and list(s) == [IDLE, IDLE]
+    assert eng.move(HOST, REMOTE, v) == (0, 2, 0)        # remote slots 0 (block 5) and 1 (block 4)
+    st = eng.get_stats()
+    assert (st["occ_hbm"], st["occ_host"], st["occ_remote"], st["demoted"]) == (3, 1, 2, 2)
+    assert states(eng, REMOTE) == [IDLE, IDLE, FREE, FREE]
+    a = eng.map_blocks([0], LOOKUP)[0]
+    assert (a["hit_len"], a["n_hit_hbm"], a["n_hit_host"], a["n_hit_remote"]) == (6, 3, 1, 2)
+    _k, tier, slot = eng.get_block_map(0)
+    assert list(tier) == [0, 0, 0, 1, 2, 2] and list(slot) == [0, 1, 2, 2, 1, 0]
+    assert states(eng, REMOTE)[:2] == [ACTIVE, ACTIVE]
+    assert eng.move(HOST, REMOTE, [2])[0] < 0            # a block in flight does not move down
+    assert eng.move(REMOTE, HBM, [1, 0]) == (0, 2, 0)    # straight up: block 4 -> HBM slot 3, block 5 -> slot 4
+    assert eng.reload([2]) == (0, 1)                     # block 3 -> HBM slot 5
+    _k, tier, slot = eng.get_block_map(0)
+    assert list(tier) == [0] * 6 and list(slot) == [0, 1, 2, 5, 3, 4]
+    for b in range(6):
+        assert np.array_equal(eng.read_block(HBM, int(slot[b])), _payload(keys[b], eng.block_bytes)), b
+    st = eng.get_stats()
+    assert (st["occ_hbm"], st["occ_host"], st["occ_remote"], st["promoted"], st["reloaded"]) == (6, 0, 0, 2, 1)
+    eng.map_blocks([0], ADMIT)
+    eng.prefill_done(0)
+    # down again, one level at a time, then one level up; dead blocks are dropped on the way down
+    assert eng.offload([4, 3]) == (0, 2, 0)              # blocks 5, 4 -> host slots 0, 1
+    assert eng.move(HOST, REMOTE, [0, 1]) == (0, 2, 0)   # -> remote slots 0, 1
+    assert eng.move(REMOTE, HOST, [1]) == (0, 1, 0)      # block 4 back to host slot 0
+    assert states(eng, HOST) == [IDLE, FREE, FREE] and states(eng, REMOTE) == [IDLE, FREE, FREE, FREE]
+    assert np.array_equal(eng.read_block(HOST, 0), _payload(keys[4], eng.block_bytes))
+    assert np.array_equal(eng.read_block(REMOTE, 0), _payload(keys[5], eng.block_bytes))
+    eng.remove(0, 0, 1)                                  # everything dies
+    assert eng.move(HOST, REMOTE, [0]) == (0, 1, 1)      # dropped, not copied
+    v, s = eng.select_victims(REMOTE, 4)
+    assert list(v) == [0] and list(s) == [DEAD]
+    eng.release(REMOTE, v)
+    st = eng.get_stats()
+    assert (st["occ_host"], st["occ_remote"], st["promoted"], st["demoted"]) == (0, 0, 3, 4)
+    # pairs that skip a level on the way down, and bad slots, are rejected
+    assert eng.move(HBM, REMOTE, [0])[0] < 0 and eng.move(REMOTE, REMOTE, [0])[0] < 0
+    assert eng.move(REMOTE, HOST, [0])[0] < 0 and eng.move(REMOTE, HOST, [9])[0] < 0
+    # the remote tier fills up: the move stops there and reports how far it got
+    eng.release(HBM, [0, 1, 2, 5])                       # the dead blocks 0..3 of the first context
+    eng.spawn(1)
+    eng.append(1, toks(rng, 96))
+    call(eng, 1)                                         # six new blocks at HBM slots 0..5
+    assert eng.offload([0, 1, 2]) == (0, 3, 0)
+    assert eng.move(HOST, REMOTE, [0, 1, 2]) == (0, 3, 0)
+    assert eng.offload([3, 4, 5]) == (0, 3, 0)
+    rc, n_done, n_dropped = eng.move(HOST, REMOTE, [0, 1, 2])
+    assert rc < 0 and (n_done, n_dropped) == (1, 0)      # one remote slot was left
+    assert eng.get_stats()["occ_remote"] == 4
+
+
 ALL = [state_machine_single_context, suffix_invalidation, fork_and_shared_kv, one_off_bypass, worked_example,
        mixed_pool_example, victim_order_bruteforce, one_state_pools_reduce_to_lru, offload_reload_round_trip,
        dead_victims_are_dropped_without_copy, compaction, raw_copy_blocks, admission_stops_when_full,
        lookup_locks_and_orphans, degenerate_inputs, pinned_retention, no_lifecycle_policy, inclusive_tiers, exchange_both_ways,
-       orphans_are_dead]
+       orphans_are_dead, three_tiers]
