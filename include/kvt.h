@@ -9,7 +9,7 @@
  *   (3) derivation of each resident block's KV-level lifecycle state from message-level states
  *       (Section 5.2 state machine; Section 6.1 "Managing Shared KV"),
  *   (4) state-prioritised, recency-ordered victim selection (Algorithm 1; Section 6.2), and
- *   (5) movement of paged KV blocks between the HBM pool and a pinned host tier (Section 7).
+ *   (5) movement of paged KV blocks between the HBM pool, a pinned host tier and an optional third tier (Section 7).
  *
  * General conventions
  *   - Plain C, no exceptions, no stdout. Every function returns an int32_t status: KVT_OK (0) or a
@@ -42,7 +42,7 @@
 extern "C" {
 #endif
 
-#define KVT_ABI_VERSION 1u
+#define KVT_ABI_VERSION 2u
 #define KVT_BLOCK_TOKENS 16u
 
 /* ---- status codes -------------------------------------------------------------------------- */
@@ -57,9 +57,11 @@ extern "C" {
 #define KVT_E_CUDA     -8  /* a CUDA runtime call failed; text via kvt_last_error */
 
 /* ---- enums --------------------------------------------------------------------------------- */
-/* Tiers (Section 7: multi-tier engine; the remote tier is not part of this library). */
+/* Tiers (Section 7: a multi-tier engine spanning GPU HBM, host memory and remote memory). */
 #define KVT_TIER_HBM   0u
 #define KVT_TIER_HOST  1u
+#define KVT_TIER_REMOTE 2u  /* third level of Section 7's hierarchy (remote memory); here one more caller-provided
+                              device-accessible buffer stands in for it: cross-node transport is out of scope */
 #define KVT_TIER_NONE  0xFFu   /* "not resident" in block maps */
 
 /* HBM pool layouts. The host pool is always block-major. */
@@ -139,7 +141,7 @@ typedef struct kvt_config {
   uint32_t pool_layout;      /* KVT_LAYOUT_* of the HBM pool */
   uint32_t n_hbm_blocks;     /* slots in the HBM tier (>= 1) */
   uint32_t n_host_blocks;    /* slots in the host tier (may be 0) */
-  uint32_t table_capacity;   /* power of two, >= 2 * (n_hbm_blocks + n_host_blocks) */
+  uint32_t table_capacity;   /* power of two, >= 2 * (n_hbm_blocks + n_host_blocks + n_remote_blocks) */
   uint32_t max_contexts;     /* context ids are 0 .. max_contexts-1 */
   uint32_t max_messages;     /* upper bound on messages with materialised positions, all contexts together */
   uint32_t max_batch_blocks; /* upper bound on the blocks hashed by one kvt_map_blocks call and on n of one list call */
@@ -148,11 +150,12 @@ typedef struct kvt_config {
   uint64_t max_key_blocks;   /* capacity of the per-context key lists, in blocks (all contexts together) */
   uint64_t hash_seed;        /* seed of the block hash */
   uint32_t suspended_order;  /* KVT_ORDER_* */
-  uint32_t reserved1;        /* must be 0 */
+  uint32_t n_remote_blocks;  /* slots in the remote tier (may be 0) */
   void *hbm_pool;  uint64_t hbm_pool_bytes;   /* device; NULL/0 = metadata-only engine (no payload is moved) */
   void *host_pool; uint64_t host_pool_bytes;  /* device-accessible pinned host memory; NULL/0 if metadata-only */
   void *dev_meta;  uint64_t dev_meta_bytes;   /* device metadata + scratch arena, 256-byte aligned */
   void *dev_tokens; uint64_t dev_tokens_bytes;/* device token arena, 256-byte aligned */
+  void *remote_pool; uint64_t remote_pool_bytes; /* device-accessible memory of the remote tier; NULL/0 if none or metadata-only */
 } kvt_config;
 
 /* Computes the byte sizes the caller must allocate for dev_meta and dev_tokens from the other
@@ -213,6 +216,7 @@ typedef struct kvt_call_info {
   uint32_t n_admitted;    /* ADMIT: blocks this call newly holds (inserted or adopted) */
   uint32_t n_held;        /* leading blocks locked in flight for this context after the call */
   uint32_t n_pinned;      /* of the admissible blocks, those touched by a Pinned message */
+  uint32_t n_hit_remote;  /* of the reusable prefix, blocks resident in the remote tier (kvt_move them up before use) */
 } kvt_call_info;
 
 /* phase KVT_MAP_LOOKUP — one LLM call begins for each listed context (Section 7: call id and
@@ -280,6 +284,16 @@ int32_t kvt_offload(kvt_engine *e, const uint32_t *hbm_slots, uint32_t n, uint32
  * KVT_E_NOSPACE + *n_done when HBM is full. Synchronises. */
 int32_t kvt_reload(kvt_engine *e, const uint32_t *host_slots, uint32_t n, uint32_t *n_done,
                    void *stream);
+
+/* Movement between neighbouring levels of the hierarchy (Section 7: HBM, host memory, remote memory) and straight
+ * up from the remote tier into HBM: (HBM, host) = kvt_offload, (host, HBM) = kvt_reload, (host, remote) moves down
+ * like an offload (dead blocks dropped, live ones to the remote slots that are free when the call begins, lowest
+ * first; blocks in flight and clean copies are rejected), (remote, host) and (remote, HBM) move up like a reload
+ * (i-th listed block to the i-th lowest free slot; blocks in flight allowed; the remote slot is freed, also with
+ * inclusive tiers). Any other pair: KVT_E_INVAL. KVT_E_NOSPACE + counts when the destination fills up.
+ * Host id array. Synchronises. */
+int32_t kvt_move(kvt_engine *e, uint32_t src_tier, uint32_t dst_tier, const uint32_t *slots, uint32_t n,
+                 uint32_t *n_done, uint32_t *n_dropped, void *stream);
 
 /* Reload and offload in one call, for the common step "bring my prefix back and push other blocks out": the
  * listed host slots move to the HBM slots that are free when the call begins (as kvt_reload does), the listed
@@ -360,6 +374,10 @@ typedef struct kvt_stats {
   uint64_t select_slots;     /* and the tier slots they scanned */
   uint64_t offloaded_clean;  /* of `offloaded`, blocks handed to an existing clean host copy (no bytes moved) */
   uint64_t blocks_rehashed;  /* of `blocks_hashed`, blocks whose digest was actually recomputed (the rest kept their keys) */
+  uint64_t occ_remote;       /* occupied slots of the remote tier */
+  uint64_t hits_remote;      /* reusable-prefix blocks found in the remote tier */
+  uint64_t demoted;          /* blocks moved host -> remote */
+  uint64_t promoted;         /* blocks moved remote -> host or remote -> HBM */
 } kvt_stats;
 int32_t kvt_get_stats(kvt_engine *e, kvt_stats *out);
 

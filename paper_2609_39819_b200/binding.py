@@ -27,7 +27,7 @@ EXPORTS = ("kvt_query_sizes", "kvt_create", "kvt_destroy", "kvt_apply_op", "kvt_
            "kvt_classify", "kvt_get_states", "kvt_select_victims", "kvt_offload", "kvt_reload", "kvt_release",
            "kvt_compact", "kvt_copy_blocks", "kvt_hash_scratch_bytes", "kvt_hash_tokens", "kvt_get_stats",
            "kvt_last_error", "kvt_get_entries", "kvt_debug_load_resident", "kvt_set_profiling",
-           "kvt_hash_tokens_noalloc", "kvt_debug_set_mover_variant", "kvt_exchange", "kvt_debug_set_lookup_variant")
+           "kvt_hash_tokens_noalloc", "kvt_debug_set_mover_variant", "kvt_exchange", "kvt_debug_set_lookup_variant", "kvt_move")
 
 
 class KvtError(RuntimeError):
@@ -42,11 +42,12 @@ class Config(C.Structure):
                                            "table_capacity", "max_contexts", "max_messages", "max_batch_blocks",
                                            "policy_flags")] + \
                [("max_tokens", C.c_uint64), ("max_key_blocks", C.c_uint64), ("hash_seed", C.c_uint64),
-                ("suspended_order", C.c_uint32), ("reserved1", C.c_uint32),
+                ("suspended_order", C.c_uint32), ("n_remote_blocks", C.c_uint32),
                 ("hbm_pool", C.c_void_p), ("hbm_pool_bytes", C.c_uint64),
                 ("host_pool", C.c_void_p), ("host_pool_bytes", C.c_uint64),
                 ("dev_meta", C.c_void_p), ("dev_meta_bytes", C.c_uint64),
-                ("dev_tokens", C.c_void_p), ("dev_tokens_bytes", C.c_uint64)]
+                ("dev_tokens", C.c_void_p), ("dev_tokens_bytes", C.c_uint64),
+                ("remote_pool", C.c_void_p), ("remote_pool_bytes", C.c_uint64)]
 
 
 class Op(C.Structure):
@@ -55,12 +56,13 @@ class Op(C.Structure):
 
 
 CALL_INFO_DTYPE = np.dtype([(n, np.uint32) for n in ("n_blocks", "hit_len", "n_hit_hbm", "n_hit_host",
-                                                       "n_admissible", "n_admitted", "n_held", "n_pinned")])
+                                                       "n_admissible", "n_admitted", "n_held", "n_pinned",
+                                                       "n_hit_remote")])
 STATS_FIELDS = ("clock", "n_contexts", "occ_hbm", "occ_host", "blocks_hashed", "hits_hbm", "hits_host", "misses",
                 "inserted", "adopted", "dropped", "offloaded", "reloaded", "compacted", "bytes_d2h", "bytes_h2d",
                 "bytes_d2d", "table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns",
                 "mover_bytes", "lookup_ns", "lookup_blocks", "select_ns", "select_slots", "offloaded_clean",
-                "blocks_rehashed")
+                "blocks_rehashed", "occ_remote", "hits_remote", "demoted", "promoted")
 
 _lib = None
 
@@ -91,6 +93,7 @@ def load_library():
             "kvt_offload": [vp, vp, u32, vp, vp, vp],
             "kvt_reload": [vp, vp, u32, vp, vp],
             "kvt_exchange": [vp, vp, u32, vp, u32, vp, vp, vp, vp],
+            "kvt_move": [vp, u32, u32, vp, u32, vp, vp, vp],
             "kvt_release": [vp, u32, vp, u32, vp],
             "kvt_compact": [vp, u32, vp, vp],
             "kvt_copy_blocks": [vp, u32, vp, u32, vp, u32, u32, vp],
@@ -161,7 +164,7 @@ class Engine:
                  n_hbm_blocks=128, n_host_blocks=512, max_contexts=64, hash_seed=0, suspended_order=ORDER_MRU,
                  metadata_only=False, table_capacity=None, max_messages=1 << 16, max_batch_blocks=None,
                  max_tokens=1 << 22, max_key_blocks=None, host_pool_on_device=False, zero_pools=True, policy_flags=0,
-                 device="cuda"):
+                 n_remote_blocks=0, device="cuda"):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2609_39819_b200 needs a CUDA device (there is no CPU fallback)")
@@ -170,12 +173,12 @@ class Engine:
         self.device = torch.device(device)
         self.n_layers, self.n_kv_heads, self.head_dim, self.elem_bytes = n_layers, n_kv_heads, head_dim, elem_bytes
         self.pool_layout = pool_layout
-        self.n_hbm_blocks, self.n_host_blocks = n_hbm_blocks, n_host_blocks
+        self.n_hbm_blocks, self.n_host_blocks, self.n_remote_blocks = n_hbm_blocks, n_host_blocks, n_remote_blocks
         self.chunk_bytes = 16 * n_kv_heads * head_dim * elem_bytes
         self.n_chunks = 2 * n_layers
         self.block_bytes = self.chunk_bytes * self.n_chunks
         self.metadata_only = metadata_only
-        n_total = n_hbm_blocks + n_host_blocks
+        n_total = n_hbm_blocks + n_host_blocks + n_remote_blocks
         if table_capacity is None:
             table_capacity = 1 << max(4, (2 * n_total - 1).bit_length())
         if max_batch_blocks is None:
@@ -183,9 +186,10 @@ class Engine:
         if max_key_blocks is None:
             max_key_blocks = max(max_tokens // 8, 64)
         cfg = Config()
-        cfg.abi_version, cfg.block_tokens = 1, 16
+        cfg.abi_version, cfg.block_tokens = 2, 16
         cfg.n_layers, cfg.n_kv_heads, cfg.head_dim, cfg.elem_bytes = n_layers, n_kv_heads, head_dim, elem_bytes
         cfg.pool_layout, cfg.n_hbm_blocks, cfg.n_host_blocks = pool_layout, n_hbm_blocks, n_host_blocks
+        cfg.n_remote_blocks = n_remote_blocks
         cfg.table_capacity, cfg.max_contexts, cfg.max_messages = table_capacity, max_contexts, max_messages
         cfg.max_batch_blocks, cfg.max_tokens, cfg.max_key_blocks = max_batch_blocks, max_tokens, max_key_blocks
         cfg.hash_seed, cfg.suspended_order, cfg.policy_flags = hash_seed, suspended_order, policy_flags
@@ -198,7 +202,7 @@ class Engine:
         cfg.dev_meta, cfg.dev_meta_bytes = self._align(self.meta), mb.value
         cfg.dev_tokens, cfg.dev_tokens_bytes = self._align(self.tokens), tb.value
         if metadata_only:
-            self.hbm_pool = self.host_pool = None
+            self.hbm_pool = self.host_pool = self.remote_pool = None
         else:
             new = torch.zeros if zero_pools else torch.empty
             self.hbm_pool = new(n_hbm_blocks * self.block_bytes, dtype=torch.uint8, device=self.device)
@@ -209,6 +213,14 @@ class Engine:
                 self.host_pool = new(nh, dtype=torch.uint8, pin_memory=True)
             cfg.hbm_pool, cfg.hbm_pool_bytes = self.hbm_pool.data_ptr(), self.hbm_pool.numel()
             cfg.host_pool, cfg.host_pool_bytes = self.host_pool.data_ptr(), self.host_pool.numel()
+            # the remote tier is stood in for by one more buffer of the same kind as the host tier
+            nr = max(n_remote_blocks, 1) * self.block_bytes
+            if host_pool_on_device:
+                self.remote_pool = new(nr, dtype=torch.uint8, device=self.device)
+            else:
+                self.remote_pool = new(nr, dtype=torch.uint8, pin_memory=True)
+            if n_remote_blocks:
+                cfg.remote_pool, cfg.remote_pool_bytes = self.remote_pool.data_ptr(), self.remote_pool.numel()
         self.cfg = cfg
         h = C.c_void_p()
         rc = self.L.kvt_create(C.byref(cfg), _stream(), C.byref(h))
@@ -224,7 +236,7 @@ class Engine:
         if getattr(self, "h", None):
             self.L.kvt_destroy(self.h)
             self.h = None
-            self.hbm_pool = self.host_pool = self.meta = self.tokens = None   # release the memory
+            self.hbm_pool = self.host_pool = self.remote_pool = self.meta = self.tokens = None   # release the memory
 
     def __del__(self):
         try:
@@ -309,7 +321,7 @@ class Engine:
         self._check(self.L.kvt_classify(self.h, _stream()), "classify")
 
     def _tier_size(self, tier):
-        return self.n_hbm_blocks if tier == TIER_HBM else self.n_host_blocks
+        return (self.n_hbm_blocks, self.n_host_blocks, self.n_remote_blocks)[tier]
 
     def get_states(self, tier):
         st = np.zeros(self._tier_size(tier), np.uint8)
@@ -334,6 +346,12 @@ class Engine:
         s = _u32(slots); nd = C.c_uint32(0)
         rc = self.L.kvt_reload(self.h, _p(s), len(s), C.byref(nd), _stream())
         return rc, nd.value
+
+    def move(self, src_tier, dst_tier, slots):
+        s = _u32(slots)
+        nd, nx = C.c_uint32(0), C.c_uint32(0)
+        rc = self.L.kvt_move(self.h, src_tier, dst_tier, _p(s), len(s), C.byref(nd), C.byref(nx), _stream())
+        return rc, nd.value, nx.value
 
     def exchange(self, out_slots, in_slots):
         o, i = _u32(out_slots), _u32(in_slots)
@@ -389,7 +407,7 @@ class Engine:
     def _chunks(self, tier, slot):
         if tier == TIER_HBM and self.pool_layout == LAYOUT_LAYER_MAJOR:
             return self.hbm_pool.view(self.n_chunks, self.n_hbm_blocks, self.chunk_bytes)[:, slot, :]
-        pool = self.hbm_pool if tier == TIER_HBM else self.host_pool
+        pool = (self.hbm_pool, self.host_pool, self.remote_pool)[tier]
         return pool.view(-1, self.n_chunks, self.chunk_bytes)[slot]
 
     # Device-side counterpart of workloads.payload_pattern for large blocks (harness helpers, torch ops only).

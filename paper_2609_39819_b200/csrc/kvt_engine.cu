@@ -69,7 +69,7 @@ struct Ctx {
   std::vector<Msg> msgs;
   std::vector<std::pair<u32, u32>> mat_bounds;  // bounds of the leading messages still valid in the materialised layout
   u32 mat_blocks = 0;      // blocks of the materialised token sequence (keys in the key segment)
-  u32 valid_blocks = 0, held = 0, hit_len = 0, n_hit_hbm = 0, n_hit_host = 0, n_admissible = 0, n_pinned = 0;
+  u32 valid_blocks = 0, held = 0, hit_len = 0, n_hit_hbm = 0, n_hit_host = 0, n_hit_remote = 0, n_admissible = 0, n_pinned = 0;
   u64 tok_off = 0, tok_cap = 0, tok_len = 0;   // device token buffer = concatenation of the current messages
   int keyseg = -1;
 };
@@ -84,7 +84,8 @@ struct DevLayout {
 
 DevLayout make_layout(const kvt_config &c) {
   DevLayout L{};
-  u64 N = (u64)c.n_hbm_blocks + c.n_host_blocks, Nt = std::max(c.n_hbm_blocks, c.n_host_blocks);
+  u64 N = (u64)c.n_hbm_blocks + c.n_host_blocks + c.n_remote_blocks;
+  u64 Nt = std::max(std::max(c.n_hbm_blocks, c.n_host_blocks), c.n_remote_blocks);
   u64 B = c.max_batch_blocks, LB = std::max<u64>(B, Nt), C = c.max_contexts, Mm = c.max_messages;
   L.LB = LB; L.Nt = Nt; L.N = N;
   u64 off = 0;
@@ -102,7 +103,7 @@ DevLayout make_layout(const kvt_config &c) {
   L.agg = take(n_chunks * 8); L.carry = take(n_chunks * 8);   // per-chunk aggregates / chain values of a LOOKUP batch
   L.cflags = take((n_chunks + 1) * 4);                         // per-chunk publication flags + the ticket word
   L.desc = take(C * 64);
-  L.ctxres = take(C * 16);
+  L.ctxres = take(C * 20);   // per context: hit_len, hits per tier (3), admission stop
   L.m_start = take(Mm * 4); L.m_end = take(Mm * 4); L.m_rank = take(Mm);
   L.keyA = take(Nt * 8); L.keyB = take(Nt * 8); L.valA = take(Nt * 4); L.valB = take(Nt * 4);
   L.rcounts = take((256ull * (Nt / SORT_TILE + 1) + 256) * 4);
@@ -131,7 +132,7 @@ struct kvt_engine {
   std::vector<int> free_segs;
   RangeAlloc tok_alloc, key_alloc;
   u32 now = 0, max_depth = 0;
-  u32 occ[2] = {0, 0};
+  u32 occ[3] = {0, 0, 0};
   u32 tombs = 0;
   bool dirty = true;
   kvt_stats st{};
@@ -145,7 +146,7 @@ struct kvt_engine {
   bool profiling = false, mover_timed = false;
   // CUDA graph of the radix-sort passes of kvt_select_victims, one per tier
   struct SortGraph { cudaGraphExec_t exec = nullptr; u32 n_pass = 0; };
-  SortGraph sort_graph[2];
+  SortGraph sort_graph[3];
   cudaStream_t capture_stream = nullptr;   // only ever used for stream capture, never executes work
   bool use_graphs = true;
   u32 mover_variant = 0;   // 0 auto, 1 CTA per chunk, 2 warp per 4 KiB tile, 3 TMA ring
@@ -154,8 +155,8 @@ struct kvt_engine {
   cudaEvent_t ev_m0 = nullptr, ev_m1 = nullptr, ev_h0 = nullptr, ev_h1 = nullptr;
 
   template <class T> T *dp(u64 off) const { return reinterpret_cast<T *>(meta + off); }
-  u32 tier_slots(u32 t) const { return t == KVT_TIER_HBM ? cfg.n_hbm_blocks : cfg.n_host_blocks; }
-  u32 tier_e0(u32 t) const { return t == KVT_TIER_HBM ? 0 : cfg.n_hbm_blocks; }
+  u32 tier_slots(u32 t) const { return t == KVT_TIER_HBM ? cfg.n_hbm_blocks : t == KVT_TIER_HOST ? cfg.n_host_blocks : cfg.n_remote_blocks; }
+  u32 tier_e0(u32 t) const { return t == KVT_TIER_HBM ? 0 : t == KVT_TIER_HOST ? cfg.n_hbm_blocks : cfg.n_hbm_blocks + cfg.n_host_blocks; }
 };
 
 namespace {
@@ -272,8 +273,8 @@ PoolView pool_view(kvt_engine *e, u32 tier) {
     if (e->cfg.pool_layout == KVT_LAYOUT_LAYER_MAJOR) { v.slot_stride = e->chunk_bytes; v.chunk_stride = e->chunk_bytes * e->cfg.n_hbm_blocks; }
     else { v.slot_stride = e->block_bytes; v.chunk_stride = e->chunk_bytes; }
   } else {
-    v.base = (u8 *)e->cfg.host_pool;
-    v.n_slots = e->cfg.n_host_blocks;
+    v.base = (u8 *)(tier == KVT_TIER_HOST ? e->cfg.host_pool : e->cfg.remote_pool);
+    v.n_slots = e->tier_slots(tier);
     v.slot_stride = e->block_bytes; v.chunk_stride = e->chunk_bytes;
   }
   return v;
@@ -458,9 +459,9 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   const kvt_config &c = *cfg;
   if (c.abi_version != KVT_ABI_VERSION || c.block_tokens != 16 || !c.n_layers || !c.n_kv_heads || !c.head_dim ||
       !c.elem_bytes || c.pool_layout > 1 || !c.n_hbm_blocks || !c.max_contexts || !c.max_batch_blocks ||
-      !c.max_messages || c.suspended_order > 1 || c.policy_flags > 7 || c.reserved1 || !c.dev_meta || !c.dev_tokens)
+      !c.max_messages || c.suspended_order > 1 || c.policy_flags > 7 || !c.dev_meta || !c.dev_tokens)
     return KVT_E_INVAL;
-  u64 N = (u64)c.n_hbm_blocks + c.n_host_blocks;
+  u64 N = (u64)c.n_hbm_blocks + c.n_host_blocks + c.n_remote_blocks;
   if (N >= CLAIM_BIT || c.max_batch_blocks >= CLAIM_BIT) return KVT_E_INVAL;
   if (c.table_capacity < 2 * N || (c.table_capacity & (c.table_capacity - 1))) return KVT_E_INVAL;
   if (((uintptr_t)c.dev_meta & 255) || ((uintptr_t)c.dev_tokens & 255)) return KVT_E_INVAL;
@@ -472,6 +473,9 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
     if (c.hbm_pool_bytes < chunk_bytes * n_chunks * c.n_hbm_blocks || ((uintptr_t)c.hbm_pool & 15)) return KVT_E_INVAL;
     if (c.n_host_blocks && (!c.host_pool || c.host_pool_bytes < chunk_bytes * n_chunks * c.n_host_blocks ||
                             ((uintptr_t)c.host_pool & 15)))
+      return KVT_E_INVAL;
+    if (c.n_remote_blocks && (!c.remote_pool || c.remote_pool_bytes < chunk_bytes * n_chunks * c.n_remote_blocks ||
+                              ((uintptr_t)c.remote_pool & 15)))
       return KVT_E_INVAL;
   }
   int dev = 0;
@@ -487,7 +491,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   e->ent.key = e->dp<u64>(L.e_key); e->ent.stamp = e->dp<u32>(L.e_stamp); e->ent.depth = e->dp<u32>(L.e_depth);
   e->ent.infl = e->dp<u32>(L.e_infl); e->ent.rank = e->dp<u32>(L.e_rank); e->ent.tslot = e->dp<u32>(L.e_tslot);
   e->ent.mark = e->dp<u32>(L.e_mark); e->ent.floor = e->dp<u8>(L.e_floor); e->ent.link = e->dp<u32>(L.e_link);
-  e->ent.n_hbm = c.n_hbm_blocks; e->ent.n_total = (u32)N;
+  e->ent.n_hbm = c.n_hbm_blocks; e->ent.n_host = c.n_host_blocks; e->ent.n_total = (u32)N;
   e->d_keys = e->dp<u64>(L.keys); e->d_status = e->dp<u32>(L.status);
   e->h0 = hash_h0(c.hash_seed);
   e->ctxs.resize(c.max_contexts);
@@ -495,7 +499,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   e->key_alloc.init(c.max_key_blocks + c.max_key_blocks / CHUNK + 64ull * c.max_contexts, 32);
   // pinned staging
   u64 C = c.max_contexts, Mm = c.max_messages, LB = L.LB;
-  u64 o_status = 0, o_desc = 256, o_ctxres = o_desc + round_up(C * 64, 256), o_ms = o_ctxres + round_up(C * 16, 256),
+  u64 o_status = 0, o_desc = 256, o_ctxres = o_desc + round_up(C * 64, 256), o_ms = o_ctxres + round_up(C * 20, 256),
       o_me = o_ms + round_up(Mm * 4, 256), o_mr = o_me + round_up(Mm * 4, 256), o_ids = o_mr + round_up(Mm, 256),
       o_ids2 = o_ids + round_up(LB * 4, 256), o_out = o_ids2 + round_up(LB * 4, 256),
       total = o_out + round_up(LB * 16, 256);
@@ -567,7 +571,7 @@ int32_t kvt_get_stats(kvt_engine *e, kvt_stats *out) {
   s.clock = e->now;
   s.n_contexts = 0;
   for (const Ctx &c : e->ctxs) s.n_contexts += c.live;
-  s.occ_hbm = e->occ[0]; s.occ_host = e->occ[1];
+  s.occ_hbm = e->occ[0]; s.occ_host = e->occ[1]; s.occ_remote = e->occ[2];
   s.tombstones = e->tombs;
   *out = s;
   return KVT_OK;
@@ -751,7 +755,8 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
   HashCtx *hd = reinterpret_cast<HashCtx *>(e->h_desc);
   std::vector<int> dev_idx(n_ctx, -1);
   u32 nd = 0, chunk_base = 0, dchunk_base = 0, blk_base = 0;
-  u32 *h_hit = e->h_ctxres, *h_hbm = e->h_ctxres + e->cfg.max_contexts, *h_host = e->h_ctxres + 2 * e->cfg.max_contexts;
+  u32 *h_hit = e->h_ctxres, *h_hbm = e->h_ctxres + e->cfg.max_contexts, *h_host = e->h_ctxres + 2 * e->cfg.max_contexts,
+      *h_remote = e->h_ctxres + 3 * e->cfg.max_contexts;
   for (u32 i = 0; i < n_ctx; ++i) {
     Ctx &c = e->ctxs[ids[i]];
     for (Msg &m : c.msgs) if (m.state == MS_SUSPENDED) m.state = MS_ACTIVE;  // reactivation (Section 5.2)
@@ -779,7 +784,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
       d.tok_off = c.tok_off; d.key_off = sg.off; d.carry_off = sg.off + sg.keycap;
       d.old_key_off = old_key_off; d.old_carry_off = old_carry_off;
       d.n_blocks = nb; d.first = first; d.chunk_base = chunk_base; d.dchunk_base = dchunk_base; d.blk_base = blk_base; d.pad = 0;
-      h_hit[nd] = nb; h_hbm[nd] = 0; h_host[nd] = 0;
+      h_hit[nd] = nb; h_hbm[nd] = 0; h_host[nd] = 0; h_remote[nd] = 0;
       dev_idx[i] = (int)nd;
       hd[nd++] = d;
       chunk_base += cdiv(nb, CHUNK);
@@ -794,7 +799,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     const u32 C = e->cfg.max_contexts;
     CU(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nd * sizeof(HashCtx), cudaMemcpyHostToDevice, s));
     CU(cudaMemcpyAsync(d_res, h_hit, nd * 4, cudaMemcpyHostToDevice, s));
-    CU(cudaMemsetAsync(d_res + C, 0, 2ull * C * 4, s));
+    CU(cudaMemsetAsync(d_res + C, 0, 3ull * C * 4, s));
     r = status_zero(e, s);
     if (r) return r;
     HashArgs ha;
@@ -803,7 +808,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     LookupArgs la;
     la.tab = e->tab; la.b_ent = e->dp<u32>(e->L.s0); la.hit_len = d_res; la.status = e->d_status;
     LockArgs lk;
-    lk.ent = e->ent; lk.b_ent = la.b_ent; lk.hit_len = d_res; lk.n_hbm = d_res + C; lk.n_host = d_res + 2 * C;
+    lk.ent = e->ent; lk.b_ent = la.b_ent; lk.hit_len = d_res; lk.n_hbm = d_res + C; lk.n_host = d_res + 2 * C; lk.n_remote = d_res + 3 * C;
     lk.now = e->now; lk.status = e->d_status;
     if (e->profiling) CU(cudaEventRecord(e->ev_h0, s));
     if (e->lookup_variant != 2) {
@@ -820,7 +825,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     KL(k_lock_hits, chunk_base, CHUNK, s, ha, lk);
     if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));
     LAUNCH_CHECK();
-    CU(cudaMemcpyAsync(h_hit, d_res, 3ull * C * 4, cudaMemcpyDeviceToHost, s));
+    CU(cudaMemcpyAsync(h_hit, d_res, 4ull * C * 4, cudaMemcpyDeviceToHost, s));
     r = status_fetch(e, s);
     if (r) return r;
     if (e->profiling) {
@@ -836,6 +841,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     c.hit_len = k >= 0 ? h_hit[k] : 0;
     c.n_hit_hbm = k >= 0 ? h_hbm[k] : 0;
     c.n_hit_host = k >= 0 ? h_host[k] : 0;
+    c.n_hit_remote = k >= 0 ? h_remote[k] : 0;
     c.held = c.hit_len;
     if (e->cfg.policy_flags & KVT_POLICY_NO_LIFECYCLE) {   // nothing is known to be Temporary or Pinned
       c.n_admissible = c.mat_blocks - c.hit_len;
@@ -845,8 +851,9 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
       c.n_pinned = count_pinned_blocks(c, c.hit_len, c.hit_len + c.n_admissible);
     }
     e->st.blocks_hashed += c.mat_blocks;
-    e->st.hits_hbm += c.n_hit_hbm; e->st.hits_host += c.n_hit_host; e->st.misses += c.mat_blocks - c.hit_len;
-    out[i] = kvt_call_info{c.mat_blocks, c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, 0, c.held, c.n_pinned};
+    e->st.hits_hbm += c.n_hit_hbm; e->st.hits_host += c.n_hit_host; e->st.hits_remote += c.n_hit_remote;
+    e->st.misses += c.mat_blocks - c.hit_len;
+    out[i] = kvt_call_info{c.mat_blocks, c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, 0, c.held, c.n_pinned, c.n_hit_remote};
   }
   return KVT_OK;
 }
@@ -867,17 +874,17 @@ static int32_t map_admit(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_info
     while (first < n_ctx && stopped[first]) ++first;
     if (first == n_ctx) break;
     // claims may fill the table: keep live + tombstones + candidates below 3/4 of the capacity
-    u64 cap = (u64)e->tab.mask + 1, used = (u64)e->occ[0] + e->occ[1] + e->tombs;
+    u64 cap = (u64)e->tab.mask + 1, used = (u64)e->occ[0] + e->occ[1] + e->occ[2] + e->tombs;
     if (used + 1 > cap * 3 / 4 || (e->tombs && used + e->cfg.max_batch_blocks > cap * 3 / 4)) {
       rc = table_rebuild(e, s);
       if (rc) break;
-      used = (u64)e->occ[0] + e->occ[1];
+      used = (u64)e->occ[0] + e->occ[1] + e->occ[2];
     }
     u64 budget = std::min<u64>(cap * 3 / 4 - used, e->cfg.max_batch_blocks);
     rc = stage_acquire(e);
     if (rc) break;
     AdmitCtx *hd = reinterpret_cast<AdmitCtx *>(e->h_desc);
-    u32 *h_stop = e->h_ctxres + 3 * C;
+    u32 *h_stop = e->h_ctxres + 4 * C;
     u32 nd = 0, n_cand = 0;
     std::vector<u32> who;
     for (u32 i = first; i < n_ctx && n_cand < budget; ++i) {
@@ -896,7 +903,7 @@ static int32_t map_admit(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_info
     AdmitArgs a;
     a.tab = e->tab; a.ent = e->ent; a.keys = e->d_keys; a.ctx = e->dp<AdmitCtx>(e->L.desc); a.n_ctx = nd; a.n_cand = n_cand;
     a.cslot = e->dp<u32>(e->L.s0); a.flag = e->dp<u32>(e->L.s1); a.aux = e->dp<u32>(e->L.s2); a.krank = e->dp<u32>(e->L.s3);
-    a.freelist = e->dp<u32>(e->L.freelist); a.n_free = n_free; a.stop = e->dp<u32>(e->L.ctxres) + 3 * C;
+    a.freelist = e->dp<u32>(e->L.freelist); a.n_free = n_free; a.stop = e->dp<u32>(e->L.ctxres) + 4 * C;
     a.now = e->now; a.status = e->d_status;
     CU(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nd * sizeof(AdmitCtx), cudaMemcpyHostToDevice, s));
     CU(cudaMemcpyAsync(a.stop, h_stop, nd * 4, cudaMemcpyHostToDevice, s));
@@ -933,7 +940,8 @@ static int32_t map_admit(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_info
   for (u32 i = 0; i < n_ctx; ++i) {
     Ctx &c = e->ctxs[ids[i]];
     c.held = cur[i];
-    out[i] = kvt_call_info{c.mat_blocks, c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, cur[i] - held0[i], c.held, c.n_pinned};
+    out[i] = kvt_call_info{c.mat_blocks, c.hit_len, c.n_hit_hbm, c.n_hit_host, c.n_admissible, cur[i] - held0[i], c.held, c.n_pinned,
+                           c.n_hit_remote};
   }
   return rc;
 }
@@ -995,7 +1003,7 @@ int32_t kvt_classify(kvt_engine *e, void *stream) {
 }
 
 int32_t kvt_get_states(kvt_engine *e, uint32_t tier, uint8_t *state, uint32_t cap, void *stream) {
-  if (!e || !state || tier > 1) return KVT_E_INVAL;
+  if (!e || !state || tier > 2) return KVT_E_INVAL;
   u32 n = e->tier_slots(tier);
   if (cap < n) return KVT_E_BUFSZ;
   if (!n) return KVT_OK;
@@ -1012,7 +1020,7 @@ int32_t kvt_get_states(kvt_engine *e, uint32_t tier, uint8_t *state, uint32_t ca
 
 int32_t kvt_get_entries(kvt_engine *e, uint32_t tier, uint64_t *keys, uint32_t *stamp, uint32_t *depth,
                         uint32_t *inflight, uint32_t *link, uint32_t cap, void *stream) {
-  if (!e || tier > 1) return KVT_E_INVAL;
+  if (!e || tier > 2) return KVT_E_INVAL;
   u32 n = e->tier_slots(tier), e0 = e->tier_e0(tier);
   if (cap < n) return KVT_E_BUFSZ;
   if (!n) return KVT_OK;
@@ -1031,7 +1039,7 @@ int32_t kvt_get_entries(kvt_engine *e, uint32_t tier, uint64_t *keys, uint32_t *
 // ---- stage 4 -----------------------------------------------------------------------------------------------
 int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_t flags, uint32_t *slots_out,
                            uint8_t *states_out, uint32_t cap, uint32_t *n_out, void *stream) {
-  if (!e || tier > 1 || flags > 1 || !n_out || (!slots_out && cap)) return KVT_E_INVAL;
+  if (!e || tier > 2 || flags > 1 || !n_out || (!slots_out && cap)) return KVT_E_INVAL;
   *n_out = 0;
   u32 n = e->tier_slots(tier);
   if (!n || !n_req) return KVT_OK;
@@ -1219,6 +1227,28 @@ int32_t kvt_reload(kvt_engine *e, const uint32_t *host_slots, uint32_t n, uint32
   return r;
 }
 
+int32_t kvt_move(kvt_engine *e, uint32_t src_tier, uint32_t dst_tier, const uint32_t *slots, uint32_t n, uint32_t *n_done,
+                 uint32_t *n_dropped, void *stream) {
+  if (!e || (!slots && n) || !n_done || !n_dropped) return KVT_E_INVAL;
+  *n_done = *n_dropped = 0;
+  if (src_tier == KVT_TIER_HBM && dst_tier == KVT_TIER_HOST) return kvt_offload(e, slots, n, n_done, n_dropped, stream);
+  if (src_tier == KVT_TIER_HOST && dst_tier == KVT_TIER_HBM) return kvt_reload(e, slots, n, n_done, stream);
+  const bool down = src_tier == KVT_TIER_HOST && dst_tier == KVT_TIER_REMOTE;
+  const bool up = src_tier == KVT_TIER_REMOTE && (dst_tier == KVT_TIER_HOST || dst_tier == KVT_TIER_HBM);
+  if (!down && !up) return KVT_E_INVAL;
+  ListMode m{};
+  m.reject_shadow = true;
+  if (down) m.drop_dead = !(e->cfg.policy_flags & KVT_POLICY_NO_LIFECYCLE);
+  else m.allow_inflight = true;
+  ListCounts c;
+  int32_t r = list_op(e, (cudaStream_t)stream, src_tier, dst_tier, slots, n, m, &c);
+  *n_done = c.done; *n_dropped = c.dropped;
+  if (down) e->st.demoted += c.copied; else e->st.promoted += c.copied;
+  if (dst_tier == KVT_TIER_HBM) e->st.bytes_h2d += c.copied * e->block_bytes;
+  if (r == KVT_E_NOSPACE) e->err = "destination tier full";
+  return r;
+}
+
 int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_out, const uint32_t *host_slots_in,
                      uint32_t n_in, uint32_t *n_out_done, uint32_t *n_dropped, uint32_t *n_in_done, void *stream) {
   if (!e || (!hbm_slots_out && n_out) || (!host_slots_in && n_in) || !n_out_done || !n_dropped || !n_in_done) return KVT_E_INVAL;
@@ -1321,7 +1351,7 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
 }
 
 int32_t kvt_release(kvt_engine *e, uint32_t tier, const uint32_t *slots, uint32_t n, void *stream) {
-  if (!e || tier > 1 || (!slots && n)) return KVT_E_INVAL;
+  if (!e || tier > 2 || (!slots && n)) return KVT_E_INVAL;
   ListMode m{};
   m.drop_all = true;
   ListCounts c;
@@ -1329,7 +1359,7 @@ int32_t kvt_release(kvt_engine *e, uint32_t tier, const uint32_t *slots, uint32_
 }
 
 int32_t kvt_compact(kvt_engine *e, uint32_t tier, uint32_t *n_moved, void *stream) {
-  if (!e || tier > 1 || !n_moved) return KVT_E_INVAL;
+  if (!e || tier > 2 || !n_moved) return KVT_E_INVAL;
   *n_moved = 0;
   cudaStream_t s = (cudaStream_t)stream;
   u32 n = e->tier_slots(tier), e0 = e->tier_e0(tier), n_occ = e->occ[tier];
@@ -1360,7 +1390,7 @@ int32_t kvt_compact(kvt_engine *e, uint32_t tier, uint32_t *n_moved, void *strea
 
 int32_t kvt_copy_blocks(kvt_engine *e, uint32_t src_tier, const uint32_t *src, uint32_t dst_tier, const uint32_t *dst,
                         uint32_t n, uint32_t flags, void *stream) {
-  if (!e || src_tier > 1 || dst_tier > 1 || ((!src || !dst) && n)) return KVT_E_INVAL;
+  if (!e || src_tier > 2 || dst_tier > 2 || ((!src || !dst) && n)) return KVT_E_INVAL;
   if (e->metadata_only) return fail(e, KVT_E_INVAL, "copy_blocks on a metadata-only engine");
   if (n == 0) return KVT_OK;
   if (n > e->L.LB) return fail(e, KVT_E_NOSPACE, "list longer than max_batch_blocks");
@@ -1444,7 +1474,7 @@ int32_t kvt_hash_tokens_noalloc(const uint32_t *d_tokens, uint64_t n_tokens, uin
 // ---- debug loader -------------------------------------------------------------------------------------------
 int32_t kvt_debug_load_resident(kvt_engine *e, const uint64_t *keys, const uint8_t *state, const uint32_t *stamp,
                                 const uint32_t *depth, const uint32_t *slot, uint32_t tier, uint32_t n, void *stream) {
-  if (!e || tier > 1 || ((!keys || !state || !stamp || !depth || !slot) && n)) return KVT_E_INVAL;
+  if (!e || tier > 2 || ((!keys || !state || !stamp || !depth || !slot) && n)) return KVT_E_INVAL;
   if (n == 0) return KVT_OK;
   u32 ns = e->tier_slots(tier);
   if (n > ns || n > e->L.LB) return fail(e, KVT_E_INVAL, "more blocks than slots");
@@ -1462,7 +1492,7 @@ int32_t kvt_debug_load_resident(kvt_engine *e, const uint64_t *keys, const uint8
       max_stamp = std::max(max_stamp, stamp[i]); max_d = std::max(max_d, depth[i]);
     }
   }
-  if ((u64)e->occ[0] + e->occ[1] + e->tombs + n > ((u64)e->tab.mask + 1) * 3 / 4) return fail(e, KVT_E_NOSPACE, "table too full");
+  if ((u64)e->occ[0] + e->occ[1] + e->occ[2] + e->tombs + n > ((u64)e->tab.mask + 1) * 3 / 4) return fail(e, KVT_E_NOSPACE, "table too full");
   cudaStream_t s = (cudaStream_t)stream;
   // stage the arrays in scratch: keys -> keyA, state -> out_states, stamp/depth/slot -> s1/s2/s3
   u64 *dk = e->dp<u64>(e->L.keyA);

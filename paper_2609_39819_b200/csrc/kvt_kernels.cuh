@@ -66,12 +66,12 @@ __device__ const PowTable g_pow_p = PowTable();
 // ---- device views -------------------------------------------------------------------------------------
 struct Table { TSlot *slots; u32 mask; u32 shift; };   // capacity = mask + 1, home = key >> shift
 
-struct Entries {            // per resident-block metadata, entry id = slot (HBM) or n_hbm + slot (host)
+struct Entries {            // per resident-block metadata, entry id = slot (HBM), n_hbm + slot (host) or n_hbm + n_host + slot (remote)
   u64 *key;                 // 0 = free
   u32 *stamp, *depth, *infl, *rank, *tslot, *mark;
   u32 *link;                // inclusive tiering: an HBM block and its clean host copy point at each other (else ENT_NONE)
   u8 *floor;
-  u32 n_hbm, n_total;
+  u32 n_hbm, n_host, n_total;
 };
 
 // A host entry that only holds a clean copy of a block whose home is in HBM.
@@ -484,15 +484,15 @@ __global__ void __launch_bounds__(CHUNK) k_hash_lookup_fused(HashArgs a, LookupA
 }
 
 // Stamps and locks the reusable prefix of every context of the batch; counts hits per tier.
-struct LockArgs { Entries ent; const u32 *b_ent; const u32 *hit_len; u32 *n_hbm; u32 *n_host; u32 now; u32 *status; };
+struct LockArgs { Entries ent; const u32 *b_ent; const u32 *hit_len; u32 *n_hbm; u32 *n_host; u32 *n_remote; u32 now; u32 *status; };
 
 __global__ void __launch_bounds__(CHUNK) k_lock_hits(HashArgs a, LockArgs l) {
-  __shared__ u32 s_hbm, s_host;
+  __shared__ u32 s_hbm, s_host, s_remote;
   const u32 tid = threadIdx.x;
   u32 ci;
   const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci);
   const u32 b = (blockIdx.x - c.chunk_base) * CHUNK + tid;
-  if (tid == 0) { s_hbm = 0; s_host = 0; }
+  if (tid == 0) { s_hbm = 0; s_host = 0; s_remote = 0; }
   __syncthreads();
   if (b < l.hit_len[ci]) {
     u32 e = l.b_ent[c.blk_base + b];
@@ -500,13 +500,14 @@ __global__ void __launch_bounds__(CHUNK) k_lock_hits(HashArgs a, LockArgs l) {
     else {
       l.ent.stamp[e] = l.now;
       atomicAdd(&l.ent.infl[e], 1u);
-      atomicAdd(e < l.ent.n_hbm ? &s_hbm : &s_host, 1u);
+      atomicAdd(e < l.ent.n_hbm ? &s_hbm : e < l.ent.n_hbm + l.ent.n_host ? &s_host : &s_remote, 1u);
     }
   }
   __syncthreads();
   if (tid == 0) {
     if (s_hbm) atomicAdd(&l.n_hbm[ci], s_hbm);
     if (s_host) atomicAdd(&l.n_host[ci], s_host);
+    if (s_remote) atomicAdd(&l.n_remote[ci], s_remote);
   }
 }
 
@@ -726,7 +727,8 @@ __global__ void k_block_map(Table t, Entries en, const u64 *keys, u32 n, u8 *tie
   u32 e = s == ENT_NONE ? ENT_NONE : t.slots[s].ent;
   if (e >= en.n_total) { tier[b] = 0xFF; slot[b] = 0xFFFFFFFFu; }
   else if (e < en.n_hbm) { tier[b] = 0; slot[b] = e; }
-  else { tier[b] = 1; slot[b] = e - en.n_hbm; }
+  else if (e < en.n_hbm + en.n_host) { tier[b] = 1; slot[b] = e - en.n_hbm; }
+  else { tier[b] = 2; slot[b] = e - en.n_hbm - en.n_host; }
 }
 
 // ======================================================================================================

@@ -41,3 +41,20 @@ def test_random_api_streams_with_long_messages(oracle, seed, flags):
     F.run([gpu, cpu], seed, steps=200, inclusive=bool(flags & 2), check_every=10, invariants=False, max_tok=6000)
     st = gpu.get_stats()
     assert st["blocks_rehashed"] < st["blocks_hashed"]
+
+
+@pytest.mark.parametrize("seed", range(12))
+@pytest.mark.parametrize("flags", [0, 1, 2, 4])
+@pytest.mark.parametrize("pools", [(24, 12, 16), (8, 4, 3), (16, 0, 8)], ids=lambda p: f"hbm{p[0]}-host{p[1]}-remote{p[2]}")
+def test_random_api_streams_with_three_tiers(oracle, seed, flags, pools):
+    """The same with a remote tier behind the host tier: blocks travel down level by level and up again,
+    straight into HBM too."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_39819_b200 import binding as B
+    kw = dict(n_hbm_blocks=pools[0], n_host_blocks=pools[1], n_remote_blocks=pools[2], max_contexts=6, policy_flags=flags,
+              suspended_order=seed % 2, pool_layout=seed % 2, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 16, max_messages=2048, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    F.run([gpu, cpu], seed, steps=300, inclusive=bool(flags & 2), check_every=10)

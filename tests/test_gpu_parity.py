@@ -655,7 +655,8 @@ def test_create_rejects_bad_configs(B):
         return rc
 
     assert attempt() == B.OK                                   # the unmodified copy is fine
-    assert attempt(abi_version=2) == B.E_INVAL
+    assert attempt(abi_version=1) == B.E_INVAL
+    assert attempt(n_remote_blocks=4) == B.E_INVAL                                # a remote tier without its pool
     assert attempt(block_tokens=32) == B.E_INVAL
     assert attempt(table_capacity=good.cfg.table_capacity + 1) == B.E_INVAL      # not a power of two
     assert attempt(table_capacity=16) == B.E_INVAL                                # < 2 * (hbm + host)
