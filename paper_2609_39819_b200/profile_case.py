@@ -9,6 +9,7 @@ larger than L2, a few GB on the device at most, a handful of launches).
     python -m paper_2609_39819_b200.profile_case lookup     # hash + table lookup of 16 x 16,128-block calls
     python -m paper_2609_39819_b200.profile_case select     # classify + select 10% of 1 Mi resident blocks
     python -m paper_2609_39819_b200.profile_case c4         # the whole metadata stress at full size (C4)
+    python -m paper_2609_39819_b200.profile_case mover_remote  # host tier <-> third tier, third tier -> HBM
     python -m paper_2609_39819_b200.profile_case sweep      # C5: movement bandwidth sweep (markdown table)
 Each prints one line with CUDA-event timings of its launches.
 """
@@ -99,6 +100,19 @@ def main(case: str):
         gb = n * geo.block_bytes / 1e9
         print(f"mover_host: {n} blocks x {geo.block_bytes} B; gather to host ms {g} = {[round(gb / (m / 1e3), 1) for m in g]} GB/s; "
               f"scatter from host ms {sc} = {[round(gb / (m / 1e3), 1) for m in sc]} GB/s")
+    elif case == "mover_remote":
+        # host tier <-> the buffer standing in for the remote tier (both pinned host memory): the mover reads over
+        # the host link and writes back over it, so both directions of the link carry the payload at once
+        geo, n = W.GEO_8B, 512
+        eng = B.Engine(n_hbm_blocks=n, n_host_blocks=n, n_remote_blocks=n, max_contexts=2, max_tokens=1 << 12,
+                       max_messages=64, max_batch_blocks=4096, zero_pools=False, **geo.kwargs())
+        src = torch.from_numpy(W.ids_c5(1, n, n, True).view(np.int32)).cuda()
+        dst = torch.from_numpy(W.ids_c5(2, n, n, True).view(np.int32)).cuda()
+        down = _events(torch, lambda: eng.copy_blocks(1, src, 2, dst), 2)
+        up = _events(torch, lambda: eng.copy_blocks(2, dst, 0, src), 2)
+        gb = n * geo.block_bytes / 1e9
+        print(f"mover_remote: {n} blocks x {geo.block_bytes} B; host -> remote ms {down} = {[round(gb / (m / 1e3), 1) for m in down]} GB/s; "
+              f"remote -> HBM ms {up} = {[round(gb / (m / 1e3), 1) for m in up]} GB/s")
     elif case == "exchange":
         geo, n = W.GEO_8B, 1024
         eng = B.Engine(n_hbm_blocks=3 * n, n_host_blocks=3 * n, max_contexts=2, max_tokens=1 << 12, max_messages=64,

@@ -319,7 +319,23 @@ def evict(eng, n, n_pinned_incoming=0, reload_slots=None):
         hv, hs = eng.select_victims(TIER_HOST, n_live - free_host)
         rec["host_victims"] = hv.copy()
         rec["host_vstates"] = hs.copy()
-        if len(hv):
+        if len(hv) and getattr(eng, "n_remote_blocks", 0):
+            # a third tier exists: the host tier's victims move down instead of being lost (clean copies of HBM
+            # blocks are simply released), after the remote tier has made room by releasing its own first victims
+            copies = hs == STATE_COPY
+            if copies.any():
+                eng.release(TIER_HOST, hv[copies])
+            down, dstates = hv[~copies], hs[~copies]
+            n_down = int(((dstates & 0x7F) > 0).sum())
+            free_remote = eng.n_remote_blocks - eng.get_stats()["occ_remote"]
+            if n_down > free_remote:
+                rv, rs = eng.select_victims(TIER_REMOTE, n_down - free_remote)
+                rec["remote_victims"] = rv.copy()
+                if len(rv):
+                    eng.release(TIER_REMOTE, rv)
+            if len(down):
+                rec["demote"] = eng.move(TIER_HOST, TIER_REMOTE, down)
+        elif len(hv):
             eng.release(TIER_HOST, hv)
     if reload_slots is not None and len(reload_slots):
         # both directions in one call; what found no free HBM slot at the start follows once the offload has made room
@@ -341,17 +357,21 @@ def run_call(eng, ctxs, opt: ReplayOptions):
     rec["lookup"] = info.copy()
     st = eng.get_stats()
     free_hbm = eng.n_hbm_blocks - st["occ_hbm"]
-    need = int(info["n_hit_host"].sum()) + int(info["n_admissible"].sum()) - free_hbm
-    host_slots = []
+    need = int(info["n_hit_host"].sum()) + int(info["n_hit_remote"].sum()) + int(info["n_admissible"].sum()) - free_hbm
+    host_slots, remote_slots = [], []
     for c, inf in zip(ctxs, info):
-        if inf["n_hit_host"]:
+        if inf["n_hit_host"] or inf["n_hit_remote"]:
             _keys, tier, slot = eng.get_block_map(c)
             h = int(inf["hit_len"])
             host_slots.append(slot[:h][tier[:h] == TIER_HOST])
-    hs = None
+            remote_slots.append(slot[:h][tier[:h] == TIER_REMOTE])
+    hs = rs = None
     if host_slots:
         hs = np.concatenate(host_slots)
         hs = hs[np.sort(np.unique(hs, return_index=True)[1])]  # a shared host block is reloaded once
+        rs = np.concatenate(remote_slots)
+        rs = rs[np.sort(np.unique(rs, return_index=True)[1])]
+        hs, rs = (hs if len(hs) else None), (rs if len(rs) else None)
     if need > 0 and opt.use_exchange and hs is not None:
         rec.update(evict(eng, need, int(info["n_pinned"].sum()), reload_slots=hs))
     else:
@@ -359,6 +379,8 @@ def run_call(eng, ctxs, opt: ReplayOptions):
             rec.update(evict(eng, need, int(info["n_pinned"].sum())))
         if hs is not None:
             rec["reload"] = eng.reload(hs)
+    if rs is not None:
+        rec["promote"] = eng.move(TIER_REMOTE, TIER_HBM, rs)   # remote hits come straight up into HBM
     adm = eng.map_blocks(ctxs, MAP_ADMIT)
     rec["admit"] = adm.copy()
     maps = []
@@ -377,17 +399,21 @@ def run_call(eng, ctxs, opt: ReplayOptions):
         eng.prefill_done(c)
     opt.counters["calls"] = opt.counters.get("calls", 0) + 1
     if opt.record_states:
-        rec["states"] = [eng.get_states(TIER_HBM).copy(), eng.get_states(TIER_HOST).copy()]
-        rec["entries"] = [eng.get_entries(TIER_HBM), eng.get_entries(TIER_HOST)]
+        rec["states"] = [eng.get_states(t).copy() for t in engine_tiers(eng)]
+        rec["entries"] = [eng.get_entries(t) for t in engine_tiers(eng)]
     rec["stats"] = {k: v for k, v in eng.get_stats().items() if k not in GPU_ONLY_STATS}
     if opt.payload is not None and opt.verify_payload_every and opt.counters["calls"] % opt.verify_payload_every == 0:
         rec["payload_ok"] = verify_payload(eng, opt.payload)
     return rec
 
 
+def engine_tiers(eng):
+    return (TIER_HBM, TIER_HOST, TIER_REMOTE) if getattr(eng, "n_remote_blocks", 0) else (TIER_HBM, TIER_HOST)
+
+
 def verify_payload(eng, payload) -> bool:
-    """Every occupied slot of both tiers holds payload(key) of the block it is registered for."""
-    for tier in (TIER_HBM, TIER_HOST):
+    """Every occupied slot of every tier holds payload(key) of the block it is registered for."""
+    for tier in engine_tiers(eng):
         keys = eng.get_entries(tier)["key"]
         for s in np.nonzero(keys)[0]:
             if not np.array_equal(eng.read_block(tier, int(s)), payload(int(keys[s]), eng.block_bytes)):

@@ -93,7 +93,7 @@ def _replay_pair(gpu, cpu, trace, payload, check_pools=True, record_states=True,
         if k not in W.GPU_ONLY_STATS:
             assert sg[k] == sc[k], k
     if check_pools and payload is not None:
-        for tier, n in ((0, gpu.n_hbm_blocks), (1, gpu.n_host_blocks)):
+        for tier in W.engine_tiers(gpu):
             keys = cpu.get_entries(tier)["key"]
             for s in np.nonzero(keys)[0]:
                 assert np.array_equal(gpu.read_block(tier, int(s)), cpu.read_block(tier, int(s))), (tier, s)
@@ -219,6 +219,31 @@ def test_trace_parity_with_unreachable_blocks_dead(B, oracle, flags):
         assert np.array_equal(gpu.get_states(tier), cpu.get_states(tier))
     vg, vc = gpu.select_victims(0, 64), cpu.select_victims(0, 64)
     assert np.array_equal(vg[0], vc[0]) and np.array_equal(vg[1], vc[1])
+
+
+@pytest.mark.parametrize("flags", [0, 2])
+def test_trace_parity_with_a_remote_tier(B, oracle, flags):
+    """Three tiers under the replay driver: host victims move down to the remote tier, remote hits come straight up
+    into HBM; every reported value, every state on all three tiers and every payload byte match the oracle."""
+    for seed in (7, 63, 86):
+        kw = dict(n_hbm_blocks=96, n_host_blocks=48, n_remote_blocks=160, max_contexts=64, policy_flags=flags,
+                  **W.GEO_TOY.kwargs())
+        gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)
+        cpu = oracle.OracleEngine(**kw)
+        _replay_pair(gpu, cpu, W.trace_c1(seed), W.payload_pattern, verify_every=1)
+    trace, n_ctx = W.trace_c3(1, n_sessions=8, scale=1 / 32)
+    kw = dict(n_hbm_blocks=256, n_host_blocks=96, n_remote_blocks=512, max_contexts=n_ctx, policy_flags=flags,
+              **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 20, max_messages=1 << 15, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    _replay_pair(gpu, cpu, trace, W.payload_pattern, verify_every=5)
+    st = gpu.get_stats()
+    assert st["demoted"] > 0 and st["promoted"] > 0 and st["hits_remote"] > 0
+    for tier in (0, 1, 2):
+        assert np.array_equal(gpu.get_states(tier), cpu.get_states(tier))
+        eg, ec = gpu.get_entries(tier), cpu.get_entries(tier)
+        for k in ec:
+            assert np.array_equal(eg[k], ec[k]), (tier, k)
 
 
 def test_scaled_c2_trace_parity(B, oracle):

@@ -127,6 +127,28 @@ def test_replay_with_exchange_moves_the_same_blocks(make, flags):
     assert np.array_equal(out[0][2][0], out[1][2][0]) and np.array_equal(out[0][2][1], out[1][2][1])
 
 
+@pytest.mark.parametrize("flags", [0, 2])
+def test_replay_with_a_remote_tier_keeps_more_blocks_reusable(make, flags):
+    """C3-shaped trace with a small host tier: without a third tier the host tier's victims are lost, with one
+    they move down and come back when their session calls again: more prefix hits, fewer dropped live blocks,
+    every payload byte intact on all three tiers."""
+    trace, n_ctx = W.trace_c3(1, n_sessions=8, scale=1 / 32)
+    res = {}
+    for n_remote in (0, 512):
+        eng = make(n_hbm_blocks=256, n_host_blocks=96, n_remote_blocks=n_remote, max_contexts=n_ctx, policy_flags=flags,
+                   **W.GEO_TOY.kwargs())
+        opt = W.ReplayOptions(payload=W.payload_pattern, record_states=False, verify_payload_every=9)
+        for _i, kind, rec in W.replay(eng, trace, opt):
+            if kind == "call":
+                assert rec.get("payload_ok", True)
+        assert W.verify_payload(eng, W.payload_pattern)
+        res[n_remote] = eng.get_stats()
+    a, b = res[0], res[512]
+    assert b["demoted"] > 0 and b["promoted"] > 0 and b["hits_remote"] > 0
+    assert b["hits_hbm"] + b["hits_host"] + b["hits_remote"] > a["hits_hbm"] + a["hits_host"]
+    assert b["dropped"] < a["dropped"]
+
+
 def test_incremental_appends_hash_like_one_shot(make, oracle):
     """Hashing a context after piecewise appends equals hashing the concatenation in one shot."""
     rng = np.random.default_rng(21)
