@@ -589,7 +589,7 @@ def test_capacity_errors_leave_the_engine_usable(B):
     st = eng.get_stats()
     assert (st["occ_hbm"], st["occ_host"]) == (12, 4)
     with pytest.raises(B.KvtError):
-        eng.select_victims(2, 1)                                 # bad tier
+        eng.select_victims(3, 1)                                 # bad tier
 
 
 @pytest.mark.parametrize("lookup_variant", [1, 2], ids=["three-kernels", "single-pass"])
