@@ -321,7 +321,8 @@ class Engine:
         self._check(self.L.kvt_classify(self.h, _stream()), "classify")
 
     def _tier_size(self, tier):
-        return (self.n_hbm_blocks, self.n_host_blocks, self.n_remote_blocks)[tier]
+        sizes = (self.n_hbm_blocks, self.n_host_blocks, self.n_remote_blocks)
+        return sizes[tier] if 0 <= tier < 3 else 0      # an unknown tier is for the library to reject
 
     def get_states(self, tier):
         st = np.zeros(self._tier_size(tier), np.uint8)
