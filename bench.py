@@ -189,25 +189,58 @@ def mem_available_bytes():
 
 
 class ClockSampler:
-    """nvidia-smi polled every 50 ms in the background; stop(t0, t1) keeps the samples taken inside the timed
-    window [t0, t1] (host wall clock), or all samples of the run if the window saw fewer than two."""
+    """SM clock and throttle reasons sampled in the background while an arm runs: NVML read-outs every 5 ms from a
+    thread (the timed region of the in-device arm lasts tens of ms), or, if NVML cannot be loaded, nvidia-smi
+    polled every 50 ms. stop(t0, t1) keeps the samples taken inside the timed window [t0, t1] (host wall clock),
+    or all samples of the arm if the window saw fewer than two. Read-only: no setting of the GPU is touched."""
     FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
+    NVML_REASONS = ((0x8, "hw_slowdown"), (0x40, "hw_thermal_slowdown"), (0x20, "sw_thermal_slowdown"), (0x4, "sw_power_cap"))
 
-    def __init__(self, gpu_index):
+    def __init__(self, gpu_index, torch=None):
+        self.rows, self.p, self.thread, self.source = [], None, None, "none"
+        try:
+            import threading
+            import pynvml
+            pynvml.nvmlInit()
+            h = None
+            if torch is not None:
+                try:
+                    uuid = str(torch.cuda.get_device_properties(torch.cuda.current_device()).uuid)
+                    h = pynvml.nvmlDeviceGetHandleByUUID(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+                except Exception:
+                    h = None
+            if h is None:
+                h = pynvml.nvmlDeviceGetHandleByIndex(gpu_index)
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(h, pynvml.NVML_CLOCK_SM))
+            self.running = True
+
+            def loop():
+                while self.running:
+                    try:
+                        mhz = float(pynvml.nvmlDeviceGetClockInfo(h, pynvml.NVML_CLOCK_SM))
+                        bits = int(pynvml.nvmlDeviceGetCurrentClocksThrottleReasons(h))
+                        self.rows.append((time.time(), mhz, self.max_mhz, [nm for b, nm in self.NVML_REASONS if bits & b]))
+                    except Exception:
+                        pass
+                    time.sleep(0.005)
+            self.thread = threading.Thread(target=loop, daemon=True)
+            self.thread.start()
+            self.source = "nvml, 5 ms"
+            return
+        except Exception:
+            self.thread = None
         self.f = tempfile.NamedTemporaryFile("w+", suffix=".csv", delete=False)
         try:
             self.p = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
                                        "-i", str(gpu_index), "-lms", "50"], stdout=self.f, stderr=subprocess.DEVNULL)
+            self.source = "nvidia-smi, 50 ms"
         except OSError:
             self.p = None
 
-    def stop(self, t0=None, t1=None):
+    def _smi_rows(self):
         import datetime
-        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": "none"}
-        if self.p is None:
-            return out
         time.sleep(0.06)
         self.p.terminate()
         try:
@@ -230,7 +263,19 @@ class ClockSampler:
                 continue
         self.f.close()
         os.unlink(self.f.name)
-        inside = [r for r in rows if t0 is not None and t0 - 0.05 <= r[0] <= t1 + 0.05]
+        return rows
+
+    def stop(self, t0=None, t1=None):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0, "window": "none", "source": self.source}
+        if self.thread is not None:
+            self.running = False
+            self.thread.join(timeout=1)
+            rows, slack = list(self.rows), 0.0
+        elif self.p is not None:
+            rows, slack = self._smi_rows(), 0.05
+        else:
+            return out
+        inside = [r for r in rows if t0 is not None and t0 - slack <= r[0] <= t1 + slack]
         use, out["window"] = (inside, "timed region") if len(inside) >= 2 else (rows, "whole arm (timed region shorter than the sampling period)")
         if use:
             out.update(sm_mhz=float(np.median([r[1] for r in use])), sm_max_mhz=float(max(r[2] for r in use)),
@@ -581,7 +626,7 @@ def main():
     hbm_now = hbm_copy_this_run(torch)
 
     # ---- value arm: everything resident in HBM ------------------------------------------------------------
-    sampler = ClockSampler(local_rank)
+    sampler = ClockSampler(local_rank, torch)
     free_b, _total = torch.cuda.mem_get_info()
     want2 = int(args.host_gib * GiB) // W.GEO_8B.block_bytes
     fit2 = int((free_b - n_hbm_blocks * W.GEO_8B.block_bytes - 6 * GiB) // W.GEO_8B.block_bytes)
@@ -602,7 +647,7 @@ def main():
             dist.all_reduce(hb, op=dist.ReduceOp.MIN)
             host_blocks = int(hb.item())
         if host_blocks >= 5000:      # the session keeps up to ~4.5 K blocks in the host tier
-            sampler = ClockSampler(local_rank)
+            sampler = ClockSampler(local_rank, torch)
             e = gpu_arm(args, torch, B, setup, turns, n_ff, True, host_blocks, n_hbm_blocks, rank, world, barrier)
             clocks_e2e = sampler.stop(*e["wall"])
 
