@@ -196,7 +196,7 @@ __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
 #pragma unroll
   for (int it = 0; it < 4; ++it) {
     u32 idx = it * CHUNK + tid;
-    v[it] = (idx >> 2) < nb ? __ldg(tok + idx) : make_uint4(0, 0, 0, 0);
+    v[it] = (idx >> 2) < nb ? __ldcs(tok + idx) : make_uint4(0, 0, 0, 0);   // read once: evict-first
   }
   // iteration `it` covers blocks it*64 .. it*64+63, four lanes per block; after the two exchange steps every
   // lane of a quad holds the four block sums, and lane q finishes the block of iteration q
@@ -381,7 +381,7 @@ __global__ void __launch_bounds__(CHUNK) k_hash_lookup_fused(HashArgs a, LookupA
 #pragma unroll
     for (int it = 0; it < 4; ++it) {
       u32 idx = it * CHUNK + tid;
-      v[it] = (idx >> 2) < nb ? __ldg(tok + idx) : make_uint4(0, 0, 0, 0);
+      v[it] = (idx >> 2) < nb ? __ldcs(tok + idx) : make_uint4(0, 0, 0, 0);
     }
     u64 mine = 0;
 #pragma unroll
