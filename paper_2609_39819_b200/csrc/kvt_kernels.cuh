@@ -91,6 +91,26 @@ __device__ __forceinline__ u32 tab_find(const Table &t, u64 key, u32 *status) {
   return ENT_NONE;
 }
 
+// Read-only probe for kernels that run while nobody writes the table: returns the entry id stored for key, or
+// ENT_NONE. Each step fetches two consecutive slots with two independent 16-byte loads (key and entry id come
+// together), so a probe sequence of length p costs ceil(p / 2) dependent memory round trips and no extra one for
+// the entry id.
+__device__ __forceinline__ u32 tab_lookup_ent(const Table &t, u64 key, u32 *status) {
+  u32 i = (u32)(key >> t.shift);
+  for (u32 n = 0; n <= t.mask; n += 2) {
+    const uint4 a = __ldg(reinterpret_cast<const uint4 *>(t.slots + i));
+    const uint4 b = __ldg(reinterpret_cast<const uint4 *>(t.slots + ((i + 1) & t.mask)));
+    const u64 ka = (u64)a.x | ((u64)a.y << 32), kb = (u64)b.x | ((u64)b.y << 32);
+    if (ka == key) return a.z;
+    if (ka == KEY_EMPTY) return ENT_NONE;
+    if (kb == key) return b.z;
+    if (kb == KEY_EMPTY) return ENT_NONE;
+    i = (i + 2) & t.mask;
+  }
+  set_err(status, DERR_PROBE);
+  return ENT_NONE;
+}
+
 // Finds key or claims the first EMPTY slot of its probe sequence for it (tombstones are skipped,
 // never reused, so two threads inserting the same key always meet in the same slot).
 __device__ __forceinline__ u32 tab_find_or_claim(const Table &t, u64 key, u32 *status) {
@@ -312,8 +332,7 @@ __global__ void __launch_bounds__(CHUNK) k_hash_finish_lookup(HashArgs a, Lookup
     }
     a.keys[c.key_off + b0 + tid] = key;
     if (l.tab.slots) {
-      u32 s = tab_find(l.tab, key, l.status);
-      u32 ent = s == ENT_NONE ? ENT_NONE : l.tab.slots[s].ent;
+      u32 ent = tab_lookup_ent(l.tab, key, l.status);
       l.b_ent[c.blk_base + b0 + tid] = ent;
       if (ent == ENT_NONE) atomicMin(&s_min, b0 + tid);
     }
@@ -474,8 +493,7 @@ __global__ void __launch_bounds__(CHUNK) k_hash_lookup_fused(HashArgs a, LookupA
   }
   if (tid < nb) {
     a.keys[c.key_off + b0 + tid] = key;
-    u32 s = tab_find(l.tab, key, l.status);
-    u32 ent = s == ENT_NONE ? ENT_NONE : l.tab.slots[s].ent;
+    u32 ent = tab_lookup_ent(l.tab, key, l.status);
     l.b_ent[c.blk_base + b0 + tid] = ent;
     if (ent == ENT_NONE) atomicMin(&s_min, b0 + tid);
   }
@@ -710,9 +728,7 @@ __global__ void k_admit_apply(AdmitArgs a) {
 __global__ void k_unlock(Table t, Entries en, const u64 *keys, u32 n, u32 now, u32 do_stamp, u32 *status) {
   u32 b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= n) return;
-  u32 s = tab_find(t, keys[b], status);
-  if (s == ENT_NONE) { set_err(status, DERR_CORRUPT); return; }
-  u32 e = t.slots[s].ent;
+  u32 e = tab_lookup_ent(t, keys[b], status);
   if (e >= en.n_total) { set_err(status, DERR_CORRUPT); return; }
   u32 old = atomicSub(&en.infl[e], 1u);
   if (old == 0) { atomicAdd(&en.infl[e], 1u); set_err(status, DERR_CORRUPT); }
@@ -723,8 +739,7 @@ __global__ void k_unlock(Table t, Entries en, const u64 *keys, u32 n, u32 now, u
 __global__ void k_block_map(Table t, Entries en, const u64 *keys, u32 n, u8 *tier, u32 *slot, u32 *status) {
   u32 b = blockIdx.x * blockDim.x + threadIdx.x;
   if (b >= n) return;
-  u32 s = tab_find(t, keys[b], status);
-  u32 e = s == ENT_NONE ? ENT_NONE : t.slots[s].ent;
+  u32 e = tab_lookup_ent(t, keys[b], status);
   if (e >= en.n_total) { tier[b] = 0xFF; slot[b] = 0xFFFFFFFFu; }
   else if (e < en.n_hbm) { tier[b] = 0; slot[b] = e; }
   else if (e < en.n_hbm + en.n_host) { tier[b] = 1; slot[b] = e - en.n_hbm; }
@@ -772,7 +787,7 @@ __global__ void k_first_miss(ClsArgs a) {
   if (g >= a.n_map) return;
   const ClsCtx c = a.ctx[lo];
   const u32 b = g - c.map_base;
-  if (tab_find(a.tab, a.keys[c.key_off + b], a.status) == ENT_NONE) atomicMin(&a.first_miss[lo], b);
+  if (tab_lookup_ent(a.tab, a.keys[c.key_off + b], a.status) == ENT_NONE) atomicMin(&a.first_miss[lo], b);
 }
 
 __global__ void k_classify(ClsArgs a) {
@@ -792,9 +807,7 @@ __global__ void k_classify(ClsArgs a) {
   for (u32 j = l; j < c.n_msgs && ms[j] < t1; ++j)
     if (me[j] > ms[j] && mr[j] > r) r = mr[j];
   if (r == 0) return;
-  u32 s = tab_find(a.tab, a.keys[c.key_off + b], a.status);
-  if (s == ENT_NONE) return;  // mapped but not resident
-  u32 e = a.tab.slots[s].ent;
+  u32 e = tab_lookup_ent(a.tab, a.keys[c.key_off + b], a.status);   // ENT_NONE: mapped but not resident
   if (e < a.ent.n_total) atomicMax(&a.ent.rank[e], r);
 }
 
