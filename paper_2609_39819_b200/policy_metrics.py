@@ -61,8 +61,7 @@ def replay_metrics(eng, trace):
         hit += int(rec["lookup"]["hit_len"].sum())
         tot += int(rec["lookup"]["n_blocks"].sum())
         occ = dead = 0
-        for tier in (0, 1):
-            st = rec["states"][tier]
+        for st in rec["states"]:                                # every tier the engine has
             occ += int((st != 0xFF).sum())
             dead += int((st == 0).sum())
         zshare.append(dead / occ if occ else 0.0)
@@ -96,6 +95,7 @@ def main():
     ap.add_argument("--hbm", type=int, default=1024)
     ap.add_argument("--host", type=int, default=1024)
     ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--remote", type=int, default=0, help="adds a row for the paper's policy with a third tier of this many blocks")
     a = ap.parse_args()
     from . import binding as B
     trace, n_ctx = W.trace_c3(a.seed, n_sessions=a.sessions, scale=a.scale)
@@ -103,10 +103,13 @@ def main():
           f"metadata-only engines on the GPU")
     print("| policy | hit ratio | zombie share mean / peak | wrong-direction evictions | judged | offloaded | dropped |")
     print("|---|---:|---:|---:|---:|---:|---:|")
-    for name, (order, flags) in POLICIES.items():
-        eng = B.Engine(n_hbm_blocks=a.hbm, n_host_blocks=a.host, max_contexts=n_ctx, metadata_only=True,
-                       suspended_order=order, policy_flags=flags, max_tokens=1 << 22, max_messages=1 << 15,
-                       **W.GEO_GLM.kwargs())
+    rows = [(name, order, flags, 0) for name, (order, flags) in POLICIES.items()]
+    if a.remote:
+        rows.append((f"lifecycle + MRU, third tier of {a.remote} blocks", 0, 0, a.remote))
+    for name, order, flags, n_remote in rows:
+        eng = B.Engine(n_hbm_blocks=a.hbm, n_host_blocks=a.host, n_remote_blocks=n_remote, max_contexts=n_ctx,
+                       metadata_only=True, suspended_order=order, policy_flags=flags, max_tokens=1 << 22,
+                       max_messages=1 << 15, **W.GEO_GLM.kwargs())
         m = replay_metrics(eng, trace)
         print(f"| {name} | {m['hit_ratio']:.3f} | {m['zombie_share_mean']:.3f} / {m['zombie_share_peak']:.3f} | "
               f"{m['wrong_direction_ratio']:.3f} | {m['evictions_judged']} | {m['offloaded']} | {m['dropped']} |")
