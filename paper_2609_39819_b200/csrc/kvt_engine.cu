@@ -102,7 +102,7 @@ DevLayout make_layout(const kvt_config &c) {
   u64 n_chunks = B / CHUNK + C + 1;
   L.agg = take(n_chunks * 8); L.carry = take(n_chunks * 8);   // per-chunk aggregates / chain values of a LOOKUP batch
   L.cflags = take((n_chunks + 1) * 4);                         // per-chunk publication flags + the ticket word
-  L.desc = take(C * 64);
+  L.desc = take(C * 64 + 2 * n_chunks * 4);   // per-context descriptors, then the chunk -> context maps of a LOOKUP batch
   L.ctxres = take(C * 20);   // per context: hit_len, hits per tier (3), admission stop
   L.m_start = take(Mm * 4); L.m_end = take(Mm * 4); L.m_rank = take(Mm);
   L.keyA = take(Nt * 8); L.keyB = take(Nt * 8); L.valA = take(Nt * 4); L.valB = take(Nt * 4);
@@ -499,7 +499,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   e->key_alloc.init(c.max_key_blocks + c.max_key_blocks / CHUNK + 64ull * c.max_contexts, 32);
   // pinned staging
   u64 C = c.max_contexts, Mm = c.max_messages, LB = L.LB;
-  u64 o_status = 0, o_desc = 256, o_ctxres = o_desc + round_up(C * 64, 256), o_ms = o_ctxres + round_up(C * 20, 256),
+  u64 o_status = 0, o_desc = 256, o_ctxres = o_desc + round_up(C * 64 + 2 * (c.max_batch_blocks / CHUNK + C + 1) * 4, 256), o_ms = o_ctxres + round_up(C * 20, 256),
       o_me = o_ms + round_up(Mm * 4, 256), o_mr = o_me + round_up(Mm * 4, 256), o_ids = o_mr + round_up(Mm, 256),
       o_ids2 = o_ids + round_up(LB * 4, 256), o_out = o_ids2 + round_up(LB * 4, 256),
       total = o_out + round_up(LB * 16, 256);
@@ -753,6 +753,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
   if (r) return r;
   e->now += 1;
   HashCtx *hd = reinterpret_cast<HashCtx *>(e->h_desc);
+  std::vector<std::pair<u32, u32>> n_seq_chunks;   // per listed sequence: chunks in the all-blocks grid / in the digest grid
   std::vector<int> dev_idx(n_ctx, -1);
   u32 nd = 0, chunk_base = 0, dchunk_base = 0, blk_base = 0;
   u32 *h_hit = e->h_ctxres, *h_hbm = e->h_ctxres + e->cfg.max_contexts, *h_host = e->h_ctxres + 2 * e->cfg.max_contexts,
@@ -789,6 +790,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
       hd[nd++] = d;
       chunk_base += cdiv(nb, CHUNK);
       dchunk_base += cdiv(nb - first, CHUNK);
+      n_seq_chunks.push_back({cdiv(nb, CHUNK), cdiv(nb - first, CHUNK)});
       blk_base += nb;
       e->st.blocks_rehashed += nb - first;
     }
@@ -797,7 +799,16 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
   if (nd) {
     u32 *d_res = e->dp<u32>(e->L.ctxres);
     const u32 C = e->cfg.max_contexts;
-    CU(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nd * sizeof(HashCtx), cudaMemcpyHostToDevice, s));
+    // chunk -> sequence maps of the two grids, right behind the descriptors (one upload)
+    u32 *h_map = reinterpret_cast<u32 *>(hd + nd), *h_dmap = h_map + chunk_base;
+    {
+      u32 k = 0, dk = 0;
+      for (u32 q = 0; q < nd; ++q) {
+        for (u32 j = 0; j < n_seq_chunks[q].first; ++j) h_map[k++] = q;
+        for (u32 j = 0; j < n_seq_chunks[q].second; ++j) h_dmap[dk++] = q;
+      }
+    }
+    CU(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nd * sizeof(HashCtx) + ((u64)chunk_base + dchunk_base) * 4, cudaMemcpyHostToDevice, s));
     CU(cudaMemcpyAsync(d_res, h_hit, nd * 4, cudaMemcpyHostToDevice, s));
     CU(cudaMemsetAsync(d_res + C, 0, 3ull * C * 4, s));
     r = status_zero(e, s);
@@ -805,6 +816,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     HashArgs ha;
     ha.tokens = e->d_tokens; ha.keys = e->d_keys; ha.carry_base = e->d_keys; ha.ctx = e->dp<HashCtx>(e->L.desc); ha.n_ctx = nd;
     ha.agg = e->dp<u64>(e->L.agg); ha.h0 = e->h0; ha.single = HashCtx{};
+    ha.chunk_ctx = reinterpret_cast<const u32 *>(ha.ctx + nd); ha.dchunk_ctx = ha.chunk_ctx + chunk_base;
     LookupArgs la;
     la.tab = e->tab; la.b_ent = e->dp<u32>(e->L.s0); la.hit_len = d_res; la.status = e->d_status;
     LockArgs lk;
@@ -1425,7 +1437,7 @@ int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t ha
   cudaStream_t s = (cudaStream_t)stream;
   u32 n_chunks = cdiv(nb, CHUNK);
   HashArgs ha;
-  ha.tokens = d_tokens; ha.keys = d_keys; ha.ctx = nullptr; ha.n_ctx = 1;
+  ha.tokens = d_tokens; ha.keys = d_keys; ha.ctx = nullptr; ha.n_ctx = 1; ha.chunk_ctx = ha.dchunk_ctx = nullptr;
   ha.single = HashCtx{};
   ha.single.n_blocks = (u32)nb;
   ha.agg = (u64 *)d_scratch; ha.carry_base = (u64 *)d_scratch + n_chunks; ha.h0 = hash_h0(hash_seed);
@@ -1460,7 +1472,7 @@ int32_t kvt_hash_tokens_noalloc(const uint32_t *d_tokens, uint64_t n_tokens, uin
   cudaStream_t s = (cudaStream_t)stream;
   u32 n_chunks = cdiv(nb, CHUNK);
   HashArgs ha;
-  ha.tokens = d_tokens; ha.keys = d_keys; ha.ctx = nullptr; ha.n_ctx = 1;
+  ha.tokens = d_tokens; ha.keys = d_keys; ha.ctx = nullptr; ha.n_ctx = 1; ha.chunk_ctx = ha.dchunk_ctx = nullptr;
   ha.single = HashCtx{};
   ha.single.n_blocks = (u32)nb;
   ha.agg = g_noalloc_ptr[dev]; ha.carry_base = g_noalloc_ptr[dev] + NOALLOC_MAX_CHUNKS; ha.h0 = hash_h0(hash_seed);

@@ -159,29 +159,16 @@ struct HashCtx {
 struct HashArgs {
   const u32 *tokens; u64 *keys; u64 *carry_base; const HashCtx *ctx; HashCtx single; u32 n_ctx;
   u64 *agg; u64 h0;
+  const u32 *chunk_ctx, *dchunk_ctx;   // batch only: sequence index of every chunk of the all-blocks / digest grid
 };
 
 // Sequence that owns chunk `chunk` of the all-blocks grid (dgrid = false) or of the digest grid (dgrid = true):
-// the last one whose base is <= chunk (sequences with no chunk of their own share a base with their successor).
-// Called by every thread of the CTA with the same arguments: the bases are staged in shared memory with one
-// round of loads, so a cold start costs one memory latency instead of one per step of the binary search.
-constexpr u32 CTX_STAGE = 1024;
+// looked up in the chunk -> sequence map the host uploads with the descriptors (two dependent loads, no search).
 __device__ __forceinline__ const HashCtx &hash_ctx_of_chunk(const HashArgs &a, u32 chunk, u32 *ctx_idx, bool dgrid = false) {
   if (!a.ctx) { *ctx_idx = 0; return a.single; }
-  __shared__ u32 s_base[CTX_STAGE];
-  const bool staged = a.n_ctx <= CTX_STAGE;
-  if (staged) {
-    for (u32 t = threadIdx.x; t < a.n_ctx; t += blockDim.x) s_base[t] = dgrid ? a.ctx[t].dchunk_base : a.ctx[t].chunk_base;
-    __syncthreads();
-  }
-  u32 lo = 0, hi = a.n_ctx;
-  while (hi - lo > 1) {
-    u32 mid = (lo + hi) >> 1;
-    u32 base = staged ? s_base[mid] : (dgrid ? a.ctx[mid].dchunk_base : a.ctx[mid].chunk_base);
-    if (base <= chunk) lo = mid; else hi = mid;
-  }
-  *ctx_idx = lo;
-  return a.ctx[lo];
+  const u32 i = dgrid ? a.dchunk_ctx[chunk] : a.chunk_ctx[chunk];
+  *ctx_idx = i;
+  return a.ctx[i];
 }
 
 // Lane multipliers K[0..15] as a constant-initialised table (read once per thread, L1-resident).
@@ -313,14 +300,12 @@ struct LookupArgs {
 };
 
 __global__ void __launch_bounds__(CHUNK) k_hash_finish_lookup(HashArgs a, LookupArgs l) {
-  __shared__ u32 s_min;
   const u32 tid = threadIdx.x;
   u32 ci;
   const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci);
   const u32 b0 = (blockIdx.x - c.chunk_base) * CHUNK;
   const u32 nb = min(CHUNK, c.n_blocks - b0);
-  if (tid == 0) s_min = 0xFFFFFFFFu;
-  __syncthreads();
+  u32 miss = 0xFFFFFFFFu;
   if (tid < nb) {
     u64 key;
     if (b0 < c.first) {          // unchanged prefix: the key of the previous list still holds
@@ -334,11 +319,20 @@ __global__ void __launch_bounds__(CHUNK) k_hash_finish_lookup(HashArgs a, Lookup
     if (l.tab.slots) {
       u32 ent = tab_lookup_ent(l.tab, key, l.status);
       l.b_ent[c.blk_base + b0 + tid] = ent;
-      if (ent == ENT_NONE) atomicMin(&s_min, b0 + tid);
+      if (ent == ENT_NONE) miss = b0 + tid;
     }
   }
-  __syncthreads();
-  if (l.tab.slots && tid == 0 && s_min != 0xFFFFFFFFu) atomicMin(&l.hit_len[ci], s_min);
+  // first miss of the CTA -> the context's reusable prefix length: warp minima meet in shared memory, one global
+  // atomic per CTA that saw a miss
+  if (l.tab.slots) {
+    __shared__ u32 s_min;
+    if (tid == 0) s_min = 0xFFFFFFFFu;
+    __syncthreads();
+    miss = __reduce_min_sync(0xFFFFFFFFu, miss);
+    if ((tid & 31) == 0 && miss != 0xFFFFFFFFu) atomicMin(&s_min, miss);
+    __syncthreads();
+    if (tid == 0 && s_min != 0xFFFFFFFFu) atomicMin(&l.hit_len[ci], s_min);
+  }
 }
 
 // ------------------------------------------------------------------------------------------------------
@@ -505,28 +499,35 @@ __global__ void __launch_bounds__(CHUNK) k_hash_lookup_fused(HashArgs a, LookupA
 struct LockArgs { Entries ent; const u32 *b_ent; const u32 *hit_len; u32 *n_hbm; u32 *n_host; u32 *n_remote; u32 now; u32 *status; };
 
 __global__ void __launch_bounds__(CHUNK) k_lock_hits(HashArgs a, LockArgs l) {
-  __shared__ u32 s_hbm, s_host, s_remote;
   const u32 tid = threadIdx.x;
   u32 ci;
   const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci);
   const u32 b = (blockIdx.x - c.chunk_base) * CHUNK + tid;
-  if (tid == 0) { s_hbm = 0; s_host = 0; s_remote = 0; }
-  __syncthreads();
+  u32 tier = 3;   // none
   if (b < l.hit_len[ci]) {
     u32 e = l.b_ent[c.blk_base + b];
     if (e >= l.ent.n_total) set_err(l.status, DERR_CORRUPT);
     else {
       l.ent.stamp[e] = l.now;
       atomicAdd(&l.ent.infl[e], 1u);
-      atomicAdd(e < l.ent.n_hbm ? &s_hbm : e < l.ent.n_hbm + l.ent.n_host ? &s_host : &s_remote, 1u);
+      tier = e < l.ent.n_hbm ? 0u : e < l.ent.n_hbm + l.ent.n_host ? 1u : 2u;
     }
   }
+  // per-tier hit counts: one ballot per tier and warp, summed in shared memory, one global atomic per CTA and tier
+  __shared__ u32 s_cnt[3];
+  if (tid < 3) s_cnt[tid] = 0;
   __syncthreads();
-  if (tid == 0) {
-    if (s_hbm) atomicAdd(&l.n_hbm[ci], s_hbm);
-    if (s_host) atomicAdd(&l.n_host[ci], s_host);
-    if (s_remote) atomicAdd(&l.n_remote[ci], s_remote);
+  const u32 m0 = __ballot_sync(0xFFFFFFFFu, tier == 0), m1 = __ballot_sync(0xFFFFFFFFu, tier == 1),
+            m2 = __ballot_sync(0xFFFFFFFFu, tier == 2);
+  if ((tid & 31) == 0) {
+    if (m0) atomicAdd(&s_cnt[0], (u32)__popc(m0));
+    if (m1) atomicAdd(&s_cnt[1], (u32)__popc(m1));
+    if (m2) atomicAdd(&s_cnt[2], (u32)__popc(m2));
   }
+  __syncthreads();
+  if (tid == 0 && s_cnt[0]) atomicAdd(&l.n_hbm[ci], s_cnt[0]);
+  if (tid == 1 && s_cnt[1]) atomicAdd(&l.n_host[ci], s_cnt[1]);
+  if (tid == 2 && s_cnt[2]) atomicAdd(&l.n_remote[ci], s_cnt[2]);
 }
 
 // ======================================================================================================
@@ -759,6 +760,7 @@ struct ClsArgs {
 
 // Context that owns mapping g (the last one whose map_base is <= g). Every thread of the CTA calls it: the
 // bases are staged in shared memory by one round of loads when they fit.
+constexpr u32 CTX_STAGE = 1024;
 __device__ __forceinline__ u32 cls_ctx_of_mapping(const ClsArgs &a, u32 g) {
   __shared__ u32 s_base[CTX_STAGE];
   const bool staged = a.n_ctx <= CTX_STAGE;
