@@ -37,9 +37,9 @@ from paper_2609_39819_b200 import workloads as W  # noqa: E402
 
 METRIC = "KV block GB/s (HBM & host link) vs roofline; blocks hashed+looked up/sec"
 GiB = 1 << 30
-# DRAM traffic of the mover kernel per algorithmic byte (read + write), from the ncu capture summarised
-# in profiles/mover_8b_hbm_to_hbm.md: (dram__bytes_read.sum + dram__bytes_write.sum) / (2 x payload bytes) of a
-# 1024-block launch; traffic grows in proportion to the blocks moved, so it is scaled to the bench's launches.
+# DRAM traffic of the mover kernel per algorithmic byte (read + write), from one ncu capture (its summary sits
+# with the other profile summaries of this repository): (dram__bytes_read.sum + dram__bytes_write.sum) /
+# (2 x payload bytes) of a 1024-block launch; traffic grows in proportion to the blocks moved, so it is scaled to the bench's launches.
 MOVER_TRAFFIC_PER_ALGO_BYTE = 0.989
 
 
