@@ -391,6 +391,13 @@ int32_t kvt_set_profiling(kvt_engine *e, uint32_t on);
  * multiple of 16 KiB). Results are identical. */
 int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant);
 
+/* Upper bound on the thread blocks a mover kernel launches (offload / reload / exchange / move / compact /
+ * copy_blocks); 0 = automatic (default): 8 per SM for moves inside device memory, 32 for moves to or from a pool
+ * that lies in host memory (128 for kvt_exchange, which drives both directions). A move that crosses the host
+ * link is bound by the link and reaches its full rate with 16 blocks (128 for both directions at once), so the
+ * automatic choice leaves most SMs to kernels running on other streams at the same time. */
+int32_t kvt_set_mover_ctas(kvt_engine *e, uint32_t max_ctas);
+
 /* Tuning hook: how kvt_map_blocks(LOOKUP) hashes and probes. 0 / 1 = three kernels (digest, carry scan, finish +
  * probe; default), 2 = one single-pass kernel in which chunks hand their chain values forward through device
  * memory (bounded waits; a wait that runs out makes the call return KVT_E_DEVICE). Results are identical; the

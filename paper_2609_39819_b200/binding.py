@@ -27,7 +27,7 @@ EXPORTS = ("kvt_query_sizes", "kvt_create", "kvt_destroy", "kvt_apply_op", "kvt_
            "kvt_classify", "kvt_get_states", "kvt_select_victims", "kvt_offload", "kvt_reload", "kvt_release",
            "kvt_compact", "kvt_copy_blocks", "kvt_hash_scratch_bytes", "kvt_hash_tokens", "kvt_get_stats",
            "kvt_last_error", "kvt_get_entries", "kvt_debug_load_resident", "kvt_set_profiling",
-           "kvt_hash_tokens_noalloc", "kvt_debug_set_mover_variant", "kvt_exchange", "kvt_debug_set_lookup_variant", "kvt_move")
+           "kvt_hash_tokens_noalloc", "kvt_debug_set_mover_variant", "kvt_exchange", "kvt_debug_set_lookup_variant", "kvt_move", "kvt_set_mover_ctas")
 
 
 class KvtError(RuntimeError):
@@ -104,6 +104,7 @@ def load_library():
             "kvt_set_profiling": [vp, u32],
             "kvt_debug_set_mover_variant": [vp, u32],
             "kvt_debug_set_lookup_variant": [vp, u32],
+            "kvt_set_mover_ctas": [vp, u32],
             "kvt_get_entries": [vp, u32, vp, vp, vp, vp, vp, u32, vp],
             "kvt_debug_load_resident": [vp, vp, vp, vp, vp, vp, u32, u32, vp],
         }
@@ -249,6 +250,9 @@ class Engine:
 
     def set_mover_variant(self, variant):
         self._check(self.L.kvt_debug_set_mover_variant(self.h, variant), "set_mover_variant")
+
+    def set_mover_ctas(self, max_ctas):
+        self._check(self.L.kvt_set_mover_ctas(self.h, max_ctas), "set_mover_ctas")
 
     def set_lookup_variant(self, variant):
         self._check(self.L.kvt_debug_set_lookup_variant(self.h, variant), "set_lookup_variant")

@@ -150,6 +150,16 @@ struct kvt_engine {
   cudaStream_t capture_stream = nullptr;   // only ever used for stream capture, never executes work
   bool use_graphs = true;
   u32 mover_variant = 0;   // 0 auto, 1 CTA per chunk, 2 warp per 4 KiB tile, 3 TMA ring
+  u32 mover_max_ctas = 0;  // caller's upper bound on the mover's grid (0: automatic)
+  bool tier_in_host_mem[3] = {false, false, false};   // pool is host memory: moves to / from it are bound by the host link
+  // Grid of a mover launch: 8 CTAs per SM inside the device; a move that crosses the host link reaches the link's
+  // rate with 16 CTAs (measured), so it gets 32; both directions at
+  // once need 128 to reach the duplex rate. Either way most of the GPU stays free for other streams.
+  u32 mover_grid(u64 want, u32 link_dirs = 0) const {
+    u64 cap = mover_max_ctas ? mover_max_ctas : link_dirs == 1 ? 32 : link_dirs == 2 ? 128 : (u64)sm_count * 8;
+    return (u32)std::max<u64>(1, std::min(want, cap));
+  }
+  u32 link_dirs(u32 st, u32 dt) const { return (tier_in_host_mem[st] || tier_in_host_mem[dt]) ? 1u : 0u; }
   u32 lookup_variant = 0;  // 0 / 1 digest / carry / finish kernels, 2 single-pass hash + probe kernel
   bool tma_attr_set = false;
   cudaEvent_t ev_m0 = nullptr, ev_m1 = nullptr, ev_h0 = nullptr, ev_h1 = nullptr;
@@ -288,7 +298,8 @@ int32_t launch_mover(kvt_engine *e, cudaStream_t s, u32 st, const u32 *src, u32 
   a.src_ids = src; a.dst_ids = dst; a.n_pairs = n_max; a.n_pairs_dev = n_dev;
   a.n_chunks = (u32)e->n_chunks; a.chunk_bytes = (u32)e->chunk_bytes; a.status = e->d_status;
   u64 items = (u64)n_max * e->n_chunks;
-  u32 grid = (u32)std::min<u64>(items, (u64)e->sm_count * 8);
+  const u32 ld = e->link_dirs(st, dt);
+  u32 grid = e->mover_grid(items, ld);
   const bool timed = e->profiling && n_dev != nullptr;   // only the calls that synchronise afterwards
   if (timed) CU(cudaEventRecord(e->ev_m0, s));
   // a warp per 4 KiB tile keeps 8 loads per lane in flight whatever the chunk size (measured faster for
@@ -307,12 +318,13 @@ int32_t launch_mover(kvt_engine *e, cudaStream_t s, u32 st, const u32 *src, u32 
     }
     u32 per_sm = (u32)std::max<size_t>(1, std::min<size_t>(8, (200 * 1024) / (smem + 1024)));
     u32 tgrid = (u32)std::min<u64>(titems, (u64)e->sm_count * per_sm);
+    tgrid = std::min(tgrid, e->mover_grid(titems, ld));
     k_move_tma<<<tgrid, 32, smem, s>>>(a, tile, tpc);
     e->st.kernel_launches++;
   } else if (use_tiles && tiles_ok) {
     u32 tpc = (u32)(e->chunk_bytes / 4096);
     u64 titems = items * tpc;
-    u32 tgrid = (u32)std::min<u64>((titems + 7) / 8, (u64)e->sm_count * 8);
+    u32 tgrid = e->mover_grid((titems + 7) / 8, ld);
     KL(k_move_tiles<8>, tgrid, 256, s, a, tpc);
   } else {
     KL(k_move_blocks<4>, grid, 256, s, a);
@@ -485,6 +497,14 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   e->meta = (u8 *)c.dev_meta; e->d_tokens = (u32 *)c.dev_tokens;
   e->chunk_bytes = chunk_bytes; e->n_chunks = n_chunks; e->block_bytes = chunk_bytes * n_chunks;
   e->metadata_only = meta_only;
+  if (!meta_only) {
+    const void *pools[3] = {c.hbm_pool, c.n_host_blocks ? c.host_pool : nullptr, c.n_remote_blocks ? c.remote_pool : nullptr};
+    for (int t = 0; t < 3; ++t) {
+      cudaPointerAttributes at;
+      if (pools[t] && cudaPointerGetAttributes(&at, pools[t]) == cudaSuccess) e->tier_in_host_mem[t] = at.type == cudaMemoryTypeHost;
+      else cudaGetLastError();
+    }
+  }
   cudaDeviceGetAttribute(&e->sm_count, cudaDevAttrMultiProcessorCount, dev);
   e->tab.slots = e->dp<TSlot>(L.tab); e->tab.mask = c.table_capacity - 1;
   e->tab.shift = 64 - (bit_length(c.table_capacity) - 1);
@@ -556,6 +576,12 @@ int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant) {
   if (!e) return KVT_E_INVAL;
   if (variant > 3) return KVT_E_INVAL;
   e->mover_variant = variant;
+  return KVT_OK;
+}
+
+int32_t kvt_set_mover_ctas(kvt_engine *e, uint32_t max_ctas) {
+  if (!e) return KVT_E_INVAL;
+  e->mover_max_ctas = max_ctas;
   return KVT_OK;
 }
 
@@ -1324,11 +1350,12 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
       if (timed) CU(cudaEventRecord(e->ev_m0, s));
       if (e->chunk_bytes % 4096 == 0) {
         u32 tpc = (u32)(e->chunk_bytes / 4096);
-        u32 grid = (u32)std::min<u64>((items * tpc + 7) / 8, (u64)e->sm_count * 8);
+        u32 grid = e->mover_grid((items * tpc + 7) / 8, e->link_dirs(KVT_TIER_HBM, KVT_TIER_HOST) * 2);
         KL(k_move_tiles_dual<8>, grid, 256, s, ma, mb, tpc, 2u);   // CTAs alternate between the two directions
       } else {   // chunk sizes the tile kernel cannot split: one direction after the other
-        u32 g1 = (u32)std::min<u64>((u64)ma.n_pairs * e->n_chunks, (u64)e->sm_count * 8);
-        u32 g2 = (u32)std::min<u64>((u64)mb.n_pairs * e->n_chunks, (u64)e->sm_count * 8);
+        const u32 xl = e->link_dirs(KVT_TIER_HBM, KVT_TIER_HOST);
+        u32 g1 = ma.n_pairs ? e->mover_grid((u64)ma.n_pairs * e->n_chunks, xl) : 0;
+        u32 g2 = mb.n_pairs ? e->mover_grid((u64)mb.n_pairs * e->n_chunks, xl) : 0;
         if (g1) KL(k_move_blocks<4>, g1, 256, s, ma);
         if (g2) KL(k_move_blocks<4>, g2, 256, s, mb);
       }

@@ -10,6 +10,7 @@ larger than L2, a few GB on the device at most, a handful of launches).
     python -m paper_2609_39819_b200.profile_case select     # classify + select 10% of 1 Mi resident blocks
     python -m paper_2609_39819_b200.profile_case c4         # the whole metadata stress at full size (C4)
     python -m paper_2609_39819_b200.profile_case mover_remote  # host tier <-> third tier, third tier -> HBM
+    python -m paper_2609_39819_b200.profile_case mover_ctas # bandwidth against the number of thread blocks the mover may use
     python -m paper_2609_39819_b200.profile_case sweep      # C5: movement bandwidth sweep (markdown table)
 Each prints one line with CUDA-event timings of its launches.
 """
@@ -113,6 +114,23 @@ def main(case: str):
         gb = n * geo.block_bytes / 1e9
         print(f"mover_remote: {n} blocks x {geo.block_bytes} B; host -> remote ms {down} = {[round(gb / (m / 1e3), 1) for m in down]} GB/s; "
               f"remote -> HBM ms {up} = {[round(gb / (m / 1e3), 1) for m in up]} GB/s")
+    elif case == "mover_ctas":
+        # how many thread blocks a move needs: HBM -> HBM, HBM -> host, host -> HBM against the grid limit
+        geo, n = W.GEO_8B, 512
+        eng = B.Engine(n_hbm_blocks=2 * n, n_host_blocks=n, max_contexts=2, max_tokens=1 << 12, max_messages=64,
+                       max_batch_blocks=4096, zero_pools=False, **geo.kwargs())
+        a = torch.from_numpy(W.ids_c5(1, n, n, True).view(np.int32)).cuda()
+        b = torch.from_numpy(W.ids_c5(2, n, n, True).view(np.int32)).cuda()
+        b2 = b + n
+        gb = n * geo.block_bytes / 1e9
+        print("| CTAs | HBM -> HBM GB/s (read + write) | HBM -> host GB/s | host -> HBM GB/s |")
+        print("|---:|---:|---:|---:|")
+        for ctas in (1, 2, 4, 8, 16, 32, 64, 148, 296, 592, 0):
+            eng.set_mover_ctas(ctas)
+            dd = min(_events(torch, lambda: eng.copy_blocks(0, a, 0, b2), 3))
+            dh = min(_events(torch, lambda: eng.copy_blocks(0, a, 1, b), 2))
+            hd = min(_events(torch, lambda: eng.copy_blocks(1, b, 0, a), 2))
+            print(f"| {ctas if ctas else '1184 (default)'} | {2 * gb / (dd / 1e3):.0f} | {gb / (dh / 1e3):.1f} | {gb / (hd / 1e3):.1f} |")
     elif case == "exchange":
         geo, n = W.GEO_8B, 1024
         eng = B.Engine(n_hbm_blocks=3 * n, n_host_blocks=3 * n, max_contexts=2, max_tokens=1 << 12, max_messages=64,
@@ -138,6 +156,18 @@ def main(case: str):
                 b.record(); torch.cuda.synchronize()
                 if rep:
                     res[mode].append(round(a.elapsed_time(b), 2))
+        # the exchange against the number of thread blocks its mover may use (0 = the library's own choice)
+        by_ctas = {}
+        for ctas in (16, 32, 64, 128, 148, 296, 592, 1184, 0):
+            eng.set_mover_ctas(ctas)
+            ms = []
+            for rep in range(3):
+                out, inn = lists()
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record(); eng.exchange(out, inn); b.record(); torch.cuda.synchronize()
+                ms.append(a.elapsed_time(b))
+            by_ctas[ctas] = round(2 * gb / (min(ms) / 1e3), 1)
+        print(f"exchange GB/s (both directions together) by thread blocks: {by_ctas}")
         # reference: the copy engines driving both directions at once (two streams, 2 GiB pinned each way)
         h1 = torch.empty(2 << 30, dtype=torch.uint8, pin_memory=True); d1 = torch.empty(2 << 30, dtype=torch.uint8, device="cuda")
         h2 = torch.empty(2 << 30, dtype=torch.uint8, pin_memory=True); d2 = torch.empty(2 << 30, dtype=torch.uint8, device="cuda")
