@@ -392,10 +392,10 @@ int32_t kvt_set_profiling(kvt_engine *e, uint32_t on);
 int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant);
 
 /* Upper bound on the thread blocks a mover kernel launches (offload / reload / exchange / move / compact /
- * copy_blocks); 0 = automatic (default): 8 per SM for moves inside device memory, 32 for moves to or from a pool
- * that lies in host memory (128 for kvt_exchange, which drives both directions). A move that crosses the host
- * link is bound by the link and reaches its full rate with 16 blocks (128 for both directions at once), so the
- * automatic choice leaves most SMs to kernels running on other streams at the same time. */
+ * copy_blocks); 0 = automatic (default): 8 blocks of 256 threads per SM for moves inside device memory; for a move
+ * to or from a pool that lies in host memory 4 blocks of 1024 threads (32 for kvt_exchange, which drives both
+ * directions). A move that crosses the host link is bound by the link, 128 warps keep it full, and packing them
+ * into a few large blocks leaves all other SMs to kernels running on other streams at the same time. */
 int32_t kvt_set_mover_ctas(kvt_engine *e, uint32_t max_ctas);
 
 /* Tuning hook: how kvt_map_blocks(LOOKUP) hashes and probes. 0 / 1 = three kernels (digest, carry scan, finish +

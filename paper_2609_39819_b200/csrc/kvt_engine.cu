@@ -152,11 +152,11 @@ struct kvt_engine {
   u32 mover_variant = 0;   // 0 auto, 1 CTA per chunk, 2 warp per 4 KiB tile, 3 TMA ring
   u32 mover_max_ctas = 0;  // caller's upper bound on the mover's grid (0: automatic)
   bool tier_in_host_mem[3] = {false, false, false};   // pool is host memory: moves to / from it are bound by the host link
-  // Grid of a mover launch: 8 CTAs per SM inside the device; a move that crosses the host link reaches the link's
-  // rate with 16 CTAs (measured), so it gets 32; both directions at
-  // once need 128 to reach the duplex rate. Either way most of the GPU stays free for other streams.
+  // Grid of a mover launch. Inside the device: 8 CTAs of 256 threads per SM. A move that crosses the host link
+  // is bound by the link: 128 warps keep it full (measured), and a GEMM on another stream loses every SM a mover
+  // CTA sits on, so those warps are packed into 4 CTAs of 1024 threads (32 for both directions at once).
   u32 mover_grid(u64 want, u32 link_dirs = 0) const {
-    u64 cap = mover_max_ctas ? mover_max_ctas : link_dirs == 1 ? 32 : link_dirs == 2 ? 128 : (u64)sm_count * 8;
+    u64 cap = mover_max_ctas ? mover_max_ctas : link_dirs == 1 ? 4 : link_dirs == 2 ? 32 : (u64)sm_count * 8;
     return (u32)std::max<u64>(1, std::min(want, cap));
   }
   u32 link_dirs(u32 st, u32 dt) const { return (tier_in_host_mem[st] || tier_in_host_mem[dt]) ? 1u : 0u; }
@@ -299,7 +299,7 @@ int32_t launch_mover(kvt_engine *e, cudaStream_t s, u32 st, const u32 *src, u32 
   a.n_chunks = (u32)e->n_chunks; a.chunk_bytes = (u32)e->chunk_bytes; a.status = e->d_status;
   u64 items = (u64)n_max * e->n_chunks;
   const u32 ld = e->link_dirs(st, dt);
-  u32 grid = e->mover_grid(items, ld);
+  u32 grid = e->mover_grid(items, ld) * (ld && !e->mover_max_ctas ? 4 : 1);   // 256-thread CTAs: four for one of 1024
   const bool timed = e->profiling && n_dev != nullptr;   // only the calls that synchronise afterwards
   if (timed) CU(cudaEventRecord(e->ev_m0, s));
   // a warp per 4 KiB tile keeps 8 loads per lane in flight whatever the chunk size (measured faster for
@@ -318,14 +318,19 @@ int32_t launch_mover(kvt_engine *e, cudaStream_t s, u32 st, const u32 *src, u32 
     }
     u32 per_sm = (u32)std::max<size_t>(1, std::min<size_t>(8, (200 * 1024) / (smem + 1024)));
     u32 tgrid = (u32)std::min<u64>(titems, (u64)e->sm_count * per_sm);
-    tgrid = std::min(tgrid, e->mover_grid(titems, ld));
+    tgrid = std::min(tgrid, e->mover_grid(titems, ld) * (ld && !e->mover_max_ctas ? 8 : 1));   // one warp per CTA here
     k_move_tma<<<tgrid, 32, smem, s>>>(a, tile, tpc);
     e->st.kernel_launches++;
   } else if (use_tiles && tiles_ok) {
     u32 tpc = (u32)(e->chunk_bytes / 4096);
     u64 titems = items * tpc;
-    u32 tgrid = e->mover_grid((titems + 7) / 8, ld);
-    KL(k_move_tiles<8>, tgrid, 256, s, a, tpc);
+    if (ld) {   // link-bound: few, large CTAs (see mover_grid)
+      u32 tgrid = e->mover_grid((titems + 31) / 32, ld);
+      KL((k_move_tiles<8, 1024>), tgrid, 1024, s, a, tpc);
+    } else {
+      u32 tgrid = e->mover_grid((titems + 7) / 8, ld);
+      KL(k_move_tiles<8>, tgrid, 256, s, a, tpc);
+    }
   } else {
     KL(k_move_blocks<4>, grid, 256, s, a);
   }
@@ -1350,8 +1355,14 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
       if (timed) CU(cudaEventRecord(e->ev_m0, s));
       if (e->chunk_bytes % 4096 == 0) {
         u32 tpc = (u32)(e->chunk_bytes / 4096);
-        u32 grid = e->mover_grid((items * tpc + 7) / 8, e->link_dirs(KVT_TIER_HBM, KVT_TIER_HOST) * 2);
-        KL(k_move_tiles_dual<8>, grid, 256, s, ma, mb, tpc, 2u);   // CTAs alternate between the two directions
+        const u32 xl = e->link_dirs(KVT_TIER_HBM, KVT_TIER_HOST) * 2;
+        if (xl) {
+          u32 grid = std::max(2u, e->mover_grid((items * tpc + 31) / 32, xl));
+          KL((k_move_tiles_dual<8, 1024>), grid, 1024, s, ma, mb, tpc, 2u);
+        } else {
+          u32 grid = e->mover_grid((items * tpc + 7) / 8, xl);
+          KL(k_move_tiles_dual<8>, grid, 256, s, ma, mb, tpc, 2u);   // CTAs alternate between the two directions
+        }
       } else {   // chunk sizes the tile kernel cannot split: one direction after the other
         const u32 xl = e->link_dirs(KVT_TIER_HBM, KVT_TIER_HOST);
         u32 g1 = ma.n_pairs ? e->mover_grid((u64)ma.n_pairs * e->n_chunks, xl) : 0;

@@ -1210,15 +1210,16 @@ __global__ void __launch_bounds__(256) k_move_blocks(MoveArgs a) {
 
 // Variant for small chunks: work item = 32 lanes x 16 B x UNROLL bytes of one chunk, one item per warp
 // at a time, so that a 4 KiB chunk keeps UNROLL loads per lane in flight instead of one.
-template <int UNROLL>
-__global__ void __launch_bounds__(256) k_move_tiles(MoveArgs a, u32 tiles_per_chunk) {
+template <int UNROLL, int THREADS = 256>
+__global__ void __launch_bounds__(THREADS) k_move_tiles(MoveArgs a, u32 tiles_per_chunk) {
+  constexpr u32 WPC = THREADS / 32;   // warps per CTA
   u32 n_pairs = a.n_pairs;
   if (a.n_pairs_dev) n_pairs = min(n_pairs, *a.n_pairs_dev);
   const u32 lane = threadIdx.x & 31;
   const u64 per_pair = (u64)a.n_chunks * tiles_per_chunk;
   const u64 n_items = (u64)n_pairs * per_pair;
-  const u64 n_warps = (u64)gridDim.x * 8;
-  for (u64 item = (u64)blockIdx.x * 8 + (threadIdx.x >> 5); item < n_items; item += n_warps) {
+  const u64 n_warps = (u64)gridDim.x * WPC;
+  for (u64 item = (u64)blockIdx.x * WPC + (threadIdx.x >> 5); item < n_items; item += n_warps) {
     u32 pair = (u32)(item / per_pair);
     u32 rem = (u32)(item - (u64)pair * per_pair);
     u32 chunk = rem / tiles_per_chunk, tile = rem - chunk * tiles_per_chunk;
@@ -1239,8 +1240,9 @@ __global__ void __launch_bounds__(256) k_move_tiles(MoveArgs a, u32 tiles_per_ch
 // Two independent pair lists in one launch (kvt_exchange): even CTAs work on list a, odd CTAs on list b (or all
 // CTAs on the one that has work), so that loads from and stores to the host tier are in flight at the same time
 // (the link is full duplex) and neither direction waits for the other's latency.
-template <int UNROLL>
-__global__ void __launch_bounds__(256) k_move_tiles_dual(MoveArgs a, MoveArgs b, u32 tiles_per_chunk, u32 b_every) {
+template <int UNROLL, int THREADS = 256>
+__global__ void __launch_bounds__(THREADS) k_move_tiles_dual(MoveArgs a, MoveArgs b, u32 tiles_per_chunk, u32 b_every) {
+  constexpr u32 WPC = THREADS / 32;
   u32 na = a.n_pairs, nb = b.n_pairs;
   if (a.n_pairs_dev) na = min(na, *a.n_pairs_dev);
   if (b.n_pairs_dev) nb = min(nb, *b.n_pairs_dev);
@@ -1265,8 +1267,8 @@ __global__ void __launch_bounds__(256) k_move_tiles_dual(MoveArgs a, MoveArgs b,
     }
     const MoveArgs &m = from_b ? b : a;
     const u64 n_items = (u64)(from_b ? nb : na) * per_pair;
-    const u64 n_warps = (u64)n_cta * 8;
-    for (u64 k = (u64)my_cta * 8 + (threadIdx.x >> 5); k < n_items; k += n_warps) {
+    const u64 n_warps = (u64)n_cta * WPC;
+    for (u64 k = (u64)my_cta * WPC + (threadIdx.x >> 5); k < n_items; k += n_warps) {
       u32 pair = (u32)(k / per_pair);
       u32 rem = (u32)(k - (u64)pair * per_pair);
       u32 chunk = rem / tiles_per_chunk, tile = rem - chunk * tiles_per_chunk;

@@ -11,6 +11,7 @@ larger than L2, a few GB on the device at most, a handful of launches).
     python -m paper_2609_39819_b200.profile_case c4         # the whole metadata stress at full size (C4)
     python -m paper_2609_39819_b200.profile_case mover_remote  # host tier <-> third tier, third tier -> HBM
     python -m paper_2609_39819_b200.profile_case mover_ctas # bandwidth against the number of thread blocks the mover may use
+    python -m paper_2609_39819_b200.profile_case overlap    # a GEMM loop beside an offload: what the mover's grid size costs
     python -m paper_2609_39819_b200.profile_case sweep      # C5: movement bandwidth sweep (markdown table)
 Each prints one line with CUDA-event timings of its launches.
 """
@@ -123,14 +124,52 @@ def main(case: str):
         b = torch.from_numpy(W.ids_c5(2, n, n, True).view(np.int32)).cuda()
         b2 = b + n
         gb = n * geo.block_bytes / 1e9
-        print("| CTAs | HBM -> HBM GB/s (read + write) | HBM -> host GB/s | host -> HBM GB/s |")
+        print("| thread blocks (256 threads inside the device, 1024 over the link) | HBM -> HBM GB/s (read + write) | HBM -> host GB/s | host -> HBM GB/s |")
         print("|---:|---:|---:|---:|")
         for ctas in (1, 2, 4, 8, 16, 32, 64, 148, 296, 592, 0):
             eng.set_mover_ctas(ctas)
             dd = min(_events(torch, lambda: eng.copy_blocks(0, a, 0, b2), 3))
             dh = min(_events(torch, lambda: eng.copy_blocks(0, a, 1, b), 2))
             hd = min(_events(torch, lambda: eng.copy_blocks(1, b, 0, a), 2))
-            print(f"| {ctas if ctas else '1184 (default)'} | {2 * gb / (dd / 1e3):.0f} | {gb / (dh / 1e3):.1f} | {gb / (hd / 1e3):.1f} |")
+            print(f"| {ctas if ctas else 'automatic'} | {2 * gb / (dd / 1e3):.0f} | {gb / (dh / 1e3):.1f} | {gb / (hd / 1e3):.1f} |")
+    elif case == "overlap":
+        # a dense bf16 GEMM loop on one stream while the mover pushes 2 GiB to the pinned host tier on another:
+        # GEMM time alone and beside movers of different grid sizes
+        geo, n = W.GEO_8B, 1024
+        eng = B.Engine(n_hbm_blocks=n, n_host_blocks=n, max_contexts=2, max_tokens=1 << 12, max_messages=64,
+                       max_batch_blocks=4096, zero_pools=False, **geo.kwargs())
+        src = torch.from_numpy(W.ids_c5(1, n, n, True).view(np.int32)).cuda()
+        dst = torch.from_numpy(W.ids_c5(2, n, n, True).view(np.int32)).cuda()
+        x = torch.randn(8192, 8192, dtype=torch.bfloat16, device="cuda")
+        y = torch.randn(8192, 8192, dtype=torch.bfloat16, device="cuda")
+        s_move, s_gemm = torch.cuda.Stream(), torch.cuda.Stream()
+        n_gemm = 40
+
+        def run(ctas):
+            torch.cuda.synchronize()
+            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            if ctas is not None:
+                eng.set_mover_ctas(ctas)
+                with torch.cuda.stream(s_move):
+                    m0.record(); eng.copy_blocks(0, src, 1, dst); m1.record()
+            with torch.cuda.stream(s_gemm):
+                g0.record()
+                for _ in range(n_gemm):
+                    torch.matmul(x, y)
+                g1.record()
+            torch.cuda.synchronize()
+            return g0.elapsed_time(g1), (m0.elapsed_time(m1) if ctas is not None else 0.0)
+
+        run(None); run(0)
+        flop = 2 * 8192 ** 3 * n_gemm
+        gb = n * geo.block_bytes / 1e9
+        cases = [("GEMM alone", None), ("beside the mover, automatic grid (4 blocks of 1024 threads)", 0)] + \
+                [(f"beside the mover on {c} blocks of 1024 threads", c) for c in (1, 2, 8, 32, 148, 296)]
+        for label, ctas in cases:
+            g, m = min(run(ctas) for _ in range(3))
+            mv = f", move {m:.1f} ms = {gb / (m / 1e3):.1f} GB/s" if ctas is not None else ""
+            print(f"overlap: {label}: {n_gemm} GEMMs in {g:.1f} ms = {flop / (g / 1e3) / 1e12:.0f} TFLOP/s{mv}")
     elif case == "exchange":
         geo, n = W.GEO_8B, 1024
         eng = B.Engine(n_hbm_blocks=3 * n, n_host_blocks=3 * n, max_contexts=2, max_tokens=1 << 12, max_messages=64,
@@ -158,7 +197,7 @@ def main(case: str):
                     res[mode].append(round(a.elapsed_time(b), 2))
         # the exchange against the number of thread blocks its mover may use (0 = the library's own choice)
         by_ctas = {}
-        for ctas in (16, 32, 64, 128, 148, 296, 592, 1184, 0):
+        for ctas in (2, 4, 8, 16, 32, 64, 148, 0):
             eng.set_mover_ctas(ctas)
             ms = []
             for rep in range(3):
