@@ -40,3 +40,23 @@ def test_struct_sizes_match_the_header():
     assert ctypes.sizeof(binding.Config) == 14 * 4 + 3 * 8 + 2 * 4 + 10 * 8
     assert ctypes.sizeof(binding.Op) == 8 * 4 + 8
     assert binding.CALL_INFO_DTYPE.itemsize == 9 * 4
+
+
+def test_stats_and_call_info_fields_follow_the_header():
+    """The bindings unpack kvt_stats / kvt_call_info by position: their field lists must be the header's, in order."""
+    import re
+    from paper_2609_39819_b200 import binding
+    from oracle import kvt_oracle
+    text = open(os.path.join(ROOT, "include", "kvt.h")).read()
+
+    def fields(struct, ctype):
+        body = text[text.index(f"typedef struct {struct}"):text.index(f"}} {struct};")]
+        out = []
+        for decl in re.findall(ctype + r"\s+([^;]+);", body):
+            out += [x.strip() for x in decl.split(",")]
+        return out
+
+    stats = fields("kvt_stats", "uint64_t")
+    assert stats == list(binding.STATS_FIELDS) == list(kvt_oracle.STATS_FIELDS)
+    info = fields("kvt_call_info", "uint32_t")
+    assert info == list(binding.CALL_INFO_DTYPE.names) == list(kvt_oracle.CALL_INFO_DTYPE.names)
