@@ -231,7 +231,7 @@ def main(case: str):
     elif case == "hash_big":
         n_tok = 64 << 20
         tok = torch.randint(0, W.VOCAB, (n_tok,), dtype=torch.int32, device="cuda")
-        ms = _events(torch, lambda: B.hash_tokens(tok, 0), 3)
+        ms = _events(torch, lambda: B.hash_tokens(tok, 0), 8)
         nb = n_tok // 16
         print(f"hash_big: {nb} blocks, ms per call {ms}, blocks/s {[round(nb / (m / 1e3)) for m in ms]}, "
               f"GB/s at 72 B per block {[round(72 * nb / (m / 1e3) / 1e9, 1) for m in ms]}")
