@@ -178,12 +178,35 @@ struct LaneTable {
 };
 __device__ const LaneTable g_lane_mult = LaneTable();
 
-// tok * K mod 2^64 for a 32-bit token: one widening multiply-add for the low word of K, one 32-bit multiply for
-// its high word (a full 64 x 64 multiply costs twice as much on the integer pipe, which bounds this kernel).
-__device__ __forceinline__ u64 mul_tok(u32 tok, u64 k) {
-  u64 lo = (u64)tok * (u32)k;
-  u32 hi = tok * (u32)(k >> 32);
-  return lo + ((u64)hi << 32);
+// Block digests of one 256-block chunk from the quad layout (lane q of a quad holds tokens 4q..4q+3 of the blocks
+// it*64 + tid/4, it = 0..3): weighted sums, quad reduction, mix; sd[blk] = d_blk (0 beyond nb).
+__device__ __forceinline__ void digest_quads(const uint4 (&v)[4], u32 q, u64 k0, u64 k1, u64 k2, u64 k3, u64 ksum,
+                                             u32 tid, u32 nb, u64 *sd) {
+  // per iteration: low words of the multipliers through widening multiply-adds into one 64-bit accumulator, high
+  // words through 32-bit multiply-adds into one 32-bit accumulator (tok * K mod 2^64 = tok*Klo + ((tok*Khi) << 32))
+  const u32 k0l = (u32)k0, k1l = (u32)k1, k2l = (u32)k2, k3l = (u32)k3;
+  const u32 k0h = (u32)(k0 >> 32), k1h = (u32)(k1 >> 32), k2h = (u32)(k2 >> 32), k3h = (u32)(k3 >> 32);
+  u64 part[4];
+#pragma unroll
+  for (int it = 0; it < 4; ++it) {
+    u64 lo = ksum;
+    lo += (u64)v[it].x * k0l; lo += (u64)v[it].y * k1l; lo += (u64)v[it].z * k2l; lo += (u64)v[it].w * k3l;
+    u32 hi = v[it].x * k0h + v[it].y * k1h + v[it].z * k2h + v[it].w * k3h;
+    part[it] = lo + ((u64)hi << 32);
+  }
+  // quad reduction that leaves lane q with the block of iteration q: two exchange steps, each lane passing on the
+  // halves it does not keep (3 64-bit shuffles instead of 8)
+  {
+    const bool up2 = q & 2, up1 = q & 1;
+    u64 keep0 = up2 ? part[2] : part[0], keep1 = up2 ? part[3] : part[1];
+    u64 send0 = up2 ? part[0] : part[2], send1 = up2 ? part[1] : part[3];
+    keep0 += __shfl_xor_sync(0xFFFFFFFFu, send0, 2);
+    keep1 += __shfl_xor_sync(0xFFFFFFFFu, send1, 2);
+    u64 keep = up1 ? keep1 : keep0, send = up1 ? keep0 : keep1;
+    keep += __shfl_xor_sync(0xFFFFFFFFu, send, 1);
+    u32 blk = (q * CHUNK + tid) >> 2;
+    sd[blk] = blk < nb ? mix64(keep) : 0;
+  }
 }
 
 __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
@@ -207,18 +230,7 @@ __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   }
   // iteration `it` covers blocks it*64 .. it*64+63, four lanes per block; after the two exchange steps every
   // lane of a quad holds the four block sums, and lane q finishes the block of iteration q
-  u64 mine = 0;
-#pragma unroll
-  for (int it = 0; it < 4; ++it) {
-    u64 s = ksum + mul_tok(v[it].x, k0) + mul_tok(v[it].y, k1) + mul_tok(v[it].z, k2) + mul_tok(v[it].w, k3);
-    s += __shfl_xor_sync(0xFFFFFFFFu, s, 1);
-    s += __shfl_xor_sync(0xFFFFFFFFu, s, 2);
-    if ((u32)it == q) mine = s;
-  }
-  {
-    u32 blk = (q * CHUNK + tid) >> 2;
-    sd[blk] = blk < nb ? mix64(mine) : 0;
-  }
+  digest_quads(v, q, k0, k1, k2, k3, ksum, tid, nb, sd);
   __syncthreads();
   // inclusive scan of c_t = sum_{i<=t} P^(t-i) d_i
   u64 cval = sd[tid];
@@ -396,18 +408,7 @@ __global__ void __launch_bounds__(CHUNK) k_hash_lookup_fused(HashArgs a, LookupA
       u32 idx = it * CHUNK + tid;
       v[it] = (idx >> 2) < nb ? __ldcs(tok + idx) : make_uint4(0, 0, 0, 0);
     }
-    u64 mine = 0;
-#pragma unroll
-    for (int it = 0; it < 4; ++it) {
-      u64 s = ksum + mul_tok(v[it].x, k0) + mul_tok(v[it].y, k1) + mul_tok(v[it].z, k2) + mul_tok(v[it].w, k3);
-      s += __shfl_xor_sync(0xFFFFFFFFu, s, 1);
-      s += __shfl_xor_sync(0xFFFFFFFFu, s, 2);
-      if ((u32)it == q) mine = s;
-    }
-    {
-      u32 blk = (q * CHUNK + tid) >> 2;
-      sd[blk] = blk < nb ? mix64(mine) : 0;
-    }
+    digest_quads(v, q, k0, k1, k2, k3, ksum, tid, nb, sd);
     __syncthreads();
     u64 cval = sd[tid];
     u64 pp = HASH_P;
