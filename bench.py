@@ -57,6 +57,7 @@ def parse_args():
     ap.add_argument("--skip-cpu", action="store_true")
     ap.add_argument("--skip-stress", action="store_true", help="skip the C4-shaped metadata measurement")
     ap.add_argument("--skip-inclusive", action="store_true", help="skip the extra end-to-end run with inclusive tiers")
+    ap.add_argument("--skip-two-tenants", action="store_true", help="skip the extra end-to-end run with two sessions")
     return ap.parse_args()
 
 
@@ -442,6 +443,73 @@ def gpu_arm(args, torch, B, setup, turns, n_ff, e2e, n_host_blocks, n_hbm_blocks
     return res
 
 
+def shift_ctx(turns, setup, by):
+    """The same session under other context ids (so that two sessions can share an engine)."""
+    def ev_(ev):
+        return (ev[0], ev[1] + by) + tuple(ev[2:])
+    return [ev_(ev) for ev in setup], [([ev_(ev) for ev in pre], [c + by for c in ctxs], [ev_(ev) for ev in post])
+                                       for pre, ctxs, post in turns]
+
+
+def two_tenant_arm(args, torch, B, n_ff, use_exchange, n_hbm_blocks=12288, n_host_blocks=12288):
+    """End-to-end side measurement without artificial pressure: two C2 sessions (seeds s, s + 1) take turns on an
+    HBM pool that holds one and a half of them (24 GiB) over a pinned host tier. Every call finds part of its prefix
+    on the host tier and has to push part of the other session out: with `use_exchange` the replay driver issues
+    the reload and the offload as one kvt_exchange (both directions of the link at once), otherwise as kvt_offload
+    followed by kvt_reload. Returns payload GB/s over the timed calls."""
+    W_, K = args.warmup, args.steps
+    sa, ta, _ = make_turns(args.seed, W_ + K + 4)
+    sb, tb, _ = make_turns(args.seed + 1, W_ + K + 4)
+    sb, tb = shift_ctx(tb, sb, 1)
+    n = min(len(ta), len(tb))
+    ff = n - (W_ + K)
+    max_tok = 1 << 22
+    eng = B.Engine(n_hbm_blocks=n_hbm_blocks, n_host_blocks=n_host_blocks, max_contexts=4, max_tokens=max_tok,
+                   max_messages=1 << 14, max_batch_blocks=max_tok // 16, zero_pools=False, **W.GEO_8B.kwargs())
+    cache = {}
+
+    def tok(arr):
+        k = id(arr)
+        if k not in cache:
+            cache[k] = torch.from_numpy(arr.view(np.int32)).pin_memory()
+        return cache[k]
+
+    opt = W.ReplayOptions(payload=None, record_states=False, use_exchange=use_exchange)
+    for ev in sa + sb:
+        apply_event(eng, ev, tok)
+
+    def call(turn):
+        pre, ctxs, post = turn
+        for ev in pre:
+            apply_event(eng, ev, tok)
+        W.run_call(eng, ctxs, opt)
+        for ev in post:
+            apply_event(eng, ev, tok)
+
+    for t in range(ff + W_):
+        call(ta[t]); call(tb[t])
+    torch.cuda.synchronize()
+    s0 = eng.get_stats()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    ev0.record()
+    for t in range(ff + W_, ff + W_ + K):
+        call(ta[t]); call(tb[t])
+    ev1.record()
+    torch.cuda.synchronize()
+    ms = ev0.elapsed_time(ev1)
+    s1 = eng.get_stats()
+    d = {k: s1[k] - s0[k] for k in s1}
+    out = {"value": kv_bytes(d, eng.block_bytes) / (ms / 1e3) / 1e9, "ms_per_call": ms / (2 * K),
+           "offloaded_per_call": d["offloaded"] / (2 * K), "reloaded_per_call": d["reloaded"] / (2 * K),
+           "dropped_per_call": d["dropped"] / (2 * K)}
+    eng.close()
+    del eng, cache
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    return out
+
+
 def metadata_stress(torch, B, hbm_peak, reps=5):
     """C4-shaped side measurement of the metadata stages at scale (the C2 calls above are launch-latency
     sized): 1 Mi resident blocks, one LOOKUP batch of 64 calls x 16,128 blocks, classification of the
@@ -724,6 +792,15 @@ def main():
             "offloaded_per_step": ist["offloaded"] / K, "offloaded_without_copy_per_step": ist["offloaded_clean"] / K,
             "reloaded_per_step": ist["reloaded"] / K, "bytes_over_link_per_step": (ist["bytes_d2h"] + ist["bytes_h2d"]) / K,
             "verified_blocks": i["verified"],
+        }
+    if e and not args.skip_two_tenants and world == 1 and mem_available_bytes() > 64 * GiB:
+        seq = two_tenant_arm(args, torch, B, n_ff, False)
+        dup = two_tenant_arm(args, torch, B, n_ff, True)
+        line["e2e_two_sessions"] = {
+            "workload": "two C2 sessions (seeds s, s+1) taking turns on a 24 GiB HBM pool (1.5 sessions) over a 24 GiB "
+                        "pinned host tier; no artificial pressure: every call reloads part of its own prefix and "
+                        "pushes part of the other session out",
+            "unit": "GB/s (blocks offloaded + reloaded)", "offload_then_reload": seq, "one_exchange_per_call": dup,
         }
     if not args.skip_stress and world == 1:
         line["metadata_stress"] = metadata_stress(torch, B, hbm_peak)

@@ -295,13 +295,16 @@ int32_t kvt_reload(kvt_engine *e, const uint32_t *host_slots, uint32_t n, uint32
 int32_t kvt_move(kvt_engine *e, uint32_t src_tier, uint32_t dst_tier, const uint32_t *slots, uint32_t n,
                  uint32_t *n_done, uint32_t *n_dropped, void *stream);
 
-/* Reload and offload in one call, for the common step "bring my prefix back and push other blocks out": the
- * listed host slots move to the HBM slots that are free when the call begins (as kvt_reload does), the listed
- * HBM slots are dropped / handed over / moved to the host slots that are free when the call begins (as
- * kvt_offload does). Because neither list depends on slots the other one frees, the two payload streams are
- * issued by ONE mover launch and cross the host link in both directions at the same time (the link is full
- * duplex). Both lists are validated before anything changes (same codes as the single calls). KVT_E_NOSPACE if
- * either direction ran out of destination slots; the three counts tell how far each got. Synchronises. */
+/* Offload and reload in one call, for the common step "push other blocks out and bring my prefix back". Both
+ * lists are validated against the state the call finds (same codes as the single calls; nothing changes on an
+ * error). After that the result is by definition that of kvt_offload(hbm_slots_out) followed by
+ * kvt_reload(host_slots_in): the victims are dropped / handed over / moved to the host slots that are free when the
+ * call begins; the listed host blocks then take the lowest free HBM slots, those the victims just left included,
+ * so the call also works on a full pool. What the single call adds: ONE mover launch carries both payload streams,
+ * so they cross the host link in both directions at the same time (the link is full duplex); where a reload lands
+ * in a slot a victim leaves, the same warp copies the victim's tile out before it writes the new tile in.
+ * KVT_E_NOSPACE if either direction ran out of destination slots; the three counts tell how far each got.
+ * Synchronises. */
 int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_out, const uint32_t *host_slots_in,
                      uint32_t n_in, uint32_t *n_out_done, uint32_t *n_dropped, uint32_t *n_in_done, void *stream);
 
@@ -393,7 +396,7 @@ int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant);
 
 /* Upper bound on the thread blocks a mover kernel launches (offload / reload / exchange / move / compact /
  * copy_blocks); 0 = automatic (default): 8 blocks of 256 threads per SM for moves inside device memory; for a move
- * to or from a pool that lies in host memory 4 blocks of 1024 threads (32 for kvt_exchange, which drives both
+ * to or from a pool that lies in host memory 4 blocks of 1024 threads (8 for kvt_exchange, which drives both
  * directions). A move that crosses the host link is bound by the link, 128 warps keep it full, and packing them
  * into a few large blocks leaves all other SMs to kernels running on other streams at the same time. */
 int32_t kvt_set_mover_ctas(kvt_engine *e, uint32_t max_ctas);

@@ -762,8 +762,11 @@ int32_t kvto_move(Engine *e, uint32_t st, uint32_t dt, const uint32_t *slots, ui
   return OK;
 }
 
-// Reload and offload in one call, both with destinations taken from the slots that are free when the call
-// begins (the two payload streams are independent, so a device can run them concurrently over a duplex link).
+// Offload and reload in one call. Both lists are checked against the state the call finds; after that the result is
+// by definition that of kvt_offload(out) followed by kvt_reload(in): victims leave first (to the host slots that
+// are free when the call begins), the listed host blocks then take the lowest free HBM slots, those the victims
+// just left included. (What a device gains from the single call is that the two payload streams can run at the
+// same time over a duplex link.)
 int32_t kvto_exchange(Engine *e, const uint32_t *out_slots, uint32_t n_out, const uint32_t *in_slots, uint32_t n_in,
                       uint32_t *n_out_done, uint32_t *n_dropped, uint32_t *n_in_done) {
   if (!e || (!out_slots && n_out) || (!in_slots && n_in) || !n_out_done || !n_dropped || !n_in_done) return E_INVAL;
@@ -772,58 +775,9 @@ int32_t kvto_exchange(Engine *e, const uint32_t *out_slots, uint32_t n_out, cons
   int32_t vb = validate_slots(e, TIER_HBM, out_slots, n_out, false);
   for (int32_t code : {E_RANGE, E_INVAL, E_STATE})
     if (va == code || vb == code) return code;
-  std::vector<uint8_t> rank[N_TIERS];
-  classify(*e, rank);
-  const bool knows_dead = !(e->cfg.policy_flags & POLICY_NO_LIFECYCLE);
-  std::vector<uint32_t> hbm_dests(e->free_slots[TIER_HBM].begin(), e->free_slots[TIER_HBM].end());
-  std::vector<uint32_t> host_dests(e->free_slots[TIER_HOST].begin(), e->free_slots[TIER_HOST].end());
-  bool full = false;
-  for (uint32_t i = 0; i < n_in; ++i) {               // incoming blocks
-    if (i == hbm_dests.size()) { full = true; break; }
-    uint32_t h = in_slots[i], d = hbm_dests[i];
-    if (e->cfg.policy_flags & POLICY_INCLUSIVE) {
-      copy_payload(*e, TIER_HOST, h, TIER_HBM, d);
-      Entry x = e->ent[TIER_HOST][h];
-      x.link = h;
-      e->ent[TIER_HBM][d] = x;
-      e->free_slots[TIER_HBM].erase(d);
-      e->ent[TIER_HOST][h].shadow = true;
-      e->ent[TIER_HOST][h].link = d;
-      e->ent[TIER_HOST][h].inflight = 0;
-      e->where[x.key] = {TIER_HBM, d};
-    } else {
-      move_entry(e, TIER_HOST, h, TIER_HBM, d);
-    }
-    e->st.reloaded++;
-    e->st.bytes_h2d += e->block_bytes;
-    (*n_in_done)++;
-  }
-  size_t next_dest = 0;
-  for (uint32_t i = 0; i < n_out; ++i) {              // outgoing blocks
-    uint32_t s = out_slots[i];
-    if (knows_dead && rank[0][s] == 0) {
-      free_slot(*e, TIER_HBM, s);
-      e->st.dropped++;
-      (*n_dropped)++;
-    } else if (e->ent[TIER_HBM][s].link >= 0) {
-      Entry x = e->ent[TIER_HBM][s];
-      Entry &h = e->ent[TIER_HOST][x.link];
-      h.shadow = false; h.link = -1; h.stamp = x.stamp; h.depth = x.depth; h.floor = x.floor; h.inflight = x.inflight;
-      e->where[x.key] = {TIER_HOST, (uint32_t)x.link};
-      e->ent[TIER_HBM][s] = Entry();
-      e->free_slots[TIER_HBM].insert(s);
-      e->st.offloaded++;
-      e->st.offloaded_clean++;
-    } else {
-      if (next_dest == host_dests.size()) { full = true; break; }
-      uint32_t d = host_dests[next_dest++];
-      move_entry(e, TIER_HBM, s, TIER_HOST, d);
-      e->st.offloaded++;
-      e->st.bytes_d2h += e->block_bytes;
-    }
-    (*n_out_done)++;
-  }
-  return full ? E_NOSPACE : OK;
+  int32_t r_out = kvto_offload(e, out_slots, n_out, n_out_done, n_dropped);
+  int32_t r_in = kvto_reload(e, in_slots, n_in, n_in_done);
+  return (r_out == E_NOSPACE || r_in == E_NOSPACE) ? E_NOSPACE : OK;
 }
 
 int32_t kvto_release(Engine *e, uint32_t tier, const uint32_t *slots, uint32_t n) {

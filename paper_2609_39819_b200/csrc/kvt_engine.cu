@@ -154,9 +154,10 @@ struct kvt_engine {
   bool tier_in_host_mem[3] = {false, false, false};   // pool is host memory: moves to / from it are bound by the host link
   // Grid of a mover launch. Inside the device: 8 CTAs of 256 threads per SM. A move that crosses the host link
   // is bound by the link: 128 warps keep it full (measured), and a GEMM on another stream loses every SM a mover
-  // CTA sits on, so those warps are packed into 4 CTAs of 1024 threads (32 for both directions at once).
+  // CTA sits on, so those warps are packed into 4 CTAs of 1024 threads (8 for an exchange, which
+  // drives both directions).
   u32 mover_grid(u64 want, u32 link_dirs = 0) const {
-    u64 cap = mover_max_ctas ? mover_max_ctas : link_dirs == 1 ? 4 : link_dirs == 2 ? 32 : (u64)sm_count * 8;
+    u64 cap = mover_max_ctas ? mover_max_ctas : link_dirs == 1 ? 4 : link_dirs == 2 ? 8 : (u64)sm_count * 8;
     return (u32)std::max<u64>(1, std::min(want, cap));
   }
   u32 link_dirs(u32 st, u32 dt) const { return (tier_in_host_mem[st] || tier_in_host_mem[dt]) ? 1u : 0u; }
@@ -1204,7 +1205,7 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
   a.w_cut = ST_CUT; a.w_nlive = ST_NLIVE; a.w_ndrop = ST_NDROP; a.w_nclean = ST_NCLEAN; a.w_nshdrop = ST_NSHDROP;
   u32 g = cdiv(n, 256);
   KL(k_list_validate, g, 256, s, a);
-  r = compact_indices(e, s, PredLive{a.live}, EmitLive{a.lidx, a.n_free, e->d_status + ST_CUT}, n, ST_TOTAL);
+  r = compact_indices(e, s, PredLive{a.live}, EmitLive{a.lidx, a.n_free, e->d_status + ST_CUT, nullptr}, n, ST_TOTAL);
   if (r) return r;
   if (!m.drop_all) {
     r = compact_indices(e, s, PredFree{e->ent.key, a.dst_e0}, EmitFree{e->dp<u32>(e->L.freelist), (u32)e->L.LB},
@@ -1312,12 +1313,14 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
   if (r) return r;
   CU(cudaMemcpyAsync(e->d_status + ST_CUT, &n_in, 4, cudaMemcpyHostToDevice, s));
   CU(cudaMemcpyAsync(e->d_status + ST_B_CUT, &n_out, 4, cudaMemcpyHostToDevice, s));
-  // list A: incoming (host -> HBM); list B: outgoing (HBM -> host). Both plans use the free slots of call begin.
+  // list A: incoming (host -> HBM); list B: outgoing (HBM -> host). Both are validated against the state the call
+  // finds; then the victims are planned and applied first, the reloads after them, so that the incoming blocks
+  // take the lowest free HBM slots including those the victims leave: the result of kvt_offload + kvt_reload.
   ListArgs a{}, b{};
   a.tab = b.tab = e->tab; a.ent = b.ent = e->ent; a.status = b.status = e->d_status;
   a.ids = d_in; a.n = n_in; a.e0 = e->tier_e0(KVT_TIER_HOST); a.n_slots = e->cfg.n_host_blocks; a.dst_e0 = 0;
   a.live = e->dp<u32>(e->L.s1); a.lidx = e->dp<u32>(e->L.s2); a.freelist = e->dp<u32>(e->L.freelist);
-  a.n_free = e->cfg.n_hbm_blocks - e->occ[0];
+  a.n_free = e->cfg.n_hbm_blocks;      // upper bound; the count after the victims have left is the device word ST_FREE
   a.pair_src = e->dp<u32>(e->L.pair_src); a.pair_dst = e->dp<u32>(e->L.pair_dst);
   a.allow_inflight = 1; a.reject_shadow = 1; a.keep_copy = (e->cfg.policy_flags & KVT_POLICY_INCLUSIVE) ? 1 : 0;
   a.w_cut = ST_CUT; a.w_nlive = ST_NLIVE; a.w_ndrop = ST_NDROP; a.w_nclean = ST_NCLEAN; a.w_nshdrop = ST_NSHDROP;
@@ -1330,22 +1333,30 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
   const u32 ga = cdiv(n_in, 256), gb = cdiv(n_out, 256);
   if (n_in) KL(k_list_validate, ga, 256, s, a);
   if (n_out) KL(k_list_validate, gb, 256, s, b);
-  if (n_in) { r = compact_indices(e, s, PredLive{a.live}, EmitLive{a.lidx, a.n_free, e->d_status + ST_CUT}, n_in, ST_TOTAL); if (r) return r; }
-  if (n_out) { r = compact_indices(e, s, PredLive{b.live}, EmitLive{b.lidx, b.n_free, e->d_status + ST_B_CUT}, n_out, ST_B_TOTAL); if (r) return r; }
-  r = compact_indices(e, s, PredFree{e->ent.key, 0}, EmitFree{e->dp<u32>(e->L.freelist), (u32)e->L.LB}, e->cfg.n_hbm_blocks, ST_FREE);
-  if (r) return r;
-  if (e->cfg.n_host_blocks) {
-    r = compact_indices(e, s, PredFree{e->ent.key, b.dst_e0}, EmitFree{e->dp<u32>(e->L.freelist2), (u32)e->L.LB}, e->cfg.n_host_blocks, ST_B_FREE);
+  if (n_out) {   // victims: plan against the host slots that are free now, apply
+    r = compact_indices(e, s, PredLive{b.live}, EmitLive{b.lidx, b.n_free, e->d_status + ST_B_CUT, nullptr}, n_out, ST_B_TOTAL);
     if (r) return r;
+    if (e->cfg.n_host_blocks) {
+      r = compact_indices(e, s, PredFree{e->ent.key, b.dst_e0}, EmitFree{e->dp<u32>(e->L.freelist2), (u32)e->L.LB}, e->cfg.n_host_blocks, ST_B_FREE);
+      if (r) return r;
+    }
+    KL(k_list_apply, gb, 256, s, b);
+    KL(k_list_unmark, gb, 256, s, b);
   }
-  if (n_in) { KL(k_list_apply, ga, 256, s, a); KL(k_list_unmark, ga, 256, s, a); }
-  if (n_out) { KL(k_list_apply, gb, 256, s, b); KL(k_list_unmark, gb, 256, s, b); }
+  if (n_in) {    // reloads: the free HBM slots now include what the victims left
+    r = compact_indices(e, s, PredFree{e->ent.key, 0}, EmitFree{e->dp<u32>(e->L.freelist), (u32)e->L.LB}, e->cfg.n_hbm_blocks, ST_FREE);
+    if (r) return r;
+    r = compact_indices(e, s, PredLive{a.live}, EmitLive{a.lidx, a.n_free, e->d_status + ST_CUT, e->d_status + ST_FREE}, n_in, ST_TOTAL);
+    if (r) return r;
+    KL(k_list_apply, ga, 256, s, a);
+    KL(k_list_unmark, ga, 256, s, a);
+  }
   LAUNCH_CHECK();
   // one mover launch for both directions
   if (!e->metadata_only) {
     MoveArgs ma{}, mb{};
     ma.src = pool_view(e, KVT_TIER_HOST); ma.dst = pool_view(e, KVT_TIER_HBM); ma.src_ids = a.pair_src; ma.dst_ids = a.pair_dst;
-    ma.n_pairs = std::min(n_in, a.n_free); ma.n_pairs_dev = e->d_status + ST_NLIVE;
+    ma.n_pairs = n_in; ma.n_pairs_dev = e->d_status + ST_NLIVE;
     mb.src = pool_view(e, KVT_TIER_HBM); mb.dst = pool_view(e, KVT_TIER_HOST); mb.src_ids = b.pair_src; mb.dst_ids = b.pair_dst;
     mb.n_pairs = std::min(n_out, b.n_free); mb.n_pairs_dev = e->d_status + ST_B_NLIVE;
     ma.n_chunks = mb.n_chunks = (u32)e->n_chunks; ma.chunk_bytes = mb.chunk_bytes = (u32)e->chunk_bytes; ma.status = mb.status = e->d_status;
@@ -1354,21 +1365,26 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
       const bool timed = e->profiling;
       if (timed) CU(cudaEventRecord(e->ev_m0, s));
       if (e->chunk_bytes % 4096 == 0) {
+        // which reload lands in a slot a victim leaves (scratch of the selection, idle during this call)
+        u32 *vic_of = e->dp<u32>(e->L.out_slots), *dep = e->dp<u32>(e->L.valA), *taken = e->dp<u32>(e->L.valB);
+        CU(cudaMemsetAsync(vic_of, 0xFF, (u64)e->cfg.n_hbm_blocks * 4, s));
+        if (mb.n_pairs) KL(k_xchg_mark, cdiv(mb.n_pairs, 256), 256, s, mb.src_ids, mb.n_pairs_dev, mb.n_pairs, vic_of, taken);
+        if (ma.n_pairs) KL(k_xchg_link, cdiv(ma.n_pairs, 256), 256, s, ma.dst_ids, ma.n_pairs_dev, ma.n_pairs, vic_of, dep, taken);
         u32 tpc = (u32)(e->chunk_bytes / 4096);
         const u32 xl = e->link_dirs(KVT_TIER_HBM, KVT_TIER_HOST) * 2;
         if (xl) {
-          u32 grid = std::max(2u, e->mover_grid((items * tpc + 31) / 32, xl));
-          KL((k_move_tiles_dual<8, 1024>), grid, 1024, s, ma, mb, tpc, 2u);
+          u32 grid = e->mover_grid((items + 31) / 32, xl);
+          KL((k_move_exchange<8, 1024>), grid, 1024, s, ma, mb, tpc, dep, taken, e->d_status + ST_QA);
         } else {
-          u32 grid = e->mover_grid((items * tpc + 7) / 8, xl);
-          KL(k_move_tiles_dual<8>, grid, 256, s, ma, mb, tpc, 2u);   // CTAs alternate between the two directions
+          u32 grid = e->mover_grid((items + 7) / 8, xl);
+          KL((k_move_exchange<8, 256>), grid, 256, s, ma, mb, tpc, dep, taken, e->d_status + ST_QA);
         }
-      } else {   // chunk sizes the tile kernel cannot split: one direction after the other
+      } else {   // chunk sizes the tile kernel cannot split: victims out, then reloads in (stream order)
         const u32 xl = e->link_dirs(KVT_TIER_HBM, KVT_TIER_HOST);
-        u32 g1 = ma.n_pairs ? e->mover_grid((u64)ma.n_pairs * e->n_chunks, xl) : 0;
-        u32 g2 = mb.n_pairs ? e->mover_grid((u64)mb.n_pairs * e->n_chunks, xl) : 0;
-        if (g1) KL(k_move_blocks<4>, g1, 256, s, ma);
-        if (g2) KL(k_move_blocks<4>, g2, 256, s, mb);
+        u32 g1 = mb.n_pairs ? e->mover_grid((u64)mb.n_pairs * e->n_chunks, xl) * (xl && !e->mover_max_ctas ? 4 : 1) : 0;
+        u32 g2 = ma.n_pairs ? e->mover_grid((u64)ma.n_pairs * e->n_chunks, xl) * (xl && !e->mover_max_ctas ? 4 : 1) : 0;
+        if (g1) KL(k_move_blocks<4>, g1, 256, s, mb);
+        if (g2) KL(k_move_blocks<4>, g2, 256, s, ma);
       }
       if (timed) { CU(cudaEventRecord(e->ev_m1, s)); e->mover_timed = true; }
       LAUNCH_CHECK();

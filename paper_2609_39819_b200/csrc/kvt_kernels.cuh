@@ -32,6 +32,7 @@ enum : int {
   ST_ERR = 0, ST_TOTAL, ST_CUT, ST_NLIVE, ST_NDROP, ST_NEW, ST_INSERTED, ST_ADOPTED, ST_TOMBS,
   ST_RANK0, ST_RANK1, ST_RANK2, ST_RANK3, ST_M, ST_NMOVED, ST_FREE, ST_AUX, ST_SHADOW, ST_NCLEAN, ST_NSHDROP,
   ST_B_CUT, ST_B_NLIVE, ST_B_NDROP, ST_B_NCLEAN, ST_B_NSHDROP, ST_B_TOTAL, ST_B_FREE,   // second list of an exchange
+  ST_QA, ST_QB,                                                                          // work queues of its mover
   ST_WORDS = 32
 };
 
@@ -1054,7 +1055,11 @@ struct PredLive { const u32 *live; __device__ bool operator()(u32 i) const { ret
 // item with rank r needs the r-th free destination slot; the first one that does not fit cuts the list
 struct EmitLive {
   u32 *lidx; u32 n_free; u32 *cut;
-  __device__ void operator()(u32 i, u32 r) const { lidx[i] = r; if (r >= n_free) atomicMin(cut, i); }
+  const u32 *n_free_dev;   // optional: the free count is a device word (computed earlier in the same call)
+  __device__ void operator()(u32 i, u32 r) const {
+    lidx[i] = r;
+    if (r >= (n_free_dev ? min(n_free, *n_free_dev) : n_free)) atomicMin(cut, i);
+  }
 };
 struct PredFree { const u64 *key; u32 e0; __device__ bool operator()(u32 i) const { return key[e0 + i] == 0; } };
 struct EmitFree { u32 *list; u32 cap; __device__ void operator()(u32 i, u32 r) const { if (r < cap) list[r] = i; } };
@@ -1238,52 +1243,98 @@ __global__ void __launch_bounds__(THREADS) k_move_tiles(MoveArgs a, u32 tiles_pe
   }
 }
 
-// Two independent pair lists in one launch (kvt_exchange): even CTAs work on list a, odd CTAs on list b (or all
-// CTAs on the one that has work), so that loads from and stores to the host tier are in flight at the same time
-// (the link is full duplex) and neither direction waits for the other's latency.
-template <int UNROLL, int THREADS = 256>
-__global__ void __launch_bounds__(THREADS) k_move_tiles_dual(MoveArgs a, MoveArgs b, u32 tiles_per_chunk, u32 b_every) {
-  constexpr u32 WPC = THREADS / 32;
+// ---- kvt_exchange: victims out and reloads in with one launch -----------------------------------------------------
+// A reload may land in the HBM slot a victim of the same call leaves. vic_of[slot] = index of the victim pair that
+// reads that slot; dep[r] = the victim pair reload r has to wait for (ENT_NONE: none); taken[v] = 1: victim v is
+// copied out by the warp that copies its successor in.
+__global__ void k_xchg_mark(const u32 *vic_src, const u32 *n_vic_dev, u32 n_vic_max, u32 *vic_of, u32 *taken) {
+  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= min(n_vic_max, *n_vic_dev)) return;
+  vic_of[vic_src[i]] = i;
+  taken[i] = 0;
+}
+__global__ void k_xchg_link(const u32 *in_dst, const u32 *n_in_dev, u32 n_in_max, const u32 *vic_of, u32 *dep, u32 *taken) {
+  u32 r = blockIdx.x * blockDim.x + threadIdx.x;
+  if (r >= min(n_in_max, *n_in_dev)) return;
+  u32 v = vic_of[in_dst[r]];
+  dep[r] = v;
+  if (v != ENT_NONE) taken[v] = 1;
+}
+
+// Mover of an exchange. Work unit = one chunk of one pair; two queues (reloads a: host -> HBM, victims b: HBM ->
+// host), every warp takes units from both in turn, so both directions of the link are busy whatever the mix. A
+// reload unit whose destination slot is being vacated copies that victim's tile out first and then its own tile
+// in: the same lane reads and writes the same 16 bytes, so program order keeps the two apart. Victims handled that
+// way are skipped in the victim queue.
+template <int UNROLL, int THREADS>
+__global__ void __launch_bounds__(THREADS) k_move_exchange(MoveArgs a, MoveArgs b, u32 tiles_per_chunk, const u32 *dep,
+                                                           const u32 *taken, u32 *queues) {
   u32 na = a.n_pairs, nb = b.n_pairs;
   if (a.n_pairs_dev) na = min(na, *a.n_pairs_dev);
   if (b.n_pairs_dev) nb = min(nb, *b.n_pairs_dev);
   const u32 lane = threadIdx.x & 31;
-  const u64 per_pair = (u64)a.n_chunks * tiles_per_chunk;
-  // CTA roles: with work on both sides and at least two CTAs the grid is split in two halves; otherwise every CTA
-  // serves list a and then list b
-  const bool split = na && nb && gridDim.x >= b_every;
-  for (int pass = 0; pass < 2; ++pass) {
-    bool from_b;
-    u32 my_cta, n_cta;
-    if (split) {
-      if (pass) break;
-      // every b_every-th CTA serves list b, the others list a
-      const u32 q = blockIdx.x / b_every, rmd = blockIdx.x % b_every;
-      from_b = rmd == b_every - 1;
-      const u32 n_b = gridDim.x / b_every, n_a = gridDim.x - n_b;
-      my_cta = from_b ? q : q * (b_every - 1) + rmd;
-      n_cta = from_b ? n_b : n_a;
-    } else {
-      from_b = pass; my_cta = blockIdx.x; n_cta = gridDim.x;
+  const u32 units_a = na * a.n_chunks, units_b = nb * b.n_chunks;
+  bool more_a = units_a != 0, more_b = units_b != 0;
+  while (more_a || more_b) {
+    if (more_a) {
+      u32 u = 0;
+      if (lane == 0) u = atomicAdd(&queues[0], 1u);
+      u = __shfl_sync(0xFFFFFFFFu, u, 0);
+      if (u >= units_a) more_a = false;
+      else {
+        const u32 r = u / a.n_chunks, chunk = u - r * a.n_chunks;
+        const u32 v = dep[r];
+        const u32 s = a.src_ids[r], d = a.dst_ids[r];
+        u32 vs = 0, vd = 0;
+        bool ok = s < a.src.n_slots && d < a.dst.n_slots;
+        if (v != ENT_NONE) { vs = b.src_ids[v]; vd = b.dst_ids[v]; ok = ok && vs < b.src.n_slots && vd < b.dst.n_slots; }
+        if (!ok) { if (lane == 0) set_err(a.status, DERR_RANGE); }
+        else {
+          const uint4 *sp = reinterpret_cast<const uint4 *>(a.src.base + s * a.src.slot_stride + chunk * a.src.chunk_stride) + lane;
+          uint4 *dp = reinterpret_cast<uint4 *>(a.dst.base + d * a.dst.slot_stride + chunk * a.dst.chunk_stride) + lane;
+          const uint4 *vsp = reinterpret_cast<const uint4 *>(b.src.base + vs * b.src.slot_stride + chunk * b.src.chunk_stride) + lane;
+          uint4 *vdp = reinterpret_cast<uint4 *>(b.dst.base + vd * b.dst.slot_stride + chunk * b.dst.chunk_stride) + lane;
+          for (u32 t = 0; t < tiles_per_chunk; ++t) {
+            const u64 o = (u64)t * 32 * UNROLL;
+            uint4 x[UNROLL];
+            if (v != ENT_NONE) {        // the victim's tile leaves before the new one overwrites it
+#pragma unroll
+              for (int q = 0; q < UNROLL; ++q) x[q] = __ldcs(vsp + o + q * 32);
+#pragma unroll
+              for (int q = 0; q < UNROLL; ++q) __stcs(vdp + o + q * 32, x[q]);
+            }
+#pragma unroll
+            for (int q = 0; q < UNROLL; ++q) x[q] = __ldcs(sp + o + q * 32);
+#pragma unroll
+            for (int q = 0; q < UNROLL; ++q) __stcs(dp + o + q * 32, x[q]);
+          }
+        }
+      }
     }
-    const MoveArgs &m = from_b ? b : a;
-    const u64 n_items = (u64)(from_b ? nb : na) * per_pair;
-    const u64 n_warps = (u64)n_cta * WPC;
-    for (u64 k = (u64)my_cta * WPC + (threadIdx.x >> 5); k < n_items; k += n_warps) {
-      u32 pair = (u32)(k / per_pair);
-      u32 rem = (u32)(k - (u64)pair * per_pair);
-      u32 chunk = rem / tiles_per_chunk, tile = rem - chunk * tiles_per_chunk;
-      u32 s = m.src_ids[pair], d = m.dst_ids[pair];
-      if (s >= m.src.n_slots || d >= m.dst.n_slots) { if (lane == 0) set_err(m.status, DERR_RANGE); continue; }
-      const uint4 *sp = reinterpret_cast<const uint4 *>(m.src.base + s * m.src.slot_stride + chunk * m.src.chunk_stride) +
-                        (u64)tile * 32 * UNROLL + lane;
-      uint4 *dp = reinterpret_cast<uint4 *>(m.dst.base + d * m.dst.slot_stride + chunk * m.dst.chunk_stride) +
-                  (u64)tile * 32 * UNROLL + lane;
-      uint4 r[UNROLL];
+    if (more_b) {
+      u32 u = 0;
+      if (lane == 0) u = atomicAdd(&queues[1], 1u);
+      u = __shfl_sync(0xFFFFFFFFu, u, 0);
+      if (u >= units_b) more_b = false;
+      else {
+        const u32 v = u / b.n_chunks, chunk = u - v * b.n_chunks;
+        if (!taken[v]) {
+          const u32 s = b.src_ids[v], d = b.dst_ids[v];
+          if (s >= b.src.n_slots || d >= b.dst.n_slots) { if (lane == 0) set_err(b.status, DERR_RANGE); }
+          else {
+            const uint4 *sp = reinterpret_cast<const uint4 *>(b.src.base + s * b.src.slot_stride + chunk * b.src.chunk_stride) + lane;
+            uint4 *dp = reinterpret_cast<uint4 *>(b.dst.base + d * b.dst.slot_stride + chunk * b.dst.chunk_stride) + lane;
+            for (u32 t = 0; t < tiles_per_chunk; ++t) {
+              const u64 o = (u64)t * 32 * UNROLL;
+              uint4 x[UNROLL];
 #pragma unroll
-      for (int u = 0; u < UNROLL; ++u) r[u] = __ldcs(sp + u * 32);
+              for (int q = 0; q < UNROLL; ++q) x[q] = __ldcs(sp + o + q * 32);
 #pragma unroll
-      for (int u = 0; u < UNROLL; ++u) __stcs(dp + u * 32, r[u]);
+              for (int q = 0; q < UNROLL; ++q) __stcs(dp + o + q * 32, x[q]);
+            }
+          }
+        }
+      }
     }
   }
 }

@@ -327,11 +327,12 @@ def exchange_both_ways(make):
             for kk, s_ in zip(k, sl):
                 eng.write_block(HBM, int(s_), _payload(kk, eng.block_bytes))
         assert eng.offload([7, 6]) == (0, 2, 0)           # context 1's blocks 3, 2 -> host slots 0, 1
-        # bring them back while pushing context 0's tail out: the incoming blocks take the HBM slots that are free
-        # now (6, 7), the outgoing ones the host slots that are free now (2, 3; 0 and 1 are still occupied)
+        # bring them back while pushing context 0's tail out, as offload then reload would: the outgoing blocks take
+        # the host slots that are free now (2, 3; 0 and 1 are still occupied), the incoming ones the lowest free HBM
+        # slots, which are the two the victims just left (2, 3), not 6 and 7
         assert eng.exchange([3, 2], [1, 0]) == (0, 2, 0, 2)
         _k, t1, s1 = eng.get_block_map(1)
-        assert list(t1) == [HBM] * 4 and list(s1) == [4, 5, 6, 7]
+        assert list(t1) == [HBM] * 4 and list(s1) == [4, 5, 2, 3]
         _k, t0, s0 = eng.get_block_map(0)
         assert list(t0) == [HBM, HBM, HOST, HOST] and list(s0) == [0, 1, 3, 2]
         st = eng.get_stats()
@@ -340,11 +341,11 @@ def exchange_both_ways(make):
             _k, t, sl = eng.get_block_map(c)
             for b in range(4):
                 assert np.array_equal(eng.read_block(int(t[b]), int(sl[b])), _payload(keys[c][b], eng.block_bytes))
-        # second exchange: context 0's tail comes back into HBM slots 2, 3 while its block 0 goes out; the host
-        # slots 0, 1 are free again without inclusive tiers, and still hold clean copies with them
+        # second exchange: context 0's block 0 goes out and its tail comes back, into the slot block 0 left and
+        # into slot 6; the host slots 0, 1 are free again without inclusive tiers, and still hold clean copies with them
         assert eng.exchange([0], [3, 2]) == (0, 1, 0, 2)
         _k, t0, s0 = eng.get_block_map(0)
-        assert list(t0) == [HOST, HBM, HBM, HBM] and list(s0) == [0 if flags == 0 else 4, 1, 2, 3]
+        assert list(t0) == [HOST, HBM, HBM, HBM] and list(s0) == [0 if flags == 0 else 4, 1, 0, 6]
         # validation covers both lists before anything moves
         watch = ("occ_hbm", "occ_host", "offloaded", "reloaded", "dropped", "bytes_d2h", "bytes_h2d")
         before = {k: eng.get_stats()[k] for k in watch}
