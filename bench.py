@@ -15,6 +15,9 @@ Two measurements of the same steps:
   e2e   : the real thing through the same C-ABI calls: tokens come from pinned host buffers, the
           second tier is pinned host memory, every offload / reload crosses the host link inside the
           timed region.
+Side measurements in the same line: `e2e_inclusive_tiers` (the e2e steps with clean host copies kept),
+`e2e_two_sessions` (two such sessions taking turns on an HBM pool that holds one and a half of them: no artificial
+pressure, offload + reload per call against one kvt_exchange per call), `metadata_stress` (C4 shape).
 `--impl reference` times the CPU oracle (plain single-threaded C++) on the same steps.
 Prints ONE JSON line.
 """
