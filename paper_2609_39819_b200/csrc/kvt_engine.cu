@@ -1364,7 +1364,8 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
     if (items) {
       const bool timed = e->profiling;
       if (timed) CU(cudaEventRecord(e->ev_m0, s));
-      if (e->chunk_bytes % 4096 == 0) {
+      const bool queues_fit = (u64)std::max(ma.n_pairs, mb.n_pairs) * e->n_chunks < (1ull << 32);   // 32-bit unit counters
+      if (e->chunk_bytes % 4096 == 0 && queues_fit) {
         // which reload lands in a slot a victim leaves (scratch of the selection, idle during this call)
         u32 *vic_of = e->dp<u32>(e->L.out_slots), *dep = e->dp<u32>(e->L.valA), *taken = e->dp<u32>(e->L.valB);
         CU(cudaMemsetAsync(vic_of, 0xFF, (u64)e->cfg.n_hbm_blocks * 4, s));
