@@ -369,6 +369,32 @@ def exchange_both_ways(make):
     assert eng.exchange([], [0, 1]) == (E_NOSPACE, 0, 0, 1)
     assert list(eng.get_block_map(0)[2]) == [0, 1, 1, 3]  # block 3 came back to HBM slot 3, block 2 still at host slot 1
     assert eng.exchange([], []) == (0, 0, 0, 0)
+    # a full pool: the incoming blocks can only go where the outgoing ones were; every byte of both survives
+    eng = make(n_hbm_blocks=4, n_host_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(23)
+    keys = {}
+    for c in (0, 1):
+        eng.spawn(c)
+        eng.append(c, toks(rng, 32))
+        call(eng, c)                                      # context 0 at HBM slots 0, 1; context 1 at slots 2, 3
+        keys[c] = eng.get_block_map(c)[0]
+        for b in range(2):
+            eng.write_block(HBM, 2 * c + b, _payload(keys[c][b], eng.block_bytes))
+    assert eng.offload([3, 2]) == (0, 2, 0)               # context 1 -> host slots 0 (block 1), 1 (block 0)
+    eng.spawn(2)
+    eng.append(2, toks(rng, 32))
+    call(eng, 2)                                          # context 2 fills HBM slots 2, 3: the pool is full
+    keys[2] = eng.get_block_map(2)[0]
+    for b in range(2):
+        eng.write_block(HBM, 2 + b, _payload(keys[2][b], eng.block_bytes))
+    assert eng.get_stats()["occ_hbm"] == 4
+    assert eng.exchange([1, 0], [1, 0]) == (0, 2, 0, 2)   # context 0 out (host slots 2, 3), context 1 into slots 0, 1
+    assert [list(x) for x in eng.get_block_map(1)[1:]] == [[HBM, HBM], [0, 1]]
+    assert [list(x) for x in eng.get_block_map(0)[1:]] == [[HOST, HOST], [3, 2]]
+    for c in (0, 1, 2):
+        _k, t, sl = eng.get_block_map(c)
+        for b in range(2):
+            assert np.array_equal(eng.read_block(int(t[b]), int(sl[b])), _payload(keys[c][b], eng.block_bytes)), (c, b)
 
 
 # ---- hand-worked lifecycle example (8-block pool) --------------------------------------------------
