@@ -796,7 +796,9 @@ def main():
             "reloaded_per_step": ist["reloaded"] / K, "bytes_over_link_per_step": (ist["bytes_d2h"] + ist["bytes_h2d"]) / K,
             "verified_blocks": i["verified"],
         }
-    if e and not args.skip_two_tenants and world == 1 and mem_available_bytes() > 64 * GiB:
+    if hasattr(torch._C, "_host_emptyCache"):
+        torch._C._host_emptyCache()      # give the pinned pools of the arms above back to the OS
+    if e and not args.skip_two_tenants and world == 1 and mem_available_bytes() > 32 * GiB:
         seq = two_tenant_arm(args, torch, B, n_ff, False)
         dup = two_tenant_arm(args, torch, B, n_ff, True)
         line["e2e_two_sessions"] = {
