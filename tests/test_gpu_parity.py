@@ -509,6 +509,19 @@ def test_mover_with_second_tier_in_hbm(B, oracle):
     del gpu, cpu
 
 
+@pytest.mark.parametrize("ctas", [1, 3, 64])
+@pytest.mark.parametrize("on_device", [False, True], ids=["pinned-host-tier", "second-tier-in-hbm"])
+def test_mover_grid_limit_does_not_change_results(B, ctas, on_device):
+    """kvt_set_mover_ctas bounds the mover's grid (one thread block has to walk every tile); offload, reload and the
+    two-directional exchange still move every byte, over the host link (1024-thread blocks) and inside the device."""
+    def make(**k):
+        eng = B.Engine(max_tokens=1 << 16, max_messages=256, host_pool_on_device=on_device, **k)
+        eng.set_mover_ctas(ctas)
+        return eng
+    S.offload_reload_round_trip(make, geos=[W.GEO_128K.kwargs()], layouts=(0,))
+    S.exchange_both_ways(make)
+
+
 # ---- table maintenance and limits -------------------------------------------------------------------------
 def test_tombstones_trigger_rebuild_and_lookups_survive(B, oracle):
     """Insert / drop cycles leave tombstones; the table is rebuilt when they pile up; every resident key is still
