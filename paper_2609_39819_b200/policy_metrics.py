@@ -95,11 +95,16 @@ def main():
     ap.add_argument("--hbm", type=int, default=1024)
     ap.add_argument("--host", type=int, default=1024)
     ap.add_argument("--seed", type=int, default=1)
+    ap.add_argument("--timed", action="store_true", help="order the calls by an event clock with tool waits (trace_c3_timed)")
+    ap.add_argument("--long-wait-p", type=float, default=0.0, help="with --timed: share of tool waits of 30-120 s")
     ap.add_argument("--remote", type=int, default=0, help="adds a row for the paper's policy with a third tier of this many blocks")
     a = ap.parse_args()
     from . import binding as B
-    trace, n_ctx = W.trace_c3(a.seed, n_sessions=a.sessions, scale=a.scale)
-    print(f"C3-shaped trace: {a.sessions} sessions, scale {a.scale}, HBM {a.hbm} blocks, host tier {a.host} blocks, "
+    if a.timed:
+        trace, n_ctx = W.trace_c3_timed(a.seed, n_sessions=a.sessions, scale=a.scale, long_wait_p=a.long_wait_p)
+    else:
+        trace, n_ctx = W.trace_c3(a.seed, n_sessions=a.sessions, scale=a.scale)
+    print(f"C3-shaped trace{' with an event clock' if a.timed else ''}: {a.sessions} sessions, scale {a.scale}, HBM {a.hbm} blocks, host tier {a.host} blocks, "
           f"metadata-only engines on the GPU")
     print("| policy | hit ratio | zombie share mean / peak | wrong-direction evictions | judged | offloaded | dropped |")
     print("|---|---:|---:|---:|---:|---:|---:|")

@@ -214,6 +214,86 @@ def trace_c3(seed: int, n_sessions: int = 32, min_len: int = 32768, max_len: int
     return ev, next_ctx
 
 
+def trace_c3_timed(seed: int, n_sessions: int = 32, min_len: int = 32768, max_len: int = 264192, scale: float = 1.0,
+                   long_wait_p: float = 0.0):
+    """C3 with a notion of time (Section 6.2: newly suspended KV waits while tools, sub-agents or other physical
+    stages run). Same sessions, turns, forks and edits as trace_c3, but every call is a batch of one and the order
+    of the calls comes from an event clock: after a call a session is busy for the call itself (0.3-1.5 s) plus a
+    tool wait, log-uniform 1-6 s, or 30-120 s with probability long_wait_p; a parent waits for its subagent, whose
+    calls take their own turns on the clock. Returns (events, number of context ids used)."""
+    import heapq
+    rng = np.random.default_rng([33, seed])
+    ev = []
+    targets = [int(_loguniform(rng, min_len, max_len) * scale) for _ in range(n_sessions)]
+    lens = [[] for _ in range(n_sessions)]
+    n_forks = [int(rng.integers(0, 5)) for _ in range(n_sessions)]
+    summaries = [[] for _ in range(n_sessions)]
+    next_ctx = n_sessions
+    ready = []          # (time, tie-break, kind, session, payload)
+    tick = 0
+
+    def wait():
+        t = 0.3 + 1.2 * rng.random()
+        t += _loguniform(rng, 30, 120) if rng.random() < long_wait_p else _loguniform(rng, 1, 6)
+        return t
+
+    for s in range(n_sessions):
+        ev.append(("spawn", s))
+        n = max(16, int(600 * scale))
+        ev.append(("append", s, _tokens(rng, n)))
+        lens[s].append(n)
+        if s % 4 == 0:
+            ev.append(("pin", s, 0, 1))
+        heapq.heappush(ready, (rng.random(), tick, "turn", s, None))
+        tick += 1
+    while ready:
+        now, _t, kind, s, pay = heapq.heappop(ready)
+        if kind == "turn":
+            for lo, hi in ((100, 2048), (200, 8192)):
+                n = max(1, int(_loguniform(rng, lo, hi) * scale))
+                ev.append(("append", s, _tokens(rng, n)))
+                lens[s].append(n)
+            if summaries[s] and rng.random() < 0.3:
+                j = summaries[s].pop(0)
+                if rng.random() < 0.5:
+                    n = max(1, int(_loguniform(rng, 100, 1024) * scale))
+                    ev.append(("replace", s, j, j + 1, _tokens(rng, n)))
+                    lens[s][j] = n
+                else:
+                    ev.append(("remove", s, j, j + 1))
+                    lens[s].pop(j)
+                    summaries[s] = [k - 1 if k > j else k for k in summaries[s]]
+            ev.append(("call", [s]))
+            if sum(lens[s]) >= targets[s]:
+                ev.append(("terminate", s))
+                continue
+            if n_forks[s] and rng.random() < 0.15:      # the parent now waits for a subagent
+                n_forks[s] -= 1
+                child = next_ctx
+                next_ctx += 1
+                ev.append(("fork", s, child, len(lens[s])))
+                heapq.heappush(ready, (now + wait(), tick, "sub", s, (child, int(rng.integers(1, 6)))))
+            else:
+                heapq.heappush(ready, (now + wait(), tick, "turn", s, None))
+            tick += 1
+        else:                                            # one call of a subagent
+            child, left = pay
+            n = max(1, int(_loguniform(rng, 200, 4096) * scale))
+            ev.append(("append", child, _tokens(rng, n)))
+            ev.append(("call", [child]))
+            if left > 1:
+                heapq.heappush(ready, (now + wait(), tick, "sub", s, (child, left - 1)))
+            else:
+                ev.append(("terminate", child))
+                n = max(1, int(_loguniform(rng, 100, 1024) * scale))
+                ev.append(("append", s, _tokens(rng, n)))
+                summaries[s].append(len(lens[s]))
+                lens[s].append(n)
+                heapq.heappush(ready, (now + wait(), tick, "turn", s, None))
+            tick += 1
+    return ev, next_ctx
+
+
 # ------------------------------------------------------------------------------------------------
 # C4: metadata-only lookup / eviction stress
 # ------------------------------------------------------------------------------------------------

@@ -151,6 +151,23 @@ def test_replay_with_a_remote_tier_keeps_more_blocks_reusable(make, flags):
     assert b["dropped"] < a["dropped"]
 
 
+def test_timed_trace_shows_the_recency_direction(make):
+    """C3 with an event clock and tool waits of 1-6 s (Section 6.2's premise: what was suspended last comes back
+    last): evicting the most recently suspended blocks first keeps more reusable KV than LRU does; with a tail of
+    very long waits the order turns around (the stragglers are what LRU evicts)."""
+    from paper_2609_39819_b200 import policy_metrics as PM
+    res = {}
+    for lw in (0.0, 0.1):
+        trace, n_ctx = W.trace_c3_timed(1, n_sessions=16, scale=1 / 32, long_wait_p=lw)
+        for order in (0, 1):
+            eng = make(n_hbm_blocks=400, n_host_blocks=400, max_contexts=n_ctx, suspended_order=order, metadata_only=True,
+                       **W.GEO_TOY.kwargs())
+            res[lw, order] = PM.replay_metrics(eng, trace)
+            check_invariants(eng)
+    assert res[0.0, 0]["hit_ratio"] > res[0.0, 1]["hit_ratio"] + 0.05 and res[0.0, 0]["dropped"] < res[0.0, 1]["dropped"]
+    assert res[0.1, 1]["hit_ratio"] > res[0.1, 0]["hit_ratio"]
+
+
 def test_incremental_appends_hash_like_one_shot(make, oracle):
     """Hashing a context after piecewise appends equals hashing the concatenation in one shot."""
     rng = np.random.default_rng(21)
