@@ -246,6 +246,17 @@ def test_trace_parity_with_a_remote_tier(B, oracle, flags):
             assert np.array_equal(eg[k], ec[k]), (tier, k)
 
 
+@pytest.mark.parametrize("order,lw", [(0, 0.0), (1, 0.1)])
+def test_timed_c3_trace_parity(B, oracle, order, lw):
+    """The C3 sessions ordered by an event clock (single-session calls, subagents interleaved with other sessions)."""
+    trace, n_ctx = W.trace_c3_timed(2, n_sessions=8, scale=1 / 32, long_wait_p=lw)
+    kw = dict(n_hbm_blocks=200, n_host_blocks=200, max_contexts=n_ctx, suspended_order=order, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 20, max_messages=1 << 15, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    n = _replay_pair(gpu, cpu, trace, W.payload_pattern, verify_every=11, use_exchange=bool(order))
+    assert n > 100 and cpu.get_stats()["reloaded"] > 0
+
+
 def test_scaled_c2_trace_parity(B, oracle):
     kw = dict(n_hbm_blocks=96, n_host_blocks=64, max_contexts=8, **W.GEO_TOY.kwargs())
     gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)
