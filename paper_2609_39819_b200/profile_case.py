@@ -171,7 +171,7 @@ def main(case: str):
             mv = f", move {m:.1f} ms = {gb / (m / 1e3):.1f} GB/s" if ctas is not None else ""
             print(f"overlap: {label}: {n_gemm} GEMMs in {g:.1f} ms = {flop / (g / 1e3) / 1e12:.0f} TFLOP/s{mv}")
     elif case == "exchange":
-        geo, n = W.GEO_8B, 1024
+        geo, n = W.GEO_8B, (int(sys.argv[2]) if len(sys.argv) > 2 else 1024)    # a smaller n for profiler captures
         eng = B.Engine(n_hbm_blocks=3 * n, n_host_blocks=3 * n, max_contexts=2, max_tokens=1 << 12, max_messages=64,
                        max_batch_blocks=4 * n, zero_pools=False, **geo.kwargs())
         ar = np.arange(n, dtype=np.uint32)
