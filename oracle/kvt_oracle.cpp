@@ -19,11 +19,13 @@
 // used here (chained 64-bit hash over 16-token blocks, lowest-free-slot-first, depth-descending then
 // slot-ascending ties, logical clock) are listed in the repository's design notes.
 //
-// Parity pins (tests marked "not gpu"): published SplitMix64 output stream for the mixing function
-// and the lane multipliers; closed form and affine-composition law of the chain; prefix / suffix
-// invariants; brute-force classification (kvto_classify_bruteforce) and brute-force victim order on
-// tiny pools; the paper's shared-KV example; Algorithm 1's order; LRU / reverse-LRU special cases;
-// byte-identical round trips. No function here is "parity unpinned".
+// What holds this file to the paper and to arithmetic, independently of the CUDA library (CPU-only tests):
+// the published SplitMix64 output stream for the mixing function and the lane multipliers; the closed
+// form and the affine-composition law of the chain; prefix / suffix invariants; the literal double loop
+// of Section 6.1 (kvto_classify_bruteforce) and a brute-force victim sort on tiny pools; the paper's
+// shared-KV example; Algorithm 1's order; LRU / reverse-LRU special cases; byte-identical round trips;
+// hand-worked scenarios for the destination slots of offload / move and for the recency stamps of a
+// call that ends in flight. Every function is covered by at least one of these.
 
 #include <algorithm>
 #include <cstdint>
@@ -743,6 +745,8 @@ int32_t kvto_move(Engine *e, uint32_t st, uint32_t dt, const uint32_t *slots, ui
   std::vector<uint8_t> rank[N_TIERS];
   classify(*e, rank);
   const bool knows_dead = !(e->cfg.policy_flags & POLICY_NO_LIFECYCLE);
+  // destinations as in kvto_offload: the slots free when the call begins. (Here that is the same set as "free at
+  // each step": a drop frees a slot of the source tier only, never one of the destination tier.)
   std::vector<uint32_t> dests(e->free_slots[dt].begin(), e->free_slots[dt].end());
   size_t next_dest = 0;
   for (uint32_t i = 0; i < n; ++i) {

@@ -842,8 +842,128 @@ def three_tiers(make):
     assert eng.get_stats()["occ_remote"] == 4
 
 
+# ---- destinations of a downward move = the slots free when the call begins (hand-worked) -----------------------
+def offload_destinations_are_fixed_at_call_begin(make):
+    """Inclusive tiers, one offload call that lists a dead block WITH a clean host copy ahead of a live block without
+    one. Dropping the dead block frees its copy's host slot (slot 0) in the middle of the call; the live block must
+    still go to the lowest slot that was free when the call began (slot 1), not to the slot the call itself freed."""
+    eng = make(n_hbm_blocks=6, n_host_blocks=6, max_contexts=4, policy_flags=2, **TOY)
+    rng = np.random.default_rng(31)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 64))
+    call(eng, 0)                                         # ctx 0: blocks 0..3 at HBM slots 0..3
+    eng.spawn(1)
+    eng.append(1, toks(rng, 32))
+    call(eng, 1)                                         # ctx 1: blocks 0, 1 at HBM slots 4, 5
+    k0 = eng.get_block_map(0)[0]
+    k1 = eng.get_block_map(1)[0]
+    for s, k in ((3, k0[3]), (4, k1[0]), (5, k1[1])):
+        eng.write_block(HBM, s, _payload(k, eng.block_bytes))
+    assert eng.offload([3]) == (0, 1, 0)                 # ctx 0's last block -> host slot 0
+    a = eng.map_blocks([0], LOOKUP)[0]
+    assert (a["hit_len"], a["n_hit_hbm"], a["n_hit_host"]) == (4, 3, 1)
+    assert eng.reload([0]) == (0, 1)                     # back to HBM slot 3; host slot 0 keeps the clean copy
+    eng.map_blocks([0], ADMIT)
+    eng.prefill_done(0)
+    eng.terminate(0)                                     # ctx 0's blocks are dead now, slot 3 still has its copy
+    assert states(eng) == [DEAD] * 4 + [IDLE] * 2
+    assert states(eng, HOST) == [SHADOW] + [FREE] * 5
+    # the call: dead-with-copy first, then two live blocks
+    assert eng.offload([3, 4, 5]) == (0, 3, 1)
+    assert states(eng) == [DEAD] * 3 + [FREE] * 3
+    assert states(eng, HOST) == [FREE, IDLE, IDLE, FREE, FREE, FREE]      # slot 0 was not free when the call began
+    _k, tier, slot = eng.get_block_map(1)
+    assert list(tier) == [HOST, HOST] and list(slot) == [1, 2]
+    assert np.array_equal(eng.read_block(HOST, 1), _payload(k1[0], eng.block_bytes))
+    assert np.array_equal(eng.read_block(HOST, 2), _payload(k1[1], eng.block_bytes))
+    st = eng.get_stats()
+    assert (st["occ_hbm"], st["occ_host"], st["dropped"]) == (3, 2, 1)
+    # the next call does see slot 0 as free
+    eng.spawn(2)
+    eng.append(2, toks(rng, 16))
+    call(eng, 2)                                         # one block at HBM slot 3 (lowest free)
+    assert eng.offload([3]) == (0, 1, 0)
+    assert list(eng.get_block_map(2)[1]) == [HOST] and list(eng.get_block_map(2)[2]) == [0]
+
+
+def move_down_with_a_dead_block_ahead(make):
+    """kvt_move(host -> remote) with a dead block listed ahead of live ones: the dead one is dropped without taking a
+    remote slot, the live ones take the lowest remote slots in list order. (No drop of such a call can free a remote
+    slot, so the slots free at call begin and the slots free at each step are the same set here.)"""
+    eng = make(n_hbm_blocks=6, n_host_blocks=4, n_remote_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(32)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 32))
+    call(eng, 0)                                         # ctx 0: HBM slots 0, 1
+    eng.spawn(1)
+    eng.append(1, toks(rng, 48))
+    call(eng, 1)                                         # ctx 1: HBM slots 2, 3, 4
+    k1 = eng.get_block_map(1)[0]
+    for b in range(3):
+        eng.write_block(HBM, 2 + b, _payload(k1[b], eng.block_bytes))
+    assert eng.offload([0, 2, 3, 4]) == (0, 4, 0)        # host slot 0: ctx 0 block 0; slots 1, 2, 3: ctx 1 blocks 0, 1, 2
+    assert eng.offload([1]) == (-5, 0, 0)                # host tier full
+    eng.release(HBM, [1])
+    # a remote slot is taken first so that "lowest free" is not slot 0
+    assert eng.move(HOST, REMOTE, [3]) == (0, 1, 0)      # ctx 1 block 2 -> remote slot 0
+    eng.terminate(0)                                     # host slot 0 is dead now
+    assert states(eng, HOST) == [DEAD, IDLE, IDLE, FREE]
+    assert eng.move(HOST, REMOTE, [0, 2, 1]) == (0, 3, 1)    # dead dropped; block 1 -> remote 1, block 0 -> remote 2
+    assert states(eng, HOST) == [FREE] * 4
+    assert states(eng, REMOTE) == [IDLE, IDLE, IDLE, FREE]
+    _k, tier, slot = eng.get_block_map(1)
+    assert list(tier) == [REMOTE] * 3 and list(slot) == [2, 1, 0]
+    for b in range(3):
+        assert np.array_equal(eng.read_block(REMOTE, int(slot[b])), _payload(k1[b], eng.block_bytes))
+    st = eng.get_stats()
+    assert (st["occ_host"], st["occ_remote"], st["demoted"]) == (0, 3, 3)
+
+
+# ---- recency stamps of a context that ends while its call is in flight (hand-worked) ----------------------------
+def stamps_of_a_call_that_is_terminated_in_flight(make):
+    """A block is stamped when a lookup hits it, when an admission inserts or adopts it and at PREFILL_DONE of a holder
+    (Section 6.2: the order of cache events). TERMINATE of an in-flight context releases its locks and stamps
+    nothing (Section 6.1: reclaimed once in-flight use completes). Clock values are worked out by hand below."""
+    eng = make(n_hbm_blocks=16, n_host_blocks=4, max_contexts=4, **TOY)
+    rng = np.random.default_rng(33)
+    eng.spawn(0)
+    eng.append(0, toks(rng, 80))
+    call(eng, 0)                                         # lookup: clock 1; done: clock 2. Slots 0..4 stamp 2
+    eng.spawn(1)
+    eng.append(1, toks(rng, 32))
+    call(eng, 1)                                         # clock 3, 4. Slots 5, 6 stamp 4
+    assert list(eng.get_entries(HBM)["stamp"][:7]) == [2] * 5 + [4] * 2
+    eng.release(HBM, [2])                                # ctx 0's blocks 3, 4 are now behind a hole
+    a = eng.map_blocks([0], LOOKUP)[0]                   # clock 5: blocks 0, 1 hit
+    assert (a["hit_len"], a["n_admissible"]) == (2, 3)
+    assert list(eng.get_entries(HBM)["stamp"][:5]) == [5, 5, 0, 2, 2]
+    b = eng.map_blocks([0], ADMIT)[0]                    # block 2 inserted at slot 2, blocks 3, 4 adopted
+    assert (b["n_admitted"], b["n_held"]) == (3, 5)
+    ent = eng.get_entries(HBM)
+    assert list(ent["stamp"][:5]) == [5] * 5 and list(ent["inflight"][:5]) == [1] * 5
+    eng.spawn(2)
+    eng.append(2, toks(rng, 16))
+    call(eng, 2)                                         # clock 6, 7. Slot 7 stamp 7
+    eng.spawn(3)
+    eng.append(3, toks(rng, 16))
+    call(eng, 3)                                         # clock 8, 9. Slot 8 stamp 9
+    eng.terminate(0)                                     # in flight: locks released, no stamp, clock stays 9
+    ent = eng.get_entries(HBM)
+    assert list(ent["stamp"][:9]) == [5, 5, 5, 5, 5, 4, 4, 7, 9]
+    assert list(ent["inflight"][:9]) == [0] * 9
+    assert eng.get_stats()["clock"] == 9
+    eng.terminate(1)
+    eng.terminate(2)
+    assert states(eng)[:9] == [DEAD] * 8 + [IDLE]
+    v, s = eng.select_victims(HBM, 16)
+    # dead, oldest stamp first, deeper block first inside one stamp: ctx 1 (stamp 4), ctx 0 (stamp 5), ctx 2 (7); then idle
+    assert list(v) == [6, 5, 4, 3, 2, 1, 0, 7, 8]
+    assert list(s) == [DEAD] * 8 + [IDLE]
+
+
 ALL = [state_machine_single_context, suffix_invalidation, fork_and_shared_kv, one_off_bypass, worked_example,
        mixed_pool_example, victim_order_bruteforce, one_state_pools_reduce_to_lru, offload_reload_round_trip,
        dead_victims_are_dropped_without_copy, compaction, raw_copy_blocks, admission_stops_when_full,
        lookup_locks_and_orphans, degenerate_inputs, pinned_retention, no_lifecycle_policy, inclusive_tiers, exchange_both_ways,
-       orphans_are_dead, three_tiers]
+       orphans_are_dead, three_tiers, offload_destinations_are_fixed_at_call_begin, move_down_with_a_dead_block_ahead,
+       stamps_of_a_call_that_is_terminated_in_flight]
