@@ -245,8 +245,13 @@ int32_t kvt_get_block_map(kvt_engine *e, uint32_t ctx, uint64_t *keys, uint8_t *
                           uint32_t *slot, uint32_t cap, uint32_t *n, void *stream);
 
 /* ---- stage 3: KV-level lifecycle state (Section 6.1 "Managing Shared KV") -------------------- */
-/* Recomputes, for every resident block, the highest-priority state over all (context, message
- * version) mappings; a block nobody maps is dead. Asynchronous on `stream`. */
+/* Brings the KV-level state of every resident block up to date: the highest-priority state over all (context,
+ * message version) mappings of its key; a block nobody maps is dead. The engine keeps, per block, the number of
+ * mappings of each priority and updates these counts by events (Section 6.1: the aggregate is updated whenever a
+ * mapped version changes state): this call applies what has happened since the last one (contexts whose messages,
+ * mapped prefix or token layout changed; contexts that ended; blocks that entered the table) and touches only the
+ * blocks of those contexts. Calls that need the states (selection, offload, ...) do the same on their own.
+ * With KVT_POLICY_ORPHANS_DEAD the states are recomputed in full. Asynchronous on `stream`. */
 int32_t kvt_classify(kvt_engine *e, void *stream);
 
 /* Copies the ranks of one tier to a host array (KVT_STATE_FREE for empty slots); classifies
@@ -263,7 +268,10 @@ int32_t kvt_get_states(kvt_engine *e, uint32_t tier, uint8_t *state, uint32_t ca
  * else, oldest first. states_out[i] is the rank, with KVT_STATE_HAS_COPY or-ed in for an HBM victim that
  * still has a clean host copy (offloading it moves no bytes and needs no host slot), or KVT_STATE_COPY.
  * With KVT_POLICY_NO_LIFECYCLE every candidate counts as rank 1. Classifies first if needed. Host output
- * arrays (states_out may be NULL). KVT_E_BUFSZ if cap < min(n_req, #candidates). Synchronises. */
+ * arrays (states_out may be NULL). KVT_E_BUFSZ if cap < min(n_req, #candidates). The order is computed on a packed
+ * key of 2 (+1 on a host tier with clean copies) + bits(clock) + bits(largest depth) bits; KVT_E_INVAL if that exceeds
+ * 63 bits (kvt_debug_load_resident refuses stamps and depths that would get there; the clock itself is 32 bits and
+ * calls that would advance it past 2^32 - 1 fail with KVT_E_NOSPACE). Synchronises. */
 int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_t flags, uint32_t *slots_out,
                            uint8_t *states_out, uint32_t cap, uint32_t *n_out, void *stream);
 
@@ -343,8 +351,9 @@ int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t ha
  *   - Limit: n_tokens <= KVT_HASH_NOALLOC_MAX_TOKENS; larger inputs are rejected with KVT_E_NOSPACE
  *     and nothing is launched. The scratch array takes 16 KiB of device memory on every GPU that
  *     loads the library, until the process exits.
- *   - The first call on each device looks up the array's device address (no allocation, but a
- *     runtime query): make that first call outside any stream capture.
+ *   - Every call asks the runtime for the array's address on the current device (no allocation). The
+ *     first call on a device is the one that makes the runtime set the library up there: make that
+ *     first call outside any stream capture.
  *   - All calls share the one array. Nothing in it has to start at zero (each call overwrites what it
  *     later reads), but two calls whose kernels overlap on the GPU (different streams, or different
  *     host threads) race on it: keep calls on one device ordered.
@@ -407,6 +416,16 @@ int32_t kvt_set_mover_ctas(kvt_engine *e, uint32_t max_ctas);
  * single pass measured slower on B200 (its CTAs live too long to keep enough token bytes in flight). */
 int32_t kvt_debug_set_lookup_variant(kvt_engine *e, uint32_t variant);
 
+/* Test / measurement hook for the classification: 0 = event-driven (default), 1 = every kvt_classify recomputes all
+ * counts from zero over all contexts, 2 = event-driven, and every update is followed by a full recomputation that must
+ * give the same counts (KVT_E_DEVICE if not). */
+int32_t kvt_debug_set_classify_mode(kvt_engine *e, uint32_t mode);
+
+/* Test hook for the bounded wait of the single-pass lookup (variant 2): the number of polls a chunk spends on its
+ * predecessors' publications before it gives up (default 2^18). With 0 every chunk that needs a predecessor gives
+ * up at once: the kernel still returns normally, the call reports KVT_E_DEVICE and the engine is unchanged. */
+int32_t kvt_debug_set_wait_limit(kvt_engine *e, uint32_t polls);
+
 /* Text of the last error of this engine (always NUL-terminated). */
 int32_t kvt_last_error(kvt_engine *e, char *buf, uint32_t cap);
 
@@ -419,8 +438,8 @@ int32_t kvt_get_entries(kvt_engine *e, uint32_t tier, uint64_t *keys, uint32_t *
 /* Test / benchmark hook: makes n blocks resident in `tier` at the given slots without running
  * calls. state[i] acts as a permanent anonymous mapping of that rank (classification never reports
  * less for the block until it is dropped). Keys must be >= 2, distinct and not resident; slots
- * free and distinct (violations: KVT_E_INVAL, state unchanged). Advances the logical clock to at
- * least max(stamp). Host arrays. Synchronises. */
+ * free and distinct, and 3 + bits(max stamp) + bits(max depth) <= 63 (violations: KVT_E_INVAL, state unchanged).
+ * Advances the logical clock to at least max(stamp). Host arrays. Synchronises. */
 int32_t kvt_debug_load_resident(kvt_engine *e, const uint64_t *keys, const uint8_t *state,
                                 const uint32_t *stamp, const uint32_t *depth,
                                 const uint32_t *slot, uint32_t tier, uint32_t n, void *stream);

@@ -11,6 +11,8 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libkvt.so")
+# KVT_LIB=<path>: load another build of the same sources instead (the checked build libkvt_debug.so, a traced build)
+ALT_LIB = os.environ.get("KVT_LIB")
 
 OK, E_INVAL, E_NOCTX, E_RANGE, E_STATE, E_NOSPACE, E_BUFSZ, E_DEVICE, E_CUDA = 0, -1, -2, -3, -4, -5, -6, -7, -8
 TIER_HBM, TIER_HOST, TIER_REMOTE, TIER_NONE = 0, 1, 2, 0xFF
@@ -27,7 +29,8 @@ EXPORTS = ("kvt_query_sizes", "kvt_create", "kvt_destroy", "kvt_apply_op", "kvt_
            "kvt_classify", "kvt_get_states", "kvt_select_victims", "kvt_offload", "kvt_reload", "kvt_release",
            "kvt_compact", "kvt_copy_blocks", "kvt_hash_scratch_bytes", "kvt_hash_tokens", "kvt_get_stats",
            "kvt_last_error", "kvt_get_entries", "kvt_debug_load_resident", "kvt_set_profiling",
-           "kvt_hash_tokens_noalloc", "kvt_debug_set_mover_variant", "kvt_exchange", "kvt_debug_set_lookup_variant", "kvt_move", "kvt_set_mover_ctas")
+           "kvt_hash_tokens_noalloc", "kvt_debug_set_mover_variant", "kvt_exchange", "kvt_debug_set_lookup_variant", "kvt_move", "kvt_set_mover_ctas",
+           "kvt_debug_set_wait_limit", "kvt_debug_set_classify_mode")
 
 
 class KvtError(RuntimeError):
@@ -71,14 +74,23 @@ def load_library():
     """Loads libkvt.so (built in-tree by paper_2609_39819_b200.build). Raises if it is missing."""
     global _lib
     if _lib is None:
-        if not os.path.exists(LIB_PATH):
-            try:                                   # a build step, not a fallback: compile the CUDA library in-tree
-                from . import build
+        if ALT_LIB:
+            if not os.path.exists(ALT_LIB):
+                raise RuntimeError(f"KVT_LIB={ALT_LIB} does not exist")
+            lib_path = ALT_LIB
+        else:
+            lib_path = LIB_PATH
+        try:                                       # a build step, not a fallback: (re)compile the CUDA library
+            from . import build                    # in-tree when it is missing or older than its sources
+            if not ALT_LIB:
                 build.build_lib()
-            except Exception as exc:
+        except Exception as exc:
+            if not os.path.exists(LIB_PATH):
                 raise RuntimeError(f"{LIB_PATH} is missing and could not be built with nvcc ({exc}); "
                                    "there is no CPU fallback") from exc
-        lib = C.CDLL(LIB_PATH)
+            import warnings
+            warnings.warn(f"libkvt.so could not be rebuilt ({exc}); loading the existing binary")
+        lib = C.CDLL(lib_path)
         vp, u32, u64, i32 = C.c_void_p, C.c_uint32, C.c_uint64, C.c_int32
         sig = {
             "kvt_query_sizes": [vp, vp, vp],
@@ -105,6 +117,8 @@ def load_library():
             "kvt_debug_set_mover_variant": [vp, u32],
             "kvt_debug_set_lookup_variant": [vp, u32],
             "kvt_set_mover_ctas": [vp, u32],
+            "kvt_debug_set_wait_limit": [vp, u32],
+            "kvt_debug_set_classify_mode": [vp, u32],
             "kvt_get_entries": [vp, u32, vp, vp, vp, vp, vp, u32, vp],
             "kvt_debug_load_resident": [vp, vp, vp, vp, vp, vp, u32, u32, vp],
         }
@@ -256,6 +270,12 @@ class Engine:
 
     def set_lookup_variant(self, variant):
         self._check(self.L.kvt_debug_set_lookup_variant(self.h, variant), "set_lookup_variant")
+
+    def set_classify_mode(self, mode):
+        self._check(self.L.kvt_debug_set_classify_mode(self.h, mode), "set_classify_mode")
+
+    def set_wait_limit(self, polls):
+        self._check(self.L.kvt_debug_set_wait_limit(self.h, polls), "set_wait_limit")
 
     def last_error(self):
         buf = C.create_string_buffer(256)

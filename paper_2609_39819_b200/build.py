@@ -11,6 +11,7 @@ SOURCES = ["kvt_engine.cu"]
 DEPS = ["kvt_kernels.cuh", os.path.join("..", "..", "include", "kvt.h")]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "-shared",
               "-Xcompiler", "-fPIC"]
+DEFINES: list = []
 
 
 def _stale() -> bool:
@@ -22,11 +23,28 @@ def _stale() -> bool:
 
 
 def build_lib(force: bool = False, verbose: bool = False) -> str:
-    if force or _stale():
-        nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
-        cmd = [nvcc] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-              ["-o", LIB] + [os.path.join(CSRC, s) for s in SOURCES]
-        subprocess.check_call(cmd)
+    """Compiles libkvt.so if it is missing or older than its sources. Safe when several processes call it at once
+    (one rank per GPU): an exclusive file lock serialises them, the compiler writes to a temporary file and the
+    result is moved into place in one step, so nobody ever loads a half-written library."""
+    if not (force or _stale()):
+        return LIB
+    import fcntl
+    with open(LIB + ".lock", "w") as lock:
+        fcntl.flock(lock, fcntl.LOCK_EX)
+        try:
+            if force or _stale():            # somebody else may have built it while we waited
+                nvcc = os.environ.get("NVCC", "/usr/local/cuda/bin/nvcc")
+                tmp = f"{LIB}.{os.getpid()}.tmp"
+                cmd = [nvcc] + NVCC_FLAGS + DEFINES + (["-Xptxas", "-v"] if verbose else []) + \
+                      ["-o", tmp] + [os.path.join(CSRC, s) for s in SOURCES]
+                try:
+                    subprocess.check_call(cmd)
+                    os.replace(tmp, LIB)
+                finally:
+                    if os.path.exists(tmp):
+                        os.remove(tmp)
+        finally:
+            fcntl.flock(lock, fcntl.LOCK_UN)
     return LIB
 
 

@@ -9,6 +9,7 @@
 
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <string>
@@ -63,8 +64,14 @@ struct Msg { u32 len; u8 state; };
 // call can resume hashing at a chunk boundary instead of block 0).
 struct KeySeg { u64 off = 0, cap = 0, keycap = 0; u32 refs = 0; };
 
+// What the per-block mapping counts currently contain for one context: the key list, the mapped prefix length and
+// the message table (slice of the device message arrays) it was accounted with. Holds a reference on the key segment.
+struct Snap { int keyseg = -1; u32 valid = 0; u64 tbl_off = 0; u32 tbl_n = 0; };
+
 struct Ctx {
   bool live = false, one_off = false, in_flight = false;
+  bool map_dirty = false;    // messages, mapped prefix or key list changed since `synced` was taken
+  Snap synced;
   bool terminated = false;   // ended but kept: it still has Pinned messages
   std::vector<Msg> msgs;
   std::vector<std::pair<u32, u32>> mat_bounds;  // bounds of the leading messages still valid in the materialised layout
@@ -75,9 +82,9 @@ struct Ctx {
 };
 
 struct DevLayout {
-  u64 tab, e_key, e_stamp, e_depth, e_infl, e_rank, e_tslot, e_mark, e_link, e_floor, keys, status;
+  u64 tab, e_key, e_stamp, e_depth, e_infl, e_cnt, e_tslot, e_mark, e_link, e_floor, cnt_chk, fresh, keys, status;
   u64 s0, s1, s2, s3, ids, ids2, pair_src, pair_dst, pair_src2, pair_dst2, freelist, freelist2, tiles, agg, carry, cflags, desc, ctxres;
-  u64 m_start, m_end, m_rank, keyA, keyB, valA, valB, rcounts, out_slots, out_states, map_tier, map_slot;
+  u64 m_start, m_end, m_rank, keyA, keyB, valA, valB, rcounts, sel_cta, sel_args, slot_key, sel_hist, sel_state, out_slots, out_states, map_tier, map_slot;
   u64 total;
   u64 LB, Nt, N;
 };
@@ -92,7 +99,9 @@ DevLayout make_layout(const kvt_config &c) {
   auto take = [&](u64 bytes) { u64 o = off; off = round_up(off + bytes, 256); return o; };
   L.tab = take((u64)c.table_capacity * 16);
   L.e_key = take(N * 8); L.e_stamp = take(N * 4); L.e_depth = take(N * 4); L.e_infl = take(N * 4);
-  L.e_rank = take(N * 4); L.e_tslot = take(N * 4); L.e_mark = take(N * 4); L.e_link = take(N * 4); L.e_floor = take(N);
+  L.e_cnt = take(N * 8); L.e_tslot = take(N * 4); L.e_mark = take(N * 4); L.e_link = take(N * 4); L.e_floor = take(N);
+  L.cnt_chk = take(N * 8);   // the counts of a full recomputation, for the cross-check mode
+  L.fresh = take(N * 4);     // entries inserted since the counts were last brought up to date
   L.keys = take((c.max_key_blocks + c.max_key_blocks / CHUNK + 64ull * c.max_contexts) * 8);   // keys + per-chunk carries
   L.status = take(ST_WORDS * 4);
   L.s0 = take(LB * 4); L.s1 = take(LB * 4); L.s2 = take(LB * 4); L.s3 = take(LB * 4);
@@ -102,11 +111,16 @@ DevLayout make_layout(const kvt_config &c) {
   u64 n_chunks = B / CHUNK + C + 1;
   L.agg = take(n_chunks * 8); L.carry = take(n_chunks * 8);   // per-chunk aggregates / chain values of a LOOKUP batch
   L.cflags = take((n_chunks + 1) * 4);                         // per-chunk publication flags + the ticket word
-  L.desc = take(C * 64 + 2 * n_chunks * 4);   // per-context descriptors, then the chunk -> context maps of a LOOKUP batch
+  L.desc = take(C * 256 + 2 * n_chunks * 4);  // per-context descriptors, then the chunk -> context maps of a LOOKUP batch
   L.ctxres = take(C * 20);   // per context: hit_len, hits per tier (3), admission stop
-  L.m_start = take(Mm * 4); L.m_end = take(Mm * 4); L.m_rank = take(Mm);
+  L.m_start = take(2 * Mm * 4); L.m_end = take(2 * Mm * 4); L.m_rank = take(2 * Mm);   // accounted-for tables + the new ones of a pass
   L.keyA = take(Nt * 8); L.keyB = take(Nt * 8); L.valA = take(Nt * 4); L.valB = take(Nt * 4);
-  L.rcounts = take((256ull * (Nt / SORT_TILE + 1) + 256) * 4);
+  L.rcounts = take(((u64)RADIX_BINS * (Nt / SORT_TILE + 1) + RADIX_BINS) * 4);
+  L.sel_cta = take((Nt / SEL_TILE + 2) * 4);
+  L.sel_args = take(sizeof(SelArgs));
+  L.slot_key = take(Nt * 8);
+  L.sel_hist = take((u64)SEL_MAX_LEVELS * SEL_BINS * 4);
+  L.sel_state = take((SEL_MAX_LEVELS + 1) * sizeof(SelState));
   L.out_slots = take(Nt * 4); L.out_states = take(Nt);
   L.map_tier = take(B); L.map_slot = take(B * 4);
   L.total = off;
@@ -134,7 +148,12 @@ struct kvt_engine {
   u32 now = 0, max_depth = 0;
   u32 occ[3] = {0, 0, 0};
   u32 tombs = 0;
-  bool dirty = true;
+  bool dirty = true;          // something below is pending: the counts are not up to date
+  bool full_dirty = true;     // the counts must be recomputed from scratch (start; debug loads; after an arena ran out)
+  std::vector<Snap> zombies;  // what is still accounted for contexts that have ended
+  u32 n_fresh = 0;            // entries in the device list L.fresh
+  RangeAlloc tbl_alloc;       // slices of the device message arrays
+  u32 classify_mode = 0;      // 0 event-driven, 1 full recomputation every time, 2 event-driven + cross-check
   kvt_stats st{};
   std::string err;
   // pinned host staging
@@ -144,11 +163,12 @@ struct kvt_engine {
   bool upload_pending = false;
   // optional timing of the mover kernel (kvt_set_profiling)
   bool profiling = false, mover_timed = false;
-  // CUDA graph of the radix-sort passes of kvt_select_victims, one per tier
-  struct SortGraph { cudaGraphExec_t exec = nullptr; u32 n_pass = 0; };
-  SortGraph sort_graph[3];
+  // CUDA graph of the kernel sequence of kvt_select_victims, one per tier
+  struct SelGraph { cudaGraphExec_t exec = nullptr; };
+  std::map<u64, SelGraph> sel_graph[3];    // keyed by (level count, pass count, sort tiles)
   cudaStream_t capture_stream = nullptr;   // only ever used for stream capture, never executes work
   bool use_graphs = true;
+  SelArgs *h_sel = nullptr;                // pinned staging of the selection's argument record
   u32 mover_variant = 0;   // 0 auto, 1 CTA per chunk, 2 warp per 4 KiB tile, 3 TMA ring
   u32 mover_max_ctas = 0;  // caller's upper bound on the mover's grid (0: automatic)
   bool tier_in_host_mem[3] = {false, false, false};   // pool is host memory: moves to / from it are bound by the host link
@@ -162,6 +182,7 @@ struct kvt_engine {
   }
   u32 link_dirs(u32 st, u32 dt) const { return (tier_in_host_mem[st] || tier_in_host_mem[dt]) ? 1u : 0u; }
   u32 lookup_variant = 0;  // 0 / 1 digest / carry / finish kernels, 2 single-pass hash + probe kernel
+  u32 wait_limit = 1u << 18;   // polls a chunk of the single-pass kernel spends on its predecessors before it gives up
   bool tma_attr_set = false;
   cudaEvent_t ev_m0 = nullptr, ev_m1 = nullptr, ev_h0 = nullptr, ev_h1 = nullptr;
 
@@ -189,6 +210,33 @@ namespace {
   } while (0)
 
 int32_t fail(kvt_engine *e, int32_t code, const char *msg) { e->err = msg; return code; }
+
+// Per-kernel timing for development builds (-DKVT_TRACE): an event after every marked launch, the gaps printed to
+// stderr once the call has synchronised. Compiles to nothing otherwise.
+#ifdef KVT_TRACE
+struct Trace { cudaEvent_t ev[64]; const char *name[64]; int n = 0; bool init = false; };
+static Trace g_trace;
+static void trace_mark(cudaStream_t s, const char *name) {
+  Trace &t = g_trace;
+  if (!t.init) { for (auto &x : t.ev) cudaEventCreate(&x); t.init = true; }
+  if (t.n < 64) { t.name[t.n] = name; cudaEventRecord(t.ev[t.n++], s); }
+}
+static void trace_dump(const char *what) {
+  Trace &t = g_trace;
+  if (t.n > 1 && getenv("KVT_TRACE")) {
+    fprintf(stderr, "[trace] %s:", what);
+    for (int i = 1; i < t.n; ++i) { float ms = 0; cudaEventElapsedTime(&ms, t.ev[i - 1], t.ev[i]); fprintf(stderr, " %s %.1f", t.name[i], ms * 1e3f); }
+    float tot = 0; cudaEventElapsedTime(&tot, t.ev[0], t.ev[t.n - 1]);
+    fprintf(stderr, " | total %.1f us\n", tot * 1e3f);
+  }
+  t.n = 0;
+}
+#define TRACE(s, name) trace_mark(s, name)
+#define TRACE_DUMP(what) trace_dump(what)
+#else
+#define TRACE(s, name) do {} while (0)
+#define TRACE_DUMP(what) do {} while (0)
+#endif
 
 int32_t launch_ok(kvt_engine *e) {
   cudaError_t x = cudaGetLastError();
@@ -352,59 +400,204 @@ void mover_account(kvt_engine *e, u64 blocks) {
 }
 
 // ---- classification -------------------------------------------------------------------------------------
-int32_t do_classify(kvt_engine *e, cudaStream_t s) {
+constexpr int32_t INT_TBL_FULL = -100;   // internal: no room for the new message tables
+
+// Message table of a context as it stands: the leading messages whose materialised bounds touch a mapped block.
+u32 build_table(const Ctx &c, u32 *ms, u32 *me, u8 *mr, u32 cap) {
+  u32 k = 0;
+  for (size_t j = 0; j < c.mat_bounds.size(); ++j) {
+    if (c.mat_bounds[j].first >= c.valid_blocks * 16ull) break;  // later messages touch no mapped block
+    if (k >= cap) return 0xFFFFFFFFu;
+    ms[k] = c.mat_bounds[j].first; me[k] = c.mat_bounds[j].second; mr[k] = msg_rank(c.msgs[j].state);
+    ++k;
+  }
+  return k;
+}
+
+void snap_release(kvt_engine *e, Snap &sn) {
+  if (sn.tbl_n) e->tbl_alloc.release(sn.tbl_off, sn.tbl_n);
+  seg_deref(e, sn.keyseg);
+  sn = Snap();
+}
+
+MsgTables msg_tables(kvt_engine *e) { return MsgTables{e->dp<u32>(e->L.m_start), e->dp<u32>(e->L.m_end), e->dp<u8>(e->L.m_rank)}; }
+
+// Runs the delta kernel over the listed contexts (nullptr = a context that has ended: everything it was accounted
+// for is taken away) and makes the current state what is accounted for. from_zero: the old side is empty for all.
+int32_t apply_deltas(kvt_engine *e, cudaStream_t s, const std::vector<Ctx *> &list, std::vector<Snap> &ended, bool from_zero) {
+  const u32 nd = (u32)(list.size() + ended.size());
+  if (!nd) return KVT_OK;
+  const u64 C = e->cfg.max_contexts, Mm = e->cfg.max_messages;
+  if (nd > 2 * C) return fail(e, KVT_E_NOSPACE, "too many contexts ended since the last classification");
+  DeltaCtx *hd = reinterpret_cast<DeltaCtx *>(e->h_desc + 2 * C * sizeof(SnapDesc));
+  u32 nm = 0, nmap = 0, k = 0;
+  std::vector<u32> tbl_n(list.size());
+  for (size_t i = 0; i < list.size(); ++i) {
+    const Ctx &c = *list[i];
+    const bool maps = c.valid_blocks && c.keyseg >= 0;
+    u32 n = maps ? build_table(c, e->h_mstart + nm, e->h_mend + nm, e->h_mrank + nm, (u32)Mm - nm) : 0;
+    if (n == 0xFFFFFFFFu) return fail(e, KVT_E_NOSPACE, "max_messages exceeded");
+    tbl_n[i] = n;
+    nm += n;
+  }
+  u64 tbl_base = 0;
+  if (nm && !e->tbl_alloc.alloc(nm, &tbl_base)) return INT_TBL_FULL;   // caller falls back to the full recomputation
+  u32 off = 0;
+  for (size_t i = 0; i < list.size(); ++i) {
+    const Ctx &c = *list[i];
+    const bool maps = c.valid_blocks && c.keyseg >= 0;
+    const Snap &o = c.synced;
+    DeltaCtx d{};
+    if (!from_zero && o.keyseg >= 0) { d.old_key_off = e->segs[o.keyseg].off; d.old_valid = o.valid; d.old_tbl = (u32)o.tbl_off; d.old_n = o.tbl_n; }
+    if (maps) { d.new_key_off = e->segs[c.keyseg].off; d.new_valid = c.valid_blocks; d.new_tbl = (u32)(tbl_base + off); d.new_n = tbl_n[i]; }
+    d.map_base = nmap;
+    nmap += std::max(d.old_valid, d.new_valid);
+    off += tbl_n[i];
+    hd[k++] = d;
+  }
+  for (const Snap &o : ended) {
+    DeltaCtx d{};
+    if (!from_zero && o.keyseg >= 0) { d.old_key_off = e->segs[o.keyseg].off; d.old_valid = o.valid; d.old_tbl = (u32)o.tbl_off; d.old_n = o.tbl_n; }
+    d.map_base = nmap;
+    nmap += d.old_valid;
+    hd[k++] = d;
+  }
+  if (nmap) {
+    DeltaCtx *dd = reinterpret_cast<DeltaCtx *>(e->dp<u8>(e->L.desc) + 2 * C * sizeof(SnapDesc));
+    CU(cudaMemcpyAsync(dd, hd, nd * sizeof(DeltaCtx), cudaMemcpyHostToDevice, s));
+    if (nm) {
+      CU(cudaMemcpyAsync(e->dp<u32>(e->L.m_start) + tbl_base, e->h_mstart, nm * 4ull, cudaMemcpyHostToDevice, s));
+      CU(cudaMemcpyAsync(e->dp<u32>(e->L.m_end) + tbl_base, e->h_mend, nm * 4ull, cudaMemcpyHostToDevice, s));
+      CU(cudaMemcpyAsync(e->dp<u8>(e->L.m_rank) + tbl_base, e->h_mrank, nm, cudaMemcpyHostToDevice, s));
+    }
+    DeltaArgs a;
+    a.tab = e->tab; a.ent = e->ent; a.keys = e->d_keys; a.ctx = dd; a.n_ctx = nd; a.n_map = nmap; a.tbl = msg_tables(e);
+    a.status = e->d_status; a.first_miss = nullptr;
+    if (from_zero && (e->cfg.policy_flags & KVT_POLICY_ORPHANS_DEAD)) {
+      a.first_miss = e->dp<u32>(e->L.freelist2);   // scratch of the list calls, free between calls (stream order)
+      if (nd > e->L.LB) return fail(e, KVT_E_NOSPACE, "more contexts than max_batch_blocks");
+      CU(cudaMemsetAsync(a.first_miss, 0xFF, nd * 4ull, s));
+      KL(k_first_miss, cdiv(nmap, 256), 256, s, a);
+    }
+    KL(k_map_delta, cdiv(nmap, 256), 256, s, a);
+    LAUNCH_CHECK();
+  }
+  // what is accounted for now
+  off = 0;
+  for (size_t i = 0; i < list.size(); ++i) {
+    Ctx &c = *list[i];
+    const bool maps = c.valid_blocks && c.keyseg >= 0;
+    Snap n;
+    if (maps) { n.keyseg = c.keyseg; e->segs[c.keyseg].refs++; n.valid = c.valid_blocks; n.tbl_off = tbl_base + off; n.tbl_n = tbl_n[i]; }
+    off += tbl_n[i];
+    snap_release(e, c.synced);
+    c.synced = n;
+    c.map_dirty = false;
+  }
+  for (Snap &o : ended) snap_release(e, o);
+  ended.clear();
+  return KVT_OK;
+}
+
+// Recomputes every count from zero over all contexts.
+int32_t full_recount(kvt_engine *e, cudaStream_t s) {
+  for (Ctx &c : e->ctxs) if (c.live) snap_release(e, c.synced);
+  for (Snap &o : e->zombies) snap_release(e, o);
+  e->zombies.clear();
+  e->tbl_alloc.init(2ull * e->cfg.max_messages, 1);
+  CU(cudaMemsetAsync(e->ent.cnt, 0, (u64)e->ent.n_total * 8, s));
+  std::vector<Ctx *> all;
+  for (Ctx &c : e->ctxs) if (c.live) all.push_back(&c);
+  int32_t r = apply_deltas(e, s, all, e->zombies, true);
+  return r == INT_TBL_FULL ? fail(e, KVT_E_NOSPACE, "max_messages exceeded") : r;
+}
+
+// Brings the per-block mapping counts up to date with everything that happened since the last time.
+int32_t do_classify(kvt_engine *e, cudaStream_t s, bool force_full = false) {
   int32_t r = stage_acquire(e);
   if (r) return r;
-  ClsCtx *hd = reinterpret_cast<ClsCtx *>(e->h_desc);
-  u32 nc = 0, nm = 0, nmap = 0;
-  for (Ctx &c : e->ctxs) {
-    if (!c.live || c.valid_blocks == 0 || c.keyseg < 0) continue;
-    ClsCtx d;
-    d.key_off = e->segs[c.keyseg].off; d.map_base = nmap; d.valid = c.valid_blocks; d.msg_base = nm;
-    u32 k = 0;
-    for (size_t j = 0; j < c.mat_bounds.size(); ++j) {
-      if (c.mat_bounds[j].first >= c.valid_blocks * 16ull) break;  // later messages touch no mapped block
-      if (nm + k >= e->cfg.max_messages) return fail(e, KVT_E_NOSPACE, "max_messages exceeded");
-      e->h_mstart[nm + k] = c.mat_bounds[j].first;
-      e->h_mend[nm + k] = c.mat_bounds[j].second;
-      e->h_mrank[nm + k] = msg_rank(c.msgs[j].state);
-      ++k;
+  const bool full = force_full || e->full_dirty || e->classify_mode == 1 || (e->cfg.policy_flags & KVT_POLICY_ORPHANS_DEAD);
+  if (full) {
+    r = full_recount(e, s);
+    if (r) return r;
+  } else {
+    const u64 C = e->cfg.max_contexts;
+    // (1) entries inserted since then get the contributions of every mapping already accounted for
+    if (e->n_fresh) {
+      SnapDesc *hs = reinterpret_cast<SnapDesc *>(e->h_desc);
+      u32 ns = 0;
+      auto add = [&](const Snap &o) {
+        if (o.keyseg < 0 || !o.valid || ns >= 2 * C) return;
+        hs[ns++] = SnapDesc{e->segs[o.keyseg].off, o.valid, (u32)o.tbl_off, o.tbl_n, 0};
+      };
+      for (const Ctx &c : e->ctxs) if (c.live) add(c.synced);
+      for (const Snap &o : e->zombies) add(o);
+      if (ns) {
+        SnapDesc *ds = reinterpret_cast<SnapDesc *>(e->dp<u8>(e->L.desc));
+        CU(cudaMemcpyAsync(ds, hs, ns * sizeof(SnapDesc), cudaMemcpyHostToDevice, s));
+        FixArgs a;
+        a.tab = e->tab; a.ent = e->ent; a.keys = e->d_keys; a.snaps = ds; a.n_snaps = ns; a.tbl = msg_tables(e);
+        a.fresh = e->dp<u32>(e->L.fresh); a.n_fresh = e->n_fresh; a.status = e->d_status;
+        KL(k_fresh_fixup, cdiv(e->n_fresh, 128), 128, s, a);
+      }
     }
-    d.n_msgs = k;
-    nm += k; nmap += c.valid_blocks;
-    hd[nc++] = d;
-  }
-  KL(k_rank_reset, cdiv(e->ent.n_total,256), 256, s, e->ent);
-  if (nmap) {
-    CU(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nc * sizeof(ClsCtx), cudaMemcpyHostToDevice, s));
-    CU(cudaMemcpyAsync(e->dp<u8>(e->L.m_start), e->h_mstart, nm * 4ull, cudaMemcpyHostToDevice, s));
-    CU(cudaMemcpyAsync(e->dp<u8>(e->L.m_end), e->h_mend, nm * 4ull, cudaMemcpyHostToDevice, s));
-    CU(cudaMemcpyAsync(e->dp<u8>(e->L.m_rank), e->h_mrank, nm, cudaMemcpyHostToDevice, s));
-    ClsArgs a;
-    a.tab = e->tab; a.ent = e->ent; a.keys = e->d_keys; a.ctx = e->dp<ClsCtx>(e->L.desc); a.n_ctx = nc; a.n_map = nmap;
-    a.m_start = e->dp<u32>(e->L.m_start); a.m_end = e->dp<u32>(e->L.m_end); a.m_rank = e->dp<u8>(e->L.m_rank);
-    a.status = e->d_status;
-    a.first_miss = nullptr;
-    if (e->cfg.policy_flags & KVT_POLICY_ORPHANS_DEAD) {
-      a.first_miss = e->dp<u32>(e->L.ctxres);   // per-call scratch of the lookup, free between calls (stream order)
-      CU(cudaMemsetAsync(a.first_miss, 0xFF, nc * 4ull, s));
-      KL(k_first_miss, cdiv(nmap,256), 256, s, a);
-    }
-    KL(k_classify, cdiv(nmap,256), 256, s, a);
-    r = stage_release(e, s);
+    // (2) contexts that changed, and contexts that ended
+    std::vector<Ctx *> list;
+    for (Ctx &c : e->ctxs) if (c.live && c.map_dirty) list.push_back(&c);
+    r = apply_deltas(e, s, list, e->zombies, false);
+    if (r == INT_TBL_FULL) r = full_recount(e, s);   // the table arena is fragmented or full: start over
     if (r) return r;
   }
+  e->n_fresh = 0;
+  r = stage_release(e, s);
+  if (r) return r;
   LAUNCH_CHECK();
   e->dirty = false;
+  e->full_dirty = false;
+  if (e->classify_mode == 2 && !full) {   // cross-check: the event-driven counts must equal a full recomputation
+    CU(cudaMemcpyAsync(e->dp<u64>(e->L.cnt_chk), e->ent.cnt, (u64)e->ent.n_total * 8, cudaMemcpyDeviceToDevice, s));
+    r = do_classify(e, s, true);
+    if (r) return r;
+    CU(cudaMemsetAsync(e->d_status + ST_CHK, 0, 4, s));
+    KL(k_cnt_compare, cdiv(e->ent.n_total, 256), 256, s, e->dp<u64>(e->L.cnt_chk), e->ent.cnt, e->ent.n_total, e->d_status + ST_CHK);
+    LAUNCH_CHECK();
+    CU(cudaMemcpyAsync(e->h_status + ST_CHK, e->d_status + ST_CHK, 4, cudaMemcpyDeviceToHost, s));
+    CU(cudaStreamSynchronize(s));
+    if (e->h_status[ST_CHK]) return fail(e, KVT_E_DEVICE, "event-driven classification differs from the full recomputation");
+  }
   return KVT_OK;
 }
 
 int32_t ensure_classified(kvt_engine *e, cudaStream_t s) { return e->dirty ? do_classify(e, s) : KVT_OK; }
 
+// A context ends: what is accounted for it is kept until the next classification takes it away.
+int32_t retire_ctx(kvt_engine *e, Ctx &c, cudaStream_t s) {
+  if (c.synced.keyseg >= 0 && c.synced.valid) {
+    if (e->zombies.size() >= e->cfg.max_contexts) {   // bounded: bring the counts up to date first
+      c.map_dirty = true;
+      int32_t r = do_classify(e, s);
+      if (r) return r;
+    }
+    e->zombies.push_back(c.synced);
+    c.synced = Snap();
+  } else {
+    snap_release(e, c.synced);
+  }
+  seg_deref(e, c.keyseg);
+  c = Ctx();
+  return KVT_OK;
+}
+
 // ---- token buffers ---------------------------------------------------------------------------------------
 int32_t copy_tokens_in(kvt_engine *e, cudaStream_t s, u64 dst_tok, const u32 *src, u32 n, bool on_device) {
   if (!n) return KVT_OK;
   CU(cudaMemcpyAsync(e->d_tokens + dst_tok, src, (u64)n * 4, on_device ? cudaMemcpyDeviceToDevice : cudaMemcpyHostToDevice, s));
+  return KVT_OK;
+}
+
+int32_t copy_tokens_dd(kvt_engine *e, cudaStream_t s, u64 dst_tok, u64 src_tok, u64 n) {
+  if (!n) return KVT_OK;
+  CU(cudaMemcpyAsync(e->d_tokens + dst_tok, e->d_tokens + src_tok, n * 4, cudaMemcpyDeviceToDevice, s));
   return KVT_OK;
 }
 
@@ -515,7 +708,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   e->tab.slots = e->dp<TSlot>(L.tab); e->tab.mask = c.table_capacity - 1;
   e->tab.shift = 64 - (bit_length(c.table_capacity) - 1);
   e->ent.key = e->dp<u64>(L.e_key); e->ent.stamp = e->dp<u32>(L.e_stamp); e->ent.depth = e->dp<u32>(L.e_depth);
-  e->ent.infl = e->dp<u32>(L.e_infl); e->ent.rank = e->dp<u32>(L.e_rank); e->ent.tslot = e->dp<u32>(L.e_tslot);
+  e->ent.infl = e->dp<u32>(L.e_infl); e->ent.cnt = e->dp<u64>(L.e_cnt); e->ent.tslot = e->dp<u32>(L.e_tslot);
   e->ent.mark = e->dp<u32>(L.e_mark); e->ent.floor = e->dp<u8>(L.e_floor); e->ent.link = e->dp<u32>(L.e_link);
   e->ent.n_hbm = c.n_hbm_blocks; e->ent.n_host = c.n_host_blocks; e->ent.n_total = (u32)N;
   e->d_keys = e->dp<u64>(L.keys); e->d_status = e->dp<u32>(L.status);
@@ -523,18 +716,23 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   e->ctxs.resize(c.max_contexts);
   e->tok_alloc.init(c.max_tokens, 64);
   e->key_alloc.init(c.max_key_blocks + c.max_key_blocks / CHUNK + 64ull * c.max_contexts, 32);
+  e->tbl_alloc.init(2ull * c.max_messages, 1);
   // pinned staging
   u64 C = c.max_contexts, Mm = c.max_messages, LB = L.LB;
-  u64 o_status = 0, o_desc = 256, o_ctxres = o_desc + round_up(C * 64 + 2 * (c.max_batch_blocks / CHUNK + C + 1) * 4, 256), o_ms = o_ctxres + round_up(C * 20, 256),
+  u64 o_status = 0, o_desc = 256, o_ctxres = o_desc + round_up(C * 256 + 2 * (c.max_batch_blocks / CHUNK + C + 1) * 4, 256), o_ms = o_ctxres + round_up(C * 20, 256),
       o_me = o_ms + round_up(Mm * 4, 256), o_mr = o_me + round_up(Mm * 4, 256), o_ids = o_mr + round_up(Mm, 256),
       o_ids2 = o_ids + round_up(LB * 4, 256), o_out = o_ids2 + round_up(LB * 4, 256),
-      total = o_out + round_up(LB * 16, 256);
+      o_sel = o_out + round_up(LB * 16, 256), total = o_sel + round_up(sizeof(SelArgs), 256);
   if (cudaHostAlloc((void **)&e->stage, total, cudaHostAllocDefault) != cudaSuccess) { delete e; return KVT_E_CUDA; }
   e->h_status = (u32 *)(e->stage + o_status); e->h_desc = e->stage + o_desc; e->h_ctxres = (u32 *)(e->stage + o_ctxres);
   e->h_mstart = (u32 *)(e->stage + o_ms); e->h_mend = (u32 *)(e->stage + o_me); e->h_mrank = e->stage + o_mr;
   e->h_ids = (u32 *)(e->stage + o_ids); e->h_ids2 = (u32 *)(e->stage + o_ids2); e->h_out = e->stage + o_out;
+  e->h_sel = (SelArgs *)(e->stage + o_sel);
   cudaStream_t s = (cudaStream_t)stream;
   if (cudaStreamCreateWithFlags(&e->capture_stream, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); e->use_graphs = false; }
+#ifdef KVT_TRACE
+  if (getenv("KVT_NO_GRAPH")) e->use_graphs = false;
+#endif
   bool ok = cudaEventCreateWithFlags(&e->ev_upload, cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreate(&e->ev_m0) == cudaSuccess && cudaEventCreate(&e->ev_m1) == cudaSuccess &&
             cudaEventCreate(&e->ev_h0) == cudaSuccess && cudaEventCreate(&e->ev_h1) == cudaSuccess;
@@ -554,7 +752,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
 int32_t kvt_destroy(kvt_engine *e) {
   if (!e) return KVT_E_INVAL;
   cudaDeviceSynchronize();
-  for (auto &g : e->sort_graph) if (g.exec) cudaGraphExecDestroy(g.exec);
+  for (auto &m : e->sel_graph) for (auto &g : m) if (g.second.exec) cudaGraphExecDestroy(g.second.exec);
   if (e->capture_stream) cudaStreamDestroy(e->capture_stream);
   if (e->ev_upload) cudaEventDestroy(e->ev_upload);
   if (e->ev_m0) cudaEventDestroy(e->ev_m0);
@@ -597,6 +795,18 @@ int32_t kvt_debug_set_lookup_variant(kvt_engine *e, uint32_t variant) {
   return KVT_OK;
 }
 
+int32_t kvt_debug_set_classify_mode(kvt_engine *e, uint32_t mode) {
+  if (!e || mode > 2) return KVT_E_INVAL;
+  e->classify_mode = mode;
+  return KVT_OK;
+}
+
+int32_t kvt_debug_set_wait_limit(kvt_engine *e, uint32_t polls) {
+  if (!e) return KVT_E_INVAL;
+  e->wait_limit = polls;
+  return KVT_OK;
+}
+
 int32_t kvt_get_stats(kvt_engine *e, kvt_stats *out) {
   if (!e || !out) return KVT_E_INVAL;
   kvt_stats s = e->st;
@@ -619,7 +829,6 @@ int32_t kvt_apply_op(kvt_engine *e, const kvt_op *op, void *stream) {
     if (id >= e->ctxs.size() || e->ctxs[id].live) return fail(e, KVT_E_INVAL, "spawn: context id out of range or in use");
     e->ctxs[id] = Ctx();
     e->ctxs[id].live = true;
-    e->dirty = true;
     return KVT_OK;
   }
   if (op->op == KVT_OP_FORK) {
@@ -646,6 +855,7 @@ int32_t kvt_apply_op(kvt_engine *e, const kvt_op *op, void *stream) {
     k.valid_blocks = std::min<u32>(Tm / 16, p->valid_blocks);
     if (k.mat_blocks && p->keyseg >= 0) { k.keyseg = p->keyseg; e->segs[p->keyseg].refs++; }  // equal prefixes, equal keys
     else { k.mat_blocks = 0; k.valid_blocks = 0; }
+    k.map_dirty = true;
     e->ctxs[id] = std::move(k);
     e->dirty = true;
     return KVT_OK;
@@ -661,15 +871,17 @@ int32_t kvt_apply_op(kvt_engine *e, const kvt_op *op, void *stream) {
       if (need > c->tok_cap) {
         u64 ncap = grow_cap(std::max<u64>(need, 2 * c->tok_cap)), noff;
         if (!e->tok_alloc.alloc(ncap, &noff)) return fail(e, KVT_E_NOSPACE, "token arena full");
-        if (c->tok_len) CU(cudaMemcpyAsync(e->d_tokens + noff, e->d_tokens + c->tok_off, c->tok_len * 4, cudaMemcpyDeviceToDevice, s));
+        int32_t r = copy_tokens_dd(e, s, noff, c->tok_off, c->tok_len);
+        if (!r) r = copy_tokens_in(e, s, noff + c->tok_len, op->tokens, op->n_tokens, on_dev);
+        if (r) { e->tok_alloc.release(noff, ncap); return r; }   // the context keeps its old buffer
         if (c->tok_cap) e->tok_alloc.release(c->tok_off, c->tok_cap);
         c->tok_off = noff; c->tok_cap = ncap;
+      } else {
+        int32_t r = copy_tokens_in(e, s, c->tok_off + c->tok_len, op->tokens, op->n_tokens, on_dev);
+        if (r) return r;
       }
-      int32_t r = copy_tokens_in(e, s, c->tok_off + c->tok_len, op->tokens, op->n_tokens, on_dev);
-      if (r) return r;
       c->tok_len = need;
-      c->msgs.push_back(Msg{op->n_tokens, (u8)(c->one_off ? MS_TEMPORARY : MS_ACTIVE)});
-      e->dirty = true;
+      c->msgs.push_back(Msg{op->n_tokens, (u8)(c->one_off ? MS_TEMPORARY : MS_ACTIVE)});   // no KV effect before the next call
       return KVT_OK;
     }
     case KVT_OP_REPLACE:
@@ -687,10 +899,10 @@ int32_t kvt_apply_op(kvt_engine *e, const kvt_op *op, void *stream) {
       } else {                                      // edit in the middle: rebuild the buffer elsewhere
         u64 ncap = grow_cap(new_len), noff;
         if (!e->tok_alloc.alloc(ncap, &noff)) return fail(e, KVT_E_NOSPACE, "token arena full");
-        if (t0) CU(cudaMemcpyAsync(e->d_tokens + noff, e->d_tokens + c->tok_off, t0 * 4, cudaMemcpyDeviceToDevice, s));
-        int32_t r = copy_tokens_in(e, s, noff + t0, op->tokens, (u32)nnew, on_dev);
-        if (r) return r;
-        if (tail) CU(cudaMemcpyAsync(e->d_tokens + noff + t0 + nnew, e->d_tokens + c->tok_off + t1, tail * 4, cudaMemcpyDeviceToDevice, s));
+        int32_t r = copy_tokens_dd(e, s, noff, c->tok_off, t0);
+        if (!r) r = copy_tokens_in(e, s, noff + t0, op->tokens, (u32)nnew, on_dev);
+        if (!r) r = copy_tokens_dd(e, s, noff + t0 + nnew, c->tok_off + t1, tail);
+        if (r) { e->tok_alloc.release(noff, ncap); return r; }   // the context keeps its old buffer
         if (c->tok_cap) e->tok_alloc.release(c->tok_off, c->tok_cap);
         c->tok_off = noff; c->tok_cap = ncap;
       }
@@ -703,6 +915,7 @@ int32_t kvt_apply_op(kvt_engine *e, const kvt_op *op, void *stream) {
       }
       c->msgs.erase(c->msgs.begin() + op->msg_start, c->msgs.begin() + op->msg_end);
       if (rep) c->msgs.insert(c->msgs.begin() + op->msg_start, Msg{op->n_tokens, (u8)(c->one_off ? MS_TEMPORARY : MS_ACTIVE)});
+      c->map_dirty = true;
       e->dirty = true;
       return KVT_OK;
     }
@@ -715,16 +928,19 @@ int32_t kvt_apply_op(kvt_engine *e, const kvt_op *op, void *stream) {
         if (!(op->msg_start < op->msg_end && op->msg_end <= c->msgs.size())) return fail(e, KVT_E_RANGE, "one_off: bad message range");
         for (u32 j = op->msg_start; j < op->msg_end; ++j) c->msgs[j].state = MS_TEMPORARY;
       }
+      c->map_dirty = true;
       e->dirty = true;
       return KVT_OK;
     }
     case KVT_OP_PREFILL_DONE: {
       if (!c->in_flight) return fail(e, KVT_E_STATE, "prefill_done: context is not in flight");
+      if (e->now == 0xFFFFFFFFu) return fail(e, KVT_E_NOSPACE, "logical clock exhausted");
       e->now += 1;
       int32_t r = unlock_held(e, *c, s, true);
       if (r) return r;
       for (Msg &m : c->msgs) if (m.state == MS_ACTIVE) m.state = MS_SUSPENDED;
       c->in_flight = false;
+      c->map_dirty = true;
       e->dirty = true;
       return KVT_OK;
     }
@@ -734,14 +950,14 @@ int32_t kvt_apply_op(kvt_engine *e, const kvt_op *op, void *stream) {
       c->tok_off = c->tok_cap = c->tok_len = 0;
       bool pinned = false;
       for (Msg &m : c->msgs) { if (m.state == MS_PINNED) pinned = true; else m.state = MS_EXPIRED; }
+      e->dirty = true;
       if (pinned) {            // Pinned messages retain their protection: keep the mapping, drop the rest
         c->terminated = true;
         c->in_flight = false;
+        c->map_dirty = true;
       } else {
-        seg_deref(e, c->keyseg);
-        *c = Ctx();
+        return retire_ctx(e, *c, s);
       }
-      e->dirty = true;
       return KVT_OK;
     }
     case KVT_OP_PIN:
@@ -756,8 +972,9 @@ int32_t kvt_apply_op(kvt_engine *e, const kvt_op *op, void *stream) {
       if (c->terminated) {
         bool pinned = false;
         for (const Msg &m : c->msgs) pinned = pinned || m.state == MS_PINNED;
-        if (!pinned) { seg_deref(e, c->keyseg); *c = Ctx(); }
+        if (!pinned) { e->dirty = true; return retire_ctx(e, *c, s); }
       }
+      c->map_dirty = true;
       e->dirty = true;
       return KVT_OK;
     }
@@ -776,13 +993,43 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     u64 nb = e->ctxs[ids[i]].tok_len / 16;
     if (!nb) continue;
     newseg[i] = seg_new(e, nb);
+    if (newseg[i] < 0 && e->dirty) {   // key lists that are only kept for the pending classification may be in the way
+      int32_t rc = do_classify(e, s);
+      if (rc) { for (u32 j = 0; j < i; ++j) seg_deref(e, newseg[j]); return rc; }
+      newseg[i] = seg_new(e, nb);
+    }
     if (newseg[i] < 0) {
       for (u32 j = 0; j < i; ++j) seg_deref(e, newseg[j]);
       return fail(e, KVT_E_NOSPACE, "key arena full");
     }
   }
   int32_t r = stage_acquire(e);
-  if (r) return r;
+  if (r) { for (int sg : newseg) seg_deref(e, sg); return r; }
+  // An error leaves the engine unchanged: the host-side changes below are made on the contexts themselves (the
+  // kernels need the new layout), with copies kept aside; a failure puts the copies back and gives the new key
+  // segments up. The old segments are only released once the call has succeeded. On the device, the kernels of a
+  // failed call have written nothing but scratch and the new segments (k_lock_hits does nothing once the error
+  // word is set).
+  if (e->now == 0xFFFFFFFFu) { for (int sg : newseg) seg_deref(e, sg); return fail(e, KVT_E_NOSPACE, "logical clock exhausted"); }
+  std::vector<Ctx> saved(n_ctx);
+  for (u32 i = 0; i < n_ctx; ++i) saved[i] = e->ctxs[ids[i]];
+  const u32 saved_now = e->now, saved_depth = e->max_depth;
+  const bool saved_dirty = e->dirty;
+  const u64 saved_rehashed = e->st.blocks_rehashed;
+  auto rollback = [&](int32_t code) {
+    for (u32 i = 0; i < n_ctx; ++i) e->ctxs[ids[i]] = std::move(saved[i]);
+    for (int sg : newseg) seg_deref(e, sg);
+    e->now = saved_now; e->max_depth = saved_depth; e->dirty = saved_dirty; e->st.blocks_rehashed = saved_rehashed;
+    return code;
+  };
+#define CUR(call)                                                                                  \
+  do {                                                                                             \
+    cudaError_t _e = (call);                                                                       \
+    if (_e != cudaSuccess) {                                                                       \
+      e->err = std::string(#call) + ": " + cudaGetErrorString(_e);                                 \
+      return rollback(KVT_E_CUDA);                                                                 \
+    }                                                                                              \
+  } while (0)
   e->now += 1;
   HashCtx *hd = reinterpret_cast<HashCtx *>(e->h_desc);
   std::vector<std::pair<u32, u32>> n_seq_chunks;   // per listed sequence: chunks in the all-blocks grid / in the digest grid
@@ -794,6 +1041,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     Ctx &c = e->ctxs[ids[i]];
     for (Msg &m : c.msgs) if (m.state == MS_SUSPENDED) m.state = MS_ACTIVE;  // reactivation (Section 5.2)
     c.in_flight = true;
+    c.map_dirty = true;
     c.mat_bounds.clear();
     u32 pos = 0;
     for (const Msg &m : c.msgs) { c.mat_bounds.push_back({pos, pos + m.len}); pos += m.len; }
@@ -807,8 +1055,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
       old_key_off = e->segs[c.keyseg].off;
       old_carry_off = old_key_off + e->segs[c.keyseg].keycap;
     }
-    seg_deref(e, c.keyseg);   // the old list stays readable for the kernels of this call (stream order)
-    c.keyseg = newseg[i];
+    c.keyseg = newseg[i];     // the old segment is released after the call has succeeded (it is read by this call's kernels)
     c.mat_blocks = c.valid_blocks = nb;
     e->max_depth = std::max(e->max_depth, nb);
     if (nb) {
@@ -840,11 +1087,11 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
         for (u32 j = 0; j < n_seq_chunks[q].second; ++j) h_dmap[dk++] = q;
       }
     }
-    CU(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nd * sizeof(HashCtx) + ((u64)chunk_base + dchunk_base) * 4, cudaMemcpyHostToDevice, s));
-    CU(cudaMemcpyAsync(d_res, h_hit, nd * 4, cudaMemcpyHostToDevice, s));
-    CU(cudaMemsetAsync(d_res + C, 0, 3ull * C * 4, s));
+    CUR(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nd * sizeof(HashCtx) + ((u64)chunk_base + dchunk_base) * 4, cudaMemcpyHostToDevice, s));
+    CUR(cudaMemcpyAsync(d_res, h_hit, nd * 4, cudaMemcpyHostToDevice, s));
+    CUR(cudaMemsetAsync(d_res + C, 0, 3ull * C * 4, s));
     r = status_zero(e, s);
-    if (r) return r;
+    if (r) return rollback(r);
     HashArgs ha;
     ha.tokens = e->d_tokens; ha.keys = e->d_keys; ha.carry_base = e->d_keys; ha.ctx = e->dp<HashCtx>(e->L.desc); ha.n_ctx = nd;
     ha.agg = e->dp<u64>(e->L.agg); ha.h0 = e->h0; ha.single = HashCtx{};
@@ -854,7 +1101,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     LockArgs lk;
     lk.ent = e->ent; lk.b_ent = la.b_ent; lk.hit_len = d_res; lk.n_hbm = d_res + C; lk.n_host = d_res + 2 * C; lk.n_remote = d_res + 3 * C;
     lk.now = e->now; lk.status = e->d_status;
-    if (e->profiling) CU(cudaEventRecord(e->ev_h0, s));
+    if (e->profiling) CUR(cudaEventRecord(e->ev_h0, s));
     if (e->lookup_variant != 2) {
       if (dchunk_base) KL(k_hash_digest, dchunk_base, CHUNK, s, ha);
       KL(k_hash_carry, nd, 1024, s, ha);
@@ -862,23 +1109,26 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     } else {
       ChainState cs;
       cs.flags = e->dp<u32>(e->L.cflags); cs.ticket = cs.flags + chunk_base; cs.incl = e->dp<u64>(e->L.carry);
-      cs.spin_limit = 1u << 18;   // x (one L2 round trip + 40 ns): far beyond any real wait, still bounded
-      CU(cudaMemsetAsync(cs.flags, 0, (chunk_base + 1) * 4ull, s));
+      cs.spin_limit = e->wait_limit;   // polls of (one L2 round trip + 40 ns): far beyond any real wait, still bounded
+      CUR(cudaMemsetAsync(cs.flags, 0, (chunk_base + 1) * 4ull, s));
       KL(k_hash_lookup_fused, chunk_base, CHUNK, s, ha, la, cs);
     }
     KL(k_lock_hits, chunk_base, CHUNK, s, ha, lk);
-    if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));
-    LAUNCH_CHECK();
-    CU(cudaMemcpyAsync(h_hit, d_res, 4ull * C * 4, cudaMemcpyDeviceToHost, s));
+    if (e->profiling) CUR(cudaEventRecord(e->ev_h1, s));
+    r = launch_ok(e);
+    if (r) return rollback(r);
+    CUR(cudaMemcpyAsync(h_hit, d_res, 4ull * C * 4, cudaMemcpyDeviceToHost, s));
     r = status_fetch(e, s);
-    if (r) return r;
+    if (r) return rollback(r);
     if (e->profiling) {
       float ms = 0.f;
       if (cudaEventElapsedTime(&ms, e->ev_h0, e->ev_h1) == cudaSuccess) { e->st.lookup_ns += (u64)((double)ms * 1e6); e->st.lookup_blocks += blk_base; }
     }
     r = status_code(e);
-    if (r) return r;
+    if (r) return rollback(r);
   }
+#undef CUR
+  for (u32 i = 0; i < n_ctx; ++i) seg_deref(e, saved[i].keyseg);
   for (u32 i = 0; i < n_ctx; ++i) {
     Ctx &c = e->ctxs[ids[i]];
     int k = dev_idx[i];
@@ -949,6 +1199,8 @@ static int32_t map_admit(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_info
     a.cslot = e->dp<u32>(e->L.s0); a.flag = e->dp<u32>(e->L.s1); a.aux = e->dp<u32>(e->L.s2); a.krank = e->dp<u32>(e->L.s3);
     a.freelist = e->dp<u32>(e->L.freelist); a.n_free = n_free; a.stop = e->dp<u32>(e->L.ctxres) + 4 * C;
     a.now = e->now; a.status = e->d_status;
+    a.fresh = e->dp<u32>(e->L.fresh); a.fresh_base = e->n_fresh;
+    if ((u64)e->n_fresh + n_free > e->ent.n_total) { rc = fail(e, KVT_E_DEVICE, "list of new entries would overflow"); break; }
     CU(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nd * sizeof(AdmitCtx), cudaMemcpyHostToDevice, s));
     CU(cudaMemcpyAsync(a.stop, h_stop, nd * 4, cudaMemcpyHostToDevice, s));
     rc = status_zero(e, s);
@@ -970,6 +1222,7 @@ static int32_t map_admit(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_info
     rc = status_code(e);
     if (rc) break;
     e->occ[0] += e->h_status[ST_INSERTED];
+    e->n_fresh += e->h_status[ST_INSERTED];
     e->tombs += e->h_status[ST_TOMBS];
     e->st.inserted += e->h_status[ST_INSERTED];
     e->st.adopted += e->h_status[ST_ADOPTED];
@@ -1043,7 +1296,7 @@ int32_t kvt_get_block_map(kvt_engine *e, uint32_t ctx, uint64_t *keys, uint8_t *
 // ---- stage 3 -----------------------------------------------------------------------------------------------
 int32_t kvt_classify(kvt_engine *e, void *stream) {
   if (!e) return KVT_E_INVAL;
-  return do_classify(e, (cudaStream_t)stream);
+  return (e->dirty || e->classify_mode == 1) ? do_classify(e, (cudaStream_t)stream) : KVT_OK;
 }
 
 int32_t kvt_get_states(kvt_engine *e, uint32_t tier, uint8_t *state, uint32_t cap, void *stream) {
@@ -1092,61 +1345,98 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   if (r) return r;
   r = status_zero(e, s);
   if (r) return r;
-  SelArgs a;
+  int32_t rr = stage_acquire(e);
+  if (rr) return rr;
+  SelArgs &a = *e->h_sel;   // pinned staging: uploaded below, read by every kernel of the sequence
+  a = SelArgs{};
   a.ent = e->ent; a.e0 = e->tier_e0(tier); a.n_slots = n; a.n_req = n_req; a.now = e->now;
   a.stamp_bits = bit_length(e->now); a.depth_bits = bit_length(e->max_depth);
   a.mru = e->cfg.suspended_order == KVT_ORDER_MRU; a.status = e->d_status;
   a.max_rank = (flags & KVT_SEL_INCLUDE_PINNED) ? 3 : 2;
   a.one_tier = (e->cfg.policy_flags & KVT_POLICY_NO_LIFECYCLE) ? 1 : 0;
   a.copy_bit = (tier == KVT_TIER_HOST && (e->cfg.policy_flags & KVT_POLICY_INCLUSIVE)) ? 1 : 0;
+  const u32 key_bits = 2 + a.copy_bit + a.stamp_bits + a.depth_bits;
+  if (key_bits > 63) return fail(e, KVT_E_INVAL, "select: stamps and depths this large do not fit the 63-bit victim key");
+  // composite = (key << slot_bits) | slot, searched most significant digit first: 11 bits, then 13 at a time
+  a.slot_bits = bit_length(n - 1);
+  {
+    u32 left = key_bits + a.slot_bits, lev = 0;
+    while (left) {
+      const u32 w = std::min(left, lev == 0 ? SEL_W0 : SEL_WN);
+      left -= w;
+      a.lev_lo[lev] = (u8)left; a.lev_w[lev] = (u8)w;
+      ++lev;
+    }
+    a.n_levels = lev;
+  }
   u64 *kA = e->dp<u64>(e->L.keyA), *kB = e->dp<u64>(e->L.keyB);
   u32 *vA = e->dp<u32>(e->L.valA), *vB = e->dp<u32>(e->L.valB), *counts = e->dp<u32>(e->L.rcounts);
-  u32 *row_total = counts + 256ull * (e->L.Nt / SORT_TILE + 1);
+  u32 *row_total = counts + (u64)RADIX_BINS * (e->L.Nt / SORT_TILE + 1);
+  a.slot_key = e->dp<u64>(e->L.slot_key); a.hist = e->dp<u32>(e->L.sel_hist); a.state = e->dp<SelState>(e->L.sel_state);
+  a.cta_count = e->dp<u32>(e->L.sel_cta);
+  a.pair_key = kA; a.pair_val = vA;
+  const u32 n_emit = std::min(n_req, n);
+  const u32 m_max = (u32)std::min<u64>((u64)n_emit + SEL_SLACK, n);   // the gathered set never exceeds this
+  a.n_emit = n_emit; a.rank_shift = a.stamp_bits + a.depth_bits;
+  a.slots_out = e->dp<u32>(e->L.out_slots); a.states_out = e->dp<u8>(e->L.out_states);
+  const SelArgs *d_args = e->dp<SelArgs>(e->L.sel_args);
+  CU(cudaMemcpyAsync((void *)d_args, &a, sizeof(SelArgs), cudaMemcpyHostToDevice, s));
+  rr = stage_release(e, s);
+  if (rr) return rr;
+  const u32 n_levels = a.n_levels, n_pass = cdiv(key_bits, RADIX_BITS);
+  // sort grids cover the bound of the gathered set rounded up to a power of two of tiles (few distinct graphs)
+  u32 tiles = 1;
+  while (tiles < cdiv(m_max, SORT_TILE)) tiles *= 2;
+  const u32 g = cdiv(n, SEL_TILE);
+  // The sequence below is short kernels with fixed grids and buffers whose arguments all live in device memory,
+  // i.e. launch-bound: it is captured once per (tier, level count, pass count) into a CUDA graph on a private
+  // stream and replayed on the caller's stream with one launch.
+  auto enqueue = [&](cudaStream_t q, bool count) {
+    if (count) TRACE(q, "start");
+    cudaMemsetAsync(a.hist, 0, (u64)n_levels * SEL_BINS * 4, q);
+    if (count) TRACE(q, "memset");
+    k_sel_keys<<<g, SEL_CTA, 0, q>>>(d_args);
+    if (count) TRACE(q, "keys");
+    for (u32 lev = 1; lev < n_levels; ++lev) { k_sel_level<<<g, SEL_CTA, 0, q>>>(d_args, lev); if (count) TRACE(q, "level"); }
+    k_sel_count<<<g, SEL_CTA, 0, q>>>(d_args);
+    if (count) TRACE(q, "count");
+    k_sel_gather<<<g, SEL_CTA, 0, q>>>(d_args);
+    if (count) TRACE(q, "gather");
+    u64 *ka = kA, *kb = kB; u32 *va = vA, *vb = vB;
+    for (u32 p = 0; p < n_pass; ++p) {
+      k_radix_hist<<<tiles, 256, 0, q>>>(ka, e->d_status, RADIX_BITS * p, counts);
+      if (count) TRACE(q, "hist");
+      k_radix_scan<<<RADIX_BINS / 8, 256, 0, q>>>(counts, row_total, e->d_status);
+      if (count) TRACE(q, "scan");
+      k_radix_scatter<<<tiles, 256, 0, q>>>(ka, va, kb, vb, e->d_status, RADIX_BITS * p, counts, row_total);
+      if (count) TRACE(q, "scatter");
+      std::swap(ka, kb); std::swap(va, vb);
+    }
+    k_sel_emit<<<std::min<u32>(cdiv(n, 256), (u32)e->sm_count * 8), 256, 0, q>>>(d_args, ka, va);
+    if (count) TRACE(q, "emit");
+    if (count) e->st.kernel_launches += 3ull + (n_levels - 1) + 3ull * n_pass + 1;
+  };
   if (e->profiling) CU(cudaEventRecord(e->ev_h0, s));
-  KL(k_sel_count, cdiv(n,256), 256, s, a);
-  r = compact_indices(e, s, PredSel{a}, EmitSel{a, kA, vA}, n, ST_M);
-  if (r) return r;
-  const u32 key_bits = 2 + a.copy_bit + a.stamp_bits + a.depth_bits, n_pass = cdiv(key_bits, 8), tiles = cdiv(n, SORT_TILE);
-  // The radix passes are a fixed sequence of short kernels (same buffers, same grids, element count read from
-  // the status block), i.e. launch-bound: they are captured once per (tier, pass count) into a CUDA graph on a
-  // private capture stream and replayed on the caller's stream with one launch.
   {
-    kvt_engine::SortGraph &g = e->sort_graph[tier];
-    if (e->use_graphs && (!g.exec || g.n_pass != n_pass)) {
-      if (g.exec) { cudaGraphExecDestroy(g.exec); g.exec = nullptr; }
+    kvt_engine::SelGraph &gr = e->sel_graph[tier][(u64)n_levels << 48 | (u64)n_pass << 32 | tiles];
+    if (e->use_graphs && !gr.exec) {
       cudaGraph_t graph = nullptr;
       bool ok = cudaStreamBeginCapture(e->capture_stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess;
       if (ok) {
-        u64 *ka = kA, *kb = kB; u32 *va = vA, *vb = vB;
-        for (u32 p = 0; p < n_pass; ++p) {
-          k_radix_hist<<<tiles, 256, 0, e->capture_stream>>>(ka, e->d_status, 8 * p, counts);
-          k_radix_scan<<<32, 256, 0, e->capture_stream>>>(counts, row_total, e->d_status);
-          k_radix_scatter<<<tiles, 256, 0, e->capture_stream>>>(ka, va, kb, vb, e->d_status, 8 * p, counts, row_total);
-          std::swap(ka, kb); std::swap(va, vb);
-        }
+        enqueue(e->capture_stream, false);
         ok = cudaStreamEndCapture(e->capture_stream, &graph) == cudaSuccess && graph;
       }
-      if (ok) ok = cudaGraphInstantiate(&g.exec, graph, 0) == cudaSuccess;
+      if (ok) ok = cudaGraphInstantiate(&gr.exec, graph, 0) == cudaSuccess;
       if (graph) cudaGraphDestroy(graph);
-      if (!ok) { cudaGetLastError(); g.exec = nullptr; e->use_graphs = false; }   // fall back to plain launches
-      g.n_pass = n_pass;
+      if (!ok) { cudaGetLastError(); gr.exec = nullptr; e->use_graphs = false; }   // fall back to plain launches
     }
-    if (e->use_graphs && g.exec) {
-      CU(cudaGraphLaunch(g.exec, s));
-      e->st.kernel_launches += 3ull * n_pass;
-      if (n_pass & 1) { std::swap(kA, kB); std::swap(vA, vB); }
+    if (e->use_graphs && gr.exec) {
+      CU(cudaGraphLaunch(gr.exec, s));
+      e->st.kernel_launches += 3ull + (n_levels - 1) + 3ull * n_pass + 1;
     } else {
-      for (u32 p = 0; p < n_pass; ++p) {
-        KL(k_radix_hist, tiles, 256, s, kA, e->d_status, 8 * p, counts);
-        KL(k_radix_scan, 32, 256, s, counts, row_total, e->d_status);
-        KL(k_radix_scatter, tiles, 256, s, kA, vA, kB, vB, e->d_status, 8 * p, counts, row_total);
-        std::swap(kA, kB); std::swap(vA, vB);
-      }
+      enqueue(s, true);
     }
   }
-  u32 n_emit = std::min(n_req, n);
-  KL(k_sel_emit, cdiv(n_emit,256), 256, s, e->ent, a.e0, n, kA, vA, n_emit, e->d_status, a.stamp_bits + a.depth_bits, a.copy_bit, e->dp<u32>(e->L.out_slots),
-                                               e->dp<u8>(e->L.out_states));
   if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));
   LAUNCH_CHECK();
   // the victim list (at most n_emit entries) travels with the status block: one synchronisation
@@ -1155,15 +1445,17 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   if (states_out) CU(cudaMemcpyAsync(h_states, e->dp<u8>(e->L.out_states), n_emit, cudaMemcpyDeviceToHost, s));
   r = status_fetch(e, s);
   if (r) return r;
+  TRACE_DUMP("select");
   if (e->profiling) {
     float ms = 0.f;
     if (cudaEventElapsedTime(&ms, e->ev_h0, e->ev_h1) == cudaSuccess) { e->st.select_ns += (u64)((double)ms * 1e6); e->st.select_slots += n; }
   }
   r = status_code(e);
   if (r) return r;
-  u64 total = (u64)e->h_status[ST_RANK0] + e->h_status[ST_RANK1] + e->h_status[ST_RANK2] + e->h_status[ST_RANK3] +
-              e->h_status[ST_SHADOW];
-  u32 k = (u32)std::min<u64>(n_req, total);
+  const u32 total = e->h_status[ST_TOTAL];   // candidates of the tier
+  if (e->h_status[ST_M] != e->h_status[ST_AUX] || e->h_status[ST_M] > m_max || e->h_status[ST_M] < std::min(n_req, total))
+    return fail(e, KVT_E_DEVICE, "selection: gathered set does not match its histogram");
+  u32 k = std::min(n_req, total);
   *n_out = k;
   if (cap < k) return KVT_E_BUFSZ;
   if (k) {
@@ -1185,7 +1477,8 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
   if (n > e->L.LB) return fail(e, KVT_E_NOSPACE, "list longer than max_batch_blocks");
   int32_t r = stage_acquire(e);
   if (r) return r;
-  if (m.drop_dead) { r = ensure_classified(e, s); if (r) return r; r = stage_acquire(e); if (r) return r; }
+  // the mapping counts are brought up to date before any entry moves or goes away (the pending updates name entries)
+  r = ensure_classified(e, s); if (r) return r; r = stage_acquire(e); if (r) return r;
   std::memcpy(e->h_ids, slots, n * 4ull);
   u32 *d_ids = e->dp<u32>(e->L.ids);
   CU(cudaMemcpyAsync(d_ids, e->h_ids, n * 4ull, cudaMemcpyHostToDevice, s));
@@ -1431,7 +1724,9 @@ int32_t kvt_compact(kvt_engine *e, uint32_t tier, uint32_t *n_moved, void *strea
   cudaStream_t s = (cudaStream_t)stream;
   u32 n = e->tier_slots(tier), e0 = e->tier_e0(tier), n_occ = e->occ[tier];
   if (!n || !n_occ || n_occ == n) return KVT_OK;
-  int32_t r = status_zero(e, s);
+  int32_t r = ensure_classified(e, s);   // before entries move
+  if (r) return r;
+  r = status_zero(e, s);
   if (r) return r;
   u32 *src = e->dp<u32>(e->L.pair_src), *dst = e->dp<u32>(e->L.pair_dst);
   r = compact_indices(e, s, PredHole{e->ent.key, e0, n_occ}, EmitList{dst}, n, ST_AUX);
@@ -1505,11 +1800,10 @@ int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t ha
 
 // ---- hasher without allocation ------------------------------------------------------------------------------
 // Scratch of the no-allocation hasher: chunk aggregates followed by chunk carries. File-scope device
-// memory: in host code this name is only a handle, so its device address is queried once per device
-// below and that pointer is what the kernels get.
+// memory: in host code this name is only a handle, so its device address is queried below (with the
+// caller's device current) and that pointer is what the kernels get.
 constexpr u64 NOALLOC_MAX_CHUNKS = KVT_HASH_NOALLOC_MAX_TOKENS / 16 / CHUNK;
 static __device__ __align__(256) unsigned long long g_noalloc_scratch[2 * NOALLOC_MAX_CHUNKS + 1];
-static u64 *g_noalloc_ptr[64] = {};   // per device ordinal
 
 int32_t kvt_hash_tokens_noalloc(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t hash_seed, uint64_t *d_keys,
                                 void *stream) {
@@ -1517,20 +1811,19 @@ int32_t kvt_hash_tokens_noalloc(const uint32_t *d_tokens, uint64_t n_tokens, uin
   u64 nb = n_tokens / 16;
   if (nb == 0) return KVT_OK;
   if (!d_tokens || !d_keys || ((uintptr_t)d_tokens & 15)) return KVT_E_INVAL;
-  int dev = -1;
-  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return KVT_E_CUDA;
-  if (!g_noalloc_ptr[dev]) {   // first call on this device: resolve the array's device address
-    void *p = nullptr;
-    if (cudaGetSymbolAddress(&p, g_noalloc_scratch) != cudaSuccess || !p) return KVT_E_CUDA;
-    g_noalloc_ptr[dev] = (u64 *)p;
-  }
+  // The array's address on the current device. Asked for on every call: after the first call on a device (which
+  // makes the runtime load this module there) it is a look-up, and nothing cached here can go stale when a device's
+  // context is reset or be raced for by two host threads.
+  void *sym = nullptr;
+  if (cudaGetSymbolAddress(&sym, g_noalloc_scratch) != cudaSuccess || !sym) return KVT_E_CUDA;
+  u64 *const scratch = (u64 *)sym;
   cudaStream_t s = (cudaStream_t)stream;
   u32 n_chunks = cdiv(nb, CHUNK);
   HashArgs ha;
   ha.tokens = d_tokens; ha.keys = d_keys; ha.ctx = nullptr; ha.n_ctx = 1; ha.chunk_ctx = ha.dchunk_ctx = nullptr;
   ha.single = HashCtx{};
   ha.single.n_blocks = (u32)nb;
-  ha.agg = g_noalloc_ptr[dev]; ha.carry_base = g_noalloc_ptr[dev] + NOALLOC_MAX_CHUNKS; ha.h0 = hash_h0(hash_seed);
+  ha.agg = scratch; ha.carry_base = scratch + NOALLOC_MAX_CHUNKS; ha.h0 = hash_h0(hash_seed);
   LookupArgs la{};
   k_hash_digest<<<n_chunks, CHUNK, 0, s>>>(ha);
   k_hash_carry<<<1, 1024, 0, s>>>(ha);
@@ -1560,6 +1853,9 @@ int32_t kvt_debug_load_resident(kvt_engine *e, const uint64_t *keys, const uint8
     }
   }
   if ((u64)e->occ[0] + e->occ[1] + e->occ[2] + e->tombs + n > ((u64)e->tab.mask + 1) * 3 / 4) return fail(e, KVT_E_NOSPACE, "table too full");
+  // the victim key packs rank, recency and depth into 63 bits: stamps and depths that would not fit are refused here
+  if (3 + bit_length(std::max(e->now, max_stamp)) + bit_length(std::max(e->max_depth, max_d)) > 63)
+    return fail(e, KVT_E_INVAL, "stamp and depth too large for the victim key");
   cudaStream_t s = (cudaStream_t)stream;
   // stage the arrays in scratch: keys -> keyA, state -> out_states, stamp/depth/slot -> s1/s2/s3
   u64 *dk = e->dp<u64>(e->L.keyA);
@@ -1583,6 +1879,7 @@ int32_t kvt_debug_load_resident(kvt_engine *e, const uint64_t *keys, const uint8
   r = status_code(e);
   if (r) return r;
   e->occ[tier] += n;
+  for (const Ctx &c : e->ctxs) if (c.live) { e->full_dirty = e->dirty = true; break; }   // existing contexts may map the new keys
   e->now = std::max(e->now, max_stamp);
   e->max_depth = std::max(e->max_depth, max_d);
   return KVT_OK;

@@ -21,8 +21,6 @@ constexpr u32 ENT_NONE = 0xFFFFFFFFu;
 constexpr u32 CLAIM_BIT = 0x80000000u;
 constexpr u32 CHUNK = 256;        // blocks hashed by one CTA
 constexpr u32 SCAN_TILE = 1024;   // items per CTA in the ordered-compaction kernels
-constexpr u32 SORT_TILE = 1024;   // items per CTA in the radix-sort kernels (8 warps x 128): small tiles keep all SMs busy
-constexpr int SORT_ITERS = SORT_TILE / 256;   // items per thread
 
 // bits of the device error word
 enum : u32 { DERR_PROBE = 1, DERR_RANGE = 2, DERR_INVAL = 4, DERR_STATE = 8, DERR_CORRUPT = 16, DERR_WAIT = 32 };
@@ -33,6 +31,7 @@ enum : int {
   ST_RANK0, ST_RANK1, ST_RANK2, ST_RANK3, ST_M, ST_NMOVED, ST_FREE, ST_AUX, ST_SHADOW, ST_NCLEAN, ST_NSHDROP,
   ST_B_CUT, ST_B_NLIVE, ST_B_NDROP, ST_B_NCLEAN, ST_B_NSHDROP, ST_B_TOTAL, ST_B_FREE,   // second list of an exchange
   ST_QA, ST_QB,                                                                          // work queues of its mover
+  ST_CHK,                                                                                // cross-check of the mapping counts
   ST_WORDS = 32
 };
 
@@ -69,11 +68,24 @@ struct Table { TSlot *slots; u32 mask; u32 shift; };   // capacity = mask + 1, h
 
 struct Entries {            // per resident-block metadata, entry id = slot (HBM), n_hbm + slot (host) or n_hbm + n_host + slot (remote)
   u64 *key;                 // 0 = free
-  u32 *stamp, *depth, *infl, *rank, *tslot, *mark;
+  u32 *stamp, *depth, *infl, *tslot, *mark;
+  u64 *cnt;                 // mappings per rank: three 21-bit fields (Suspended, Active, Pinned), see entry_rank()
   u32 *link;                // inclusive tiering: an HBM block and its clean host copy point at each other (else ENT_NONE)
   u8 *floor;
   u32 n_hbm, n_host, n_total;
 };
+
+// KV-level state of a resident block (Section 6.1): the highest-priority state over all (context, message version)
+// mappings of its key, dead when there is none. cnt[e] counts the mappings per rank, so the state is the highest
+// rank with a non-zero count (or the floor installed by the debug loader, whichever is higher).
+constexpr u32 CNT_BITS = 21;
+constexpr u64 CNT_MASK = (1ull << CNT_BITS) - 1;
+__host__ __device__ __forceinline__ u64 cnt_unit(u32 rank) { return rank ? 1ull << (CNT_BITS * (rank - 1)) : 0ull; }
+__device__ __forceinline__ u32 rank_of(u64 cnt, u32 floor) {
+  const u32 r = (cnt >> (2 * CNT_BITS)) ? 3u : ((cnt >> CNT_BITS) & CNT_MASK) ? 2u : (cnt & CNT_MASK) ? 1u : 0u;
+  return max(r, floor);
+}
+__device__ __forceinline__ u32 entry_rank(const Entries &en, u32 e) { return rank_of(en.cnt[e], en.floor[e]); }
 
 // A host entry that only holds a clean copy of a block whose home is in HBM.
 __device__ __forceinline__ bool is_shadow(const Entries &en, u32 e) { return e >= en.n_hbm && en.link[e] != ENT_NONE; }
@@ -441,15 +453,14 @@ __global__ void __launch_bounds__(CHUNK) k_hash_lookup_fused(HashArgs a, LookupA
         while (true) {
           const int k = k_hi - (int)lane;
           u64 m = 1, ad = 0;
-          u32 f = 2;
           const bool mine_k = k >= (int)g0;
           const u32 idx = c.chunk_base + (u32)(mine_k ? k : 0);
-          u32 it = 0;
-          do {
+          u32 f = mine_k ? 0u : 2u;   // nothing seen yet
+          for (u32 it = 0; it < cs.spin_limit; ++it) {   // bounded: a limit of 0 gives up without looking
             f = mine_k ? ld_acquire_u32(cs.flags + idx) : 2u;
             if (!__any_sync(0xFFFFFFFFu, f == 0)) break;
             __nanosleep(40);
-          } while (++it < cs.spin_limit);
+          }
           if (mine_k) {
             if (f == 2) { m = 0; ad = __ldcg(cs.incl + idx); }
             else if (f == 1) { m = A; ad = __ldcg(a.agg + idx); }
@@ -506,6 +517,11 @@ __global__ void __launch_bounds__(CHUNK) k_lock_hits(HashArgs a, LockArgs l) {
   const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci);
   const u32 b = (blockIdx.x - c.chunk_base) * CHUNK + tid;
   u32 tier = 3;   // none
+  // the hash / probe kernels failed: the call changes nothing. One read per CTA, so that the whole CTA agrees.
+  __shared__ u32 s_err;
+  if (tid == 0) s_err = l.status[ST_ERR];
+  __syncthreads();
+  if (s_err) return;
   if (b < l.hit_len[ci]) {
     u32 e = l.b_ent[c.blk_base + b];
     if (e >= l.ent.n_total) set_err(l.status, DERR_CORRUPT);
@@ -627,6 +643,7 @@ struct AdmitArgs {
   Table tab; Entries ent; const u64 *keys; const AdmitCtx *ctx; u32 n_ctx; u32 n_cand;
   u32 *cslot, *flag, *aux, *krank;   // per candidate scratch
   const u32 *freelist; u32 n_free;   // lowest free HBM slots, ascending; n_free = free HBM slots
+  u32 *fresh; u32 fresh_base;         // list of the entries created since the mapping counts were last brought up to date
   u32 *stop;                          // per context (indexed by AdmitCtx.res)
   u32 now; u32 *status;
 };
@@ -712,10 +729,10 @@ __global__ void k_admit_apply(AdmitArgs a) {
     if (held) {
       u32 e = a.freelist[a.krank[g]];
       a.ent.key[e] = a.keys[c.key_off + b];
-      a.ent.stamp[e] = a.now; a.ent.depth[e] = b; a.ent.rank[e] = 2; a.ent.floor[e] = 0; a.ent.tslot[e] = s; a.ent.link[e] = ENT_NONE;
+      a.ent.stamp[e] = a.now; a.ent.depth[e] = b; a.ent.cnt[e] = 0; a.ent.floor[e] = 0; a.ent.tslot[e] = s; a.ent.link[e] = ENT_NONE;
       atomicAdd(&a.ent.infl[e], 1u);
       a.tab.slots[s].ent = e;
-      atomicAdd(&a.status[ST_INSERTED], 1u);
+      a.fresh[a.fresh_base + atomicAdd(&a.status[ST_INSERTED], 1u)] = e;
     } else {
       a.tab.slots[s].key = KEY_TOMB;
       a.tab.slots[s].ent = ENT_NONE;
@@ -750,20 +767,47 @@ __global__ void k_block_map(Table t, Entries en, const u64 *keys, u32 n, u8 *tie
 }
 
 // ======================================================================================================
-// K3: classifier. rank[e] = max(floor[e], max over mappings (context, block) of the block's rank), where a
-// block's rank under a context is the highest message rank over the messages whose token span touches it.
+// K3: classifier (Section 6.1). The engine keeps, per resident block, how many (context, block) mappings of each
+// rank point at its key (Entries.cnt); the block's state is read off those counts. A mapping's rank is the highest
+// message rank over the messages whose token span touches the block. The counts are updated by events, not
+// recomputed: for every context whose messages, mapped prefix or key list changed since it was last accounted
+// for, one thread per block takes the old contribution away and adds the new one (k_map_delta); keys that entered
+// the table since then receive the contributions of every context that already mapped them (k_run_filter /
+// k_run_fixup). The full recomputation is the same delta kernel run from zero counts over all contexts.
 // ======================================================================================================
-struct ClsCtx { u64 key_off; u32 map_base; u32 valid; u32 msg_base; u32 n_msgs; };
-struct ClsArgs {
-  Table tab; Entries ent; const u64 *keys; const ClsCtx *ctx; u32 n_ctx; u32 n_map;
-  const u32 *m_start, *m_end; const u8 *m_rank; u32 *status;
+struct MsgTables { const u32 *start, *end; const u8 *rank; };   // message spans of all accounted-for contexts, by offset
+
+// Rank of block b under a message table slice [off, off + n): highest rank over the messages touching tokens [16 b, 16 b + 16).
+__device__ __forceinline__ u32 block_rank(const MsgTables &t, u32 off, u32 n, u32 b) {
+  const u32 t0 = b * 16, t1 = t0 + 16;
+  const u32 *ms = t.start + off, *me = t.end + off;
+  const u8 *mr = t.rank + off;
+  u32 l = 0, h = n;   // first message whose end is beyond t0 (ends are non-decreasing)
+  while (l < h) { const u32 mid = (l + h) >> 1; if (me[mid] > t0) h = mid; else l = mid + 1; }
+  u32 r = 0;
+  for (u32 j = l; j < n && ms[j] < t1; ++j)
+    if (me[j] > ms[j] && mr[j] > r) r = mr[j];
+  return r;
+}
+
+// One context of a delta pass: what was accounted for (old) and what holds now (new).
+struct DeltaCtx {
+  u64 old_key_off, new_key_off;        // key lists (u64 index into keys)
+  u32 old_valid, new_valid;            // mapped prefix lengths
+  u32 old_tbl, old_n, new_tbl, new_n;  // message table slices
+  u32 map_base;                        // first item of this context in the flattened (context, block) index space
+  u32 pad;
+};
+struct DeltaArgs {
+  Table tab; Entries ent; const u64 *keys; const DeltaCtx *ctx; u32 n_ctx; u32 n_map;
+  MsgTables tbl; u32 *status;
   u32 *first_miss;   // per listed context: index of its first non-resident block; nullptr = orphans keep their state
 };
 
-// Context that owns mapping g (the last one whose map_base is <= g). Every thread of the CTA calls it: the
+// Context that owns item g (the last one whose map_base is <= g). Every thread of the CTA calls it: the
 // bases are staged in shared memory by one round of loads when they fit.
 constexpr u32 CTX_STAGE = 1024;
-__device__ __forceinline__ u32 cls_ctx_of_mapping(const ClsArgs &a, u32 g) {
+__device__ __forceinline__ u32 delta_ctx_of_item(const DeltaArgs &a, u32 g) {
   __shared__ u32 s_base[CTX_STAGE];
   const bool staged = a.n_ctx <= CTX_STAGE;
   if (staged) {
@@ -778,136 +822,387 @@ __device__ __forceinline__ u32 cls_ctx_of_mapping(const ClsArgs &a, u32 g) {
   return lo;
 }
 
-__global__ void k_rank_reset(Entries en) {
-  u32 e = blockIdx.x * blockDim.x + threadIdx.x;
-  if (e < en.n_total) en.rank[e] = en.floor[e];
+// Reachability pre-pass of the full recomputation: the first block of every context's mapped prefix that is resident
+// in no tier. A lookup stops there, so the blocks behind it cannot be reused through this context.
+__global__ void k_first_miss(DeltaArgs a) {
+  u32 g = blockIdx.x * blockDim.x + threadIdx.x;
+  const u32 lo = delta_ctx_of_item(a, g);
+  if (g >= a.n_map) return;
+  const DeltaCtx c = a.ctx[lo];
+  const u32 b = g - c.map_base;
+  if (b >= c.new_valid) return;
+  if (tab_lookup_ent(a.tab, a.keys[c.new_key_off + b], a.status) == ENT_NONE) atomicMin(&a.first_miss[lo], b);
 }
 
-// Reachability pre-pass: the first block of every context's mapped prefix that is resident in no tier. A lookup
-// stops there, so the blocks behind it cannot be reused through this context.
-__global__ void k_first_miss(ClsArgs a) {
-  u32 g = blockIdx.x * blockDim.x + threadIdx.x;
-  const u32 lo = cls_ctx_of_mapping(a, g);
-  if (g >= a.n_map) return;
-  const ClsCtx c = a.ctx[lo];
-  const u32 b = g - c.map_base;
-  if (tab_lookup_ent(a.tab, a.keys[c.key_off + b], a.status) == ENT_NONE) atomicMin(&a.first_miss[lo], b);
+__device__ __forceinline__ void cnt_add(const DeltaArgs &a, u64 key, u64 delta) {
+  const u32 e = tab_lookup_ent(a.tab, key, a.status);   // ENT_NONE: mapped but not resident
+  if (e < a.ent.n_total) atomicAdd((unsigned long long *)&a.ent.cnt[e], (unsigned long long)delta);
 }
 
-__global__ void k_classify(ClsArgs a) {
+__global__ void k_map_delta(DeltaArgs a) {
   u32 g = blockIdx.x * blockDim.x + threadIdx.x;
-  const u32 lo = cls_ctx_of_mapping(a, g);
+  const u32 lo = delta_ctx_of_item(a, g);
   if (g >= a.n_map) return;
-  const ClsCtx c = a.ctx[lo];
+  const DeltaCtx c = a.ctx[lo];
   const u32 b = g - c.map_base;
-  if (a.first_miss && b >= a.first_miss[lo]) return;   // behind a missing block: unreachable through this context
-  const u32 t0 = b * 16, t1 = t0 + 16;
-  const u32 *ms = a.m_start + c.msg_base, *me = a.m_end + c.msg_base;
-  const u8 *mr = a.m_rank + c.msg_base;
-  // first message whose end is beyond t0 (ends are non-decreasing)
-  u32 l = 0, h = c.n_msgs;
-  while (l < h) { u32 mid = (l + h) >> 1; if (me[mid] > t0) h = mid; else l = mid + 1; }
-  u32 r = 0;
-  for (u32 j = l; j < c.n_msgs && ms[j] < t1; ++j)
-    if (me[j] > ms[j] && mr[j] > r) r = mr[j];
-  if (r == 0) return;
-  u32 e = tab_lookup_ent(a.tab, a.keys[c.key_off + b], a.status);   // ENT_NONE: mapped but not resident
-  if (e < a.ent.n_total) atomicMax(&a.ent.rank[e], r);
+  const bool has_old = b < c.old_valid, has_new = b < c.new_valid && !(a.first_miss && b >= a.first_miss[lo]);
+  const u64 k_old = has_old ? a.keys[c.old_key_off + b] : 0, k_new = has_new ? a.keys[c.new_key_off + b] : 0;
+  const u32 r_old = has_old ? block_rank(a.tbl, c.old_tbl, c.old_n, b) : 0;
+  const u32 r_new = has_new ? block_rank(a.tbl, c.new_tbl, c.new_n, b) : 0;
+  if (k_old == k_new) {
+    if (r_old != r_new && k_new) cnt_add(a, k_new, cnt_unit(r_new) - cnt_unit(r_old));
+  } else {
+    if (r_old) cnt_add(a, k_old, 0ull - cnt_unit(r_old));
+    if (r_new) cnt_add(a, k_new, cnt_unit(r_new));
+  }
+}
+
+// Entries created since the counts were last brought up to date start at zero. Each of them receives, once, the
+// contribution of every accounted-for mapping (snapshot) whose key at the entry's chain depth is the entry's key.
+// Between two such passes entries are neither moved nor dropped, so the list holds valid, distinct entry ids.
+struct SnapDesc { u64 key_off; u32 valid, tbl, n, pad; };
+struct FixArgs {
+  Table tab; Entries ent; const u64 *keys; const SnapDesc *snaps; u32 n_snaps;
+  MsgTables tbl; const u32 *fresh; u32 n_fresh; u32 *status;
+};
+
+__global__ void k_fresh_fixup(FixArgs a) {
+  const u32 i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= a.n_fresh) return;
+  const u32 e = a.fresh[i];
+  if (e >= a.ent.n_total) { set_err(a.status, DERR_CORRUPT); return; }
+  const u64 key = a.ent.key[e];
+  const u32 d = a.ent.depth[e];
+  u64 sum = 0;
+  for (u32 q = 0; q < a.n_snaps; ++q) {
+    const SnapDesc sn = a.snaps[q];
+    if (d < sn.valid && a.keys[sn.key_off + d] == key) sum += cnt_unit(block_rank(a.tbl, sn.tbl, sn.n, d));
+  }
+  if (sum) a.ent.cnt[e] += sum;   // nobody else touches this entry in this kernel
+}
+
+// Cross-check of the event-driven counts against a full recomputation (debug mode): any difference is an error.
+__global__ void k_cnt_compare(const u64 *a, const u64 *b, u32 n, u32 *status) {
+  const u32 e = blockIdx.x * blockDim.x + threadIdx.x;
+  if (e < n && a[e] != b[e]) set_err(status, DERR_CORRUPT);
 }
 
 // ======================================================================================================
-// K4: victim selection. Candidates of a tier: resident, not in flight, rank <= max_rank (2, or 3 when the
-// incoming KV is Pinned). Whole ranks below the
-// boundary rank are taken, the ordered compaction keeps slot order, and a stable LSD radix sort on the
-// packed (rank, recency, inverted depth) key orders them; ties therefore end slot-ascending.
+// K4: victim selection (Algorithm 1 order; Section 6.2 recency). Candidates of a tier: resident, not in
+// flight, rank <= max_rank (2, or 3 when the incoming KV is Pinned). The order is the ascending order of the
+// composite (packed key, slot), packed key = [copy bit] rank | recency | inverted depth. The first k of that
+// order are found without sorting the tier:
+//   keys    : one pass over the tier writes every slot's packed key and counts the composite's top digit;
+//   level l : MSB-first radix select. Each level kernel first turns the previous level's histogram into the bin
+//             in which the k-th smallest composite lies (every CTA does this small scan itself, so no kernel
+//             waits for another), then counts the next digit of the slots inside that bin. The search stops as
+//             soon as the bin holds at most SEL_SLACK slots; the composite is unique per slot, so the last
+//             level always ends it;
+//   gather  : the slots below the bin (all selected) and the slots of the bin go into the pair list in slot
+//             order (per-CTA counts, then every CTA adds up the counts before it): k <= M <= k + SEL_SLACK pairs;
+//   sort    : stable LSD radix sort of those M pairs on the key bits, 10 bits per pass; ties end slot-ascending;
+//   emit    : the first k pairs, with their states.
+// Every kernel reads its arguments from one record in device memory, so the whole sequence is a fixed CUDA graph
+// per (tier, level count, pass count) and a call is one upload and one graph launch. Work scales with k, not with
+// the number of candidates.
 // ======================================================================================================
+typedef unsigned __int128 u128;
+constexpr u32 SEL_W0 = 11, SEL_WN = 13;            // digit widths of level 0 and of the later levels
+constexpr u32 SEL_BINS = 1u << SEL_WN;            // bins of a histogram (level 0 uses the first 2^11)
+constexpr u32 SEL_SLACK = 4096;                   // a boundary bin this small ends the search
+constexpr u32 SEL_MAX_LEVELS = 9;                 // 11 + 8 * 13 = 115 bits >= 63 key bits + 31 slot bits
+constexpr u32 SEL_ITEMS = 4, SEL_CTA = 1024;      // slots per thread / threads per CTA of the tier-wide passes
+constexpr u32 SEL_TILE = SEL_ITEMS * SEL_CTA;     // slots per CTA
+constexpr u64 SEL_NOT_KEY = ~0ull;                // packed key of a slot that is not a candidate (real keys have bit 63 clear)
+constexpr u32 RADIX_BITS = 10, RADIX_BINS = 1u << RADIX_BITS;
+constexpr u32 SORT_TILE = 1024;                   // pairs per CTA in the radix-sort kernels (8 warps x 128)
+constexpr int SORT_ITERS = SORT_TILE / 256;       // pairs per thread
+
+struct SelState { u32 done, need, below, lo; u32 pfx[4]; };   // after the boundaries of levels 0 .. j-1
 struct SelArgs {
   Entries ent; u32 e0, n_slots;       // entry range of the tier
   u32 n_req; u32 now; u32 stamp_bits, depth_bits; u32 mru; u32 max_rank; u32 one_tier;
   u32 copy_bit;                       // 1: the key carries a leading "resident block" bit (host tier with clean copies)
+  u32 slot_bits;                      // bits of a slot number; the composite is (key << slot_bits) | slot
+  u32 n_levels; u8 lev_lo[SEL_MAX_LEVELS], lev_w[SEL_MAX_LEVELS];   // level l looks at composite bits [lo, lo + w)
+  u64 *slot_key;                      // per slot of the tier: packed key or SEL_NOT_KEY
+  u32 *hist;                          // n_levels x SEL_BINS counters, zero at the start of a call
+  SelState *state;                    // n_levels + 1 records; record 0 is unused
+  u32 *cta_count;                     // per CTA of the tier-wide passes: slots it contributes to the gathered set
+  u64 *pair_key; u32 *pair_val;       // gathered pairs
+  u32 n_emit, rank_shift; u32 *slots_out; u8 *states_out;   // victim list
   u32 *status;
 };
 
-// Class of slot i for the selection: 0..3 = candidate of that rank, SEL_SHADOW = clean host copy of an HBM
-// block (always a candidate, goes first: dropping it loses nothing), SEL_NOT = not a candidate.
-constexpr u32 SEL_SHADOW = 0xFE, SEL_NOT = 0xFF;
-__device__ __forceinline__ u32 sel_class(const SelArgs &a, u32 i) {
-  u32 e = a.e0 + i;
-  if (!a.ent.key[e]) return SEL_NOT;
-  if (is_shadow(a.ent, e)) return SEL_SHADOW;
-  if (a.ent.infl[e]) return SEL_NOT;
-  u32 r = a.one_tier ? 1u : a.ent.rank[e];   // without lifecycle tracking every block is one tier
-  return r <= a.max_rank ? r : SEL_NOT;
-}
-
-__global__ void k_sel_count(SelArgs a) {
-  __shared__ u32 s[5];
-  if (threadIdx.x < 5) s[threadIdx.x] = 0;
+// The argument record of a call, staged once per CTA in shared memory (a per-thread copy would land in local
+// memory, because the level tables are indexed at run time).
+__device__ __forceinline__ const SelArgs &sel_args(const SelArgs *pa) {
+  __shared__ SelArgs s_args;
+  const u32 *src = reinterpret_cast<const u32 *>(pa);
+  u32 *dst = reinterpret_cast<u32 *>(&s_args);
+  for (u32 i = threadIdx.x; i < sizeof(SelArgs) / 4; i += blockDim.x) dst[i] = __ldg(src + i);
   __syncthreads();
-  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
-  u32 c = i < a.n_slots ? sel_class(a, i) : SEL_NOT;
-  for (u32 k = 0; k < 5; ++k) {
-    u32 m = __ballot_sync(0xFFFFFFFFu, c == (k == 4 ? SEL_SHADOW : k));
-    if ((threadIdx.x & 31) == 0 && m) atomicAdd(&s[k], __popc(m));
+  return s_args;
+}
+
+__device__ __forceinline__ u128 sel_comp(const SelArgs &a, u64 key, u32 slot) { return ((u128)key << a.slot_bits) | slot; }
+__device__ __forceinline__ u128 sel_prefix(const SelState &s) {
+  return ((u128)(((u64)s.pfx[3] << 32) | s.pfx[2]) << 64) | (((u64)s.pfx[1] << 32) | s.pfx[0]);
+}
+
+// Adds one to bin d of the CTA's shared histogram for every lane with ok set. A warp whose lanes all hold the same
+// digit (pools with few distinct stamps) adds once; otherwise every lane adds for itself.
+__device__ __forceinline__ void sel_count_digit(u32 *h, bool ok, u32 d) {
+  int same = 0;
+  __match_all_sync(0xFFFFFFFFu, ok ? d : 0xFFFFFFFFu, &same);
+  if (same) { if (ok && (threadIdx.x & 31) == 0) atomicAdd(&h[d], 32u); }
+  else if (ok) atomicAdd(&h[d], 1u);
+}
+
+__device__ __forceinline__ void sel_flush_hist(const u32 *h, u32 bins, u32 *ghist) {
+  for (u32 b = threadIdx.x; b < bins; b += SEL_CTA) { const u32 v = h[b]; if (v) atomicAdd(&ghist[b], v); }
+}
+
+// Every thread of a SEL_CTA-thread CTA calls this. Applies the boundary of level `lev` (its histogram is complete:
+// it was written by an earlier kernel) to the state before it and returns the state after it. The state says which
+// composite prefix still has to be searched (pfx, above bit lo), how many of the wanted slots lie in it (need) and
+// how many candidates lie below it (below); done ends the search: every candidate whose composite, shifted right
+// by lo, is <= pfx belongs to the gathered set.
+__device__ SelState sel_apply_level(const SelArgs &a, u32 lev, SelState in) {
+  __shared__ u32 s_warp[32];
+  __shared__ SelState s_out;
+  if (in.done) return in;
+  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const u32 bins = 1u << a.lev_w[lev];
+  const u32 per = (bins + SEL_CTA - 1) / SEL_CTA;   // consecutive bins per thread (<= 8)
+  const u32 *h = a.hist + (u64)lev * SEL_BINS;
+  u32 mine = 0;
+  for (u32 q = 0; q < per; ++q) { const u32 b = tid * per + q; if (b < bins) mine += h[b]; }
+  u32 x = mine;
+#pragma unroll
+  for (u32 o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(0xFFFFFFFFu, x, o); if (lane >= o) x += y; }
+  if (lane == 31) s_warp[warp] = x;
+  __syncthreads();
+  if (warp == 0) {
+    u32 w = s_warp[lane], z = w;
+#pragma unroll
+    for (u32 o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(0xFFFFFFFFu, z, o); if (lane >= o) z += y; }
+    s_warp[lane] = z - w;
+    if (lane == 31) {   // all candidates of this level: fewer than wanted means "take everything"
+      const u32 total = z;
+      if (lev == 0) a.status[ST_TOTAL] = total;   // same value from every CTA
+      if (total < in.need || total == 0) {
+        SelState o = in;
+        o.done = 1; o.below = in.below + total; o.need = 0; o.lo = 0;
+        o.pfx[0] = o.pfx[1] = o.pfx[2] = o.pfx[3] = 0xFFFFFFFFu;   // every composite is below this
+        a.status[ST_AUX] = o.below;                                  // size of the gathered set
+        s_out = o;
+      } else {
+        s_out.done = 2;   // marker: a bin will be found below
+      }
+    }
   }
   __syncthreads();
-  if (threadIdx.x < 4 && s[threadIdx.x]) atomicAdd(&a.status[ST_RANK0 + threadIdx.x], s[threadIdx.x]);
-  if (threadIdx.x == 4 && s[4]) atomicAdd(&a.status[ST_SHADOW], s[4]);
+  const bool take_all = s_out.done == 1;
+  const u32 before = s_warp[warp] + x - mine;   // candidates in the bins of earlier threads
+  __syncthreads();
+  if (!take_all && before < in.need && in.need <= before + mine) {   // exactly one thread
+    u32 cum = before;
+    for (u32 q = 0; q < per; ++q) {
+      const u32 b = tid * per + q;
+      const u32 c = b < bins ? h[b] : 0;
+      if (in.need <= cum + c) {
+        SelState o;
+        const u128 p = (sel_prefix(in) << a.lev_w[lev]) | b;
+        o.pfx[0] = (u32)p; o.pfx[1] = (u32)(p >> 32); o.pfx[2] = (u32)(p >> 64); o.pfx[3] = (u32)(p >> 96);
+        o.below = in.below + cum;
+        o.need = in.need - cum;
+        o.lo = a.lev_lo[lev];
+        o.done = (c <= SEL_SLACK || lev + 1 == a.n_levels) ? 1u : 0u;
+        if (o.done) a.status[ST_AUX] = o.below + c;   // size of the gathered set (same value from every CTA)
+        s_out = o;
+        break;
+      }
+      cum += c;
+    }
+  }
+  __syncthreads();
+  SelState out = s_out;
+  __syncthreads();
+  return out;
 }
 
-// Highest rank that must be looked at to serve n_req victims (Algorithm 1: lower ranks go first; clean host
-// copies go before everything). -1: the copies alone suffice.
-__device__ __forceinline__ int sel_boundary_rank(const u32 *status, u32 n_req) {
-  u32 cum = status[ST_SHADOW];
-  if (cum >= n_req) return -1;
-  cum += status[ST_RANK0];
-  if (cum >= n_req) return 0;
-  cum += status[ST_RANK1];
-  if (cum >= n_req) return 1;
-  cum += status[ST_RANK2];
-  if (cum >= n_req) return 2;
-  return 3;
+__device__ __forceinline__ SelState sel_initial(const SelArgs &a) {
+  SelState in;
+  in.done = 0; in.need = a.n_req; in.below = 0; in.lo = 0; in.pfx[0] = in.pfx[1] = in.pfx[2] = in.pfx[3] = 0;
+  return in;
 }
 
-struct PredSel {
-  SelArgs a;
-  __device__ bool operator()(u32 i) const {
-    u32 c = sel_class(a, i);
-    if (c == SEL_NOT) return false;
-    return c == SEL_SHADOW || (int)c <= sel_boundary_rank(a.status, a.n_req);
+// Pass over the tier: packed key of every slot, histogram of the composite's top digit. All fields of the SEL_ITEMS
+// slots of a thread are fetched before any of them is looked at, so the loads are in flight together.
+__global__ void __launch_bounds__(SEL_CTA) k_sel_keys(const SelArgs *pa) {
+  __shared__ u32 h[1u << SEL_W0];
+  const SelArgs &a = sel_args(pa);
+  for (u32 b = threadIdx.x; b < (1u << SEL_W0); b += SEL_CTA) h[b] = 0;
+  const u32 lo = a.lev_lo[0], mask = (1u << a.lev_w[0]) - 1;
+  u64 ekey[SEL_ITEMS];
+  u32 link[SEL_ITEMS], infl[SEL_ITEMS], rank[SEL_ITEMS], stamp[SEL_ITEMS], depth[SEL_ITEMS];
+#pragma unroll
+  for (u32 it = 0; it < SEL_ITEMS; ++it) {
+    const u32 i = (blockIdx.x * SEL_ITEMS + it) * SEL_CTA + threadIdx.x;
+    const u32 e = a.e0 + min(i, a.n_slots - 1);
+    ekey[it] = a.ent.key[e]; link[it] = a.ent.link[e]; infl[it] = a.ent.infl[e]; rank[it] = entry_rank(a.ent, e);
+    stamp[it] = a.ent.stamp[e]; depth[it] = a.ent.depth[e];
   }
-};
-struct EmitSel {
-  SelArgs a; u64 *keys; u32 *vals;
-  __device__ void operator()(u32 i, u32 pos) const {
-    u32 e = a.e0 + i;
-    const bool sh = is_shadow(a.ent, e);
-    u64 r = sh ? 0u : (a.one_tier ? 1u : a.ent.rank[e]);
-    u64 st = a.ent.stamp[e];
-    u64 rec = (r == 1 && a.mru && !sh) ? (u64)a.now - st : st;  // newest first inside the idle tier
-    u64 dinv = ((1ull << a.depth_bits) - 1) - a.ent.depth[e];   // chain tail first
-    u64 primary = sh ? 0u : 1u;                                  // copies sort before resident blocks
-    keys[pos] = (a.copy_bit ? primary << (2 + a.stamp_bits + a.depth_bits) : 0) | (r << (a.stamp_bits + a.depth_bits)) |
-                (rec << a.depth_bits) | dinv;
-    vals[pos] = i;
+  __syncthreads();
+#pragma unroll
+  for (u32 it = 0; it < SEL_ITEMS; ++it) {
+    const u32 i = (blockIdx.x * SEL_ITEMS + it) * SEL_CTA + threadIdx.x;
+    bool ok = false;
+    u32 d = 0;
+    if (i < a.n_slots) {
+      const bool sh = a.e0 + i >= a.ent.n_hbm && link[it] != ENT_NONE;       // clean host copy of an HBM block
+      const u32 r = a.one_tier ? 1u : rank[it];
+      u64 key = SEL_NOT_KEY;
+      if (ekey[it] && (sh || (!infl[it] && r <= a.max_rank))) {
+        const u64 rr = sh ? 0u : r;
+        const u64 rec = (rr == 1 && a.mru && !sh) ? (u64)a.now - stamp[it] : (u64)stamp[it];   // newest first inside the idle tier
+        const u64 dinv = ((1ull << a.depth_bits) - 1) - depth[it];                              // chain tail first
+        key = (a.copy_bit ? (u64)(sh ? 0u : 1u) << (2 + a.stamp_bits + a.depth_bits) : 0) |    // copies before resident blocks
+              (rr << (a.stamp_bits + a.depth_bits)) | (rec << a.depth_bits) | dinv;
+        ok = true;
+        d = (u32)(sel_comp(a, key, i) >> lo) & mask;
+      }
+      a.slot_key[i] = key;
+    }
+    sel_count_digit(h, ok, d);
   }
-};
+  __syncthreads();
+  sel_flush_hist(h, 1u << a.lev_w[0], a.hist);
+}
 
-// ---- stable LSD radix sort, 8 bits per pass; element count read from the status block ----------------
+// Level lev >= 1: boundary of level lev - 1, then the histogram of digit lev inside the boundary bin.
+__global__ void __launch_bounds__(SEL_CTA) k_sel_level(const SelArgs *pa, u32 lev) {
+  __shared__ u32 h[SEL_BINS];
+  const SelArgs &a = sel_args(pa);
+  if (lev >= a.n_levels) return;
+  const SelState st = sel_apply_level(a, lev - 1, lev == 1 ? sel_initial(a) : a.state[lev - 1]);
+  if (blockIdx.x == 0 && threadIdx.x == 0) a.state[lev] = st;
+  if (st.done) return;
+  const u32 bins = 1u << a.lev_w[lev];
+  for (u32 b = threadIdx.x; b < bins; b += SEL_CTA) h[b] = 0;
+  __syncthreads();
+  const u128 pfx = sel_prefix(st);
+  const u32 lo = a.lev_lo[lev], mask = bins - 1;
+  bool any = false;
+#pragma unroll
+  for (u32 it = 0; it < SEL_ITEMS; ++it) {
+    const u32 i = (blockIdx.x * SEL_ITEMS + it) * SEL_CTA + threadIdx.x;
+    bool ok = false;
+    u32 d = 0;
+    if (i < a.n_slots) {
+      const u64 key = a.slot_key[i];
+      if (key != SEL_NOT_KEY) {
+        const u128 c = sel_comp(a, key, i);
+        if ((c >> st.lo) == pfx) { ok = true; d = (u32)(c >> lo) & mask; }
+      }
+    }
+    sel_count_digit(h, ok, d);
+    any = any || ok;
+  }
+  if (__syncthreads_or(any)) sel_flush_hist(h, bins, a.hist + (u64)lev * SEL_BINS);
+}
+
+// Last boundary, then how many slots of every CTA's stretch belong to the gathered set (every candidate whose
+// composite prefix is at or below the boundary bin).
+__global__ void __launch_bounds__(SEL_CTA) k_sel_count(const SelArgs *pa) {
+  __shared__ u32 s_cnt;
+  const SelArgs &a = sel_args(pa);
+  const SelState st = sel_apply_level(a, a.n_levels - 1, a.n_levels == 1 ? sel_initial(a) : a.state[a.n_levels - 1]);
+  if (blockIdx.x == 0 && threadIdx.x == 0) a.state[a.n_levels] = st;   // always done: the last level's bins hold one slot each
+  if (threadIdx.x == 0) s_cnt = 0;
+  __syncthreads();
+  const u128 pfx = sel_prefix(st);
+  u32 mine = 0;
+#pragma unroll
+  for (u32 it = 0; it < SEL_ITEMS; ++it) {
+    const u32 i = (blockIdx.x * SEL_ITEMS + it) * SEL_CTA + threadIdx.x;
+    const u64 key = i < a.n_slots ? a.slot_key[i] : SEL_NOT_KEY;
+    mine += key != SEL_NOT_KEY && (sel_comp(a, key, i) >> st.lo) <= pfx;
+  }
+  mine = __reduce_add_sync(0xFFFFFFFFu, mine);
+  if ((threadIdx.x & 31) == 0 && mine) atomicAdd(&s_cnt, mine);
+  __syncthreads();
+  if (threadIdx.x == 0) a.cta_count[blockIdx.x] = s_cnt;
+}
+
+// The gathered set in slot order: a CTA's first pair goes behind the pairs of all CTAs before it.
+__global__ void __launch_bounds__(SEL_CTA) k_sel_gather(const SelArgs *pa) {
+  __shared__ u32 s_warp[SEL_ITEMS][32];   // pairs per (iteration, warp), then their exclusive prefix in slot order
+  __shared__ u32 s_red[32];
+  const SelArgs &a = sel_args(pa);
+  const SelState st = a.state[a.n_levels];
+  const u128 pfx = sel_prefix(st);
+  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  u32 before = 0;   // pairs of the CTAs before this one
+  for (u32 c = tid; c < blockIdx.x; c += SEL_CTA) before += a.cta_count[c];
+  before = __reduce_add_sync(0xFFFFFFFFu, before);
+  if (lane == 0) s_red[warp] = before;
+  u64 key[SEL_ITEMS];
+  u32 m[SEL_ITEMS];
+#pragma unroll
+  for (u32 it = 0; it < SEL_ITEMS; ++it) {
+    const u32 i = (blockIdx.x * SEL_ITEMS + it) * SEL_CTA + tid;
+    key[it] = i < a.n_slots ? a.slot_key[i] : SEL_NOT_KEY;
+    const bool in_set = key[it] != SEL_NOT_KEY && (sel_comp(a, key[it], i) >> st.lo) <= pfx;
+    m[it] = __ballot_sync(0xFFFFFFFFu, in_set);
+    if (lane == 0) s_warp[it][warp] = __popc(m[it]);
+  }
+  __syncthreads();
+  if (warp == 0) {
+    u32 base = s_red[lane];
+#pragma unroll
+    for (u32 o = 16; o > 0; o >>= 1) base += __shfl_xor_sync(0xFFFFFFFFu, base, o);
+    // exclusive scan over (iteration, warp) in that order = ascending slot
+    u32 run = base;
+#pragma unroll
+    for (u32 it = 0; it < SEL_ITEMS; ++it) {
+      const u32 w = s_warp[it][lane];
+      u32 z = w;
+#pragma unroll
+      for (u32 o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(0xFFFFFFFFu, z, o); if (lane >= o) z += y; }
+      s_warp[it][lane] = run + z - w;
+      run += __shfl_sync(0xFFFFFFFFu, z, 31);
+    }
+    if (blockIdx.x == gridDim.x - 1 && lane == 0) a.status[ST_M] = run;   // size of the gathered set
+  }
+  __syncthreads();
+#pragma unroll
+  for (u32 it = 0; it < SEL_ITEMS; ++it) {
+    if (!((m[it] >> lane) & 1)) continue;
+    const u32 i = (blockIdx.x * SEL_ITEMS + it) * SEL_CTA + tid;
+    const u32 p = s_warp[it][warp] + __popc(m[it] & ((1u << lane) - 1));
+    if (p >= a.n_slots) { set_err(a.status, DERR_CORRUPT); continue; }   // cannot happen: at most one pair per slot
+    a.pair_key[p] = key[it];
+    a.pair_val[p] = i;
+  }
+}
+
+// ---- stable LSD radix sort, RADIX_BITS per pass; element count read from the status block ----------------
 __global__ void __launch_bounds__(256) k_radix_hist(const u64 *keys, const u32 *status, u32 shift, u32 *counts) {
-  __shared__ u32 h[256];
+  __shared__ u32 h[RADIX_BINS];
   const u32 m = status[ST_M];
   const u32 n_tiles = (m + SORT_TILE - 1) / SORT_TILE;
   if (blockIdx.x >= n_tiles) return;
-  h[threadIdx.x] = 0;
+  for (u32 d = threadIdx.x; d < RADIX_BINS; d += 256) h[d] = 0;
   __syncthreads();
   u32 base = blockIdx.x * SORT_TILE;
   for (u32 k = threadIdx.x; k < SORT_TILE; k += 256) {
     u32 i = base + k;
-    if (i < m) atomicAdd(&h[(u32)(keys[i] >> shift) & 255u], 1u);
+    if (i < m) atomicAdd(&h[(u32)(keys[i] >> shift) & (RADIX_BINS - 1)], 1u);
   }
   __syncthreads();
-  counts[threadIdx.x * n_tiles + blockIdx.x] = h[threadIdx.x];   // digit-major
+  for (u32 d = threadIdx.x; d < RADIX_BINS; d += 256) counts[d * n_tiles + blockIdx.x] = h[d];   // digit-major
 }
 
 // One warp per digit: exclusive scan of that digit's per-tile counts in place, digit total to row_total.
@@ -915,7 +1210,7 @@ __global__ void __launch_bounds__(256) k_radix_scan(u32 *counts, u32 *row_total,
   const u32 m = status[ST_M];
   const u32 n_tiles = (m + SORT_TILE - 1) / SORT_TILE;
   const u32 lane = threadIdx.x & 31, d = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-  if (d >= 256) return;
+  if (d >= RADIX_BINS) return;
   u32 *row = counts + d * n_tiles;
   u32 run = 0;
   for (u32 t0 = 0; t0 < n_tiles; t0 += 32) {
@@ -933,14 +1228,15 @@ __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const
                                                        const u32 *status, u32 shift, const u32 *offsets, const u32 *row_total) {
   // each warp owns SORT_TILE / 8 consecutive items of the tile and walks them in order, so equal digits keep
   // their input order (stable)
-  __shared__ u32 cnt[8][256];
-  __shared__ u32 dbase[256];
+  __shared__ u32 cnt[8][RADIX_BINS];
+  __shared__ u32 dbase[RADIX_BINS];
   __shared__ u32 wsum[8];
+  constexpr u32 DPT = RADIX_BINS / 256;   // digits per thread in the digit scans
   const u32 m = status[ST_M];
   const u32 n_tiles = (m + SORT_TILE - 1) / SORT_TILE;
   if (blockIdx.x >= n_tiles) return;
   const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  for (u32 k = tid; k < 8 * 256; k += 256) (&cnt[0][0])[k] = 0;
+  for (u32 k = tid; k < 8 * RADIX_BINS; k += 256) (&cnt[0][0])[k] = 0;
   __syncthreads();
   const u32 base = blockIdx.x * SORT_TILE + warp * (SORT_TILE / 8);
   u64 kreg[SORT_ITERS];
@@ -951,25 +1247,28 @@ __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const
     bool ok = i < m;
     kreg[it] = ok ? keys_in[i] : 0;
     vreg[it] = ok ? vals_in[i] : 0;
-    u32 d = (u32)(kreg[it] >> shift) & 255u;
-    u32 peers = __match_any_sync(0xFFFFFFFFu, ok ? d : 256u);
+    u32 d = (u32)(kreg[it] >> shift) & (RADIX_BINS - 1);
+    u32 peers = __match_any_sync(0xFFFFFFFFu, ok ? d : RADIX_BINS);
     if (ok && (peers & ((1u << lane) - 1)) == 0) cnt[warp][d] += __popc(peers);
     __syncwarp();
   }
   __syncthreads();
-  {  // first position of every digit = exclusive scan of the 256 digit totals
-    u32 v = row_total[tid], x = v;
+  {  // first position of every digit = exclusive scan of the digit totals (DPT consecutive digits per thread)
+    u32 v[DPT], sum = 0;
+#pragma unroll
+    for (u32 q = 0; q < DPT; ++q) { v[q] = row_total[tid * DPT + q]; sum += v[q]; }
+    u32 x = sum;
 #pragma unroll
     for (u32 o = 1; o < 32; o <<= 1) { u32 y = __shfl_up_sync(0xFFFFFFFFu, x, o); if (lane >= o) x += y; }
     if (lane == 31) wsum[warp] = x;
     __syncthreads();
-    u32 before = 0;
-    for (u32 w = 0; w < warp; ++w) before += wsum[w];
-    dbase[tid] = before + x - v;
+    u32 run = x - sum;
+    for (u32 w = 0; w < warp; ++w) run += wsum[w];
+#pragma unroll
+    for (u32 q = 0; q < DPT; ++q) { dbase[tid * DPT + q] = run; run += v[q]; }
   }
   __syncthreads();
-  {  // per digit: exclusive scan across the 8 warps, plus the tile's offset inside the digit
-    u32 d = tid;
+  for (u32 d = tid; d < RADIX_BINS; d += 256) {   // per digit: exclusive scan across the 8 warps, plus the tile's offset inside the digit
     u32 run = dbase[d] + offsets[d * n_tiles + blockIdx.x];
 #pragma unroll
     for (int w = 0; w < 8; ++w) { u32 c = cnt[w][d]; cnt[w][d] = run; run += c; }
@@ -979,8 +1278,8 @@ __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const
   for (int it = 0; it < SORT_ITERS; ++it) {
     u32 i = base + it * 32 + lane;
     bool ok = i < m;
-    u32 d = (u32)(kreg[it] >> shift) & 255u;
-    u32 peers = __match_any_sync(0xFFFFFFFFu, ok ? d : 256u);
+    u32 d = (u32)(kreg[it] >> shift) & (RADIX_BINS - 1);
+    u32 peers = __match_any_sync(0xFFFFFFFFu, ok ? d : RADIX_BINS);
     u32 before = __popc(peers & ((1u << lane) - 1));
     u32 pos = 0;
     if (ok) pos = cnt[warp][d] + before;
@@ -993,17 +1292,18 @@ __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const
 
 // Victim list for the caller: slot, and its state: the rank, | 0x80 for an HBM block that still has a clean host
 // copy (moving it out needs no copy), or 0xFE for a host slot that is such a copy.
-__global__ void k_sel_emit(Entries en, u32 e0, u32 n_slots, const u64 *keys, const u32 *vals, u32 n, const u32 *status,
-                           u32 rank_shift, u32 copy_bit, u32 *slots_out, u8 *states_out) {
-  u32 i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i >= n || i >= status[ST_M]) return;   // only the first ST_M entries of the sorted list exist
-  u32 slot = vals[i];
-  if (slot >= n_slots) return;
-  slots_out[i] = slot;
-  u64 k = keys[i] >> rank_shift;
-  bool primary = copy_bit ? (k >> 2) & 1 : true;
-  u32 link = en.link[e0 + slot];
-  states_out[i] = !primary ? (u8)0xFE : (u8)((k & 3) | (link != ENT_NONE ? 0x80 : 0));
+__global__ void k_sel_emit(const SelArgs *pa, const u64 *keys, const u32 *vals) {
+  const SelArgs &a = sel_args(pa);
+  const u32 n = min(a.n_emit, a.status[ST_M]);   // only the first ST_M pairs exist
+  for (u32 i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
+    const u32 slot = vals[i];
+    if (slot >= a.n_slots) continue;
+    a.slots_out[i] = slot;
+    const u64 k = keys[i] >> a.rank_shift;
+    const bool primary = a.copy_bit ? (k >> 2) & 1 : true;
+    const u32 link = a.ent.link[a.e0 + slot];
+    a.states_out[i] = !primary ? (u8)0xFE : (u8)((k & 3) | (link != ENT_NONE ? 0x80 : 0));
+  }
 }
 
 // ======================================================================================================
@@ -1039,7 +1339,7 @@ __global__ void k_list_validate(ListArgs a) {
   }
   if (a.ent.infl[e] && !a.allow_inflight) set_err(a.status, DERR_STATE);
   u32 cat = LIST_COPY;
-  if (a.drop_all || (a.drop_dead && a.ent.rank[e] == 0)) cat = LIST_DROP;
+  if (a.drop_all || (a.drop_dead && entry_rank(a.ent, e) == 0)) cat = LIST_DROP;
   else if (a.clean_ok && a.ent.link[e] != ENT_NONE) cat = LIST_CLEAN;
   a.live[i] = cat;
 }
@@ -1065,14 +1365,14 @@ struct PredFree { const u64 *key; u32 e0; __device__ bool operator()(u32 i) cons
 struct EmitFree { u32 *list; u32 cap; __device__ void operator()(u32 i, u32 r) const { if (r < cap) list[r] = i; } };
 
 __device__ __forceinline__ void entry_clear(const Entries &en, u32 e) {
-  en.key[e] = 0; en.stamp[e] = 0; en.depth[e] = 0; en.infl[e] = 0; en.rank[e] = 0; en.floor[e] = 0; en.tslot[e] = ENT_NONE;
+  en.key[e] = 0; en.stamp[e] = 0; en.depth[e] = 0; en.infl[e] = 0; en.cnt[e] = 0; en.floor[e] = 0; en.tslot[e] = ENT_NONE;
   en.link[e] = ENT_NONE;
 }
 
 // Moves an entry (and whatever points at it: its table slot, its linked copy / block) to a free entry.
 __device__ __forceinline__ void entry_move(const Table &t, const Entries &en, u32 src, u32 dst) {
   en.key[dst] = en.key[src]; en.stamp[dst] = en.stamp[src]; en.depth[dst] = en.depth[src];
-  en.infl[dst] = en.infl[src]; en.rank[dst] = en.rank[src]; en.floor[dst] = en.floor[src];
+  en.infl[dst] = en.infl[src]; en.cnt[dst] = en.cnt[src]; en.floor[dst] = en.floor[src];
   u32 s = en.tslot[src];
   en.tslot[dst] = s;
   if (s != ENT_NONE) t.slots[s].ent = dst;
@@ -1106,7 +1406,7 @@ __global__ void k_list_apply(ListArgs a) {
   } else if (cat == LIST_CLEAN) {        // hand the block over to its clean host copy: metadata only
     u32 h = a.ent.link[e];
     a.ent.stamp[h] = a.ent.stamp[e]; a.ent.depth[h] = a.ent.depth[e]; a.ent.infl[h] = a.ent.infl[e];
-    a.ent.rank[h] = a.ent.rank[e]; a.ent.floor[h] = a.ent.floor[e];
+    a.ent.cnt[h] = a.ent.cnt[e]; a.ent.floor[h] = a.ent.floor[e];
     u32 s = a.ent.tslot[e];
     a.ent.tslot[h] = s;
     a.tab.slots[s].ent = h;
@@ -1121,12 +1421,12 @@ __global__ void k_list_apply(ListArgs a) {
     u32 de = a.dst_e0 + d;
     if (a.keep_copy) {                   // the block moves to HBM, the host slot stays behind as its clean copy
       a.ent.key[de] = a.ent.key[e]; a.ent.stamp[de] = a.ent.stamp[e]; a.ent.depth[de] = a.ent.depth[e];
-      a.ent.infl[de] = a.ent.infl[e]; a.ent.rank[de] = a.ent.rank[e]; a.ent.floor[de] = a.ent.floor[e];
+      a.ent.infl[de] = a.ent.infl[e]; a.ent.cnt[de] = a.ent.cnt[e]; a.ent.floor[de] = a.ent.floor[e];
       u32 s = a.ent.tslot[e];
       a.ent.tslot[de] = s;
       a.tab.slots[s].ent = de;
       a.ent.link[de] = e;
-      a.ent.link[e] = de; a.ent.tslot[e] = ENT_NONE; a.ent.infl[e] = 0;
+      a.ent.link[e] = de; a.ent.tslot[e] = ENT_NONE; a.ent.infl[e] = 0; a.ent.cnt[e] = 0;   // a copy carries no state of its own
     } else {
       entry_move(a.tab, a.ent, e, de);
     }
@@ -1165,12 +1465,12 @@ __global__ void k_load_apply(LoadArgs a) {
   if (s == ENT_NONE) return;
   a.tab.slots[s].ent = e;
   a.ent.key[e] = a.keys[i]; a.ent.stamp[e] = a.stamp[i]; a.ent.depth[e] = a.depth[i];
-  a.ent.infl[e] = 0; a.ent.rank[e] = a.state[i]; a.ent.floor[e] = a.state[i]; a.ent.tslot[e] = s; a.ent.link[e] = ENT_NONE;
+  a.ent.infl[e] = 0; a.ent.cnt[e] = 0; a.ent.floor[e] = a.state[i]; a.ent.tslot[e] = s; a.ent.link[e] = ENT_NONE;
 }
 
 __global__ void k_states_out(Entries en, u32 e0, u32 n, u8 *out) {
   u32 i = blockIdx.x * blockDim.x + threadIdx.x;
-  if (i < n) out[i] = en.key[e0 + i] ? (is_shadow(en, e0 + i) ? (u8)0xFE : (u8)en.rank[e0 + i]) : (u8)0xFF;
+  if (i < n) out[i] = en.key[e0 + i] ? (is_shadow(en, e0 + i) ? (u8)0xFE : (u8)entry_rank(en, e0 + i)) : (u8)0xFF;
 }
 
 // ======================================================================================================

@@ -20,6 +20,7 @@ def test_random_api_streams_match_the_oracle(oracle, seed, flags, pools):
     kw = dict(n_hbm_blocks=pools[0], n_host_blocks=pools[1], max_contexts=6, policy_flags=flags, suspended_order=seed % 2,
               pool_layout=seed % 2, **W.GEO_TOY.kwargs())
     gpu = B.Engine(max_tokens=1 << 16, max_messages=2048, **kw)
+    gpu.set_classify_mode((2, 1, 0)[seed % 3])    # event-driven counts cross-checked / recomputed in full / on their own
     cpu = oracle.OracleEngine(**kw)
     F.run([gpu, cpu], seed, steps=300, inclusive=bool(flags & 2), check_every=10)
 
@@ -37,6 +38,7 @@ def test_random_api_streams_with_long_messages(oracle, seed, flags):
               **W.GEO_TOY.kwargs())
     gpu = B.Engine(max_tokens=1 << 20, max_messages=4096, **kw)
     gpu.set_lookup_variant(1 + seed % 2)      # both forms of the hash + probe stage
+    gpu.set_classify_mode((2, 0, 1)[seed % 3])
     cpu = oracle.OracleEngine(**kw)
     F.run([gpu, cpu], seed, steps=200, inclusive=bool(flags & 2), check_every=10, invariants=False, max_tok=6000)
     st = gpu.get_stats()
@@ -56,5 +58,6 @@ def test_random_api_streams_with_three_tiers(oracle, seed, flags, pools):
     kw = dict(n_hbm_blocks=pools[0], n_host_blocks=pools[1], n_remote_blocks=pools[2], max_contexts=6, policy_flags=flags,
               suspended_order=seed % 2, pool_layout=seed % 2, **W.GEO_TOY.kwargs())
     gpu = B.Engine(max_tokens=1 << 16, max_messages=2048, **kw)
+    gpu.set_classify_mode((2, 1, 0)[seed % 3])    # event-driven counts cross-checked / recomputed in full / on their own
     cpu = oracle.OracleEngine(**kw)
     F.run([gpu, cpu], seed, steps=300, inclusive=bool(flags & 2), check_every=10)

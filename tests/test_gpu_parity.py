@@ -80,6 +80,8 @@ def _replay_pair(gpu, cpu, trace, payload, check_pools=True, record_states=True,
                          use_exchange=use_exchange)
     oc = W.ReplayOptions(payload=payload, record_states=record_states, verify_payload_every=verify_every,
                          use_exchange=use_exchange)
+    if gpu.n_hbm_blocks + gpu.n_host_blocks <= 8192:
+        gpu.set_classify_mode(2)      # small pools: every event-driven update is cross-checked against a full recomputation
     n_calls = 0
     for (i, kind, rg), (_, _, rc) in zip(W.replay(gpu, trace, og), W.replay(cpu, trace, oc)):
         if kind == "call":
@@ -443,6 +445,115 @@ def test_c4_lookup_and_select_parity(B, oracle, n_resident, chain_blocks, n_call
     for k in ec:
         assert np.array_equal(eg[k], ec[k]), k
     assert np.array_equal(gpu.get_states(0), cpu.get_states(0))
+    sg, sc = gpu.get_stats(), cpu.get_stats()
+    for k in sc:
+        if k not in W.GPU_ONLY_STATS:
+            assert sg[k] == sc[k], k
+
+
+def test_wide_stamps_and_depths_order_like_the_oracle(B, oracle):
+    """Stamps up to 2^31 and depths up to 2^24 make the packed victim key 59 bits wide; the order still equals the
+    oracle's comparator. A stamp / depth pair beyond 63 bits is refused by the loader."""
+    n = 3000
+    kw = dict(n_hbm_blocks=n, n_host_blocks=0, max_contexts=4, metadata_only=True, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 16, max_messages=64, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    rng = np.random.default_rng(123)
+    keys = rng.integers(2, 1 << 63, n, dtype=np.uint64)
+    state = rng.integers(0, 4, n).astype(np.uint8)
+    stamp = rng.integers(0, 1 << 31, n, dtype=np.uint32)
+    stamp[: n // 3] = stamp[0]                                   # many ties on the stamp: depth, then slot decide
+    depth = rng.integers(0, 1 << 24, n, dtype=np.uint32)
+    depth[: n // 6] = depth[0]
+    slot = rng.permutation(n).astype(np.uint32)
+    for eng in (gpu, cpu):
+        eng.debug_load_resident(keys, state, stamp, depth, slot, 0)
+    for n_req, pinned in ((1, False), (n // 10, False), (n // 2, False), (n, False), (n, True)):
+        vg, sg = gpu.select_victims(0, n_req, include_pinned=pinned)
+        vc, sc = cpu.select_victims(0, n_req, include_pinned=pinned)
+        assert np.array_equal(vg, vc) and np.array_equal(sg, sc), (n_req, pinned)
+    big = gpu.debug_load_resident_rc(np.array([5], np.uint64), [0], [0xFFFFFFFF], [0xFFFFFFFF], [0], 0)
+    assert big == B.E_INVAL                                      # 3 + 32 + 32 bits
+    vg, _ = gpu.select_victims(0, 5)
+    assert np.array_equal(vg, cpu.select_victims(0, 5)[0])       # and nothing changed
+
+
+def test_pool_beyond_one_scan_round(B, oracle):
+    """3.2 M slots: every ordered compaction over the tier (selection, free lists, compaction plan) needs more than
+    one 1024-tile round of the tile scan, and the slot count is not a multiple of any tile size."""
+    n_resident, chain_blocks, n_calls = 3 * (1 << 20) + 54321, 16128, 3
+    inp, gpu, cpu = _c4_setup(B, oracle, n_resident, chain_blocks, n_calls)
+    for frac in (0.10, 0.75):
+        n = int(n_resident * frac)
+        vg, sg = gpu.select_victims(0, n)
+        vc, sc = cpu.select_victims(0, n)
+        assert np.array_equal(vg, vc) and np.array_equal(sg, sc), frac
+    # release a scattered quarter of the pool, then fill the holes
+    rng = np.random.default_rng(77)
+    drop = rng.permutation(n_resident)[: n_resident // 4].astype(np.uint32)
+    gpu.release(0, drop)
+    cpu.release(0, drop)
+    assert np.array_equal(gpu.get_states(0), cpu.get_states(0))
+    assert gpu.compact(0) == cpu.compact(0)
+    eg, ec = gpu.get_entries(0), cpu.get_entries(0)
+    for k in ec:
+        assert np.array_equal(eg[k], ec[k]), k
+    assert np.array_equal(gpu.get_states(0), cpu.get_states(0))
+    ids = list(range(n_calls))
+    assert np.array_equal(gpu.map_blocks(ids, 0), cpu.map_blocks(ids, 0))
+    assert np.array_equal(gpu.map_blocks(ids, 1), cpu.map_blocks(ids, 1))
+    n = n_resident // 3
+    vg, sg = gpu.select_victims(0, n)
+    vc, sc = cpu.select_victims(0, n)
+    assert np.array_equal(vg, vc) and np.array_equal(sg, sc)
+    sg, sc = gpu.get_stats(), cpu.get_stats()
+    for k in sc:
+        if k not in W.GPU_ONLY_STATS:
+            assert sg[k] == sc[k], k
+
+
+def test_wait_that_runs_out_reports_a_device_error_and_changes_nothing(B, oracle):
+    """The single-pass lookup's chunks wait, bounded, for their predecessors. With the limit set to zero polls every
+    chunk behind the first one of a sequence gives up at once: the kernel returns normally, the call reports
+    KVT_E_DEVICE, and neither the host nor the device state of the engine has changed. Nothing faults or hangs."""
+    kw = dict(n_hbm_blocks=4096, n_host_blocks=64, max_contexts=8, metadata_only=True, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 18, max_messages=256, **kw)
+    cpu = oracle.OracleEngine(**kw)
+    rng = np.random.default_rng(99)
+    t0, t1 = (rng.integers(0, W.VOCAB, n, dtype=np.uint32) for n in (16 * 700 + 5, 16 * 300))
+    for eng in (gpu, cpu):
+        eng.spawn(0); eng.append(0, t0)
+        eng.spawn(1); eng.append(1, t1)
+        eng.map_blocks([0], 0); eng.map_blocks([0], 1); eng.prefill_done(0)     # context 0 is resident and idle
+        eng.append(0, t1[:160])
+    before = (gpu.get_stats(), gpu.get_entries(0), gpu.get_states(0), gpu.get_block_map(0))
+    gpu.set_lookup_variant(2)
+    gpu.set_wait_limit(0)
+    rc, _ = gpu.map_blocks_rc([0, 1], 0)
+    assert rc == B.E_DEVICE and "wait" in gpu.last_error()
+    after = (gpu.get_stats(), gpu.get_entries(0), gpu.get_states(0), gpu.get_block_map(0))
+    for k in before[0]:
+        if k != "kernel_launches":
+            assert before[0][k] == after[0][k], k
+    for k in before[1]:
+        assert np.array_equal(before[1][k], after[1][k]), k
+    assert np.array_equal(before[2], after[2])
+    for a, b in zip(before[3], after[3]):
+        assert np.array_equal(a, b)
+    assert gpu.map_blocks_rc([0], 1)[0] == B.E_STATE                 # nobody is in flight
+    # the same call with the default kernels, then with the single pass and its normal limit, matches the oracle
+    gpu.set_lookup_variant(1)
+    assert np.array_equal(gpu.map_blocks([0, 1], 0), cpu.map_blocks([0, 1], 0))
+    assert np.array_equal(gpu.map_blocks([0, 1], 1), cpu.map_blocks([0, 1], 1))
+    for eng in (gpu, cpu):
+        eng.prefill_done(0); eng.prefill_done(1)
+        eng.append(1, t0[:999])
+    gpu.set_lookup_variant(2)
+    gpu.set_wait_limit(1 << 18)
+    assert np.array_equal(gpu.map_blocks([1, 0], 0), cpu.map_blocks([1, 0], 0))
+    eg, ec = gpu.get_entries(0), cpu.get_entries(0)
+    for k in ec:
+        assert np.array_equal(eg[k], ec[k]), k
     sg, sc = gpu.get_stats(), cpu.get_stats()
     for k in sc:
         if k not in W.GPU_ONLY_STATS:

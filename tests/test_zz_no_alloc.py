@@ -15,14 +15,18 @@ def test_noalloc_hasher_matches_the_ordinary_one_twice_in_a_row():
     from paper_2609_39819_b200 import binding as B
     B.load_library()
     rng = np.random.default_rng(2024)
-    # first a long input (many chunks), then a short one: stale scratch of the first call must not matter
-    for n_tokens, seed in ((16 * 5000 + 11, 0), (16 * 300 + 5, 7)):
-        tok = torch.from_numpy(rng.integers(0, 151552, n_tokens, dtype=np.uint32).view(np.int32)).cuda()
+    from oracle import kvt_oracle
+    # first a long input (many chunks), then shorter ones: stale scratch of an earlier call must not matter. Also an
+    # exact multiple of the 256-block chunk and a single block.
+    for n_tokens, seed in ((16 * 5000 + 11, 0), (16 * 300 + 5, 7), (16 * 256 * 3, 1), (16, 5)):
+        host = rng.integers(0, 151552, n_tokens, dtype=np.uint32)
+        tok = torch.from_numpy(host.view(np.int32)).cuda()
         want = B.hash_tokens(tok, seed)                       # existing entry point, caller-provided scratch
         got = torch.zeros(n_tokens // 16, dtype=torch.int64, device="cuda")
         assert B.hash_tokens_noalloc(tok, got, seed) == B.OK  # through the C ABI, built-in scratch
         torch.cuda.synchronize()
         assert torch.equal(got, want)                         # integer keys: bit-exact
+        assert np.array_equal(got.cpu().numpy().view(np.uint64), kvt_oracle.hash_tokens(host, seed))   # and the CPU definition
     # sizes beyond the built-in scratch are refused, nothing is written
     big = torch.empty(B.HASH_NOALLOC_MAX_TOKENS + 16, dtype=torch.int32, device="cuda")
     out = torch.full((1,), 123, dtype=torch.int64, device="cuda")
