@@ -519,7 +519,7 @@ def metadata_stress(torch, B, hbm_peak, reps=5):
     resulting 1.03 M mappings, selection of 10% of the pool. Kernel times come from the library's own
     CUDA events, call times from events around the C-ABI call. Algorithmic bytes per unit: hash 72 B per
     block (64 B tokens + 8 B key), fused lookup 64 B per block (two 32-byte table sectors), classify 16 B
-    per mapping + 9 B per entry, select 8 B per resident block + 4 B per victim."""
+    per mapping (8 B key + one 8-byte count update), select 8 B per resident block + 4 B per victim."""
     n_res, n_calls, cb = 1 << 20, 64, 16128
     inp = W.inputs_c4(1, n_resident=n_res, chain_blocks=cb, n_calls=n_calls)
     eng = B.Engine(n_hbm_blocks=n_res, n_host_blocks=0, max_contexts=n_calls + 1, metadata_only=True,
@@ -537,7 +537,7 @@ def metadata_stress(torch, B, hbm_peak, reps=5):
         a.record(); r = fn(); b.record(); torch.cuda.synchronize()
         return a.elapsed_time(b), r
 
-    look_ms, cls_ms, sel_ms = [], [], []
+    look_ms, cls_ms, sel_ms, cls_edit_ms, cls_full_ms, cls_done_ms = [], [], [], [], [], []
     s0 = None
     flush = torch.empty(1 << 29, dtype=torch.uint8, device="cuda")   # 512 MiB > L2: every timed call starts cold
     for rep in range(reps + 1):
@@ -550,9 +550,19 @@ def metadata_stress(torch, B, hbm_peak, reps=5):
         ms, info = timed(lambda: eng.map_blocks(ids, 0))
         look_ms.append(ms)
         flush.fill_(rep + 1)
-        cls_ms.append(timed(lambda: eng.classify())[0])
+        cls_ms.append(timed(lambda: eng.classify())[0])      # event-driven: the 64 contexts of the batch are new mappings
+        eng.set_classify_mode(1)                             # the full recomputation over all contexts, for comparison
+        flush.fill_(rep + 1)
+        cls_full_ms.append(timed(lambda: eng.classify())[0])
+        eng.set_classify_mode(0)
         for c in ids:
             eng.prefill_done(c)
+        flush.fill_(rep + 1)
+        cls_done_ms.append(timed(lambda: eng.classify())[0])  # every context's messages went from Active to Suspended
+        eng.pin(0, 0, 1)                                     # one context's message changes state: 16,128 of its blocks
+        flush.fill_(rep + 1)
+        cls_edit_ms.append(timed(lambda: eng.classify())[0])
+        eng.unpin(0, 0, 1)
         eng.classify()
         flush.fill_(rep + 2)
         torch.cuda.synchronize()
@@ -560,6 +570,7 @@ def metadata_stress(torch, B, hbm_peak, reps=5):
         sel_ms.append(ms)
         for i in ids:
             eng.terminate(i)
+        eng.classify()                    # takes the ended contexts' mappings away (not timed)
     s1 = eng.get_stats()
     d = {k: s1[k] - s0[k] for k in s1}
     n_blocks = int(info["n_blocks"].sum())
@@ -576,8 +587,12 @@ def metadata_stress(torch, B, hbm_peak, reps=5):
                         "algorithmic_bytes_per_block": 136, "achieved_GBs": n_blocks * 136 / (look_k / 1e3) / 1e9,
                         "frac_hbm": n_blocks * 136 / (look_k / 1e3) / 1e9 / hbm_peak},
         "classify": {"mappings": n_blocks, "entries": n_res, "call_ms": med(cls_ms),
-                     "achieved_GBs": (16 * n_blocks + 9 * n_res) / (med(cls_ms) / 1e3) / 1e9,
-                     "frac_hbm": (16 * n_blocks + 9 * n_res) / (med(cls_ms) / 1e3) / 1e9 / hbm_peak},
+                     "what": "event-driven update after the LOOKUP batch: 64 new contexts x 16,128 mappings",
+                     "achieved_GBs": 16 * n_blocks / (med(cls_ms) / 1e3) / 1e9,
+                     "frac_hbm": 16 * n_blocks / (med(cls_ms) / 1e3) / 1e9 / hbm_peak,
+                     "after_one_context_changed_state_ms": med(cls_edit_ms),
+                     "after_all_contexts_suspended_ms": med(cls_done_ms),
+                     "full_recomputation_ms": med(cls_full_ms)},
         "select": {"resident": n_res, "victims": len(v), "call_ms": med(sel_ms), "kernels_ms": sel_k,
                    "resident_blocks_per_s": n_res / (med(sel_ms) / 1e3),
                    "achieved_GBs": (8 * n_res + 4 * len(v)) / (sel_k / 1e3) / 1e9,

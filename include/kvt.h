@@ -42,7 +42,7 @@
 extern "C" {
 #endif
 
-#define KVT_ABI_VERSION 2u
+#define KVT_ABI_VERSION 3u
 #define KVT_BLOCK_TOKENS 16u
 
 /* ---- status codes -------------------------------------------------------------------------- */
@@ -156,6 +156,12 @@ typedef struct kvt_config {
   void *dev_meta;  uint64_t dev_meta_bytes;   /* device metadata + scratch arena, 256-byte aligned */
   void *dev_tokens; uint64_t dev_tokens_bytes;/* device token arena, 256-byte aligned */
   void *remote_pool; uint64_t remote_pool_bytes; /* device-accessible memory of the remote tier; NULL/0 if none or metadata-only */
+  void *stage_buf; uint64_t stage_bytes;         /* optional device memory (16-byte aligned; 64-512 MiB is plenty) for moves
+                                                    between device memory and a pool in host memory: the mover kernel
+                                                    gathers / scatters whole blocks through it and the copy engines carry
+                                                    them over the link in large transfers, on two streams the library
+                                                    creates, one per direction. NULL/0: the kernel reads / writes host
+                                                    memory directly. Used for blocks of at least 512 KiB. */
 } kvt_config;
 
 /* Computes the byte sizes the caller must allocate for dev_meta and dev_tokens from the other
@@ -400,7 +406,9 @@ int32_t kvt_set_profiling(kvt_engine *e, uint32_t on);
 /* Tuning hook: which mover kernel offload / reload / compact / copy_blocks launch. 0 = automatic (variant 2
  * whenever it applies, default), 1 = one CTA per (block, chunk), 2 = one warp per 4 KiB tile (needs chunk_bytes % 4096 == 0,
  * otherwise variant 1 is used), 3 = TMA bulk copies through a shared-memory ring (chunks of at most 16 KiB or a
- * multiple of 16 KiB). Results are identical. */
+ * multiple of 16 KiB), 4 = copy engines through the staging ring for every block size (needs kvt_config.stage_buf;
+ * only offload / reload / move between device memory and a pool in host memory). With 1-3 the staging ring is not
+ * used. Results are identical. */
 int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant);
 
 /* Upper bound on the thread blocks a mover kernel launches (offload / reload / exchange / move / compact /

@@ -50,7 +50,8 @@ class Config(C.Structure):
                 ("host_pool", C.c_void_p), ("host_pool_bytes", C.c_uint64),
                 ("dev_meta", C.c_void_p), ("dev_meta_bytes", C.c_uint64),
                 ("dev_tokens", C.c_void_p), ("dev_tokens_bytes", C.c_uint64),
-                ("remote_pool", C.c_void_p), ("remote_pool_bytes", C.c_uint64)]
+                ("remote_pool", C.c_void_p), ("remote_pool_bytes", C.c_uint64),
+                ("stage_buf", C.c_void_p), ("stage_bytes", C.c_uint64)]
 
 
 class Op(C.Structure):
@@ -179,7 +180,7 @@ class Engine:
                  n_hbm_blocks=128, n_host_blocks=512, max_contexts=64, hash_seed=0, suspended_order=ORDER_MRU,
                  metadata_only=False, table_capacity=None, max_messages=1 << 16, max_batch_blocks=None,
                  max_tokens=1 << 22, max_key_blocks=None, host_pool_on_device=False, zero_pools=True, policy_flags=0,
-                 n_remote_blocks=0, device="cuda"):
+                 n_remote_blocks=0, stage_mib=256, device="cuda"):
         import torch
         if not torch.cuda.is_available():
             raise RuntimeError("paper_2609_39819_b200 needs a CUDA device (there is no CPU fallback)")
@@ -201,7 +202,7 @@ class Engine:
         if max_key_blocks is None:
             max_key_blocks = max(max_tokens // 8, 64)
         cfg = Config()
-        cfg.abi_version, cfg.block_tokens = 2, 16
+        cfg.abi_version, cfg.block_tokens = 3, 16
         cfg.n_layers, cfg.n_kv_heads, cfg.head_dim, cfg.elem_bytes = n_layers, n_kv_heads, head_dim, elem_bytes
         cfg.pool_layout, cfg.n_hbm_blocks, cfg.n_host_blocks = pool_layout, n_hbm_blocks, n_host_blocks
         cfg.n_remote_blocks = n_remote_blocks
@@ -236,6 +237,11 @@ class Engine:
                 self.remote_pool = new(nr, dtype=torch.uint8, pin_memory=True)
             if n_remote_blocks:
                 cfg.remote_pool, cfg.remote_pool_bytes = self.remote_pool.data_ptr(), self.remote_pool.numel()
+            # staging ring for copy-engine transfers between HBM and a host-memory tier (large blocks only)
+            self.stage_buf = None
+            if stage_mib and not host_pool_on_device and (n_host_blocks or n_remote_blocks):
+                self.stage_buf = torch.empty(stage_mib << 20, dtype=torch.uint8, device=self.device)
+                cfg.stage_buf, cfg.stage_bytes = self.stage_buf.data_ptr(), self.stage_buf.numel()
         self.cfg = cfg
         h = C.c_void_p()
         rc = self.L.kvt_create(C.byref(cfg), _stream(), C.byref(h))
@@ -251,7 +257,7 @@ class Engine:
         if getattr(self, "h", None):
             self.L.kvt_destroy(self.h)
             self.h = None
-            self.hbm_pool = self.host_pool = self.remote_pool = self.meta = self.tokens = None   # release the memory
+            self.hbm_pool = self.host_pool = self.remote_pool = self.meta = self.tokens = self.stage_buf = None   # release the memory
 
     def __del__(self):
         try:

@@ -169,7 +169,16 @@ struct kvt_engine {
   cudaStream_t capture_stream = nullptr;   // only ever used for stream capture, never executes work
   bool use_graphs = true;
   SelArgs *h_sel = nullptr;                // pinned staging of the selection's argument record
-  u32 mover_variant = 0;   // 0 auto, 1 CTA per chunk, 2 warp per 4 KiB tile, 3 TMA ring
+  u32 mover_variant = 0;   // 0 auto, 1 CTA per chunk, 2 warp per 4 KiB tile, 3 TMA ring, 4 copy engines through the staging ring
+  // Staging ring for moves between device memory and a pool in host memory: the payload is gathered into (scattered
+  // from) contiguous device memory by the mover kernel and crosses the link as large copy-engine transfers on the
+  // library's own two copy streams (one per direction, so an exchange drives the link in both directions).
+  static constexpr int N_STAGES = 4;
+  struct Staging {
+    u8 *buf = nullptr; u32 blocks_per_stage = 0; bool ok = false;
+    cudaStream_t cs[2] = {nullptr, nullptr};                 // [0] device -> host, [1] host -> device
+    cudaEvent_t ready[2][N_STAGES] = {}, free_[2][N_STAGES] = {}, begin = nullptr;
+  } stg;
   u32 mover_max_ctas = 0;  // caller's upper bound on the mover's grid (0: automatic)
   bool tier_in_host_mem[3] = {false, false, false};   // pool is host memory: moves to / from it are bound by the host link
   // Grid of a mover launch. Inside the device: 8 CTAs of 256 threads per SM. A move that crosses the host link
@@ -339,23 +348,38 @@ PoolView pool_view(kvt_engine *e, u32 tier) {
   return v;
 }
 
+// View of one stage of the staging ring as a block-major pool of `blocks` slots.
+PoolView stage_view(kvt_engine *e, int dir, int stage, u32 blocks) {
+  PoolView v;
+  v.base = e->stg.buf + ((u64)dir * kvt_engine::N_STAGES + stage) * e->stg.blocks_per_stage * e->block_bytes;
+  v.n_slots = blocks; v.slot_stride = e->block_bytes; v.chunk_stride = e->chunk_bytes;
+  return v;
+}
+
+int32_t launch_mover_views(kvt_engine *e, cudaStream_t s, const PoolView &sv, const u32 *src, const PoolView &dv, const u32 *dst,
+                           u32 n_max, const u32 *n_dev, u32 ld, bool timed);
+
 int32_t launch_mover(kvt_engine *e, cudaStream_t s, u32 st, const u32 *src, u32 dt, const u32 *dst, u32 n_max,
                      const u32 *n_dev) {
   if (e->metadata_only || n_max == 0) return KVT_OK;
+  return launch_mover_views(e, s, pool_view(e, st), src, pool_view(e, dt), dst, n_max, n_dev, e->link_dirs(st, dt),
+                            e->profiling && n_dev != nullptr);   // only the calls that synchronise afterwards are timed
+}
+
+int32_t launch_mover_views(kvt_engine *e, cudaStream_t s, const PoolView &sv, const u32 *src, const PoolView &dv, const u32 *dst,
+                           u32 n_max, const u32 *n_dev, u32 ld, bool timed) {
   MoveArgs a;
-  a.src = pool_view(e, st); a.dst = pool_view(e, dt);
+  a.src = sv; a.dst = dv;
   a.src_ids = src; a.dst_ids = dst; a.n_pairs = n_max; a.n_pairs_dev = n_dev;
   a.n_chunks = (u32)e->n_chunks; a.chunk_bytes = (u32)e->chunk_bytes; a.status = e->d_status;
   u64 items = (u64)n_max * e->n_chunks;
-  const u32 ld = e->link_dirs(st, dt);
   u32 grid = e->mover_grid(items, ld) * (ld && !e->mover_max_ctas ? 4 : 1);   // 256-thread CTAs: four for one of 1024
-  const bool timed = e->profiling && n_dev != nullptr;   // only the calls that synchronise afterwards
   if (timed) CU(cudaEventRecord(e->ev_m0, s));
   // a warp per 4 KiB tile keeps 8 loads per lane in flight whatever the chunk size (measured faster for
   // 4 KiB and 32 KiB chunks alike); chunks that are not a multiple of 4 KiB take the CTA-per-chunk kernel
   const bool tiles_ok = e->chunk_bytes % 4096 == 0;
   const bool use_tiles = e->mover_variant != 1;
-  if (e->mover_variant == 3 && e->chunk_bytes % 16 == 0) {   // TMA ring (experimental variant)
+  if (e->mover_variant == 3 && e->chunk_bytes % 16 == 0 && src && dst) {   // TMA ring (experimental variant)
     u32 tile = (u32)(e->chunk_bytes <= 16384 ? e->chunk_bytes : (e->chunk_bytes % 16384 == 0 ? 16384 : 0));
     if (tile == 0 || tile > 49152) return fail(e, KVT_E_INVAL, "chunk size not supported by the TMA mover");
     u32 tpc = (u32)(e->chunk_bytes / tile);
@@ -385,6 +409,98 @@ int32_t launch_mover(kvt_engine *e, cudaStream_t s, u32 st, const u32 *src, u32 
   }
   if (timed) { CU(cudaEventRecord(e->ev_m1, s)); e->mover_timed = true; }
   LAUNCH_CHECK();
+  return KVT_OK;
+}
+
+// Whether a move of n blocks between these tiers goes through the staging ring: a staging buffer is configured,
+// exactly one side is a pool in host memory, and the blocks are large enough for one copy-engine transfer each.
+bool staged_applies(const kvt_engine *e, u32 st, u32 dt) {
+  if (!e->stg.ok || e->metadata_only) return false;
+  if (e->tier_in_host_mem[st] == e->tier_in_host_mem[dt]) return false;
+  if (e->mover_variant != 0 && e->mover_variant != 4) return false;      // a kernel variant was asked for
+  return e->mover_variant == 4 || e->block_bytes >= (512u << 10);
+}
+
+// Moves n blocks src_tier[h_src[i]] -> dst_tier[h_dst[i]] through the staging ring. d_src / d_dst: the same id lists
+// in device memory (for the gather / scatter kernel); h_src / h_dst: on the host (for the copy-engine transfers).
+// dir 0: device -> host (gather into a stage on `s`, then transfers on the copy stream); dir 1: host -> device
+// (transfers into a stage on the copy stream, then scatter on `s`). Consecutive host slots travel as one transfer.
+// When this returns, `s` waits for everything the copy stream still has to do.
+int32_t staged_move(kvt_engine *e, cudaStream_t s, u32 st, const u32 *d_src, const u32 *h_src, u32 dt, const u32 *d_dst,
+                    const u32 *h_dst, u32 n) {
+  if (!n) return KVT_OK;
+  const int dir = e->tier_in_host_mem[st] ? 1 : 0;
+  kvt_engine::Staging &g = e->stg;
+  const u32 SB = g.blocks_per_stage;
+  const u64 BB = e->block_bytes;
+  u8 *host_pool = (u8 *)(dir ? (st == KVT_TIER_HOST ? e->cfg.host_pool : e->cfg.remote_pool)
+                             : (dt == KVT_TIER_HOST ? e->cfg.host_pool : e->cfg.remote_pool));
+  const u32 *h_ids = dir ? h_src : h_dst;     // slots of the pool in host memory
+  const u32 n_host_slots = e->tier_slots(dir ? st : dt);
+  for (u32 i = 0; i < n; ++i) if (h_ids[i] >= n_host_slots) return fail(e, KVT_E_RANGE, "slot id out of range");
+  // Inside a batch the blocks sit in the stage in the order of their host slots, whatever the order of the list, so
+  // that every stretch of consecutive host slots is one transfer: pos[i] = place of list item i in its batch's stage.
+  const u32 n_batches = cdiv(n, SB);
+  u32 *h_pos = e->h_ids2, *d_pos = e->dp<u32>(e->L.ids2);
+  std::vector<u32> order(std::min(SB, n));
+  for (u32 k = 0; k < n_batches; ++k) {
+    const u32 b0 = k * SB, nb = std::min(SB, n - b0);
+    for (u32 i = 0; i < nb; ++i) order[i] = i;
+    std::sort(order.begin(), order.begin() + nb, [&](u32 x, u32 y) { return h_ids[b0 + x] < h_ids[b0 + y]; });
+    for (u32 p = 0; p < nb; ++p) h_pos[b0 + order[p]] = p;
+  }
+  CU(cudaMemcpyAsync(d_pos, h_pos, n * 4ull, cudaMemcpyHostToDevice, s));
+  {
+    int32_t r = stage_release(e, s);   // the next call that stages ids waits for this upload
+    if (r) return r;
+  }
+  const bool timed = e->profiling;
+  if (timed) CU(cudaEventRecord(e->ev_m0, s));
+  if (dir == 1) {   // the host pool holds what earlier work on `s` put there
+    CU(cudaEventRecord(g.begin, s));
+    CU(cudaStreamWaitEvent(g.cs[1], g.begin, 0));
+  }
+  std::vector<u32> sorted_slots(std::min(SB, n));
+  for (u32 k = 0; k < n_batches; ++k) {
+    const int sg = (int)(k % kvt_engine::N_STAGES);
+    const u32 b0 = k * SB, nb = std::min(SB, n - b0);
+    u8 *stage = stage_view(e, dir, sg, nb).base;
+    for (u32 i = 0; i < nb; ++i) sorted_slots[h_pos[b0 + i]] = h_ids[b0 + i];
+    auto transfers = [&]() -> int32_t {
+      for (u32 p = 0; p < nb;) {
+        u32 run = 1;
+        while (p + run < nb && sorted_slots[p + run] == sorted_slots[p] + run) ++run;
+        u8 *hp = host_pool + (u64)sorted_slots[p] * BB, *sp = stage + (u64)p * BB;
+        if (dir == 0) CU(cudaMemcpyAsync(hp, sp, run * BB, cudaMemcpyDeviceToHost, g.cs[0]));
+        else CU(cudaMemcpyAsync(sp, hp, run * BB, cudaMemcpyHostToDevice, g.cs[1]));
+        p += run;
+      }
+      return KVT_OK;
+    };
+    if (dir == 0) {
+      if (k >= (u32)kvt_engine::N_STAGES) CU(cudaStreamWaitEvent(s, g.free_[0][sg], 0));   // the stage's transfers are done
+      int32_t r = launch_mover_views(e, s, pool_view(e, st), d_src + b0, stage_view(e, 0, sg, nb), d_pos + b0, nb, nullptr, 0, false);
+      if (r) return r;
+      CU(cudaEventRecord(g.ready[0][sg], s));
+      CU(cudaStreamWaitEvent(g.cs[0], g.ready[0][sg], 0));
+      r = transfers();
+      if (r) return r;
+      CU(cudaEventRecord(g.free_[0][sg], g.cs[0]));
+    } else {
+      if (k >= (u32)kvt_engine::N_STAGES) CU(cudaStreamWaitEvent(g.cs[1], g.free_[1][sg], 0));   // the stage was scattered
+      int32_t r = transfers();
+      if (r) return r;
+      CU(cudaEventRecord(g.ready[1][sg], g.cs[1]));
+      CU(cudaStreamWaitEvent(s, g.ready[1][sg], 0));
+      r = launch_mover_views(e, s, stage_view(e, 1, sg, nb), d_pos + b0, pool_view(e, dt), d_dst + b0, nb, nullptr, 0, false);
+      if (r) return r;
+      CU(cudaEventRecord(g.free_[1][sg], s));
+    }
+  }
+  if (dir == 0)   // the caller's stream continues once the last transfers have landed
+    for (u32 k = n_batches > (u32)kvt_engine::N_STAGES ? n_batches - kvt_engine::N_STAGES : 0; k < n_batches; ++k)
+      CU(cudaStreamWaitEvent(s, g.free_[0][k % kvt_engine::N_STAGES], 0));
+  if (timed) { CU(cudaEventRecord(e->ev_m1, s)); e->mover_timed = true; }
   return KVT_OK;
 }
 
@@ -681,6 +797,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   u64 chunk_bytes = 16ull * c.n_kv_heads * c.head_dim * c.elem_bytes, n_chunks = 2ull * c.n_layers;
   bool meta_only = c.hbm_pool == nullptr;
   if (!meta_only) {
+    if (c.stage_buf && ((uintptr_t)c.stage_buf & 15)) return KVT_E_INVAL;
     if (c.hbm_pool_bytes < chunk_bytes * n_chunks * c.n_hbm_blocks || ((uintptr_t)c.hbm_pool & 15)) return KVT_E_INVAL;
     if (c.n_host_blocks && (!c.host_pool || c.host_pool_bytes < chunk_bytes * n_chunks * c.n_host_blocks ||
                             ((uintptr_t)c.host_pool & 15)))
@@ -705,6 +822,21 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
     }
   }
   cudaDeviceGetAttribute(&e->sm_count, cudaDevAttrMultiProcessorCount, dev);
+  if (!meta_only && c.stage_buf && c.stage_bytes) {
+    kvt_engine::Staging &g = e->stg;
+    g.buf = (u8 *)c.stage_buf;
+    g.blocks_per_stage = (u32)std::min<u64>(c.stage_bytes / (2ull * kvt_engine::N_STAGES) / e->block_bytes, 0x7FFFFFFFu);
+    bool okk = g.blocks_per_stage > 0;
+    for (int d = 0; d < 2 && okk; ++d) {
+      okk = cudaStreamCreateWithFlags(&g.cs[d], cudaStreamNonBlocking) == cudaSuccess;
+      for (int k = 0; k < kvt_engine::N_STAGES && okk; ++k)
+        okk = cudaEventCreateWithFlags(&g.ready[d][k], cudaEventDisableTiming) == cudaSuccess &&
+              cudaEventCreateWithFlags(&g.free_[d][k], cudaEventDisableTiming) == cudaSuccess;
+    }
+    okk = okk && cudaEventCreateWithFlags(&g.begin, cudaEventDisableTiming) == cudaSuccess;
+    if (!okk) cudaGetLastError();
+    g.ok = okk;
+  }
   e->tab.slots = e->dp<TSlot>(L.tab); e->tab.mask = c.table_capacity - 1;
   e->tab.shift = 64 - (bit_length(c.table_capacity) - 1);
   e->ent.key = e->dp<u64>(L.e_key); e->ent.stamp = e->dp<u32>(L.e_stamp); e->ent.depth = e->dp<u32>(L.e_depth);
@@ -754,6 +886,14 @@ int32_t kvt_destroy(kvt_engine *e) {
   cudaDeviceSynchronize();
   for (auto &m : e->sel_graph) for (auto &g : m) if (g.second.exec) cudaGraphExecDestroy(g.second.exec);
   if (e->capture_stream) cudaStreamDestroy(e->capture_stream);
+  for (int d = 0; d < 2; ++d) {
+    if (e->stg.cs[d]) cudaStreamDestroy(e->stg.cs[d]);
+    for (int k = 0; k < kvt_engine::N_STAGES; ++k) {
+      if (e->stg.ready[d][k]) cudaEventDestroy(e->stg.ready[d][k]);
+      if (e->stg.free_[d][k]) cudaEventDestroy(e->stg.free_[d][k]);
+    }
+  }
+  if (e->stg.begin) cudaEventDestroy(e->stg.begin);
   if (e->ev_upload) cudaEventDestroy(e->ev_upload);
   if (e->ev_m0) cudaEventDestroy(e->ev_m0);
   if (e->ev_m1) cudaEventDestroy(e->ev_m1);
@@ -778,7 +918,7 @@ int32_t kvt_set_profiling(kvt_engine *e, uint32_t on) {
 
 int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant) {
   if (!e) return KVT_E_INVAL;
-  if (variant > 3) return KVT_E_INVAL;
+  if (variant > 4) return KVT_E_INVAL;
   e->mover_variant = variant;
   return KVT_OK;
 }
@@ -1508,14 +1648,26 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
   KL(k_list_apply, g, 256, s, a);
   KL(k_list_unmark, g, 256, s, a);
   LAUNCH_CHECK();
-  if (!m.drop_all) {
-    r = launch_mover(e, s, src_tier, a.pair_src, dst_tier, a.pair_dst, std::min(n, a.n_free), e->d_status + ST_NLIVE);
+  const bool staged = !m.drop_all && staged_applies(e, src_tier, dst_tier);
+  const u32 n_pairs_max = std::min(n, a.n_free);
+  u32 *h_psrc = (u32 *)e->h_out, *h_pdst = h_psrc + e->L.LB;
+  if (!m.drop_all && !staged) {
+    r = launch_mover(e, s, src_tier, a.pair_src, dst_tier, a.pair_dst, n_pairs_max, e->d_status + ST_NLIVE);
     if (r) return r;
+  }
+  if (staged && n_pairs_max) {   // the copy-engine transfers are issued from the host: it needs the planned pairs
+    CU(cudaMemcpyAsync(h_psrc, a.pair_src, n_pairs_max * 4ull, cudaMemcpyDeviceToHost, s));
+    CU(cudaMemcpyAsync(h_pdst, a.pair_dst, n_pairs_max * 4ull, cudaMemcpyDeviceToHost, s));
   }
   r = status_fetch(e, s);
   if (r) return r;
   r = status_code(e);
   if (r) return r;
+  if (staged && e->h_status[ST_NLIVE]) {
+    r = staged_move(e, s, src_tier, a.pair_src, h_psrc, dst_tier, a.pair_dst, h_pdst, std::min(e->h_status[ST_NLIVE], n_pairs_max));
+    if (r) return r;
+    CU(cudaStreamSynchronize(s));
+  }
   out->copied = e->h_status[ST_NLIVE];
   out->dropped = e->h_status[ST_NDROP];
   out->clean = e->h_status[ST_NCLEAN];

@@ -1494,7 +1494,7 @@ __global__ void __launch_bounds__(256) k_move_blocks(MoveArgs a) {
   const u32 vec_per_chunk = a.chunk_bytes >> 4;
   for (u64 item = blockIdx.x; item < n_items; item += gridDim.x) {
     u32 pair = (u32)(item / a.n_chunks), chunk = (u32)(item % a.n_chunks);
-    u32 s = a.src_ids[pair], d = a.dst_ids[pair];
+    u32 s = a.src_ids ? a.src_ids[pair] : pair, d = a.dst_ids ? a.dst_ids[pair] : pair;   // no list: the pair's own index
     if (s >= a.src.n_slots || d >= a.dst.n_slots) { if (threadIdx.x == 0) set_err(a.status, DERR_RANGE); continue; }
     const uint4 *sp = reinterpret_cast<const uint4 *>(a.src.base + s * a.src.slot_stride + chunk * a.src.chunk_stride);
     uint4 *dp = reinterpret_cast<uint4 *>(a.dst.base + d * a.dst.slot_stride + chunk * a.dst.chunk_stride);
@@ -1529,7 +1529,7 @@ __global__ void __launch_bounds__(THREADS) k_move_tiles(MoveArgs a, u32 tiles_pe
     u32 pair = (u32)(item / per_pair);
     u32 rem = (u32)(item - (u64)pair * per_pair);
     u32 chunk = rem / tiles_per_chunk, tile = rem - chunk * tiles_per_chunk;
-    u32 s = a.src_ids[pair], d = a.dst_ids[pair];
+    u32 s = a.src_ids ? a.src_ids[pair] : pair, d = a.dst_ids ? a.dst_ids[pair] : pair;   // no list: the pair's own index
     if (s >= a.src.n_slots || d >= a.dst.n_slots) { if (lane == 0) set_err(a.status, DERR_RANGE); continue; }
     const uint4 *sp = reinterpret_cast<const uint4 *>(a.src.base + s * a.src.slot_stride + chunk * a.src.chunk_stride) +
                       (u64)tile * 32 * UNROLL + lane;

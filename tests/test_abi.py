@@ -23,7 +23,7 @@ def test_query_sizes_needs_no_gpu():
     from paper_2609_39819_b200 import binding
     lib = binding.load_library()
     cfg = binding.Config()
-    cfg.abi_version, cfg.block_tokens = 2, 16
+    cfg.abi_version, cfg.block_tokens = 3, 16
     cfg.n_layers, cfg.n_kv_heads, cfg.head_dim, cfg.elem_bytes = 2, 2, 64, 2
     cfg.n_hbm_blocks, cfg.n_host_blocks, cfg.table_capacity = 128, 512, 2048
     cfg.max_contexts, cfg.max_messages, cfg.max_batch_blocks = 64, 1024, 4096
@@ -37,7 +37,7 @@ def test_query_sizes_needs_no_gpu():
 
 def test_struct_sizes_match_the_header():
     from paper_2609_39819_b200 import binding
-    assert ctypes.sizeof(binding.Config) == 14 * 4 + 3 * 8 + 2 * 4 + 10 * 8
+    assert ctypes.sizeof(binding.Config) == 14 * 4 + 3 * 8 + 2 * 4 + 12 * 8
     assert ctypes.sizeof(binding.Op) == 8 * 4 + 8
     assert binding.CALL_INFO_DTYPE.itemsize == 9 * 4
 

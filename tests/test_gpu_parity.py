@@ -631,6 +631,53 @@ def test_mover_with_second_tier_in_hbm(B, oracle):
     del gpu, cpu
 
 
+@pytest.mark.parametrize("geo,stage_mib", [(W.GEO_TOY, 1), (W.GEO_128K, 2), (W.GEO_8B, 64)], ids=["toy", "128K", "8B"])
+@pytest.mark.parametrize("layout", [0, 1])
+def test_moves_through_the_staging_ring_are_byte_exact(B, oracle, geo, stage_mib, layout):
+    """Offload, reload and the moves to and from a third tier with the copy engines carrying the payload: the mover
+    kernel gathers whole blocks into the staging ring (scatters them out of it) and the link sees large transfers.
+    The ring is sized so that the lists wrap around it several times; lists are permuted, so transfers of one block
+    and of several consecutive host slots both occur. Same results as the oracle, every byte checked."""
+    n = 96
+    kw = dict(n_hbm_blocks=n, n_host_blocks=n, n_remote_blocks=n // 2, max_contexts=4, pool_layout=layout, **geo.kwargs())
+    gpu = B.Engine(max_tokens=1 << 16, max_messages=256, stage_mib=stage_mib, **kw)
+    gpu.set_mover_variant(4)
+    cpu = oracle.OracleEngine(**kw)
+    rng = np.random.default_rng(5)
+    tok = rng.integers(0, W.VOCAB, 16 * n, dtype=np.uint32)
+    for eng in (gpu, cpu):
+        eng.spawn(0); eng.append(0, tok)
+        eng.map_blocks([0], 0); eng.map_blocks([0], 1); eng.prefill_done(0)
+    keys = cpu.get_block_map(0)[0]
+    for b in range(n):
+        gpu.fill_block_pattern(0, b, int(keys[b]))
+
+    def same_maps():
+        for a, b in zip(gpu.get_block_map(0), cpu.get_block_map(0)):
+            assert np.array_equal(a, b)
+        _k, tier, slot = cpu.get_block_map(0)
+        bad = [b for b in range(n) if tier[b] != 0xFF and not gpu.check_block_pattern(int(tier[b]), int(slot[b]), int(keys[b]))]
+        assert not bad, bad[:8]
+
+    out = rng.permutation(n)[: 3 * n // 4].astype(np.uint32)
+    assert gpu.offload(out) == cpu.offload(out)
+    same_maps()
+    back = rng.permutation(3 * n // 4)[: n // 2].astype(np.uint32)                     # host slots, in any order
+    assert gpu.reload(back) == cpu.reload(back)
+    same_maps()
+    host_occ = np.nonzero(cpu.get_entries(1)["key"])[0].astype(np.uint32)
+    down = rng.permutation(host_occ)
+    assert gpu.move(1, 2, down) == cpu.move(1, 2, down)                                # host -> remote: both in host memory
+    same_maps()
+    up = rng.permutation(len(down)).astype(np.uint32)[: len(down) // 2]
+    assert gpu.move(2, 0, up) == cpu.move(2, 0, up)                                    # remote -> HBM through the ring
+    same_maps()
+    sg, sc = gpu.get_stats(), cpu.get_stats()
+    for k in sc:
+        if k not in W.GPU_ONLY_STATS:
+            assert sg[k] == sc[k], k
+
+
 @pytest.mark.parametrize("ctas", [1, 3, 64])
 @pytest.mark.parametrize("on_device", [False, True], ids=["pinned-host-tier", "second-tier-in-hbm"])
 def test_mover_grid_limit_does_not_change_results(B, ctas, on_device):
