@@ -930,7 +930,7 @@ int32_t kvt_set_mover_ctas(kvt_engine *e, uint32_t max_ctas) {
 }
 
 int32_t kvt_debug_set_lookup_variant(kvt_engine *e, uint32_t variant) {
-  if (!e || variant > 2) return KVT_E_INVAL;
+  if (!e || variant > 4) return KVT_E_INVAL;
   e->lookup_variant = variant;
   return KVT_OK;
 }
@@ -1245,7 +1245,11 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     if (e->lookup_variant != 2) {
       if (dchunk_base) KL(k_hash_digest, dchunk_base, CHUNK, s, ha);
       KL(k_hash_carry, nd, 1024, s, ha);
-      KL(k_hash_finish_lookup, chunk_base, CHUNK, s, ha, la);
+      // one key per thread by default; two or four (more table loads in flight per thread) measured the same: the
+      // probes of a cold table are bound by the rate of random 32-byte sectors, not by latency per thread
+      if (e->lookup_variant == 3) KL(k_hash_finish_lookup<2>, chunk_base, CHUNK / 2, s, ha, la);
+      else if (e->lookup_variant == 4) KL(k_hash_finish_lookup<4>, chunk_base, CHUNK / 4, s, ha, la);
+      else KL(k_hash_finish_lookup<1>, chunk_base, CHUNK, s, ha, la);
     } else {
       ChainState cs;
       cs.flags = e->dp<u32>(e->L.cflags); cs.ticket = cs.flags + chunk_base; cs.incl = e->dp<u64>(e->L.carry);
@@ -1946,7 +1950,7 @@ int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t ha
   LookupArgs la{};
   k_hash_digest<<<n_chunks, CHUNK, 0, s>>>(ha);
   k_hash_carry<<<1, 1024, 0, s>>>(ha);
-  k_hash_finish_lookup<<<n_chunks, CHUNK, 0, s>>>(ha, la);
+  k_hash_finish_lookup<1><<<n_chunks, CHUNK, 0, s>>>(ha, la);
   return cudaGetLastError() == cudaSuccess ? KVT_OK : KVT_E_CUDA;
 }
 
@@ -1979,7 +1983,7 @@ int32_t kvt_hash_tokens_noalloc(const uint32_t *d_tokens, uint64_t n_tokens, uin
   LookupArgs la{};
   k_hash_digest<<<n_chunks, CHUNK, 0, s>>>(ha);
   k_hash_carry<<<1, 1024, 0, s>>>(ha);
-  k_hash_finish_lookup<<<n_chunks, CHUNK, 0, s>>>(ha, la);
+  k_hash_finish_lookup<1><<<n_chunks, CHUNK, 0, s>>>(ha, la);
   return cudaGetLastError() == cudaSuccess ? KVT_OK : KVT_E_CUDA;
 }
 

@@ -324,40 +324,86 @@ struct LookupArgs {
   u32 *status;
 };
 
-__global__ void __launch_bounds__(CHUNK) k_hash_finish_lookup(HashArgs a, LookupArgs l) {
+// Read-only probes of ILP keys at once: the first two slots of every key are fetched before any of them is looked
+// at (2 * ILP independent 16-byte loads in flight per thread), later steps only for the keys still unresolved.
+template <int ILP>
+__device__ __forceinline__ void tab_lookup_ents(const Table &t, const u64 (&key)[ILP], const bool (&active)[ILP], u32 (&ent)[ILP],
+                                                u32 *status) {
+  u32 i[ILP];
+  bool open[ILP];
+  bool any = false;
+#pragma unroll
+  for (int q = 0; q < ILP; ++q) { i[q] = (u32)(key[q] >> t.shift); open[q] = active[q]; ent[q] = ENT_NONE; any = any || open[q]; }
+  for (u32 n = 0; any && n <= t.mask; n += 2) {
+    uint4 a[ILP], b[ILP];
+#pragma unroll
+    for (int q = 0; q < ILP; ++q)
+      if (open[q]) {
+        a[q] = __ldg(reinterpret_cast<const uint4 *>(t.slots + i[q]));
+        b[q] = __ldg(reinterpret_cast<const uint4 *>(t.slots + ((i[q] + 1) & t.mask)));
+      }
+    any = false;
+#pragma unroll
+    for (int q = 0; q < ILP; ++q)
+      if (open[q]) {
+        const u64 ka = (u64)a[q].x | ((u64)a[q].y << 32), kb = (u64)b[q].x | ((u64)b[q].y << 32);
+        if (ka == key[q]) { ent[q] = a[q].z; open[q] = false; }
+        else if (ka == KEY_EMPTY) open[q] = false;
+        else if (kb == key[q]) { ent[q] = b[q].z; open[q] = false; }
+        else if (kb == KEY_EMPTY) open[q] = false;
+        else { i[q] = (i[q] + 2) & t.mask; any = true; }
+      }
+  }
+  if (any) set_err(status, DERR_PROBE);
+}
+
+// One CTA of CHUNK / ILP threads per 256-block chunk; thread t finishes and probes blocks t, t + CHUNK / ILP, ...
+template <int ILP>
+__global__ void __launch_bounds__(CHUNK / ILP) k_hash_finish_lookup(HashArgs a, LookupArgs l) {
+  constexpr u32 T = CHUNK / ILP;
   const u32 tid = threadIdx.x;
   u32 ci;
   const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci);
   const u32 b0 = (blockIdx.x - c.chunk_base) * CHUNK;
   const u32 nb = min(CHUNK, c.n_blocks - b0);
-  u32 miss = 0xFFFFFFFFu;
-  if (tid < nb) {
-    u64 key;
-    if (b0 < c.first) {          // unchanged prefix: the key of the previous list still holds
-      key = a.keys[c.old_key_off + b0 + tid];
-    } else {
-      u64 h = g_pow_p.v[tid + 1] * a.carry_base[c.carry_off + (blockIdx.x - c.chunk_base)] + a.keys[c.key_off + b0 + tid];
-      key = mix64(h);
-      if (key < 2) key += 2;
-    }
-    a.keys[c.key_off + b0 + tid] = key;
-    if (l.tab.slots) {
-      u32 ent = tab_lookup_ent(l.tab, key, l.status);
-      l.b_ent[c.blk_base + b0 + tid] = ent;
-      if (ent == ENT_NONE) miss = b0 + tid;
+  u64 key[ILP];
+  bool act[ILP];
+  const bool kept = b0 < c.first;                                   // unchanged prefix: the keys of the previous list still hold
+  const u64 carry = kept ? 0 : a.carry_base[c.carry_off + (blockIdx.x - c.chunk_base)];
+#pragma unroll
+  for (int q = 0; q < ILP; ++q) {
+    const u32 j = tid + q * T;
+    act[q] = j < nb;
+    key[q] = 0;
+    if (act[q]) {
+      if (kept) key[q] = a.keys[c.old_key_off + b0 + j];
+      else {
+        key[q] = mix64(g_pow_p.v[j + 1] * carry + a.keys[c.key_off + b0 + j]);
+        if (key[q] < 2) key[q] += 2;
+      }
+      a.keys[c.key_off + b0 + j] = key[q];
     }
   }
+  if (!l.tab.slots) return;
+  u32 ent[ILP];
+  tab_lookup_ents<ILP>(l.tab, key, act, ent, l.status);
+  u32 miss = 0xFFFFFFFFu;
+#pragma unroll
+  for (int q = 0; q < ILP; ++q)
+    if (act[q]) {
+      const u32 j = tid + q * T;
+      l.b_ent[c.blk_base + b0 + j] = ent[q];
+      if (ent[q] == ENT_NONE) miss = min(miss, b0 + j);
+    }
   // first miss of the CTA -> the context's reusable prefix length: warp minima meet in shared memory, one global
   // atomic per CTA that saw a miss
-  if (l.tab.slots) {
-    __shared__ u32 s_min;
-    if (tid == 0) s_min = 0xFFFFFFFFu;
-    __syncthreads();
-    miss = __reduce_min_sync(0xFFFFFFFFu, miss);
-    if ((tid & 31) == 0 && miss != 0xFFFFFFFFu) atomicMin(&s_min, miss);
-    __syncthreads();
-    if (tid == 0 && s_min != 0xFFFFFFFFu) atomicMin(&l.hit_len[ci], s_min);
-  }
+  __shared__ u32 s_min;
+  if (tid == 0) s_min = 0xFFFFFFFFu;
+  __syncthreads();
+  miss = __reduce_min_sync(0xFFFFFFFFu, miss);
+  if ((tid & 31) == 0 && miss != 0xFFFFFFFFu) atomicMin(&s_min, miss);
+  __syncthreads();
+  if (tid == 0 && s_min != 0xFFFFFFFFu) atomicMin(&l.hit_len[ci], s_min);
 }
 
 // ------------------------------------------------------------------------------------------------------
