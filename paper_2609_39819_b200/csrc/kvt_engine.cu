@@ -504,6 +504,108 @@ int32_t staged_move(kvt_engine *e, cudaStream_t s, u32 st, const u32 *d_src, con
   return KVT_OK;
 }
 
+// Both directions at once through the staging ring: victims (HBM -> host) are gathered and sent on copy stream 0,
+// reloads (host -> HBM) arrive and are scattered on copy stream 1, so both copy engines work. A reload may land in
+// the HBM slot a victim of the same call leaves; payload copies are independent of the list order, so the victims
+// are gathered in the order the reload batches need their slots, and the scatter of a batch waits for the gather
+// of the last victim it depends on. All lists are host copies of what the plan kernels produced; in_dst stays on
+// the device (d_in_dst). When this returns, `s` waits for both copy streams.
+int32_t staged_exchange(kvt_engine *e, cudaStream_t s, u32 n_in, const u32 *in_src, const u32 *in_dst, const u32 *d_in_dst,
+                        u32 n_out, const u32 *out_src, const u32 *out_dst) {
+  kvt_engine::Staging &g = e->stg;
+  const u32 SB = g.blocks_per_stage;
+  const u64 BB = e->block_bytes;
+  const u32 NS = kvt_engine::N_STAGES;
+  for (u32 i = 0; i < n_in; ++i) if (in_src[i] >= e->cfg.n_host_blocks) return fail(e, KVT_E_RANGE, "slot id out of range");
+  for (u32 i = 0; i < n_out; ++i) if (out_dst[i] >= e->cfg.n_host_blocks) return fail(e, KVT_E_RANGE, "slot id out of range");
+  const u32 nbi = cdiv(n_in, SB), nbo = cdiv(n_out, SB);
+  // order of the victims: those whose slots the first reload batches need come first
+  std::map<u32, u32> vic_of;
+  for (u32 v = 0; v < n_out; ++v) vic_of[out_src[v]] = v;
+  std::vector<u32> order; order.reserve(n_out);
+  std::vector<char> taken(n_out, 0);
+  std::vector<u32> need(nbi, 0);
+  for (u32 j = 0; j < nbi; ++j) {
+    for (u32 r = j * SB; r < std::min(n_in, (j + 1) * SB); ++r) {
+      auto it = vic_of.find(in_dst[r]);
+      if (it != vic_of.end() && !taken[it->second]) { taken[it->second] = 1; order.push_back(it->second); }
+    }
+    need[j] = (u32)order.size();
+  }
+  for (u32 v = 0; v < n_out; ++v) if (!taken[v]) order.push_back(v);
+  // device lists: victims' HBM slots in that order, and the place of every block inside its batch's stage (blocks
+  // sit in the order of their host slots, so that consecutive host slots are one transfer)
+  u32 *h_osrc = e->h_ids, *h_opos = e->h_ids2, *h_ipos = (u32 *)e->h_out;
+  u32 *d_osrc = e->dp<u32>(e->L.ids), *d_opos = e->dp<u32>(e->L.ids2), *d_ipos = e->dp<u32>(e->L.s0);
+  std::vector<u32> ohost(n_out), isorted(n_in), osorted(n_out), idx(SB);
+  for (u32 i = 0; i < n_out; ++i) { h_osrc[i] = out_src[order[i]]; ohost[i] = out_dst[order[i]]; }
+  auto place = [&](const u32 *slots, u32 n, u32 *pos, std::vector<u32> &sorted) {
+    for (u32 b0 = 0; b0 < n; b0 += SB) {
+      const u32 nb = std::min(SB, n - b0);
+      for (u32 i = 0; i < nb; ++i) idx[i] = i;
+      std::sort(idx.begin(), idx.begin() + nb, [&](u32 x, u32 y) { return slots[b0 + x] < slots[b0 + y]; });
+      for (u32 p = 0; p < nb; ++p) { pos[b0 + idx[p]] = p; sorted[b0 + p] = slots[b0 + idx[p]]; }
+    }
+  };
+  std::vector<u32> in_src_copy(in_src, in_src + n_in);   // in_src lives in the staging area h_ipos is about to reuse
+  place(ohost.data(), n_out, h_opos, osorted);
+  place(in_src_copy.data(), n_in, h_ipos, isorted);
+  if (n_out) {
+    CU(cudaMemcpyAsync(d_osrc, h_osrc, n_out * 4ull, cudaMemcpyHostToDevice, s));
+    CU(cudaMemcpyAsync(d_opos, h_opos, n_out * 4ull, cudaMemcpyHostToDevice, s));
+  }
+  if (n_in) CU(cudaMemcpyAsync(d_ipos, h_ipos, n_in * 4ull, cudaMemcpyHostToDevice, s));
+  {
+    int32_t r = stage_release(e, s);
+    if (r) return r;
+  }
+  const bool timed = e->profiling;
+  if (timed) CU(cudaEventRecord(e->ev_m0, s));
+  CU(cudaEventRecord(g.begin, s));
+  CU(cudaStreamWaitEvent(g.cs[0], g.begin, 0));
+  CU(cudaStreamWaitEvent(g.cs[1], g.begin, 0));
+  u8 *host_pool = (u8 *)e->cfg.host_pool;
+  auto transfers = [&](int dir, const std::vector<u32> &sorted, u32 b0, u32 nb, u8 *stage) -> int32_t {
+    for (u32 p = 0; p < nb;) {
+      u32 run = 1;
+      while (p + run < nb && sorted[b0 + p + run] == sorted[b0 + p] + run) ++run;
+      u8 *hp = host_pool + (u64)sorted[b0 + p] * BB, *sp = stage + (u64)p * BB;
+      if (dir == 0) CU(cudaMemcpyAsync(hp, sp, run * BB, cudaMemcpyDeviceToHost, g.cs[0]));
+      else CU(cudaMemcpyAsync(sp, hp, run * BB, cudaMemcpyHostToDevice, g.cs[1]));
+      p += run;
+    }
+    return KVT_OK;
+  };
+  auto issue_out = [&](u32 k) -> int32_t {   // gather + transfers of victim batch k, in order on copy stream 0
+    const u32 b0 = k * SB, nb = std::min(SB, n_out - b0);
+    const int sg = (int)(k % NS);
+    int32_t r = launch_mover_views(e, g.cs[0], pool_view(e, KVT_TIER_HBM), d_osrc + b0, stage_view(e, 0, sg, nb), d_opos + b0, nb,
+                                   nullptr, 0, false);
+    if (r) return r;
+    CU(cudaEventRecord(g.ready[0][sg], g.cs[0]));
+    return transfers(0, osorted, b0, nb, stage_view(e, 0, sg, nb).base);
+  };
+  u32 ko = 0;
+  for (u32 j = 0; j < nbi; ++j) {
+    while (ko < nbo && ko * SB < need[j]) { int32_t r = issue_out(ko++); if (r) return r; }
+    const u32 b0 = j * SB, nb = std::min(SB, n_in - b0);
+    const int sg = (int)(j % NS);
+    int32_t r = transfers(1, isorted, b0, nb, stage_view(e, 1, sg, nb).base);
+    if (r) return r;
+    if (need[j]) CU(cudaStreamWaitEvent(g.cs[1], g.ready[0][(ko - 1) % NS], 0));   // the victims in the way have been gathered
+    r = launch_mover_views(e, g.cs[1], stage_view(e, 1, sg, nb), d_ipos + b0, pool_view(e, KVT_TIER_HBM), d_in_dst + b0, nb, nullptr, 0,
+                           false);
+    if (r) return r;
+  }
+  while (ko < nbo) { int32_t r = issue_out(ko++); if (r) return r; }
+  CU(cudaEventRecord(g.free_[0][0], g.cs[0]));
+  CU(cudaEventRecord(g.free_[1][0], g.cs[1]));
+  CU(cudaStreamWaitEvent(s, g.free_[0][0], 0));
+  CU(cudaStreamWaitEvent(s, g.free_[1][0], 0));
+  if (timed) { CU(cudaEventRecord(e->ev_m1, s)); e->mover_timed = true; }
+  return KVT_OK;
+}
+
 // After the stream has been synchronised: adds the timed mover kernel to the statistics.
 void mover_account(kvt_engine *e, u64 blocks) {
   if (!e->mover_timed) return;
@@ -1801,8 +1903,34 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
     KL(k_list_unmark, ga, 256, s, a);
   }
   LAUNCH_CHECK();
+  const bool staged = staged_applies(e, KVT_TIER_HBM, KVT_TIER_HOST);
+  if (staged) {   // copy engines, both directions: the transfers are issued from the host, which needs the planned pairs
+    u32 *h_isrc = (u32 *)e->h_out, *h_idst = h_isrc + e->L.LB, *h_osrc = h_idst + e->L.LB, *h_odst = h_osrc + e->L.LB;
+    const u32 n_out_max = std::min(n_out, b.n_free);
+    if (n_in) {
+      CU(cudaMemcpyAsync(h_isrc, a.pair_src, n_in * 4ull, cudaMemcpyDeviceToHost, s));
+      CU(cudaMemcpyAsync(h_idst, a.pair_dst, n_in * 4ull, cudaMemcpyDeviceToHost, s));
+    }
+    if (n_out_max) {
+      CU(cudaMemcpyAsync(h_osrc, b.pair_src, n_out_max * 4ull, cudaMemcpyDeviceToHost, s));
+      CU(cudaMemcpyAsync(h_odst, b.pair_dst, n_out_max * 4ull, cudaMemcpyDeviceToHost, s));
+    }
+    r = status_fetch(e, s);
+    if (r) return r;
+    r = status_code(e);
+    if (r) return r;
+    const u32 ni = std::min(e->h_status[ST_NLIVE], n_in), no = std::min(e->h_status[ST_B_NLIVE], n_out_max);
+    if (ni + no) {
+      std::vector<u32> v_idst(h_idst, h_idst + ni), v_osrc(h_osrc, h_osrc + no), v_odst(h_odst, h_odst + no);   // the staging area is reused
+      r = stage_acquire(e);
+      if (r) return r;
+      r = staged_exchange(e, s, ni, h_isrc, v_idst.data(), a.pair_dst, no, v_osrc.data(), v_odst.data());
+      if (r) return r;
+      CU(cudaStreamSynchronize(s));
+    }
+  }
   // one mover launch for both directions
-  if (!e->metadata_only) {
+  if (!e->metadata_only && !staged) {
     MoveArgs ma{}, mb{};
     ma.src = pool_view(e, KVT_TIER_HOST); ma.dst = pool_view(e, KVT_TIER_HBM); ma.src_ids = a.pair_src; ma.dst_ids = a.pair_dst;
     ma.n_pairs = n_in; ma.n_pairs_dev = e->d_status + ST_NLIVE;
@@ -1840,10 +1968,12 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
       LAUNCH_CHECK();
     }
   }
-  r = status_fetch(e, s);
-  if (r) return r;
-  r = status_code(e);
-  if (r) return r;
+  if (!staged) {
+    r = status_fetch(e, s);
+    if (r) return r;
+    r = status_code(e);
+    if (r) return r;
+  }
   const u32 *h = e->h_status;
   const u32 in_copied = h[ST_NLIVE], out_copied = h[ST_B_NLIVE], out_drop = h[ST_B_NDROP], out_clean = h[ST_B_NCLEAN];
   mover_account(e, (u64)in_copied + out_copied);

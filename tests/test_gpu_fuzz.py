@@ -19,8 +19,10 @@ def test_random_api_streams_match_the_oracle(oracle, seed, flags, pools):
     from paper_2609_39819_b200 import binding as B
     kw = dict(n_hbm_blocks=pools[0], n_host_blocks=pools[1], max_contexts=6, policy_flags=flags, suspended_order=seed % 2,
               pool_layout=seed % 2, **W.GEO_TOY.kwargs())
-    gpu = B.Engine(max_tokens=1 << 16, max_messages=2048, **kw)
+    gpu = B.Engine(max_tokens=1 << 16, max_messages=2048, stage_mib=1, **kw)
     gpu.set_classify_mode((2, 1, 0)[seed % 3])    # event-driven counts cross-checked / recomputed in full / on their own
+    if seed % 2:
+        gpu.set_mover_variant(4)                  # payload through the staging ring and the copy engines (8 blocks per stage)
     cpu = oracle.OracleEngine(**kw)
     F.run([gpu, cpu], seed, steps=300, inclusive=bool(flags & 2), check_every=10)
 
@@ -57,7 +59,9 @@ def test_random_api_streams_with_three_tiers(oracle, seed, flags, pools):
     from paper_2609_39819_b200 import binding as B
     kw = dict(n_hbm_blocks=pools[0], n_host_blocks=pools[1], n_remote_blocks=pools[2], max_contexts=6, policy_flags=flags,
               suspended_order=seed % 2, pool_layout=seed % 2, **W.GEO_TOY.kwargs())
-    gpu = B.Engine(max_tokens=1 << 16, max_messages=2048, **kw)
+    gpu = B.Engine(max_tokens=1 << 16, max_messages=2048, stage_mib=1, **kw)
     gpu.set_classify_mode((2, 1, 0)[seed % 3])    # event-driven counts cross-checked / recomputed in full / on their own
+    if seed % 2:
+        gpu.set_mover_variant(4)                  # payload through the staging ring and the copy engines (8 blocks per stage)
     cpu = oracle.OracleEngine(**kw)
     F.run([gpu, cpu], seed, steps=300, inclusive=bool(flags & 2), check_every=10)

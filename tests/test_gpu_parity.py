@@ -672,10 +672,43 @@ def test_moves_through_the_staging_ring_are_byte_exact(B, oracle, geo, stage_mib
     up = rng.permutation(len(down)).astype(np.uint32)[: len(down) // 2]
     assert gpu.move(2, 0, up) == cpu.move(2, 0, up)                                    # remote -> HBM through the ring
     same_maps()
+    # both directions in one call, on a full HBM tier: every reload lands in a slot a victim is leaving
+    for eng in (gpu, cpu):
+        eng.spawn(1); eng.append(1, tok[::-1].copy())
+        eng.map_blocks([1], 0)
+        eng.map_blocks([1], 1); eng.prefill_done(1)
+    st = cpu.get_stats()
+    assert st["occ_hbm"] == n                                                          # context 1 filled what was free
+    keys1 = cpu.get_block_map(1)[0]
+    _k, t1, s1 = cpu.get_block_map(1)
+    for b in range(len(keys1)):
+        if t1[b] == 0:
+            gpu.fill_block_pattern(0, int(s1[b]), int(keys1[b]))
+    host_occ = np.nonzero(cpu.get_entries(1)["key"])[0].astype(np.uint32)
+    ins = rng.permutation(host_occ)[: max(1, len(host_occ) // 2)]
+    vg, _ = gpu.select_victims(0, len(ins) + 5)
+    vc, _ = cpu.select_victims(0, len(ins) + 5)
+    assert np.array_equal(vg, vc)
+    assert gpu.exchange(vg, ins) == cpu.exchange(vc, ins)
+    same_maps()
+    _k, t1, s1 = cpu.get_block_map(1)
+    bad = [b for b in range(len(keys1)) if t1[b] != 0xFF and not gpu.check_block_pattern(int(t1[b]), int(s1[b]), int(keys1[b]))]
+    assert not bad, bad[:8]
     sg, sc = gpu.get_stats(), cpu.get_stats()
     for k in sc:
         if k not in W.GPU_ONLY_STATS:
             assert sg[k] == sc[k], k
+
+
+def test_exchange_scenario_through_the_staging_ring(B):
+    def make(**k):
+        eng = B.Engine(max_tokens=1 << 16, max_messages=256, stage_mib=1, **k)
+        eng.set_mover_variant(4)
+        return eng
+    S.exchange_both_ways(make)
+    S.offload_reload_round_trip(make)
+    S.inclusive_tiers(make)
+    S.three_tiers(make)
 
 
 @pytest.mark.parametrize("ctas", [1, 3, 64])
