@@ -40,10 +40,20 @@ from paper_2609_39819_b200 import workloads as W  # noqa: E402
 
 METRIC = "KV block GB/s (HBM & host link) vs roofline; blocks hashed+looked up/sec"
 GiB = 1 << 30
-# DRAM traffic of the mover kernel per algorithmic byte (read + write), from one ncu capture (its summary sits
-# with the other profile summaries of this repository): (dram__bytes_read.sum + dram__bytes_write.sum) /
-# (2 x payload bytes) of a 1024-block launch; traffic grows in proportion to the blocks moved, so it is scaled to the bench's launches.
-MOVER_TRAFFIC_PER_ALGO_BYTE = 0.989
+
+
+def mover_traffic_ratio():
+    """DRAM traffic of the mover kernel per algorithmic byte (read + write), taken from the tracked summary of its
+    ncu capture: (dram__bytes_read.sum + dram__bytes_write.sum) / (2 x payload bytes) of a 1024-block launch, the
+    row "traffic / algorithmic" of the summary's counter table. Traffic grows in proportion to the blocks moved, so
+    the ratio is scaled to the bench's launches. None if the summary is missing."""
+    import re
+    try:
+        text = open(os.path.join(ROOT, "profiles", "mover_8b_hbm_to_hbm.md")).read()
+    except OSError:
+        return None
+    m = re.search(r"^\|\s*traffic / algorithmic\s*\|\s*([0-9.]+)\s*\|", text, flags=re.M)
+    return float(m.group(1)) if m else None
 
 
 def parse_args():
@@ -61,6 +71,8 @@ def parse_args():
     ap.add_argument("--skip-stress", action="store_true", help="skip the C4-shaped metadata measurement")
     ap.add_argument("--skip-inclusive", action="store_true", help="skip the extra end-to-end run with inclusive tiers")
     ap.add_argument("--skip-two-tenants", action="store_true", help="skip the extra end-to-end run with two sessions")
+    ap.add_argument("--skip-c3", action="store_true", help="skip the C3 arm (32 sessions, GLM-scale blocks, 120 GiB pool)")
+    ap.add_argument("--c3-host-gib", type=float, default=48.0, help="pinned host tier of the C3 arm")
     return ap.parse_args()
 
 
@@ -513,6 +525,116 @@ def two_tenant_arm(args, torch, B, n_ff, use_exchange, n_hbm_blocks=12288, n_hos
     return out
 
 
+def c3_arm(args, torch, B, link):
+    """C3 at full size, as a timed run: 32 concurrent agent sessions with subagents (32 K - 258 K tokens each,
+    ~216 K blocks of demand), GLM-scale KV (92 x 8 x 128 bf16, 5.75 MiB per block), HBM pool 120 GiB = 21,370
+    blocks, pinned host tier. No pressure is added: the sessions do not fit, so every round evicts in the engine's
+    victim order, offloads what is live, drops what is dead and reloads prefixes on the sessions' next calls. Tokens
+    come from pageable host arrays through the C ABI; payload bytes are whatever the pools hold (the movement is
+    real, the content is not produced). The whole trace is timed with the wall clock (every call synchronises)."""
+    import gc
+    gc.collect()
+    torch.cuda.empty_cache()
+    if hasattr(torch._C, "_host_emptyCache"):
+        torch._C._host_emptyCache()
+    geo = W.GEO_GLM
+    free_b, _ = torch.cuda.mem_get_info()
+    n_hbm = min(21370, int((free_b - 8 * GiB) // geo.block_bytes))
+    n_host = min(int(args.c3_host_gib * GiB), int(mem_available_bytes() * 0.4)) // geo.block_bytes
+    if n_hbm < 4000 or n_host < 1000:
+        return {"skipped": f"needs memory: {n_hbm} HBM blocks, {n_host} host blocks possible"}
+    trace, n_ctx = W.trace_c3(args.seed)
+    eng = B.Engine(n_hbm_blocks=n_hbm, n_host_blocks=n_host, max_contexts=n_ctx, max_tokens=1 << 24, max_messages=1 << 16,
+                   zero_pools=False, **geo.kwargs())
+    eng.set_profiling(True)
+    opt = W.ReplayOptions(payload=None, record_states=False)
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    n_calls = 0
+    for _i, kind, _rec in W.replay(eng, trace, opt):
+        n_calls += kind == "call"
+    torch.cuda.synchronize()
+    sec = time.perf_counter() - t0
+    st = eng.get_stats()
+    moved = (st["offloaded"] - st["offloaded_clean"] + st["reloaded"]) * eng.block_bytes
+    mover_s = st["mover_ns"] / 1e9
+    out = {
+        "workload": f"C3: 32 sessions + subagents, seed {args.seed}, {n_calls} batched calls, GLM-scale blocks of "
+                    f"{eng.block_bytes} B, HBM pool {n_hbm} blocks ({n_hbm * eng.block_bytes / GiB:.0f} GiB), pinned host "
+                    f"tier {n_host} blocks ({n_host * eng.block_bytes / GiB:.0f} GiB); natural pressure only",
+        "value": moved / sec / 1e9, "unit": "GB/s (payload offloaded + reloaded over the host link / wall time of the whole trace)",
+        "seconds": sec, "blocks_hashed": st["blocks_hashed"], "blocks_hashed_looked_up_per_s": st["blocks_hashed"] / sec,
+        "inserted": st["inserted"], "offloaded": st["offloaded"], "reloaded": st["reloaded"], "dropped": st["dropped"],
+        "hit_ratio": (st["hits_hbm"] + st["hits_host"]) / max(st["blocks_hashed"], 1),
+        "host_link": {"achieved": st["mover_bytes"] / mover_s / 1e9 if mover_s else 0.0, "unit": "GB/s while a move is running",
+                      "frac": (st["mover_bytes"] / mover_s / 1e9) / (0.5 * (link["h2d"] + link["d2h"])) if mover_s else 0.0},
+        "lookup_kernels_blocks_per_s": st["lookup_blocks"] / (st["lookup_ns"] / 1e9) if st["lookup_ns"] else None,
+        "gpu_launches": st["kernel_launches"],
+    }
+    eng.close()
+    del eng
+    gc.collect()
+    torch.cuda.empty_cache()
+    if hasattr(torch._C, "_host_emptyCache"):
+        torch._C._host_emptyCache()
+    return out
+
+
+def cpu_stage_arm():
+    """The oracle, as it stands, on the C4 inputs stage by stage and on a C5-sized block gather, on this machine's
+    host cores: one thread (the oracle's own engine calls), plus an all-cores figure for the two embarrassingly
+    parallel stages (block digests, block copies) with plain std::thread."""
+    from oracle import kvt_oracle as O
+    O.build()
+    n_res, cb, n_calls = 1 << 20, 16128, 64
+    inp = W.inputs_c4(1, n_resident=n_res, chain_blocks=cb, n_calls=n_calls)
+    eng = O.OracleEngine(n_hbm_blocks=n_res, n_host_blocks=0, max_contexts=n_calls + 1, metadata_only=True, **W.GEO_TOY.kwargs())
+    keys = np.concatenate([O.hash_tokens(c) for c in inp.chain_tokens])
+    eng.debug_load_resident(keys, inp.state, inp.stamp, inp.depth, inp.slot, 0)
+    for i, t in enumerate(inp.calls):
+        eng.spawn(i)
+        eng.append(i, t)
+
+    def timed(fn):
+        t0 = time.perf_counter()
+        r = fn()
+        return time.perf_counter() - t0, r
+    t_look, info = timed(lambda: eng.map_blocks(list(range(n_calls)), 0))
+    t_cls, _ = timed(lambda: eng.get_states(0))
+    t_sel, (v, _s) = timed(lambda: eng.select_victims(0, n_res // 10))
+    n_blocks = int(info["n_blocks"].sum())
+    cores = os.cpu_count() or 1
+    tok = np.concatenate(inp.calls)
+    t_hash1, _ = timed(lambda: O.hash_tokens(tok))
+    t_dig1, _ = timed(lambda: O.par_digests(tok, 0, 1))
+    t_digN, _ = timed(lambda: O.par_digests(tok, 0, cores))
+    # C5-shaped gather: 256 permuted 2 MiB blocks (0.5 GiB, far beyond the caches) out of a 320-block pool into a contiguous tier
+    bb, n_pool, n = W.GEO_8B.block_bytes, 320, 256
+    rng = np.random.default_rng(5)
+    src = np.ones(n_pool * bb, dtype=np.uint8)
+    dst = np.ones(n * bb, dtype=np.uint8)
+    ids = rng.permutation(n_pool)[:n]
+    O.par_copy_blocks(dst, src, bb, ids[:64], np.arange(64), 1)          # touch the code path once
+    t_cp1, _ = timed(lambda: O.par_copy_blocks(dst, src, bb, ids, np.arange(n), 1))
+    t_cpN, _ = timed(lambda: O.par_copy_blocks(dst, src, bb, ids, np.arange(n), cores))
+    return {
+        "metadata_c4": {
+            "workload": f"the C4 inputs of metadata_stress: {n_res} resident blocks, {n_calls} calls x {cb} blocks, select 10%",
+            "cores": 1,
+            "hash_lookup_blocks_per_s": n_blocks / t_look, "hash_lookup_s": t_look,
+            "classify_s": t_cls, "classify_mappings_per_s": n_blocks / t_cls,
+            "select_s": t_sel, "select_resident_blocks_per_s": n_res / t_sel, "victims": int(len(v)),
+            "hash_only_blocks_per_s": len(tok) // 16 / t_hash1,
+            "digests_blocks_per_s_1_thread": len(tok) // 16 / t_dig1,
+            "digests_blocks_per_s_all_cores": len(tok) // 16 / t_digN, "all_cores": cores,
+        },
+        "mover_c5": {
+            "workload": f"{n} permuted blocks of {bb} B gathered from a {n_pool}-block pool into a contiguous tier (memcpy)",
+            "GBs_1_thread": n * bb / t_cp1 / 1e9, "GBs_all_cores": n * bb / t_cpN / 1e9, "all_cores": cores,
+        },
+    }
+
+
 def metadata_stress(torch, B, hbm_peak, reps=5):
     """C4-shaped side measurement of the metadata stages at scale (the C2 calls above are launch-latency
     sized): 1 Mi resident blocks, one LOOKUP batch of 64 calls x 16,128 blocks, classification of the
@@ -697,8 +819,7 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
     torch.cuda.set_device(local_rank)
     from paper_2609_39819_b200 import build as kbuild
-    if rank == 0 or not os.path.exists(kbuild.LIB):
-        kbuild.build_lib()
+    kbuild.build_lib()       # every rank asks; a file lock lets one of them compile and the others wait for the result
     barrier = None
     if world > 1:
         import torch.distributed as dist
@@ -754,13 +875,15 @@ def main():
     mover_s = st["mover_ns"] / 1e9
     achieved = 2 * st["mover_bytes"] / mover_s / 1e9 if mover_s else 0.0
     per_launch_bytes = 2 * st["mover_bytes"] / max(st["mover_launches"], 1)
+    traffic_ratio = mover_traffic_ratio()
     roofline = {
         "bound": "hbm", "kernel": "k_move_tiles<8>", "achieved": achieved, "peak": hbm_peak, "unit": "GB/s",
         "frac": achieved / hbm_peak, "peak_kind": f"{peak_kind} copy bandwidth (MEASURED_PEAKS.json hbm_gbs)",
         "frac_of_nominal_8TBs": achieved / 8000.0, "torch_copy_gbs_this_run": hbm_now,
         "launches": st["mover_launches"], "avg_launch_ms": mover_s * 1e3 / max(st["mover_launches"], 1),
         "algorithmic_bytes_per_launch": per_launch_bytes,
-        "traffic": None if MOVER_TRAFFIC_PER_ALGO_BYTE is None else MOVER_TRAFFIC_PER_ALGO_BYTE * per_launch_bytes,
+        "traffic": None if traffic_ratio is None else traffic_ratio * per_launch_bytes,
+        "traffic_source": "profiles/mover_8b_hbm_to_hbm.md (ncu capture of a 1024-block launch, scaled by blocks moved)",
     }
     line = {
         "metric": METRIC, "value": tot_bytes / (ms / 1e3) / 1e9, "unit": "GB/s", "n_gpus": args.gpus, "steps": K,
@@ -822,6 +945,8 @@ def main():
                         "pushes part of the other session out",
             "unit": "GB/s (blocks offloaded + reloaded)", "offload_then_reload": seq, "one_exchange_per_call": dup,
         }
+    if e and not args.skip_c3 and world == 1:
+        line["c3"] = c3_arm(args, torch, B, link)
     if not args.skip_stress and world == 1:
         line["metadata_stress"] = metadata_stress(torch, B, hbm_peak)
     if not args.skip_cpu and world == 1:
@@ -837,6 +962,7 @@ def main():
             "stage_wall_ms_per_step": {k: round(x / min(args.cpu_steps, K), 3) for k, x in c["stage_ms"].items()},
             "host": host_info(),
         }
+        line["cpu_baseline"].update(cpu_stage_arm())
     print(json.dumps(line))
 
 

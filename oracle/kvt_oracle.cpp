@@ -33,6 +33,7 @@
 #include <map>
 #include <set>
 #include <string>
+#include <thread>
 #include <utility>
 #include <vector>
 
@@ -865,6 +866,40 @@ int32_t kvto_debug_load_resident(Engine *e, const uint64_t *keys, const uint8_t 
     e->where[keys[i]] = {tier, slot[i]};
     if (stamp[i] > e->now) e->now = stamp[i];
   }
+  return OK;
+}
+
+// ---- all-cores timing helpers --------------------------------------------------------------------------------
+// The two embarrassingly parallel stages (block digests, block copies) spread over plain std::threads, for the
+// benchmark's "all host cores" figures. They are not part of the engine above and nothing else calls them.
+int32_t kvto_par_digests(const uint32_t *tokens, uint64_t n_tokens, uint64_t seed, uint64_t *digests, uint32_t n_threads) {
+  if ((!tokens || !digests) && n_tokens >= 16) return E_INVAL;
+  if (!n_threads) return E_INVAL;
+  const HashParams hp = make_params(seed);
+  const uint64_t nb = n_tokens / 16;
+  std::vector<std::thread> th;
+  for (uint32_t t = 0; t < n_threads; ++t)
+    th.emplace_back([=, &hp]() {
+      for (uint64_t b = nb * t / n_threads; b < nb * (t + 1) / n_threads; ++b) {
+        uint64_t sum = 0;
+        for (int k = 0; k < 16; ++k) sum += ((uint64_t)tokens[16 * b + k] + 1ull) * hp.K[k];
+        digests[b] = mix64(sum);
+      }
+    });
+  for (auto &x : th) x.join();
+  return OK;
+}
+
+int32_t kvto_par_copy_blocks(uint8_t *dst, const uint8_t *src, uint64_t block_bytes, const uint32_t *src_ids,
+                             const uint32_t *dst_ids, uint32_t n, uint32_t n_threads) {
+  if (!dst || !src || !src_ids || !dst_ids || !n_threads) return E_INVAL;
+  std::vector<std::thread> th;
+  for (uint32_t t = 0; t < n_threads; ++t)
+    th.emplace_back([=]() {
+      for (uint64_t i = (uint64_t)n * t / n_threads; i < (uint64_t)n * (t + 1) / n_threads; ++i)
+        std::memcpy(dst + (uint64_t)dst_ids[i] * block_bytes, src + (uint64_t)src_ids[i] * block_bytes, block_bytes);
+    });
+  for (auto &x : th) x.join();
   return OK;
 }
 

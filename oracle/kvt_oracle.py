@@ -35,7 +35,7 @@ class OracleError(RuntimeError):
 def build(force: bool = False) -> str:
     """Compiles the oracle with g++ (plain -O2, one thread) if the library is missing or stale."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        subprocess.check_call(["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-o", _LIB, _SRC])
+        subprocess.check_call(["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-pthread", "-o", _LIB, _SRC])
     return _LIB
 
 
@@ -89,6 +89,26 @@ def hash_tokens(tokens, seed: int = 0) -> np.ndarray:
     if rc:
         raise OracleError(rc, "hash_tokens")
     return keys
+
+
+def par_digests(tokens, seed: int = 0, n_threads: int = 1) -> np.ndarray:
+    """Block digests d_b of a token sequence, blocks spread over n_threads threads (timing helper)."""
+    tok = _u32(tokens)
+    out = np.zeros(len(tok) // 16, dtype=np.uint64)
+    lib().kvto_par_digests.argtypes = [C.c_void_p, C.c_uint64, C.c_uint64, C.c_void_p, C.c_uint32]
+    rc = lib().kvto_par_digests(_p(tok), len(tok), seed, _p(out), n_threads)
+    if rc:
+        raise OracleError(rc, "par_digests")
+    return out
+
+
+def par_copy_blocks(dst, src, block_bytes, src_ids, dst_ids, n_threads: int = 1):
+    """dst[dst_ids[i]] = src[src_ids[i]] for whole blocks (uint8 arrays), over n_threads threads (timing helper)."""
+    s, d = _u32(src_ids), _u32(dst_ids)
+    lib().kvto_par_copy_blocks.argtypes = [C.c_void_p, C.c_void_p, C.c_uint64, C.c_void_p, C.c_void_p, C.c_uint32, C.c_uint32]
+    rc = lib().kvto_par_copy_blocks(_p(dst), _p(src), block_bytes, _p(s), _p(d), len(s), n_threads)
+    if rc:
+        raise OracleError(rc, "par_copy_blocks")
 
 
 def hash_constants(seed: int = 0, x: int = 0):

@@ -125,3 +125,26 @@ def test_prefix_suffix_position_seed_properties(oracle):
     # no collisions in a modest sample
     big = oracle.hash_tokens(rng.integers(0, 151552, 16 * 20000))
     assert len(np.unique(big)) == len(big)
+
+
+def test_parallel_digests_and_copies_match_the_plain_ones(oracle):
+    """The all-cores timing helpers compute the same things: the chain over their digests gives the block keys, and
+    the threaded block copy equals a plain gather."""
+    rng = np.random.default_rng(11)
+    tok = rng.integers(0, 151552, 16 * 1000 + 9, dtype=np.uint32)
+    for seed in (0, 5):
+        _K, P, H0, _ = oracle.hash_constants(seed)
+        d = oracle.par_digests(tok, seed, n_threads=3)
+        h, keys = H0, []
+        for x in d:
+            h = (P * h + int(x)) & (2**64 - 1)
+            k = oracle.hash_constants(seed, h)[3]
+            keys.append(k + 2 if k < 2 else k)
+        assert keys == [int(k) for k in oracle.hash_tokens(tok, seed)]
+    src = rng.integers(0, 256, 64 * 4096, dtype=np.uint8)
+    dst = np.zeros(32 * 4096, dtype=np.uint8)
+    si, di = rng.permutation(64)[:32], rng.permutation(32)
+    oracle.par_copy_blocks(dst, src, 4096, si, di, n_threads=4)
+    want = np.zeros_like(dst).reshape(32, 4096)
+    want[di] = src.reshape(64, 4096)[si]
+    assert np.array_equal(dst.reshape(32, 4096), want)
