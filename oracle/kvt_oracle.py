@@ -14,7 +14,10 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "kvt_oracle.cpp")
-_LIB = os.path.join(_HERE, "libkvt_oracle.so")
+# KVT_ORACLE_SANITIZE=1: a separate build with AddressSanitizer and UndefinedBehaviorSanitizer (the process must
+# then run with the ASan runtime preloaded; the sanitizer test starts such a process)
+_SANITIZE = os.environ.get("KVT_ORACLE_SANITIZE") == "1"
+_LIB = os.path.join(_HERE, "libkvt_oracle_asan.so" if _SANITIZE else "libkvt_oracle.so")
 
 OK, E_INVAL, E_NOCTX, E_RANGE, E_STATE, E_NOSPACE, E_BUFSZ = 0, -1, -2, -3, -4, -5, -6
 TIER_HBM, TIER_HOST, TIER_REMOTE, TIER_NONE = 0, 1, 2, 0xFF
@@ -35,7 +38,9 @@ class OracleError(RuntimeError):
 def build(force: bool = False) -> str:
     """Compiles the oracle with g++ (plain -O2, one thread) if the library is missing or stale."""
     if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
-        subprocess.check_call(["g++", "-O2", "-std=c++17", "-shared", "-fPIC", "-pthread", "-o", _LIB, _SRC])
+        flags = ["-O1", "-g", "-fsanitize=address,undefined", "-fno-sanitize-recover=undefined", "-fno-omit-frame-pointer"] \
+            if _SANITIZE else ["-O2"]
+        subprocess.check_call(["g++"] + flags + ["-std=c++17", "-shared", "-fPIC", "-pthread", "-o", _LIB, _SRC])
     return _LIB
 
 

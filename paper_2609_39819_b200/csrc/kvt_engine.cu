@@ -21,6 +21,17 @@ using namespace kvt;
 
 namespace {
 
+// Threads per block of the element-wise kernels. The checked build (-DKVT_DEBUG) runs every launch in another
+// shape (small blocks, a handful of mover CTAs, no CUDA graph): results do not depend on the shape, and a kernel
+// that secretly relied on it shows up as a difference from the CPU reference in the tests.
+#ifdef KVT_DEBUG
+constexpr u32 TPB = 64;
+constexpr bool CHECKED_BUILD = true;
+#else
+constexpr u32 TPB = 256;
+constexpr bool CHECKED_BUILD = false;
+#endif
+
 constexpr u32 MS_ACTIVE = 0, MS_SUSPENDED = 1, MS_EXPIRED = 2, MS_TEMPORARY = 3, MS_PINNED = 4;
 // Priority of a message state in the block aggregate: Algorithm 1's release order.
 inline u8 msg_rank(u8 s) { return s == MS_PINNED ? 3 : (s == MS_ACTIVE ? 2 : (s == MS_SUSPENDED ? 1 : 0)); }
@@ -186,7 +197,7 @@ struct kvt_engine {
   // CTA sits on, so those warps are packed into 4 CTAs of 1024 threads (8 for an exchange, which
   // drives both directions).
   u32 mover_grid(u64 want, u32 link_dirs = 0) const {
-    u64 cap = mover_max_ctas ? mover_max_ctas : link_dirs == 1 ? 4 : link_dirs == 2 ? 8 : (u64)sm_count * 8;
+    u64 cap = mover_max_ctas ? mover_max_ctas : CHECKED_BUILD ? 5 : link_dirs == 1 ? 4 : link_dirs == 2 ? 8 : (u64)sm_count * 8;
     return (u32)std::max<u64>(1, std::min(want, cap));
   }
   u32 link_dirs(u32 st, u32 dt) const { return (tier_in_host_mem[st] || tier_in_host_mem[dt]) ? 1u : 0u; }
@@ -320,8 +331,8 @@ int32_t compact_indices(kvt_engine *e, cudaStream_t s, Pred pred, Emit emit, u32
 }
 
 int32_t table_rebuild(kvt_engine *e, cudaStream_t s) {
-  KL(k_table_clear, cdiv((u64)e->tab.mask + 1,256), 256, s, e->tab);
-  KL(k_table_reinsert, cdiv(e->ent.n_total,256), 256, s, e->tab, e->ent, e->d_status);
+  KL(k_table_clear, cdiv((u64)e->tab.mask + 1, TPB), TPB, s, e->tab);
+  KL(k_table_reinsert, cdiv(e->ent.n_total, TPB), TPB, s, e->tab, e->ent, e->d_status);
   LAUNCH_CHECK();
   e->tombs = 0;
   e->st.table_rebuilds++;
@@ -695,9 +706,9 @@ int32_t apply_deltas(kvt_engine *e, cudaStream_t s, const std::vector<Ctx *> &li
       a.first_miss = e->dp<u32>(e->L.freelist2);   // scratch of the list calls, free between calls (stream order)
       if (nd > e->L.LB) return fail(e, KVT_E_NOSPACE, "more contexts than max_batch_blocks");
       CU(cudaMemsetAsync(a.first_miss, 0xFF, nd * 4ull, s));
-      KL(k_first_miss, cdiv(nmap, 256), 256, s, a);
+      KL(k_first_miss, cdiv(nmap, TPB), TPB, s, a);
     }
-    KL(k_map_delta, cdiv(nmap, 256), 256, s, a);
+    KL(k_map_delta, cdiv(nmap, TPB), TPB, s, a);
     LAUNCH_CHECK();
   }
   // what is accounted for now
@@ -777,7 +788,7 @@ int32_t do_classify(kvt_engine *e, cudaStream_t s, bool force_full = false) {
     r = do_classify(e, s, true);
     if (r) return r;
     CU(cudaMemsetAsync(e->d_status + ST_CHK, 0, 4, s));
-    KL(k_cnt_compare, cdiv(e->ent.n_total, 256), 256, s, e->dp<u64>(e->L.cnt_chk), e->ent.cnt, e->ent.n_total, e->d_status + ST_CHK);
+    KL(k_cnt_compare, cdiv(e->ent.n_total, TPB), TPB, s, e->dp<u64>(e->L.cnt_chk), e->ent.cnt, e->ent.n_total, e->d_status + ST_CHK);
     LAUNCH_CHECK();
     CU(cudaMemcpyAsync(e->h_status + ST_CHK, e->d_status + ST_CHK, 4, cudaMemcpyDeviceToHost, s));
     CU(cudaStreamSynchronize(s));
@@ -823,7 +834,7 @@ u64 grow_cap(u64 need) { return round_up(std::max<u64>(need + need / 4, 1024), 6
 
 int32_t unlock_held(kvt_engine *e, Ctx &c, cudaStream_t s, bool stamp) {
   if (c.held && c.keyseg >= 0) {
-    KL(k_unlock, cdiv(c.held,256), 256, s, e->tab, e->ent, e->d_keys + e->segs[c.keyseg].off, c.held, e->now,
+    KL(k_unlock, cdiv(c.held, TPB), TPB, s, e->tab, e->ent, e->d_keys + e->segs[c.keyseg].off, c.held, e->now,
                                                 stamp ? 1u : 0u, e->d_status);
     LAUNCH_CHECK();
   }
@@ -967,6 +978,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
 #ifdef KVT_TRACE
   if (getenv("KVT_NO_GRAPH")) e->use_graphs = false;
 #endif
+  if (CHECKED_BUILD) e->use_graphs = false;
   bool ok = cudaEventCreateWithFlags(&e->ev_upload, cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreate(&e->ev_m0) == cudaSuccess && cudaEventCreate(&e->ev_m1) == cudaSuccess &&
             cudaEventCreate(&e->ev_h0) == cudaSuccess && cudaEventCreate(&e->ev_h1) == cudaSuccess;
@@ -975,7 +987,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   ok = ok && cudaMemsetAsync(e->d_status, 0, ST_WORDS * 4, s) == cudaSuccess;
   ok = ok && cudaMemsetAsync(e->ent.link, 0xFF, N * 4, s) == cudaSuccess;   // no links
   if (ok) {
-    KL(k_table_clear, cdiv((u64)c.table_capacity,256), 256, s, e->tab);
+    KL(k_table_clear, cdiv((u64)c.table_capacity, TPB), TPB, s, e->tab);
     ok = cudaGetLastError() == cudaSuccess && cudaStreamSynchronize(s) == cudaSuccess;
   }
   if (!ok) { cudaFreeHost(e->stage); if (e->ev_upload) cudaEventDestroy(e->ev_upload); delete e; return KVT_E_CUDA; }
@@ -1451,15 +1463,15 @@ static int32_t map_admit(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_info
     CU(cudaMemcpyAsync(a.stop, h_stop, nd * 4, cudaMemcpyHostToDevice, s));
     rc = status_zero(e, s);
     if (rc) break;
-    u32 g = cdiv(n_cand, 256);
-    KL(k_admit_claim, g, 256, s, a);
-    KL(k_admit_resolve, g, 256, s, a);
+    u32 g = cdiv(n_cand, TPB);
+    KL(k_admit_claim, g, TPB, s, a);
+    KL(k_admit_resolve, g, TPB, s, a);
     rc = compact_indices(e, s, PredOwner{a.flag}, EmitRank{a.krank}, n_cand, ST_NEW);
     if (rc) break;
     rc = compact_indices(e, s, PredFree{e->ent.key, 0}, EmitFree{e->dp<u32>(e->L.freelist), (u32)e->L.LB}, e->cfg.n_hbm_blocks, ST_FREE);
     if (rc) break;
-    KL(k_admit_stop, g, 256, s, a);
-    KL(k_admit_apply, g, 256, s, a);
+    KL(k_admit_stop, g, TPB, s, a);
+    KL(k_admit_apply, g, TPB, s, a);
     rc = launch_ok(e);
     if (rc) break;
     CU(cudaMemcpyAsync(h_stop, a.stop, nd * 4, cudaMemcpyDeviceToHost, s));
@@ -1522,7 +1534,7 @@ int32_t kvt_get_block_map(kvt_engine *e, uint32_t ctx, uint64_t *keys, uint8_t *
   const u64 *dk = e->d_keys + e->segs[c->keyseg].off;
   int32_t r = status_zero(e, s);
   if (r) return r;
-  KL(k_block_map, cdiv(nb,256), 256, s, e->tab, e->ent, dk, nb, e->dp<u8>(e->L.map_tier), e->dp<u32>(e->L.map_slot), e->d_status);
+  KL(k_block_map, cdiv(nb, TPB), TPB, s, e->tab, e->ent, dk, nb, e->dp<u8>(e->L.map_tier), e->dp<u32>(e->L.map_slot), e->d_status);
   LAUNCH_CHECK();
   // results go through pinned staging: one synchronisation for everything
   u64 *hk = (u64 *)e->h_out; u32 *hs = (u32 *)(e->h_out + nb * 8ull); u8 *ht = e->h_out + nb * 12ull;
@@ -1554,7 +1566,7 @@ int32_t kvt_get_states(kvt_engine *e, uint32_t tier, uint8_t *state, uint32_t ca
   int32_t r = ensure_classified(e, s);
   if (r) return r;
   u8 *d_out = e->dp<u8>(e->L.out_states);
-  KL(k_states_out, cdiv(n,256), 256, s, e->ent, e->tier_e0(tier), n, d_out);
+  KL(k_states_out, cdiv(n, TPB), TPB, s, e->ent, e->tier_e0(tier), n, d_out);
   LAUNCH_CHECK();
   CU(cudaMemcpyAsync(state, d_out, n, cudaMemcpyDeviceToHost, s));
   CU(cudaStreamSynchronize(s));
@@ -1742,8 +1754,8 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
   a.allow_inflight = m.allow_inflight; a.drop_dead = m.drop_dead; a.drop_all = m.drop_all;
   a.reject_shadow = m.reject_shadow; a.clean_ok = m.clean_ok; a.keep_copy = m.keep_copy; a.status = e->d_status;
   a.w_cut = ST_CUT; a.w_nlive = ST_NLIVE; a.w_ndrop = ST_NDROP; a.w_nclean = ST_NCLEAN; a.w_nshdrop = ST_NSHDROP;
-  u32 g = cdiv(n, 256);
-  KL(k_list_validate, g, 256, s, a);
+  u32 g = cdiv(n, TPB);
+  KL(k_list_validate, g, TPB, s, a);
   r = compact_indices(e, s, PredLive{a.live}, EmitLive{a.lidx, a.n_free, e->d_status + ST_CUT, nullptr}, n, ST_TOTAL);
   if (r) return r;
   if (!m.drop_all) {
@@ -1751,8 +1763,8 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
                         e->tier_slots(dst_tier), ST_FREE);
     if (r) return r;
   }
-  KL(k_list_apply, g, 256, s, a);
-  KL(k_list_unmark, g, 256, s, a);
+  KL(k_list_apply, g, TPB, s, a);
+  KL(k_list_unmark, g, TPB, s, a);
   LAUNCH_CHECK();
   const bool staged = !m.drop_all && staged_applies(e, src_tier, dst_tier);
   const u32 n_pairs_max = std::min(n, a.n_free);
@@ -1881,9 +1893,9 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
   b.pair_src = e->dp<u32>(e->L.pair_src2); b.pair_dst = e->dp<u32>(e->L.pair_dst2);
   b.drop_dead = !(e->cfg.policy_flags & KVT_POLICY_NO_LIFECYCLE); b.clean_ok = 1;
   b.w_cut = ST_B_CUT; b.w_nlive = ST_B_NLIVE; b.w_ndrop = ST_B_NDROP; b.w_nclean = ST_B_NCLEAN; b.w_nshdrop = ST_B_NSHDROP;
-  const u32 ga = cdiv(n_in, 256), gb = cdiv(n_out, 256);
-  if (n_in) KL(k_list_validate, ga, 256, s, a);
-  if (n_out) KL(k_list_validate, gb, 256, s, b);
+  const u32 ga = cdiv(n_in, TPB), gb = cdiv(n_out, TPB);
+  if (n_in) KL(k_list_validate, ga, TPB, s, a);
+  if (n_out) KL(k_list_validate, gb, TPB, s, b);
   if (n_out) {   // victims: plan against the host slots that are free now, apply
     r = compact_indices(e, s, PredLive{b.live}, EmitLive{b.lidx, b.n_free, e->d_status + ST_B_CUT, nullptr}, n_out, ST_B_TOTAL);
     if (r) return r;
@@ -1891,16 +1903,16 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
       r = compact_indices(e, s, PredFree{e->ent.key, b.dst_e0}, EmitFree{e->dp<u32>(e->L.freelist2), (u32)e->L.LB}, e->cfg.n_host_blocks, ST_B_FREE);
       if (r) return r;
     }
-    KL(k_list_apply, gb, 256, s, b);
-    KL(k_list_unmark, gb, 256, s, b);
+    KL(k_list_apply, gb, TPB, s, b);
+    KL(k_list_unmark, gb, TPB, s, b);
   }
   if (n_in) {    // reloads: the free HBM slots now include what the victims left
     r = compact_indices(e, s, PredFree{e->ent.key, 0}, EmitFree{e->dp<u32>(e->L.freelist), (u32)e->L.LB}, e->cfg.n_hbm_blocks, ST_FREE);
     if (r) return r;
     r = compact_indices(e, s, PredLive{a.live}, EmitLive{a.lidx, a.n_free, e->d_status + ST_CUT, e->d_status + ST_FREE}, n_in, ST_TOTAL);
     if (r) return r;
-    KL(k_list_apply, ga, 256, s, a);
-    KL(k_list_unmark, ga, 256, s, a);
+    KL(k_list_apply, ga, TPB, s, a);
+    KL(k_list_unmark, ga, TPB, s, a);
   }
   LAUNCH_CHECK();
   const bool staged = staged_applies(e, KVT_TIER_HBM, KVT_TIER_HOST);
@@ -1946,8 +1958,8 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
         // which reload lands in a slot a victim leaves (scratch of the selection, idle during this call)
         u32 *vic_of = e->dp<u32>(e->L.out_slots), *dep = e->dp<u32>(e->L.valA), *taken = e->dp<u32>(e->L.valB);
         CU(cudaMemsetAsync(vic_of, 0xFF, (u64)e->cfg.n_hbm_blocks * 4, s));
-        if (mb.n_pairs) KL(k_xchg_mark, cdiv(mb.n_pairs, 256), 256, s, mb.src_ids, mb.n_pairs_dev, mb.n_pairs, vic_of, taken);
-        if (ma.n_pairs) KL(k_xchg_link, cdiv(ma.n_pairs, 256), 256, s, ma.dst_ids, ma.n_pairs_dev, ma.n_pairs, vic_of, dep, taken);
+        if (mb.n_pairs) KL(k_xchg_mark, cdiv(mb.n_pairs, TPB), TPB, s, mb.src_ids, mb.n_pairs_dev, mb.n_pairs, vic_of, taken);
+        if (ma.n_pairs) KL(k_xchg_link, cdiv(ma.n_pairs, TPB), TPB, s, ma.dst_ids, ma.n_pairs_dev, ma.n_pairs, vic_of, dep, taken);
         u32 tpc = (u32)(e->chunk_bytes / 4096);
         const u32 xl = e->link_dirs(KVT_TIER_HBM, KVT_TIER_HOST) * 2;
         if (xl) {
@@ -2020,7 +2032,7 @@ int32_t kvt_compact(kvt_engine *e, uint32_t tier, uint32_t *n_moved, void *strea
   r = compact_indices(e, s, PredMover{e->ent.key, e0, n_occ}, EmitList{src}, n, ST_NMOVED);
   if (r) return r;
   u32 n_max = std::min(n_occ, n - n_occ);
-  KL(k_compact_apply, cdiv(n_max,256), 256, s, e->tab, e->ent, e0, src, dst, e->d_status);
+  KL(k_compact_apply, cdiv(n_max, TPB), TPB, s, e->tab, e->ent, e0, src, dst, e->d_status);
   LAUNCH_CHECK();
   r = launch_mover(e, s, tier, src, tier, dst, n_max, e->d_status + ST_NMOVED);
   if (r) return r;
@@ -2157,8 +2169,8 @@ int32_t kvt_debug_load_resident(kvt_engine *e, const uint64_t *keys, const uint8
   LoadArgs a;
   a.tab = e->tab; a.ent = e->ent; a.keys = dk; a.state = dst_state; a.stamp = dsp; a.depth = ddp; a.slot = dsl;
   a.n = n; a.e0 = e->tier_e0(tier); a.n_slots = ns; a.status = e->d_status;
-  KL(k_load_check, cdiv(n,256), 256, s, a);
-  KL(k_load_apply, cdiv(n,256), 256, s, a);
+  KL(k_load_check, cdiv(n, TPB), TPB, s, a);
+  KL(k_load_apply, cdiv(n, TPB), TPB, s, a);
   LAUNCH_CHECK();
   r = status_fetch(e, s);
   if (r) return r;

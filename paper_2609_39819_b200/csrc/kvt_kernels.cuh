@@ -92,6 +92,14 @@ __device__ __forceinline__ bool is_shadow(const Entries &en, u32 e) { return e >
 
 __device__ __forceinline__ void set_err(u32 *status, u32 bits) { atomicOr(&status[ST_ERR], bits); }
 
+// Index and invariant checks of the checked build (-DKVT_DEBUG): a violation sets the error word and skips the
+// access (never a trap, never a wild store); the call then reports KVT_E_DEVICE. They compile to nothing otherwise.
+#ifdef KVT_DEBUG
+#define KVT_CHECK(cond, status, action) do { if (!(cond)) { set_err((status), DERR_CORRUPT); action; } } while (0)
+#else
+#define KVT_CHECK(cond, status, action) do { } while (0)
+#endif
+
 // Finds key; returns its table slot index or ENT_NONE. Stops at the first EMPTY slot.
 __device__ __forceinline__ u32 tab_find(const Table &t, u64 key, u32 *status) {
   u32 i = (u32)(key >> t.shift);
@@ -773,7 +781,9 @@ __global__ void k_admit_apply(AdmitArgs a) {
   } else if (f == CAND_OWNER) {
     u32 s = a.cslot[g];
     if (held) {
+      KVT_CHECK(a.krank[g] < a.n_free, a.status, return);
       u32 e = a.freelist[a.krank[g]];
+      KVT_CHECK(e < a.ent.n_hbm && a.ent.key[e] == 0 && s <= a.tab.mask, a.status, return);
       a.ent.key[e] = a.keys[c.key_off + b];
       a.ent.stamp[e] = a.now; a.ent.depth[e] = b; a.ent.cnt[e] = 0; a.ent.floor[e] = 0; a.ent.tslot[e] = s; a.ent.link[e] = ENT_NONE;
       atomicAdd(&a.ent.infl[e], 1u);
@@ -882,6 +892,7 @@ __global__ void k_first_miss(DeltaArgs a) {
 
 __device__ __forceinline__ void cnt_add(const DeltaArgs &a, u64 key, u64 delta) {
   const u32 e = tab_lookup_ent(a.tab, key, a.status);   // ENT_NONE: mapped but not resident
+  KVT_CHECK(e == ENT_NONE || (e < a.ent.n_total && a.ent.key[e] == key), a.status, return);
   if (e < a.ent.n_total) atomicAdd((unsigned long long *)&a.ent.cnt[e], (unsigned long long)delta);
 }
 
@@ -1332,6 +1343,7 @@ __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const
     __syncwarp();
     if (ok && before == 0) cnt[warp][d] += __popc(peers);
     __syncwarp();
+    KVT_CHECK(!ok || pos < m, const_cast<u32 *>(status), continue);
     if (ok) { keys_out[pos] = kreg[it]; vals_out[pos] = vreg[it]; }
   }
 }
@@ -1461,7 +1473,9 @@ __global__ void k_list_apply(ListArgs a) {
     atomicAdd(&a.status[a.w_nclean], 1u);
   } else {
     u32 r = a.lidx[i];
+    KVT_CHECK(r < a.n_free, a.status, return);
     u32 d = a.freelist[r];
+    KVT_CHECK(a.ent.key[a.dst_e0 + d] == 0 && a.dst_e0 + d < a.ent.n_total, a.status, return);
     a.pair_src[r] = id;
     a.pair_dst[r] = d;
     u32 de = a.dst_e0 + d;
@@ -1488,6 +1502,8 @@ struct EmitList { u32 *list; __device__ void operator()(u32 i, u32 r) const { li
 __global__ void k_compact_apply(Table t, Entries en, u32 e0, const u32 *src, const u32 *dst, const u32 *status) {
   u32 i = blockIdx.x * blockDim.x + threadIdx.x;
   if (i >= status[ST_NMOVED] || status[ST_ERR]) return;
+  KVT_CHECK(e0 + src[i] < en.n_total && e0 + dst[i] < en.n_total && en.key[e0 + src[i]] != 0 && en.key[e0 + dst[i]] == 0,
+            const_cast<u32 *>(status), return);
   entry_move(t, en, e0 + src[i], e0 + dst[i]);
 }
 

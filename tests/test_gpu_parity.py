@@ -906,3 +906,27 @@ def test_create_rejects_bad_configs(B):
     assert attempt(suspended_order=2) == B.E_INVAL and attempt(policy_flags=8) == B.E_INVAL
     assert attempt(n_hbm_blocks=0) == B.E_INVAL and attempt(max_contexts=0) == B.E_INVAL
     assert lib.kvt_create(None, None, None) == B.E_INVAL
+
+
+# ---- the checked build: device-side index checks, every launch in another shape -----------------------------
+def test_checked_build_in_another_launch_shape():
+    """The same scenario expectations and a slice of the random differential streams, in a child process that loads
+    libkvt_debug.so (-DKVT_DEBUG): 64-thread blocks for the element-wise kernels, at most five mover thread blocks,
+    plain launches instead of the selection's CUDA graph, and index / invariant checks that set the device error
+    word. Results must not depend on the launch shape, and no check may fire."""
+    import os
+    import subprocess
+    import sys
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_39819_b200 import build
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = dict(os.environ, KVT_LIB=build.build_debug_lib())
+    cmd = [sys.executable, "-m", "pytest", "-x", "-q", "-p", "no:cacheprovider", "-m", "gpu",
+           os.path.join(root, "tests", "test_gpu_parity.py"), os.path.join(root, "tests", "test_gpu_fuzz.py"),
+           "-k", "test_scenario or c1_trace_parity or (random_api_streams_match and hbm24 and (0-0 or 2-1 or 4-2 or 7-3)) "
+                 "or staging_ring or c4_lookup_and_select_parity and 5000"]
+    r = subprocess.run(cmd, env=env, cwd=root, capture_output=True, text=True, timeout=1500)
+    assert r.returncode == 0, (r.stdout[-3000:], r.stderr[-2000:])
+    assert "passed" in r.stdout
