@@ -432,13 +432,13 @@ bool staged_applies(const kvt_engine *e, u32 st, u32 dt) {
   return e->mover_variant == 4 || e->block_bytes >= (512u << 10);
 }
 
-// Moves n blocks src_tier[h_src[i]] -> dst_tier[h_dst[i]] through the staging ring. d_src / d_dst: the same id lists
-// in device memory (for the gather / scatter kernel); h_src / h_dst: on the host (for the copy-engine transfers).
-// dir 0: device -> host (gather into a stage on `s`, then transfers on the copy stream); dir 1: host -> device
-// (transfers into a stage on the copy stream, then scatter on `s`). Consecutive host slots travel as one transfer.
-// When this returns, `s` waits for everything the copy stream still has to do.
-int32_t staged_move(kvt_engine *e, cudaStream_t s, u32 st, const u32 *d_src, const u32 *h_src, u32 dt, const u32 *d_dst,
-                    const u32 *h_dst, u32 n) {
+// Moves n blocks src_tier[h_src[i]] -> dst_tier[h_dst[i]] through the staging ring; h_src / h_dst are the planned
+// pairs on the host. The blocks travel in the order of their slots in the host-memory pool, whatever the order of
+// the list (the copies are independent of each other), so that every stretch of consecutive host slots is one
+// copy-engine transfer. dir 0: device -> host (gather into a stage on `s`, then transfers on the copy stream);
+// dir 1: host -> device (transfers into a stage on the copy stream, then scatter on `s`). When this returns, `s`
+// waits for everything the copy stream still has to do.
+int32_t staged_move(kvt_engine *e, cudaStream_t s, u32 st, const u32 *h_src, u32 dt, const u32 *h_dst, u32 n) {
   if (!n) return KVT_OK;
   const int dir = e->tier_in_host_mem[st] ? 1 : 0;
   kvt_engine::Staging &g = e->stg;
@@ -446,42 +446,35 @@ int32_t staged_move(kvt_engine *e, cudaStream_t s, u32 st, const u32 *d_src, con
   const u64 BB = e->block_bytes;
   u8 *host_pool = (u8 *)(dir ? (st == KVT_TIER_HOST ? e->cfg.host_pool : e->cfg.remote_pool)
                              : (dt == KVT_TIER_HOST ? e->cfg.host_pool : e->cfg.remote_pool));
-  const u32 *h_ids = dir ? h_src : h_dst;     // slots of the pool in host memory
+  const u32 *h_host = dir ? h_src : h_dst, *h_dev = dir ? h_dst : h_src;   // slots of the host-memory pool / of the device pool
   const u32 n_host_slots = e->tier_slots(dir ? st : dt);
-  for (u32 i = 0; i < n; ++i) if (h_ids[i] >= n_host_slots) return fail(e, KVT_E_RANGE, "slot id out of range");
-  // Inside a batch the blocks sit in the stage in the order of their host slots, whatever the order of the list, so
-  // that every stretch of consecutive host slots is one transfer: pos[i] = place of list item i in its batch's stage.
-  const u32 n_batches = cdiv(n, SB);
-  u32 *h_pos = e->h_ids2, *d_pos = e->dp<u32>(e->L.ids2);
-  std::vector<u32> order(std::min(SB, n));
-  for (u32 k = 0; k < n_batches; ++k) {
-    const u32 b0 = k * SB, nb = std::min(SB, n - b0);
-    for (u32 i = 0; i < nb; ++i) order[i] = i;
-    std::sort(order.begin(), order.begin() + nb, [&](u32 x, u32 y) { return h_ids[b0 + x] < h_ids[b0 + y]; });
-    for (u32 p = 0; p < nb; ++p) h_pos[b0 + order[p]] = p;
-  }
-  CU(cudaMemcpyAsync(d_pos, h_pos, n * 4ull, cudaMemcpyHostToDevice, s));
-  {
-    int32_t r = stage_release(e, s);   // the next call that stages ids waits for this upload
-    if (r) return r;
-  }
+  for (u32 i = 0; i < n; ++i) if (h_host[i] >= n_host_slots) return fail(e, KVT_E_RANGE, "slot id out of range");
+  std::vector<u32> order(n), host_sorted(n);
+  for (u32 i = 0; i < n; ++i) order[i] = i;
+  std::sort(order.begin(), order.end(), [&](u32 x, u32 y) { return h_host[x] < h_host[y]; });
+  int32_t r = stage_acquire(e);
+  if (r) return r;
+  u32 *h_ids = e->h_ids2, *d_ids = e->dp<u32>(e->L.ids2);    // device-pool slots in travelling order
+  for (u32 p = 0; p < n; ++p) { h_ids[p] = h_dev[order[p]]; host_sorted[p] = h_host[order[p]]; }
+  CU(cudaMemcpyAsync(d_ids, h_ids, n * 4ull, cudaMemcpyHostToDevice, s));
+  r = stage_release(e, s);   // the next call that stages ids waits for this upload
+  if (r) return r;
   const bool timed = e->profiling;
   if (timed) CU(cudaEventRecord(e->ev_m0, s));
   if (dir == 1) {   // the host pool holds what earlier work on `s` put there
     CU(cudaEventRecord(g.begin, s));
     CU(cudaStreamWaitEvent(g.cs[1], g.begin, 0));
   }
-  std::vector<u32> sorted_slots(std::min(SB, n));
+  const u32 n_batches = cdiv(n, SB);
   for (u32 k = 0; k < n_batches; ++k) {
     const int sg = (int)(k % kvt_engine::N_STAGES);
     const u32 b0 = k * SB, nb = std::min(SB, n - b0);
     u8 *stage = stage_view(e, dir, sg, nb).base;
-    for (u32 i = 0; i < nb; ++i) sorted_slots[h_pos[b0 + i]] = h_ids[b0 + i];
     auto transfers = [&]() -> int32_t {
       for (u32 p = 0; p < nb;) {
         u32 run = 1;
-        while (p + run < nb && sorted_slots[p + run] == sorted_slots[p] + run) ++run;
-        u8 *hp = host_pool + (u64)sorted_slots[p] * BB, *sp = stage + (u64)p * BB;
+        while (p + run < nb && host_sorted[b0 + p + run] == host_sorted[b0 + p] + run) ++run;
+        u8 *hp = host_pool + (u64)host_sorted[b0 + p] * BB, *sp = stage + (u64)p * BB;
         if (dir == 0) CU(cudaMemcpyAsync(hp, sp, run * BB, cudaMemcpyDeviceToHost, g.cs[0]));
         else CU(cudaMemcpyAsync(sp, hp, run * BB, cudaMemcpyHostToDevice, g.cs[1]));
         p += run;
@@ -490,7 +483,7 @@ int32_t staged_move(kvt_engine *e, cudaStream_t s, u32 st, const u32 *d_src, con
     };
     if (dir == 0) {
       if (k >= (u32)kvt_engine::N_STAGES) CU(cudaStreamWaitEvent(s, g.free_[0][sg], 0));   // the stage's transfers are done
-      int32_t r = launch_mover_views(e, s, pool_view(e, st), d_src + b0, stage_view(e, 0, sg, nb), d_pos + b0, nb, nullptr, 0, false);
+      r = launch_mover_views(e, s, pool_view(e, st), d_ids + b0, stage_view(e, 0, sg, nb), nullptr, nb, nullptr, 0, false);
       if (r) return r;
       CU(cudaEventRecord(g.ready[0][sg], s));
       CU(cudaStreamWaitEvent(g.cs[0], g.ready[0][sg], 0));
@@ -499,11 +492,11 @@ int32_t staged_move(kvt_engine *e, cudaStream_t s, u32 st, const u32 *d_src, con
       CU(cudaEventRecord(g.free_[0][sg], g.cs[0]));
     } else {
       if (k >= (u32)kvt_engine::N_STAGES) CU(cudaStreamWaitEvent(g.cs[1], g.free_[1][sg], 0));   // the stage was scattered
-      int32_t r = transfers();
+      r = transfers();
       if (r) return r;
       CU(cudaEventRecord(g.ready[1][sg], g.cs[1]));
       CU(cudaStreamWaitEvent(s, g.ready[1][sg], 0));
-      r = launch_mover_views(e, s, stage_view(e, 1, sg, nb), d_pos + b0, pool_view(e, dt), d_dst + b0, nb, nullptr, 0, false);
+      r = launch_mover_views(e, s, stage_view(e, 1, sg, nb), nullptr, pool_view(e, dt), d_ids + b0, nb, nullptr, 0, false);
       if (r) return r;
       CU(cudaEventRecord(g.free_[1][sg], s));
     }
@@ -519,10 +512,10 @@ int32_t staged_move(kvt_engine *e, cudaStream_t s, u32 st, const u32 *d_src, con
 // reloads (host -> HBM) arrive and are scattered on copy stream 1, so both copy engines work. A reload may land in
 // the HBM slot a victim of the same call leaves; payload copies are independent of the list order, so the victims
 // are gathered in the order the reload batches need their slots, and the scatter of a batch waits for the gather
-// of the last victim it depends on. All lists are host copies of what the plan kernels produced; in_dst stays on
-// the device (d_in_dst). When this returns, `s` waits for both copy streams.
-int32_t staged_exchange(kvt_engine *e, cudaStream_t s, u32 n_in, const u32 *in_src, const u32 *in_dst, const u32 *d_in_dst,
-                        u32 n_out, const u32 *out_src, const u32 *out_dst) {
+// of the last victim it depends on. All lists are host copies of what the plan kernels produced. When this
+// returns, `s` waits for both copy streams.
+int32_t staged_exchange(kvt_engine *e, cudaStream_t s, u32 n_in, const u32 *in_src, const u32 *in_dst, u32 n_out,
+                        const u32 *out_src, const u32 *out_dst) {
   kvt_engine::Staging &g = e->stg;
   const u32 SB = g.blocks_per_stage;
   const u64 BB = e->block_bytes;
@@ -530,6 +523,12 @@ int32_t staged_exchange(kvt_engine *e, cudaStream_t s, u32 n_in, const u32 *in_s
   for (u32 i = 0; i < n_in; ++i) if (in_src[i] >= e->cfg.n_host_blocks) return fail(e, KVT_E_RANGE, "slot id out of range");
   for (u32 i = 0; i < n_out; ++i) if (out_dst[i] >= e->cfg.n_host_blocks) return fail(e, KVT_E_RANGE, "slot id out of range");
   const u32 nbi = cdiv(n_in, SB), nbo = cdiv(n_out, SB);
+  // the reloads travel in the order of their host slots (long transfers); their HBM destinations follow that order
+  std::vector<u32> in_order(n_in), in_src_s(n_in), in_dst_s(n_in);
+  for (u32 i = 0; i < n_in; ++i) in_order[i] = i;
+  std::sort(in_order.begin(), in_order.end(), [&](u32 x, u32 y) { return in_src[x] < in_src[y]; });
+  for (u32 p = 0; p < n_in; ++p) { in_src_s[p] = in_src[in_order[p]]; in_dst_s[p] = in_dst[in_order[p]]; }
+  in_src = in_src_s.data(); in_dst = in_dst_s.data();
   // order of the victims: those whose slots the first reload batches need come first
   std::map<u32, u32> vic_of;
   for (u32 v = 0; v < n_out; ++v) vic_of[out_src[v]] = v;
@@ -546,8 +545,8 @@ int32_t staged_exchange(kvt_engine *e, cudaStream_t s, u32 n_in, const u32 *in_s
   for (u32 v = 0; v < n_out; ++v) if (!taken[v]) order.push_back(v);
   // device lists: victims' HBM slots in that order, and the place of every block inside its batch's stage (blocks
   // sit in the order of their host slots, so that consecutive host slots are one transfer)
-  u32 *h_osrc = e->h_ids, *h_opos = e->h_ids2, *h_ipos = (u32 *)e->h_out;
-  u32 *d_osrc = e->dp<u32>(e->L.ids), *d_opos = e->dp<u32>(e->L.ids2), *d_ipos = e->dp<u32>(e->L.s0);
+  u32 *h_osrc = e->h_ids, *h_opos = e->h_ids2, *h_ipos = (u32 *)e->h_out, *h_idst = h_ipos + e->L.LB;
+  u32 *d_osrc = e->dp<u32>(e->L.ids), *d_opos = e->dp<u32>(e->L.ids2), *d_ipos = e->dp<u32>(e->L.s0), *d_idst = e->dp<u32>(e->L.s1);
   std::vector<u32> ohost(n_out), isorted(n_in), osorted(n_out), idx(SB);
   for (u32 i = 0; i < n_out; ++i) { h_osrc[i] = out_src[order[i]]; ohost[i] = out_dst[order[i]]; }
   auto place = [&](const u32 *slots, u32 n, u32 *pos, std::vector<u32> &sorted) {
@@ -558,14 +557,17 @@ int32_t staged_exchange(kvt_engine *e, cudaStream_t s, u32 n_in, const u32 *in_s
       for (u32 p = 0; p < nb; ++p) { pos[b0 + idx[p]] = p; sorted[b0 + p] = slots[b0 + idx[p]]; }
     }
   };
-  std::vector<u32> in_src_copy(in_src, in_src + n_in);   // in_src lives in the staging area h_ipos is about to reuse
   place(ohost.data(), n_out, h_opos, osorted);
-  place(in_src_copy.data(), n_in, h_ipos, isorted);
+  place(in_src, n_in, h_ipos, isorted);
+  for (u32 p = 0; p < n_in; ++p) h_idst[p] = in_dst[p];
   if (n_out) {
     CU(cudaMemcpyAsync(d_osrc, h_osrc, n_out * 4ull, cudaMemcpyHostToDevice, s));
     CU(cudaMemcpyAsync(d_opos, h_opos, n_out * 4ull, cudaMemcpyHostToDevice, s));
   }
-  if (n_in) CU(cudaMemcpyAsync(d_ipos, h_ipos, n_in * 4ull, cudaMemcpyHostToDevice, s));
+  if (n_in) {
+    CU(cudaMemcpyAsync(d_ipos, h_ipos, n_in * 4ull, cudaMemcpyHostToDevice, s));
+    CU(cudaMemcpyAsync(d_idst, h_idst, n_in * 4ull, cudaMemcpyHostToDevice, s));
+  }
   {
     int32_t r = stage_release(e, s);
     if (r) return r;
@@ -604,7 +606,7 @@ int32_t staged_exchange(kvt_engine *e, cudaStream_t s, u32 n_in, const u32 *in_s
     int32_t r = transfers(1, isorted, b0, nb, stage_view(e, 1, sg, nb).base);
     if (r) return r;
     if (need[j]) CU(cudaStreamWaitEvent(g.cs[1], g.ready[0][(ko - 1) % NS], 0));   // the victims in the way have been gathered
-    r = launch_mover_views(e, g.cs[1], stage_view(e, 1, sg, nb), d_ipos + b0, pool_view(e, KVT_TIER_HBM), d_in_dst + b0, nb, nullptr, 0,
+    r = launch_mover_views(e, g.cs[1], stage_view(e, 1, sg, nb), d_ipos + b0, pool_view(e, KVT_TIER_HBM), d_idst + b0, nb, nullptr, 0,
                            false);
     if (r) return r;
   }
@@ -1782,7 +1784,7 @@ static int32_t list_op(kvt_engine *e, cudaStream_t s, u32 src_tier, u32 dst_tier
   r = status_code(e);
   if (r) return r;
   if (staged && e->h_status[ST_NLIVE]) {
-    r = staged_move(e, s, src_tier, a.pair_src, h_psrc, dst_tier, a.pair_dst, h_pdst, std::min(e->h_status[ST_NLIVE], n_pairs_max));
+    r = staged_move(e, s, src_tier, h_psrc, dst_tier, h_pdst, std::min(e->h_status[ST_NLIVE], n_pairs_max));
     if (r) return r;
     CU(cudaStreamSynchronize(s));
   }
@@ -1933,10 +1935,11 @@ int32_t kvt_exchange(kvt_engine *e, const uint32_t *hbm_slots_out, uint32_t n_ou
     if (r) return r;
     const u32 ni = std::min(e->h_status[ST_NLIVE], n_in), no = std::min(e->h_status[ST_B_NLIVE], n_out_max);
     if (ni + no) {
-      std::vector<u32> v_idst(h_idst, h_idst + ni), v_osrc(h_osrc, h_osrc + no), v_odst(h_odst, h_odst + no);   // the staging area is reused
+      // the staging area is reused by the call below: keep the lists aside
+      std::vector<u32> v_isrc(h_isrc, h_isrc + ni), v_idst(h_idst, h_idst + ni), v_osrc(h_osrc, h_osrc + no), v_odst(h_odst, h_odst + no);
       r = stage_acquire(e);
       if (r) return r;
-      r = staged_exchange(e, s, ni, h_isrc, v_idst.data(), a.pair_dst, no, v_osrc.data(), v_odst.data());
+      r = staged_exchange(e, s, ni, v_isrc.data(), v_idst.data(), no, v_osrc.data(), v_odst.data());
       if (r) return r;
       CU(cudaStreamSynchronize(s));
     }

@@ -102,6 +102,26 @@ def main(case: str):
         gb = n * geo.block_bytes / 1e9
         print(f"mover_host: {n} blocks x {geo.block_bytes} B; gather to host ms {g} = {[round(gb / (m / 1e3), 1) for m in g]} GB/s; "
               f"scatter from host ms {sc} = {[round(gb / (m / 1e3), 1) for m in sc]} GB/s")
+    elif case == "mover_staged":
+        # offload / reload through the staging ring and the copy engines (the default for blocks >= 512 KiB between HBM
+        # and a pinned host tier), against the same lists through the kernel that reads / writes host memory itself
+        geo, n = W.GEO_8B, 512
+        eng = B.Engine(n_hbm_blocks=n, n_host_blocks=n, max_contexts=2, max_tokens=1 << 16, max_messages=64,
+                       max_batch_blocks=4096, zero_pools=False, **geo.kwargs())
+        rng = np.random.default_rng(3)
+        eng.spawn(0)
+        eng.append(0, rng.integers(0, W.VOCAB, 16 * n, dtype=np.uint32))
+        eng.map_blocks([0], 0); eng.map_blocks([0], 1); eng.prefill_done(0)
+        gb = n * geo.block_bytes / 1e9
+        for variant, name in ((0, "staging ring + copy engines"), (2, "kernel over mapped host memory")):
+            eng.set_mover_variant(variant)
+            out = rng.permutation(n).astype(np.uint32)
+            for rep in range(2):
+                o = _events(torch, lambda: eng.offload(out), 1)
+                back = rng.permutation(n).astype(np.uint32)
+                r = _events(torch, lambda: eng.reload(back), 1)
+                print(f"mover_staged [{name}]: {n} blocks x {geo.block_bytes} B, permuted lists; offload {o[0]:.2f} ms = "
+                      f"{gb / (o[0] / 1e3):.1f} GB/s, reload {r[0]:.2f} ms = {gb / (r[0] / 1e3):.1f} GB/s")
     elif case == "mover_remote":
         # host tier <-> the buffer standing in for the remote tier (both pinned host memory): the mover reads over
         # the host link and writes back over it, so both directions of the link carry the payload at once
@@ -289,7 +309,10 @@ def main(case: str):
         for frac in (0.10, 0.35, 0.75):
             res[f"select_{int(frac * 100)}pct_ms"] = _events(torch, lambda: eng.select_victims(0, int(n_res * frac)), 3)
         res["lookup_batch_ms"] = _events(torch, lambda: eng.map_blocks(ids, 0), 1)
-        res["classify_ms"] = _events(torch, lambda: eng.classify(), 3)
+        res["classify_after_lookup_ms"] = _events(torch, lambda: eng.classify(), 1)      # event-driven: the batch's contexts
+        eng.set_classify_mode(1)
+        res["classify_full_ms"] = _events(torch, lambda: eng.classify(), 2)              # recomputed from zero
+        eng.set_classify_mode(0)
         v, _s = eng.select_victims(0, n_res // 10)
         res["drop_10pct_ms"] = _events(torch, lambda: eng.offload(v), 1)
         res["admit_batch_ms"] = _events(torch, lambda: eng.map_blocks(ids, 1), 1)
