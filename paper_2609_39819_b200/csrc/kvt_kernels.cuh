@@ -100,9 +100,13 @@ __device__ __forceinline__ void set_err(u32 *status, u32 bits) { atomicOr(&statu
 #define KVT_CHECK(cond, status, action) do { } while (0)
 #endif
 
+// Home slot of a key: the even slot of the pair its top bits select. Probe sequences start at an aligned pair, so
+// every two-slot step of a read-only probe reads one 32-byte sector.
+__device__ __forceinline__ u32 tab_home(const Table &t, u64 key) { return (u32)(key >> t.shift) & ~1u; }
+
 // Finds key; returns its table slot index or ENT_NONE. Stops at the first EMPTY slot.
 __device__ __forceinline__ u32 tab_find(const Table &t, u64 key, u32 *status) {
-  u32 i = (u32)(key >> t.shift);
+  u32 i = tab_home(t, key);
   for (u32 n = 0; n <= t.mask; ++n, i = (i + 1) & t.mask) {
     u64 k = t.slots[i].key;
     if (k == key) return i;
@@ -117,7 +121,7 @@ __device__ __forceinline__ u32 tab_find(const Table &t, u64 key, u32 *status) {
 // together), so a probe sequence of length p costs ceil(p / 2) dependent memory round trips and no extra one for
 // the entry id.
 __device__ __forceinline__ u32 tab_lookup_ent(const Table &t, u64 key, u32 *status) {
-  u32 i = (u32)(key >> t.shift);
+  u32 i = tab_home(t, key);
   for (u32 n = 0; n <= t.mask; n += 2) {
     const uint4 a = __ldg(reinterpret_cast<const uint4 *>(t.slots + i));
     const uint4 b = __ldg(reinterpret_cast<const uint4 *>(t.slots + ((i + 1) & t.mask)));
@@ -135,7 +139,7 @@ __device__ __forceinline__ u32 tab_lookup_ent(const Table &t, u64 key, u32 *stat
 // Finds key or claims the first EMPTY slot of its probe sequence for it (tombstones are skipped,
 // never reused, so two threads inserting the same key always meet in the same slot).
 __device__ __forceinline__ u32 tab_find_or_claim(const Table &t, u64 key, u32 *status) {
-  u32 i = (u32)(key >> t.shift);
+  u32 i = tab_home(t, key);
   for (u32 n = 0; n <= t.mask;) {
     u64 k = *(volatile u64 *)&t.slots[i].key;
     if (k == key) return i;
@@ -341,7 +345,7 @@ __device__ __forceinline__ void tab_lookup_ents(const Table &t, const u64 (&key)
   bool open[ILP];
   bool any = false;
 #pragma unroll
-  for (int q = 0; q < ILP; ++q) { i[q] = (u32)(key[q] >> t.shift); open[q] = active[q]; ent[q] = ENT_NONE; any = any || open[q]; }
+  for (int q = 0; q < ILP; ++q) { i[q] = tab_home(t, key[q]); open[q] = active[q]; ent[q] = ENT_NONE; any = any || open[q]; }
   for (u32 n = 0; any && n <= t.mask; n += 2) {
     uint4 a[ILP], b[ILP];
 #pragma unroll
