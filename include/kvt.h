@@ -7,7 +7,7 @@
  *       (Section 4.1, Table 3: append / replace / remove / fork / spawn / one_off),
  *   (2) lookup of those hashes in a GPU-resident open-addressing block table (reusable prefix),
  *   (3) derivation of each resident block's KV-level lifecycle state from message-level states
- *       (Section 5.2 state machine; Section 6.1 "Managing Shared KV"),
+ *       (Section 5.2 state machine; Section 6.1, the paragraph on KV shared between contexts),
  *   (4) state-prioritised, recency-ordered victim selection (Algorithm 1; Section 6.2), and
  *   (5) movement of paged KV blocks between the HBM pool, a pinned host tier and an optional third tier (Section 7).
  *
@@ -250,7 +250,7 @@ int32_t kvt_map_blocks(kvt_engine *e, const uint32_t *ctx_ids, uint32_t n_ctx, u
 int32_t kvt_get_block_map(kvt_engine *e, uint32_t ctx, uint64_t *keys, uint8_t *tier,
                           uint32_t *slot, uint32_t cap, uint32_t *n, void *stream);
 
-/* ---- stage 3: KV-level lifecycle state (Section 6.1 "Managing Shared KV") -------------------- */
+/* ---- stage 3: KV-level lifecycle state (Section 6.1, KV shared between contexts) ------------- */
 /* Brings the KV-level state of every resident block up to date: the highest-priority state over all (context,
  * message version) mappings of its key; a block nobody maps is dead. The engine keeps, per block, the number of
  * mappings of each priority and updates these counts by events (Section 6.1: the aggregate is updated whenever a

@@ -10,7 +10,7 @@
 //     Section 5.1 (KV scope resolution: suffix invalidation, KV-existence gating, program order)
 //     and Section 5.2 (runtime transitions; remove/replace; fork; one_off);
 //   - KV-level state of a shared block = highest-priority mapped message state, dead when every
-//     mapped version is Discarded: Section 6.1 "Managing Shared KV";
+//     mapped version is Discarded: Section 6.1 (KV shared between contexts);
 //   - release order Expired/Temporary -> Suspended -> Active and "admit iff Delta <= 0":
 //     Algorithm 1; most-recently-suspended-first inside the Suspended tier: Section 6.2; the
 //     oldest-first switch is the "w/o RO" variant of Section 8.3;
@@ -48,7 +48,7 @@ enum : uint32_t { ORDER_MRU = 0, ORDER_LRU = 1 };
 enum : uint32_t {
   POLICY_NO_LIFECYCLE = 1,   // the "w/o LT" variant of Section 8.3
   POLICY_ORPHANS_DEAD = 4,   // a context's mappings stop counting at its first non-resident block
-  POLICY_INCLUSIVE = 2       // a reloaded block keeps its host copy (Section 7: per-tier caching keeps a fast copy)
+  POLICY_INCLUSIVE = 2       // a reloaded block keeps its host copy (Section 7: a tier may keep a copy of a page that has moved on)
 };
 enum : uint32_t {
   OP_SPAWN = 1, OP_FORK, OP_APPEND, OP_REPLACE, OP_REMOVE, OP_ONE_OFF, OP_PREFILL_DONE,

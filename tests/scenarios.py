@@ -106,7 +106,7 @@ def fork_and_shared_kv(make):
     # the child still holds a Suspended reference to blocks 2,3 -> they stay Suspended.
     eng.remove(0, 1, 2)
     assert states(eng)[:8] == [IDLE, IDLE, IDLE, IDLE, DEAD, DEAD, IDLE, IDLE]
-    # Discarded only when all mapped versions are: now the child goes too
+    # the block dies only once nobody maps it any more (Section 6.1): now the child goes too
     eng.terminate(1)
     assert states(eng)[:8] == [IDLE, IDLE] + [DEAD] * 6
     # execution in one context does not touch the other's message states
