@@ -75,12 +75,13 @@ def test_hash_full_size_batch_matches_oracle(B, oracle):
 
 
 # ---- whole path on C1 traces: every reported value and every payload byte ----------------------------
-def _replay_pair(gpu, cpu, trace, payload, check_pools=True, record_states=True, verify_every=0, use_exchange=False):
+def _replay_pair(gpu, cpu, trace, payload, check_pools=True, record_states=True, verify_every=0, use_exchange=False,
+                 cross_check=True):
     og = W.ReplayOptions(payload=payload, record_states=record_states, verify_payload_every=verify_every,
                          use_exchange=use_exchange)
     oc = W.ReplayOptions(payload=payload, record_states=record_states, verify_payload_every=verify_every,
                          use_exchange=use_exchange)
-    if gpu.n_hbm_blocks + gpu.n_host_blocks <= 8192:
+    if cross_check and gpu.n_hbm_blocks + gpu.n_host_blocks <= 8192:
         gpu.set_classify_mode(2)      # small pools: every event-driven update is cross-checked against a full recomputation
     n_calls = 0
     for (i, kind, rg), (_, _, rc) in zip(W.replay(gpu, trace, og), W.replay(cpu, trace, oc)):
@@ -108,6 +109,17 @@ def test_c1_trace_parity(B, oracle, seed):
     gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)
     cpu = oracle.OracleEngine(**kw)
     _replay_pair(gpu, cpu, W.trace_c1(seed), W.payload_normal_bf16, verify_every=2)
+
+
+@pytest.mark.parametrize("first", [1, 51, 101, 151])
+def test_c1_trace_parity_seeds_1_to_200(B, oracle, first):
+    """The tiny configuration on seeds 1 .. 200 (fifty per case), metadata and payload bytes, one engine pair per seed."""
+    kw = dict(n_hbm_blocks=128, n_host_blocks=512, max_contexts=64, **W.GEO_TOY.kwargs())
+    for seed in range(first, first + 50):
+        gpu = B.Engine(max_tokens=1 << 18, max_messages=4096, **kw)
+        cpu = oracle.OracleEngine(**kw)
+        _replay_pair(gpu, cpu, W.trace_c1(seed), W.payload_normal_bf16, record_states=False)
+        gpu.close()
 
 
 @pytest.mark.parametrize("layout,order", [(0, 1), (1, 0), (1, 1)])
