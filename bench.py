@@ -659,7 +659,7 @@ def metadata_stress(torch, B, hbm_peak, reps=5):
         a.record(); r = fn(); b.record(); torch.cuda.synchronize()
         return a.elapsed_time(b), r
 
-    look_ms, cls_ms, sel_ms, cls_edit_ms, cls_full_ms, cls_done_ms = [], [], [], [], [], []
+    look_ms, cls_ms, sel_ms, cls_edit_ms, cls_full_ms, cls_done_ms, cls_k, cls_edit_k, cls_edit_warm_ms, cls_edit_warm_k = [], [], [], [], [], [], [], [], [], []
     s0 = None
     flush = torch.empty(1 << 29, dtype=torch.uint8, device="cuda")   # 512 MiB > L2: every timed call starts cold
     for rep in range(reps + 1):
@@ -672,7 +672,9 @@ def metadata_stress(torch, B, hbm_peak, reps=5):
         ms, info = timed(lambda: eng.map_blocks(ids, 0))
         look_ms.append(ms)
         flush.fill_(rep + 1)
+        c0 = eng.get_stats()
         cls_ms.append(timed(lambda: eng.classify())[0])      # event-driven: the 64 contexts of the batch are new mappings
+        cls_k.append((eng.get_stats()["classify_ns"] - c0["classify_ns"]) / 1e6)
         eng.set_classify_mode(1)                             # the full recomputation over all contexts, for comparison
         flush.fill_(rep + 1)
         cls_full_ms.append(timed(lambda: eng.classify())[0])
@@ -683,9 +685,13 @@ def metadata_stress(torch, B, hbm_peak, reps=5):
         cls_done_ms.append(timed(lambda: eng.classify())[0])  # every context's messages went from Active to Suspended
         eng.pin(0, 0, 1)                                     # one context's message changes state: 16,128 of its blocks
         flush.fill_(rep + 1)
+        c0 = eng.get_stats()
         cls_edit_ms.append(timed(lambda: eng.classify())[0])
-        eng.unpin(0, 0, 1)
-        eng.classify()
+        cls_edit_k.append((eng.get_stats()["classify_ns"] - c0["classify_ns"]) / 1e6)
+        eng.unpin(0, 0, 1)                                   # and back, this time with whatever the caches hold
+        c0 = eng.get_stats()
+        cls_edit_warm_ms.append(timed(lambda: eng.classify())[0])
+        cls_edit_warm_k.append((eng.get_stats()["classify_ns"] - c0["classify_ns"]) / 1e6)
         flush.fill_(rep + 2)
         torch.cuda.synchronize()
         ms, (v, _st) = timed(lambda: eng.select_victims(0, n_res // 10))
@@ -710,9 +716,13 @@ def metadata_stress(torch, B, hbm_peak, reps=5):
                         "frac_hbm": n_blocks * 136 / (look_k / 1e3) / 1e9 / hbm_peak},
         "classify": {"mappings": n_blocks, "entries": n_res, "call_ms": med(cls_ms),
                      "what": "event-driven update after the LOOKUP batch: 64 new contexts x 16,128 mappings",
-                     "achieved_GBs": 16 * n_blocks / (med(cls_ms) / 1e3) / 1e9,
-                     "frac_hbm": 16 * n_blocks / (med(cls_ms) / 1e3) / 1e9 / hbm_peak,
+                     "kernels_ms": med(cls_k),
+                     "achieved_GBs": 16 * n_blocks / (med(cls_k) / 1e3) / 1e9,
+                     "frac_hbm": 16 * n_blocks / (med(cls_k) / 1e3) / 1e9 / hbm_peak,
                      "after_one_context_changed_state_ms": med(cls_edit_ms),
+                     "after_one_context_changed_state_kernels_ms": med(cls_edit_k),
+                     "after_one_context_changed_state_warm_l2_ms": med(cls_edit_warm_ms),
+                     "after_one_context_changed_state_warm_l2_kernels_ms": med(cls_edit_warm_k),
                      "after_all_contexts_suspended_ms": med(cls_done_ms),
                      "full_recomputation_ms": med(cls_full_ms)},
         "select": {"resident": n_res, "victims": len(v), "call_ms": med(sel_ms), "kernels_ms": sel_k,

@@ -396,6 +396,8 @@ typedef struct kvt_stats {
   uint64_t hits_remote;      /* reusable-prefix blocks found in the remote tier */
   uint64_t demoted;          /* blocks moved host -> remote */
   uint64_t promoted;         /* blocks moved remote -> host or remote -> HBM */
+  uint64_t classify_ns;      /* with profiling on: device time of the classification kernels */
+  uint64_t classify_items;   /* and the (context, block) mappings they visited */
 } kvt_stats;
 int32_t kvt_get_stats(kvt_engine *e, kvt_stats *out);
 

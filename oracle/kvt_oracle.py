@@ -64,7 +64,7 @@ STATS_FIELDS = ("clock", "n_contexts", "occ_hbm", "occ_host", "blocks_hashed", "
                 "inserted", "adopted", "dropped", "offloaded", "reloaded", "compacted", "bytes_d2h", "bytes_h2d",
                 "bytes_d2d", "table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns",
                 "mover_bytes", "lookup_ns", "lookup_blocks", "select_ns", "select_slots", "offloaded_clean",
-                "blocks_rehashed", "occ_remote", "hits_remote", "demoted", "promoted")
+                "blocks_rehashed", "occ_remote", "hits_remote", "demoted", "promoted", "classify_ns", "classify_items")
 
 _lib = None
 

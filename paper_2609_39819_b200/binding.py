@@ -66,7 +66,7 @@ STATS_FIELDS = ("clock", "n_contexts", "occ_hbm", "occ_host", "blocks_hashed", "
                 "inserted", "adopted", "dropped", "offloaded", "reloaded", "compacted", "bytes_d2h", "bytes_h2d",
                 "bytes_d2d", "table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns",
                 "mover_bytes", "lookup_ns", "lookup_blocks", "select_ns", "select_slots", "offloaded_clean",
-                "blocks_rehashed", "occ_remote", "hits_remote", "demoted", "promoted")
+                "blocks_rehashed", "occ_remote", "hits_remote", "demoted", "promoted", "classify_ns", "classify_items")
 
 _lib = None
 
@@ -341,7 +341,7 @@ class Engine:
         if rc not in (OK, E_BUFSZ):
             self._check(rc, "get_block_map")
         nb = n.value
-        keys = np.zeros(nb, np.uint64); tier = np.zeros(nb, np.uint8); slot = np.zeros(nb, np.uint32)
+        keys = np.empty(nb, np.uint64); tier = np.empty(nb, np.uint8); slot = np.empty(nb, np.uint32)
         self._check(self.L.kvt_get_block_map(self.h, ctx, _p(keys), _p(tier), _p(slot), nb, C.byref(n), _stream()),
                     "get_block_map")
         return keys, tier, slot
@@ -361,11 +361,11 @@ class Engine:
 
     def select_victims(self, tier, n_req, include_pinned=False):
         cap = min(n_req, self._tier_size(tier))
-        slots = np.zeros(cap, np.uint32); states = np.zeros(cap, np.uint8)
+        slots = np.empty(cap, np.uint32); states = np.empty(cap, np.uint8)     # filled by the call up to n
         n = C.c_uint32(0)
         self._check(self.L.kvt_select_victims(self.h, tier, n_req, 1 if include_pinned else 0, _p(slots), _p(states),
                                               cap, C.byref(n), _stream()), "select_victims")
-        return slots[:n.value].copy(), states[:n.value].copy()
+        return slots[:n.value], states[:n.value]
 
     # ---- movement -------------------------------------------------------------------------------
     def offload(self, slots):

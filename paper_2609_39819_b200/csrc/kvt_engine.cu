@@ -204,7 +204,8 @@ struct kvt_engine {
   u32 lookup_variant = 0;  // 0 / 1 digest / carry / finish kernels, 2 single-pass hash + probe kernel
   u32 wait_limit = 1u << 18;   // polls a chunk of the single-pass kernel spends on its predecessors before it gives up
   bool tma_attr_set = false;
-  cudaEvent_t ev_m0 = nullptr, ev_m1 = nullptr, ev_h0 = nullptr, ev_h1 = nullptr;
+  cudaEvent_t ev_m0 = nullptr, ev_m1 = nullptr, ev_h0 = nullptr, ev_h1 = nullptr, ev_c0 = nullptr, ev_c1 = nullptr;
+  bool classify_timed = false; u64 classify_pending_items = 0;   // a timed classification whose events have not been read yet
 
   template <class T> T *dp(u64 off) const { return reinterpret_cast<T *>(meta + off); }
   u32 tier_slots(u32 t) const { return t == KVT_TIER_HBM ? cfg.n_hbm_blocks : t == KVT_TIER_HOST ? cfg.n_host_blocks : cfg.n_remote_blocks; }
@@ -710,7 +711,10 @@ int32_t apply_deltas(kvt_engine *e, cudaStream_t s, const std::vector<Ctx *> &li
       CU(cudaMemsetAsync(a.first_miss, 0xFF, nd * 4ull, s));
       KL(k_first_miss, cdiv(nmap, TPB), TPB, s, a);
     }
+    const bool timed = e->profiling && !e->classify_timed;
+    if (timed) CU(cudaEventRecord(e->ev_c0, s));
     KL(k_map_delta, cdiv(nmap, TPB), TPB, s, a);
+    if (timed) { CU(cudaEventRecord(e->ev_c1, s)); e->classify_timed = true; e->classify_pending_items = nmap; }
     LAUNCH_CHECK();
   }
   // what is accounted for now
@@ -983,7 +987,8 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   if (CHECKED_BUILD) e->use_graphs = false;
   bool ok = cudaEventCreateWithFlags(&e->ev_upload, cudaEventDisableTiming) == cudaSuccess &&
             cudaEventCreate(&e->ev_m0) == cudaSuccess && cudaEventCreate(&e->ev_m1) == cudaSuccess &&
-            cudaEventCreate(&e->ev_h0) == cudaSuccess && cudaEventCreate(&e->ev_h1) == cudaSuccess;
+            cudaEventCreate(&e->ev_h0) == cudaSuccess && cudaEventCreate(&e->ev_h1) == cudaSuccess &&
+            cudaEventCreate(&e->ev_c0) == cudaSuccess && cudaEventCreate(&e->ev_c1) == cudaSuccess;
   // everything except the key arena and scratch must start at zero; the table needs ent = NONE
   ok = ok && cudaMemsetAsync(e->meta + L.e_key, 0, L.keys - L.e_key, s) == cudaSuccess;
   ok = ok && cudaMemsetAsync(e->d_status, 0, ST_WORDS * 4, s) == cudaSuccess;
@@ -1015,6 +1020,8 @@ int32_t kvt_destroy(kvt_engine *e) {
   if (e->ev_m1) cudaEventDestroy(e->ev_m1);
   if (e->ev_h0) cudaEventDestroy(e->ev_h0);
   if (e->ev_h1) cudaEventDestroy(e->ev_h1);
+  if (e->ev_c0) cudaEventDestroy(e->ev_c0);
+  if (e->ev_c1) cudaEventDestroy(e->ev_c1);
   if (e->stage) cudaFreeHost(e->stage);
   delete e;
   return KVT_OK;
@@ -1065,6 +1072,13 @@ int32_t kvt_debug_set_wait_limit(kvt_engine *e, uint32_t polls) {
 
 int32_t kvt_get_stats(kvt_engine *e, kvt_stats *out) {
   if (!e || !out) return KVT_E_INVAL;
+  if (e->classify_timed && cudaEventQuery(e->ev_c1) == cudaSuccess) {   // classification is asynchronous: its time is read here
+    float ms = 0.f;
+    if (cudaEventElapsedTime(&ms, e->ev_c0, e->ev_c1) == cudaSuccess) {
+      e->st.classify_ns += (u64)((double)ms * 1e6); e->st.classify_items += e->classify_pending_items;
+    }
+    e->classify_timed = false;
+  }
   kvt_stats s = e->st;
   s.clock = e->now;
   s.n_contexts = 0;
@@ -1621,12 +1635,12 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   a.slot_bits = bit_length(n - 1);
   {
     u32 left = key_bits + a.slot_bits, lev = 0;
-    while (left) {
+    do {   // the search needs no further level once a bin cannot hold more than SEL_SLACK composites (they are unique)
       const u32 w = std::min(left, lev == 0 ? SEL_W0 : SEL_WN);
       left -= w;
       a.lev_lo[lev] = (u8)left; a.lev_w[lev] = (u8)w;
       ++lev;
-    }
+    } while (left && (1ull << left) > SEL_SLACK);
     a.n_levels = lev;
   }
   u64 *kA = e->dp<u64>(e->L.keyA), *kB = e->dp<u64>(e->L.keyB);

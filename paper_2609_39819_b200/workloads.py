@@ -22,7 +22,7 @@ TIER_HBM, TIER_HOST, TIER_REMOTE, TIER_NONE = 0, 1, 2, 0xFF
 MAP_LOOKUP, MAP_ADMIT = 0, 1
 GiB = 1 << 30
 GPU_ONLY_STATS = ("table_rebuilds", "tombstones", "kernel_launches", "mover_launches", "mover_ns", "mover_bytes",
-                  "lookup_ns", "lookup_blocks", "select_ns", "select_slots", "blocks_rehashed")
+                  "lookup_ns", "lookup_blocks", "select_ns", "select_slots", "blocks_rehashed", "classify_ns", "classify_items")
 STATE_COPY, STATE_HAS_COPY = 0xFE, 0x80
 
 
