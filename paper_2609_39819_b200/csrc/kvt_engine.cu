@@ -1652,7 +1652,10 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   const u32 n_emit = std::min(n_req, n);
   const u32 m_max = (u32)std::min<u64>((u64)n_emit + SEL_SLACK, n);   // the gathered set never exceeds this
   a.n_emit = n_emit; a.rank_shift = a.stamp_bits + a.depth_bits;
-  a.slots_out = e->dp<u32>(e->L.out_slots); a.states_out = e->dp<u8>(e->L.out_states);
+  // the victim list is written by the last kernel straight into the pinned staging area (mapped into the device's
+  // address space like every pinned allocation): no copy after the kernels, the list is there when the stream is
+  u32 *h_slots = (u32 *)e->h_out; u8 *h_states = e->h_out + n_emit * 4ull;
+  a.slots_out = h_slots; a.states_out = h_states;
   const SelArgs *d_args = e->dp<SelArgs>(e->L.sel_args);
   CU(cudaMemcpyAsync((void *)d_args, &a, sizeof(SelArgs), cudaMemcpyHostToDevice, s));
   rr = stage_release(e, s);
@@ -1686,10 +1689,11 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
       if (count) TRACE(q, "scatter");
       std::swap(ka, kb); std::swap(va, vb);
     }
-    k_sel_emit<<<std::min<u32>(cdiv(n, 256), (u32)e->sm_count * 8), 256, 0, q>>>(d_args, ka, va);
-    if (count) TRACE(q, "emit");
-    if (count) e->st.kernel_launches += 3ull + (n_levels - 1) + 3ull * n_pass + 1;
+    if (count) e->st.kernel_launches += 3ull + (n_levels - 1) + 3ull * n_pass;
   };
+  // where the sorted pairs end up: the passes swap the two buffers
+  const u64 *k_final = (n_pass & 1) ? kB : kA;
+  const u32 *v_final = (n_pass & 1) ? vB : vA;
   if (e->profiling) CU(cudaEventRecord(e->ev_h0, s));
   {
     kvt_engine::SelGraph &gr = e->sel_graph[tier][(u64)n_levels << 48 | (u64)n_pass << 32 | tiles];
@@ -1706,17 +1710,14 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
     }
     if (e->use_graphs && gr.exec) {
       CU(cudaGraphLaunch(gr.exec, s));
-      e->st.kernel_launches += 3ull + (n_levels - 1) + 3ull * n_pass + 1;
+      e->st.kernel_launches += 3ull + (n_levels - 1) + 3ull * n_pass;
     } else {
       enqueue(s, true);
     }
   }
-  if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));
+  if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));   // selection and sort; the list's way to the host comes after
+  KL(k_sel_emit, std::min<u32>(cdiv(n_emit, 256), (u32)e->sm_count * 8), 256, s, d_args, k_final, v_final);
   LAUNCH_CHECK();
-  // the victim list (at most n_emit entries) travels with the status block: one synchronisation
-  u32 *h_slots = (u32 *)e->h_out; u8 *h_states = e->h_out + n_emit * 4ull;
-  CU(cudaMemcpyAsync(h_slots, e->dp<u32>(e->L.out_slots), n_emit * 4ull, cudaMemcpyDeviceToHost, s));
-  if (states_out) CU(cudaMemcpyAsync(h_states, e->dp<u8>(e->L.out_states), n_emit, cudaMemcpyDeviceToHost, s));
   r = status_fetch(e, s);
   if (r) return r;
   TRACE_DUMP("select");
