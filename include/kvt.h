@@ -420,11 +420,12 @@ int32_t kvt_debug_set_mover_variant(kvt_engine *e, uint32_t variant);
  * into a few large blocks leaves all other SMs to kernels running on other streams at the same time. */
 int32_t kvt_set_mover_ctas(kvt_engine *e, uint32_t max_ctas);
 
-/* Tuning hook: how kvt_map_blocks(LOOKUP) hashes and probes. 0 / 1 = three kernels (digest, carry scan, finish +
+/* Tuning hook: how kvt_map_blocks(LOOKUP) hashes and probes. 0 / 1 = two kernels (digest; chunk carry + finish +
  * probe; default), 2 = one single-pass kernel in which chunks hand their chain values forward through device
- * memory (bounded waits; a wait that runs out makes the call return KVT_E_DEVICE), 3 / 4 = the three kernels with
- * two / four keys per thread in the probe. Results are identical; on B200 the single pass measured slower (its CTAs
- * live too long to keep enough token bytes in flight) and the wider probes the same as the default. */
+ * memory (bounded waits; a wait that runs out makes the call return KVT_E_DEVICE), 3 / 4 = the default kernels with
+ * one / four keys per thread in the probe instead of two. Results are identical; on B200 the single pass measured
+ * slower (its CTAs live too long to keep enough token bytes in flight) and the other probe widths within 3 % of the
+ * default. */
 int32_t kvt_debug_set_lookup_variant(kvt_engine *e, uint32_t variant);
 
 /* Test / measurement hook for the classification: 0 = event-driven (default), 1 = every kvt_classify recomputes all

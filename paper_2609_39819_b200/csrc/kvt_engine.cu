@@ -1374,12 +1374,11 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     if (e->profiling) CUR(cudaEventRecord(e->ev_h0, s));
     if (e->lookup_variant != 2) {
       if (dchunk_base) KL(k_hash_digest, dchunk_base, CHUNK, s, ha);
-      KL(k_hash_carry, nd, 1024, s, ha);
-      // one key per thread by default; two or four (more table loads in flight per thread) measured the same: the
-      // probes of a cold table are bound by the rate of random 32-byte sectors, not by latency per thread
-      if (e->lookup_variant == 3) KL(k_hash_finish_lookup<2>, chunk_base, CHUNK / 2, s, ha, la);
+      // two keys per thread by default; one or four measured within 3 % of it: the probes of a cold table are bound
+      // by the number of outstanding misses the memory system carries, not by what a thread issues
+      if (e->lookup_variant == 3) KL(k_hash_finish_lookup<1>, chunk_base, CHUNK, s, ha, la);
       else if (e->lookup_variant == 4) KL(k_hash_finish_lookup<4>, chunk_base, CHUNK / 4, s, ha, la);
-      else KL(k_hash_finish_lookup<1>, chunk_base, CHUNK, s, ha, la);
+      else KL(k_hash_finish_lookup<2>, chunk_base, CHUNK / 2, s, ha, la);
     } else {
       ChainState cs;
       cs.flags = e->dp<u32>(e->L.cflags); cs.ticket = cs.flags + chunk_base; cs.incl = e->dp<u64>(e->L.carry);
@@ -2109,7 +2108,6 @@ int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t ha
   ha.agg = (u64 *)d_scratch; ha.carry_base = (u64 *)d_scratch + n_chunks; ha.h0 = hash_h0(hash_seed);
   LookupArgs la{};
   k_hash_digest<<<n_chunks, CHUNK, 0, s>>>(ha);
-  k_hash_carry<<<1, 1024, 0, s>>>(ha);
   k_hash_finish_lookup<1><<<n_chunks, CHUNK, 0, s>>>(ha, la);
   return cudaGetLastError() == cudaSuccess ? KVT_OK : KVT_E_CUDA;
 }
@@ -2142,7 +2140,6 @@ int32_t kvt_hash_tokens_noalloc(const uint32_t *d_tokens, uint64_t n_tokens, uin
   ha.agg = scratch; ha.carry_base = scratch + NOALLOC_MAX_CHUNKS; ha.h0 = hash_h0(hash_seed);
   LookupArgs la{};
   k_hash_digest<<<n_chunks, CHUNK, 0, s>>>(ha);
-  k_hash_carry<<<1, 1024, 0, s>>>(ha);
   k_hash_finish_lookup<1><<<n_chunks, CHUNK, 0, s>>>(ha, la);
   return cudaGetLastError() == cudaSuccess ? KVT_OK : KVT_E_CUDA;
 }

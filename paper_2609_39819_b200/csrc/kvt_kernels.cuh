@@ -156,13 +156,13 @@ __device__ __forceinline__ u32 tab_find_or_claim(const Table &t, u64 key, u32 *s
 }
 
 // ======================================================================================================
-// K1: block hasher. 3 phases, no inter-CTA waits:
+// K1: block hasher. Two kernels, no inter-CTA waits:
 //   digest : per 256-block chunk, 4 lanes per block read 16 B each, weighted sums, mix, then a CTA-wide
 //            scan of the affine chain with zero carry-in -> partial chain values + chunk aggregate
-//   carry  : one CTA per context scans its chunk aggregates, 1024 chunks per step
+//   finish : every chunk's CTA folds the aggregates of the chunks before it into the chain value entering its
+//            chunk (carry), then h = P^(i+1) * carry + partial, key = mix64(h); fused with the table probe
 // Incremental: a sequence whose leading blocks are unchanged since its previous key list only digests from the
 // last chunk boundary before the first changed block (the chain restarts from the carry kept for that chunk).
-//   finish : h = P^(i+1) * carry + partial, key = mix64(h); fused with the table probe
 // ======================================================================================================
 // One sequence of a batch. Blocks [0, first) keep the keys of the previous key list (first is a multiple of
 // CHUNK): only chunks from first / CHUNK on are digested, restarting the chain from the carry stored for that
@@ -276,59 +276,6 @@ __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   if (tid == nb - 1) a.agg[blockIdx.x] = cval;
 }
 
-// One CTA per sequence: the chain value entering chunk g0 + j is A^j * C0 + sum_{i<j} A^(j-1-i) * agg_i with
-// A = P^CHUNK (every chunk before the last is full) and C0 the value entering chunk g0 = first / CHUNK (H0, or the
-// carry kept from the previous key list), evaluated 1024 chunks at a time: a warp scan per 32 chunks, a scan of
-// the 32 warp totals, then the carry of the previous 1024. Also copies the kept carries of chunks < g0.
-__global__ void __launch_bounds__(1024) k_hash_carry(HashArgs a) {
-  __shared__ u64 wtot[32], wpre[32], sv[1024];
-  const u32 i = blockIdx.x;
-  if (i >= a.n_ctx) return;
-  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const HashCtx c = a.ctx ? a.ctx[i] : a.single;
-  const u32 g0 = c.first / CHUNK;
-  const u32 n_chunks = (c.n_blocks - c.first + CHUNK - 1) / CHUNK;   // chunks that were digested
-  for (u32 k = tid; k < g0; k += 1024) a.carry_base[c.carry_off + k] = a.carry_base[c.old_carry_off + k];
-  const u64 A = g_pow_p.v[CHUNK];
-  const u64 A32 = pow_u64(A, 32);
-  const u64 a_lane = pow_u64(A, lane + 1);          // A^(lane+1)
-  const u64 a_tid = pow_u64(A32, warp) * a_lane;    // A^(tid+1)
-  u64 carry = g0 ? a.carry_base[c.old_carry_off + g0] : a.h0;
-  if (n_chunks == 0 && tid == 0) a.carry_base[c.carry_off + g0] = carry;   // nothing new: keep the resume point
-  for (u32 base = 0; base < n_chunks; base += 1024) {
-    const u32 j = base + tid;
-    u64 x = j < n_chunks ? a.agg[c.dchunk_base + j] : 0;
-    u64 pp = A;
-#pragma unroll
-    for (u32 o = 1; o < 32; o <<= 1) {
-      u64 up = __shfl_up_sync(0xFFFFFFFFu, x, o);
-      if (lane >= o) x += pp * up;
-      pp *= pp;
-    }
-    if (lane == 31) wtot[warp] = x;
-    __syncthreads();
-    if (warp == 0) {   // value at the end of every earlier warp of this round, with zero carry-in
-      u64 y = wtot[lane], qq = A32;
-#pragma unroll
-      for (u32 o = 1; o < 32; o <<= 1) {
-        u64 up = __shfl_up_sync(0xFFFFFFFFu, y, o);
-        if (lane >= o) y += qq * up;
-        qq *= qq;
-      }
-      u64 e = __shfl_up_sync(0xFFFFFFFFu, y, 1);
-      wpre[lane] = lane ? e : 0;
-    }
-    __syncthreads();
-    sv[tid] = a_tid * carry + a_lane * wpre[warp] + x;   // chain value after chunk g0 + j
-    __syncthreads();
-    if (j < n_chunks) a.carry_base[c.carry_off + g0 + j] = tid ? sv[tid - 1] : carry;
-    // value after the last chunk: the resume point of a later call if that chunk is full
-    if (j == n_chunks - 1) a.carry_base[c.carry_off + g0 + n_chunks] = sv[tid];
-    carry = sv[1023];
-    __syncthreads();
-  }
-}
-
 struct LookupArgs {
   Table tab;            // slots == nullptr: hash only
   u32 *b_ent;           // per batch block: entry id or ENT_NONE
@@ -369,31 +316,69 @@ __device__ __forceinline__ void tab_lookup_ents(const Table &t, const u64 (&key)
   if (any) set_err(status, DERR_PROBE);
 }
 
+// Chain value entering chunk j of a sequence (j counted from the first digested chunk g0 = first / CHUNK):
+// A^m C0 + sum_{i<m} A^(m-1-i) agg_i with m = j - g0, A = P^CHUNK (every chunk before the last is full) and C0 the
+// value entering chunk g0 (H0, or the carry kept from the previous key list). Every thread of the CTA calls it;
+// the terms are spread over the threads and summed.
+template <u32 T>
+__device__ __forceinline__ u64 chunk_carry(const HashArgs &a, const HashCtx &c, u32 j) {
+  __shared__ u64 s_part[T / 32];
+  const u32 g0 = c.first / CHUNK, m = j - g0, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const u64 A = g_pow_p.v[CHUNK];
+  u64 sum = 0;
+  for (u32 i = tid; i < m; i += T) sum += pow_u64(A, m - 1 - i) * a.agg[c.dchunk_base + i];
+  if (tid == 0) sum += pow_u64(A, m) * (g0 ? a.carry_base[c.old_carry_off + g0] : a.h0);
+#pragma unroll
+  for (u32 o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
+  if (lane == 0) s_part[warp] = sum;
+  __syncthreads();
+  u64 total = 0;
+#pragma unroll
+  for (u32 w = 0; w < T / 32; ++w) total += s_part[w];
+  return total;
+}
+
 // One CTA of CHUNK / ILP threads per 256-block chunk; thread t finishes and probes blocks t, t + CHUNK / ILP, ...
+// The CTA first works out the chain value entering its chunk from the chunk aggregates of the digest kernel (no
+// separate scan kernel) and stores it next to the keys, where a later call resumes from it.
 template <int ILP>
 __global__ void __launch_bounds__(CHUNK / ILP) k_hash_finish_lookup(HashArgs a, LookupArgs l) {
   constexpr u32 T = CHUNK / ILP;
   const u32 tid = threadIdx.x;
   u32 ci;
   const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci);
-  const u32 b0 = (blockIdx.x - c.chunk_base) * CHUNK;
+  const u32 j = blockIdx.x - c.chunk_base;
+  const u32 b0 = j * CHUNK;
   const u32 nb = min(CHUNK, c.n_blocks - b0);
   u64 key[ILP];
   bool act[ILP];
   const bool kept = b0 < c.first;                                   // unchanged prefix: the keys of the previous list still hold
-  const u64 carry = kept ? 0 : a.carry_base[c.carry_off + (blockIdx.x - c.chunk_base)];
+  u64 carry = 0;
+  if (kept) {
+    if (tid == 0) {
+      a.carry_base[c.carry_off + j] = a.carry_base[c.old_carry_off + j];
+      if (b0 + CHUNK == c.n_blocks) a.carry_base[c.carry_off + j + 1] = a.carry_base[c.old_carry_off + j + 1];   // nothing new: the resume point
+    }
+  } else {
+    carry = chunk_carry<T>(a, c, j);
+    if (tid == 0) {
+      a.carry_base[c.carry_off + j] = carry;
+      if (b0 + nb == c.n_blocks)   // value after the last chunk: the resume point of a later call if that chunk is full
+        a.carry_base[c.carry_off + j + 1] = g_pow_p.v[nb] * carry + a.agg[c.dchunk_base + (j - c.first / CHUNK)];
+    }
+  }
 #pragma unroll
   for (int q = 0; q < ILP; ++q) {
-    const u32 j = tid + q * T;
-    act[q] = j < nb;
+    const u32 jj = tid + q * T;
+    act[q] = jj < nb;
     key[q] = 0;
     if (act[q]) {
-      if (kept) key[q] = a.keys[c.old_key_off + b0 + j];
+      if (kept) key[q] = a.keys[c.old_key_off + b0 + jj];
       else {
-        key[q] = mix64(g_pow_p.v[j + 1] * carry + a.keys[c.key_off + b0 + j]);
+        key[q] = mix64(g_pow_p.v[jj + 1] * carry + a.keys[c.key_off + b0 + jj]);
         if (key[q] < 2) key[q] += 2;
       }
-      a.keys[c.key_off + b0 + j] = key[q];
+      a.keys[c.key_off + b0 + jj] = key[q];
     }
   }
   if (!l.tab.slots) return;
@@ -403,9 +388,9 @@ __global__ void __launch_bounds__(CHUNK / ILP) k_hash_finish_lookup(HashArgs a, 
 #pragma unroll
   for (int q = 0; q < ILP; ++q)
     if (act[q]) {
-      const u32 j = tid + q * T;
-      l.b_ent[c.blk_base + b0 + j] = ent[q];
-      if (ent[q] == ENT_NONE) miss = min(miss, b0 + j);
+      const u32 jj = tid + q * T;
+      l.b_ent[c.blk_base + b0 + jj] = ent[q];
+      if (ent[q] == ENT_NONE) miss = min(miss, b0 + jj);
     }
   // first miss of the CTA -> the context's reusable prefix length: warp minima meet in shared memory, one global
   // atomic per CTA that saw a miss

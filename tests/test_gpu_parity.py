@@ -420,7 +420,7 @@ def _c4_setup(B, oracle, n_resident, chain_blocks, n_calls):
     return inp, gpu, cpu
 
 
-@pytest.mark.parametrize("lookup_variant", [1, 2, 3, 4], ids=["three-kernels", "single-pass", "two-keys-per-thread", "four-keys-per-thread"])
+@pytest.mark.parametrize("lookup_variant", [1, 2, 3, 4], ids=["default", "single-pass", "one-key-per-thread", "four-keys-per-thread"])
 @pytest.mark.parametrize("n_resident,chain_blocks,n_calls", [(5000, 700, 9), (1 << 20, 16128, 64)])
 def test_c4_lookup_and_select_parity(B, oracle, n_resident, chain_blocks, n_calls, lookup_variant):
     inp, gpu, cpu = _c4_setup(B, oracle, n_resident, chain_blocks, n_calls)
@@ -819,7 +819,7 @@ def test_capacity_errors_leave_the_engine_usable(B):
         eng.select_victims(3, 1)                                 # bad tier
 
 
-@pytest.mark.parametrize("lookup_variant", [1, 2, 4], ids=["three-kernels", "single-pass", "four-keys-per-thread"])
+@pytest.mark.parametrize("lookup_variant", [1, 2, 4], ids=["default", "single-pass", "four-keys-per-thread"])
 def test_incremental_hashing_resumes_at_chunk_boundaries(B, oracle, lookup_variant):
     """Appends, edits, forks and repeated calls around multiples of 256 blocks: only the changed tail is digested
     again, and every key still equals the one-shot hash of the whole sequence."""
@@ -863,7 +863,7 @@ def test_incremental_hashing_resumes_at_chunk_boundaries(B, oracle, lookup_varia
     assert st["blocks_rehashed"] < st["blocks_hashed"]
 
 
-@pytest.mark.parametrize("lookup_variant", [1, 2], ids=["three-kernels", "single-pass"])
+@pytest.mark.parametrize("lookup_variant", [1, 2], ids=["default", "single-pass"])
 def test_adjacent_key_lists_do_not_overlap(B, oracle, lookup_variant):
     """Key lists of one batch sit back to back in the key arena, each followed by its per-chunk carries and the
     resume point: sizes whose rounded lists leave no slack (e.g. 7,937..7,968 blocks) must not spill into the
