@@ -428,6 +428,13 @@ int32_t kvt_set_mover_ctas(kvt_engine *e, uint32_t max_ctas);
  * default. */
 int32_t kvt_debug_set_lookup_variant(kvt_engine *e, uint32_t variant);
 
+/* L2 residency of the metadata (default on where the device supports it): the kernels that probe the block table and
+ * the per-entry arrays are launched with an access-policy window over them, so those lines sit in the persisting part
+ * of L2 (up to the device's maximum, 79 MiB on B200; the process-wide limit cudaLimitPersistingL2CacheSize is raised to
+ * what the engine needs, never lowered) while KV payload and token streams, which are read and written with
+ * streaming accesses, pass through the rest. 0 switches it off and gives the persisting lines back. */
+int32_t kvt_set_l2_residency(kvt_engine *e, uint32_t on);
+
 /* Test / measurement hook for the classification: 0 = event-driven (default), 1 = every kvt_classify recomputes all
  * counts from zero over all contexts, 2 = event-driven, and every update is followed by a full recomputation that must
  * give the same counts (KVT_E_DEVICE if not). */

@@ -201,6 +201,12 @@ struct kvt_engine {
     return (u32)std::max<u64>(1, std::min(want, cap));
   }
   u32 link_dirs(u32 st, u32 dt) const { return (tier_in_host_mem[st] || tier_in_host_mem[dt]) ? 1u : 0u; }
+  // L2 residency of the block table and the hot per-entry arrays (key, stamp, depth, in-flight, counts): the kernels
+  // that probe them are launched with an access-policy window over that range, so the lines they touch stay in the
+  // persisting part of L2 while KV payload and token streams pass through the rest
+  cudaAccessPolicyWindow l2_win{};
+  bool l2_on = false;
+  bool overlap_launches = !CHECKED_BUILD;   // dependent launches inside one call (digest -> finish -> lock)
   u32 lookup_variant = 0;  // 0 / 1 digest / carry / finish kernels, 2 single-pass hash + probe kernel
   u32 wait_limit = 1u << 18;   // polls a chunk of the single-pass kernel spends on its predecessors before it gives up
   bool tma_attr_set = false;
@@ -229,6 +235,33 @@ namespace {
     kern<<<(grid), (block), 0, (stream)>>>(__VA_ARGS__);       \
     e->st.kernel_launches++;                                   \
   } while (0)
+
+// Launch of a kernel that works on the block table / per-entry metadata: carries the L2 access-policy window.
+// after_kernel: the launch directly follows, in the same stream, a kernel that releases its dependents early; this
+// kernel's CTAs may then take the SM slots the tail of that kernel leaves free and wait (dep_wait() in the kernel)
+// for its results there, instead of starting after the last CTA has drained.
+template <typename... Exp, typename... Act>
+void launch_meta(kvt_engine *e, bool after_kernel, void (*kern)(Exp...), u32 grid, u32 block, cudaStream_t s, Act &&...args) {
+  cudaLaunchConfig_t cfg{};
+  cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.stream = s;
+  cudaLaunchAttribute at[2];
+  u32 n = 0;
+  if (e->l2_on) {
+    at[n].id = cudaLaunchAttributeAccessPolicyWindow;
+    at[n].val.accessPolicyWindow = e->l2_win;
+    ++n;
+  }
+  if (after_kernel && e->overlap_launches) {
+    at[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[n].val.programmaticStreamSerializationAllowed = 1;
+    ++n;
+  }
+  cfg.attrs = at; cfg.numAttrs = n;
+  cudaLaunchKernelEx(&cfg, kern, std::forward<Act>(args)...);
+  e->st.kernel_launches++;
+}
+#define KLM(kern, grid, block, stream, ...) launch_meta(e, false, kern, (grid), (block), (stream), __VA_ARGS__)
+#define KLD(kern, grid, block, stream, ...) launch_meta(e, true, kern, (grid), (block), (stream), __VA_ARGS__)
 
 int32_t fail(kvt_engine *e, int32_t code, const char *msg) { e->err = msg; return code; }
 
@@ -709,11 +742,11 @@ int32_t apply_deltas(kvt_engine *e, cudaStream_t s, const std::vector<Ctx *> &li
       a.first_miss = e->dp<u32>(e->L.freelist2);   // scratch of the list calls, free between calls (stream order)
       if (nd > e->L.LB) return fail(e, KVT_E_NOSPACE, "more contexts than max_batch_blocks");
       CU(cudaMemsetAsync(a.first_miss, 0xFF, nd * 4ull, s));
-      KL(k_first_miss, cdiv(nmap, TPB), TPB, s, a);
+      KLM(k_first_miss, cdiv(nmap, TPB), TPB, s, a);
     }
     const bool timed = e->profiling && !e->classify_timed;
     if (timed) CU(cudaEventRecord(e->ev_c0, s));
-    KL(k_map_delta, cdiv(nmap, TPB), TPB, s, a);
+    KLM(k_map_delta, cdiv(nmap, TPB), TPB, s, a);
     if (timed) { CU(cudaEventRecord(e->ev_c1, s)); e->classify_timed = true; e->classify_pending_items = nmap; }
     LAUNCH_CHECK();
   }
@@ -773,7 +806,7 @@ int32_t do_classify(kvt_engine *e, cudaStream_t s, bool force_full = false) {
         FixArgs a;
         a.tab = e->tab; a.ent = e->ent; a.keys = e->d_keys; a.snaps = ds; a.n_snaps = ns; a.tbl = msg_tables(e);
         a.fresh = e->dp<u32>(e->L.fresh); a.n_fresh = e->n_fresh; a.status = e->d_status;
-        KL(k_fresh_fixup, cdiv(e->n_fresh, 128), 128, s, a);
+        KLM(k_fresh_fixup, cdiv(e->n_fresh, 128), 128, s, a);
       }
     }
     // (2) contexts that changed, and contexts that ended
@@ -840,8 +873,8 @@ u64 grow_cap(u64 need) { return round_up(std::max<u64>(need + need / 4, 1024), 6
 
 int32_t unlock_held(kvt_engine *e, Ctx &c, cudaStream_t s, bool stamp) {
   if (c.held && c.keyseg >= 0) {
-    KL(k_unlock, cdiv(c.held, TPB), TPB, s, e->tab, e->ent, e->d_keys + e->segs[c.keyseg].off, c.held, e->now,
-                                                stamp ? 1u : 0u, e->d_status);
+    KLM(k_unlock, cdiv(c.held, TPB), TPB, s, e->tab, e->ent, (const u64 *)(e->d_keys + e->segs[c.keyseg].off), c.held, e->now,
+        stamp ? 1u : 0u, e->d_status);
     LAUNCH_CHECK();
   }
   c.held = 0;
@@ -964,6 +997,25 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   e->ent.n_hbm = c.n_hbm_blocks; e->ent.n_host = c.n_host_blocks; e->ent.n_total = (u32)N;
   e->d_keys = e->dp<u64>(L.keys); e->d_status = e->dp<u32>(L.status);
   e->h0 = hash_h0(c.hash_seed);
+  {   // L2 residency window: table, keys, stamps, depths, in-flight counts, mapping counts (contiguous in the arena)
+    int max_persist = 0, max_win = 0;
+    cudaDeviceGetAttribute(&max_persist, cudaDevAttrMaxPersistingL2CacheSize, dev);
+    cudaDeviceGetAttribute(&max_win, cudaDevAttrMaxAccessPolicyWindowSize, dev);
+    const u64 bytes = std::min<u64>(L.e_tslot - L.tab, (u64)std::max(max_win, 0));
+    const u64 want = std::min<u64>(bytes, (u64)std::max(max_persist, 0));
+    size_t cur = 0;
+    if (bytes && want && cudaDeviceGetLimit(&cur, cudaLimitPersistingL2CacheSize) == cudaSuccess &&
+        (cur >= want || cudaDeviceSetLimit(cudaLimitPersistingL2CacheSize, want) == cudaSuccess)) {
+      e->l2_win.base_ptr = e->meta + L.tab;
+      e->l2_win.num_bytes = bytes;
+      e->l2_win.hitRatio = (float)std::min(1.0, (double)want / (double)bytes);
+      e->l2_win.hitProp = cudaAccessPropertyPersisting;
+      e->l2_win.missProp = cudaAccessPropertyNormal;
+      e->l2_on = true;
+    } else {
+      cudaGetLastError();
+    }
+  }
   e->ctxs.resize(c.max_contexts);
   e->tok_alloc.init(c.max_tokens, 64);
   e->key_alloc.init(c.max_key_blocks + c.max_key_blocks / CHUNK + 64ull * c.max_contexts, 32);
@@ -1005,6 +1057,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
 int32_t kvt_destroy(kvt_engine *e) {
   if (!e) return KVT_E_INVAL;
   cudaDeviceSynchronize();
+  if (e->l2_win.num_bytes) cudaCtxResetPersistingL2Cache();   // the lines this engine kept resident are ordinary lines again
   for (auto &m : e->sel_graph) for (auto &g : m) if (g.second.exec) cudaGraphExecDestroy(g.second.exec);
   if (e->capture_stream) cudaStreamDestroy(e->capture_stream);
   for (int d = 0; d < 2; ++d) {
@@ -1055,6 +1108,14 @@ int32_t kvt_set_mover_ctas(kvt_engine *e, uint32_t max_ctas) {
 int32_t kvt_debug_set_lookup_variant(kvt_engine *e, uint32_t variant) {
   if (!e || variant > 4) return KVT_E_INVAL;
   e->lookup_variant = variant;
+  return KVT_OK;
+}
+
+int32_t kvt_set_l2_residency(kvt_engine *e, uint32_t on) {
+  if (!e) return KVT_E_INVAL;
+  if (on && !e->l2_win.num_bytes) return fail(e, KVT_E_INVAL, "this device offers no persisting L2");
+  e->l2_on = on != 0;
+  if (!on) cudaCtxResetPersistingL2Cache();
   return KVT_OK;
 }
 
@@ -1373,12 +1434,13 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     lk.now = e->now; lk.status = e->d_status;
     if (e->profiling) CUR(cudaEventRecord(e->ev_h0, s));
     if (e->lookup_variant != 2) {
-      if (dchunk_base) KL(k_hash_digest, dchunk_base, CHUNK, s, ha);
+      const bool dg = dchunk_base != 0;
+      if (dg) KL(k_hash_digest, dchunk_base, CHUNK, s, ha);
       // two keys per thread by default; one or four measured within 3 % of it: the probes of a cold table are bound
       // by the number of outstanding misses the memory system carries, not by what a thread issues
-      if (e->lookup_variant == 3) KL(k_hash_finish_lookup<1>, chunk_base, CHUNK, s, ha, la);
-      else if (e->lookup_variant == 4) KL(k_hash_finish_lookup<4>, chunk_base, CHUNK / 4, s, ha, la);
-      else KL(k_hash_finish_lookup<2>, chunk_base, CHUNK / 2, s, ha, la);
+      if (e->lookup_variant == 3) launch_meta(e, dg, k_hash_finish_lookup<1>, chunk_base, CHUNK, s, ha, la);
+      else if (e->lookup_variant == 4) launch_meta(e, dg, k_hash_finish_lookup<4>, chunk_base, CHUNK / 4, s, ha, la);
+      else launch_meta(e, dg, k_hash_finish_lookup<2>, chunk_base, CHUNK / 2, s, ha, la);
     } else {
       ChainState cs;
       cs.flags = e->dp<u32>(e->L.cflags); cs.ticket = cs.flags + chunk_base; cs.incl = e->dp<u64>(e->L.carry);
@@ -1386,7 +1448,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
       CUR(cudaMemsetAsync(cs.flags, 0, (chunk_base + 1) * 4ull, s));
       KL(k_hash_lookup_fused, chunk_base, CHUNK, s, ha, la, cs);
     }
-    KL(k_lock_hits, chunk_base, CHUNK, s, ha, lk);
+    KLD(k_lock_hits<4>, chunk_base, CHUNK / 4, s, ha, lk);
     if (e->profiling) CUR(cudaEventRecord(e->ev_h1, s));
     r = launch_ok(e);
     if (r) return rollback(r);
@@ -1479,14 +1541,14 @@ static int32_t map_admit(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_info
     rc = status_zero(e, s);
     if (rc) break;
     u32 g = cdiv(n_cand, TPB);
-    KL(k_admit_claim, g, TPB, s, a);
-    KL(k_admit_resolve, g, TPB, s, a);
+    KLM(k_admit_claim, g, TPB, s, a);
+    KLM(k_admit_resolve, g, TPB, s, a);
     rc = compact_indices(e, s, PredOwner{a.flag}, EmitRank{a.krank}, n_cand, ST_NEW);
     if (rc) break;
     rc = compact_indices(e, s, PredFree{e->ent.key, 0}, EmitFree{e->dp<u32>(e->L.freelist), (u32)e->L.LB}, e->cfg.n_hbm_blocks, ST_FREE);
     if (rc) break;
     KL(k_admit_stop, g, TPB, s, a);
-    KL(k_admit_apply, g, TPB, s, a);
+    KLM(k_admit_apply, g, TPB, s, a);
     rc = launch_ok(e);
     if (rc) break;
     CU(cudaMemcpyAsync(h_stop, a.stop, nd * 4, cudaMemcpyDeviceToHost, s));

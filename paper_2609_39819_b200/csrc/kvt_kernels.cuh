@@ -234,9 +234,17 @@ __device__ __forceinline__ void digest_quads(const uint4 (&v)[4], u32 q, u64 k0,
   }
 }
 
+// Dependent launches inside one call: a kernel releases the next launch of its stream at its start (the next
+// kernel's CTAs then fill the SM slots this kernel's tail leaves free), and the next kernel waits, before it touches
+// anything this one writes, until this grid has finished and its writes are visible. Both are no-ops for a launch
+// without the attribute.
+__device__ __forceinline__ void dep_release() { asm volatile("griddepcontrol.launch_dependents;"); }
+__device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   __shared__ u64 sd[CHUNK];
   __shared__ u64 wagg[CHUNK / 32];
+  dep_release();
   const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   u32 ci;
   const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci, true);
@@ -354,6 +362,8 @@ __global__ void __launch_bounds__(CHUNK / ILP) k_hash_finish_lookup(HashArgs a, 
   bool act[ILP];
   const bool kept = b0 < c.first;                                   // unchanged prefix: the keys of the previous list still hold
   u64 carry = 0;
+  dep_release();
+  dep_wait();   // the digest kernel's keys and aggregates
   if (kept) {
     if (tid == 0) {
       a.carry_base[c.carry_off + j] = a.carry_base[c.old_carry_off + j];
@@ -554,36 +564,45 @@ __global__ void __launch_bounds__(CHUNK) k_hash_lookup_fused(HashArgs a, LookupA
 // Stamps and locks the reusable prefix of every context of the batch; counts hits per tier.
 struct LockArgs { Entries ent; const u32 *b_ent; const u32 *hit_len; u32 *n_hbm; u32 *n_host; u32 *n_remote; u32 now; u32 *status; };
 
-__global__ void __launch_bounds__(CHUNK) k_lock_hits(HashArgs a, LockArgs l) {
+// One CTA of CHUNK / ILP threads per 256-block chunk (the whole grid is resident at once at C4 scale with ILP = 4).
+template <int ILP>
+__global__ void __launch_bounds__(CHUNK / ILP) k_lock_hits(HashArgs a, LockArgs l) {
+  constexpr u32 T = CHUNK / ILP;
   const u32 tid = threadIdx.x;
   u32 ci;
   const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci);
-  const u32 b = (blockIdx.x - c.chunk_base) * CHUNK + tid;
-  u32 tier = 3;   // none
   // the hash / probe kernels failed: the call changes nothing. One read per CTA, so that the whole CTA agrees.
   __shared__ u32 s_err;
-  if (tid == 0) s_err = l.status[ST_ERR];
-  __syncthreads();
-  if (s_err) return;
-  if (b < l.hit_len[ci]) {
-    u32 e = l.b_ent[c.blk_base + b];
-    if (e >= l.ent.n_total) set_err(l.status, DERR_CORRUPT);
-    else {
-      l.ent.stamp[e] = l.now;
-      atomicAdd(&l.ent.infl[e], 1u);
-      tier = e < l.ent.n_hbm ? 0u : e < l.ent.n_hbm + l.ent.n_host ? 1u : 2u;
-    }
-  }
-  // per-tier hit counts: one ballot per tier and warp, summed in shared memory, one global atomic per CTA and tier
   __shared__ u32 s_cnt[3];
+  dep_wait();   // the probe kernel's entry ids, prefix lengths and error word
+  if (tid == 0) s_err = l.status[ST_ERR];
   if (tid < 3) s_cnt[tid] = 0;
   __syncthreads();
-  const u32 m0 = __ballot_sync(0xFFFFFFFFu, tier == 0), m1 = __ballot_sync(0xFFFFFFFFu, tier == 1),
-            m2 = __ballot_sync(0xFFFFFFFFu, tier == 2);
+  if (s_err) return;
+  const u32 hit_len = l.hit_len[ci];
+  const u32 b0 = (blockIdx.x - c.chunk_base) * CHUNK;
+  u32 e[ILP];
+#pragma unroll
+  for (int q = 0; q < ILP; ++q) {
+    const u32 b = b0 + tid + q * T;
+    e[q] = b < hit_len ? l.b_ent[c.blk_base + b] : ENT_NONE;
+  }
+  u32 n0 = 0, n1 = 0, n2 = 0;
+#pragma unroll
+  for (int q = 0; q < ILP; ++q) {
+    const u32 b = b0 + tid + q * T;
+    if (b >= hit_len) continue;
+    if (e[q] >= l.ent.n_total) { set_err(l.status, DERR_CORRUPT); continue; }
+    l.ent.stamp[e[q]] = l.now;
+    atomicAdd(&l.ent.infl[e[q]], 1u);
+    if (e[q] < l.ent.n_hbm) ++n0; else if (e[q] < l.ent.n_hbm + l.ent.n_host) ++n1; else ++n2;
+  }
+  // per-tier hit counts: warp sums meet in shared memory, one global atomic per CTA and tier
+  n0 = __reduce_add_sync(0xFFFFFFFFu, n0); n1 = __reduce_add_sync(0xFFFFFFFFu, n1); n2 = __reduce_add_sync(0xFFFFFFFFu, n2);
   if ((tid & 31) == 0) {
-    if (m0) atomicAdd(&s_cnt[0], (u32)__popc(m0));
-    if (m1) atomicAdd(&s_cnt[1], (u32)__popc(m1));
-    if (m2) atomicAdd(&s_cnt[2], (u32)__popc(m2));
+    if (n0) atomicAdd(&s_cnt[0], n0);
+    if (n1) atomicAdd(&s_cnt[1], n1);
+    if (n2) atomicAdd(&s_cnt[2], n2);
   }
   __syncthreads();
   if (tid == 0 && s_cnt[0]) atomicAdd(&l.n_hbm[ci], s_cnt[0]);
