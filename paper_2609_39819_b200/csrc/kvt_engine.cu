@@ -236,17 +236,26 @@ namespace {
     e->st.kernel_launches++;                                   \
   } while (0)
 
+template <typename... Exp, typename... Act>
+void launch_attr(kvt_engine *e, bool window, bool after_kernel, void (*kern)(Exp...), u32 grid, u32 block, cudaStream_t s,
+                 Act &&...args);
 // Launch of a kernel that works on the block table / per-entry metadata: carries the L2 access-policy window.
 // after_kernel: the launch directly follows, in the same stream, a kernel that releases its dependents early; this
 // kernel's CTAs may then take the SM slots the tail of that kernel leaves free and wait (dep_wait() in the kernel)
 // for its results there, instead of starting after the last CTA has drained.
 template <typename... Exp, typename... Act>
 void launch_meta(kvt_engine *e, bool after_kernel, void (*kern)(Exp...), u32 grid, u32 block, cudaStream_t s, Act &&...args) {
+  launch_attr(e, true, after_kernel, kern, grid, block, s, std::forward<Act>(args)...);
+  e->st.kernel_launches++;
+}
+template <typename... Exp, typename... Act>
+void launch_attr(kvt_engine *e, bool window, bool after_kernel, void (*kern)(Exp...), u32 grid, u32 block, cudaStream_t s,
+                 Act &&...args) {
   cudaLaunchConfig_t cfg{};
   cfg.gridDim = dim3(grid); cfg.blockDim = dim3(block); cfg.stream = s;
   cudaLaunchAttribute at[2];
   u32 n = 0;
-  if (e->l2_on) {
+  if (window && e->l2_on) {
     at[n].id = cudaLaunchAttributeAccessPolicyWindow;
     at[n].val.accessPolicyWindow = e->l2_win;
     ++n;
@@ -258,7 +267,6 @@ void launch_meta(kvt_engine *e, bool after_kernel, void (*kern)(Exp...), u32 gri
   }
   cfg.attrs = at; cfg.numAttrs = n;
   cudaLaunchKernelEx(&cfg, kern, std::forward<Act>(args)...);
-  e->st.kernel_launches++;
 }
 #define KLM(kern, grid, block, stream, ...) launch_meta(e, false, kern, (grid), (block), (stream), __VA_ARGS__)
 #define KLD(kern, grid, block, stream, ...) launch_meta(e, true, kern, (grid), (block), (stream), __VA_ARGS__)
@@ -1733,7 +1741,9 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
     if (count) TRACE(q, "start");
     cudaMemsetAsync(a.hist, 0, (u64)n_levels * SEL_BINS * 4, q);
     if (count) TRACE(q, "memset");
-    k_sel_keys<<<g, SEL_CTA, 0, q>>>(d_args);
+    // (dependent launches were tried for this chain and lose: with kernels of 3-10 us the programmatic completion
+    // costs more than the tail overlap saves, 85 -> 135 us; the key kernel alone carries the L2 window)
+    launch_attr(e, true, false, k_sel_keys, g, SEL_CTA, q, d_args);
     if (count) TRACE(q, "keys");
     for (u32 lev = 1; lev < n_levels; ++lev) { k_sel_level<<<g, SEL_CTA, 0, q>>>(d_args, lev); if (count) TRACE(q, "level"); }
     k_sel_count<<<g, SEL_CTA, 0, q>>>(d_args);

@@ -62,6 +62,19 @@ struct PowTable {
   constexpr PowTable() : v() { u64 p = 1; for (u32 i = 0; i <= CHUNK; ++i) { v[i] = p; p *= HASH_P; } }
 };
 __device__ const PowTable g_pow_p = PowTable();
+// A^0 .. A^64 with A = P^CHUNK: the weights of the chunk aggregates of sequences of up to 64 chunks (16 Ki blocks);
+// longer ones fall back to square-and-multiply.
+struct ChunkPowTable {
+  u64 v[65];
+  constexpr ChunkPowTable() : v() {
+    u64 a = 1;
+    for (u32 i = 0; i < CHUNK; ++i) a *= HASH_P;
+    u64 p = 1;
+    for (u32 i = 0; i <= 64; ++i) { v[i] = p; p *= a; }
+  }
+};
+__device__ const ChunkPowTable g_pow_a = ChunkPowTable();
+__device__ __forceinline__ u64 pow_a(u32 e) { return e <= 64 ? g_pow_a.v[e] : pow_u64(g_pow_p.v[CHUNK], e); }
 
 // ---- device views -------------------------------------------------------------------------------------
 struct Table { TSlot *slots; u32 mask; u32 shift; };   // capacity = mask + 1, home = key >> shift
@@ -234,12 +247,64 @@ __device__ __forceinline__ void digest_quads(const uint4 (&v)[4], u32 q, u64 k0,
   }
 }
 
+// ---- untiled bulk copies (cp.async.bulk) and the mbarriers they complete on; every wait is bounded -----------
+constexpr u32 TMA_WAIT_LIMIT = 1u << 20;
+
+__device__ __forceinline__ u32 smem_u32(const void *p) { return (u32)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(u64 *bar, u32 count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(u64 *bar, u32 bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+// Polls the barrier's phase; gives up after TMA_WAIT_LIMIT polls (returns false).
+__device__ __forceinline__ bool mbar_wait(u64 *bar, u32 parity) {
+  u32 done = 0;
+  for (u32 n = 0; n < TMA_WAIT_LIMIT && !done; ++n) {
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+  }
+  return done != 0;
+}
+__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, u32 bytes, u64 *bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+               ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void bulk_store(void *gdst, const void *smem_src, u32 bytes) {
+  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(smem_src)), "r"(bytes) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+
 // Dependent launches inside one call: a kernel releases the next launch of its stream at its start (the next
 // kernel's CTAs then fill the SM slots this kernel's tail leaves free), and the next kernel waits, before it touches
 // anything this one writes, until this grid has finished and its writes are visible. Both are no-ops for a launch
 // without the attribute.
 __device__ __forceinline__ void dep_release() { asm volatile("griddepcontrol.launch_dependents;"); }
 __device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
+// Chain values of a chunk with zero carry-in from its block digests sd[] (an inclusive scan of
+// c_t = sum_{i<=t} P^(t-i) d_i over the CTA), stored where the keys will be; the last one is the chunk's aggregate.
+__device__ __forceinline__ void chunk_scan_store(const HashArgs &a, const HashCtx &c, u32 b0, u32 nb, u32 dchunk, const u64 *sd,
+                                                 u64 *wagg) {
+  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  u64 cval = sd[tid];
+  u64 pp = HASH_P;
+#pragma unroll
+  for (u32 o = 1; o < 32; o <<= 1) {
+    u64 up = __shfl_up_sync(0xFFFFFFFFu, cval, o);
+    if (lane >= o) cval += pp * up;
+    pp *= pp;
+  }
+  if (lane == 31) wagg[warp] = cval;
+  __syncthreads();
+  u64 carry = 0;  // chain value at the end of the previous warp, with zero chunk carry-in
+  const u64 p32 = pp;  // after 5 squarings pp = P^32
+  for (u32 w = 0; w < warp; ++w) carry = p32 * carry + wagg[w];
+  cval += g_pow_p.v[lane + 1] * carry;
+  if (tid < nb) a.keys[c.key_off + b0 + tid] = cval;
+  if (tid == nb - 1) a.agg[dchunk] = cval;
+}
 
 __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   __shared__ u64 sd[CHUNK];
@@ -265,23 +330,7 @@ __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   // lane of a quad holds the four block sums, and lane q finishes the block of iteration q
   digest_quads(v, q, k0, k1, k2, k3, ksum, tid, nb, sd);
   __syncthreads();
-  // inclusive scan of c_t = sum_{i<=t} P^(t-i) d_i
-  u64 cval = sd[tid];
-  u64 pp = HASH_P;
-#pragma unroll
-  for (u32 o = 1; o < 32; o <<= 1) {
-    u64 up = __shfl_up_sync(0xFFFFFFFFu, cval, o);
-    if (lane >= o) cval += pp * up;
-    pp *= pp;
-  }
-  if (lane == 31) wagg[warp] = cval;
-  __syncthreads();
-  u64 carry = 0;  // chain value at the end of the previous warp, with zero chunk carry-in
-  const u64 p32 = pp;  // after 5 squarings pp = P^32
-  for (u32 w = 0; w < warp; ++w) carry = p32 * carry + wagg[w];
-  cval += g_pow_p.v[lane + 1] * carry;
-  if (tid < nb) a.keys[c.key_off + b0 + tid] = cval;
-  if (tid == nb - 1) a.agg[blockIdx.x] = cval;
+  chunk_scan_store(a, c, b0, nb, blockIdx.x, sd, wagg);
 }
 
 struct LookupArgs {
@@ -332,10 +381,9 @@ template <u32 T>
 __device__ __forceinline__ u64 chunk_carry(const HashArgs &a, const HashCtx &c, u32 j) {
   __shared__ u64 s_part[T / 32];
   const u32 g0 = c.first / CHUNK, m = j - g0, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const u64 A = g_pow_p.v[CHUNK];
   u64 sum = 0;
-  for (u32 i = tid; i < m; i += T) sum += pow_u64(A, m - 1 - i) * a.agg[c.dchunk_base + i];
-  if (tid == 0) sum += pow_u64(A, m) * (g0 ? a.carry_base[c.old_carry_off + g0] : a.h0);
+  for (u32 i = tid; i < m; i += T) sum += pow_a(m - 1 - i) * a.agg[c.dchunk_base + i];
+  if (tid == 0) sum += pow_a(m) * (g0 ? a.carry_base[c.old_carry_off + g0] : a.h0);
 #pragma unroll
   for (u32 o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xFFFFFFFFu, sum, o);
   if (lane == 0) s_part[warp] = sum;
@@ -364,6 +412,12 @@ __global__ void __launch_bounds__(CHUNK / ILP) k_hash_finish_lookup(HashArgs a, 
   u64 carry = 0;
   dep_release();
   dep_wait();   // the digest kernel's keys and aggregates
+  u64 loc[ILP];   // chain values with zero carry-in (or, in the unchanged prefix, the old keys): fetched before the carry is known
+#pragma unroll
+  for (int q = 0; q < ILP; ++q) {
+    const u32 jj = tid + q * T;
+    loc[q] = jj < nb ? a.keys[(kept ? c.old_key_off : c.key_off) + b0 + jj] : 0;
+  }
   if (kept) {
     if (tid == 0) {
       a.carry_base[c.carry_off + j] = a.carry_base[c.old_carry_off + j];
@@ -383,9 +437,9 @@ __global__ void __launch_bounds__(CHUNK / ILP) k_hash_finish_lookup(HashArgs a, 
     act[q] = jj < nb;
     key[q] = 0;
     if (act[q]) {
-      if (kept) key[q] = a.keys[c.old_key_off + b0 + jj];
+      if (kept) key[q] = loc[q];
       else {
-        key[q] = mix64(g_pow_p.v[jj + 1] * carry + a.keys[c.key_off + b0 + jj]);
+        key[q] = mix64(g_pow_p.v[jj + 1] * carry + loc[q]);
         if (key[q] < 2) key[q] += 2;
       }
       a.keys[c.key_off + b0 + jj] = key[q];
@@ -1715,33 +1769,6 @@ __global__ void __launch_bounds__(THREADS) k_move_exchange(MoveArgs a, MoveArgs 
 // carry payload; every wait is bounded and reports through the status word. Every copy is CTA-local: one source, one destination, no clusters.
 // ------------------------------------------------------------------------------------------------------
 constexpr int TMA_STAGES = 4;
-constexpr u32 TMA_WAIT_LIMIT = 1u << 20;
-
-__device__ __forceinline__ u32 smem_u32(const void *p) { return (u32)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(u64 *bar, u32 count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(u64 *bar, u32 bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-// Polls the barrier's phase; gives up after TMA_WAIT_LIMIT polls (returns false).
-__device__ __forceinline__ bool mbar_wait(u64 *bar, u32 parity) {
-  u32 done = 0;
-  for (u32 n = 0; n < TMA_WAIT_LIMIT && !done; ++n) {
-    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
-                 : "=r"(done) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-  }
-  return done != 0;
-}
-__device__ __forceinline__ void bulk_load(void *smem_dst, const void *gsrc, u32 bytes, u64 *bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-               ::"r"(smem_u32(smem_dst)), "l"(gsrc), "r"(bytes), "r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void bulk_store(void *gdst, const void *smem_src, u32 bytes) {
-  asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" ::"l"(gdst), "r"(smem_u32(smem_src)), "r"(bytes) : "memory");
-  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
-}
 
 __global__ void __launch_bounds__(32) k_move_tma(MoveArgs a, u32 tile_bytes, u32 tiles_per_chunk) {
   extern __shared__ __align__(128) u8 smem[];
