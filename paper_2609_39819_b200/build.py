@@ -58,6 +58,19 @@ def build_lib(force: bool = False, verbose: bool = False, lib: str = LIB, define
     return lib
 
 
+TRACE_LIB = os.path.join(_HERE, "libkvt_trace.so")
+
+
+def build_trace_lib(force: bool = False) -> str:
+    """Development build with per-kernel event timing (-DKVT_TRACE): with KVT_TRACE=1 in the environment the LOOKUP
+    and selection calls print the time between their launches to stderr; KVT_NO_OVERLAP=1 launches the LOOKUP kernels
+    without the tail overlap, KVT_NO_GRAPH=1 the selection without its CUDA graph. Load it with KVT_LIB=<path>."""
+    return build_lib(force, lib=TRACE_LIB, defines=["-DKVT_TRACE"])
+
+
 if __name__ == "__main__":
     import sys
-    print(build_lib(force=True, verbose="-v" in sys.argv))
+    if "--trace" in sys.argv:
+        print(build_trace_lib(force=True))
+    else:
+        print(build_lib(force=True, verbose="-v" in sys.argv))

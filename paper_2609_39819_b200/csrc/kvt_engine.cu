@@ -1042,6 +1042,7 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   cudaStream_t s = (cudaStream_t)stream;
   if (cudaStreamCreateWithFlags(&e->capture_stream, cudaStreamNonBlocking) != cudaSuccess) { cudaGetLastError(); e->use_graphs = false; }
 #ifdef KVT_TRACE
+  if (getenv("KVT_NO_OVERLAP")) e->overlap_launches = false;
   if (getenv("KVT_NO_GRAPH")) e->use_graphs = false;
 #endif
   if (CHECKED_BUILD) e->use_graphs = false;
@@ -1443,7 +1444,9 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     if (e->profiling) CUR(cudaEventRecord(e->ev_h0, s));
     if (e->lookup_variant != 2) {
       const bool dg = dchunk_base != 0;
+      TRACE(s, "start");
       if (dg) KL(k_hash_digest, dchunk_base, CHUNK, s, ha);
+      TRACE(s, "digest");
       // two keys per thread by default; one or four measured within 3 % of it: the probes of a cold table are bound
       // by the number of outstanding misses the memory system carries, not by what a thread issues
       if (e->lookup_variant == 3) launch_meta(e, dg, k_hash_finish_lookup<1>, chunk_base, CHUNK, s, ha, la);
@@ -1456,7 +1459,9 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
       CUR(cudaMemsetAsync(cs.flags, 0, (chunk_base + 1) * 4ull, s));
       KL(k_hash_lookup_fused, chunk_base, CHUNK, s, ha, la, cs);
     }
+    TRACE(s, "finish");
     KLD(k_lock_hits<4>, chunk_base, CHUNK / 4, s, ha, lk);
+    TRACE(s, "lock");
     if (e->profiling) CUR(cudaEventRecord(e->ev_h1, s));
     r = launch_ok(e);
     if (r) return rollback(r);
@@ -1467,6 +1472,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
       float ms = 0.f;
       if (cudaEventElapsedTime(&ms, e->ev_h0, e->ev_h1) == cudaSuccess) { e->st.lookup_ns += (u64)((double)ms * 1e6); e->st.lookup_blocks += blk_base; }
     }
+    TRACE_DUMP("lookup");
     r = status_code(e);
     if (r) return rollback(r);
   }

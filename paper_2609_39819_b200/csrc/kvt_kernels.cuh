@@ -310,7 +310,7 @@ __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   __shared__ u64 sd[CHUNK];
   __shared__ u64 wagg[CHUNK / 32];
   dep_release();
-  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const u32 tid = threadIdx.x;
   u32 ci;
   const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci, true);
   const u32 b0 = c.first + (blockIdx.x - c.dchunk_base) * CHUNK;
