@@ -114,7 +114,11 @@ DevLayout make_layout(const kvt_config &c) {
   L.cnt_chk = take(N * 8);   // the counts of a full recomputation, for the cross-check mode
   L.fresh = take(N * 4);     // entries inserted since the counts were last brought up to date
   L.keys = take((c.max_key_blocks + c.max_key_blocks / CHUNK + 64ull * c.max_contexts) * 8);   // keys + per-chunk carries
+  // status words, per-context results and call descriptors sit in one stretch, on the device and in the pinned
+  // staging area alike, so that a LOOKUP call uploads all three with one copy and reads two of them back with one
   L.status = take(ST_WORDS * 4);
+  L.ctxres = take(C * 20);   // per context: hit_len, hits per tier (3), admission stop
+  L.desc = take(C * 256 + 2 * (B / CHUNK + C + 1) * 4);  // per-context descriptors, then the chunk -> context maps of a LOOKUP batch
   L.s0 = take(LB * 4); L.s1 = take(LB * 4); L.s2 = take(LB * 4); L.s3 = take(LB * 4);
   L.ids = take(LB * 4); L.ids2 = take(LB * 4); L.pair_src = take(LB * 4); L.pair_dst = take(LB * 4);
   L.freelist = take(LB * 4); L.freelist2 = take(LB * 4); L.pair_src2 = take(LB * 4); L.pair_dst2 = take(LB * 4);
@@ -122,8 +126,6 @@ DevLayout make_layout(const kvt_config &c) {
   u64 n_chunks = B / CHUNK + C + 1;
   L.agg = take(n_chunks * 8); L.carry = take(n_chunks * 8);   // per-chunk aggregates / chain values of a LOOKUP batch
   L.cflags = take((n_chunks + 1) * 4);                         // per-chunk publication flags + the ticket word
-  L.desc = take(C * 256 + 2 * n_chunks * 4);  // per-context descriptors, then the chunk -> context maps of a LOOKUP batch
-  L.ctxres = take(C * 20);   // per context: hit_len, hits per tier (3), admission stop
   L.m_start = take(2 * Mm * 4); L.m_end = take(2 * Mm * 4); L.m_rank = take(2 * Mm);   // accounted-for tables + the new ones of a pass
   L.keyA = take(Nt * 8); L.keyB = take(Nt * 8); L.valA = take(Nt * 4); L.valB = take(Nt * 4);
   L.rcounts = take(((u64)RADIX_BINS * (Nt / SORT_TILE + 1) + RADIX_BINS) * 4);
@@ -1030,7 +1032,8 @@ int32_t kvt_create(const kvt_config *cfg, void *stream, kvt_engine **out) {
   e->tbl_alloc.init(2ull * c.max_messages, 1);
   // pinned staging
   u64 C = c.max_contexts, Mm = c.max_messages, LB = L.LB;
-  u64 o_status = 0, o_desc = 256, o_ctxres = o_desc + round_up(C * 256 + 2 * (c.max_batch_blocks / CHUNK + C + 1) * 4, 256), o_ms = o_ctxres + round_up(C * 20, 256),
+  u64 o_status = 0, o_ctxres = L.ctxres - L.status, o_desc = L.desc - L.status,
+      o_ms = o_desc + round_up(C * 256 + 2 * (c.max_batch_blocks / CHUNK + C + 1) * 4, 256),
       o_me = o_ms + round_up(Mm * 4, 256), o_mr = o_me + round_up(Mm * 4, 256), o_ids = o_mr + round_up(Mm, 256),
       o_ids2 = o_ids + round_up(LB * 4, 256), o_out = o_ids2 + round_up(LB * 4, 256),
       o_sel = o_out + round_up(LB * 16, 256), total = o_sel + round_up(sizeof(SelArgs), 256);
@@ -1427,11 +1430,14 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
         for (u32 j = 0; j < n_seq_chunks[q].second; ++j) h_dmap[dk++] = q;
       }
     }
-    CUR(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nd * sizeof(HashCtx) + ((u64)chunk_base + dchunk_base) * 4, cudaMemcpyHostToDevice, s));
-    CUR(cudaMemcpyAsync(d_res, h_hit, nd * 4, cudaMemcpyHostToDevice, s));
-    CUR(cudaMemsetAsync(d_res + C, 0, 3ull * C * 4, s));
-    r = status_zero(e, s);
-    if (r) return rollback(r);
+    TRACE(s, "begin");
+    // one upload: zeroed status words, the per-context result words (prefix length = all blocks, no hits yet),
+    // descriptors and chunk maps
+    std::memset(e->h_status, 0, ST_WORDS * 4);
+    {
+      const u32 n16 = (u32)cdiv((e->L.desc - e->L.status) + nd * sizeof(HashCtx) + ((u64)chunk_base + dchunk_base) * 4, 16);
+      KL(k_copy_words, std::min<u32>(cdiv(n16, 256), 64u), 256, s, (const uint4 *)e->h_status, (uint4 *)e->d_status, n16);
+    }
     HashArgs ha;
     ha.tokens = e->d_tokens; ha.keys = e->d_keys; ha.carry_base = e->d_keys; ha.ctx = e->dp<HashCtx>(e->L.desc); ha.n_ctx = nd;
     ha.agg = e->dp<u64>(e->L.agg); ha.h0 = e->h0; ha.single = HashCtx{};
@@ -1444,14 +1450,14 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     if (e->profiling) CUR(cudaEventRecord(e->ev_h0, s));
     if (e->lookup_variant != 2) {
       const bool dg = dchunk_base != 0;
-      TRACE(s, "start");
-      if (dg) KL(k_hash_digest, dchunk_base, CHUNK, s, ha);
+      TRACE(s, "uploads");
+      if (dg) { launch_attr(e, false, true, k_hash_digest, dchunk_base, CHUNK, s, ha); e->st.kernel_launches++; }
       TRACE(s, "digest");
       // two keys per thread by default; one or four measured within 3 % of it: the probes of a cold table are bound
       // by the number of outstanding misses the memory system carries, not by what a thread issues
-      if (e->lookup_variant == 3) launch_meta(e, dg, k_hash_finish_lookup<1>, chunk_base, CHUNK, s, ha, la);
-      else if (e->lookup_variant == 4) launch_meta(e, dg, k_hash_finish_lookup<4>, chunk_base, CHUNK / 4, s, ha, la);
-      else launch_meta(e, dg, k_hash_finish_lookup<2>, chunk_base, CHUNK / 2, s, ha, la);
+      if (e->lookup_variant == 3) launch_meta(e, true, k_hash_finish_lookup<1>, chunk_base, CHUNK, s, ha, la);
+      else if (e->lookup_variant == 4) launch_meta(e, true, k_hash_finish_lookup<4>, chunk_base, CHUNK / 4, s, ha, la);
+      else launch_meta(e, true, k_hash_finish_lookup<2>, chunk_base, CHUNK / 2, s, ha, la);
     } else {
       ChainState cs;
       cs.flags = e->dp<u32>(e->L.cflags); cs.ticket = cs.flags + chunk_base; cs.incl = e->dp<u64>(e->L.carry);
@@ -1465,9 +1471,16 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     if (e->profiling) CUR(cudaEventRecord(e->ev_h1, s));
     r = launch_ok(e);
     if (r) return rollback(r);
-    CUR(cudaMemcpyAsync(h_hit, d_res, 4ull * C * 4, cudaMemcpyDeviceToHost, s));
-    r = status_fetch(e, s);
+    // one read-back: status words and result words, written into the staging area by a kernel
+    {
+      const u32 n16 = (u32)cdiv((e->L.ctxres - e->L.status) + 4ull * C * 4, 16);
+      launch_attr(e, false, true, k_copy_words, std::min<u32>(cdiv(n16, 256), 64u), 256, s, (const uint4 *)e->d_status, (uint4 *)e->h_status, n16);
+      e->st.kernel_launches++;
+    }
+    r = launch_ok(e);
     if (r) return rollback(r);
+    CUR(cudaStreamSynchronize(s));
+    TRACE(s, "results");
     if (e->profiling) {
       float ms = 0.f;
       if (cudaEventElapsedTime(&ms, e->ev_h0, e->ev_h1) == cudaSuccess) { e->st.lookup_ns += (u64)((double)ms * 1e6); e->st.lookup_blocks += blk_base; }

@@ -306,10 +306,21 @@ __device__ __forceinline__ void chunk_scan_store(const HashArgs &a, const HashCt
   if (tid == nb - 1) a.agg[dchunk] = cval;
 }
 
+// Small control records between the pinned staging area and device memory (either direction; both are in the
+// device's address space): the descriptors of a call going up, status and result words coming back. A kernel
+// reaches a few tens of KB over the host link in about a third of the time a copy-engine transfer of that size
+// takes to start and finish, and it can be a dependent launch on both sides.
+__global__ void __launch_bounds__(256) k_copy_words(const uint4 *src, uint4 *dst, u32 n16) {
+  dep_release();
+  dep_wait();
+  for (u32 i = blockIdx.x * 256 + threadIdx.x; i < n16; i += gridDim.x * 256) dst[i] = src[i];
+}
+
 __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   __shared__ u64 sd[CHUNK];
   __shared__ u64 wagg[CHUNK / 32];
   dep_release();
+  dep_wait();   // the descriptors, when the kernel that brings them up is the launch before this one
   const u32 tid = threadIdx.x;
   u32 ci;
   const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci, true);

@@ -40,6 +40,7 @@ def test_random_api_streams_with_long_messages(oracle, seed, flags):
               **W.GEO_TOY.kwargs())
     gpu = B.Engine(max_tokens=1 << 20, max_messages=4096, **kw)
     gpu.set_lookup_variant(1 + seed % 4)      # every form of the hash + probe stage
+    gpu.set_l2_residency(seed % 5 != 0)       # with and without the L2 window on the metadata kernels
     gpu.set_classify_mode((2, 0, 1)[seed % 3])
     cpu = oracle.OracleEngine(**kw)
     F.run([gpu, cpu], seed, steps=200, inclusive=bool(flags & 2), check_every=10, invariants=False, max_tok=6000)
