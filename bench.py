@@ -662,6 +662,7 @@ def metadata_stress(torch, B, hbm_peak, reps=5):
     look_ms, cls_ms, sel_ms, cls_edit_ms, cls_full_ms, cls_done_ms, cls_k, cls_edit_k, cls_edit_warm_ms, cls_edit_warm_k = [], [], [], [], [], [], [], [], [], []
     s0 = None
     flush = torch.empty(1 << 29, dtype=torch.uint8, device="cuda")   # 512 MiB > L2: every timed call starts cold
+    vbuf = eng.victim_buffers(n_res // 10)   # pinned output arrays: the victim list is written there by the last kernel
     for rep in range(reps + 1):
         if rep == 1:
             s0 = eng.get_stats()          # the first repetition is the warm-up
@@ -694,7 +695,7 @@ def metadata_stress(torch, B, hbm_peak, reps=5):
         cls_edit_warm_k.append((eng.get_stats()["classify_ns"] - c0["classify_ns"]) / 1e6)
         flush.fill_(rep + 2)
         torch.cuda.synchronize()
-        ms, (v, _st) = timed(lambda: eng.select_victims(0, n_res // 10))
+        ms, (v, _st) = timed(lambda: eng.select_victims(0, n_res // 10, out=vbuf))
         sel_ms.append(ms)
         for i in ids:
             eng.terminate(i)

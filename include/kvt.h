@@ -274,7 +274,11 @@ int32_t kvt_get_states(kvt_engine *e, uint32_t tier, uint8_t *state, uint32_t ca
  * else, oldest first. states_out[i] is the rank, with KVT_STATE_HAS_COPY or-ed in for an HBM victim that
  * still has a clean host copy (offloading it moves no bytes and needs no host slot), or KVT_STATE_COPY.
  * With KVT_POLICY_NO_LIFECYCLE every candidate counts as rank 1. Classifies first if needed. Host output
- * arrays (states_out may be NULL). KVT_E_BUFSZ if cap < min(n_req, #candidates). The order is computed on a packed
+ * arrays (states_out may be NULL). If both are pinned host memory (or device / managed memory) and
+ * cap >= min(n_req, slots of the tier), the last kernel writes the list straight into them; otherwise it is staged
+ * in the engine's pinned area and copied by the CPU, which for a long list costs more than the selection itself
+ * (0.4 ms for 786 K victims). After an error the arrays' contents are unspecified.
+ * KVT_E_BUFSZ if cap < min(n_req, #candidates). The order is computed on a packed
  * key of 2 (+1 on a host tier with clean copies) + bits(clock) + bits(largest depth) bits; KVT_E_INVAL if that exceeds
  * 63 bits (kvt_debug_load_resident refuses stamps and depths that would get there; the clock itself is 32 bits and
  * calls that would advance it past 2^32 - 1 fail with KVT_E_NOSPACE). Synchronises. */

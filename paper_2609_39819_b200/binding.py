@@ -363,9 +363,22 @@ class Engine:
         self._check(self.L.kvt_get_states(self.h, tier, _p(st), len(st), _stream()), "get_states")
         return st
 
-    def select_victims(self, tier, n_req, include_pinned=False):
+    def victim_buffers(self, n):
+        """A pair of pinned host arrays (slots, states) for `out=` of select_victims: the selection's last kernel
+        writes the list straight into them instead of staging it for a CPU copy."""
+        import torch
+        ts = torch.empty(n, dtype=torch.int32, pin_memory=True); tt = torch.empty(n, dtype=torch.uint8, pin_memory=True)
+        self._victim_bufs = getattr(self, "_victim_bufs", []) + [(ts, tt)]     # the arrays below do not own the memory
+        return ts.numpy().view(np.uint32), tt.numpy()
+
+    def select_victims(self, tier, n_req, include_pinned=False, out=None):
         cap = min(n_req, self._tier_size(tier))
-        slots = np.empty(cap, np.uint32); states = np.empty(cap, np.uint8)     # filled by the call up to n
+        if out is None:
+            slots = np.empty(cap, np.uint32); states = np.empty(cap, np.uint8)     # filled by the call up to n
+        else:
+            slots, states = out
+            if len(slots) < cap or len(states) < cap or slots.dtype != np.uint32 or states.dtype != np.uint8:
+                raise ValueError("select_victims: out arrays too small or of the wrong type")
         n = C.c_uint32(0)
         self._check(self.L.kvt_select_victims(self.h, tier, n_req, 1 if include_pinned else 0, _p(slots), _p(states),
                                               cap, C.byref(n), _stream()), "select_victims")

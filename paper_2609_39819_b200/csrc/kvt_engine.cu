@@ -320,6 +320,27 @@ int32_t stage_release(kvt_engine *e, cudaStream_t s) {
   return KVT_OK;
 }
 
+// Control records between the pinned staging area and device memory, carried by one small kernel instead of one
+// copy-engine transfer each (a transfer of a few KB costs 8-11 us of stream time, the kernel 3-5 us for all of them).
+// Host-side pointers must lie in the staging area; a pending list is sent with flush().
+struct SegCopy {
+  kvt_engine *e; cudaStream_t s; CopySegs c{}; bool after_kernel;
+  SegCopy(kvt_engine *e_, cudaStream_t s_, bool after_kernel_ = false) : e(e_), s(s_), after_kernel(after_kernel_) { c.n = 0; }
+  void add(void *dst, const void *src, u64 bytes) {
+    if (!bytes) return;
+    if (c.n == 6) flush();
+    c.src[c.n] = src; c.dst[c.n] = dst; c.bytes[c.n] = (u32)bytes; ++c.n;
+  }
+  void flush() {
+    if (!c.n) return;
+    u64 most = 0;
+    for (u32 k = 0; k < c.n; ++k) most = std::max<u64>(most, c.bytes[k]);
+    launch_attr(e, false, after_kernel, k_copy_segs, (u32)std::min<u64>(std::max<u64>(cdiv(most / 16, 256), 1), 64), 256u, s, c);
+    e->st.kernel_launches++;
+    c.n = 0; after_kernel = true;
+  }
+};
+
 int32_t status_zero(kvt_engine *e, cudaStream_t s) {
   CU(cudaMemsetAsync(e->d_status, 0, ST_WORDS * 4, s));
   return KVT_OK;
@@ -739,11 +760,13 @@ int32_t apply_deltas(kvt_engine *e, cudaStream_t s, const std::vector<Ctx *> &li
   }
   if (nmap) {
     DeltaCtx *dd = reinterpret_cast<DeltaCtx *>(e->dp<u8>(e->L.desc) + 2 * C * sizeof(SnapDesc));
-    CU(cudaMemcpyAsync(dd, hd, nd * sizeof(DeltaCtx), cudaMemcpyHostToDevice, s));
-    if (nm) {
-      CU(cudaMemcpyAsync(e->dp<u32>(e->L.m_start) + tbl_base, e->h_mstart, nm * 4ull, cudaMemcpyHostToDevice, s));
-      CU(cudaMemcpyAsync(e->dp<u32>(e->L.m_end) + tbl_base, e->h_mend, nm * 4ull, cudaMemcpyHostToDevice, s));
-      CU(cudaMemcpyAsync(e->dp<u8>(e->L.m_rank) + tbl_base, e->h_mrank, nm, cudaMemcpyHostToDevice, s));
+    {
+      SegCopy up(e, s);
+      up.add(dd, hd, nd * sizeof(DeltaCtx));
+      up.add(e->dp<u32>(e->L.m_start) + tbl_base, e->h_mstart, nm * 4ull);
+      up.add(e->dp<u32>(e->L.m_end) + tbl_base, e->h_mend, nm * 4ull);
+      up.add(e->dp<u8>(e->L.m_rank) + tbl_base, e->h_mrank, nm);
+      up.flush();
     }
     DeltaArgs a;
     a.tab = e->tab; a.ent = e->ent; a.keys = e->d_keys; a.ctx = dd; a.n_ctx = nd; a.n_map = nmap; a.tbl = msg_tables(e);
@@ -812,7 +835,7 @@ int32_t do_classify(kvt_engine *e, cudaStream_t s, bool force_full = false) {
       for (const Snap &o : e->zombies) add(o);
       if (ns) {
         SnapDesc *ds = reinterpret_cast<SnapDesc *>(e->dp<u8>(e->L.desc));
-        CU(cudaMemcpyAsync(ds, hs, ns * sizeof(SnapDesc), cudaMemcpyHostToDevice, s));
+        { SegCopy up(e, s); up.add(ds, hs, ns * sizeof(SnapDesc)); up.flush(); }
         FixArgs a;
         a.tab = e->tab; a.ent = e->ent; a.keys = e->d_keys; a.snaps = ds; a.n_snaps = ns; a.tbl = msg_tables(e);
         a.fresh = e->dp<u32>(e->L.fresh); a.n_fresh = e->n_fresh; a.status = e->d_status;
@@ -1696,6 +1719,14 @@ int32_t kvt_get_entries(kvt_engine *e, uint32_t tier, uint64_t *keys, uint32_t *
 }
 
 // ---- stage 4 -----------------------------------------------------------------------------------------------
+// The address under which a kernel can write to `p`, or nullptr if `p` is ordinary pageable host memory.
+static void *device_view(const void *p) {
+  cudaPointerAttributes at{};
+  if (!p || cudaPointerGetAttributes(&at, p) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+  if (at.type == cudaMemoryTypeHost || at.type == cudaMemoryTypeDevice || at.type == cudaMemoryTypeManaged) return at.devicePointer;
+  return nullptr;
+}
+
 int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_t flags, uint32_t *slots_out,
                            uint8_t *states_out, uint32_t cap, uint32_t *n_out, void *stream) {
   if (!e || tier > 2 || flags > 1 || !n_out || (!slots_out && cap)) return KVT_E_INVAL;
@@ -1704,8 +1735,6 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   if (!n || !n_req) return KVT_OK;
   cudaStream_t s = (cudaStream_t)stream;
   int32_t r = ensure_classified(e, s);
-  if (r) return r;
-  r = status_zero(e, s);
   if (r) return r;
   int32_t rr = stage_acquire(e);
   if (rr) return rr;
@@ -1742,10 +1771,24 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   a.n_emit = n_emit; a.rank_shift = a.stamp_bits + a.depth_bits;
   // the victim list is written by the last kernel straight into the pinned staging area (mapped into the device's
   // address space like every pinned allocation): no copy after the kernels, the list is there when the stream is
+  // ... and when the caller's arrays are themselves memory a kernel can write (pinned host or device memory, large
+  // enough for min(n_req, slots)), the list goes straight there and nothing is copied afterwards
   u32 *h_slots = (u32 *)e->h_out; u8 *h_states = e->h_out + n_emit * 4ull;
   a.slots_out = h_slots; a.states_out = h_states;
+  bool direct = false;
+  if (cap >= n_emit) {
+    void *ds = device_view(slots_out), *dt = states_out ? device_view(states_out) : nullptr;
+    if (ds && (dt || !states_out)) { direct = true; a.slots_out = (u32 *)ds; if (dt) a.states_out = (u8 *)dt; }
+  }
   const SelArgs *d_args = e->dp<SelArgs>(e->L.sel_args);
-  CU(cudaMemcpyAsync((void *)d_args, &a, sizeof(SelArgs), cudaMemcpyHostToDevice, s));
+  {   // argument record up, status words zeroed: one small kernel
+    static_assert(sizeof(SelArgs) % 4 == 0, "argument record is copied in words");
+    std::memset(e->h_status, 0, ST_WORDS * 4);
+    SegCopy up(e, s);
+    up.add((void *)d_args, &a, sizeof(SelArgs));
+    up.add(e->d_status, e->h_status, ST_WORDS * 4);
+    up.flush();
+  }
   rr = stage_release(e, s);
   if (rr) return rr;
   const u32 n_levels = a.n_levels, n_pass = cdiv(key_bits, RADIX_BITS);
@@ -1807,9 +1850,9 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   }
   if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));   // selection and sort; the list's way to the host comes after
   KL(k_sel_emit, std::min<u32>(cdiv(n_emit, 256), (u32)e->sm_count * 8), 256, s, d_args, k_final, v_final);
+  { SegCopy down(e, s, true); down.add(e->h_status, e->d_status, ST_WORDS * 4); down.flush(); }   // status words beside the list
   LAUNCH_CHECK();
-  r = status_fetch(e, s);
-  if (r) return r;
+  CU(cudaStreamSynchronize(s));
   TRACE_DUMP("select");
   if (e->profiling) {
     float ms = 0.f;
@@ -1823,7 +1866,7 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
   u32 k = std::min(n_req, total);
   *n_out = k;
   if (cap < k) return KVT_E_BUFSZ;
-  if (k) {
+  if (k && !direct) {
     std::memcpy(slots_out, h_slots, k * 4ull);
     if (states_out) std::memcpy(states_out, h_states, k);
   }

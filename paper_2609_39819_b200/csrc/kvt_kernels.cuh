@@ -316,6 +316,27 @@ __global__ void __launch_bounds__(256) k_copy_words(const uint4 *src, uint4 *dst
   for (u32 i = blockIdx.x * 256 + threadIdx.x; i < n16; i += gridDim.x * 256) dst[i] = src[i];
 }
 
+// The same for up to six stretches at once, of any alignment (16-byte, 4-byte or single-byte steps).
+struct CopySegs { const void *src[6]; void *dst[6]; u32 bytes[6]; u32 n; };
+__global__ void __launch_bounds__(256) k_copy_segs(CopySegs c) {
+  dep_release();
+  dep_wait();
+  const u32 t = blockIdx.x * 256 + threadIdx.x, T = gridDim.x * 256;
+  for (u32 k = 0; k < c.n; ++k) {
+    const uintptr_t both = (uintptr_t)c.src[k] | (uintptr_t)c.dst[k] | c.bytes[k];
+    if (!(both & 15)) {
+      const uint4 *s = (const uint4 *)c.src[k]; uint4 *d = (uint4 *)c.dst[k];
+      for (u32 i = t; i < c.bytes[k] / 16; i += T) d[i] = s[i];
+    } else if (!(both & 3)) {
+      const u32 *s = (const u32 *)c.src[k]; u32 *d = (u32 *)c.dst[k];
+      for (u32 i = t; i < c.bytes[k] / 4; i += T) d[i] = s[i];
+    } else {
+      const u8 *s = (const u8 *)c.src[k]; u8 *d = (u8 *)c.dst[k];
+      for (u32 i = t; i < c.bytes[k]; i += T) d[i] = s[i];
+    }
+  }
+}
+
 __global__ void __launch_bounds__(CHUNK) k_hash_digest(HashArgs a) {
   __shared__ u64 sd[CHUNK];
   __shared__ u64 wagg[CHUNK / 32];

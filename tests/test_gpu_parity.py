@@ -428,9 +428,10 @@ def test_c4_lookup_and_select_parity(B, oracle, n_resident, chain_blocks, n_call
     ids = list(range(n_calls))
     # selection before any call: the whole pool is a candidate; 10% stays in the dead tier,
     # 35% crosses into the idle (MRU) tier, 75% into the active tier
+    bufs = gpu.victim_buffers(n_resident)        # pinned: the list is written there by the last kernel, no staging copy
     for frac in (0.10, 0.35, 0.75):
         n = int(n_resident * frac)
-        vg, sg = gpu.select_victims(0, n)
+        vg, sg = gpu.select_victims(0, n, out=bufs if frac != 0.10 else None)
         vc, sc = cpu.select_victims(0, n)
         assert np.array_equal(vg, vc) and np.array_equal(sg, sc), frac
     ig = gpu.map_blocks(ids, 0)
