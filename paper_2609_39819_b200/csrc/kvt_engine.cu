@@ -1586,10 +1586,14 @@ static int32_t map_admit(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_info
     a.now = e->now; a.status = e->d_status;
     a.fresh = e->dp<u32>(e->L.fresh); a.fresh_base = e->n_fresh;
     if ((u64)e->n_fresh + n_free > e->ent.n_total) { rc = fail(e, KVT_E_DEVICE, "list of new entries would overflow"); break; }
-    CU(cudaMemcpyAsync(e->dp<u8>(e->L.desc), hd, nd * sizeof(AdmitCtx), cudaMemcpyHostToDevice, s));
-    CU(cudaMemcpyAsync(a.stop, h_stop, nd * 4, cudaMemcpyHostToDevice, s));
-    rc = status_zero(e, s);
-    if (rc) break;
+    {   // descriptors and stop words up, status words zeroed: one small kernel
+      std::memset(e->h_status, 0, ST_WORDS * 4);
+      SegCopy up(e, s);
+      up.add(e->dp<u8>(e->L.desc), hd, nd * sizeof(AdmitCtx));
+      up.add(a.stop, h_stop, nd * 4ull);
+      up.add(e->d_status, e->h_status, ST_WORDS * 4);
+      up.flush();
+    }
     u32 g = cdiv(n_cand, TPB);
     KLM(k_admit_claim, g, TPB, s, a);
     KLM(k_admit_resolve, g, TPB, s, a);
@@ -1601,9 +1605,15 @@ static int32_t map_admit(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_info
     KLM(k_admit_apply, g, TPB, s, a);
     rc = launch_ok(e);
     if (rc) break;
-    CU(cudaMemcpyAsync(h_stop, a.stop, nd * 4, cudaMemcpyDeviceToHost, s));
-    rc = status_fetch(e, s);
+    {
+      SegCopy down(e, s);
+      down.add(h_stop, a.stop, nd * 4ull);
+      down.add(e->h_status, e->d_status, ST_WORDS * 4);
+      down.flush();
+    }
+    rc = launch_ok(e);
     if (rc) break;
+    CU(cudaStreamSynchronize(s));
     rc = status_code(e);
     if (rc) break;
     e->occ[0] += e->h_status[ST_INSERTED];
