@@ -279,7 +279,9 @@ __device__ __forceinline__ void bulk_store(void *gdst, const void *smem_src, u32
 // Dependent launches inside one call: a kernel releases the next launch of its stream at its start (the next
 // kernel's CTAs then fill the SM slots this kernel's tail leaves free), and the next kernel waits, before it touches
 // anything this one writes, until this grid has finished and its writes are visible. Both are no-ops for a launch
-// without the attribute.
+// without the attribute. In a chain A -> B -> C of such launches C may start while B still waits for A, so a kernel
+// of a chain reads nothing that any earlier kernel of the chain writes before its own wait, and every CTA waits
+// (then "B has finished" implies "A has finished").
 __device__ __forceinline__ void dep_release() { asm volatile("griddepcontrol.launch_dependents;"); }
 __device__ __forceinline__ void dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 
@@ -433,6 +435,10 @@ template <int ILP>
 __global__ void __launch_bounds__(CHUNK / ILP) k_hash_finish_lookup(HashArgs a, LookupArgs l) {
   constexpr u32 T = CHUNK / ILP;
   const u32 tid = threadIdx.x;
+  // Nothing is read before the wait, not even the descriptors: a dependent launch may start as soon as the grid
+  // before it has started, and that grid may itself still be waiting for the kernel that brings the descriptors up.
+  dep_release();
+  dep_wait();
   u32 ci;
   const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci);
   const u32 j = blockIdx.x - c.chunk_base;
@@ -442,8 +448,6 @@ __global__ void __launch_bounds__(CHUNK / ILP) k_hash_finish_lookup(HashArgs a, 
   bool act[ILP];
   const bool kept = b0 < c.first;                                   // unchanged prefix: the keys of the previous list still hold
   u64 carry = 0;
-  dep_release();
-  dep_wait();   // the digest kernel's keys and aggregates
   u64 loc[ILP];   // chain values with zero carry-in (or, in the unchanged prefix, the old keys): fetched before the carry is known
 #pragma unroll
   for (int q = 0; q < ILP; ++q) {
@@ -655,12 +659,12 @@ template <int ILP>
 __global__ void __launch_bounds__(CHUNK / ILP) k_lock_hits(HashArgs a, LockArgs l) {
   constexpr u32 T = CHUNK / ILP;
   const u32 tid = threadIdx.x;
+  dep_wait();   // before anything is read: the descriptors, the probe kernel's entry ids, prefix lengths and error word
   u32 ci;
   const HashCtx c = hash_ctx_of_chunk(a, blockIdx.x, &ci);
   // the hash / probe kernels failed: the call changes nothing. One read per CTA, so that the whole CTA agrees.
   __shared__ u32 s_err;
   __shared__ u32 s_cnt[3];
-  dep_wait();   // the probe kernel's entry ids, prefix lengths and error word
   if (tid == 0) s_err = l.status[ST_ERR];
   if (tid < 3) s_cnt[tid] = 0;
   __syncthreads();
