@@ -439,6 +439,11 @@ int32_t kvt_debug_set_lookup_variant(kvt_engine *e, uint32_t variant);
  * streaming accesses, pass through the rest. 0 switches it off and gives the persisting lines back. */
 int32_t kvt_set_l2_residency(kvt_engine *e, uint32_t on);
 
+/* Test hook for the ordering of a call's kernels: the small kernels that carry a call's control records between the
+ * pinned staging area and the device start their copy delay_ns later (at most 1,000,000). Results must not depend on
+ * it; a kernel of the same call that read a record before it is entitled to would see the previous call's. */
+int32_t kvt_debug_set_copy_delay(kvt_engine *e, uint32_t delay_ns);
+
 /* Test / measurement hook for the classification: 0 = event-driven (default), 1 = every kvt_classify recomputes all
  * counts from zero over all contexts, 2 = event-driven, and every update is followed by a full recomputation that must
  * give the same counts (KVT_E_DEVICE if not). */

@@ -30,7 +30,7 @@ EXPORTS = ("kvt_query_sizes", "kvt_create", "kvt_destroy", "kvt_apply_op", "kvt_
            "kvt_compact", "kvt_copy_blocks", "kvt_hash_scratch_bytes", "kvt_hash_tokens", "kvt_get_stats",
            "kvt_last_error", "kvt_get_entries", "kvt_debug_load_resident", "kvt_set_profiling",
            "kvt_hash_tokens_noalloc", "kvt_debug_set_mover_variant", "kvt_exchange", "kvt_debug_set_lookup_variant", "kvt_move", "kvt_set_mover_ctas",
-           "kvt_debug_set_wait_limit", "kvt_debug_set_classify_mode", "kvt_set_l2_residency")
+           "kvt_debug_set_wait_limit", "kvt_debug_set_classify_mode", "kvt_set_l2_residency", "kvt_debug_set_copy_delay")
 
 
 class KvtError(RuntimeError):
@@ -121,6 +121,7 @@ def load_library():
             "kvt_debug_set_wait_limit": [vp, u32],
             "kvt_debug_set_classify_mode": [vp, u32],
             "kvt_set_l2_residency": [vp, u32],
+            "kvt_debug_set_copy_delay": [vp, u32],
             "kvt_get_entries": [vp, u32, vp, vp, vp, vp, vp, u32, vp],
             "kvt_debug_load_resident": [vp, vp, vp, vp, vp, vp, u32, u32, vp],
         }
@@ -277,6 +278,9 @@ class Engine:
 
     def set_lookup_variant(self, variant):
         self._check(self.L.kvt_debug_set_lookup_variant(self.h, variant), "set_lookup_variant")
+
+    def set_copy_delay(self, delay_ns):
+        self._check(self.L.kvt_debug_set_copy_delay(self.h, int(delay_ns)), "set_copy_delay")
 
     def set_l2_residency(self, on=True):
         self._check(self.L.kvt_set_l2_residency(self.h, 1 if on else 0), "set_l2_residency")

@@ -208,6 +208,7 @@ struct kvt_engine {
   // persisting part of L2 while KV payload and token streams pass through the rest
   cudaAccessPolicyWindow l2_win{};
   bool l2_on = false;
+  u32 copy_delay_ns = 0;   // test hook: the control-record copy kernels start their copy this much later
   bool overlap_launches = !CHECKED_BUILD;   // dependent launches inside one call (digest -> finish -> lock)
   u32 lookup_variant = 0;  // 0 / 1 digest / carry / finish kernels, 2 single-pass hash + probe kernel
   u32 wait_limit = 1u << 18;   // polls a chunk of the single-pass kernel spends on its predecessors before it gives up
@@ -335,7 +336,7 @@ struct SegCopy {
     if (!c.n) return;
     u64 most = 0;
     for (u32 k = 0; k < c.n; ++k) most = std::max<u64>(most, c.bytes[k]);
-    launch_attr(e, false, after_kernel, k_copy_segs, (u32)std::min<u64>(std::max<u64>(cdiv(most / 16, 256), 1), 64), 256u, s, c);
+    launch_attr(e, false, after_kernel, k_copy_segs, (u32)std::min<u64>(std::max<u64>(cdiv(most / 16, 256), 1), 64), 256u, s, c, e->copy_delay_ns);
     e->st.kernel_launches++;
     c.n = 0; after_kernel = true;
   }
@@ -1154,6 +1155,12 @@ int32_t kvt_set_l2_residency(kvt_engine *e, uint32_t on) {
   return KVT_OK;
 }
 
+int32_t kvt_debug_set_copy_delay(kvt_engine *e, uint32_t delay_ns) {
+  if (!e || delay_ns > 1000000u) return KVT_E_INVAL;
+  e->copy_delay_ns = delay_ns;
+  return KVT_OK;
+}
+
 int32_t kvt_debug_set_classify_mode(kvt_engine *e, uint32_t mode) {
   if (!e || mode > 2) return KVT_E_INVAL;
   e->classify_mode = mode;
@@ -1459,7 +1466,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     std::memset(e->h_status, 0, ST_WORDS * 4);
     {
       const u32 n16 = (u32)cdiv((e->L.desc - e->L.status) + nd * sizeof(HashCtx) + ((u64)chunk_base + dchunk_base) * 4, 16);
-      KL(k_copy_words, std::min<u32>(cdiv(n16, 256), 64u), 256, s, (const uint4 *)e->h_status, (uint4 *)e->d_status, n16);
+      KL(k_copy_words, std::min<u32>(cdiv(n16, 256), 64u), 256, s, (const uint4 *)e->h_status, (uint4 *)e->d_status, n16, e->copy_delay_ns);
     }
     HashArgs ha;
     ha.tokens = e->d_tokens; ha.keys = e->d_keys; ha.carry_base = e->d_keys; ha.ctx = e->dp<HashCtx>(e->L.desc); ha.n_ctx = nd;
@@ -1497,7 +1504,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     // one read-back: status words and result words, written into the staging area by a kernel
     {
       const u32 n16 = (u32)cdiv((e->L.ctxres - e->L.status) + 4ull * C * 4, 16);
-      launch_attr(e, false, true, k_copy_words, std::min<u32>(cdiv(n16, 256), 64u), 256, s, (const uint4 *)e->d_status, (uint4 *)e->h_status, n16);
+      launch_attr(e, false, true, k_copy_words, std::min<u32>(cdiv(n16, 256), 64u), 256, s, (const uint4 *)e->d_status, (uint4 *)e->h_status, n16, e->copy_delay_ns);
       e->st.kernel_launches++;
     }
     r = launch_ok(e);

@@ -312,17 +312,27 @@ __device__ __forceinline__ void chunk_scan_store(const HashArgs &a, const HashCt
 // device's address space): the descriptors of a call going up, status and result words coming back. A kernel
 // reaches a few tens of KB over the host link in about a third of the time a copy-engine transfer of that size
 // takes to start and finish, and it can be a dependent launch on both sides.
-__global__ void __launch_bounds__(256) k_copy_words(const uint4 *src, uint4 *dst, u32 n16) {
+// delay_ns (a test hook, at most a millisecond): the copy starts that much later, so that a kernel launched behind
+// it which looks at the records before it is entitled to sees the previous call's.
+__device__ __forceinline__ void copy_delay(u32 delay_ns) {
+  if (!delay_ns) return;
+  u64 t0, t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t0));
+  do { asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); } while (t - t0 < delay_ns);
+}
+__global__ void __launch_bounds__(256) k_copy_words(const uint4 *src, uint4 *dst, u32 n16, u32 delay_ns) {
   dep_release();
   dep_wait();
+  copy_delay(delay_ns);
   for (u32 i = blockIdx.x * 256 + threadIdx.x; i < n16; i += gridDim.x * 256) dst[i] = src[i];
 }
 
 // The same for up to six stretches at once, of any alignment (16-byte, 4-byte or single-byte steps).
 struct CopySegs { const void *src[6]; void *dst[6]; u32 bytes[6]; u32 n; };
-__global__ void __launch_bounds__(256) k_copy_segs(CopySegs c) {
+__global__ void __launch_bounds__(256) k_copy_segs(CopySegs c, u32 delay_ns) {
   dep_release();
   dep_wait();
+  copy_delay(delay_ns);
   const u32 t = blockIdx.x * 256 + threadIdx.x, T = gridDim.x * 256;
   for (u32 k = 0; k < c.n; ++k) {
     const uintptr_t both = (uintptr_t)c.src[k] | (uintptr_t)c.dst[k] | c.bytes[k];

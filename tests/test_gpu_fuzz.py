@@ -66,3 +66,30 @@ def test_random_api_streams_with_three_tiers(oracle, seed, flags, pools):
         gpu.set_mover_variant(4)                  # payload through the staging ring and the copy engines (8 blocks per stage)
     cpu = oracle.OracleEngine(**kw)
     F.run([gpu, cpu], seed, steps=300, inclusive=bool(flags & 2), check_every=10)
+
+
+@pytest.mark.parametrize("seed", range(8))
+@pytest.mark.parametrize("long_messages", [False, True], ids=["short", "long"])
+def test_results_do_not_depend_on_when_control_records_arrive(oracle, seed, long_messages):
+    """The descriptors, message tables and status words of a call are carried by small kernels, and the kernels
+    behind them are dependent launches that may start early. With those copies held back by 0.2 ms, a kernel that
+    looked at a record before its wait would see the previous call's: every result must still equal the oracle's."""
+    import torch
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2609_39819_b200 import binding as B
+    if long_messages:
+        kw = dict(n_hbm_blocks=1500, n_host_blocks=600, max_contexts=6, policy_flags=(0, 2)[seed % 2], metadata_only=True,
+                  **W.GEO_TOY.kwargs())
+        gpu = B.Engine(max_tokens=1 << 20, max_messages=4096, **kw)
+    else:
+        kw = dict(n_hbm_blocks=24, n_host_blocks=16, max_contexts=6, policy_flags=(0, 1, 2, 4)[seed % 4], suspended_order=seed % 2,
+                  **W.GEO_TOY.kwargs())
+        gpu = B.Engine(max_tokens=1 << 16, max_messages=2048, stage_mib=1, **kw)
+    gpu.set_copy_delay(200_000)
+    gpu.set_classify_mode((0, 2)[seed % 2])
+    cpu = oracle.OracleEngine(**kw)
+    if long_messages:
+        F.run([gpu, cpu], 1000 + seed, steps=120, inclusive=bool(kw["policy_flags"] & 2), check_every=10, invariants=False, max_tok=6000)
+    else:
+        F.run([gpu, cpu], 1000 + seed, steps=200, inclusive=bool(kw["policy_flags"] & 2), check_every=10)
