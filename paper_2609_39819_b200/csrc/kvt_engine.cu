@@ -1408,6 +1408,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
   std::vector<std::pair<u32, u32>> n_seq_chunks;   // per listed sequence: chunks in the all-blocks grid / in the digest grid
   std::vector<int> dev_idx(n_ctx, -1);
   u32 nd = 0, chunk_base = 0, dchunk_base = 0, blk_base = 0;
+  bool long_seq = false;   // some sequence has so many chunks to digest that its carries come from the scan kernel
   u32 *h_hit = e->h_ctxres, *h_hbm = e->h_ctxres + e->cfg.max_contexts, *h_host = e->h_ctxres + 2 * e->cfg.max_contexts,
       *h_remote = e->h_ctxres + 3 * e->cfg.max_contexts;
   for (u32 i = 0; i < n_ctx; ++i) {
@@ -1442,6 +1443,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
       hd[nd++] = d;
       chunk_base += cdiv(nb, CHUNK);
       dchunk_base += cdiv(nb - first, CHUNK);
+      long_seq = long_seq || cdiv(nb - first, CHUNK) > FOLD_MAX_CHUNKS;
       n_seq_chunks.push_back({cdiv(nb, CHUNK), cdiv(nb - first, CHUNK)});
       blk_base += nb;
       e->st.blocks_rehashed += nb - first;
@@ -1470,7 +1472,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
     }
     HashArgs ha;
     ha.tokens = e->d_tokens; ha.keys = e->d_keys; ha.carry_base = e->d_keys; ha.ctx = e->dp<HashCtx>(e->L.desc); ha.n_ctx = nd;
-    ha.agg = e->dp<u64>(e->L.agg); ha.h0 = e->h0; ha.single = HashCtx{};
+    ha.agg = e->dp<u64>(e->L.agg); ha.h0 = e->h0; ha.single = HashCtx{}; ha.carries_ready = long_seq;
     ha.chunk_ctx = reinterpret_cast<const u32 *>(ha.ctx + nd); ha.dchunk_ctx = ha.chunk_ctx + chunk_base;
     LookupArgs la;
     la.tab = e->tab; la.b_ent = e->dp<u32>(e->L.s0); la.hit_len = d_res; la.status = e->d_status;
@@ -1482,6 +1484,7 @@ static int32_t map_lookup(kvt_engine *e, const u32 *ids, u32 n_ctx, kvt_call_inf
       const bool dg = dchunk_base != 0;
       TRACE(s, "uploads");
       if (dg) { launch_attr(e, false, true, k_hash_digest, dchunk_base, CHUNK, s, ha); e->st.kernel_launches++; }
+      if (long_seq) KL(k_hash_carry, nd, 1024, s, ha);
       TRACE(s, "digest");
       // two keys per thread by default; one or four measured within 3 % of it: the probes of a cold table are bound
       // by the number of outstanding misses the memory system carries, not by what a thread issues
@@ -2258,7 +2261,9 @@ int32_t kvt_hash_tokens(const uint32_t *d_tokens, uint64_t n_tokens, uint64_t ha
   ha.single.n_blocks = (u32)nb;
   ha.agg = (u64 *)d_scratch; ha.carry_base = (u64 *)d_scratch + n_chunks; ha.h0 = hash_h0(hash_seed);
   LookupArgs la{};
+  ha.carries_ready = n_chunks > FOLD_MAX_CHUNKS;   // a long sequence: its chunk carries come from the scan kernel
   k_hash_digest<<<n_chunks, CHUNK, 0, s>>>(ha);
+  if (ha.carries_ready) k_hash_carry<<<1, 1024, 0, s>>>(ha);
   k_hash_finish_lookup<1><<<n_chunks, CHUNK, 0, s>>>(ha, la);
   return cudaGetLastError() == cudaSuccess ? KVT_OK : KVT_E_CUDA;
 }
@@ -2290,7 +2295,9 @@ int32_t kvt_hash_tokens_noalloc(const uint32_t *d_tokens, uint64_t n_tokens, uin
   ha.single.n_blocks = (u32)nb;
   ha.agg = scratch; ha.carry_base = scratch + NOALLOC_MAX_CHUNKS; ha.h0 = hash_h0(hash_seed);
   LookupArgs la{};
+  ha.carries_ready = n_chunks > FOLD_MAX_CHUNKS;   // a long sequence: its chunk carries come from the scan kernel
   k_hash_digest<<<n_chunks, CHUNK, 0, s>>>(ha);
+  if (ha.carries_ready) k_hash_carry<<<1, 1024, 0, s>>>(ha);
   k_hash_finish_lookup<1><<<n_chunks, CHUNK, 0, s>>>(ha, la);
   return cudaGetLastError() == cudaSuccess ? KVT_OK : KVT_E_CUDA;
 }

@@ -198,6 +198,7 @@ struct HashArgs {
   const u32 *tokens; u64 *keys; u64 *carry_base; const HashCtx *ctx; HashCtx single; u32 n_ctx;
   u64 *agg; u64 h0;
   const u32 *chunk_ctx, *dchunk_ctx;   // batch only: sequence index of every chunk of the all-blocks / digest grid
+  u32 carries_ready;   // the chunk carries were written by k_hash_carry (long sequences): the finish kernel reads them
 };
 
 // Sequence that owns chunk `chunk` of the all-blocks grid (dgrid = false) or of the digest grid (dgrid = true):
@@ -438,6 +439,59 @@ __device__ __forceinline__ u64 chunk_carry(const HashArgs &a, const HashCtx &c, 
   return total;
 }
 
+// The chunk carries of every sequence by a scan, one CTA per sequence: used instead of the fold above when a sequence
+// has more than FOLD_MAX_CHUNKS chunks to digest (the fold reads every aggregate before a chunk, which is quadratic
+// in the sequence length: 64 Mi tokens are 16,384 chunks). Also copies the kept carries and writes the resume point.
+constexpr u32 FOLD_MAX_CHUNKS = 128;
+__global__ void __launch_bounds__(1024) k_hash_carry(HashArgs a) {
+  __shared__ u64 wtot[32], wpre[32], sv[1024];
+  const u32 i = blockIdx.x;
+  if (i >= a.n_ctx) return;
+  const u32 tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const HashCtx c = a.ctx ? a.ctx[i] : a.single;
+  const u32 g0 = c.first / CHUNK;
+  const u32 n_chunks = (c.n_blocks - c.first + CHUNK - 1) / CHUNK;   // chunks that were digested
+  for (u32 k = tid; k < g0; k += 1024) a.carry_base[c.carry_off + k] = a.carry_base[c.old_carry_off + k];
+  const u64 A = g_pow_p.v[CHUNK];
+  const u64 A32 = pow_u64(A, 32);
+  const u64 a_lane = pow_u64(A, lane + 1);          // A^(lane+1)
+  const u64 a_tid = pow_u64(A32, warp) * a_lane;    // A^(tid+1)
+  u64 carry = g0 ? a.carry_base[c.old_carry_off + g0] : a.h0;
+  if (n_chunks == 0 && tid == 0) a.carry_base[c.carry_off + g0] = carry;   // nothing new: keep the resume point
+  for (u32 base = 0; base < n_chunks; base += 1024) {
+    const u32 j = base + tid;
+    u64 x = j < n_chunks ? a.agg[c.dchunk_base + j] : 0;
+    u64 pp = A;
+#pragma unroll
+    for (u32 o = 1; o < 32; o <<= 1) {
+      u64 up = __shfl_up_sync(0xFFFFFFFFu, x, o);
+      if (lane >= o) x += pp * up;
+      pp *= pp;
+    }
+    if (lane == 31) wtot[warp] = x;
+    __syncthreads();
+    if (warp == 0) {   // value at the end of every earlier warp of this round, with zero carry-in
+      u64 y = wtot[lane], qq = A32;
+#pragma unroll
+      for (u32 o = 1; o < 32; o <<= 1) {
+        u64 up = __shfl_up_sync(0xFFFFFFFFu, y, o);
+        if (lane >= o) y += qq * up;
+        qq *= qq;
+      }
+      u64 e = __shfl_up_sync(0xFFFFFFFFu, y, 1);
+      wpre[lane] = lane ? e : 0;
+    }
+    __syncthreads();
+    sv[tid] = a_tid * carry + a_lane * wpre[warp] + x;   // chain value after chunk g0 + j
+    __syncthreads();
+    if (j < n_chunks) a.carry_base[c.carry_off + g0 + j] = tid ? sv[tid - 1] : carry;
+    // value after the last chunk: the resume point of a later call if that chunk is full
+    if (j == n_chunks - 1) a.carry_base[c.carry_off + g0 + n_chunks] = sv[tid];
+    carry = sv[1023];
+    __syncthreads();
+  }
+}
+
 // One CTA of CHUNK / ILP threads per 256-block chunk; thread t finishes and probes blocks t, t + CHUNK / ILP, ...
 // The CTA first works out the chain value entering its chunk from the chunk aggregates of the digest kernel (no
 // separate scan kernel) and stores it next to the keys, where a later call resumes from it.
@@ -464,7 +518,9 @@ __global__ void __launch_bounds__(CHUNK / ILP) k_hash_finish_lookup(HashArgs a, 
     const u32 jj = tid + q * T;
     loc[q] = jj < nb ? a.keys[(kept ? c.old_key_off : c.key_off) + b0 + jj] : 0;
   }
-  if (kept) {
+  if (a.carries_ready) {
+    if (!kept) carry = a.carry_base[c.carry_off + j];
+  } else if (kept) {
     if (tid == 0) {
       a.carry_base[c.carry_off + j] = a.carry_base[c.old_carry_off + j];
       if (b0 + CHUNK == c.n_blocks) a.carry_base[c.carry_off + j + 1] = a.carry_base[c.old_carry_off + j + 1];   // nothing new: the resume point

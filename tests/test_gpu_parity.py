@@ -821,6 +821,31 @@ def test_capacity_errors_leave_the_engine_usable(B):
 
 
 @pytest.mark.parametrize("lookup_variant", [1, 2, 4], ids=["default", "single-pass", "four-keys-per-thread"])
+def test_a_sequence_of_several_hundred_chunks(B, oracle, lookup_variant):
+    """A context of 40,000+ blocks (more than 128 hash chunks: its chunk carries come from the scan kernel instead of
+    the per-chunk fold), next to a short one in the same batch, then a call that resumes near its end."""
+    kw = dict(n_hbm_blocks=50_000, n_host_blocks=0, max_contexts=4, metadata_only=True, **W.GEO_TOY.kwargs())
+    gpu = B.Engine(max_tokens=1 << 21, max_messages=64, max_batch_blocks=60_000, **kw)
+    gpu.set_lookup_variant(lookup_variant)
+    rng = np.random.default_rng(31)
+    long_tok = rng.integers(0, W.VOCAB, 16 * 40_001 + 5, dtype=np.uint32)
+    short_tok = rng.integers(0, W.VOCAB, 16 * 300, dtype=np.uint32)
+    gpu.spawn(0); gpu.append(0, long_tok)
+    gpu.spawn(1); gpu.append(1, short_tok)
+    gpu.map_blocks([0, 1], 0); gpu.map_blocks([0, 1], 1)
+    assert np.array_equal(gpu.get_block_map(0)[0], oracle.hash_tokens(long_tok))
+    assert np.array_equal(gpu.get_block_map(1)[0], oracle.hash_tokens(short_tok))
+    gpu.prefill_done(0); gpu.prefill_done(1)
+    more = rng.integers(0, W.VOCAB, 16 * 700, dtype=np.uint32)
+    gpu.append(0, more)
+    before = gpu.get_stats()["blocks_rehashed"]
+    info = gpu.map_blocks([0], 0)
+    assert gpu.get_stats()["blocks_rehashed"] - before == 40_701 - 40_001 // 256 * 256     # resumed at the last chunk boundary
+    assert int(info["hit_len"][0]) == 40_001
+    assert np.array_equal(gpu.get_block_map(0)[0], oracle.hash_tokens(np.concatenate([long_tok[:16 * 40_001 + 5], more]))[:40_701])
+
+
+@pytest.mark.parametrize("lookup_variant", [1, 2, 4], ids=["default", "single-pass", "four-keys-per-thread"])
 def test_incremental_hashing_resumes_at_chunk_boundaries(B, oracle, lookup_variant):
     """Appends, edits, forks and repeated calls around multiples of 256 blocks: only the changed tail is digested
     again, and every key still equals the one-shot hash of the whole sequence."""
