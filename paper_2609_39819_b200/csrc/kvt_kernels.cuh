@@ -1417,11 +1417,13 @@ __global__ void __launch_bounds__(256) k_radix_hist(const u64 *keys, const u32 *
   if (blockIdx.x >= n_tiles) return;
   for (u32 d = threadIdx.x; d < RADIX_BINS; d += 256) h[d] = 0;
   __syncthreads();
-  u32 base = blockIdx.x * SORT_TILE;
-  for (u32 k = threadIdx.x; k < SORT_TILE; k += 256) {
-    u32 i = base + k;
-    if (i < m) atomicAdd(&h[(u32)(keys[i] >> shift) & (RADIX_BINS - 1)], 1u);
-  }
+  const u32 base = blockIdx.x * SORT_TILE + threadIdx.x;
+  u64 kreg[SORT_ITERS];
+#pragma unroll
+  for (int it = 0; it < SORT_ITERS; ++it) kreg[it] = base + it * 256 < m ? keys[base + it * 256] : 0;   // loads first, then the atomics
+#pragma unroll
+  for (int it = 0; it < SORT_ITERS; ++it)
+    if (base + it * 256 < m) atomicAdd(&h[(u32)(kreg[it] >> shift) & (RADIX_BINS - 1)], 1u);
   __syncthreads();
   for (u32 d = threadIdx.x; d < RADIX_BINS; d += 256) counts[d * n_tiles + blockIdx.x] = h[d];   // digit-major
 }
@@ -1463,11 +1465,15 @@ __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const
   u64 kreg[SORT_ITERS];
   u32 vreg[SORT_ITERS];
 #pragma unroll
+  for (int it = 0; it < SORT_ITERS; ++it) {   // all loads first: the ranking loop below synchronises the warp in every step
+    u32 i = base + it * 32 + lane;
+    kreg[it] = i < m ? keys_in[i] : 0;
+    vreg[it] = i < m ? vals_in[i] : 0;
+  }
+#pragma unroll
   for (int it = 0; it < SORT_ITERS; ++it) {
     u32 i = base + it * 32 + lane;
     bool ok = i < m;
-    kreg[it] = ok ? keys_in[i] : 0;
-    vreg[it] = ok ? vals_in[i] : 0;
     u32 d = (u32)(kreg[it] >> shift) & (RADIX_BINS - 1);
     u32 peers = __match_any_sync(0xFFFFFFFFu, ok ? d : RADIX_BINS);
     if (ok && (peers & ((1u << lane) - 1)) == 0) cnt[warp][d] += __popc(peers);
