@@ -437,7 +437,7 @@ class Engine:
     def get_stats(self):
         out = np.zeros(len(STATS_FIELDS), np.uint64)
         self._check(self.L.kvt_get_stats(self.h, _p(out)), "get_stats")
-        return {k: int(v) for k, v in zip(STATS_FIELDS, out)}
+        return dict(zip(STATS_FIELDS, out.tolist()))
 
     def get_entries(self, tier):
         n = self._tier_size(tier)
