@@ -1869,7 +1869,7 @@ int32_t kvt_select_victims(kvt_engine *e, uint32_t tier, uint32_t n_req, uint32_
     }
   }
   if (e->profiling) CU(cudaEventRecord(e->ev_h1, s));   // selection and sort; the list's way to the host comes after
-  KL(k_sel_emit, std::min<u32>(cdiv(n_emit, 256), (u32)e->sm_count * 8), 256, s, d_args, k_final, v_final);
+  KL(k_sel_emit, std::min<u32>(cdiv(n_emit, 1024), (u32)e->sm_count * 8), 256, s, d_args, k_final, v_final);
   { SegCopy down(e, s, true); down.add(e->h_status, e->d_status, ST_WORDS * 4); down.flush(); }   // status words beside the list
   LAUNCH_CHECK();
   CU(cudaStreamSynchronize(s));

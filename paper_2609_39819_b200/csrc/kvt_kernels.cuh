@@ -1523,14 +1523,32 @@ __global__ void __launch_bounds__(256) k_radix_scatter(const u64 *keys_in, const
 __global__ void k_sel_emit(const SelArgs *pa, const u64 *keys, const u32 *vals) {
   const SelArgs &a = sel_args(pa);
   const u32 n = min(a.n_emit, a.status[ST_M]);   // only the first ST_M pairs exist
-  for (u32 i = blockIdx.x * blockDim.x + threadIdx.x; i < n; i += gridDim.x * blockDim.x) {
-    const u32 slot = vals[i];
-    if (slot >= a.n_slots) continue;
-    a.slots_out[i] = slot;
-    const u64 k = keys[i] >> a.rank_shift;
-    const bool primary = a.copy_bit ? (k >> 2) & 1 : true;
-    const u32 link = a.ent.link[a.e0 + slot];
-    a.states_out[i] = !primary ? (u8)0xFE : (u8)((k & 3) | (link != ENT_NONE ? 0x80 : 0));
+  // four victims per thread: the list usually goes over the host link, where one 16-byte and one 4-byte store per
+  // thread travel better than four 4-byte and four single-byte ones
+  const bool wide = !((uintptr_t)a.slots_out & 15) && !((uintptr_t)a.states_out & 3);
+  for (u32 i0 = (blockIdx.x * blockDim.x + threadIdx.x) * 4; i0 < n; i0 += gridDim.x * blockDim.x * 4) {
+    u32 slot[4];
+    u8 st[4];
+    bool all = true;
+#pragma unroll
+    for (u32 j = 0; j < 4; ++j) {
+      const u32 i = i0 + j;
+      slot[j] = i < n ? vals[i] : 0xFFFFFFFFu;
+      st[j] = 0;
+      if (slot[j] >= a.n_slots) { all = false; continue; }
+      const u64 k = keys[i] >> a.rank_shift;
+      const bool primary = a.copy_bit ? (k >> 2) & 1 : true;
+      const u32 link = a.ent.link[a.e0 + slot[j]];
+      st[j] = !primary ? (u8)0xFE : (u8)((k & 3) | (link != ENT_NONE ? 0x80 : 0));
+    }
+    if (wide && all) {
+      *reinterpret_cast<uint4 *>(a.slots_out + i0) = make_uint4(slot[0], slot[1], slot[2], slot[3]);
+      *reinterpret_cast<uchar4 *>(a.states_out + i0) = make_uchar4(st[0], st[1], st[2], st[3]);
+    } else {
+#pragma unroll
+      for (u32 j = 0; j < 4; ++j)
+        if (slot[j] < a.n_slots) { a.slots_out[i0 + j] = slot[j]; a.states_out[i0 + j] = st[j]; }
+    }
   }
 }
 
